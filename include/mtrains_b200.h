@@ -1,0 +1,231 @@
+/*
+ * mtrains_b200 — C ABI of the sparse-embedding step of MTrainS-style DLRM training on one
+ * NVIDIA B200 (sm_100a): pooled multi-table embedding lookup, backward fused with row-wise
+ * Adagrad on the touched rows, and a software-managed set-associative row cache in HBM in
+ * front of pinned host memory.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers unless the name starts with host_ or the comment says
+ *     "host".  The caller owns every buffer it passes; the library allocates device memory
+ *     only inside mts_tables_create and mts_cache_create and frees it in the matching
+ *     destroy call.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Work is
+ *     enqueued asynchronously; no entry point synchronises the device except where stated.
+ *   - Return value: MTS_OK (0) or a negative MTS_ERR_* code.  Nothing throws, exits, aborts or
+ *     traps on the device.  mts_last_error_string() describes the calling thread's last error.
+ *   - Layouts: weights of table t are a row-major [rows[t], dim[t]] array of the storage type
+ *     (fp32 or IEEE binary16) starting at element weight_offset[t] of its backing buffer;
+ *     dim[t] * sizeof(element) must be a multiple of 16 bytes and every base pointer 16-byte
+ *     aligned.  Pooled outputs and their gradients are fp32 [B, out_stride] row-major, table t
+ *     occupying columns [out_offset[t], out_offset[t] + dim[t]) with out_offset the prefix sum
+ *     of dim.  Sparse input is CSR: `indices` int64 [N] and `offsets` int64 [T*B + 1] over bag
+ *     id t*B + b (table-major), offsets[T*B] == N.
+ */
+#ifndef MTRAINS_B200_H_
+#define MTRAINS_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MTS_OK 0
+#define MTS_ERR_INVALID_ARG (-1)
+#define MTS_ERR_ALIGNMENT (-2)
+#define MTS_ERR_WORKSPACE (-3)
+#define MTS_ERR_CAPACITY (-4)
+#define MTS_ERR_CUDA (-5)
+#define MTS_ERR_TIMEOUT (-6)
+#define MTS_ERR_UNSUPPORTED (-7)
+
+#define MTS_DTYPE_FP32 0
+#define MTS_DTYPE_FP16 1
+
+#define MTS_POOL_SUM 0
+#define MTS_POOL_MEAN 1
+
+#define MTS_POLICY_LRU 0
+#define MTS_POLICY_LFU 1
+
+#define MTS_MAX_CACHES 8
+#define MTS_CACHE_WAYS 32
+#define MTS_NUM_COUNTERS 10
+
+/* Indices into the counter block written by mts_cache_lookup_insert. */
+enum {
+  MTS_CNT_LOOKUPS = 0,       /* N */
+  MTS_CNT_UNIQUE = 1,        /* distinct keys in the call */
+  MTS_CNT_HIT_LOOKUPS = 2,   /* lookups whose key was resident before the call */
+  MTS_CNT_MISS_LOOKUPS = 3,
+  MTS_CNT_UNIQUE_HITS = 4,
+  MTS_CNT_UNIQUE_MISSES = 5,
+  MTS_CNT_INSERTED = 6,      /* length of the miss list */
+  MTS_CNT_EVICTED = 7,       /* length of the evict list */
+  MTS_CNT_EVICTED_DIRTY = 8,
+  MTS_CNT_OVERFLOW = 9       /* distinct missing keys that found no evictable way */
+};
+
+const char* mts_last_error_string(void);
+
+/* ---------------------------------------------------------------------------------------
+ * Tables.  The paper's model: T embedding tables, table t a 2-D tensor of H_t rows and D
+ * columns of p bytes (Section 2.1.2, Eq. 1), the same structure in every memory that holds
+ * it (Section 5.2), plus per-table metadata that says which memory serves it (Section 5.8).
+ * ------------------------------------------------------------------------------------- */
+typedef struct {
+  int32_t T;                      /* number of tables (>= 1) */
+  int32_t dtype;                  /* MTS_DTYPE_*: storage type of all weights */
+  const int64_t* host_rows;       /* host [T]  rows per table (>= 1) */
+  const int32_t* host_dim;        /* host [T]  columns per table */
+  const int64_t* host_weight_offset; /* host [T]  element offset of table t in its buffer */
+  const int32_t* host_cache_id;   /* host [T] or NULL.  -1: rows live in dev_weights.
+                                     c >= 0: rows live in the host tier (host_weights_mapped)
+                                     and are served through cache c (see mts_cache_*). */
+  void* dev_weights;              /* device buffer of the HBM-resident tables (may be NULL
+                                     when every table is cached) */
+  void* host_weights_mapped;      /* device-visible address of the pinned, mapped host buffer
+                                     holding the host-tier tables (NULL when none) */
+  float* momentum;                /* device fp32 [sum rows]: one Adagrad state per row, indexed
+                                     by linear row id row_offset[t] + r (prefix sum of rows).
+                                     Optimizer state stays in HBM (Section 5.6). */
+} mts_table_desc;
+
+typedef struct mts_tables mts_tables;
+
+/* Validates the description, copies the per-table metadata to the device (one small
+ * allocation) and returns a handle.  Synchronous.  Errors: INVALID_ARG (null, T < 1,
+ * rows < 1, cache id out of range), UNSUPPORTED (sum rows >= 2^32, dim > 1024), ALIGNMENT
+ * (row bytes or a base pointer not a multiple of 16), CUDA. */
+int mts_tables_create(const mts_table_desc* desc, mts_tables** out);
+int mts_tables_destroy(mts_tables* tables);
+
+/* Reads and clears the handle's sticky device status word.  Synchronises `stream`.
+ * *host_status receives a bit mask: bit 0 = an index outside [0, rows[t]) was seen (the
+ * lookup was clamped to a valid row, never read out of bounds). */
+int mts_tables_status(mts_tables* tables, int32_t* host_status, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Forward: pooled lookup (Section 2.1.1: an embedding operator selects rows of a table and
+ * pools them by sum, mean or max; sum and mean are provided).
+ *   out[b, out_offset[t] + d] = sum over the lookups i of bag (t, b) of W_t[indices[i], d]
+ * accumulated in fp32; MTS_POOL_MEAN divides by the bag length; an empty bag gives 0; an id
+ * that occurs twice in a bag counts twice.
+ * slot_of_lookup (int32 [N], may be NULL when no table is cached): for a lookup of a cached
+ * table, the cache slot holding its row, or -1 = read the row from the host tier directly.
+ * host_cache_data: host array [n_caches] of device pointers to each cache's row storage.
+ * Errors: INVALID_ARG, ALIGNMENT, CUDA (launch failure). */
+int mts_tbe_forward(const mts_tables* tables, int32_t B, const int64_t* indices,
+                    const int64_t* offsets, int64_t N, int32_t pooling_mode,
+                    const int32_t* slot_of_lookup, void* const* host_cache_data, int32_t n_caches,
+                    float* out, int64_t out_stride, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Backward fused with row-wise Adagrad on the touched rows (Section 2.1.2: an Adagrad-type
+ * optimizer with few states per row; Section 5.9: the backward pass aggregates gradients,
+ * runs the optimizer and writes the rows back to whichever memory holds them).  For every
+ * distinct row r of table t in the batch:
+ *   g_r[d]  = sum over all occurrences i of r of s_i * grad_out[b(i), out_offset[t] + d]
+ *             (s_i = 1, or 1 / bag length for mean pooling)
+ *   m_r    += (1 / D_t) * sum_d g_r[d]^2
+ *   W[r,d] -= lr * g_r[d] / (sqrt(m_r) + eps)      with the new m_r
+ * One step per row per batch; other rows and states keep their bits.  fp32 arithmetic, fp16
+ * rows stored with round-to-nearest-even.  The result is deterministic: occurrences are
+ * summed in a fixed order that depends only on the batch.
+ * Cached rows are updated in their slot and host_cache_dirty[c][slot] is set to 1; rows with
+ * slot -1 are updated in the host tier directly.
+ * workspace: device scratch of at least mts_tbe_backward_workspace_bytes(...) bytes, 256-byte
+ * aligned, contents undefined on entry and exit.
+ * uniq_rows_out / n_unique_out (both or neither; nullable, device int64 [N] / [1]): ascending
+ * distinct linear row ids of the batch and their count.
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE (too small), CUDA. */
+size_t mts_tbe_backward_workspace_bytes(const mts_tables* tables, int32_t B, int64_t N);
+int mts_tbe_backward_rowwise_adagrad(const mts_tables* tables, int32_t B, const int64_t* indices,
+                                     const int64_t* offsets, int64_t N, int32_t pooling_mode,
+                                     const float* grad_out, int64_t grad_stride, float lr, float eps,
+                                     const int32_t* slot_of_lookup, void* const* host_cache_data,
+                                     uint8_t* const* host_cache_dirty, int32_t n_caches,
+                                     void* workspace, size_t workspace_bytes,
+                                     int64_t* uniq_rows_out, int64_t* n_unique_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Row cache (Section 5.3.1 cache class: row-granular cache memory, tags, per-entry timestamp
+ * states; Section 5.5 GPU-managed cache kernels).  One level: HBM in front of pinned host
+ * memory.  32-way set associative; set of a key = floor(((key * 0x9E3779B97F4A7C15) mod 2^64)
+ * * num_sets / 2^64).  Keys are row ids relative to the cache's table group (tables of one
+ * dim, contiguous in the host buffer): row `key` starts at element key * dim of
+ * host_rows_mapped.
+ * ------------------------------------------------------------------------------------- */
+typedef struct mts_cache mts_cache;
+
+/* Allocates tags, states, dirty bytes and num_sets*32 rows of `dim` elements in HBM.
+ * key_space: number of rows of the table group the cache serves; keys are in [0, key_space).
+ * lock_depth: a way stamped at step >= step - lock_depth is not evictable (Section 5.7: a
+ * prefetched row is not evicted before its batch has trained).  Synchronous.
+ * Errors: INVALID_ARG (num_sets < 1 or num_sets*32 >= 2^31, key_space >= 2^32 - 1, ways != 32),
+ * ALIGNMENT, CUDA. */
+int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_space, int32_t ways, int32_t dim,
+                     int32_t dtype, int32_t policy, int32_t lock_depth);
+int mts_cache_destroy(mts_cache* cache);
+void* mts_cache_data(mts_cache* cache);        /* device [num_sets*32, dim] */
+uint8_t* mts_cache_dirty(mts_cache* cache);    /* device [num_sets*32] */
+
+/* Row keys of the lookups of tables [t_begin, t_end) relative to that group:
+ * keys_out[i - lookup_begin] = row_offset[t] - row_offset[t_begin] + indices[i] for the n
+ * lookups i in [lookup_begin, lookup_begin + n) = [offsets[t_begin*B], offsets[t_end*B]).
+ * (The metadata consulted on every lookup, Section 5.8.) */
+int mts_linearize_keys(const mts_tables* tables, int32_t t_begin, int32_t t_end, int32_t B,
+                       const int64_t* indices, const int64_t* offsets, int64_t lookup_begin,
+                       int64_t n, int64_t* keys_out, void* stream);
+
+/* Tag/state lookup and replacement for one batch at time `step` (Sections 5.5.1, 5.5.2):
+ *  1. every distinct key is probed in its set; a lookup is a hit iff its key was resident
+ *     before the call;
+ *  2. all hits are refreshed (timestamp = step);
+ *  3. per set, the missing keys in ascending order take the set's evictable ways (timestamp
+ *     < step - lock_depth; free ways first) in (timestamp, way) order [LFU: (count, timestamp,
+ *     way)]; a victim with a valid tag is appended to the evict list with its dirty byte, which
+ *     is cleared; missing keys beyond the evictable ways are not inserted (slot -1, counted as
+ *     overflow);
+ *  4. slot = set * 32 + way; slot_of_lookup[i] = slot of keys[i].
+ * miss list {key, slot} is ordered by (set, key); evict list {old key, slot, dirty} by (set,
+ * order of the misses that displaced them).  list_capacity >= number of distinct keys is always
+ * enough; entries beyond the capacity are dropped while MTS_CNT_INSERTED / MTS_CNT_EVICTED
+ * keep counting, so a counter above list_capacity tells the caller that a list was cut.
+ * counters: device int64 [MTS_NUM_COUNTERS], overwritten.  `step` must not decrease between calls.
+ * workspace: at least mts_cache_workspace_bytes(cache, N) bytes, 256-byte aligned.
+ * Errors: INVALID_ARG, WORKSPACE, CUDA. */
+size_t mts_cache_workspace_bytes(const mts_cache* cache, int64_t N);
+int mts_cache_lookup_insert(mts_cache* cache, const int64_t* keys, int64_t N, int64_t step,
+                            int32_t* slot_of_lookup, int64_t* miss_keys, int32_t* miss_slots,
+                            int64_t* evict_keys, int32_t* evict_slots, uint8_t* evict_dirty,
+                            int64_t list_capacity, int64_t* counters, void* workspace,
+                            size_t workspace_bytes, void* stream);
+
+/* Data movement for one lookup_insert result (Sections 5.5.3, 5.5.4): first the rows of dirty
+ * victims are saved, slot -> evict_staging[k] (k = position in the evict list), then every
+ * missed row is pulled from the host tier into its slot.  List lengths are read on the device
+ * from `counters`.  evict_staging: device [list_capacity, dim]. */
+int mts_cache_prefetch_misses(mts_cache* cache, const void* host_rows_mapped, const int64_t* miss_keys,
+                              const int32_t* miss_slots, const int32_t* evict_slots,
+                              const uint8_t* evict_dirty, int64_t list_capacity,
+                              const int64_t* counters, void* evict_staging, void* stream);
+
+/* Evicted dirty rows go back to the host tier: evict_staging[k] -> host row evict_keys[k]. */
+int mts_cache_writeback_evicted(mts_cache* cache, void* host_rows_mapped, const int64_t* evict_keys,
+                                const uint8_t* evict_dirty, int64_t list_capacity,
+                                const int64_t* counters, const void* evict_staging, void* stream);
+
+/* Writes every dirty resident row to the host tier and clears its dirty byte. */
+int mts_cache_flush(mts_cache* cache, void* host_rows_mapped, void* stream);
+
+/* Copies tags (int64 [sets*32], -1 = free), timestamps (int64, -1 = free), use counts (int64)
+ * and dirty bytes to caller buffers (device); any pointer may be NULL. */
+int mts_cache_export_state(mts_cache* cache, int64_t* tags, int64_t* timestamps, int64_t* counts,
+                           uint8_t* dirty, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MTRAINS_B200_H_ */

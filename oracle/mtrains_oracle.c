@@ -7,10 +7,10 @@
  * product never calls it.
  *
  * What is defined here, and where the paper defines it:
- *   - pooled embedding lookup (sum / mean over the rows a sample selects)   Section 2.1
- *     ("Embedding tables": look up a subset of rows and pool the result)
+ *   - pooled embedding lookup (sum / mean over the rows a sample selects)   Section 2.1.1
+ *     (embedding table operators: select rows of a table, pool them)
  *   - backward: aggregate the gradients of every row a batch touched, run a
- *     row-wise Adagrad step with one state per row, write the row back      Section 2.1.1
+ *     row-wise Adagrad step with one state per row, write the row back      Section 2.1.2
  *     (optimizer with few states per row), Section 5.9 (aggregations and
  *     optimizers, then update the weights in their memories)
  *   - row cache with tags and per-entry timestamps, LRU in three steps       Section 5.3.1,

@@ -1,0 +1,259 @@
+"""Thin ctypes binding of libmtrains_b200.so: same names as include/mtrains_b200.h, argument
+marshalling only.  Every step of the path runs in the library's CUDA kernels; there is no
+fallback: a missing library or a failing call raises.
+
+Pointer arguments accept a torch tensor (its data_ptr is passed), an int address, or None.
+`stream` accepts a torch.cuda.Stream, an int handle or None (legacy default stream).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libmtrains_b200.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CAPACITY, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = (
+    -1, -2, -3, -4, -5, -6, -7)
+DTYPE_FP32, DTYPE_FP16 = 0, 1
+POOL_SUM, POOL_MEAN = 0, 1
+POLICY_LRU, POLICY_LFU = 0, 1
+MAX_CACHES, CACHE_WAYS, NUM_COUNTERS = 8, 32, 10
+COUNTER_NAMES = ("lookups", "unique", "hit_lookups", "miss_lookups", "unique_hits",
+                 "unique_misses", "inserted", "evicted", "evicted_dirty", "overflow")
+
+EXPORTS = (
+    "mts_last_error_string", "mts_tables_create", "mts_tables_destroy", "mts_tables_status",
+    "mts_tbe_forward", "mts_tbe_backward_workspace_bytes", "mts_tbe_backward_rowwise_adagrad",
+    "mts_cache_create", "mts_cache_destroy", "mts_cache_data", "mts_cache_dirty",
+    "mts_linearize_keys", "mts_cache_workspace_bytes", "mts_cache_lookup_insert",
+    "mts_cache_prefetch_misses", "mts_cache_writeback_evicted", "mts_cache_flush",
+    "mts_cache_export_state",
+)
+
+
+class MtsError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"mtrains_b200 error {code}: {msg}")
+        self.code = code
+
+
+class TableDesc(C.Structure):
+    _fields_ = [("T", C.c_int32), ("dtype", C.c_int32),
+                ("host_rows", C.POINTER(C.c_int64)), ("host_dim", C.POINTER(C.c_int32)),
+                ("host_weight_offset", C.POINTER(C.c_int64)), ("host_cache_id", C.POINTER(C.c_int32)),
+                ("dev_weights", C.c_void_p), ("host_weights_mapped", C.c_void_p),
+                ("momentum", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library.  Raises if it has not been built (python __graft_entry__.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python __graft_entry__.py` "
+                "(nvcc, sm_100a); there is no CPU fallback")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
+        L.mts_last_error_string.restype = C.c_char_p
+        L.mts_last_error_string.argtypes = []
+        L.mts_tables_create.argtypes = [C.POINTER(TableDesc), C.POINTER(vp)]
+        L.mts_tables_destroy.argtypes = [vp]
+        L.mts_tables_status.argtypes = [vp, C.POINTER(i32), vp]
+        L.mts_tbe_forward.argtypes = [vp, i32, vp, vp, i64, i32, vp, C.POINTER(vp), i32, vp, i64, vp]
+        L.mts_tbe_backward_workspace_bytes.restype = sz
+        L.mts_tbe_backward_workspace_bytes.argtypes = [vp, i32, i64]
+        L.mts_tbe_backward_rowwise_adagrad.argtypes = [vp, i32, vp, vp, i64, i32, vp, i64, f32, f32, vp,
+                                                       C.POINTER(vp), C.POINTER(vp), i32, vp, sz, vp, vp, vp]
+        L.mts_cache_create.argtypes = [C.POINTER(vp), i64, i64, i32, i32, i32, i32, i32]
+        L.mts_cache_destroy.argtypes = [vp]
+        L.mts_cache_data.restype = vp
+        L.mts_cache_data.argtypes = [vp]
+        L.mts_cache_dirty.restype = vp
+        L.mts_cache_dirty.argtypes = [vp]
+        L.mts_linearize_keys.argtypes = [vp, i32, i32, i32, vp, vp, i64, i64, vp, vp]
+        L.mts_cache_workspace_bytes.restype = sz
+        L.mts_cache_workspace_bytes.argtypes = [vp, i64]
+        L.mts_cache_lookup_insert.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
+        L.mts_cache_prefetch_misses.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
+        L.mts_cache_writeback_evicted.argtypes = [vp, vp, vp, vp, i64, vp, vp, vp]
+        L.mts_cache_flush.argtypes = [vp, vp, vp]
+        L.mts_cache_export_state.argtypes = [vp, vp, vp, vp, vp, vp]
+        for name in EXPORTS:
+            getattr(L, name)            # raises AttributeError when a declared symbol is missing
+        _lib = L
+    return _lib
+
+
+def last_error_string() -> str:
+    return lib().mts_last_error_string().decode()
+
+
+def _check(rc: int) -> None:
+    if rc != OK:
+        raise MtsError(rc, last_error_string())
+
+
+def _ptr(x):
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    return x.data_ptr()
+
+
+def _stream(s):
+    if s is None:
+        return None
+    if isinstance(s, int):
+        return s
+    return s.cuda_stream
+
+
+def _ptr_array(items: Optional[Sequence], n: int):
+    if items is None:
+        return None
+    arr = (C.c_void_p * max(n, 1))()
+    for i, it in enumerate(items):
+        arr[i] = _ptr(it)
+    return arr
+
+
+class Tables:
+    """Handle returned by mts_tables_create; keeps the host arrays of the description alive."""
+
+    def __init__(self, dtype: int, rows, dim, weight_offset, cache_id, dev_weights, host_weights_mapped,
+                 momentum):
+        T = len(rows)
+        self._rows = (C.c_int64 * T)(*[int(r) for r in rows])
+        self._dim = (C.c_int32 * T)(*[int(d) for d in dim])
+        self._woff = (C.c_int64 * T)(*[int(w) for w in weight_offset])
+        self._cid = (C.c_int32 * T)(*[int(c) for c in cache_id]) if cache_id is not None else None
+        self._keep = (dev_weights, host_weights_mapped, momentum)
+        d = TableDesc(T, dtype, self._rows, self._dim, self._woff,
+                      self._cid if self._cid is not None else C.POINTER(C.c_int32)(),
+                      _ptr(dev_weights), _ptr(host_weights_mapped), _ptr(momentum))
+        h = C.c_void_p()
+        _check(lib().mts_tables_create(C.byref(d), C.byref(h)))
+        self.handle = h
+        self.T = T
+        self.total_dim = int(sum(int(x) for x in dim))
+
+    def status(self, stream=None) -> int:
+        st = C.c_int32(0)
+        _check(lib().mts_tables_status(self.handle, C.byref(st), _stream(stream)))
+        return int(st.value)
+
+    def destroy(self):
+        if self.handle:
+            _check(lib().mts_tables_destroy(self.handle))
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def tables_create(dtype, rows, dim, weight_offset, cache_id, dev_weights, host_weights_mapped, momentum) -> Tables:
+    return Tables(dtype, rows, dim, weight_offset, cache_id, dev_weights, host_weights_mapped, momentum)
+
+
+def tbe_forward(tables: Tables, B: int, indices, offsets, N: int, pooling_mode: int, slot_of_lookup,
+                cache_data: Optional[Sequence], out, out_stride: int, stream=None) -> None:
+    n_caches = len(cache_data) if cache_data is not None else 0
+    _check(lib().mts_tbe_forward(tables.handle, B, _ptr(indices), _ptr(offsets), N, pooling_mode,
+                                 _ptr(slot_of_lookup), _ptr_array(cache_data, n_caches), n_caches, _ptr(out),
+                                 out_stride, _stream(stream)))
+
+
+def tbe_backward_workspace_bytes(tables: Tables, B: int, N: int) -> int:
+    return int(lib().mts_tbe_backward_workspace_bytes(tables.handle, B, N))
+
+
+def tbe_backward_rowwise_adagrad(tables: Tables, B: int, indices, offsets, N: int, pooling_mode: int, grad_out,
+                                 grad_stride: int, lr: float, eps: float, slot_of_lookup,
+                                 cache_data: Optional[Sequence], cache_dirty: Optional[Sequence], workspace,
+                                 workspace_bytes: int, uniq_rows_out=None, n_unique_out=None, stream=None) -> None:
+    n_caches = len(cache_data) if cache_data is not None else 0
+    _check(lib().mts_tbe_backward_rowwise_adagrad(
+        tables.handle, B, _ptr(indices), _ptr(offsets), N, pooling_mode, _ptr(grad_out), grad_stride, lr, eps,
+        _ptr(slot_of_lookup), _ptr_array(cache_data, n_caches), _ptr_array(cache_dirty, n_caches), n_caches,
+        _ptr(workspace), workspace_bytes, _ptr(uniq_rows_out), _ptr(n_unique_out), _stream(stream)))
+
+
+class Cache:
+    """Handle returned by mts_cache_create."""
+
+    def __init__(self, num_sets: int, key_space: int, dim: int, dtype: int, policy: int = POLICY_LRU,
+                 lock_depth: int = 0, ways: int = CACHE_WAYS):
+        h = C.c_void_p()
+        _check(lib().mts_cache_create(C.byref(h), num_sets, key_space, ways, dim, dtype, policy, lock_depth))
+        self.handle = h
+        self.num_sets, self.ways, self.dim, self.dtype = num_sets, ways, dim, dtype
+        self.data_ptr = int(lib().mts_cache_data(h))
+        self.dirty_ptr = int(lib().mts_cache_dirty(h))
+
+    def destroy(self):
+        if self.handle:
+            _check(lib().mts_cache_destroy(self.handle))
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def cache_create(num_sets, key_space, dim, dtype, policy=POLICY_LRU, lock_depth=0) -> Cache:
+    return Cache(num_sets, key_space, dim, dtype, policy, lock_depth)
+
+
+def linearize_keys(tables: Tables, t_begin: int, t_end: int, B: int, indices, offsets, lookup_begin: int, n: int,
+                   keys_out, stream=None) -> None:
+    _check(lib().mts_linearize_keys(tables.handle, t_begin, t_end, B, _ptr(indices), _ptr(offsets), lookup_begin,
+                                    n, _ptr(keys_out), _stream(stream)))
+
+
+def cache_workspace_bytes(cache: Cache, N: int) -> int:
+    return int(lib().mts_cache_workspace_bytes(cache.handle, N))
+
+
+def cache_lookup_insert(cache: Cache, keys, N: int, step: int, slot_of_lookup, miss_keys, miss_slots, evict_keys,
+                        evict_slots, evict_dirty, list_capacity: int, counters, workspace, workspace_bytes: int,
+                        stream=None) -> None:
+    _check(lib().mts_cache_lookup_insert(cache.handle, _ptr(keys), N, step, _ptr(slot_of_lookup), _ptr(miss_keys),
+                                         _ptr(miss_slots), _ptr(evict_keys), _ptr(evict_slots), _ptr(evict_dirty),
+                                         list_capacity, _ptr(counters), _ptr(workspace), workspace_bytes,
+                                         _stream(stream)))
+
+
+def cache_prefetch_misses(cache: Cache, host_rows_mapped, miss_keys, miss_slots, evict_slots, evict_dirty,
+                          list_capacity: int, counters, evict_staging, stream=None) -> None:
+    _check(lib().mts_cache_prefetch_misses(cache.handle, _ptr(host_rows_mapped), _ptr(miss_keys), _ptr(miss_slots),
+                                           _ptr(evict_slots), _ptr(evict_dirty), list_capacity, _ptr(counters),
+                                           _ptr(evict_staging), _stream(stream)))
+
+
+def cache_writeback_evicted(cache: Cache, host_rows_mapped, evict_keys, evict_dirty, list_capacity: int, counters,
+                            evict_staging, stream=None) -> None:
+    _check(lib().mts_cache_writeback_evicted(cache.handle, _ptr(host_rows_mapped), _ptr(evict_keys),
+                                             _ptr(evict_dirty), list_capacity, _ptr(counters), _ptr(evict_staging),
+                                             _stream(stream)))
+
+
+def cache_flush(cache: Cache, host_rows_mapped, stream=None) -> None:
+    _check(lib().mts_cache_flush(cache.handle, _ptr(host_rows_mapped), _stream(stream)))
+
+
+def cache_export_state(cache: Cache, tags, timestamps, counts, dirty, stream=None) -> None:
+    _check(lib().mts_cache_export_state(cache.handle, _ptr(tags), _ptr(timestamps), _ptr(counts), _ptr(dirty),
+                                        _stream(stream)))

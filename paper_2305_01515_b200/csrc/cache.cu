@@ -1,0 +1,659 @@
+// Software-managed row cache in HBM in front of pinned host memory: the cache class of
+// Section 5.3.1 (row-granular data, tags, per-entry timestamp states) and the GPU cache
+// kernels of Section 5.5 (tag/state lookup, LRU/LFU replacement, data lookup/update, data
+// movement), one level deep.
+//
+// lookup_insert, all on the caller's stream and without host synchronisation:
+//   keys -> stable sort by key -> distinct keys (U, on the device) -> set index of each
+//   distinct key -> stable sort of the distinct keys by set (keeps ascending key inside a
+//   set) -> one warp per touched set: probe (lane = way), refresh hits, order the evictable
+//   ways, hand them to the set's misses -> ordered compaction of the miss and evict lists
+//   (prefix sums, no atomics on list positions) -> slot of every lookup.
+// Every decision is a pure function of the cache state and the batch, so the slots, lists and
+// counters are reproducible bit for bit.
+#include <algorithm>
+
+#include "common.cuh"
+
+struct mts_cache {
+  int64_t S = 0;
+  int64_t key_space = 0;
+  int32_t ways = MTS_CACHE_WAYS;
+  int32_t dim = 0, dtype = 0, elem_bytes = 4, policy = 0, lock_depth = 0;
+  int32_t row_bytes = 0;
+  int32_t sm_count = 148;
+  uint32_t* tags = nullptr;      // [S*32]  0xffffffff = free
+  int32_t* ts = nullptr;         // [S*32]  -1 = free
+  uint32_t* freq = nullptr;      // [S*32]
+  uint8_t* dirty = nullptr;      // [S*32]
+  char* data = nullptr;          // [S*32, row_bytes]
+};
+
+namespace mts {
+
+constexpr uint32_t FREE_TAG = 0xffffffffu;
+constexpr int CACHE_THREADS = 256;
+
+__device__ __forceinline__ uint32_t set_of_key(uint32_t key, uint64_t S) {
+  const uint64_t x = (uint64_t)key * 0x9E3779B97F4A7C15ull;
+  return (uint32_t)__umul64hi(x, S);
+}
+
+__global__ void cache_init_state(uint32_t* tags, int32_t* ts, uint32_t* freq, uint8_t* dirty, int64_t n) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    tags[i] = FREE_TAG; ts[i] = -1; freq[i] = 0; dirty[i] = 0;
+  }
+}
+
+__global__ void cache_prepare_keys(const int64_t* __restrict__ keys, int64_t n, uint32_t* __restrict__ k32,
+                                   uint32_t* __restrict__ pos, int64_t* __restrict__ counters) {
+  const int64_t i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i0 < MTS_NUM_COUNTERS) counters[i0] = i0 == MTS_CNT_LOOKUPS ? n : 0;
+  for (int64_t i = i0; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    k32[i] = (uint32_t)keys[i];
+    pos[i] = (uint32_t)i;
+  }
+}
+
+// Distinct key u: its value, multiplicity and set.  Entries u >= U of the sort input are not
+// touched: the second sort runs on the device-side count U.
+__global__ void cache_describe_unique(const uint32_t* __restrict__ sorted_keys,
+                                      const uint32_t* __restrict__ seg_start,
+                                      const uint32_t* __restrict__ n_unique, uint64_t S,
+                                      uint32_t* __restrict__ ukey, uint32_t* __restrict__ mult,
+                                      uint32_t* __restrict__ set_keys, uint32_t* __restrict__ set_vals) {
+  const uint32_t U = *n_unique;
+  for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < U; u += (int64_t)gridDim.x * blockDim.x) {
+    const uint32_t s0 = seg_start[u];
+    const uint32_t k = sorted_keys[s0];
+    ukey[u] = k;
+    mult[u] = seg_start[u + 1] - s0;
+    set_keys[u] = set_of_key(k, S);
+    set_vals[u] = (uint32_t)u;
+  }
+}
+
+// One warp per touched set; lane = way.
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of member j (ascending)
+                    const uint32_t* __restrict__ member_uidx,     // distinct-key index of member j
+                    const uint32_t* __restrict__ sseg_start, const uint32_t* __restrict__ n_sets,
+                    const uint32_t* __restrict__ ukey, const uint32_t* __restrict__ mult,
+                    uint32_t* __restrict__ tags, int32_t* __restrict__ ts, uint32_t* __restrict__ freq,
+                    uint8_t* __restrict__ dirty, int32_t step, int32_t lock_depth, int32_t policy,
+                    int32_t* __restrict__ slot_of_uniq, uint8_t* __restrict__ member_flag,
+                    uint32_t* __restrict__ member_old_key, uint8_t* __restrict__ member_old_dirty,
+                    int32_t* __restrict__ member_slot, unsigned long long* __restrict__ counters) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const uint32_t NS = *n_sets;
+  unsigned long long c_hit_lookups = 0, c_uhits = 0, c_dirty = 0, c_overflow = 0;
+  for (int64_t si = warp0; si < NS; si += nwarps) {
+    const uint32_t j0 = sseg_start[si], j1 = sseg_start[si + 1];
+    const uint32_t set = set_sorted[j0];
+    const int64_t slot0 = (int64_t)set * 32;
+    uint32_t tag = tags[slot0 + lane];
+    int32_t stamp = ts[slot0 + lane];
+    uint32_t cnt = freq[slot0 + lane];
+    bool touched = false;
+    // pass 1: probe every member against the state before the call, refresh the hits
+    for (uint32_t jb = j0; jb < j1; jb += 32) {
+      const uint32_t j = jb + lane;
+      uint32_t u = 0, k = 0, mu = 0;
+      if (j < j1) { u = member_uidx[j]; k = ukey[u]; mu = mult[u]; }
+      const int m = (int)min(32u, j1 - jb);
+      uint8_t my_flag = 0;
+      int32_t my_slot = -1;
+      for (int q = 0; q < m; ++q) {
+        const uint32_t kq = __shfl_sync(0xffffffffu, k, q);
+        const uint32_t mq = __shfl_sync(0xffffffffu, mu, q);
+        const uint32_t hit = __ballot_sync(0xffffffffu, tag == kq && tag != FREE_TAG);
+        if (hit) {
+          const int way = __ffs(hit) - 1;
+          if (lane == way) { stamp = step; cnt += mq; touched = true; }
+          if (lane == q) { my_flag = 3; my_slot = (int32_t)(slot0 + way); }
+          c_hit_lookups += mq;
+          c_uhits += 1;
+        }
+      }
+      if (j < j1) {
+        member_flag[j] = my_flag;          // 3 = hit, rewritten below for misses
+        member_slot[j] = my_slot;
+      }
+    }
+    // candidates after the refresh: ways outside the lock window, free ways first by their -1 stamp
+    const bool cand = stamp < step - lock_depth;
+    const uint32_t cand_mask = __ballot_sync(0xffffffffu, cand);
+    const int ncand = __popc(cand_mask);
+    int rank = 0;
+    for (int q = 0; q < 32; ++q) {
+      const int32_t sq = __shfl_sync(0xffffffffu, stamp, q);
+      const uint32_t fq = __shfl_sync(0xffffffffu, cnt, q);
+      if ((cand_mask >> q) & 1u) {
+        bool before;
+        if (policy == MTS_POLICY_LFU && fq != cnt) before = fq < cnt;
+        else if (sq != stamp) before = sq < stamp;
+        else before = q < lane;
+        rank += before ? 1 : 0;
+      }
+    }
+    // pass 2: the k-th missing key (ascending) takes the k-th candidate
+    int placed = 0;
+    uint8_t dirty_reg = 0;
+    bool dirty_loaded = false;
+    for (uint32_t jb = j0; jb < j1; jb += 32) {
+      const uint32_t j = jb + lane;
+      uint32_t u = 0, k = 0, mu = 0;
+      uint8_t fl = 3;
+      if (j < j1) { u = member_uidx[j]; k = ukey[u]; mu = mult[u]; fl = member_flag[j]; }
+      const int m = (int)min(32u, j1 - jb);
+      const uint32_t miss_mask = __ballot_sync(0xffffffffu, j < j1 && fl == 0);
+      uint8_t my_flag = fl;
+      int32_t my_slot = -1;
+      uint32_t my_old = FREE_TAG;
+      uint8_t my_old_dirty = 0;
+      for (int q = 0; q < m; ++q) {
+        if (!((miss_mask >> q) & 1u)) continue;
+        const uint32_t kq = __shfl_sync(0xffffffffu, k, q);
+        const uint32_t mq = __shfl_sync(0xffffffffu, mu, q);
+        if (placed < ncand) {
+          const uint32_t sel = __ballot_sync(0xffffffffu, cand && rank == placed);
+          const int way = __ffs(sel) - 1;
+          uint32_t old_tag = 0;
+          uint8_t old_dirty = 0;
+          if (lane == way) {
+            old_tag = tag;
+            if (!dirty_loaded) { dirty_reg = dirty[slot0 + lane]; dirty_loaded = true; }
+            old_dirty = tag != FREE_TAG ? dirty_reg : 0;
+            tag = kq; stamp = step; cnt = mq; dirty_reg = 0; touched = true;
+          }
+          old_tag = __shfl_sync(0xffffffffu, old_tag, way);
+          old_dirty = (uint8_t)__shfl_sync(0xffffffffu, (uint32_t)old_dirty, way);
+          if (lane == q) { my_flag = 1; my_slot = (int32_t)(slot0 + way); my_old = old_tag; my_old_dirty = old_dirty; }
+          if (old_tag != FREE_TAG && old_dirty) c_dirty += 1;
+          ++placed;
+        } else {
+          if (lane == q) { my_flag = 2; my_slot = -1; }
+          c_overflow += 1;
+        }
+      }
+      if (j < j1 && fl == 0) {
+        member_flag[j] = my_flag;          // 1 = placed, 2 = overflow
+        member_slot[j] = my_slot;
+        member_old_key[j] = my_old;
+        member_old_dirty[j] = my_old_dirty;
+      }
+      if (j < j1) slot_of_uniq[u] = (fl == 0) ? my_slot : member_slot[j];
+    }
+    if (touched) {
+      tags[slot0 + lane] = tag;
+      ts[slot0 + lane] = stamp;
+      freq[slot0 + lane] = cnt;
+      if (dirty_loaded) dirty[slot0 + lane] = dirty_reg;
+    }
+  }
+  if (lane == 0) {
+    if (c_hit_lookups) atomicAdd(&counters[MTS_CNT_HIT_LOOKUPS], c_hit_lookups);
+    if (c_uhits) atomicAdd(&counters[MTS_CNT_UNIQUE_HITS], c_uhits);
+    if (c_dirty) atomicAdd(&counters[MTS_CNT_EVICTED_DIRTY], c_dirty);
+    if (c_overflow) atomicAdd(&counters[MTS_CNT_OVERFLOW], c_overflow);
+  }
+}
+
+// Ordered compaction of the members flagged "placed" (miss list) and of those whose victim
+// held a row (evict list): count per block, scan the block counts, write.
+__device__ __forceinline__ uint32_t block_scan_256(uint32_t v, uint32_t* sh, uint32_t* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += y;
+  }
+  if (lane == 31) sh[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t w = lane < 8 ? sh[lane] : 0u;
+    uint32_t winc = w;
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) {
+      uint32_t y = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += y;
+    }
+    if (lane < 8) sh[lane] = winc - w;
+    if (lane == 7) sh[8] = winc;
+  }
+  __syncthreads();
+  const uint32_t res = sh[warp] + inc - v;
+  *total = sh[8];
+  __syncthreads();
+  return res;
+}
+
+constexpr int LIST_BLOCKS = 1024;
+
+__device__ __forceinline__ int64_t list_per_block(int64_t n, int G) {
+  const int64_t per = (n + G - 1) / G;
+  return (per + CACHE_THREADS - 1) / CACHE_THREADS * CACHE_THREADS;
+}
+
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_count_lists(const uint8_t* __restrict__ member_flag, const uint32_t* __restrict__ member_old_key,
+                  const uint32_t* __restrict__ n_unique, uint32_t* __restrict__ cnt_miss,
+                  uint32_t* __restrict__ cnt_evict) {
+  __shared__ uint32_t sh[9];
+  const int64_t n = *n_unique;
+  const int64_t per = list_per_block(n, gridDim.x);
+  const int64_t begin = (int64_t)blockIdx.x * per, end = min(n, begin + per);
+  uint32_t a = 0, b = 0;
+  for (int64_t j = begin + threadIdx.x; j < end; j += CACHE_THREADS) {
+    if (member_flag[j] == 1) { a += 1; b += member_old_key[j] != FREE_TAG ? 1u : 0u; }
+  }
+  uint32_t ta, tb;
+  block_scan_256(a, sh, &ta);
+  block_scan_256(b, sh, &tb);
+  if (threadIdx.x == 0) { cnt_miss[blockIdx.x] = ta; cnt_evict[blockIdx.x] = tb; }
+}
+
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_scan_lists(uint32_t* __restrict__ cnt_miss, uint32_t* __restrict__ cnt_evict, int G,
+                 const uint32_t* __restrict__ n_unique, int64_t n_lookups, int64_t* __restrict__ counters) {
+  __shared__ uint32_t sh[9];
+  constexpr int PER = LIST_BLOCKS / CACHE_THREADS;
+  const int j0 = threadIdx.x * PER;
+  for (int which = 0; which < 2; ++which) {
+    uint32_t* cnt = which == 0 ? cnt_miss : cnt_evict;
+    uint32_t v[PER];
+    uint32_t s = 0;
+#pragma unroll
+    for (int k = 0; k < PER; ++k) { v[k] = j0 + k < G ? cnt[j0 + k] : 0u; s += v[k]; }
+    uint32_t total;
+    uint32_t ex = block_scan_256(s, sh, &total);
+#pragma unroll
+    for (int k = 0; k < PER; ++k) { if (j0 + k < G) cnt[j0 + k] = ex; ex += v[k]; }
+    if (threadIdx.x == 0) counters[which == 0 ? MTS_CNT_INSERTED : MTS_CNT_EVICTED] = (int64_t)total;
+  }
+  if (threadIdx.x == 0) {
+    const int64_t U = *n_unique;
+    counters[MTS_CNT_UNIQUE] = U;
+    counters[MTS_CNT_MISS_LOOKUPS] = n_lookups - counters[MTS_CNT_HIT_LOOKUPS];
+    counters[MTS_CNT_UNIQUE_MISSES] = U - counters[MTS_CNT_UNIQUE_HITS];
+  }
+}
+
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_write_lists(const uint8_t* __restrict__ member_flag, const uint32_t* __restrict__ member_old_key,
+                  const uint8_t* __restrict__ member_old_dirty, const int32_t* __restrict__ member_slot,
+                  const uint32_t* __restrict__ member_uidx, const uint32_t* __restrict__ ukey,
+                  const uint32_t* __restrict__ n_unique, const uint32_t* __restrict__ base_miss,
+                  const uint32_t* __restrict__ base_evict, int64_t capacity,
+                  int64_t* __restrict__ miss_keys, int32_t* __restrict__ miss_slots,
+                  int64_t* __restrict__ evict_keys, int32_t* __restrict__ evict_slots,
+                  uint8_t* __restrict__ evict_dirty) {
+  __shared__ uint32_t sh[9];
+  const int64_t n = *n_unique;
+  const int64_t per = list_per_block(n, gridDim.x);
+  const int64_t begin = (int64_t)blockIdx.x * per, end = min(n, begin + per);
+  uint32_t bm = base_miss[blockIdx.x], be = base_evict[blockIdx.x];
+  for (int64_t t0 = begin; t0 < end; t0 += CACHE_THREADS) {
+    const int64_t j = t0 + threadIdx.x;
+    const bool placed = j < end && member_flag[j] == 1;
+    const bool ev = placed && member_old_key[j] != FREE_TAG;
+    uint32_t ta, tb;
+    const uint32_t pa = block_scan_256(placed ? 1u : 0u, sh, &ta);
+    const uint32_t pb = block_scan_256(ev ? 1u : 0u, sh, &tb);
+    if (placed && (int64_t)(bm + pa) < capacity) {
+      miss_keys[bm + pa] = (int64_t)ukey[member_uidx[j]];
+      miss_slots[bm + pa] = member_slot[j];
+    }
+    if (ev && (int64_t)(be + pb) < capacity) {
+      evict_keys[be + pb] = (int64_t)member_old_key[j];
+      evict_slots[be + pb] = member_slot[j];
+      evict_dirty[be + pb] = member_old_dirty[j];
+    }
+    bm += ta;
+    be += tb;
+  }
+}
+
+__global__ void cache_scatter_slots(const uint32_t* __restrict__ sorted_pos, const uint32_t* __restrict__ uniq_idx,
+                                    const int32_t* __restrict__ slot_of_uniq, int64_t n,
+                                    int32_t* __restrict__ slot_of_lookup) {
+  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += (int64_t)gridDim.x * blockDim.x)
+    slot_of_lookup[sorted_pos[p]] = slot_of_uniq[uniq_idx[p]];
+}
+
+// ------------------------------------------------------------------------------------ data movement
+// Row copies in 16-byte pieces; thread i of the flattened (row, piece) space moves one piece,
+// UNROLL independent pieces per thread are in flight before the first store.
+
+constexpr int COPY_UNROLL = 4;
+
+template <typename SrcOf, typename DstOf>
+__device__ __forceinline__ void copy_rows(int64_t n_rows, int vec16, SrcOf src_of, DstOf dst_of) {
+  const int64_t total = n_rows * vec16;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride * COPY_UNROLL) {
+    uint4 v[COPY_UNROLL];
+    char* dst[COPY_UNROLL];
+#pragma unroll
+    for (int u = 0; u < COPY_UNROLL; ++u) {
+      const int64_t e = i + u * stride;
+      dst[u] = nullptr;
+      if (e < total) {
+        const int64_t r = e / vec16;
+        const int c = (int)(e - r * vec16);
+        const char* s = src_of(r);
+        dst[u] = dst_of(r);
+        if (s != nullptr && dst[u] != nullptr) {
+          v[u] = *reinterpret_cast<const uint4*>(s + (int64_t)c * 16);
+          dst[u] += (int64_t)c * 16;
+        } else {
+          dst[u] = nullptr;
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < COPY_UNROLL; ++u)
+      if (dst[u] != nullptr) *reinterpret_cast<uint4*>(dst[u]) = v[u];
+  }
+}
+
+__device__ __forceinline__ int64_t list_len(const int64_t* counters, int which, int64_t capacity) {
+  const int64_t n = counters[which];
+  return n < capacity ? n : capacity;
+}
+
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_save_victims(const char* __restrict__ data, int row_bytes, const int32_t* __restrict__ evict_slots,
+                   const uint8_t* __restrict__ evict_dirty, const int64_t* __restrict__ counters,
+                   int64_t capacity, char* __restrict__ staging) {
+  const int64_t n = list_len(counters, MTS_CNT_EVICTED, capacity);
+  copy_rows(n, row_bytes / 16,
+            [&](int64_t k) { return evict_dirty[k] ? data + (int64_t)evict_slots[k] * row_bytes : nullptr; },
+            [&](int64_t k) { return staging + k * row_bytes; });
+}
+
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_fetch_misses(char* __restrict__ data, int row_bytes, const char* __restrict__ host_rows,
+                   const int64_t* __restrict__ miss_keys, const int32_t* __restrict__ miss_slots,
+                   const int64_t* __restrict__ counters, int64_t capacity) {
+  const int64_t n = list_len(counters, MTS_CNT_INSERTED, capacity);
+  copy_rows(n, row_bytes / 16,
+            [&](int64_t k) { return host_rows + miss_keys[k] * row_bytes; },
+            [&](int64_t k) { return data + (int64_t)miss_slots[k] * row_bytes; });
+}
+
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_write_victims(char* __restrict__ host_rows, int row_bytes, const int64_t* __restrict__ evict_keys,
+                    const uint8_t* __restrict__ evict_dirty, const int64_t* __restrict__ counters,
+                    int64_t capacity, const char* __restrict__ staging) {
+  const int64_t n = list_len(counters, MTS_CNT_EVICTED, capacity);
+  copy_rows(n, row_bytes / 16,
+            [&](int64_t k) { return evict_dirty[k] ? staging + k * row_bytes : nullptr; },
+            [&](int64_t k) { return host_rows + evict_keys[k] * row_bytes; });
+}
+
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_flush_rows(const char* __restrict__ data, int row_bytes, const uint32_t* __restrict__ tags,
+                 const uint8_t* __restrict__ dirty, int64_t n_slots, char* __restrict__ host_rows) {
+  copy_rows(n_slots, row_bytes / 16,
+            [&](int64_t s) { return (tags[s] != FREE_TAG && dirty[s]) ? data + s * row_bytes : nullptr; },
+            [&](int64_t s) { return host_rows + (int64_t)tags[s] * row_bytes; });
+}
+
+__global__ void cache_clear_dirty(uint8_t* dirty, int64_t n) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    dirty[i] = 0;
+}
+
+__global__ void cache_export(const uint32_t* __restrict__ tags, const int32_t* __restrict__ ts,
+                             const uint32_t* __restrict__ freq, const uint8_t* __restrict__ dirty, int64_t n,
+                             int64_t* o_tags, int64_t* o_ts, int64_t* o_freq, uint8_t* o_dirty) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    if (o_tags) o_tags[i] = tags[i] == FREE_TAG ? -1 : (int64_t)tags[i];
+    if (o_ts) o_ts[i] = (int64_t)ts[i];
+    if (o_freq) o_freq[i] = (int64_t)freq[i];
+    if (o_dirty) o_dirty[i] = dirty[i];
+  }
+}
+
+struct CacheLayout {
+  size_t keys_a, keys_b, vals_a, vals_b, uniq_idx, seg_start, ukey, mult, set_a, set_b, sval_a, sval_b,
+      sseg_start, slot_of_uniq, member_flag, member_old_key, member_old_dirty, member_slot, hist, scan, cnt_miss,
+      cnt_evict, n_unique, n_sets, total;
+};
+
+static CacheLayout cache_layout(int64_t N) {
+  CacheLayout L;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t n = (size_t)(N > 0 ? N : 1);
+  L.keys_a = take(n * 4); L.keys_b = take(n * 4); L.vals_a = take(n * 4); L.vals_b = take(n * 4);
+  L.uniq_idx = take(n * 4); L.seg_start = take((n + 1) * 4);
+  L.ukey = take(n * 4); L.mult = take(n * 4);
+  L.set_a = take(n * 4); L.set_b = take(n * 4); L.sval_a = take(n * 4); L.sval_b = take(n * 4);
+  L.sseg_start = take((n + 1) * 4);
+  L.slot_of_uniq = take(n * 4);
+  L.member_flag = take(n); L.member_old_key = take(n * 4); L.member_old_dirty = take(n); L.member_slot = take(n * 4);
+  L.hist = take(sort_hist_words() * 4);
+  L.scan = take(scan_scratch_words() * 4);
+  L.cnt_miss = take(LIST_BLOCKS * 4); L.cnt_evict = take(LIST_BLOCKS * 4);
+  L.n_unique = take(256); L.n_sets = take(256);
+  L.total = off;
+  return L;
+}
+
+}  // namespace mts
+
+using namespace mts;
+
+extern "C" int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_space, int32_t ways, int32_t dim,
+                                int32_t dtype, int32_t policy, int32_t lock_depth) {
+  if (!out) return set_error(MTS_ERR_INVALID_ARG, "cache_create: null out");
+  *out = nullptr;
+  if (ways != MTS_CACHE_WAYS) return set_error(MTS_ERR_INVALID_ARG, "cache_create: ways must be %d", MTS_CACHE_WAYS);
+  if (num_sets < 1 || num_sets * MTS_CACHE_WAYS >= (1ll << 31))
+    return set_error(MTS_ERR_INVALID_ARG, "cache_create: num_sets %lld out of range", (long long)num_sets);
+  if (key_space < 1 || key_space >= (1ll << 32) - 1)
+    return set_error(MTS_ERR_INVALID_ARG, "cache_create: key_space %lld out of range", (long long)key_space);
+  if (dtype != MTS_DTYPE_FP32 && dtype != MTS_DTYPE_FP16) return set_error(MTS_ERR_INVALID_ARG, "cache_create: dtype");
+  if (policy != MTS_POLICY_LRU && policy != MTS_POLICY_LFU) return set_error(MTS_ERR_INVALID_ARG, "cache_create: policy");
+  if (lock_depth < 0 || dim < 1) return set_error(MTS_ERR_INVALID_ARG, "cache_create: lock_depth / dim");
+  const int eb = dtype == MTS_DTYPE_FP32 ? 4 : 2;
+  if ((dim * eb) % 16) return set_error(MTS_ERR_ALIGNMENT, "cache_create: row bytes %d not a multiple of 16", dim * eb);
+  mts_cache* c = new mts_cache();
+  c->S = num_sets; c->key_space = key_space; c->dim = dim; c->dtype = dtype; c->elem_bytes = eb;
+  c->policy = policy; c->lock_depth = lock_depth; c->row_bytes = dim * eb;
+  const int64_t n = num_sets * MTS_CACHE_WAYS;
+  int dev = 0, sms = 0;
+  int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
+  if (rc == MTS_OK) rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "sm count");
+  if (rc == MTS_OK && sms > 0) c->sm_count = sms;
+  if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->tags, n * 4), "cudaMalloc(tags)");
+  if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->ts, n * 4), "cudaMalloc(timestamps)");
+  if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->freq, n * 4), "cudaMalloc(counts)");
+  if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->dirty, n), "cudaMalloc(dirty)");
+  if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->data, (size_t)n * c->row_bytes), "cudaMalloc(cache rows)");
+  if (rc == MTS_OK) {
+    cache_init_state<<<c->sm_count * 4, 256>>>(c->tags, c->ts, c->freq, c->dirty, n);
+    rc = check_launch("cache_init_state");
+  }
+  if (rc == MTS_OK) rc = check_cuda(cudaMemset(c->data, 0, (size_t)n * c->row_bytes), "cudaMemset(cache rows)");
+  if (rc == MTS_OK) rc = check_cuda(cudaDeviceSynchronize(), "cache_create sync");
+  if (rc != MTS_OK) { mts_cache_destroy(c); return rc; }
+  *out = c;
+  return MTS_OK;
+}
+
+extern "C" int mts_cache_destroy(mts_cache* c) {
+  if (!c) return MTS_OK;
+  cudaFree(c->tags); cudaFree(c->ts); cudaFree(c->freq); cudaFree(c->dirty); cudaFree(c->data);
+  delete c;
+  return MTS_OK;
+}
+
+extern "C" void* mts_cache_data(mts_cache* c) { return c ? c->data : nullptr; }
+extern "C" uint8_t* mts_cache_dirty(mts_cache* c) { return c ? c->dirty : nullptr; }
+
+__global__ void linearize_group_keys(const TableMeta* __restrict__ meta, int32_t t_begin, int64_t n_bags, int32_t B,
+                                     const int64_t* __restrict__ indices, const int64_t* __restrict__ offsets,
+                                     int64_t lookup_begin, int64_t n, int64_t* __restrict__ keys_out,
+                                     int32_t* status) {
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t gb = gid / 8;
+  if (gb >= n_bags) return;
+  const int sub = (int)(gid % 8);
+  const int64_t bag = (int64_t)t_begin * B + gb;
+  const int32_t t = (int32_t)(bag / B);
+  const int64_t rows = meta[t].rows;
+  const int64_t roff = meta[t].row_offset - meta[t_begin].row_offset;
+  const int64_t i1 = offsets[bag + 1];
+  for (int64_t i = offsets[bag] + sub; i < i1; i += 8) {
+    const int64_t o = i - lookup_begin;
+    if (o >= 0 && o < n) keys_out[o] = roff + clamp_index(indices[i], rows, status);
+  }
+}
+
+extern "C" int mts_linearize_keys(const mts_tables* h, int32_t t_begin, int32_t t_end, int32_t B,
+                                  const int64_t* indices, const int64_t* offsets, int64_t lookup_begin, int64_t n,
+                                  int64_t* keys_out, void* stream) {
+  if (!h || !offsets || B < 1 || t_begin < 0 || t_end > h->T || t_begin >= t_end || n < 0 || lookup_begin < 0 ||
+      (n > 0 && (!indices || !keys_out)))
+    return set_error(MTS_ERR_INVALID_ARG, "linearize_keys: bad argument");
+  if (n == 0) return MTS_OK;
+  const int64_t n_bags = (int64_t)(t_end - t_begin) * B;
+  linearize_group_keys<<<(unsigned)ceil_div(n_bags * 8, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      h->d_meta, t_begin, n_bags, B, indices, offsets, lookup_begin, n, keys_out, h->d_status);
+  return check_launch("linearize_group_keys");
+}
+
+extern "C" size_t mts_cache_workspace_bytes(const mts_cache* c, int64_t N) {
+  if (!c || N < 0) return 0;
+  return cache_layout(N).total;
+}
+
+extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_t N, int64_t step,
+                                       int32_t* slot_of_lookup, int64_t* miss_keys, int32_t* miss_slots,
+                                       int64_t* evict_keys, int32_t* evict_slots, uint8_t* evict_dirty,
+                                       int64_t list_capacity, int64_t* counters, void* workspace,
+                                       size_t workspace_bytes, void* stream) {
+  if (!c || !counters || N < 0 || list_capacity < 0 || step < 0 || step >= (1ll << 31) - 1)
+    return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert: bad argument");
+  if (N > 0 && (!keys || !slot_of_lookup))
+    return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert: null keys / slot_of_lookup");
+  if (list_capacity > 0 && (!miss_keys || !miss_slots || !evict_keys || !evict_slots || !evict_dirty))
+    return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert: null list buffer");
+  if (N >= (1ll << 32) - 1) return set_error(MTS_ERR_UNSUPPORTED, "cache_lookup_insert: N must fit 32 bits");
+  const CacheLayout L = cache_layout(N);
+  if (!workspace || ((uintptr_t)workspace & 255))
+    return set_error(MTS_ERR_ALIGNMENT, "cache_lookup_insert: workspace must be non-null and 256-byte aligned");
+  if (workspace_bytes < L.total)
+    return set_error(MTS_ERR_WORKSPACE, "cache_lookup_insert: workspace of %zu bytes, %zu needed", workspace_bytes, L.total);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  auto U32 = [&](size_t off) { return reinterpret_cast<uint32_t*>(ws + off); };
+  const int grid = c->sm_count * 8;
+  cache_prepare_keys<<<grid, 256, 0, s>>>(keys, N, U32(L.keys_a), U32(L.vals_a), counters);
+  int rc = check_launch("cache_prepare_keys");
+  if (rc != MTS_OK) return rc;
+  uint32_t* n_unique = U32(L.n_unique);
+  uint32_t* n_sets = U32(L.n_sets);
+  if (N == 0) {
+    return MTS_OK;   // counters already written: all zero
+  }
+  int key_bits = 1;
+  while (key_bits < 32 && (1ll << key_bits) < c->key_space) ++key_bits;
+  uint32_t *sk = nullptr, *sp = nullptr;
+  rc = radix_sort_pairs(U32(L.keys_a), U32(L.vals_a), U32(L.keys_b), U32(L.vals_b), N, nullptr, key_bits,
+                        U32(L.hist), &sk, &sp, s);
+  if (rc != MTS_OK) return rc;
+  rc = unique_segments(sk, N, nullptr, U32(L.seg_start), U32(L.uniq_idx), n_unique, U32(L.scan), s);
+  if (rc != MTS_OK) return rc;
+  cache_describe_unique<<<grid, 256, 0, s>>>(sk, U32(L.seg_start), n_unique, (uint64_t)c->S, U32(L.ukey),
+                                             U32(L.mult), U32(L.set_a), U32(L.sval_a));
+  rc = check_launch("cache_describe_unique");
+  if (rc != MTS_OK) return rc;
+  int set_bits = 0;
+  while ((1ll << set_bits) < c->S) ++set_bits;
+  uint32_t *ss = nullptr, *su = nullptr;
+  rc = radix_sort_pairs(U32(L.set_a), U32(L.sval_a), U32(L.set_b), U32(L.sval_b), N, n_unique, set_bits,
+                        U32(L.hist), &ss, &su, s);
+  if (rc != MTS_OK) return rc;
+  rc = unique_segments(ss, N, n_unique, U32(L.sseg_start), nullptr, n_sets, U32(L.scan), s);
+  if (rc != MTS_OK) return rc;
+  int32_t* slot_of_uniq = reinterpret_cast<int32_t*>(ws + L.slot_of_uniq);
+  uint8_t* member_flag = reinterpret_cast<uint8_t*>(ws + L.member_flag);
+  uint8_t* member_old_dirty = reinterpret_cast<uint8_t*>(ws + L.member_old_dirty);
+  int32_t* member_slot = reinterpret_cast<int32_t*>(ws + L.member_slot);
+  cache_probe_replace<<<grid, CACHE_THREADS, 0, s>>>(
+      ss, su, U32(L.sseg_start), n_sets, U32(L.ukey), U32(L.mult), c->tags, c->ts, c->freq, c->dirty, (int32_t)step,
+      c->lock_depth, c->policy, slot_of_uniq, member_flag, U32(L.member_old_key), member_old_dirty, member_slot,
+      reinterpret_cast<unsigned long long*>(counters));
+  rc = check_launch("cache_probe_replace");
+  if (rc != MTS_OK) return rc;
+  const int G = (int)std::min<int64_t>((int64_t)LIST_BLOCKS, ceil_div(N, CACHE_THREADS * 4));
+  cache_count_lists<<<G, CACHE_THREADS, 0, s>>>(member_flag, U32(L.member_old_key), n_unique, U32(L.cnt_miss),
+                                                U32(L.cnt_evict));
+  cache_scan_lists<<<1, CACHE_THREADS, 0, s>>>(U32(L.cnt_miss), U32(L.cnt_evict), G, n_unique, N, counters);
+  cache_write_lists<<<G, CACHE_THREADS, 0, s>>>(member_flag, U32(L.member_old_key), member_old_dirty, member_slot, su,
+                                                U32(L.ukey), n_unique, U32(L.cnt_miss), U32(L.cnt_evict),
+                                                list_capacity, miss_keys, miss_slots, evict_keys, evict_slots,
+                                                evict_dirty);
+  cache_scatter_slots<<<grid, 256, 0, s>>>(sp, U32(L.uniq_idx), slot_of_uniq, N, slot_of_lookup);
+  return check_launch("cache lists / scatter");
+}
+
+extern "C" int mts_cache_prefetch_misses(mts_cache* c, const void* host_rows_mapped, const int64_t* miss_keys,
+                                         const int32_t* miss_slots, const int32_t* evict_slots,
+                                         const uint8_t* evict_dirty, int64_t list_capacity, const int64_t* counters,
+                                         void* evict_staging, void* stream) {
+  if (!c || !host_rows_mapped || !counters || list_capacity < 0 ||
+      (list_capacity > 0 && (!miss_keys || !miss_slots || !evict_slots || !evict_dirty || !evict_staging)))
+    return set_error(MTS_ERR_INVALID_ARG, "cache_prefetch_misses: null argument");
+  if (((uintptr_t)host_rows_mapped | (uintptr_t)evict_staging) & 15)
+    return set_error(MTS_ERR_ALIGNMENT, "cache_prefetch_misses: buffers must be 16-byte aligned");
+  if (list_capacity == 0) return MTS_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int grid = c->sm_count * 8;
+  cache_save_victims<<<grid, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, evict_slots, evict_dirty, counters,
+                                                    list_capacity, static_cast<char*>(evict_staging));
+  cache_fetch_misses<<<grid, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, static_cast<const char*>(host_rows_mapped),
+                                                    miss_keys, miss_slots, counters, list_capacity);
+  return check_launch("cache_save_victims / cache_fetch_misses");
+}
+
+extern "C" int mts_cache_writeback_evicted(mts_cache* c, void* host_rows_mapped, const int64_t* evict_keys,
+                                           const uint8_t* evict_dirty, int64_t list_capacity,
+                                           const int64_t* counters, const void* evict_staging, void* stream) {
+  if (!c || !host_rows_mapped || !counters || list_capacity < 0 ||
+      (list_capacity > 0 && (!evict_keys || !evict_dirty || !evict_staging)))
+    return set_error(MTS_ERR_INVALID_ARG, "cache_writeback_evicted: null argument");
+  if (((uintptr_t)host_rows_mapped | (uintptr_t)evict_staging) & 15)
+    return set_error(MTS_ERR_ALIGNMENT, "cache_writeback_evicted: buffers must be 16-byte aligned");
+  if (list_capacity == 0) return MTS_OK;
+  cache_write_victims<<<c->sm_count * 8, CACHE_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<char*>(host_rows_mapped), c->row_bytes, evict_keys, evict_dirty, counters, list_capacity,
+      static_cast<const char*>(evict_staging));
+  return check_launch("cache_write_victims");
+}
+
+extern "C" int mts_cache_flush(mts_cache* c, void* host_rows_mapped, void* stream) {
+  if (!c || !host_rows_mapped) return set_error(MTS_ERR_INVALID_ARG, "cache_flush: null argument");
+  if ((uintptr_t)host_rows_mapped & 15) return set_error(MTS_ERR_ALIGNMENT, "cache_flush: host buffer alignment");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int64_t n = c->S * MTS_CACHE_WAYS;
+  cache_flush_rows<<<c->sm_count * 8, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, c->tags, c->dirty, n,
+                                                             static_cast<char*>(host_rows_mapped));
+  cache_clear_dirty<<<c->sm_count * 4, 256, 0, s>>>(c->dirty, n);
+  return check_launch("cache_flush");
+}
+
+extern "C" int mts_cache_export_state(mts_cache* c, int64_t* tags, int64_t* timestamps, int64_t* counts,
+                                      uint8_t* dirty, void* stream) {
+  if (!c) return set_error(MTS_ERR_INVALID_ARG, "cache_export_state: null cache");
+  cache_export<<<c->sm_count * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      c->tags, c->ts, c->freq, c->dirty, c->S * MTS_CACHE_WAYS, tags, timestamps, counts, dirty);
+  return check_launch("cache_export");
+}

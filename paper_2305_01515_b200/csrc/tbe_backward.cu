@@ -1,0 +1,465 @@
+// Backward of the pooled lookup fused with row-wise Adagrad on the touched rows (Section 2.1.2:
+// optimizer with few states per row; Section 5.9: aggregate, optimize, write rows back).
+//
+// Steps, all on the caller's stream, no host synchronisation:
+//   1. linearize_lookups : key = linear row id of every lookup, value = its position,
+//                          bag_of_pos[position] = bag id
+//   2. radix_sort_pairs  : stable sort by key; equal rows keep ascending position
+//   3. reduce_chunks     : one warp per CHUNK consecutive sorted lookups.  Gradients of a row
+//                          are summed in sorted order; a row whose lookups lie inside the
+//                          chunk is updated at once (Adagrad fused); the piece of a row that
+//                          continues over a chunk border is written as a partial sum
+//   4. combine_partials  : the chunk in which such a row starts adds the partial sums in
+//                          chunk order and applies the update
+// The summation tree depends only on the sorted order and CHUNK, so two runs give the same
+// bits.  No thread ever writes a word another thread of the same launch writes.
+#include "common.cuh"
+
+namespace mts {
+
+constexpr int BWD_CHUNK = 128;
+constexpr int BWD_WARPS = 4;
+constexpr int LIN_GROUP = 8;     // lanes per bag in linearize_lookups
+
+__global__ void __launch_bounds__(256)
+linearize_lookups(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B,
+                  const int64_t* __restrict__ indices, const int64_t* __restrict__ offsets,
+                  uint32_t* __restrict__ keys, uint32_t* __restrict__ vals,
+                  uint32_t* __restrict__ bag_of_pos, int32_t* status) {
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t bag = gid / LIN_GROUP;
+  if (bag >= n_bags) return;
+  const int sub = (int)(gid % LIN_GROUP);
+  const int32_t t = (int32_t)(bag / B);
+  const int64_t rows = meta[t].rows;
+  const int64_t roff = meta[t].row_offset;
+  const int64_t i1 = offsets[bag + 1];
+  for (int64_t i = offsets[bag] + sub; i < i1; i += LIN_GROUP) {
+    const int64_t idx = clamp_index(indices[i], rows, status);
+    keys[i] = (uint32_t)(roff + idx);
+    vals[i] = (uint32_t)i;
+    bag_of_pos[i] = (uint32_t)bag;
+  }
+}
+
+// Table that owns a linear row id (largest t with row_offset[t] <= key).
+__device__ __forceinline__ int table_of_key(const TableMeta* __restrict__ meta, int T, int64_t key) {
+  int lo = 0, hi = T - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (meta[mid].row_offset <= key) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+struct RowTarget {
+  char* w;            // row storage (HBM table, cache slot, or host tier)
+  uint8_t* dirty;     // dirty byte to set, or nullptr
+};
+
+__device__ __forceinline__ RowTarget row_target(const TableMeta& m, int64_t key, uint32_t pos, int eb,
+                                                const int32_t* __restrict__ slot_of_lookup,
+                                                const CachePtrs& caches, char* dev_w, char* host_w) {
+  RowTarget r;
+  const int64_t row_bytes = (int64_t)m.dim * eb;
+  const int64_t idx = key - m.row_offset;
+  r.dirty = nullptr;
+  if (m.cache_id < 0) {
+    r.w = dev_w + m.weight_offset * eb + idx * row_bytes;
+  } else {
+    const int32_t s = slot_of_lookup[pos];
+    if (s >= 0) {
+      r.w = static_cast<char*>(caches.data[m.cache_id]) + (int64_t)s * row_bytes;
+      r.dirty = caches.dirty[m.cache_id] ? caches.dirty[m.cache_id] + s : nullptr;
+    } else {
+      r.w = host_w + m.weight_offset * eb + idx * row_bytes;
+    }
+  }
+  return r;
+}
+
+// Row-wise Adagrad on one row held across the warp: lane owns columns (q*32 + lane)*4 .. +3.
+// m += mean(g^2); W -= lr * g / (sqrt(m) + eps).
+template <bool FP16, int NV>
+__device__ __forceinline__ void adagrad_row(const float4 (&g)[NV], const uint4 (&wraw)[NV], float m_old,
+                                            int dim, float lr, float eps, char* wptr, float* mom_ptr,
+                                            uint8_t* dirty) {
+  const int lane = threadIdx.x & 31;
+  float sq = 0.f;
+#pragma unroll
+  for (int q = 0; q < NV; ++q) sq += g[q].x * g[q].x + g[q].y * g[q].y + g[q].z * g[q].z + g[q].w * g[q].w;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+  const float m_new = m_old + sq / (float)dim;
+  const float step = lr / (sqrtf(m_new) + eps);
+#pragma unroll
+  for (int q = 0; q < NV; ++q) {
+    const int d = (q * 32 + lane) * 4;
+    if (d < dim) {
+      if (FP16) {
+        const __half2* h = reinterpret_cast<const __half2*>(&wraw[q]);
+        float2 a = __half22float2(h[0]), b = __half22float2(h[1]);
+        a.x -= step * g[q].x; a.y -= step * g[q].y; b.x -= step * g[q].z; b.y -= step * g[q].w;
+        uint2 o;
+        __half2 ha = __floats2half2_rn(a.x, a.y), hb = __floats2half2_rn(b.x, b.y);
+        o.x = *reinterpret_cast<uint32_t*>(&ha);
+        o.y = *reinterpret_cast<uint32_t*>(&hb);
+        *reinterpret_cast<uint2*>(wptr + (int64_t)d * 2) = o;
+      } else {
+        float4 w = *reinterpret_cast<const float4*>(&wraw[q]);
+        w.x -= step * g[q].x; w.y -= step * g[q].y; w.z -= step * g[q].z; w.w -= step * g[q].w;
+        *reinterpret_cast<float4*>(wptr + (int64_t)d * 4) = w;
+      }
+    }
+  }
+  if (lane == 0) {
+    *mom_ptr = m_new;
+    if (dirty) *dirty = 1;
+  }
+}
+
+template <bool FP16, int NV>
+__device__ __forceinline__ void load_row(uint4 (&wraw)[NV], const char* wptr, int dim) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int q = 0; q < NV; ++q) {
+    const int d = (q * 32 + lane) * 4;
+    wraw[q] = make_uint4(0u, 0u, 0u, 0u);
+    if (d < dim) {
+      if (FP16) {
+        const uint2 v = *reinterpret_cast<const uint2*>(wptr + (int64_t)d * 2);
+        wraw[q].x = v.x; wraw[q].y = v.y;
+      } else {
+        wraw[q] = *reinterpret_cast<const uint4*>(wptr + (int64_t)d * 4);
+      }
+    }
+  }
+}
+
+template <bool FP16, int NV, int GROUP>
+__global__ void __launch_bounds__(BWD_WARPS * 32)
+reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
+              const uint32_t* __restrict__ keys, const uint32_t* __restrict__ pos,
+              const uint32_t* __restrict__ bag_of_pos, int64_t n,
+              const int64_t* __restrict__ offsets, int32_t pooling_mode,
+              const float* __restrict__ grad, int64_t grad_stride, float lr, float eps,
+              const int32_t* __restrict__ slot_of_lookup, CachePtrs caches, char* dev_w, char* host_w,
+              float* __restrict__ momentum, float* __restrict__ partial_head,
+              float* __restrict__ partial_tail) {
+  constexpr int EB = FP16 ? 2 : 4;
+  constexpr int PSTRIDE = NV * 128;
+  const int lane = threadIdx.x & 31;
+  const int64_t chunk = (int64_t)blockIdx.x * BWD_WARPS + (threadIdx.x >> 5);
+  const int64_t p0 = chunk * BWD_CHUNK;
+  if (p0 >= n) return;
+  const int64_t p1 = min(n, p0 + BWD_CHUNK);
+  const bool first_open = p0 > 0 && keys[p0 - 1] == keys[p0];
+  bool seen_end = false;
+  float4 acc[NV];
+#pragma unroll
+  for (int q = 0; q < NV; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+  bool last_is_end = true;
+
+  for (int64_t base = p0; base < p1; base += 32) {
+    const int cnt = (int)min((int64_t)32, p1 - base);
+    // per-lane description of lookup base + lane
+    const float* my_g = grad;
+    float my_scale = 1.f;
+    char* my_w = nullptr;
+    uint8_t* my_dirty = nullptr;
+    uint32_t my_key = 0;
+    int my_dim = 4;
+    bool my_end = false;
+    if (lane < cnt) {
+      const int64_t p = base + lane;
+      my_key = keys[p];
+      my_end = (p + 1 >= n) || keys[p + 1] != my_key;
+      const uint32_t ps = pos[p];
+      const uint32_t bag = bag_of_pos[ps];
+      const int t = (int)(bag / (uint32_t)B);
+      const int b = (int)(bag - (uint32_t)t * (uint32_t)B);
+      const TableMeta m = meta[t];
+      my_dim = m.dim;
+      my_g = grad + (int64_t)b * grad_stride + m.out_offset;
+      if (pooling_mode == MTS_POOL_MEAN) my_scale = 1.f / (float)(offsets[bag + 1] - offsets[bag]);
+      if (my_end) {
+        const RowTarget rt = row_target(m, (int64_t)my_key, ps, EB, slot_of_lookup, caches, dev_w, host_w);
+        my_w = rt.w;
+        my_dirty = rt.dirty;
+      }
+    }
+    const uint32_t ends = __ballot_sync(0xffffffffu, my_end);
+    if (base + 32 >= p1) last_is_end = (ends >> (cnt - 1)) & 1u;
+
+    for (int r = 0; r < cnt; r += GROUP) {
+      float4 g[GROUP][NV];
+      uint4 w[GROUP][NV];
+      float mo[GROUP];
+      float sc[GROUP];
+      int dm[GROUP];
+#pragma unroll
+      for (int u = 0; u < GROUP; ++u) {
+        const int j = (r + u) & 31;
+        const float* gp = reinterpret_cast<const float*>(
+            __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_g, j));
+        const char* wp = reinterpret_cast<const char*>(
+            __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_w, j));
+        const uint32_t k = __shfl_sync(0xffffffffu, my_key, j);
+        sc[u] = __shfl_sync(0xffffffffu, my_scale, j);
+        dm[u] = __shfl_sync(0xffffffffu, my_dim, j);
+        const bool valid = r + u < cnt;
+        const bool is_end = valid && ((ends >> j) & 1u);
+#pragma unroll
+        for (int q = 0; q < NV; ++q) {
+          const int d = (q * 32 + lane) * 4;
+          g[u][q] = (valid && d < dm[u]) ? __ldg(reinterpret_cast<const float4*>(gp + d))
+                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        mo[u] = 0.f;
+        if (is_end) {
+          load_row<FP16, NV>(w[u], wp, dm[u]);
+          mo[u] = momentum[k];
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < GROUP; ++u) {
+        const int j = (r + u) & 31;
+        const bool valid = r + u < cnt;
+        if (valid) {
+#pragma unroll
+          for (int q = 0; q < NV; ++q) {
+            acc[q].x = fmaf(sc[u], g[u][q].x, acc[q].x);
+            acc[q].y = fmaf(sc[u], g[u][q].y, acc[q].y);
+            acc[q].z = fmaf(sc[u], g[u][q].z, acc[q].z);
+            acc[q].w = fmaf(sc[u], g[u][q].w, acc[q].w);
+          }
+        }
+        const bool is_end = valid && ((ends >> j) & 1u);
+        if (is_end) {
+          if (first_open && !seen_end) {
+            // the row started in an earlier chunk: leave its piece for combine_partials
+#pragma unroll
+            for (int q = 0; q < NV; ++q)
+              *reinterpret_cast<float4*>(partial_head + chunk * PSTRIDE + (q * 32 + lane) * 4) = acc[q];
+          } else {
+            char* wp = reinterpret_cast<char*>(
+                __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_w, j));
+            uint8_t* dp = reinterpret_cast<uint8_t*>(
+                __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_dirty, j));
+            const uint32_t k = __shfl_sync(0xffffffffu, my_key, j);
+            adagrad_row<FP16, NV>(acc, w[u], mo[u], dm[u], lr, eps, wp, momentum + k, dp);
+          }
+          seen_end = true;
+#pragma unroll
+          for (int q = 0; q < NV; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+    }
+  }
+  if (!last_is_end) {
+    float* dst = (first_open && !seen_end) ? partial_head : partial_tail;
+#pragma unroll
+    for (int q = 0; q < NV; ++q)
+      *reinterpret_cast<float4*>(dst + chunk * PSTRIDE + (q * 32 + lane) * 4) = acc[q];
+  }
+}
+
+// One warp per chunk.  The chunk owns a row iff the row's lookups start in it and run past
+// its end; the owner adds tail[c] + head[c+1] + ... in chunk order and applies the update.
+template <bool FP16, int NV>
+__global__ void __launch_bounds__(BWD_WARPS * 32)
+combine_partials(const TableMeta* __restrict__ meta, int T, const uint32_t* __restrict__ keys,
+                 const uint32_t* __restrict__ pos, int64_t n, float lr, float eps,
+                 const int32_t* __restrict__ slot_of_lookup, CachePtrs caches, char* dev_w, char* host_w,
+                 float* __restrict__ momentum, const float* __restrict__ partial_head,
+                 const float* __restrict__ partial_tail) {
+  constexpr int EB = FP16 ? 2 : 4;
+  constexpr int PSTRIDE = NV * 128;
+  const int lane = threadIdx.x & 31;
+  const int64_t chunk = (int64_t)blockIdx.x * BWD_WARPS + (threadIdx.x >> 5);
+  const int64_t p0 = chunk * BWD_CHUNK;
+  const int64_t pe = p0 + BWD_CHUNK;           // first position of the next chunk
+  if (pe >= n) return;                         // no later chunk: nothing can continue
+  const uint32_t key = keys[pe - 1];
+  if (keys[pe] != key) return;                 // last row of the chunk ends here
+  if (p0 > 0 && keys[p0 - 1] == key) return;   // started earlier: an earlier chunk owns it
+  // number of later chunks the row reaches into
+  int64_t nc = 0;
+  for (;;) {
+    const int64_t start = pe + (nc + lane) * (int64_t)BWD_CHUNK;
+    const bool in = start < n && keys[start] == key;
+    const uint32_t bal = __ballot_sync(0xffffffffu, in);
+    const int lead = __ffs(~bal) - 1;          // leading run of chunks that continue the row
+    if (bal == 0xffffffffu) { nc += 32; continue; }
+    nc += lead;
+    break;
+  }
+  float4 acc[NV];
+#pragma unroll
+  for (int q = 0; q < NV; ++q)
+    acc[q] = *reinterpret_cast<const float4*>(partial_tail + chunk * PSTRIDE + (q * 32 + lane) * 4);
+  constexpr int U = 4;
+  for (int64_t c = 1; c <= nc; c += U) {
+    float4 v[U][NV];
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+      for (int q = 0; q < NV; ++q)
+        v[u][q] = (c + u <= nc)
+                      ? *reinterpret_cast<const float4*>(partial_head + (chunk + c + u) * PSTRIDE + (q * 32 + lane) * 4)
+                      : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (c + u <= nc) {
+#pragma unroll
+        for (int q = 0; q < NV; ++q) {
+          acc[q].x += v[u][q].x; acc[q].y += v[u][q].y; acc[q].z += v[u][q].z; acc[q].w += v[u][q].w;
+        }
+      }
+  }
+  const int t = table_of_key(meta, T, (int64_t)key);
+  const TableMeta m = meta[t];
+  const RowTarget rt = row_target(m, (int64_t)key, pos[pe - 1], EB, slot_of_lookup, caches, dev_w, host_w);
+  uint4 w[NV];
+  load_row<FP16, NV>(w, rt.w, m.dim);
+  adagrad_row<FP16, NV>(acc, w, momentum[key], m.dim, lr, eps, rt.w, momentum + key, rt.dirty);
+}
+
+__global__ void export_unique(const uint32_t* __restrict__ keys, const uint32_t* __restrict__ seg_start,
+                              const uint32_t* __restrict__ n_unique, int64_t* __restrict__ uniq_rows_out,
+                              int64_t* __restrict__ n_unique_out) {
+  const uint32_t U = *n_unique;
+  for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < U; u += (int64_t)gridDim.x * blockDim.x)
+    uniq_rows_out[u] = (int64_t)keys[seg_start[u]];
+  if (blockIdx.x == 0 && threadIdx.x == 0) *n_unique_out = (int64_t)U;
+}
+
+struct BwdLayout {
+  size_t keys_a, keys_b, vals_a, vals_b, bag_of_pos, hist, scan, seg_start, n_unique, head, tail, total;
+};
+
+static BwdLayout bwd_layout(const mts_tables* h, int64_t N) {
+  BwdLayout L;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t n = (size_t)(N > 0 ? N : 1);
+  L.keys_a = take(n * 4); L.keys_b = take(n * 4); L.vals_a = take(n * 4); L.vals_b = take(n * 4);
+  L.bag_of_pos = take(n * 4);
+  L.hist = take(sort_hist_words() * 4);
+  L.scan = take(scan_scratch_words() * 4);
+  L.seg_start = take((n + 1) * 4);
+  L.n_unique = take(256);
+  const int nv = (h->max_dim + 127) / 128;
+  const int nvp = nv <= 1 ? 1 : nv <= 2 ? 2 : nv <= 4 ? 4 : 8;
+  const size_t chunks = (size_t)ceil_div((int64_t)n, BWD_CHUNK);
+  L.head = take(chunks * nvp * 128 * 4);
+  L.tail = take(chunks * nvp * 128 * 4);
+  L.total = off;
+  return L;
+}
+
+template <bool FP16, int NV, int GROUP>
+static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys, const uint32_t* pos,
+                           const uint32_t* bag_of_pos, int64_t N, const int64_t* offsets, int32_t pooling_mode,
+                           const float* grad, int64_t grad_stride, float lr, float eps,
+                           const int32_t* slot_of_lookup, const CachePtrs& caches, float* head, float* tail,
+                           cudaStream_t s) {
+  const int64_t chunks = ceil_div(N, BWD_CHUNK);
+  const unsigned grid = (unsigned)ceil_div(chunks, BWD_WARPS);
+  reduce_chunks<FP16, NV, GROUP><<<grid, BWD_WARPS * 32, 0, s>>>(
+      h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad, grad_stride, lr, eps,
+      slot_of_lookup, caches, static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights),
+      h->momentum, head, tail);
+  combine_partials<FP16, NV><<<grid, BWD_WARPS * 32, 0, s>>>(
+      h->d_meta, h->T, keys, pos, N, lr, eps, slot_of_lookup, caches, static_cast<char*>(h->dev_weights),
+      static_cast<char*>(h->host_weights), h->momentum, head, tail);
+  return check_launch("reduce_chunks / combine_partials");
+}
+
+}  // namespace mts
+
+using namespace mts;
+
+extern "C" size_t mts_tbe_backward_workspace_bytes(const mts_tables* h, int32_t B, int64_t N) {
+  (void)B;
+  if (!h || N < 0) return 0;
+  return bwd_layout(h, N).total;
+}
+
+extern "C" int mts_tbe_backward_rowwise_adagrad(
+    const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets, int64_t N,
+    int32_t pooling_mode, const float* grad_out, int64_t grad_stride, float lr, float eps,
+    const int32_t* slot_of_lookup, void* const* host_cache_data, uint8_t* const* host_cache_dirty,
+    int32_t n_caches, void* workspace, size_t workspace_bytes, int64_t* uniq_rows_out,
+    int64_t* n_unique_out, void* stream) {
+  if (!h || !offsets || !grad_out || B < 1 || N < 0 || (N > 0 && !indices))
+    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward: null argument or bad size");
+  if (pooling_mode != MTS_POOL_SUM && pooling_mode != MTS_POOL_MEAN)
+    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward: pooling mode %d", pooling_mode);
+  if ((uniq_rows_out == nullptr) != (n_unique_out == nullptr))
+    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward: pass both uniq_rows_out and n_unique_out or neither");
+  if (grad_stride < h->total_dim || (grad_stride & 3) || ((uintptr_t)grad_out & 15))
+    return set_error(MTS_ERR_ALIGNMENT, "tbe_backward: grad_out must be 16-byte aligned, grad_stride >= %d and a multiple of 4",
+                     h->total_dim);
+  if (N >= (1ll << 32) - BWD_CHUNK || (int64_t)h->T * B >= (1ll << 32))
+    return set_error(MTS_ERR_UNSUPPORTED, "tbe_backward: lookup positions and bag ids must fit 32 bits");
+  const BwdLayout L = bwd_layout(h, N);
+  if (!workspace || ((uintptr_t)workspace & 255))
+    return set_error(MTS_ERR_ALIGNMENT, "tbe_backward: workspace must be non-null and 256-byte aligned");
+  if (workspace_bytes < L.total)
+    return set_error(MTS_ERR_WORKSPACE, "tbe_backward: workspace of %zu bytes, %zu needed", workspace_bytes, L.total);
+  CachePtrs caches;
+  int rc = fill_cache_ptrs(h, host_cache_data, host_cache_dirty, n_caches, slot_of_lookup, &caches);
+  if (rc != MTS_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  if (N == 0) {
+    if (n_unique_out) return check_cuda(cudaMemsetAsync(n_unique_out, 0, sizeof(int64_t), s), "memset(n_unique_out)");
+    return MTS_OK;
+  }
+  uint32_t* keys_a = reinterpret_cast<uint32_t*>(ws + L.keys_a);
+  uint32_t* keys_b = reinterpret_cast<uint32_t*>(ws + L.keys_b);
+  uint32_t* vals_a = reinterpret_cast<uint32_t*>(ws + L.vals_a);
+  uint32_t* vals_b = reinterpret_cast<uint32_t*>(ws + L.vals_b);
+  uint32_t* bag_of_pos = reinterpret_cast<uint32_t*>(ws + L.bag_of_pos);
+  const int64_t n_bags = (int64_t)h->T * B;
+  {
+    const int64_t threads = n_bags * LIN_GROUP;
+    linearize_lookups<<<(unsigned)ceil_div(threads, 256), 256, 0, s>>>(h->d_meta, n_bags, B, indices, offsets, keys_a,
+                                                                       vals_a, bag_of_pos, h->d_status);
+    rc = check_launch("linearize_lookups");
+    if (rc != MTS_OK) return rc;
+  }
+  int key_bits = 1;
+  while (key_bits < 32 && (1ll << key_bits) < h->total_rows) ++key_bits;
+  uint32_t *keys = nullptr, *pos = nullptr;
+  rc = radix_sort_pairs(keys_a, vals_a, keys_b, vals_b, N, nullptr, key_bits, reinterpret_cast<uint32_t*>(ws + L.hist), &keys,
+                        &pos, s);
+  if (rc != MTS_OK) return rc;
+  if (uniq_rows_out) {
+    uint32_t* seg_start = reinterpret_cast<uint32_t*>(ws + L.seg_start);
+    uint32_t* n_unique = reinterpret_cast<uint32_t*>(ws + L.n_unique);
+    rc = unique_segments(keys, N, nullptr, seg_start, nullptr, n_unique, reinterpret_cast<uint32_t*>(ws + L.scan), s);
+    if (rc != MTS_OK) return rc;
+    export_unique<<<h->sm_count * 4, 256, 0, s>>>(keys, seg_start, n_unique, uniq_rows_out, n_unique_out);
+    rc = check_launch("export_unique");
+    if (rc != MTS_OK) return rc;
+  }
+  float* head = reinterpret_cast<float*>(ws + L.head);
+  float* tail = reinterpret_cast<float*>(ws + L.tail);
+  const int nv = (h->max_dim + 127) / 128;
+  const bool fp16 = h->dtype == MTS_DTYPE_FP16;
+#define MTS_BWD(F, V, G) return launch_backward<F, V, G>(h, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad_out, grad_stride, lr, eps, slot_of_lookup, caches, head, tail, s)
+  if (fp16) {
+    if (nv <= 1) MTS_BWD(true, 1, 8);
+    if (nv <= 2) MTS_BWD(true, 2, 4);
+    if (nv <= 4) MTS_BWD(true, 4, 2);
+    MTS_BWD(true, 8, 1);
+  } else {
+    if (nv <= 1) MTS_BWD(false, 1, 8);
+    if (nv <= 2) MTS_BWD(false, 2, 4);
+    if (nv <= 4) MTS_BWD(false, 4, 2);
+    MTS_BWD(false, 8, 1);
+  }
+#undef MTS_BWD
+}

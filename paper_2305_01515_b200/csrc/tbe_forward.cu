@@ -1,0 +1,173 @@
+// Pooled multi-table embedding lookup (Section 2.1.1 of the paper: an embedding operator
+// selects rows of a table and pools them).  One warp per bag (table t, sample b); a row of
+// vec16 16-byte chunks is read by a group of G = pow2(vec16) lanes, so 32 / G rows are in
+// flight per load instruction and UNROLL of those instructions are issued back to back.
+// Accumulation in fp32 registers, one 16-byte store per lane group member at the end.
+#include "common.cuh"
+
+namespace mts {
+
+constexpr int FWD_WARPS = 8;
+constexpr int FWD_UNROLL = 4;
+
+template <bool FP16, int NV>
+__global__ void __launch_bounds__(FWD_WARPS * 32)
+tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B,
+                   const int64_t* __restrict__ indices, const int64_t* __restrict__ offsets,
+                   const int32_t* __restrict__ slot_of_lookup, CachePtrs caches,
+                   const char* __restrict__ dev_w, const char* __restrict__ host_w,
+                   int32_t pooling_mode, float* __restrict__ out, int64_t out_stride,
+                   int32_t* status) {
+  constexpr int EPC = FP16 ? 8 : 4;       // elements per 16-byte chunk
+  constexpr int EB = FP16 ? 2 : 4;
+  const int lane = threadIdx.x & 31;
+  const int64_t bag = (int64_t)blockIdx.x * FWD_WARPS + (threadIdx.x >> 5);
+  if (bag >= n_bags) return;
+  const int32_t t = (int32_t)(bag / B);
+  const int32_t b = (int32_t)(bag - (int64_t)t * B);
+  const TableMeta m = meta[t];
+  const int vec16 = m.vec16;
+  // lanes per row: smallest power of two >= vec16, at most 32
+  int logG = 0;
+  while ((1 << logG) < vec16 && logG < 5) ++logG;
+  const int G = 1 << logG;
+  const int R = 32 >> logG;               // rows per load instruction
+  const int sub = lane >> logG;
+  const int cl = lane & (G - 1);
+  const int64_t i0 = offsets[bag], i1 = offsets[bag + 1];
+  const int64_t row_bytes = (int64_t)m.dim * EB;
+  const char* table_base = (m.cache_id < 0 ? dev_w : host_w) + m.weight_offset * EB;
+  const char* cache_base = m.cache_id >= 0 ? static_cast<const char*>(caches.data[m.cache_id]) : nullptr;
+
+  float acc[NV][EPC];
+#pragma unroll
+  for (int v = 0; v < NV; ++v)
+#pragma unroll
+    for (int k = 0; k < EPC; ++k) acc[v][k] = 0.f;
+
+  for (int64_t base = i0; base < i1; base += 32) {
+    const int cnt = (int)min((int64_t)32, i1 - base);
+    const char* my_ptr = table_base;
+    if (lane < cnt) {
+      int64_t idx = clamp_index(indices[base + lane], m.rows, status);
+      my_ptr = table_base + idx * row_bytes;
+      if (cache_base != nullptr) {
+        int32_t s = slot_of_lookup[base + lane];
+        if (s >= 0) my_ptr = cache_base + (int64_t)s * row_bytes;
+      }
+    }
+    for (int r = 0; r < cnt; r += R * FWD_UNROLL) {
+      uint4 v[FWD_UNROLL][NV];
+#pragma unroll
+      for (int u = 0; u < FWD_UNROLL; ++u) {
+        const int j = r + u * R + sub;
+        const unsigned long long p =
+            __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_ptr, j & 31);
+        const bool valid = j < cnt;
+#pragma unroll
+        for (int q = 0; q < NV; ++q) {
+          const int c = cl + q * 32;
+          if (valid && c < vec16) v[u][q] = ld_nc_16(reinterpret_cast<const char*>(p) + (int64_t)c * 16);
+          else v[u][q] = make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < FWD_UNROLL; ++u)
+#pragma unroll
+        for (int q = 0; q < NV; ++q) {
+          if (FP16) add_half8(acc[q], v[u][q]);
+          else add_float4(acc[q], v[u][q]);
+        }
+    }
+  }
+  // fold the row groups of the warp together
+  for (int o = G; o < 32; o <<= 1) {
+#pragma unroll
+    for (int q = 0; q < NV; ++q)
+#pragma unroll
+      for (int k = 0; k < EPC; ++k) acc[q][k] += __shfl_xor_sync(0xffffffffu, acc[q][k], o);
+  }
+  if (sub == 0) {
+    float scale = 1.f;
+    if (pooling_mode == MTS_POOL_MEAN && i1 > i0) scale = 1.f / (float)(i1 - i0);
+    float* o = out + (int64_t)b * out_stride + m.out_offset;
+#pragma unroll
+    for (int q = 0; q < NV; ++q) {
+      const int c = cl + q * 32;
+      if (c < vec16) {
+        float4* dst = reinterpret_cast<float4*>(o + c * EPC);
+        dst[0] = make_float4(acc[q][0] * scale, acc[q][1] * scale, acc[q][2] * scale, acc[q][3] * scale);
+        if (FP16)
+          dst[1] = make_float4(acc[q][4] * scale, acc[q][5] * scale, acc[q][6] * scale, acc[q][7] * scale);
+      }
+    }
+  }
+}
+
+template <bool FP16, int NV>
+static int launch_forward(const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets,
+                          int32_t pooling_mode, const int32_t* slot_of_lookup, const CachePtrs& caches,
+                          float* out, int64_t out_stride, cudaStream_t stream) {
+  const int64_t n_bags = (int64_t)h->T * B;
+  const int64_t grid = ceil_div(n_bags, FWD_WARPS);
+  tbe_forward_kernel<FP16, NV><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
+      h->d_meta, n_bags, B, indices, offsets, slot_of_lookup, caches,
+      static_cast<const char*>(h->dev_weights), static_cast<const char*>(h->host_weights), pooling_mode,
+      out, out_stride, h->d_status);
+  return check_launch("tbe_forward_kernel");
+}
+
+int fill_cache_ptrs(const mts_tables* h, void* const* host_cache_data, uint8_t* const* host_cache_dirty,
+                    int32_t n_caches, const int32_t* slot_of_lookup, CachePtrs* out) {
+  for (int c = 0; c < MTS_MAX_CACHES; ++c) { out->data[c] = nullptr; out->dirty[c] = nullptr; }
+  if (!h->any_cached) return MTS_OK;
+  if (!slot_of_lookup || !host_cache_data || n_caches < h->n_cache_ids || n_caches > MTS_MAX_CACHES)
+    return set_error(MTS_ERR_INVALID_ARG,
+                     "cached tables need slot_of_lookup and %d cache data pointers (got %d)",
+                     h->n_cache_ids, n_caches);
+  for (int c = 0; c < n_caches; ++c) {
+    if (!host_cache_data[c] || ((uintptr_t)host_cache_data[c] & 15))
+      return set_error(MTS_ERR_ALIGNMENT, "cache %d: data pointer null or not 16-byte aligned", c);
+    out->data[c] = host_cache_data[c];
+    out->dirty[c] = host_cache_dirty ? host_cache_dirty[c] : nullptr;
+  }
+  return MTS_OK;
+}
+
+}  // namespace mts
+
+using namespace mts;
+
+extern "C" int mts_tbe_forward(const mts_tables* h, int32_t B, const int64_t* indices,
+                               const int64_t* offsets, int64_t N, int32_t pooling_mode,
+                               const int32_t* slot_of_lookup, void* const* host_cache_data,
+                               int32_t n_caches, float* out, int64_t out_stride, void* stream) {
+  if (!h || !offsets || !out || B < 1 || N < 0 || (N > 0 && !indices))
+    return set_error(MTS_ERR_INVALID_ARG, "tbe_forward: null argument or bad size");
+  if (pooling_mode != MTS_POOL_SUM && pooling_mode != MTS_POOL_MEAN)
+    return set_error(MTS_ERR_INVALID_ARG, "tbe_forward: pooling mode %d", pooling_mode);
+  if (out_stride < h->total_dim || (out_stride & 3) || ((uintptr_t)out & 15))
+    return set_error(MTS_ERR_ALIGNMENT, "tbe_forward: out must be 16-byte aligned, out_stride >= %d and a multiple of 4",
+                     h->total_dim);
+  if ((int64_t)h->T * B >= (1ll << 31) * FWD_WARPS)
+    return set_error(MTS_ERR_UNSUPPORTED, "tbe_forward: too many bags");
+  CachePtrs caches;
+  int rc = fill_cache_ptrs(h, host_cache_data, nullptr, n_caches, slot_of_lookup, &caches);
+  if (rc != MTS_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int max_vec = h->max_dim * h->elem_bytes / 16;
+  const int nv = max_vec <= 32 ? 1 : max_vec <= 64 ? 2 : max_vec <= 128 ? 4 : 8;
+  const bool fp16 = h->dtype == MTS_DTYPE_FP16;
+#define MTS_FWD(F, V) return launch_forward<F, V>(h, B, indices, offsets, pooling_mode, slot_of_lookup, caches, out, out_stride, s)
+  if (fp16) {
+    if (nv == 1) MTS_FWD(true, 1);
+    if (nv == 2) MTS_FWD(true, 2);
+    MTS_FWD(true, 4);
+  } else {
+    if (nv == 1) MTS_FWD(false, 1);
+    if (nv == 2) MTS_FWD(false, 2);
+    if (nv == 4) MTS_FWD(false, 4);
+    MTS_FWD(false, 8);
+  }
+#undef MTS_FWD
+}

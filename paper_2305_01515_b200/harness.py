@@ -1,0 +1,160 @@
+"""Torch plumbing around the C ABI: device buffers for one model, one call per step of the path.
+
+Nothing here computes anything on its own; every step is a call into libmtrains_b200.so.
+"""
+from __future__ import annotations
+
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as mb
+from . import workload as wl
+
+
+class DeviceModel:
+    """Weights, optimizer state and scratch of one ModelSpec on one GPU.
+
+    Uncached specs keep all tables in one flat HBM buffer.  Cached specs keep them in one flat
+    pinned host buffer (device-visible through unified addressing) behind one cache per
+    embedding dim."""
+
+    def __init__(self, spec: wl.ModelSpec, device="cuda:0", max_lookups: int = 0, weights: Optional[np.ndarray] = None,
+                 lock_depth: int = 0, policy: int = mb.POLICY_LRU, cache_sets: Optional[List[int]] = None):
+        self.spec = spec
+        self.device = torch.device(device)
+        self.tdtype = torch.float32 if spec.dtype == wl.FP32 else torch.float16
+        n_elem = int(spec.weight_offset[-1])
+        self.cached = spec.cached
+        if self.cached:
+            self.host_weights = torch.empty(n_elem, dtype=self.tdtype, pin_memory=True)
+            self.dev_weights = None
+            store = self.host_weights
+        else:
+            self.dev_weights = torch.empty(n_elem, dtype=self.tdtype, device=self.device)
+            self.host_weights = None
+            store = self.dev_weights
+        if weights is not None:
+            store.copy_(torch.from_numpy(weights))
+        else:
+            for t in range(spec.T):
+                a, b = int(spec.weight_offset[t]), int(spec.weight_offset[t + 1])
+                dst = store[a:b].view(-1, int(spec.dims[t]))
+                step = 1 << 22
+                for r0 in range(0, int(spec.rows[t]), step):
+                    r1 = min(r0 + step, int(spec.rows[t]))
+                    dst[r0:r1].copy_(wl.weights_torch(spec, t, self.device, r0, r1))
+        self.momentum = torch.zeros(int(spec.row_offset[-1]), dtype=torch.float32, device=self.device)
+        self.caches: List[mb.Cache] = []
+        self.groups = spec.dim_groups() if self.cached else []
+        cache_id = None
+        if self.cached:
+            cache_id = np.zeros(spec.T, np.int32)
+            for g, (dim, t0, t1) in enumerate(self.groups):
+                cache_id[t0:t1] = g
+                rows_g = int(spec.row_offset[t1] - spec.row_offset[t0])
+                sets = cache_sets[g] if cache_sets is not None else wl.cache_sets_for(rows_g, spec.cache_fraction)
+                self.caches.append(mb.cache_create(sets, rows_g, dim, spec.dtype, policy, lock_depth))
+        self.tables = mb.tables_create(spec.dtype, spec.rows, spec.dims, spec.weight_offset[:-1], cache_id,
+                                       self.dev_weights, self.host_weights, self.momentum)
+        self.cache_data = [c.data_ptr for c in self.caches] if self.cached else None
+        self.cache_dirty = [c.dirty_ptr for c in self.caches] if self.cached else None
+        self.max_lookups = 0
+        self.workspace = None
+        self.ws_bytes = 0
+        if max_lookups:
+            self.reserve(max_lookups)
+
+    # ------------------------------------------------------------------ scratch
+    def reserve(self, max_lookups: int) -> None:
+        if max_lookups <= self.max_lookups:
+            return
+        self.max_lookups = max_lookups
+        B = self.spec.batch
+        self.ws_bytes = mb.tbe_backward_workspace_bytes(self.tables, B, max_lookups)
+        self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=self.device)
+        # the cache calls may run on a side stream while backward runs: scratch of their own
+        self.cache_ws_bytes = max([mb.cache_workspace_bytes(c, max_lookups) for c in self.caches] + [256])
+        self.cache_ws = torch.empty(self.cache_ws_bytes, dtype=torch.uint8, device=self.device)
+        if self.cached:
+            n = max_lookups
+            dev = self.device
+            self.slot_of_lookup = torch.full((n,), -1, dtype=torch.int32, device=dev)
+            self.keys = torch.empty(n, dtype=torch.int64, device=dev)
+            self.lists = []
+            for c in self.caches:
+                esz = 4 if self.spec.dtype == wl.FP32 else 2
+                self.lists.append(dict(
+                    miss_keys=torch.empty(n, dtype=torch.int64, device=dev),
+                    miss_slots=torch.empty(n, dtype=torch.int32, device=dev),
+                    evict_keys=torch.empty(n, dtype=torch.int64, device=dev),
+                    evict_slots=torch.empty(n, dtype=torch.int32, device=dev),
+                    evict_dirty=torch.empty(n, dtype=torch.uint8, device=dev),
+                    counters=torch.zeros(mb.NUM_COUNTERS, dtype=torch.int64, device=dev),
+                    staging=torch.empty(n * c.dim * esz, dtype=torch.uint8, device=dev),
+                    capacity=n))
+
+    # ------------------------------------------------------------------ steps of the path
+    def forward(self, indices, offsets, N: int, out=None, pooling_mode: int = mb.POOL_SUM, stream=None):
+        if out is None:
+            out = torch.empty((self.spec.batch, self.spec.total_dim), dtype=torch.float32, device=self.device)
+        mb.tbe_forward(self.tables, self.spec.batch, indices, offsets, N, pooling_mode,
+                       self.slot_of_lookup if self.cached else None, self.cache_data, out, out.shape[1], stream)
+        return out
+
+    def backward(self, indices, offsets, N: int, grad_out, lr: Optional[float] = None, eps: Optional[float] = None,
+                 pooling_mode: int = mb.POOL_SUM, uniq_rows_out=None, n_unique_out=None, stream=None) -> None:
+        self.reserve(N)
+        mb.tbe_backward_rowwise_adagrad(
+            self.tables, self.spec.batch, indices, offsets, N, pooling_mode, grad_out, grad_out.shape[1],
+            self.spec.lr if lr is None else lr, self.spec.eps if eps is None else eps,
+            self.slot_of_lookup if self.cached else None, self.cache_data, self.cache_dirty, self.workspace,
+            self.ws_bytes, uniq_rows_out, n_unique_out, stream)
+
+    def group_range(self, g: int, offsets_host: np.ndarray):
+        """Lookup range [begin, begin + n) of cache group g in one batch (host-side CSR)."""
+        _, t0, t1 = self.groups[g]
+        B = self.spec.batch
+        begin = int(offsets_host[t0 * B])
+        return begin, int(offsets_host[t1 * B]) - begin
+
+    def host_rows_ptr(self, g: int) -> int:
+        _, t0, _ = self.groups[g]
+        esz = 4 if self.spec.dtype == wl.FP32 else 2
+        return self.host_weights.data_ptr() + int(self.spec.weight_offset[t0]) * esz
+
+    def cache_step(self, indices, offsets, offsets_host: np.ndarray, step: int, stream=None,
+                   do_prefetch: bool = True) -> None:
+        """lookup_insert + prefetch + writeback of every cache for one batch."""
+        B = self.spec.batch
+        for g, c in enumerate(self.caches):
+            _, t0, t1 = self.groups[g]
+            begin, n = self.group_range(g, offsets_host)
+            L = self.lists[g]
+            keys = self.keys[begin:begin + n] if n else self.keys[:0]
+            mb.linearize_keys(self.tables, t0, t1, B, indices, offsets, begin, n, keys if n else None, stream)
+            mb.cache_lookup_insert(c, keys if n else None, n, step,
+                                   self.slot_of_lookup[begin:begin + n] if n else None, L["miss_keys"],
+                                   L["miss_slots"], L["evict_keys"], L["evict_slots"], L["evict_dirty"],
+                                   L["capacity"], L["counters"], self.cache_ws, self.cache_ws_bytes, stream)
+            if do_prefetch:
+                hp = self.host_rows_ptr(g)
+                mb.cache_prefetch_misses(c, hp, L["miss_keys"], L["miss_slots"], L["evict_slots"], L["evict_dirty"],
+                                         L["capacity"], L["counters"], L["staging"], stream)
+                mb.cache_writeback_evicted(c, hp, L["evict_keys"], L["evict_dirty"], L["capacity"], L["counters"],
+                                           L["staging"], stream)
+
+    def flush(self, stream=None) -> None:
+        for g, c in enumerate(self.caches):
+            mb.cache_flush(c, self.host_rows_ptr(g), stream)
+
+    def weights_numpy(self) -> np.ndarray:
+        torch.cuda.synchronize(self.device)
+        src = self.host_weights if self.cached else self.dev_weights
+        return src.cpu().numpy().copy()
+
+    def close(self) -> None:
+        self.tables.destroy()
+        for c in self.caches:
+            c.destroy()

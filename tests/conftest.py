@@ -21,3 +21,17 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Build the CUDA library (nvcc cross-compiles without a GPU) and the C oracle once."""
+    import shutil
+
+    import oracle
+    from paper_2305_01515_b200 import build
+
+    oracle.build()
+    if shutil.which("nvcc") or os.path.exists("/usr/local/cuda/bin/nvcc"):
+        build.build_library()
+    yield

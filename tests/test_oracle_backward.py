@@ -1,4 +1,4 @@
-"""Pins for the oracle's backward + row-wise Adagrad (Section 2.1.1: optimizer with few states
+"""Pins for the oracle's backward + row-wise Adagrad (Section 2.1.2: optimizer with few states
 per row; Section 5.9: aggregate, run the optimizer, update the touched rows)."""
 import numpy as np
 import pytest

@@ -1,4 +1,4 @@
-"""Pins for the oracle's pooled lookup (Section 2.1: look up a subset of rows and pool them)."""
+"""Pins for the oracle's pooled lookup (Section 2.1.1: select rows of a table and pool them)."""
 import numpy as np
 import pytest
 import torch
