@@ -29,3 +29,41 @@ def assert_close_mag(got, ref, mag, rtol, what=""):
         raise AssertionError(
             f"{what}: {int(bad.sum())} of {bad.size} elements out of tolerance; worst at flat index "
             f"{k}: got {got.flat[k]!r} ref {ref.flat[k]!r} err {err.flat[k]:.3e} bound {bound.flat[k]:.3e}")
+
+
+# ---------------------------------------------------------------------------- GPU-side plumbing
+FWD_RTOL = {0: 1e-5, 1: 2e-3}      # storage dtype -> tolerance of |got - ref| <= rtol * (|ref| + mag)
+
+
+def to_dev(a, device="cuda:0"):
+    import torch
+
+    return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+
+
+def oracle_args(spec):
+    return (spec.dtype, spec.dims, spec.out_offset[:-1], spec.weight_offset[:-1])
+
+
+def custom_spec(rows, dims, B, dtype, poolings=None, alphas=None, bag_dist="poisson", seed=0, name="custom"):
+    poolings = poolings or [4.0] * len(rows)
+    alphas = alphas or [0.0] * len(rows)
+    tabs = [wl.TableSpec(rows=int(r), dim=int(d), pooling=float(p), alpha=float(a))
+            for r, d, p, a in zip(rows, dims, poolings, alphas)]
+    tabs = wl._finish_tables(tabs, np.random.default_rng([seed, 17]))
+    return wl.ModelSpec(name, tabs, dtype, B, bag_dist, seed=seed)
+
+
+def as_tensor(ptr, n, dtype):
+    """A torch view of device memory owned by the library (test plumbing only)."""
+    import torch
+
+    class _Holder:
+        pass
+
+    h = _Holder()
+    itemsize = torch.empty((), dtype=dtype).element_size()
+    h.__cuda_array_interface__ = {"shape": (n,), "typestr": {1: "|u1", 2: "<f2", 4: "<f4"}[itemsize],
+                                  "data": (ptr, False), "version": 2}
+    t = torch.as_tensor(h, device="cuda:0")
+    return t.view(dtype) if t.dtype != dtype else t

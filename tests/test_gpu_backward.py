@@ -1,0 +1,174 @@
+"""GPU backward + row-wise Adagrad vs the CPU oracle through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2305_01515_b200 import binding as mb
+from paper_2305_01515_b200 import workload as wl
+from paper_2305_01515_b200.harness import DeviceModel
+from helpers import FWD_RTOL, assert_close_mag, custom_spec, oracle_args, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _weights_f64(spec, W):
+    return W.astype(np.float64)
+
+
+def _run_steps(spec, n_steps=2, mode=0, batches=None, lr=None):
+    """n_steps train steps on GPU and oracle; compares weights, momentum and unique rows."""
+    lr = spec.lr if lr is None else lr
+    W0 = wl.all_weights_numpy(spec)
+    W_ref = W0.copy()
+    m_ref = np.zeros(int(spec.row_offset[-1]), np.float32)
+    model = DeviceModel(spec, weights=W0)
+    for k in range(n_steps):
+        idx, off = batches[k] if batches is not None else wl.gen_batch(spec, k)
+        grad = wl.gen_grad(spec, k)
+        N = len(idx)
+        W_before = W_ref.copy()
+        m_before = m_ref.copy()
+        uniq_ref = oracle.tbe_backward_rowwise_adagrad(*oracle_args(spec), spec.row_offset, W_ref, m_ref,
+                                                       spec.batch, idx, off, grad, lr, spec.eps, mode)
+        uniq = torch.full((max(N, 1),), -1, dtype=torch.int64, device="cuda:0")
+        nu = torch.full((1,), -1, dtype=torch.int64, device="cuda:0")
+        model.backward(to_dev(idx), to_dev(off), N, to_dev(grad), lr=lr, pooling_mode=mode,
+                       uniq_rows_out=uniq, n_unique_out=nu)
+        torch.cuda.synchronize()
+        assert model.tables.status() == 0
+        U = int(nu.item())
+        assert U == len(uniq_ref)
+        np.testing.assert_array_equal(uniq[:U].cpu().numpy(), uniq_ref)          # bit-exact unique-row set
+        W_gpu = model.weights_numpy()
+        m_gpu = model.momentum.cpu().numpy()
+        rtol = FWD_RTOL[spec.dtype]
+        # tolerance: |got - ref| <= rtol * (|ref| + |W_old| + |step|); momentum: relative to m_new
+        mag_w = np.abs(_weights_f64(spec, W_before)) + np.abs(_weights_f64(spec, W_ref) - _weights_f64(spec, W_before))
+        assert_close_mag(W_gpu, W_ref, mag_w, rtol, f"weights after step {k}")
+        assert_close_mag(m_gpu, m_ref, m_ref, 1e-5, f"momentum after step {k}")
+        # untouched rows keep their bits
+        touched = np.zeros(len(m_ref), bool); touched[uniq_ref] = True
+        assert (m_gpu[~touched] == m_before[~touched]).all()
+        for t in range(spec.T):
+            D = int(spec.dims[t])
+            a = W_gpu[spec.weight_offset[t]:spec.weight_offset[t + 1]].reshape(-1, D)
+            b = W_before[spec.weight_offset[t]:spec.weight_offset[t + 1]].reshape(-1, D)
+            tt = touched[spec.row_offset[t]:spec.row_offset[t + 1]]
+            assert (a[~tt].view(np.uint8) == b[~tt].view(np.uint8)).all()
+        # keep both sides on the same trajectory: continue from the oracle's state
+        store = model.dev_weights
+        store.copy_(torch.from_numpy(W_ref))
+        model.momentum.copy_(torch.from_numpy(m_ref))
+    model.close()
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_config1_full(mode):
+    _run_steps(wl.config1(), n_steps=2, mode=mode)
+
+
+@pytest.mark.parametrize("dtype", [wl.FP32, wl.FP16])
+def test_mixed_dims_skew_and_long_segments(dtype):
+    """Rows hit thousands of times (segments spanning many 128-lookup chunks), rows hit once,
+    every column-group width, chunk borders inside and between rows."""
+    dims = [8, 64, 128, 200, 256, 512] if dtype == wl.FP16 else [4, 64, 128, 100, 256, 512]
+    rows = [3, 5000, 20000, 7, 777, 129]
+    pool = [40, 30, 20, 90, 33, 2]
+    spec = custom_spec(rows, dims, 193, dtype, pool, [0, 1.3, 0.9, 0, 1.2, 0], seed=11)
+    _run_steps(spec, n_steps=2)
+
+
+def test_mean_pooling_fp16():
+    spec = custom_spec([100, 3000], [64, 128], 65, wl.FP16, [5, 25], [1.1, 1.05], seed=2)
+    _run_steps(spec, n_steps=2, mode=1)
+
+
+def test_single_row_table_one_giant_segment():
+    spec = custom_spec([1, 2], [128, 64], 300, wl.FP32, [30, 7], seed=4)
+    _run_steps(spec, n_steps=1)
+
+
+def test_lookup_counts_around_chunk_and_tile_borders():
+    """N = 1, 127, 128, 129, 4095, 4096, 4097 lookups (chunk = 128 lookups, sort tile = 4096)."""
+    for n in (1, 127, 128, 129, 4095, 4096, 4097):
+        spec = custom_spec([50], [64], 1, wl.FP32, [n], bag_dist="fixed", seed=n)
+        _run_steps(spec, n_steps=1)
+
+
+def test_empty_batch_is_a_no_op():
+    spec = custom_spec([10, 20], [64, 128], 16, wl.FP16, [3, 3])
+    off = np.zeros(2 * 16 + 1, np.int64)
+    _run_steps(spec, n_steps=1, batches=[(np.zeros(0, np.int64), off)])
+
+
+def test_config2_scaled_and_config3_scaled():
+    _run_steps(wl.config2(row_scale=0.02, batch=256), n_steps=2)
+    _run_steps(wl.config3(row_scale=0.01, batch=128, tables=16), n_steps=2)
+
+
+def test_two_runs_are_bit_identical():
+    spec = wl.config2(row_scale=0.01, batch=512, tables=6)
+    idx, off = wl.gen_batch(spec, 0)
+    grad = wl.gen_grad(spec, 0)
+    res = []
+    for _ in range(2):
+        m = DeviceModel(spec)
+        m.backward(to_dev(idx), to_dev(off), len(idx), to_dev(grad))
+        res.append((m.weights_numpy(), m.momentum.cpu().numpy()))
+        m.close()
+    assert (res[0][0].view(np.uint16) == res[1][0].view(np.uint16)).all()
+    assert (res[0][1].view(np.uint32) == res[1][1].view(np.uint32)).all()
+
+
+def test_workspace_too_small_and_misaligned_are_rejected():
+    spec = custom_spec([10], [64], 2, wl.FP32, [2], bag_dist="fixed")
+    m = DeviceModel(spec)
+    idx, off = wl.gen_batch(spec, 0)
+    grad = to_dev(wl.gen_grad(spec, 0))
+    ws = torch.empty(1024, dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(mb.MtsError) as e:
+        mb.tbe_backward_rowwise_adagrad(m.tables, 2, to_dev(idx), to_dev(off), len(idx), 0, grad, 64, 0.01, 1e-8,
+                                        None, None, None, ws, 1024)
+    assert e.value.code == mb.ERR_WORKSPACE
+    m.close()
+
+
+def test_config2_full_size_sampled_rows():
+    """Full configuration 2 as bench.py runs it: the oracle replays a sample of rows (all their
+    lookups in the batch) from the counter-based initial weights."""
+    spec = wl.config2()
+    idx, off = wl.gen_batch(spec, 0)
+    grad = wl.gen_grad(spec, 0)
+    m = DeviceModel(spec)
+    m.backward(to_dev(idx), to_dev(off), len(idx), to_dev(grad))
+    torch.cuda.synchronize()
+    B = spec.batch
+    rng = np.random.default_rng(1)
+    for t in (0, 13, 25):
+        seg = idx[off[t * B]:off[(t + 1) * B]]
+        counts = np.bincount(seg, minlength=int(spec.rows[t]))
+        hot = np.argsort(counts)[-3:]                                  # the hottest rows (long segments)
+        cold = rng.choice(np.nonzero(counts == 1)[0], 40, replace=False)
+        mid = rng.choice(np.nonzero(counts > 1)[0], 40, replace=False)
+        untouched = rng.choice(np.nonzero(counts == 0)[0], 10, replace=False)
+        sample = np.unique(np.concatenate([hot, cold, mid, untouched]))
+        keep = np.isin(seg, sample)
+        lens = np.diff(off[t * B:(t + 1) * B + 1])
+        bag_of = np.repeat(np.arange(B), lens)
+        sub_idx = np.searchsorted(sample, seg[keep])
+        sub_len = np.bincount(bag_of[keep], minlength=B)
+        sub_off = np.concatenate([[0], np.cumsum(sub_len)]).astype(np.int64)
+        Wsub = wl.weights_numpy(spec, t, sample).reshape(-1)
+        W_before = Wsub.copy()
+        msub = np.zeros(len(sample), np.float32)
+        g = np.ascontiguousarray(grad[:, spec.out_offset[t]:spec.out_offset[t + 1]])
+        oracle.tbe_backward_rowwise_adagrad(spec.dtype, [128], [0], [0], [0, len(sample)], Wsub, msub, B, sub_idx,
+                                            sub_off, g, spec.lr, spec.eps)
+        base = int(spec.weight_offset[t])
+        got_w = m.dev_weights[base:base + int(spec.rows[t]) * 128].view(-1, 128)[to_dev(sample)].cpu().numpy().reshape(-1)
+        got_m = m.momentum[int(spec.row_offset[t]) + to_dev(sample)].cpu().numpy()
+        mag = np.abs(W_before.astype(np.float64)) + np.abs(Wsub.astype(np.float64) - W_before.astype(np.float64))
+        assert_close_mag(got_w, Wsub, mag, FWD_RTOL[spec.dtype], f"table {t} weights")
+        assert_close_mag(got_m, msub, msub, 1e-5, f"table {t} momentum")
+    m.close()

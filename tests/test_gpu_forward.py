@@ -1,0 +1,95 @@
+"""GPU pooled lookup vs the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2305_01515_b200 import binding as mb
+from paper_2305_01515_b200 import workload as wl
+from paper_2305_01515_b200.harness import DeviceModel
+from helpers import FWD_RTOL, assert_close_mag, custom_spec, oracle_args, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_and_compare(spec, k=0, mode=0, batch=None):
+    W = wl.all_weights_numpy(spec)
+    idx, off = batch if batch is not None else wl.gen_batch(spec, k)
+    ref, mag = oracle.tbe_forward(*oracle_args(spec), W, spec.batch, idx, off, mode, want_mag=True)
+    m = DeviceModel(spec, weights=W)
+    out = torch.full((spec.batch, spec.total_dim), float("nan"), dtype=torch.float32, device="cuda:0")
+    m.forward(to_dev(idx), to_dev(off), len(idx), out=out, pooling_mode=mode)
+    torch.cuda.synchronize()
+    assert m.tables.status() == 0
+    assert_close_mag(out.cpu().numpy(), ref, mag, FWD_RTOL[spec.dtype], "forward")
+    m.close()
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_config1_full(mode):
+    _run_and_compare(wl.config1(), mode=mode)
+
+
+@pytest.mark.parametrize("dtype", [wl.FP32, wl.FP16])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_mixed_dims_and_ragged_bags(dtype, mode):
+    """Every lane-group width (1..32 chunks and rows wider than one warp pass), bags from empty
+    to several 32-lookup tiles with a ragged tail."""
+    dims = [8, 16, 24, 64, 128, 200, 256, 512] if dtype == wl.FP16 else [4, 8, 12, 64, 128, 100, 256, 512]
+    rows = [50, 1000, 37, 5000, 20000, 300, 777, 129]
+    pool = [0.7, 3, 40, 70, 20, 5, 33, 2]
+    spec = custom_spec(rows, dims, 97, dtype, pool, [0, 1.1, 0, 1.05, 0.9, 0, 1.3, 0], seed=3)
+    _run_and_compare(spec, mode=mode)
+
+
+def test_dim_1024_fp32_and_fp16():
+    for dtype in (wl.FP32, wl.FP16):
+        _run_and_compare(custom_spec([300, 40], [1024, 64], 33, dtype, [6, 2], seed=5))
+
+
+def test_empty_batch_and_all_empty_bags():
+    spec = custom_spec([10, 20], [64, 128], 16, wl.FP16, [3, 3])
+    off = np.zeros(2 * 16 + 1, np.int64)
+    _run_and_compare(spec, batch=(np.zeros(0, np.int64), off))
+
+
+def test_config2_scaled_and_config3_scaled():
+    _run_and_compare(wl.config2(row_scale=0.02, batch=256))
+    _run_and_compare(wl.config3(row_scale=0.01, batch=128, tables=16))
+
+
+def test_out_of_range_index_is_clamped_and_flagged():
+    spec = custom_spec([10], [64], 2, wl.FP32, [2], bag_dist="fixed")
+    W = wl.all_weights_numpy(spec)
+    idx = np.array([3, 10_000, -5, 9], np.int64)
+    off = np.array([0, 2, 4], np.int64)
+    m = DeviceModel(spec, weights=W)
+    out = m.forward(to_dev(idx), to_dev(off), 4)
+    torch.cuda.synchronize()
+    assert m.tables.status() == 1 and m.tables.status() == 0      # sticky, cleared by the read
+    ref = oracle.tbe_forward(*oracle_args(spec), W, 2, np.array([3, 9, 0, 9], np.int64), off)
+    np.testing.assert_allclose(out.cpu().numpy(), ref, rtol=1e-6)
+    m.close()
+
+
+def test_config2_full_size_sampled_bags():
+    """Full configuration 2 as bench.py runs it; the oracle recomputes a sample of bags from
+    the counter-based weights (compact sub-problem: only the rows those bags touch)."""
+    spec = wl.config2()
+    idx, off = wl.gen_batch(spec, 0)
+    m = DeviceModel(spec)
+    out = m.forward(to_dev(idx), to_dev(off), len(idx)).cpu().numpy()
+    assert m.tables.status() == 0
+    rng = np.random.default_rng(0)
+    B = spec.batch
+    for t in rng.choice(spec.T, 4, replace=False):
+        bs = np.sort(rng.choice(B, 64, replace=False))
+        rows_needed = np.unique(np.concatenate([idx[off[t * B + b]:off[t * B + b + 1]] for b in bs] + [np.zeros(1, np.int64)]))
+        Wsub = wl.weights_numpy(spec, int(t), rows_needed).reshape(-1)
+        sub_idx = np.concatenate([np.searchsorted(rows_needed, idx[off[t * B + b]:off[t * B + b + 1]]) for b in bs])
+        lens = np.array([off[t * B + b + 1] - off[t * B + b] for b in bs])
+        sub_off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+        ref, mag = oracle.tbe_forward(spec.dtype, [128], [0], [0], Wsub, len(bs), sub_idx, sub_off, 0, want_mag=True)
+        got = out[bs][:, spec.out_offset[t]:spec.out_offset[t + 1]]
+        assert_close_mag(got, ref, mag, FWD_RTOL[spec.dtype], f"table {t}")
+    m.close()
