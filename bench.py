@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the sparse-embedding train step (pooled lookup forward + backward with fused
+row-wise Adagrad) on seeded synthetic input.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl native|reference] [--workload cfg2]
+
+One step = one pass of the whole path over one batch.  Prints ONE JSON line on rank 0.
+`value` is whole-job throughput with inputs resident in HBM; `e2e` is the same metric through
+the C ABI with inputs in pinned host memory (host->device copies and the device->host read of
+the pooled output inside the timed region).  `--impl reference` times the CPU oracle on a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2305_01515_b200 import workload as wl  # noqa: E402
+
+METRIC = "train_step_embedding_lookups_per_sec"
+UNIT = "lookups/s"
+
+
+def make_spec(name: str, rank: int):
+    if name == "cfg1":
+        return wl.config1(seed=rank)
+    if name == "cfg2":
+        return wl.config2(seed=rank)
+    if name == "cfg3":
+        return wl.config3(seed=rank)
+    raise SystemExit(f"unknown workload {name}")
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.idx = gpu_index
+        self.t0 = self.t1 = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i",
+                 str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def mark(self, begin: bool):
+        if begin:
+            self.t0 = time.time()
+        else:
+            self.t1 = time.time()
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        for ts, line in self.rows:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            inside = self.t0 is not None and self.t0 - 0.05 <= ts <= (self.t1 or ts) + 0.15
+            try:
+                if inside:
+                    sm.append(float(f[1]))
+                mx = float(f[2])
+            except ValueError:
+                continue
+            if inside:
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+        if not sm:       # region shorter than one sample: use every sample taken
+            for ts, line in self.rows:
+                f = [x.strip() for x in line.split(",")]
+                try:
+                    sm.append(float(f[1]))
+                except (ValueError, IndexError):
+                    pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_sample(spec, idx, off, grad, tables):
+    """Compact sub-problem for the CPU oracle: the lookups of `tables` over the whole batch, the
+    table shrunk to the rows those lookups touch (initial weights from the counter-based
+    generator)."""
+    B = spec.batch
+    dims, woff, roff, ooff, widx, soff, sgrad, Ws = [], [0], [0], [0], [], [0], [], []
+    for t in tables:
+        seg = idx[off[t * B]:off[(t + 1) * B]]
+        rows = np.unique(seg)
+        Ws.append(wl.weights_numpy(spec, t, rows).reshape(-1))
+        widx.append(np.searchsorted(rows, seg))
+        lens = np.diff(off[t * B:(t + 1) * B + 1])
+        soff.extend((soff[-1] + np.cumsum(lens)).tolist())
+        D = int(spec.dims[t])
+        dims.append(D)
+        woff.append(woff[-1] + len(rows) * D)
+        roff.append(roff[-1] + len(rows))
+        ooff.append(ooff[-1] + D)
+        sgrad.append(grad[:, spec.out_offset[t]:spec.out_offset[t + 1]])
+    return dict(dtype=spec.dtype, dim=np.array(dims, np.int32), out_offset=np.array(ooff[:-1], np.int32),
+                weight_offset=np.array(woff[:-1], np.int64), row_offset=np.array(roff, np.int64),
+                W=np.concatenate(Ws), idx=np.concatenate(widx).astype(np.int64), off=np.array(soff, np.int64),
+                grad=np.ascontiguousarray(np.concatenate(sgrad, axis=1)), B=B, lr=spec.lr, eps=spec.eps)
+
+
+def time_oracle(sample, steps: int, warmup: int):
+    """Oracle forward + backward on the sample, `steps` times; returns (lookups/s, threads)."""
+    import oracle
+
+    threads = oracle.max_threads()
+    oracle.set_threads(threads)
+    n = len(sample["idx"])
+    W = sample["W"].copy()
+    m = np.zeros(int(sample["row_offset"][-1]), np.float32)
+    args = (sample["dtype"], sample["dim"], sample["out_offset"], sample["weight_offset"])
+
+    def step():
+        oracle.tbe_forward(*args, W, sample["B"], sample["idx"], sample["off"])
+        oracle.tbe_backward_rowwise_adagrad(*args, sample["row_offset"], W, m, sample["B"], sample["idx"],
+                                            sample["off"], sample["grad"], sample["lr"], sample["eps"])
+
+    for _ in range(warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = time.perf_counter() - t0
+    return n * steps / dt, threads, dt / steps
+
+
+def run_reference(args, rank: int, world: int):
+    if rank != 0:
+        return
+    spec = make_spec(args.workload, 0)
+    idx, off = wl.gen_batch(spec, 0)
+    grad = wl.gen_grad(spec, 0)
+    tables = list(range(min(8, spec.T)))
+    sample = oracle_sample(spec, idx, off, grad, tables)
+    value, threads, sec = time_oracle(sample, args.steps, args.warmup)
+    desc = (f"tables {tables} of batch 0 ({len(sample['idx'])} of {len(idx)} lookups), tables compacted to the rows "
+            f"touched; forward + backward per step")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": spec.name, "sample": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def run_native(args, rank: int, world: int, local_rank: int):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2305_01515_b200 import binding as mb
+    from paper_2305_01515_b200.harness import DeviceModel
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    spec = make_spec(args.workload, rank)
+    model = DeviceModel(spec, device=dev)
+    R = args.rotate
+    host, devb = [], []
+    for k in range(R):
+        idx, off = wl.gen_batch(spec, k)
+        grad = wl.gen_grad(spec, k)
+        h = (torch.from_numpy(idx).pin_memory(), torch.from_numpy(off).pin_memory(), torch.from_numpy(grad).pin_memory())
+        host.append(h)
+        devb.append(tuple(x.to(dev) for x in h))
+    n_max = max(len(h[0]) for h in host)
+    model.reserve(n_max)
+    B, TD = spec.batch, spec.total_dim
+    out = torch.empty((B, TD), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def step(k):
+        i, o, g = devb[k % R]
+        model.forward(i, o, i.numel(), out=out, stream=stream)
+        model.backward(i, o, i.numel(), g, stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    for k in range(args.warmup):
+        step(k)
+    torch.cuda.synchronize(dev)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    lookups = sum(host[k % R][0].numel() for k in range(args.steps))
+    launches0 = mb.launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps + 1)]
+    barrier()
+    torch.cuda.synchronize(dev)
+    sampler.mark(True)
+    ev[0].record(stream)
+    for k in range(args.steps):
+        i, o, g = devb[k % R]
+        model.forward(i, o, i.numel(), out=out, stream=stream)
+        ev[2 * k + 1].record(stream)
+        model.backward(i, o, i.numel(), g, stream=stream)
+        ev[2 * k + 2].record(stream)
+    torch.cuda.synchronize(dev)
+    sampler.mark(False)
+    barrier()
+    launches = mb.launch_count() - launches0
+    ms_total = ev[0].elapsed_time(ev[-1])
+    fwd_ms = sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(args.steps)) / args.steps
+    bwd_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(args.steps)) / args.steps
+    clocks = sampler.stop()
+
+    # per-kernel device times over the same K steps, bracketed by CUDA events on the launch stream
+    mb.trace_enable(True)
+    for k in range(args.steps):
+        step(k)
+    trace = mb.trace_report()
+    mb.trace_enable(False)
+
+    # end to end: inputs in pinned host memory, output read back to the host, every step
+    h_out = torch.empty((B, TD), dtype=torch.float32).pin_memory()
+    d_idx = torch.empty(n_max, dtype=torch.int64, device=dev)
+    d_off = torch.empty(spec.T * B + 1, dtype=torch.int64, device=dev)
+    d_grad = torch.empty((B, TD), dtype=torch.float32, device=dev)
+
+    def e2e_step(k):
+        hi, ho, hg = host[k % R]
+        n = hi.numel()
+        d_idx[:n].copy_(hi, non_blocking=True)
+        d_off.copy_(ho, non_blocking=True)
+        d_grad.copy_(hg, non_blocking=True)
+        model.forward(d_idx, d_off, n, out=out, stream=stream)
+        model.backward(d_idx, d_off, n, d_grad, stream=stream)
+        h_out.copy_(out, non_blocking=True)
+        return n * 8 + ho.numel() * 8 + hg.numel() * 4, h_out.numel() * 4
+
+    for k in range(min(2, args.warmup)):
+        e2e_step(k)
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    h2d = d2h = 0
+    for k in range(args.steps):
+        a, b = e2e_step(k)
+        h2d += a
+        d2h += b
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=dev)
+    tot = torch.tensor([float(lookups)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
+    ms_total, e2e_ms = float(t[0]), float(t[1])
+    all_lookups = float(tot[0])
+
+    if rank == 0:
+        peak, peak_src = measured_peaks()
+        eb = spec.elem_bytes
+        # per-launch algorithmic bytes (Eq. 3: one row of D*p bytes per lookup and pass)
+        n_avg = lookups / args.steps
+        per_lookup = sum(float(spec.tables[t].dim) * eb * spec.tables[t].pooling for t in range(spec.T)) / \
+            sum(spec.tables[t].pooling for t in range(spec.T))
+        alg = {
+            "tbe_forward_kernel": n_avg * (per_lookup + 8) + 8 * (spec.T * B + 1) + 4.0 * B * TD,
+            "reduce_chunks": n_avg * (per_lookup + 12),
+        }
+        top = max(trace.items(), key=lambda kv: kv[1][0]) if trace else (None, (0.0, 0))
+        kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps} for k, v in trace.items()}
+        roof = None
+        if top[0] in alg:
+            avg_ms = top[1][0] / top[1][1]
+            ach = alg[top[0]] / (avg_ms * 1e-3) / 1e9
+            roof = {"kernel": top[0], "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
+                    "frac": ach / peak, "traffic": None, "peak_source": peak_src,
+                    "algorithmic_bytes_per_launch": alg[top[0]], "avg_launch_ms": avg_ms,
+                    "timing": "CUDA events around every launch, separate pass of the same K steps"}
+        step_bytes = 2.0 * n_avg * per_lookup
+        ms_step = ms_total / args.steps
+        line = {
+            "metric": METRIC, "value": all_lookups / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": spec.name, "tables": spec.T, "rows_per_table": int(spec.rows[0]),
+                       "dim": int(spec.dims[0]), "storage": "fp16" if spec.dtype == wl.FP16 else "fp32",
+                       "batch": B, "lookups_per_step": n_avg, "parallelism": f"{world} replica(s), own batches",
+                       "l2": f"inputs larger than L2: {spec.weight_bytes / 1e9:.2f} GB of weights, {R} batches rotate"},
+            "samples_per_sec": world * B / (ms_step * 1e-3),
+            "forward_ms": fwd_ms, "backward_ms": bwd_ms,
+            "forward_lookups_per_sec": n_avg / (fwd_ms * 1e-3),
+            "step_eq3_gbs": step_bytes / (ms_step * 1e-3) / 1e9, "step_eq3_frac_of_peak": step_bytes / (ms_step * 1e-3) / 1e9 / peak,
+            "clocks": clocks, "gpu_launches": int(launches), "kernels": kernels, "roofline": roof,
+            "e2e": {"value": all_lookups / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d // args.steps,
+                    "d2h_bytes_per_step": d2h // args.steps, "ms_per_step": e2e_ms / args.steps},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            idx0, off0, g0 = (x.numpy() for x in host[0])
+            tables = list(range(min(8, spec.T)))
+            sample = oracle_sample(spec, idx0, off0, g0, tables)
+            v, threads, sec = time_oracle(sample, 3, 1)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                    "sample": f"tables {tables} of batch 0 ({len(sample['idx'])} lookups), tables "
+                                              f"compacted to the rows touched, 3 steps of forward + backward"}
+        print(json.dumps(line), flush=True)
+    model.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--rotate", type=int, default=4, help="distinct batches that take turns")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+    if world == 1 and args.gpus > 1:
+        raise SystemExit("launch with torch.distributed.run for --gpus > 1")
+    run_native(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -70,6 +70,21 @@ enum {
 const char* mts_last_error_string(void);
 
 /* ---------------------------------------------------------------------------------------
+ * Instrumentation (the paper has no counterpart; it reports external tools only).
+ * mts_launch_count: kernels this library has launched in this process so far.
+ * mts_trace_enable(1) makes every later launch record a CUDA event before and after itself on
+ * its stream (a few microseconds of host time per launch); mts_trace_enable(0) stops it; both
+ * drop unreported records.  mts_trace_report waits for the recorded launches and returns, per
+ * kernel id in [0, mts_trace_kernel_count()), the summed device time in milliseconds and the
+ * number of launches since the last enable/report (host arrays of n >= kernel count entries).
+ * Do not enable tracing while a stream is being captured into a CUDA graph. */
+int64_t mts_launch_count(void);
+int mts_trace_enable(int32_t enable);
+int32_t mts_trace_kernel_count(void);
+const char* mts_trace_kernel_name(int32_t kernel);
+int mts_trace_report(double* host_total_ms, int64_t* host_launches, int32_t n);
+
+/* ---------------------------------------------------------------------------------------
  * Tables.  The paper's model: T embedding tables, table t a 2-D tensor of H_t rows and D
  * columns of p bytes (Section 2.1.2, Eq. 1), the same structure in every memory that holds
  * it (Section 5.2), plus per-table metadata that says which memory serves it (Section 5.8).

@@ -133,9 +133,11 @@ def tbe_forward(dtype: int, dim, out_offset, weight_offset, weights: np.ndarray,
 def tbe_backward_rowwise_adagrad(dtype: int, dim, out_offset, weight_offset, row_offset,
                                  weights: np.ndarray, momentum: np.ndarray, B: int, indices, offsets,
                                  grad_out: np.ndarray, lr: float, eps: float, pooling_mode: int = 0,
-                                 slot_of_lookup=None, cache_data=None, cache_dirty=None) -> np.ndarray:
+                                 slot_of_lookup=None, cache_data=None, cache_dirty=None,
+                                 step_mag: Optional[np.ndarray] = None) -> np.ndarray:
     """In-place update of `weights` (or cache data) and `momentum`; returns the ascending
-    distinct linear row ids the batch touched."""
+    distinct linear row ids the batch touched.  step_mag (fp64, one entry per weight element)
+    receives the cancellation-free step size of every touched element."""
     dim = _i32(dim); out_offset = _i32(out_offset); weight_offset = _i64(weight_offset)
     row_offset = _i64(row_offset); indices = _i64(indices); offsets = _i64(offsets)
     assert grad_out.dtype == np.float32 and grad_out.flags["C_CONTIGUOUS"]
@@ -145,13 +147,15 @@ def tbe_backward_rowwise_adagrad(dtype: int, dim, out_offset, weight_offset, row
     if slot_of_lookup is not None:
         slot_of_lookup = _i32(slot_of_lookup)
     uniq = np.zeros(max(N, 1), dtype=np.int64)
+    if step_mag is not None:
+        assert step_mag.dtype == np.float64 and step_mag.size == weights.size
     cd, _k1 = _ptr_array(cache_data)
     cdirty, _k2 = _ptr_array(cache_dirty)
     U = lib().orc_tbe_backward_rowwise_adagrad(
         C.c_int32(T), C.c_int32(dtype), _p(dim), _p(out_offset), _p(weight_offset), _p(row_offset),
         _p(weights), _p(momentum), C.c_int32(B), _p(indices), _p(offsets), C.c_int32(pooling_mode),
         _p(grad_out), C.c_int64(grad_out.shape[1]), C.c_float(lr), C.c_float(eps),
-        _p(slot_of_lookup), cd, cdirty, _p(uniq))
+        _p(slot_of_lookup), cd, cdirty, _p(uniq), _p(step_mag))
     return uniq[:U].copy()
 
 

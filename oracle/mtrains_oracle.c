@@ -192,14 +192,18 @@ static int pair_cmp(const void* a, const void* b) {
  * momentum is indexed by the linear row id row_offset[t] + r.  Cached rows are updated in
  * their cache slot and the slot's dirty byte is set; overflowed rows in the flat buffer.
  * uniq_out (nullable, capacity N) receives the ascending distinct linear row ids;
- * returns their count U. */
+ * returns their count U.
+ * step_mag (nullable, double, indexed like the flat weight buffer: weight_offset[t] + r*D + d,
+ * wherever the row lives) receives lr * sum_i |s_i * grad_i[d]| / (sqrt(m_r) + eps): the size
+ * of the step had no two gradient terms cancelled, which bounds what a single-precision
+ * summation of the same terms may lose. */
 int64_t orc_tbe_backward_rowwise_adagrad(
         int32_t T, int32_t dtype, const int32_t* dim, const int32_t* out_offset,
         const int64_t* weight_offset, const int64_t* row_offset, void* weights, float* momentum,
         int32_t B, const int64_t* indices, const int64_t* offsets, int32_t pooling_mode,
         const float* grad_out, int64_t grad_stride, float lr, float eps,
         const int32_t* slot_of_lookup, void* const* cache_data, uint8_t* const* cache_dirty,
-        int64_t* uniq_out) {
+        int64_t* uniq_out, double* step_mag) {
     int64_t N = offsets[(int64_t)T * B];
     if (N == 0) return 0;
     orc_pair* pairs = (orc_pair*)malloc((size_t)N * sizeof(orc_pair));
@@ -230,10 +234,14 @@ int64_t orc_tbe_backward_rowwise_adagrad(
         int32_t t = tab_of[p0];
         int32_t D = dim[t];
         double* g = (double*)calloc((size_t)D, sizeof(double));
+        double* gabs = (double*)calloc((size_t)D, sizeof(double));
         for (int64_t j = seg[u]; j < seg[u + 1]; ++j) {
             int64_t i = pairs[j].pos;
             const float* go = grad_out + (int64_t)smp_of[i] * grad_stride + out_offset[t];
-            for (int32_t d = 0; d < D; ++d) g[d] += scale_of[i] * (double)go[d];
+            for (int32_t d = 0; d < D; ++d) {
+                g[d] += scale_of[i] * (double)go[d];
+                gabs[d] += fabs(scale_of[i] * (double)go[d]);
+            }
         }
         double sq = 0.0;
         for (int32_t d = 0; d < D; ++d) sq += g[d] * g[d];
@@ -249,7 +257,11 @@ int64_t orc_tbe_backward_rowwise_adagrad(
             store_elem(base, dtype, e0 + d, w - dlr * g[d] / denom);
         }
         if (slot >= 0 && cache_dirty && cache_dirty[t]) cache_dirty[t][slot] = 1;
+        if (step_mag)
+            for (int32_t d = 0; d < D; ++d)
+                step_mag[weight_offset[t] + indices[p0] * D + d] = dlr * gabs[d] / denom;
         if (uniq_out) uniq_out[u] = key;
+        free(gabs);
         free(g);
     }
     free(seg); free(scale_of); free(smp_of); free(tab_of); free(pairs);

@@ -25,7 +25,8 @@ COUNTER_NAMES = ("lookups", "unique", "hit_lookups", "miss_lookups", "unique_hit
                  "unique_misses", "inserted", "evicted", "evicted_dirty", "overflow")
 
 EXPORTS = (
-    "mts_last_error_string", "mts_tables_create", "mts_tables_destroy", "mts_tables_status",
+    "mts_last_error_string", "mts_launch_count", "mts_trace_enable", "mts_trace_kernel_count",
+    "mts_trace_kernel_name", "mts_trace_report", "mts_tables_create", "mts_tables_destroy", "mts_tables_status",
     "mts_tbe_forward", "mts_tbe_backward_workspace_bytes", "mts_tbe_backward_rowwise_adagrad",
     "mts_cache_create", "mts_cache_destroy", "mts_cache_data", "mts_cache_dirty",
     "mts_linearize_keys", "mts_cache_workspace_bytes", "mts_cache_lookup_insert",
@@ -63,6 +64,14 @@ def lib():
         vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
         L.mts_last_error_string.restype = C.c_char_p
         L.mts_last_error_string.argtypes = []
+        L.mts_launch_count.restype = i64
+        L.mts_launch_count.argtypes = []
+        L.mts_trace_enable.argtypes = [i32]
+        L.mts_trace_kernel_count.restype = i32
+        L.mts_trace_kernel_count.argtypes = []
+        L.mts_trace_kernel_name.restype = C.c_char_p
+        L.mts_trace_kernel_name.argtypes = [i32]
+        L.mts_trace_report.argtypes = [C.POINTER(C.c_double), C.POINTER(i64), i32]
         L.mts_tables_create.argtypes = [C.POINTER(TableDesc), C.POINTER(vp)]
         L.mts_tables_destroy.argtypes = [vp]
         L.mts_tables_status.argtypes = [vp, C.POINTER(i32), vp]
@@ -93,6 +102,23 @@ def lib():
 
 def last_error_string() -> str:
     return lib().mts_last_error_string().decode()
+
+
+def launch_count() -> int:
+    return int(lib().mts_launch_count())
+
+
+def trace_enable(enable: bool) -> None:
+    _check(lib().mts_trace_enable(1 if enable else 0))
+
+
+def trace_report() -> dict:
+    """{kernel name: (total device ms, launches)} since the last enable/report; synchronises."""
+    n = int(lib().mts_trace_kernel_count())
+    ms = (C.c_double * n)()
+    cnt = (C.c_int64 * n)()
+    _check(lib().mts_trace_report(ms, cnt, n))
+    return {lib().mts_trace_kernel_name(k).decode(): (float(ms[k]), int(cnt[k])) for k in range(n) if cnt[k]}
 
 
 def _check(rc: int) -> None:

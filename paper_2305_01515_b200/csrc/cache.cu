@@ -477,7 +477,10 @@ extern "C" int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_s
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->dirty, n), "cudaMalloc(dirty)");
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->data, (size_t)n * c->row_bytes), "cudaMalloc(cache rows)");
   if (rc == MTS_OK) {
-    cache_init_state<<<c->sm_count * 4, 256>>>(c->tags, c->ts, c->freq, c->dirty, n);
+    {
+      LaunchScope scope(K_OTHER, nullptr);
+      cache_init_state<<<c->sm_count * 4, 256>>>(c->tags, c->ts, c->freq, c->dirty, n);
+    }
     rc = check_launch("cache_init_state");
   }
   if (rc == MTS_OK) rc = check_cuda(cudaMemset(c->data, 0, (size_t)n * c->row_bytes), "cudaMemset(cache rows)");
@@ -524,8 +527,11 @@ extern "C" int mts_linearize_keys(const mts_tables* h, int32_t t_begin, int32_t 
     return set_error(MTS_ERR_INVALID_ARG, "linearize_keys: bad argument");
   if (n == 0) return MTS_OK;
   const int64_t n_bags = (int64_t)(t_end - t_begin) * B;
-  linearize_group_keys<<<(unsigned)ceil_div(n_bags * 8, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      h->d_meta, t_begin, n_bags, B, indices, offsets, lookup_begin, n, keys_out, h->d_status);
+  {
+    LaunchScope scope(K_LINEARIZE, static_cast<cudaStream_t>(stream));
+    linearize_group_keys<<<(unsigned)ceil_div(n_bags * 8, 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        h->d_meta, t_begin, n_bags, B, indices, offsets, lookup_begin, n, keys_out, h->d_status);
+  }
   return check_launch("linearize_group_keys");
 }
 
@@ -555,7 +561,10 @@ extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_
   char* ws = static_cast<char*>(workspace);
   auto U32 = [&](size_t off) { return reinterpret_cast<uint32_t*>(ws + off); };
   const int grid = c->sm_count * 8;
-  cache_prepare_keys<<<grid, 256, 0, s>>>(keys, N, U32(L.keys_a), U32(L.vals_a), counters);
+  {
+    LaunchScope scope(K_CACHE_PREPARE, s);
+    cache_prepare_keys<<<grid, 256, 0, s>>>(keys, N, U32(L.keys_a), U32(L.vals_a), counters);
+  }
   int rc = check_launch("cache_prepare_keys");
   if (rc != MTS_OK) return rc;
   uint32_t* n_unique = U32(L.n_unique);
@@ -571,8 +580,11 @@ extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_
   if (rc != MTS_OK) return rc;
   rc = unique_segments(sk, N, nullptr, U32(L.seg_start), U32(L.uniq_idx), n_unique, U32(L.scan), s);
   if (rc != MTS_OK) return rc;
-  cache_describe_unique<<<grid, 256, 0, s>>>(sk, U32(L.seg_start), n_unique, (uint64_t)c->S, U32(L.ukey),
-                                             U32(L.mult), U32(L.set_a), U32(L.sval_a));
+  {
+    LaunchScope scope(K_CACHE_DESCRIBE, s);
+    cache_describe_unique<<<grid, 256, 0, s>>>(sk, U32(L.seg_start), n_unique, (uint64_t)c->S, U32(L.ukey),
+                                               U32(L.mult), U32(L.set_a), U32(L.sval_a));
+  }
   rc = check_launch("cache_describe_unique");
   if (rc != MTS_OK) return rc;
   int set_bits = 0;
@@ -587,21 +599,36 @@ extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_
   uint8_t* member_flag = reinterpret_cast<uint8_t*>(ws + L.member_flag);
   uint8_t* member_old_dirty = reinterpret_cast<uint8_t*>(ws + L.member_old_dirty);
   int32_t* member_slot = reinterpret_cast<int32_t*>(ws + L.member_slot);
-  cache_probe_replace<<<grid, CACHE_THREADS, 0, s>>>(
-      ss, su, U32(L.sseg_start), n_sets, U32(L.ukey), U32(L.mult), c->tags, c->ts, c->freq, c->dirty, (int32_t)step,
-      c->lock_depth, c->policy, slot_of_uniq, member_flag, U32(L.member_old_key), member_old_dirty, member_slot,
-      reinterpret_cast<unsigned long long*>(counters));
+  {
+    LaunchScope scope(K_CACHE_PROBE_REPLACE, s);
+    cache_probe_replace<<<grid, CACHE_THREADS, 0, s>>>(
+        ss, su, U32(L.sseg_start), n_sets, U32(L.ukey), U32(L.mult), c->tags, c->ts, c->freq, c->dirty, (int32_t)step,
+        c->lock_depth, c->policy, slot_of_uniq, member_flag, U32(L.member_old_key), member_old_dirty, member_slot,
+        reinterpret_cast<unsigned long long*>(counters));
+  }
   rc = check_launch("cache_probe_replace");
   if (rc != MTS_OK) return rc;
   const int G = (int)std::min<int64_t>((int64_t)LIST_BLOCKS, ceil_div(N, CACHE_THREADS * 4));
-  cache_count_lists<<<G, CACHE_THREADS, 0, s>>>(member_flag, U32(L.member_old_key), n_unique, U32(L.cnt_miss),
-                                                U32(L.cnt_evict));
-  cache_scan_lists<<<1, CACHE_THREADS, 0, s>>>(U32(L.cnt_miss), U32(L.cnt_evict), G, n_unique, N, counters);
-  cache_write_lists<<<G, CACHE_THREADS, 0, s>>>(member_flag, U32(L.member_old_key), member_old_dirty, member_slot, su,
-                                                U32(L.ukey), n_unique, U32(L.cnt_miss), U32(L.cnt_evict),
-                                                list_capacity, miss_keys, miss_slots, evict_keys, evict_slots,
-                                                evict_dirty);
-  cache_scatter_slots<<<grid, 256, 0, s>>>(sp, U32(L.uniq_idx), slot_of_uniq, N, slot_of_lookup);
+  {
+    LaunchScope scope(K_CACHE_LISTS, s);
+    cache_count_lists<<<G, CACHE_THREADS, 0, s>>>(member_flag, U32(L.member_old_key), n_unique, U32(L.cnt_miss),
+                                                  U32(L.cnt_evict));
+  }
+  {
+    LaunchScope scope(K_CACHE_LISTS, s);
+    cache_scan_lists<<<1, CACHE_THREADS, 0, s>>>(U32(L.cnt_miss), U32(L.cnt_evict), G, n_unique, N, counters);
+  }
+  {
+    LaunchScope scope(K_CACHE_LISTS, s);
+    cache_write_lists<<<G, CACHE_THREADS, 0, s>>>(member_flag, U32(L.member_old_key), member_old_dirty, member_slot, su,
+                                                  U32(L.ukey), n_unique, U32(L.cnt_miss), U32(L.cnt_evict),
+                                                  list_capacity, miss_keys, miss_slots, evict_keys, evict_slots,
+                                                  evict_dirty);
+  }
+  {
+    LaunchScope scope(K_CACHE_SCATTER_SLOTS, s);
+    cache_scatter_slots<<<grid, 256, 0, s>>>(sp, U32(L.uniq_idx), slot_of_uniq, N, slot_of_lookup);
+  }
   return check_launch("cache lists / scatter");
 }
 
@@ -617,10 +644,16 @@ extern "C" int mts_cache_prefetch_misses(mts_cache* c, const void* host_rows_map
   if (list_capacity == 0) return MTS_OK;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int grid = c->sm_count * 8;
-  cache_save_victims<<<grid, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, evict_slots, evict_dirty, counters,
-                                                    list_capacity, static_cast<char*>(evict_staging));
-  cache_fetch_misses<<<grid, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, static_cast<const char*>(host_rows_mapped),
-                                                    miss_keys, miss_slots, counters, list_capacity);
+  {
+    LaunchScope scope(K_CACHE_SAVE_VICTIMS, s);
+    cache_save_victims<<<grid, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, evict_slots, evict_dirty, counters,
+                                                      list_capacity, static_cast<char*>(evict_staging));
+  }
+  {
+    LaunchScope scope(K_CACHE_FETCH_MISSES, s);
+    cache_fetch_misses<<<grid, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, static_cast<const char*>(host_rows_mapped),
+                                                      miss_keys, miss_slots, counters, list_capacity);
+  }
   return check_launch("cache_save_victims / cache_fetch_misses");
 }
 
@@ -633,9 +666,12 @@ extern "C" int mts_cache_writeback_evicted(mts_cache* c, void* host_rows_mapped,
   if (((uintptr_t)host_rows_mapped | (uintptr_t)evict_staging) & 15)
     return set_error(MTS_ERR_ALIGNMENT, "cache_writeback_evicted: buffers must be 16-byte aligned");
   if (list_capacity == 0) return MTS_OK;
-  cache_write_victims<<<c->sm_count * 8, CACHE_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
-      static_cast<char*>(host_rows_mapped), c->row_bytes, evict_keys, evict_dirty, counters, list_capacity,
-      static_cast<const char*>(evict_staging));
+  {
+    LaunchScope scope(K_CACHE_WRITE_VICTIMS, nullptr);
+    cache_write_victims<<<c->sm_count * 8, CACHE_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<char*>(host_rows_mapped), c->row_bytes, evict_keys, evict_dirty, counters, list_capacity,
+        static_cast<const char*>(evict_staging));
+  }
   return check_launch("cache_write_victims");
 }
 
@@ -644,16 +680,25 @@ extern "C" int mts_cache_flush(mts_cache* c, void* host_rows_mapped, void* strea
   if ((uintptr_t)host_rows_mapped & 15) return set_error(MTS_ERR_ALIGNMENT, "cache_flush: host buffer alignment");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int64_t n = c->S * MTS_CACHE_WAYS;
-  cache_flush_rows<<<c->sm_count * 8, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, c->tags, c->dirty, n,
-                                                             static_cast<char*>(host_rows_mapped));
-  cache_clear_dirty<<<c->sm_count * 4, 256, 0, s>>>(c->dirty, n);
+  {
+    LaunchScope scope(K_CACHE_FLUSH, nullptr);
+    cache_flush_rows<<<c->sm_count * 8, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, c->tags, c->dirty, n,
+                                                               static_cast<char*>(host_rows_mapped));
+  }
+  {
+    LaunchScope scope(K_CACHE_FLUSH, nullptr);
+    cache_clear_dirty<<<c->sm_count * 4, 256, 0, s>>>(c->dirty, n);
+  }
   return check_launch("cache_flush");
 }
 
 extern "C" int mts_cache_export_state(mts_cache* c, int64_t* tags, int64_t* timestamps, int64_t* counts,
                                       uint8_t* dirty, void* stream) {
   if (!c) return set_error(MTS_ERR_INVALID_ARG, "cache_export_state: null cache");
-  cache_export<<<c->sm_count * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
-      c->tags, c->ts, c->freq, c->dirty, c->S * MTS_CACHE_WAYS, tags, timestamps, counts, dirty);
+  {
+    LaunchScope scope(K_OTHER, nullptr);
+    cache_export<<<c->sm_count * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        c->tags, c->ts, c->freq, c->dirty, c->S * MTS_CACHE_WAYS, tags, timestamps, counts, dirty);
+  }
   return check_launch("cache_export");
 }

@@ -17,6 +17,22 @@ int set_error(int code, const char* fmt, ...);
 int check_cuda(cudaError_t e, const char* what);
 inline int check_launch(const char* what) { return check_cuda(cudaGetLastError(), what); }
 
+// ----------------------------------------------------------------------------- instrumentation
+// Every kernel launch of the library sits inside a LaunchScope: it counts the launch and, when
+// tracing is on, brackets it with CUDA events on the launching stream.
+enum KernelId {
+  K_FORWARD = 0, K_LINEARIZE, K_SORT_HISTOGRAM, K_SORT_SCAN, K_SORT_SCATTER, K_UNIQUE, K_REDUCE_CHUNKS,
+  K_COMBINE_PARTIALS, K_CACHE_PREPARE, K_CACHE_DESCRIBE, K_CACHE_PROBE_REPLACE, K_CACHE_LISTS, K_CACHE_SCATTER_SLOTS,
+  K_CACHE_SAVE_VICTIMS, K_CACHE_FETCH_MISSES, K_CACHE_WRITE_VICTIMS, K_CACHE_FLUSH, K_OTHER, K_COUNT
+};
+
+struct LaunchScope {
+  LaunchScope(int kernel_id, cudaStream_t stream);
+  ~LaunchScope();
+  int slot;
+  cudaStream_t stream;
+};
+
 // ----------------------------------------------------------------------------- tables
 // Per-table metadata as the kernels see it (device array of T entries).
 struct TableMeta {

@@ -212,9 +212,18 @@ int radix_sort_pairs(uint32_t* keys_a, uint32_t* vals_a, uint32_t* keys_b, uint3
     const int shift = 8 * p;
     const int bits = min(8, key_bits - shift);
     const uint32_t mask = (1u << bits) - 1u;
-    digit_histogram<<<G, SORT_THREADS, 0, stream>>>(ki, n_max, n_dev, shift, mask, hist, G);
-    scan_histogram<<<SORT_BINS, SORT_THREADS, 0, stream>>>(hist, totals, G);
-    scatter_by_digit<<<G, SORT_THREADS, 0, stream>>>(ki, vi, ko, vo, n_max, n_dev, shift, mask, hist, totals, G);
+    {
+      LaunchScope scope(K_SORT_HISTOGRAM, stream);
+      digit_histogram<<<G, SORT_THREADS, 0, stream>>>(ki, n_max, n_dev, shift, mask, hist, G);
+    }
+    {
+      LaunchScope scope(K_SORT_SCAN, stream);
+      scan_histogram<<<SORT_BINS, SORT_THREADS, 0, stream>>>(hist, totals, G);
+    }
+    {
+      LaunchScope scope(K_SORT_SCATTER, stream);
+      scatter_by_digit<<<G, SORT_THREADS, 0, stream>>>(ki, vi, ko, vo, n_max, n_dev, shift, mask, hist, totals, G);
+    }
     uint32_t* t;
     t = ki; ki = ko; ko = t;
     t = vi; vi = vo; vo = t;
@@ -307,9 +316,18 @@ int unique_segments(const uint32_t* sorted_keys, int64_t n_max, const uint32_t* 
   }
   const int64_t nchunks = ceil_div(n_max, UNIQ_THREADS * 8);
   const int G = (int)std::min<int64_t>(nchunks, SORT_MAX_BLOCKS);
-  count_heads<<<G, UNIQ_THREADS, 0, stream>>>(sorted_keys, n_max, n_dev, scratch);
-  scan_block_counts<<<1, UNIQ_THREADS, 0, stream>>>(scratch, G, n_unique, seg_start, n_max, n_dev);
-  write_heads<<<G, UNIQ_THREADS, 0, stream>>>(sorted_keys, n_max, n_dev, scratch, seg_start, uniq_idx);
+  {
+    LaunchScope scope(K_UNIQUE, stream);
+    count_heads<<<G, UNIQ_THREADS, 0, stream>>>(sorted_keys, n_max, n_dev, scratch);
+  }
+  {
+    LaunchScope scope(K_UNIQUE, stream);
+    scan_block_counts<<<1, UNIQ_THREADS, 0, stream>>>(scratch, G, n_unique, seg_start, n_max, n_dev);
+  }
+  {
+    LaunchScope scope(K_UNIQUE, stream);
+    write_heads<<<G, UNIQ_THREADS, 0, stream>>>(sorted_keys, n_max, n_dev, scratch, seg_start, uniq_idx);
+  }
   return check_launch("unique_segments");
 }
 

@@ -1,8 +1,10 @@
 // Table handle: validation of the caller's description and the per-table metadata block
 // that every lookup consults (which memory serves a table, Section 5.8 of the paper).
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -23,11 +25,81 @@ int check_cuda(cudaError_t e, const char* what) {
   return set_error(MTS_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
 
+// ------------------------------------------------------------------------------- instrumentation
+static const char* const kKernelNames[K_COUNT] = {
+    "tbe_forward_kernel", "linearize_lookups", "digit_histogram", "scan_histogram", "scatter_by_digit",
+    "unique_segments", "reduce_chunks", "combine_partials", "cache_prepare_keys", "cache_describe_unique",
+    "cache_probe_replace", "cache_lists", "cache_scatter_slots", "cache_save_victims", "cache_fetch_misses",
+    "cache_write_victims", "cache_flush", "other"};
+
+struct TraceRecord { int kernel; cudaEvent_t start, stop; };
+
+static std::mutex g_trace_mu;
+static std::atomic<long long> g_launches{0};
+static std::atomic<int> g_trace_on{0};
+static std::vector<TraceRecord> g_records;      // events are reused across enable/report cycles
+static size_t g_used = 0;
+
+LaunchScope::LaunchScope(int kernel_id, cudaStream_t s) : slot(-1), stream(s) {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (!g_trace_on.load(std::memory_order_relaxed)) return;
+  std::lock_guard<std::mutex> lk(g_trace_mu);
+  if (g_used == g_records.size()) {
+    TraceRecord r;
+    r.kernel = kernel_id;
+    if (cudaEventCreate(&r.start) != cudaSuccess) return;
+    if (cudaEventCreate(&r.stop) != cudaSuccess) { cudaEventDestroy(r.start); return; }
+    g_records.push_back(r);
+  }
+  g_records[g_used].kernel = kernel_id;
+  slot = (int)g_used++;
+  cudaEventRecord(g_records[slot].start, stream);
+}
+
+LaunchScope::~LaunchScope() {
+  if (slot < 0) return;
+  std::lock_guard<std::mutex> lk(g_trace_mu);
+  cudaEventRecord(g_records[slot].stop, stream);
+}
+
 }  // namespace mts
 
 using namespace mts;
 
 extern "C" const char* mts_last_error_string(void) { return g_err; }
+
+extern "C" int64_t mts_launch_count(void) { return (int64_t)g_launches.load(); }
+
+extern "C" int mts_trace_enable(int32_t enable) {
+  std::lock_guard<std::mutex> lk(g_trace_mu);
+  g_used = 0;
+  g_trace_on.store(enable ? 1 : 0);
+  return MTS_OK;
+}
+
+extern "C" int32_t mts_trace_kernel_count(void) { return K_COUNT; }
+
+extern "C" const char* mts_trace_kernel_name(int32_t kernel) {
+  return (kernel >= 0 && kernel < K_COUNT) ? kKernelNames[kernel] : "";
+}
+
+extern "C" int mts_trace_report(double* host_total_ms, int64_t* host_launches, int32_t n) {
+  if (!host_total_ms || !host_launches || n < K_COUNT)
+    return set_error(MTS_ERR_INVALID_ARG, "trace_report: need %d entries", (int)K_COUNT);
+  std::lock_guard<std::mutex> lk(g_trace_mu);
+  for (int k = 0; k < n; ++k) { host_total_ms[k] = 0.0; host_launches[k] = 0; }
+  for (size_t i = 0; i < g_used; ++i) {
+    int rc = check_cuda(cudaEventSynchronize(g_records[i].stop), "cudaEventSynchronize(trace)");
+    if (rc != MTS_OK) return rc;
+    float ms = 0.f;
+    rc = check_cuda(cudaEventElapsedTime(&ms, g_records[i].start, g_records[i].stop), "cudaEventElapsedTime(trace)");
+    if (rc != MTS_OK) return rc;
+    host_total_ms[g_records[i].kernel] += ms;
+    host_launches[g_records[i].kernel] += 1;
+  }
+  g_used = 0;
+  return MTS_OK;
+}
 
 extern "C" int mts_tables_create(const mts_table_desc* desc, mts_tables** out) {
   if (!desc || !out) return set_error(MTS_ERR_INVALID_ARG, "tables_create: null argument");

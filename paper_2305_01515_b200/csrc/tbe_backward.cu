@@ -366,13 +366,19 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
                            cudaStream_t s) {
   const int64_t chunks = ceil_div(N, BWD_CHUNK);
   const unsigned grid = (unsigned)ceil_div(chunks, BWD_WARPS);
-  reduce_chunks<FP16, NV, GROUP><<<grid, BWD_WARPS * 32, 0, s>>>(
-      h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad, grad_stride, lr, eps,
-      slot_of_lookup, caches, static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights),
-      h->momentum, head, tail);
-  combine_partials<FP16, NV><<<grid, BWD_WARPS * 32, 0, s>>>(
-      h->d_meta, h->T, keys, pos, N, lr, eps, slot_of_lookup, caches, static_cast<char*>(h->dev_weights),
-      static_cast<char*>(h->host_weights), h->momentum, head, tail);
+  {
+    LaunchScope scope(K_REDUCE_CHUNKS, s);
+    reduce_chunks<FP16, NV, GROUP><<<grid, BWD_WARPS * 32, 0, s>>>(
+        h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad, grad_stride, lr, eps,
+        slot_of_lookup, caches, static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights),
+        h->momentum, head, tail);
+  }
+  {
+    LaunchScope scope(K_COMBINE_PARTIALS, s);
+    combine_partials<FP16, NV><<<grid, BWD_WARPS * 32, 0, s>>>(
+        h->d_meta, h->T, keys, pos, N, lr, eps, slot_of_lookup, caches, static_cast<char*>(h->dev_weights),
+        static_cast<char*>(h->host_weights), h->momentum, head, tail);
+  }
   return check_launch("reduce_chunks / combine_partials");
 }
 
@@ -425,8 +431,11 @@ extern "C" int mts_tbe_backward_rowwise_adagrad(
   const int64_t n_bags = (int64_t)h->T * B;
   {
     const int64_t threads = n_bags * LIN_GROUP;
-    linearize_lookups<<<(unsigned)ceil_div(threads, 256), 256, 0, s>>>(h->d_meta, n_bags, B, indices, offsets, keys_a,
-                                                                       vals_a, bag_of_pos, h->d_status);
+    {
+      LaunchScope scope(K_LINEARIZE, s);
+      linearize_lookups<<<(unsigned)ceil_div(threads, 256), 256, 0, s>>>(h->d_meta, n_bags, B, indices, offsets, keys_a,
+                                                                         vals_a, bag_of_pos, h->d_status);
+    }
     rc = check_launch("linearize_lookups");
     if (rc != MTS_OK) return rc;
   }
@@ -441,7 +450,10 @@ extern "C" int mts_tbe_backward_rowwise_adagrad(
     uint32_t* n_unique = reinterpret_cast<uint32_t*>(ws + L.n_unique);
     rc = unique_segments(keys, N, nullptr, seg_start, nullptr, n_unique, reinterpret_cast<uint32_t*>(ws + L.scan), s);
     if (rc != MTS_OK) return rc;
-    export_unique<<<h->sm_count * 4, 256, 0, s>>>(keys, seg_start, n_unique, uniq_rows_out, n_unique_out);
+    {
+      LaunchScope scope(K_UNIQUE, nullptr);
+      export_unique<<<h->sm_count * 4, 256, 0, s>>>(keys, seg_start, n_unique, uniq_rows_out, n_unique_out);
+    }
     rc = check_launch("export_unique");
     if (rc != MTS_OK) return rc;
   }

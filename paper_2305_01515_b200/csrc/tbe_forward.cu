@@ -110,10 +110,13 @@ static int launch_forward(const mts_tables* h, int32_t B, const int64_t* indices
                           float* out, int64_t out_stride, cudaStream_t stream) {
   const int64_t n_bags = (int64_t)h->T * B;
   const int64_t grid = ceil_div(n_bags, FWD_WARPS);
-  tbe_forward_kernel<FP16, NV><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
-      h->d_meta, n_bags, B, indices, offsets, slot_of_lookup, caches,
-      static_cast<const char*>(h->dev_weights), static_cast<const char*>(h->host_weights), pooling_mode,
-      out, out_stride, h->d_status);
+  {
+    LaunchScope scope(K_FORWARD, stream);
+    tbe_forward_kernel<FP16, NV><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
+        h->d_meta, n_bags, B, indices, offsets, slot_of_lookup, caches,
+        static_cast<const char*>(h->dev_weights), static_cast<const char*>(h->host_weights), pooling_mode,
+        out, out_stride, h->d_status);
+  }
   return check_launch("tbe_forward_kernel");
 }
 

@@ -68,6 +68,7 @@ class DeviceModel:
 
     # ------------------------------------------------------------------ scratch
     def reserve(self, max_lookups: int) -> None:
+        max_lookups = max(int(max_lookups), 1)
         if max_lookups <= self.max_lookups:
             return
         self.max_lookups = max_lookups

@@ -29,8 +29,10 @@ def _run_steps(spec, n_steps=2, mode=0, batches=None, lr=None):
         N = len(idx)
         W_before = W_ref.copy()
         m_before = m_ref.copy()
+        step_mag = np.zeros(W_ref.size, np.float64)
         uniq_ref = oracle.tbe_backward_rowwise_adagrad(*oracle_args(spec), spec.row_offset, W_ref, m_ref,
-                                                       spec.batch, idx, off, grad, lr, spec.eps, mode)
+                                                       spec.batch, idx, off, grad, lr, spec.eps, mode,
+                                                       step_mag=step_mag)
         uniq = torch.full((max(N, 1),), -1, dtype=torch.int64, device="cuda:0")
         nu = torch.full((1,), -1, dtype=torch.int64, device="cuda:0")
         model.backward(to_dev(idx), to_dev(off), N, to_dev(grad), lr=lr, pooling_mode=mode,
@@ -43,8 +45,9 @@ def _run_steps(spec, n_steps=2, mode=0, batches=None, lr=None):
         W_gpu = model.weights_numpy()
         m_gpu = model.momentum.cpu().numpy()
         rtol = FWD_RTOL[spec.dtype]
-        # tolerance: |got - ref| <= rtol * (|ref| + |W_old| + |step|); momentum: relative to m_new
-        mag_w = np.abs(_weights_f64(spec, W_before)) + np.abs(_weights_f64(spec, W_ref) - _weights_f64(spec, W_before))
+        # tolerance: |got - ref| <= rtol * (|ref| + |W_old| + lr * sum|grad terms| / (sqrt(m) + eps));
+        # momentum: relative to m_new
+        mag_w = np.abs(_weights_f64(spec, W_before)) + step_mag
         assert_close_mag(W_gpu, W_ref, mag_w, rtol, f"weights after step {k}")
         assert_close_mag(m_gpu, m_ref, m_ref, 1e-5, f"momentum after step {k}")
         # untouched rows keep their bits
@@ -163,12 +166,13 @@ def test_config2_full_size_sampled_rows():
         W_before = Wsub.copy()
         msub = np.zeros(len(sample), np.float32)
         g = np.ascontiguousarray(grad[:, spec.out_offset[t]:spec.out_offset[t + 1]])
+        smag = np.zeros(Wsub.size, np.float64)
         oracle.tbe_backward_rowwise_adagrad(spec.dtype, [128], [0], [0], [0, len(sample)], Wsub, msub, B, sub_idx,
-                                            sub_off, g, spec.lr, spec.eps)
+                                            sub_off, g, spec.lr, spec.eps, step_mag=smag)
         base = int(spec.weight_offset[t])
         got_w = m.dev_weights[base:base + int(spec.rows[t]) * 128].view(-1, 128)[to_dev(sample)].cpu().numpy().reshape(-1)
         got_m = m.momentum[int(spec.row_offset[t]) + to_dev(sample)].cpu().numpy()
-        mag = np.abs(W_before.astype(np.float64)) + np.abs(Wsub.astype(np.float64) - W_before.astype(np.float64))
+        mag = np.abs(W_before.astype(np.float64)) + smag
         assert_close_mag(got_w, Wsub, mag, FWD_RTOL[spec.dtype], f"table {t} weights")
         assert_close_mag(got_m, msub, msub, 1e-5, f"table {t} momentum")
     m.close()
