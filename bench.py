@@ -32,11 +32,11 @@ METRIC = "train_step_embedding_lookups_per_sec"
 UNIT = "lookups/s"
 
 
-def make_spec(name: str, rank: int):
+def make_spec(name: str, rank: int, tables: int = 0):
     if name == "cfg1":
         return wl.config1(seed=rank)
     if name == "cfg2":
-        return wl.config2(seed=rank)
+        return wl.config2(seed=rank, tables=tables) if tables else wl.config2(seed=rank)
     if name == "cfg3":
         return wl.config3(seed=rank)
     raise SystemExit(f"unknown workload {name}")
@@ -200,7 +200,7 @@ def run_native(args, rank: int, world: int, local_rank: int):
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    spec = make_spec(args.workload, rank)
+    spec = make_spec(args.workload, rank, args.tables)
     model = DeviceModel(spec, device=dev)
     R = args.rotate
     host, devb = [], []
@@ -364,6 +364,8 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--rotate", type=int, default=4, help="distinct batches that take turns")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tables", type=int, default=0,
+                    help="cfg2 only: fewer tables (a small case for profiler captures; not a bench line)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
     rank = int(os.environ.get("RANK", "0"))

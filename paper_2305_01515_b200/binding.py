@@ -12,7 +12,7 @@ import os
 from typing import Optional, Sequence
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libmtrains_b200.so")
+LIB_PATH = os.environ.get("MTRAINS_B200_LIB", os.path.join(HERE, "libmtrains_b200.so"))
 
 OK = 0
 ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CAPACITY, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = (

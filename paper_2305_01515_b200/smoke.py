@@ -66,6 +66,8 @@ def run() -> None:
         assert got == res["counters"], (got, res["counters"])
         cm.forward(d_idx, d_off, len(idx))
         cm.backward(d_idx, d_off, len(idx), torch.from_numpy(wl.gen_grad(cspec, k)).to(dev))
+        used = res["slot_of_lookup"][res["slot_of_lookup"] >= 0]
+        oc.dirty[used] = 1                       # the backward pass dirties every slot it updates
     cm.flush()
     torch.cuda.synchronize()
     oc.close()
