@@ -17,7 +17,16 @@
 
 namespace mts {
 
-constexpr int BWD_CHUNK = 128;
+#ifndef MTS_BWD_CHUNK
+#define MTS_BWD_CHUNK 128
+#endif
+#ifndef MTS_BWD_GROUP1
+#define MTS_BWD_GROUP1 4        // lookups whose loads are issued together when a row fits one warp pass
+#endif
+#ifndef MTS_BWD_MINBLK
+#define MTS_BWD_MINBLK 8        // resident blocks per SM the register allocation is bounded for
+#endif
+constexpr int BWD_CHUNK = MTS_BWD_CHUNK;
 constexpr int BWD_WARPS = 4;
 constexpr int LIN_GROUP = 8;     // lanes per bag in linearize_lookups
 
@@ -90,8 +99,8 @@ __device__ __forceinline__ void adagrad_row(const float4 (&g)[NV], const uint4 (
   for (int q = 0; q < NV; ++q) sq += g[q].x * g[q].x + g[q].y * g[q].y + g[q].z * g[q].z + g[q].w * g[q].w;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-  const float m_new = m_old + sq / (float)dim;
-  const float step = lr / (sqrtf(m_new) + eps);
+  const float m_new = m_old + sq * __frcp_rn((float)dim);
+  const float step = __fdividef(lr, __fsqrt_rn(m_new) + eps);
 #pragma unroll
   for (int q = 0; q < NV; ++q) {
     const int d = (q * 32 + lane) * 4;
@@ -136,20 +145,29 @@ __device__ __forceinline__ void load_row(uint4 (&wraw)[NV], const char* wptr, in
   }
 }
 
-template <bool FP16, int NV, int GROUP>
-__global__ void __launch_bounds__(BWD_WARPS * 32)
+// reduce_chunks: one warp per CHUNK consecutive sorted lookups, 32 at a time.  Each lane first
+// resolves one lookup (gradient slice, row address, "last lookup of its row") and stages the
+// result in shared memory; then the warp walks the 32 lookups in order, GROUP at a time: the
+// loads of a whole group (gradient slices, and row + Adagrad state where a row ends) are issued
+// before the first one is used.
+template <bool FP16, int NV, int GROUP, bool MEAN>
+__global__ void __launch_bounds__(BWD_WARPS * 32, (NV == 1 ? MTS_BWD_MINBLK : 1))
 reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
               const uint32_t* __restrict__ keys, const uint32_t* __restrict__ pos,
               const uint32_t* __restrict__ bag_of_pos, int64_t n,
-              const int64_t* __restrict__ offsets, int32_t pooling_mode,
+              const int64_t* __restrict__ offsets,
               const float* __restrict__ grad, int64_t grad_stride, float lr, float eps,
               const int32_t* __restrict__ slot_of_lookup, CachePtrs caches, char* dev_w, char* host_w,
               float* __restrict__ momentum, float* __restrict__ partial_head,
               float* __restrict__ partial_tail) {
   constexpr int EB = FP16 ? 2 : 4;
   constexpr int PSTRIDE = NV * 128;
+  __shared__ uint4 s_desc[BWD_WARPS][32];      // {gradient float offset, key, row address lo, hi}
+  __shared__ uint2 s_aux[BWD_WARPS][32];       // {dim, mean-pooling scale bits}
+  __shared__ uint8_t* s_dirty[BWD_WARPS][32];
   const int lane = threadIdx.x & 31;
-  const int64_t chunk = (int64_t)blockIdx.x * BWD_WARPS + (threadIdx.x >> 5);
+  const int wib = threadIdx.x >> 5;
+  const int64_t chunk = (int64_t)blockIdx.x * BWD_WARPS + wib;
   const int64_t p0 = chunk * BWD_CHUNK;
   if (p0 >= n) return;
   const int64_t p1 = min(n, p0 + BWD_CHUNK);
@@ -162,99 +180,107 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
 
   for (int64_t base = p0; base < p1; base += 32) {
     const int cnt = (int)min((int64_t)32, p1 - base);
-    // per-lane description of lookup base + lane
-    const float* my_g = grad;
-    float my_scale = 1.f;
-    char* my_w = nullptr;
-    uint8_t* my_dirty = nullptr;
-    uint32_t my_key = 0;
-    int my_dim = 4;
     bool my_end = false;
+    bool my_dirty = false;
+    int my_dim = 0;
     if (lane < cnt) {
       const int64_t p = base + lane;
-      my_key = keys[p];
-      my_end = (p + 1 >= n) || keys[p + 1] != my_key;
+      const uint32_t key = keys[p];
+      my_end = (p + 1 >= n) || keys[p + 1] != key;
       const uint32_t ps = pos[p];
       const uint32_t bag = bag_of_pos[ps];
       const int t = (int)(bag / (uint32_t)B);
       const int b = (int)(bag - (uint32_t)t * (uint32_t)B);
       const TableMeta m = meta[t];
       my_dim = m.dim;
-      my_g = grad + (int64_t)b * grad_stride + m.out_offset;
-      if (pooling_mode == MTS_POOL_MEAN) my_scale = 1.f / (float)(offsets[bag + 1] - offsets[bag]);
+      uint4 d;
+      d.x = (uint32_t)((int64_t)b * grad_stride + m.out_offset);
+      d.y = key;
+      d.z = 0u; d.w = 0u;
+      uint8_t* dirty = nullptr;
       if (my_end) {
-        const RowTarget rt = row_target(m, (int64_t)my_key, ps, EB, slot_of_lookup, caches, dev_w, host_w);
-        my_w = rt.w;
-        my_dirty = rt.dirty;
+        const RowTarget rt = row_target(m, (int64_t)key, ps, EB, slot_of_lookup, caches, dev_w, host_w);
+        d.z = (uint32_t)(uintptr_t)rt.w;
+        d.w = (uint32_t)((uintptr_t)rt.w >> 32);
+        dirty = rt.dirty;
       }
+      uint2 a;
+      a.x = (uint32_t)m.dim;
+      a.y = MEAN ? __float_as_uint(1.f / (float)(offsets[bag + 1] - offsets[bag])) : 0u;
+      s_desc[wib][lane] = d;
+      s_aux[wib][lane] = a;
+      s_dirty[wib][lane] = dirty;
+      my_dirty = dirty != nullptr;
     }
+    __syncwarp();                                                  // staged descriptions visible to the warp
     const uint32_t ends = __ballot_sync(0xffffffffu, my_end);
+    const bool any_dirty = __any_sync(0xffffffffu, my_dirty);
+    // one dim for the whole batch unless it straddles tables of different width
+    const int dim0 = __shfl_sync(0xffffffffu, my_dim, 0);
+    const bool uniform = __all_sync(0xffffffffu, lane >= cnt || my_dim == dim0);
     if (base + 32 >= p1) last_is_end = (ends >> (cnt - 1)) & 1u;
 
     for (int r = 0; r < cnt; r += GROUP) {
       float4 g[GROUP][NV];
       uint4 w[GROUP][NV];
       float mo[GROUP];
-      float sc[GROUP];
-      int dm[GROUP];
 #pragma unroll
       for (int u = 0; u < GROUP; ++u) {
-        const int j = (r + u) & 31;
-        const float* gp = reinterpret_cast<const float*>(
-            __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_g, j));
-        const char* wp = reinterpret_cast<const char*>(
-            __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_w, j));
-        const uint32_t k = __shfl_sync(0xffffffffu, my_key, j);
-        sc[u] = __shfl_sync(0xffffffffu, my_scale, j);
-        dm[u] = __shfl_sync(0xffffffffu, my_dim, j);
-        const bool valid = r + u < cnt;
-        const bool is_end = valid && ((ends >> j) & 1u);
+        const int j = r + u;
+        if (j < cnt) {
+          const uint4 d = s_desc[wib][j];
+          const int dim = uniform ? dim0 : (int)s_aux[wib][j].x;
+          const float* gp = grad + d.x;
 #pragma unroll
-        for (int q = 0; q < NV; ++q) {
-          const int d = (q * 32 + lane) * 4;
-          g[u][q] = (valid && d < dm[u]) ? __ldg(reinterpret_cast<const float4*>(gp + d))
-                                         : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        mo[u] = 0.f;
-        if (is_end) {
-          load_row<FP16, NV>(w[u], wp, dm[u]);
-          mo[u] = momentum[k];
+          for (int q = 0; q < NV; ++q) {
+            const int c = (q * 32 + lane) * 4;
+            g[u][q] = c < dim ? __ldg(reinterpret_cast<const float4*>(gp + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+          if ((ends >> j) & 1u) {
+            const char* wp = reinterpret_cast<const char*>((uintptr_t)d.z | ((uintptr_t)d.w << 32));
+            load_row<FP16, NV>(w[u], wp, dim);
+            mo[u] = momentum[d.y];
+          }
         }
       }
 #pragma unroll
       for (int u = 0; u < GROUP; ++u) {
-        const int j = (r + u) & 31;
-        const bool valid = r + u < cnt;
-        if (valid) {
+        const int j = r + u;
+        if (j < cnt) {
+          if (MEAN) {
+            const float sc = __uint_as_float(s_aux[wib][j].y);
 #pragma unroll
-          for (int q = 0; q < NV; ++q) {
-            acc[q].x = fmaf(sc[u], g[u][q].x, acc[q].x);
-            acc[q].y = fmaf(sc[u], g[u][q].y, acc[q].y);
-            acc[q].z = fmaf(sc[u], g[u][q].z, acc[q].z);
-            acc[q].w = fmaf(sc[u], g[u][q].w, acc[q].w);
-          }
-        }
-        const bool is_end = valid && ((ends >> j) & 1u);
-        if (is_end) {
-          if (first_open && !seen_end) {
-            // the row started in an earlier chunk: leave its piece for combine_partials
-#pragma unroll
-            for (int q = 0; q < NV; ++q)
-              *reinterpret_cast<float4*>(partial_head + chunk * PSTRIDE + (q * 32 + lane) * 4) = acc[q];
+            for (int q = 0; q < NV; ++q) {
+              acc[q].x = fmaf(sc, g[u][q].x, acc[q].x); acc[q].y = fmaf(sc, g[u][q].y, acc[q].y);
+              acc[q].z = fmaf(sc, g[u][q].z, acc[q].z); acc[q].w = fmaf(sc, g[u][q].w, acc[q].w);
+            }
           } else {
-            char* wp = reinterpret_cast<char*>(
-                __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_w, j));
-            uint8_t* dp = reinterpret_cast<uint8_t*>(
-                __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_dirty, j));
-            const uint32_t k = __shfl_sync(0xffffffffu, my_key, j);
-            adagrad_row<FP16, NV>(acc, w[u], mo[u], dm[u], lr, eps, wp, momentum + k, dp);
-          }
-          seen_end = true;
 #pragma unroll
-          for (int q = 0; q < NV; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int q = 0; q < NV; ++q) {
+              acc[q].x += g[u][q].x; acc[q].y += g[u][q].y; acc[q].z += g[u][q].z; acc[q].w += g[u][q].w;
+            }
+          }
+          if ((ends >> j) & 1u) {
+            if (first_open && !seen_end) {
+              // the row started in an earlier chunk: leave its piece for combine_partials
+#pragma unroll
+              for (int q = 0; q < NV; ++q)
+                *reinterpret_cast<float4*>(partial_head + chunk * PSTRIDE + (q * 32 + lane) * 4) = acc[q];
+            } else {
+              const uint4 d = s_desc[wib][j];
+              const int dim = uniform ? dim0 : (int)s_aux[wib][j].x;
+              char* wp = reinterpret_cast<char*>((uintptr_t)d.z | ((uintptr_t)d.w << 32));
+              adagrad_row<FP16, NV>(acc, w[u], mo[u], dim, lr, eps, wp, momentum + d.y,
+                                    any_dirty ? s_dirty[wib][j] : nullptr);
+            }
+            seen_end = true;
+#pragma unroll
+            for (int q = 0; q < NV; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
         }
       }
     }
+    __syncwarp();      // the next batch overwrites the staged descriptions
   }
   if (!last_is_end) {
     float* dst = (first_open && !seen_end) ? partial_head : partial_tail;
@@ -368,10 +394,14 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
   const unsigned grid = (unsigned)ceil_div(chunks, BWD_WARPS);
   {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
-    reduce_chunks<FP16, NV, GROUP><<<grid, BWD_WARPS * 32, 0, s>>>(
-        h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad, grad_stride, lr, eps,
-        slot_of_lookup, caches, static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights),
-        h->momentum, head, tail);
+    if (pooling_mode == MTS_POOL_MEAN)
+      reduce_chunks<FP16, NV, GROUP, true><<<grid, BWD_WARPS * 32, 0, s>>>(
+          h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
+          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail);
+    else
+      reduce_chunks<FP16, NV, GROUP, false><<<grid, BWD_WARPS * 32, 0, s>>>(
+          h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
+          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail);
   }
   {
     LaunchScope scope(K_COMBINE_PARTIALS, s);
@@ -407,8 +437,9 @@ extern "C" int mts_tbe_backward_rowwise_adagrad(
   if (grad_stride < h->total_dim || (grad_stride & 3) || ((uintptr_t)grad_out & 15))
     return set_error(MTS_ERR_ALIGNMENT, "tbe_backward: grad_out must be 16-byte aligned, grad_stride >= %d and a multiple of 4",
                      h->total_dim);
-  if (N >= (1ll << 32) - BWD_CHUNK || (int64_t)h->T * B >= (1ll << 32))
-    return set_error(MTS_ERR_UNSUPPORTED, "tbe_backward: lookup positions and bag ids must fit 32 bits");
+  if (N >= (1ll << 32) - BWD_CHUNK || (int64_t)h->T * B >= (1ll << 32) || (int64_t)B * grad_stride >= (1ll << 32))
+    return set_error(MTS_ERR_UNSUPPORTED,
+                     "tbe_backward: lookup positions, bag ids and grad_out element offsets must fit 32 bits");
   const BwdLayout L = bwd_layout(h, N);
   if (!workspace || ((uintptr_t)workspace & 255))
     return set_error(MTS_ERR_ALIGNMENT, "tbe_backward: workspace must be non-null and 256-byte aligned");
@@ -463,12 +494,12 @@ extern "C" int mts_tbe_backward_rowwise_adagrad(
   const bool fp16 = h->dtype == MTS_DTYPE_FP16;
 #define MTS_BWD(F, V, G) return launch_backward<F, V, G>(h, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad_out, grad_stride, lr, eps, slot_of_lookup, caches, head, tail, s)
   if (fp16) {
-    if (nv <= 1) MTS_BWD(true, 1, 8);
+    if (nv <= 1) MTS_BWD(true, 1, MTS_BWD_GROUP1);
     if (nv <= 2) MTS_BWD(true, 2, 4);
     if (nv <= 4) MTS_BWD(true, 4, 2);
     MTS_BWD(true, 8, 1);
   } else {
-    if (nv <= 1) MTS_BWD(false, 1, 8);
+    if (nv <= 1) MTS_BWD(false, 1, MTS_BWD_GROUP1);
     if (nv <= 2) MTS_BWD(false, 2, 4);
     if (nv <= 4) MTS_BWD(false, 4, 2);
     MTS_BWD(false, 8, 1);
