@@ -164,6 +164,33 @@ int mts_tbe_backward_rowwise_adagrad(const mts_tables* tables, int32_t B, const 
                                      void* workspace, size_t workspace_bytes,
                                      int64_t* uniq_rows_out, int64_t* n_unique_out, void* stream);
 
+/* Backward without a workspace argument and without any allocation (the paper has no
+ * counterpart; this exists for callers of this library that cannot allocate device memory).
+ * Such callers are, for example, a training or serving loop embedded in a framework that
+ * has reserved the whole device for its own pool, so that cudaMalloc fails or is forbidden by
+ * policy; a step function that must not trigger the device-wide synchronisation an allocation
+ * can imply; or plain C code that has no allocator to size the workspace with.
+ * Same computation, arguments and errors as mts_tbe_backward_rowwise_adagrad, except that the
+ * scratch memory is a fixed array of MTS_STATIC_SCRATCH_BYTES bytes inside the library image
+ * (every GPU that loads the library holds that much until the process exits).
+ *   - Limit: the batch must satisfy mts_tbe_backward_workspace_bytes(tables, B, N) <=
+ *     MTS_STATIC_SCRATCH_BYTES (about 83,000 lookups at dim <= 1024, about 229,000 at dim <= 128);
+ *     larger batches are rejected with MTS_ERR_CAPACITY before anything is launched.
+ *   - The first call on each device looks up the array's device address (no allocation).  Make
+ *     that first call outside of any stream capture.
+ *   - The call itself calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - All calls share the one array and it keeps the previous call's contents; the kernels
+ *     write every scratch word before reading it, so nothing needs clearing, but two calls whose
+ *     kernels overlap on the GPU (different streams, or different host threads) race on it.
+ *     Issue these calls on one stream, or order them with events. */
+#define MTS_STATIC_SCRATCH_BYTES (8u << 20)
+int mts_tbe_backward_rowwise_adagrad_static(const mts_tables* tables, int32_t B, const int64_t* indices,
+                                            const int64_t* offsets, int64_t N, int32_t pooling_mode,
+                                            const float* grad_out, int64_t grad_stride, float lr, float eps,
+                                            const int32_t* slot_of_lookup, void* const* host_cache_data,
+                                            uint8_t* const* host_cache_dirty, int32_t n_caches,
+                                            int64_t* uniq_rows_out, int64_t* n_unique_out, void* stream);
+
 /* ---------------------------------------------------------------------------------------
  * Row cache (Section 5.3.1 cache class: row-granular cache memory, tags, per-entry timestamp
  * states; Section 5.5 GPU-managed cache kernels).  One level: HBM in front of pinned host

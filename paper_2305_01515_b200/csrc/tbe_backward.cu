@@ -13,6 +13,8 @@
 //                          chunk order and applies the update
 // The summation tree depends only on the sorted order and CHUNK, so two runs give the same
 // bits.  No thread ever writes a word another thread of the same launch writes.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace mts {
@@ -505,4 +507,51 @@ extern "C" int mts_tbe_backward_rowwise_adagrad(
     MTS_BWD(false, 8, 1);
   }
 #undef MTS_BWD
+}
+
+// ---------------------------------------------------------------------------------------------
+// Backward without a caller-provided workspace: the scratch lives in a fixed array that is part
+// of the library image.
+static __device__ __align__(256) unsigned char g_static_scratch[MTS_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices] = {};      // device address of g_static_scratch, per device
+}  // namespace
+
+extern "C" int mts_tbe_backward_rowwise_adagrad_static(
+    const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets, int64_t N,
+    int32_t pooling_mode, const float* grad_out, int64_t grad_stride, float lr, float eps,
+    const int32_t* slot_of_lookup, void* const* host_cache_data, uint8_t* const* host_cache_dirty,
+    int32_t n_caches, int64_t* uniq_rows_out, int64_t* n_unique_out, void* stream) {
+  if (!h || N < 0) return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_static: null tables or negative N");
+  const size_t need = mts_tbe_backward_workspace_bytes(h, B, N);
+  if (need > (size_t)MTS_STATIC_SCRATCH_BYTES)
+    return set_error(MTS_ERR_CAPACITY,
+                     "tbe_backward_static: %lld lookups need %zu bytes of scratch, the built-in array holds %zu; "
+                     "use mts_tbe_backward_rowwise_adagrad with a workspace of your own",
+                     (long long)N, need, (size_t)MTS_STATIC_SCRATCH_BYTES);
+  int dev = 0;
+  int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
+  if (rc != MTS_OK) return rc;
+  if (dev < 0 || dev >= kMaxDevices) return set_error(MTS_ERR_UNSUPPORTED, "tbe_backward_static: device %d", dev);
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    if (g_static_ptr[dev] == nullptr) {
+      // In host code the array's name is only a handle; its device address has to be asked for,
+      // once per device, with that device current.
+      void* p = nullptr;
+      rc = check_cuda(cudaGetSymbolAddress(&p, g_static_scratch), "cudaGetSymbolAddress(static scratch)");
+      if (rc != MTS_OK) return rc;
+      g_static_ptr[dev] = p;
+    }
+    scratch = g_static_ptr[dev];
+  }
+  // Every scratch word the kernels read is written earlier in the same call, so nothing has to
+  // be cleared even though the array still holds the previous call's contents.
+  return mts_tbe_backward_rowwise_adagrad(h, B, indices, offsets, N, pooling_mode, grad_out, grad_stride, lr, eps,
+                                          slot_of_lookup, host_cache_data, host_cache_dirty, n_caches, scratch,
+                                          (size_t)MTS_STATIC_SCRATCH_BYTES, uniq_rows_out, n_unique_out, stream);
 }
