@@ -189,6 +189,19 @@ def run_reference(args, rank: int, world: int):
     print(json.dumps(line), flush=True)
 
 
+def reduce_over_ranks(times_ms, counts, world: int, device):
+    """Whole-job figures from per-rank ones: MAX over ranks of every time, SUM of every count."""
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    c = torch.tensor(list(counts), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return [float(x) for x in t], [float(x) for x in c]
+
+
 def run_native(args, rank: int, world: int, local_rank: int):
     import torch
     import torch.distributed as dist
@@ -294,13 +307,7 @@ def run_native(args, rank: int, world: int, local_rank: int):
     barrier()
     e2e_ms = e0.elapsed_time(e1)
 
-    t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=dev)
-    tot = torch.tensor([float(lookups)], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
-    ms_total, e2e_ms = float(t[0]), float(t[1])
-    all_lookups = float(tot[0])
+    (ms_total, e2e_ms), (all_lookups,) = reduce_over_ranks([ms_total, e2e_ms], [float(lookups)], world, dev)
 
     if rank == 0:
         peak, peak_src = measured_peaks()
@@ -313,6 +320,12 @@ def run_native(args, rank: int, world: int, local_rank: int):
             "tbe_forward_kernel": n_avg * (per_lookup + 8) + 8 * (spec.T * B + 1) + 4.0 * B * TD,
             "reduce_chunks": n_avg * (per_lookup + 12),
         }
+        # dram__bytes_read + dram__bytes_write per lookup from the ncu capture summarised in
+        # profiles/ncu_full_cfg2_8tables_top_kernels.md (1.967 M lookups per launch there); DRAM traffic
+        # grows with the lookups processed, so a launch's traffic is this figure times its lookups.
+        # Set an entry to None when its kernel changes after the capture.
+        ncu_dram_bytes_per_lookup = {"reduce_chunks": (214.897664e6 + 158.551552e6) / 1.9667e6,
+                                     "tbe_forward_kernel": (149.063168e6 + 26.262272e6) / 1.9667e6}
         top = max(trace.items(), key=lambda kv: kv[1][0]) if trace else (None, (0.0, 0))
         kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps} for k, v in trace.items()}
         roof = None
@@ -320,7 +333,11 @@ def run_native(args, rank: int, world: int, local_rank: int):
             avg_ms = top[1][0] / top[1][1]
             ach = alg[top[0]] / (avg_ms * 1e-3) / 1e9
             roof = {"kernel": top[0], "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
-                    "frac": ach / peak, "traffic": None, "peak_source": peak_src,
+                    "frac": ach / peak,
+                    "traffic": (ncu_dram_bytes_per_lookup[top[0]] * n_avg
+                                if spec.name == "cfg2" and ncu_dram_bytes_per_lookup.get(top[0]) else None),
+                    "traffic_source": "ncu capture on 8 of 26 tables, scaled by lookups per launch",
+                    "peak_source": peak_src,
                     "algorithmic_bytes_per_launch": alg[top[0]], "avg_launch_ms": avg_ms,
                     "timing": "CUDA events around every launch, separate pass of the same K steps"}
         step_bytes = 2.0 * n_avg * per_lookup
