@@ -79,38 +79,55 @@ class DeviceModel:
         self.cache_ws_bytes = max([mb.cache_workspace_bytes(c, max_lookups) for c in self.caches] + [256])
         self.cache_ws = torch.empty(self.cache_ws_bytes, dtype=torch.uint8, device=self.device)
         if self.cached:
-            n = max_lookups
-            dev = self.device
-            self.slot_of_lookup = torch.full((n,), -1, dtype=torch.int32, device=dev)
-            self.keys = torch.empty(n, dtype=torch.int64, device=dev)
-            self.lists = []
-            for c in self.caches:
-                esz = 4 if self.spec.dtype == wl.FP32 else 2
-                self.lists.append(dict(
-                    miss_keys=torch.empty(n, dtype=torch.int64, device=dev),
-                    miss_slots=torch.empty(n, dtype=torch.int32, device=dev),
-                    evict_keys=torch.empty(n, dtype=torch.int64, device=dev),
-                    evict_slots=torch.empty(n, dtype=torch.int32, device=dev),
-                    evict_dirty=torch.empty(n, dtype=torch.uint8, device=dev),
-                    counters=torch.zeros(mb.NUM_COUNTERS, dtype=torch.int64, device=dev),
-                    staging=torch.empty(n * c.dim * esz, dtype=torch.uint8, device=dev),
-                    capacity=n))
+            # two batch contexts, so that the cache calls of batch t+1 can run while batch t trains
+            self.ctx = [self._new_context(max_lookups) for _ in range(2)]
+            self.cur = 0
+
+    def _new_context(self, n: int):
+        dev = self.device
+        esz = 4 if self.spec.dtype == wl.FP32 else 2
+        lists = []
+        for c in self.caches:
+            cap = min(n, c.num_sets * c.ways)        # a call can place at most one row per slot
+            lists.append(dict(
+                miss_keys=torch.empty(cap, dtype=torch.int64, device=dev),
+                miss_slots=torch.empty(cap, dtype=torch.int32, device=dev),
+                evict_keys=torch.empty(cap, dtype=torch.int64, device=dev),
+                evict_slots=torch.empty(cap, dtype=torch.int32, device=dev),
+                evict_dirty=torch.empty(cap, dtype=torch.uint8, device=dev),
+                counters=torch.zeros(mb.NUM_COUNTERS, dtype=torch.int64, device=dev),
+                staging=torch.empty(cap * c.dim * esz, dtype=torch.uint8, device=dev),
+                capacity=cap))
+        return dict(slot=torch.full((n,), -1, dtype=torch.int32, device=dev),
+                    keys=torch.empty(n, dtype=torch.int64, device=dev), lists=lists)
+
+    @property
+    def slot_of_lookup(self):
+        return self.ctx[self.cur]["slot"]
+
+    @property
+    def lists(self):
+        return self.ctx[self.cur]["lists"]
 
     # ------------------------------------------------------------------ steps of the path
-    def forward(self, indices, offsets, N: int, out=None, pooling_mode: int = mb.POOL_SUM, stream=None):
+    def forward(self, indices, offsets, N: int, out=None, pooling_mode: int = mb.POOL_SUM, stream=None,
+                ctx: Optional[int] = None):
         if out is None:
             out = torch.empty((self.spec.batch, self.spec.total_dim), dtype=torch.float32, device=self.device)
-        mb.tbe_forward(self.tables, self.spec.batch, indices, offsets, N, pooling_mode,
-                       self.slot_of_lookup if self.cached else None, self.cache_data, out, out.shape[1], stream)
+        slot = self.ctx[self.cur if ctx is None else ctx]["slot"] if self.cached else None
+        mb.tbe_forward(self.tables, self.spec.batch, indices, offsets, N, pooling_mode, slot, self.cache_data, out,
+                       out.shape[1], stream)
         return out
 
     def backward(self, indices, offsets, N: int, grad_out, lr: Optional[float] = None, eps: Optional[float] = None,
-                 pooling_mode: int = mb.POOL_SUM, uniq_rows_out=None, n_unique_out=None, stream=None) -> None:
+                 pooling_mode: int = mb.POOL_SUM, uniq_rows_out=None, n_unique_out=None, stream=None,
+                 ctx: Optional[int] = None) -> None:
         self.reserve(N)
+        slot = self.ctx[self.cur if ctx is None else ctx]["slot"] if self.cached else None
         mb.tbe_backward_rowwise_adagrad(
             self.tables, self.spec.batch, indices, offsets, N, pooling_mode, grad_out, grad_out.shape[1],
             self.spec.lr if lr is None else lr, self.spec.eps if eps is None else eps,
-            self.slot_of_lookup if self.cached else None, self.cache_data, self.cache_dirty, self.workspace,
+            slot, self.cache_data, self.cache_dirty, self.workspace,
             self.ws_bytes, uniq_rows_out, n_unique_out, stream)
 
     def group_range(self, g: int, offsets_host: np.ndarray):
@@ -125,26 +142,39 @@ class DeviceModel:
         esz = 4 if self.spec.dtype == wl.FP32 else 2
         return self.host_weights.data_ptr() + int(self.spec.weight_offset[t0]) * esz
 
-    def cache_step(self, indices, offsets, offsets_host: np.ndarray, step: int, stream=None,
-                   do_prefetch: bool = True) -> None:
-        """lookup_insert + prefetch + writeback of every cache for one batch."""
+    def cache_lookup(self, indices, offsets, offsets_host: np.ndarray, step: int, stream=None,
+                     ctx: Optional[int] = None) -> None:
+        """Tag path of one batch: keys, lookup_insert of every cache (slots, miss and evict lists)."""
         B = self.spec.batch
+        cx = self.ctx[self.cur if ctx is None else ctx]
         for g, c in enumerate(self.caches):
             _, t0, t1 = self.groups[g]
             begin, n = self.group_range(g, offsets_host)
-            L = self.lists[g]
-            keys = self.keys[begin:begin + n] if n else self.keys[:0]
+            L = cx["lists"][g]
+            keys = cx["keys"][begin:begin + n]
             mb.linearize_keys(self.tables, t0, t1, B, indices, offsets, begin, n, keys if n else None, stream)
-            mb.cache_lookup_insert(c, keys if n else None, n, step,
-                                   self.slot_of_lookup[begin:begin + n] if n else None, L["miss_keys"],
-                                   L["miss_slots"], L["evict_keys"], L["evict_slots"], L["evict_dirty"],
-                                   L["capacity"], L["counters"], self.cache_ws, self.cache_ws_bytes, stream)
-            if do_prefetch:
-                hp = self.host_rows_ptr(g)
-                mb.cache_prefetch_misses(c, hp, L["miss_keys"], L["miss_slots"], L["evict_slots"], L["evict_dirty"],
-                                         L["capacity"], L["counters"], L["staging"], stream)
-                mb.cache_writeback_evicted(c, hp, L["evict_keys"], L["evict_dirty"], L["capacity"], L["counters"],
-                                           L["staging"], stream)
+            mb.cache_lookup_insert(c, keys if n else None, n, step, cx["slot"][begin:begin + n] if n else None,
+                                   L["miss_keys"], L["miss_slots"], L["evict_keys"], L["evict_slots"],
+                                   L["evict_dirty"], L["capacity"], L["counters"], self.cache_ws, self.cache_ws_bytes,
+                                   stream)
+
+    def cache_move(self, stream=None, ctx: Optional[int] = None) -> None:
+        """Data path of one batch: save dirty victims, pull missed rows from the host tier, write victims back."""
+        cx = self.ctx[self.cur if ctx is None else ctx]
+        for g, c in enumerate(self.caches):
+            L = cx["lists"][g]
+            hp = self.host_rows_ptr(g)
+            mb.cache_prefetch_misses(c, hp, L["miss_keys"], L["miss_slots"], L["evict_slots"], L["evict_dirty"],
+                                     L["capacity"], L["counters"], L["staging"], stream)
+            mb.cache_writeback_evicted(c, hp, L["evict_keys"], L["evict_dirty"], L["capacity"], L["counters"],
+                                       L["staging"], stream)
+
+    def cache_step(self, indices, offsets, offsets_host: np.ndarray, step: int, stream=None,
+                   do_prefetch: bool = True, ctx: Optional[int] = None) -> None:
+        """lookup_insert + prefetch + writeback of every cache for one batch."""
+        self.cache_lookup(indices, offsets, offsets_host, step, stream, ctx)
+        if do_prefetch:
+            self.cache_move(stream, ctx)
 
     def flush(self, stream=None) -> None:
         for g, c in enumerate(self.caches):

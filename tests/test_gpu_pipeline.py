@@ -1,0 +1,63 @@
+"""Pipelined cached training (cache work of batch t+1 on a side stream while batch t trains) must
+give the same bits as the sequential schedule, and the same cache decisions as the oracle."""
+import copy
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2305_01515_b200 import binding as mb
+from paper_2305_01515_b200 import workload as wl
+from paper_2305_01515_b200.harness import DeviceModel
+from paper_2305_01515_b200.pipeline import CachedTrainer
+from helpers import custom_spec, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("frac", [0.2, 0.004])       # roomy cache; cache smaller than a batch (overflow path)
+def test_pipelined_equals_sequential_and_oracle_tags(frac):
+    rows, dims = [20000, 9000, 4000, 12000], [64, 64, 128, 128]
+    spec = custom_spec(rows, dims, 256, wl.FP16, [8, 12, 20, 5], [1.05, 0.9, 1.2, 1.0], seed=77)
+    spec.cached = True
+    spec.cache_fraction = frac
+    spec.reuse_prob, spec.reuse_window = 0.7, 4
+    stream = wl.BatchStream(spec)
+    K = 10
+    host_batches = [stream.next() for _ in range(K)]
+    grads = [to_dev(wl.gen_grad(spec, k)) for k in range(K)]
+    W0 = wl.all_weights_numpy(spec)
+    results = []
+    for pipelined in (False, True):
+        m = DeviceModel(spec, weights=W0, lock_depth=1)
+        m.reserve(max(len(b[0]) for b in host_batches))
+        batches = [(to_dev(i), to_dev(o), o) for i, o in host_batches]
+        tr = CachedTrainer(m, pipelined=pipelined)
+        tr.run(batches, grads)
+        m.flush()
+        torch.cuda.synchronize()
+        results.append((m.weights_numpy(), m.momentum.cpu().numpy(), np.stack(tr.history)))
+        m.close()
+    (Wa, ma, ha), (Wb, mb_, hb) = results
+    assert (ha == hb).all()
+    assert (Wa.view(np.uint16) == Wb.view(np.uint16)).all()
+    assert (ma.view(np.uint32) == mb_.view(np.uint32)).all()
+    # the oracle's tag-only simulation makes the same decisions (the backward dirties every placed slot)
+    groups = spec.dim_groups()
+    B = spec.batch
+    overflow = 0
+    for g, (dim, t0, t1) in enumerate(groups):
+        rows_g = int(spec.row_offset[t1] - spec.row_offset[t0])
+        oc = oracle.Cache(wl.cache_sets_for(rows_g, frac), 32, dim, spec.dtype, 0, 1, with_data=False)
+        for k, (idx, off) in enumerate(host_batches):
+            keys = np.concatenate([spec.row_offset[t] - spec.row_offset[t0] + idx[off[t * B]:off[(t + 1) * B]]
+                                   for t in range(t0, t1)])
+            res = oc.lookup_insert(keys, k)
+            used = res["slot_of_lookup"][res["slot_of_lookup"] >= 0]
+            oc.dirty[used] = 1
+            assert dict(zip(mb.COUNTER_NAMES, hb[k, g].tolist())) == res["counters"], (g, k)
+            overflow += res["counters"]["overflow"]
+        oc.close()
+    if frac < 0.01:
+        assert overflow > 0
