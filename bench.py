@@ -372,6 +372,125 @@ def run_native(args, rank: int, world: int, local_rank: int):
         dist.destroy_process_group()
 
 
+def host_link_bandwidth(dev, nbytes: int = 1 << 30):
+    """Measured pinned host<->device copy bandwidth (GB/s), one direction at a time."""
+    import torch
+
+    h = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    d = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    res = []
+    for src, dst in ((h, d), (d, h)):
+        dst.copy_(src, non_blocking=True)
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(3):
+            dst.copy_(src, non_blocking=True)
+        e1.record()
+        torch.cuda.synchronize(dev)
+        res.append(3 * nbytes / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    return res[0], res[1]
+
+
+def run_cached(args, rank: int, world: int, local_rank: int):
+    """Configurations 4 and 5: rows in pinned host memory behind HBM caches, pipelined train step."""
+    import torch
+
+    from paper_2305_01515_b200 import binding as mb
+    from paper_2305_01515_b200.harness import DeviceModel
+    from paper_2305_01515_b200.pipeline import CachedTrainer
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if args.workload == "cfg4":
+        spec = wl.config4(seed=rank, hbm_budget_gb=args.budget_gb, n_batches=args.warmup + args.steps)
+    else:
+        spec = wl.config5(seed=rank, rows=args.rows, batch=args.batch, pooling=args.pooling, alpha=args.alpha,
+                          cache_fraction=args.cache_fraction, n_batches=args.warmup + args.steps)
+        spec.reuse_prob, spec.reuse_window = 0.0, 0
+    t_setup = time.time()
+    model = DeviceModel(spec, device=dev, lock_depth=1)
+    h2d_gbs, d2h_gbs = host_link_bandwidth(dev)
+    stream = wl.BatchStream(spec)
+    K = args.warmup + args.steps
+    host = [stream.next() for _ in range(K)]
+    n_max = max(len(b[0]) for b in host)
+    model.reserve(n_max)
+    batches = [(torch.from_numpy(i).to(dev), torch.from_numpy(o).to(dev), o) for i, o in host]
+    R = min(4, K)
+    grads = [torch.from_numpy(wl.gen_grad(spec, k)).to(dev) for k in range(R)]
+    glist = [grads[k % R] for k in range(K)]
+    setup_s = time.time() - t_setup
+    trainer = CachedTrainer(model, pipelined=not args.sequential)
+    main = torch.cuda.current_stream(dev)
+    marks = {}
+
+    def on_step(t):
+        if t == args.warmup - 1 or t == K - 1:
+            e = torch.cuda.Event(enable_timing=True)
+            e.record(main)
+            marks[t] = e
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = mb.launch_count()
+    if args.trace:
+        mb.trace_enable(True)
+    sampler.mark(True)
+    trainer.run(batches, glist, on_step=on_step)
+    torch.cuda.synchronize(dev)
+    sampler.mark(False)
+    kernels = None
+    if args.trace:
+        kernels = {k: {"ms_per_step": v[0] / K, "launches_per_step": v[1] / K} for k, v in mb.trace_report().items()}
+        mb.trace_enable(False)
+    clocks = sampler.stop()
+    launches = mb.launch_count() - launches0
+    ms = marks[args.warmup - 1].elapsed_time(marks[K - 1])
+    hist = np.stack(trainer.history)[args.warmup:]                      # [steps, caches, counters]
+    lookups = float(hist[:, :, 0].sum())
+    hit = float(hist[:, :, 2].sum()) / max(lookups, 1.0)
+    eb = spec.elem_bytes
+    dims = [d for d, _, _ in model.groups]
+    miss_bytes = sum(float(hist[:, g, 6].sum()) * dims[g] * eb for g in range(len(dims)))
+    dirty_bytes = sum(float(hist[:, g, 8].sum()) * dims[g] * eb for g in range(len(dims)))
+    B = spec.batch
+    eq3 = 0.0
+    for k in range(args.warmup, K):
+        off = host[k][1]
+        for t in range(spec.T):
+            eq3 += 2.0 * float(off[(t + 1) * B] - off[t * B]) * float(spec.dims[t]) * eb
+    peak, peak_src = measured_peaks()
+    t_hbm = eq3 / (peak * 1e9)
+    t_h2d = miss_bytes / (h2d_gbs * 1e9)
+    t_d2h = dirty_bytes / (d2h_gbs * 1e9)
+    t_roof = max(t_hbm, t_h2d, t_d2h)
+    t_meas = ms * 1e-3
+    line = {
+        "metric": METRIC, "value": lookups / t_meas, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": spec.name, "note": spec.note, "tables": spec.T, "rows_total": int(spec.row_offset[-1]),
+                   "host_weight_gb": spec.weight_bytes / 1e9, "cache_fraction": spec.cache_fraction, "batch": B,
+                   "lookups_per_step": lookups / args.steps, "schedule": "sequential" if args.sequential else "pipelined",
+                   "l2": "inputs larger than L2 (host tier and caches are GBs)", "setup_seconds": setup_s},
+        "samples_per_sec": B * args.steps / t_meas, "hit_rate_per_lookup": hit,
+        "unique_hit_rate": float(hist[:, :, 4].sum()) / max(float(hist[:, :, 1].sum()), 1.0),
+        "overflow_rows": float(hist[:, :, 9].sum()),
+        "host_link": {"h2d_gbs": h2d_gbs, "d2h_gbs": d2h_gbs, "miss_gb_per_step": miss_bytes / args.steps / 1e9,
+                      "dirty_evict_gb_per_step": dirty_bytes / args.steps / 1e9,
+                      "achieved_h2d_gbs": miss_bytes / t_meas / 1e9},
+        "roofline": {"bound": "host-link" if t_roof != t_hbm else "hbm", "t_hbm_ms": t_hbm * 1e3 / args.steps,
+                     "t_h2d_ms": t_h2d * 1e3 / args.steps, "t_d2h_ms": t_d2h * 1e3 / args.steps,
+                     "achieved": t_roof / t_meas, "peak": 1.0, "unit": "fraction of the slower of HBM and host-link time",
+                     "frac": t_roof / t_meas, "traffic": None, "peak_source": peak_src},
+        "clocks": clocks, "gpu_launches": int(launches), "e2e": None, "kernels": kernels,
+    }
+    print(json.dumps(line), flush=True)
+    model.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -381,6 +500,15 @@ def main():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--rotate", type=int, default=4, help="distinct batches that take turns")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--budget-gb", type=float, default=8.0, help="cfg4: HBM budget; host weights are 4x this")
+    ap.add_argument("--rows", type=int, default=50_000_000, help="cfg5: rows of the single table")
+    ap.add_argument("--batch", type=int, default=16384, help="cfg5: batch size")
+    ap.add_argument("--pooling", type=int, default=50, help="cfg5: lookups per bag")
+    ap.add_argument("--alpha", type=float, default=1.0, help="cfg5: Zipf exponent")
+    ap.add_argument("--cache-fraction", type=float, default=0.10, help="cfg5: cache slots / rows")
+    ap.add_argument("--sequential", action="store_true", help="cached workloads: no side stream")
+    ap.add_argument("--trace", action="store_true",
+                    help="cached workloads: CUDA events around every launch of the run (perturbs the timing)")
     ap.add_argument("--tables", type=int, default=0,
                     help="cfg2 only: fewer tables (a small case for profiler captures; not a bench line)")
     args = ap.parse_args()
@@ -393,6 +521,11 @@ def main():
         return
     if world == 1 and args.gpus > 1:
         raise SystemExit("launch with torch.distributed.run for --gpus > 1")
+    if args.workload in ("cfg4", "cfg5"):
+        if world > 1:
+            raise SystemExit("cached workloads are single-GPU bench lines")
+        run_cached(args, rank, world, local_rank)
+        return
     run_native(args, rank, world, local_rank)
 
 

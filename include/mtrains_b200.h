@@ -210,6 +210,10 @@ typedef struct mts_cache mts_cache;
 int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_space, int32_t ways, int32_t dim,
                      int32_t dtype, int32_t policy, int32_t lock_depth);
 int mts_cache_destroy(mts_cache* cache);
+/* Reads and clears the cache's sticky device status word; synchronises `stream`.  Bit 0: a
+ * bounded wait for a bulk copy of missed rows ran out (the kernel gave up instead of hanging; the
+ * rows of that call are incomplete) — also reported as MTS_ERR_TIMEOUT. */
+int mts_cache_status(mts_cache* cache, int32_t* host_status, void* stream);
 void* mts_cache_data(mts_cache* cache);        /* device [num_sets*32, dim] */
 uint8_t* mts_cache_dirty(mts_cache* cache);    /* device [num_sets*32] */
 

@@ -29,7 +29,7 @@ EXPORTS = (
     "mts_trace_kernel_name", "mts_trace_report", "mts_tables_create", "mts_tables_destroy", "mts_tables_status",
     "mts_tbe_forward", "mts_tbe_backward_workspace_bytes", "mts_tbe_backward_rowwise_adagrad",
     "mts_tbe_backward_rowwise_adagrad_static",
-    "mts_cache_create", "mts_cache_destroy", "mts_cache_data", "mts_cache_dirty",
+    "mts_cache_create", "mts_cache_destroy", "mts_cache_status", "mts_cache_data", "mts_cache_dirty",
     "mts_linearize_keys", "mts_cache_workspace_bytes", "mts_cache_lookup_insert",
     "mts_cache_prefetch_misses", "mts_cache_writeback_evicted", "mts_cache_flush",
     "mts_cache_export_state",
@@ -85,6 +85,7 @@ def lib():
                                                               C.POINTER(vp), C.POINTER(vp), i32, vp, vp, vp]
         L.mts_cache_create.argtypes = [C.POINTER(vp), i64, i64, i32, i32, i32, i32, i32]
         L.mts_cache_destroy.argtypes = [vp]
+        L.mts_cache_status.argtypes = [vp, C.POINTER(i32), vp]
         L.mts_cache_data.restype = vp
         L.mts_cache_data.argtypes = [vp]
         L.mts_cache_dirty.restype = vp
@@ -247,6 +248,11 @@ class Cache:
         self.num_sets, self.ways, self.dim, self.dtype = num_sets, ways, dim, dtype
         self.data_ptr = int(lib().mts_cache_data(h))
         self.dirty_ptr = int(lib().mts_cache_dirty(h))
+
+    def status(self, stream=None) -> int:
+        st = C.c_int32(0)
+        _check(lib().mts_cache_status(self.handle, C.byref(st), _stream(stream)))
+        return int(st.value)
 
     def destroy(self):
         if self.handle:

@@ -27,6 +27,7 @@ struct mts_cache {
   uint32_t* freq = nullptr;      // [S*32]
   uint8_t* dirty = nullptr;      // [S*32]
   char* data = nullptr;          // [S*32, row_bytes]
+  int32_t* d_status = nullptr;   // sticky status bits (bit 0: a bounded wait on a bulk copy ran out)
 };
 
 namespace mts {
@@ -328,7 +329,13 @@ __global__ void cache_scatter_slots(const uint32_t* __restrict__ sorted_pos, con
 // Row copies in 16-byte pieces; thread i of the flattened (row, piece) space moves one piece,
 // UNROLL independent pieces per thread are in flight before the first store.
 
-constexpr int COPY_UNROLL = 4;
+#ifndef MTS_COPY_UNROLL
+#define MTS_COPY_UNROLL 4
+#endif
+#ifndef MTS_COPY_BLOCKS_PER_SM
+#define MTS_COPY_BLOCKS_PER_SM 8
+#endif
+constexpr int COPY_UNROLL = MTS_COPY_UNROLL;
 
 template <typename SrcOf, typename DstOf>
 __device__ __forceinline__ void copy_rows(int64_t n_rows, int vec16, SrcOf src_of, DstOf dst_of) {
@@ -383,6 +390,85 @@ cache_fetch_misses(char* __restrict__ data, int row_bytes, const char* __restric
   copy_rows(n, row_bytes / 16,
             [&](int64_t k) { return host_rows + miss_keys[k] * row_bytes; },
             [&](int64_t k) { return data + (int64_t)miss_slots[k] * row_bytes; });
+}
+
+// ---- missed rows through the bulk-copy engine (TMA, non-tensor form) ------------------------
+// Plain 16-byte loads from mapped host memory top out far below the host link's bandwidth (the
+// requests that reach the link are small).  Here one warp per block asks the bulk-copy engine for
+// whole rows (host memory -> shared memory, completion counted in bytes on an mbarrier); the block
+// then stores the tile to the rows' cache slots.  The wait on the mbarrier is bounded: if it ever
+// ran out, the block raises the cache's status bit, waits once more (bounded) for its copies in
+// flight and leaves, so the kernel cannot hang.
+#ifndef MTS_FETCH_BLOCKS_PER_SM
+#define MTS_FETCH_BLOCKS_PER_SM 8
+#endif
+constexpr int FETCH_THREADS = 128;
+constexpr int FETCH_TILE_BYTES = 16384;
+constexpr uint32_t FETCH_WAIT_LIMIT = 1u << 22;
+
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+
+__global__ void __launch_bounds__(FETCH_THREADS)
+cache_fetch_misses_bulk(char* __restrict__ data, int row_bytes, const char* __restrict__ host_rows,
+                        const int64_t* __restrict__ miss_keys, const int32_t* __restrict__ miss_slots,
+                        const int64_t* __restrict__ counters, int64_t capacity, int32_t* status) {
+  __shared__ __align__(128) unsigned char tile[FETCH_TILE_BYTES];
+  __shared__ __align__(8) unsigned long long bar_storage;
+  const int64_t n = list_len(counters, MTS_CNT_INSERTED, capacity);
+  const int rows_per_tile = FETCH_TILE_BYTES / row_bytes;
+  const int64_t n_tiles = (n + rows_per_tile - 1) / rows_per_tile;
+  const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&bar_storage);
+  const uint32_t tile_s = (uint32_t)__cvta_generic_to_shared(tile);
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  uint32_t parity = 0;
+  const int vec = row_bytes / 16;
+  for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+    const int64_t r0 = t * rows_per_tile;
+    const int nr = (int)min((int64_t)rows_per_tile, n - r0);
+    if (threadIdx.x < 32) {
+      // writes of the engine into the tile must be ordered after the block's reads of the last tile
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      if (threadIdx.x == 0)
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)(nr * row_bytes))
+                     : "memory");
+      __syncwarp();
+      for (int k = threadIdx.x; k < nr; k += 32) {
+        const char* src = host_rows + miss_keys[r0 + k] * (int64_t)row_bytes;
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(tile_s + (uint32_t)(k * row_bytes)), "l"(src), "r"((uint32_t)row_bytes), "r"(bar)
+                     : "memory");
+      }
+    }
+    bool ok = mbar_wait_bounded(bar, parity, FETCH_WAIT_LIMIT);
+    if (!__syncthreads_and(ok)) {
+      if (threadIdx.x == 0) atomicOr(status, 1);
+      mbar_wait_bounded(bar, parity, FETCH_WAIT_LIMIT);
+      return;
+    }
+    parity ^= 1u;
+    const int total = nr * vec;
+    for (int e = threadIdx.x; e < total; e += FETCH_THREADS) {
+      const int k = e / vec, c = e - k * vec;
+      *reinterpret_cast<uint4*>(data + (int64_t)miss_slots[r0 + k] * row_bytes + c * 16) =
+          *reinterpret_cast<const uint4*>(tile + k * row_bytes + c * 16);
+    }
+    __syncthreads();
+  }
 }
 
 __global__ void __launch_bounds__(CACHE_THREADS)
@@ -476,6 +562,8 @@ extern "C" int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_s
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->freq, n * 4), "cudaMalloc(counts)");
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->dirty, n), "cudaMalloc(dirty)");
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->data, (size_t)n * c->row_bytes), "cudaMalloc(cache rows)");
+  if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->d_status, 256), "cudaMalloc(cache status)");
+  if (rc == MTS_OK) rc = check_cuda(cudaMemset(c->d_status, 0, 256), "cudaMemset(cache status)");
   if (rc == MTS_OK) {
     {
       LaunchScope scope(K_OTHER, nullptr);
@@ -492,9 +580,20 @@ extern "C" int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_s
 
 extern "C" int mts_cache_destroy(mts_cache* c) {
   if (!c) return MTS_OK;
-  cudaFree(c->tags); cudaFree(c->ts); cudaFree(c->freq); cudaFree(c->dirty); cudaFree(c->data);
+  cudaFree(c->tags); cudaFree(c->ts); cudaFree(c->freq); cudaFree(c->dirty); cudaFree(c->data); cudaFree(c->d_status);
   delete c;
   return MTS_OK;
+}
+
+extern "C" int mts_cache_status(mts_cache* c, int32_t* host_status, void* stream) {
+  if (!c || !host_status) return set_error(MTS_ERR_INVALID_ARG, "cache_status: null argument");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int rc = check_cuda(cudaMemcpyAsync(host_status, c->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, s),
+                      "cudaMemcpyAsync(cache status)");
+  if (rc == MTS_OK) rc = check_cuda(cudaMemsetAsync(c->d_status, 0, sizeof(int32_t), s), "cudaMemsetAsync(cache status)");
+  if (rc == MTS_OK) rc = check_cuda(cudaStreamSynchronize(s), "cudaStreamSynchronize(cache status)");
+  if (rc == MTS_OK && (*host_status & 1)) return set_error(MTS_ERR_TIMEOUT, "cache: a bounded wait on a bulk copy ran out");
+  return rc;
 }
 
 extern "C" void* mts_cache_data(mts_cache* c) { return c ? c->data : nullptr; }
@@ -651,8 +750,14 @@ extern "C" int mts_cache_prefetch_misses(mts_cache* c, const void* host_rows_map
   }
   {
     LaunchScope scope(K_CACHE_FETCH_MISSES, s);
+#ifdef MTS_FETCH_PLAIN_LOADS
     cache_fetch_misses<<<grid, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, static_cast<const char*>(host_rows_mapped),
                                                       miss_keys, miss_slots, counters, list_capacity);
+#else
+    cache_fetch_misses_bulk<<<c->sm_count * MTS_FETCH_BLOCKS_PER_SM, FETCH_THREADS, 0, s>>>(
+        c->data, c->row_bytes, static_cast<const char*>(host_rows_mapped), miss_keys, miss_slots, counters,
+        list_capacity, c->d_status);
+#endif
   }
   return check_launch("cache_save_victims / cache_fetch_misses");
 }
