@@ -441,6 +441,19 @@ def run_cached(args, rank: int, world: int, local_rank: int):
     trainer.run(batches, glist, on_step=on_step)
     torch.cuda.synchronize(dev)
     sampler.mark(False)
+    # diagnostics on the last batch, GPU otherwise idle: lookups that bypass the cache, forward alone
+    last_ctx = (K - 1) & 1
+    n_last = batches[K - 1][0].numel()
+    bypass = int((model.ctx[last_ctx]["slot"][:n_last] < 0).sum().item())
+    out_d = torch.empty((spec.batch, spec.total_dim), dtype=torch.float32, device=dev)
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    model.forward(batches[K - 1][0], batches[K - 1][1], n_last, out=out_d, stream=main, ctx=last_ctx)
+    f0.record(main)
+    for _ in range(3):
+        model.forward(batches[K - 1][0], batches[K - 1][1], n_last, out=out_d, stream=main, ctx=last_ctx)
+    f1.record(main)
+    torch.cuda.synchronize(dev)
+    fwd_alone_ms = f0.elapsed_time(f1) / 3
     kernels = None
     if args.trace:
         kernels = {k: {"ms_per_step": v[0] / K, "launches_per_step": v[1] / K} for k, v in mb.trace_report().items()}
@@ -477,7 +490,8 @@ def run_cached(args, rank: int, world: int, local_rank: int):
                    "l2": "inputs larger than L2 (host tier and caches are GBs)", "setup_seconds": setup_s},
         "samples_per_sec": B * args.steps / t_meas, "hit_rate_per_lookup": hit,
         "unique_hit_rate": float(hist[:, :, 4].sum()) / max(float(hist[:, :, 1].sum()), 1.0),
-        "overflow_rows": float(hist[:, :, 9].sum()),
+        "overflow_rows": float(hist[:, :, 9].sum()), "lookups_bypassing_cache_last_step": bypass,
+        "forward_alone_ms_last_step": fwd_alone_ms,
         "host_link": {"h2d_gbs": h2d_gbs, "d2h_gbs": d2h_gbs, "miss_gb_per_step": miss_bytes / args.steps / 1e9,
                       "dirty_evict_gb_per_step": dirty_bytes / args.steps / 1e9,
                       "achieved_h2d_gbs": miss_bytes / t_meas / 1e9},

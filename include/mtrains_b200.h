@@ -229,8 +229,8 @@ int mts_linearize_keys(const mts_tables* tables, int32_t t_begin, int32_t t_end,
  *  1. every distinct key is probed in its set; a lookup is a hit iff its key was resident
  *     before the call;
  *  2. all hits are refreshed (timestamp = step);
- *  3. per set, the missing keys in ascending order take the set's evictable ways (timestamp
- *     < step - lock_depth; free ways first) in (timestamp, way) order [LFU: (count, timestamp,
+ *  3. per set, the missing keys in ascending order take the set's evictable ways (free ways,
+ *     then ways with timestamp < step - lock_depth) in (timestamp, way) order [LFU: (count, timestamp,
  *     way)]; a victim with a valid tag is appended to the evict list with its dirty byte, which
  *     is cleared; missing keys beyond the evictable ways are not inserted (slot -1, counted as
  *     overflow);

@@ -337,8 +337,8 @@ static int64_t find_way(const orc_cache* c, int64_t set, int64_t key) {
  *     before this call.
  *  2. All hits are refreshed first (ts = step; LFU: count += occurrences in the batch).
  *  3. Then, set by set (ascending), the set's missing keys in ascending order are paired
- *     with the set's evictable ways.  A way is evictable iff ts < step - lock_depth (free
- *     ways have ts = -1).  Candidates are ordered by (ts, way) for LRU and by
+ *     with the set's evictable ways.  A way is evictable iff it is free or its ts <
+ *     step - lock_depth (free ways have ts = -1, so they are taken first).  Candidates are ordered by (ts, way) for LRU and by
  *     (count, ts, way) for LFU; the k-th missing key takes the k-th candidate.  A victim
  *     with a valid tag is appended to the evict list with its dirty byte, which is then
  *     cleared.  Misses beyond the candidates are not inserted: slot -1 (overflow).
@@ -396,7 +396,7 @@ int64_t orc_cache_lookup_insert(orc_cache* c, const int64_t* keys, int64_t N, in
         int64_t set = ms[a].set;
         int32_t nc = 0;
         for (int32_t w = 0; w < c->ways; ++w)
-            if (c->ts[set * c->ways + w] < step - c->lock_depth) cand[nc++] = w;
+            if (c->tag[set * c->ways + w] == -1 || c->ts[set * c->ways + w] < step - c->lock_depth) cand[nc++] = w;
         /* order candidates; insertion sort keeps it plain */
         for (int32_t x = 1; x < nc; ++x) {
             int32_t w = cand[x]; int32_t y = x - 1;

@@ -124,7 +124,7 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
       }
     }
     // candidates after the refresh: ways outside the lock window, free ways first by their -1 stamp
-    const bool cand = stamp < step - lock_depth;
+    const bool cand = tag == FREE_TAG || stamp < step - lock_depth;
     const uint32_t cand_mask = __ballot_sync(0xffffffffu, cand);
     const int ncand = __popc(cand_mask);
     int rank = 0;
@@ -399,8 +399,8 @@ cache_fetch_misses(char* __restrict__ data, int row_bytes, const char* __restric
 // then stores the tile to the rows' cache slots.  The wait on the mbarrier is bounded: if it ever
 // ran out, the block raises the cache's status bit, waits once more (bounded) for its copies in
 // flight and leaves, so the kernel cannot hang.
-#ifndef MTS_FETCH_BLOCKS_PER_SM
-#define MTS_FETCH_BLOCKS_PER_SM 8
+#ifndef MTS_FETCH_BLOCKS
+#define MTS_FETCH_BLOCKS 32      // blocks of the bulk-copy fetch: the host link needs few copies in flight
 #endif
 constexpr int FETCH_THREADS = 128;
 constexpr int FETCH_TILE_BYTES = 16384;
@@ -754,7 +754,7 @@ extern "C" int mts_cache_prefetch_misses(mts_cache* c, const void* host_rows_map
     cache_fetch_misses<<<grid, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, static_cast<const char*>(host_rows_mapped),
                                                       miss_keys, miss_slots, counters, list_capacity);
 #else
-    cache_fetch_misses_bulk<<<c->sm_count * MTS_FETCH_BLOCKS_PER_SM, FETCH_THREADS, 0, s>>>(
+    cache_fetch_misses_bulk<<<MTS_FETCH_BLOCKS, FETCH_THREADS, 0, s>>>(
         c->data, c->row_bytes, static_cast<const char*>(host_rows_mapped), miss_keys, miss_slots, counters,
         list_capacity, c->d_status);
 #endif

@@ -1,14 +1,23 @@
-"""Schedule of the cached train step: the cache work of batch t+1 (tag lookup, miss prefetch,
-dirty writeback) runs on a side stream while batch t trains on the main stream (Section 5.7 of
-the paper: prefetch into the cache ahead of training; Section 6.1: cache kernels on their own
-streams, synchronised with the next batch's lookups).  Only events order the two streams.
+"""Schedule of the cached train step (Section 5.7 of the paper: prefetch into the cache ahead of
+training; Section 6.1: cache kernels on their own streams, synchronised with the next batch's
+lookups).  Three streams, ordered by events only:
 
-Why this is safe with lock_depth >= 1: the replacement of batch t+1 may only take ways whose
-timestamp is older than t, so it never touches a slot batch t reads or updates; its decisions depend
-on tags and timestamps only, which batch t's forward/backward do not write.  The one data hazard is
-a row that found no evictable way in batch t (served from host memory directly) and is fetched from
-host memory for batch t+1: when batch t reported such overflow, the data movement of batch t+1 waits
-for batch t's backward.
+    main : forward(t), backward(t)
+    move : save victims / fetch missed rows / write victims back for batch t+1   (host link)
+    tag  : tag lookup and replacement for batch t+2                              (HBM, small)
+
+so the host-link traffic of the next batch and the tag work of the one after it overlap the
+training of the current batch.
+
+Why this is safe with lock_depth >= 1.  The tag step of batch t+2 waits for backward(t); it may only
+take ways stamped at t or earlier, i.e. rows whose batches have trained, and never a way of batch
+t+1 (stamped t+1), which is still waiting to train.  Its decisions read and write tags, timestamps
+and the dirty bytes of its victims only; forward/backward write none of the first two and only the
+dirty bytes of their own batch's slots.  The data movement of batch t+1 touches victim slots (trained
+at t-1 or earlier, complete because the tag step waited for backward(t-1)) and the slots of missed
+rows, which no batch in flight uses.  One hazard is left: a row that found no evictable way in batch
+t (it is read and updated in host memory directly) and is fetched from host memory for batch t+1.
+When batch t reported such overflow, the data movement of batch t+1 waits for backward(t).
 """
 from __future__ import annotations
 
@@ -28,25 +37,37 @@ class CachedTrainer:
         self.pipelined = pipelined
         self.dev = model.device
         self.main = torch.cuda.current_stream(self.dev)
-        self.side = torch.cuda.Stream(self.dev) if pipelined else self.main
+        self.tag = torch.cuda.Stream(self.dev) if pipelined else self.main
+        self.move = torch.cuda.Stream(self.dev) if pipelined else self.main
         n_c = len(model.caches)
         self.host_counters = [torch.zeros((n_c, mb.NUM_COUNTERS), dtype=torch.int64).pin_memory() for _ in range(2)]
         self.history: List[np.ndarray] = []           # per batch [n_caches, NUM_COUNTERS]
 
-    def _prepare(self, t, batch, ctx, ev_tags, ev_ready, wait_bwd_prev, wait_bwd_cur_if_overflow):
-        """Cache work of batch t into context ctx on the side stream."""
-        m, s = self.m, self.side
-        idx, off, off_host = batch[0], batch[1], batch[2]
-        if wait_bwd_prev is not None:
-            s.wait_event(wait_bwd_prev)                 # victims' rows and dirty bytes are final
-        m.cache_lookup(idx, off, off_host, t, stream=s, ctx=ctx)
-        for g in range(len(m.caches)):
-            self.host_counters[ctx][g].copy_(m.ctx[ctx]["lists"][g]["counters"], non_blocking=True)
+    def _lookup(self, t, step, batch, ev_tags, wait_event):
+        """Tag path of batch t on the tag stream (into context t mod 2)."""
+        m, s, ctx = self.m, self.tag, t & 1
+        if wait_event is not None:
+            s.wait_event(wait_event)
+        m.cache_lookup(batch[0], batch[1], batch[2], step, stream=s, ctx=ctx)
+        with torch.cuda.stream(s):
+            for g in range(len(m.caches)):
+                self.host_counters[ctx][g].copy_(m.ctx[ctx]["lists"][g]["counters"], non_blocking=True)
         ev_tags.record(s)
-        if wait_bwd_cur_if_overflow is not None:
-            s.wait_event(wait_bwd_cur_if_overflow)
-        m.cache_move(stream=s, ctx=ctx)
+
+    def _move(self, t, ev_tags, ev_ready, wait_event):
+        """Data path of batch t on the move stream."""
+        s = self.move
+        s.wait_event(ev_tags)
+        if wait_event is not None:
+            s.wait_event(wait_event)
+        self.m.cache_move(stream=s, ctx=t & 1)
         ev_ready.record(s)
+
+    def _counters(self, t, ev_tags) -> bool:
+        ev_tags.synchronize()                        # counters of batch t are on the host
+        cnt = self.host_counters[t & 1].numpy().copy()
+        self.history.append(cnt)
+        return bool(cnt[:, mb.COUNTER_NAMES.index("overflow")].sum() > 0)
 
     def run(self, batches, grads, out: Optional[torch.Tensor] = None,
             on_step: Optional[Callable[[int], None]] = None, first_step: int = 0) -> None:
@@ -55,40 +76,46 @@ class CachedTrainer:
         K = len(batches)
         if K == 0:
             return
-        with torch.cuda.stream(self.side):
-            pass
         ev_tags = [torch.cuda.Event() for _ in range(K)]
         ev_ready = [torch.cuda.Event() for _ in range(K)]
         ev_bwd = [torch.cuda.Event() for _ in range(K)]
         if out is None:
             out = torch.empty((m.spec.batch, m.spec.total_dim), dtype=torch.float32, device=self.dev)
-        prev_overflow = False
-        # side stream must see the inputs produced on the main stream
+        if not self.pipelined:
+            for t in range(K):
+                idx, off, _ = batches[t]
+                self._lookup(t, first_step + t, batches[t], ev_tags[t], None)
+                self._move(t, ev_tags[t], ev_ready[t], None)
+                m.forward(idx, off, idx.numel(), out=out, stream=self.main, ctx=t & 1)
+                m.backward(idx, off, idx.numel(), grads[t], stream=self.main, ctx=t & 1)
+                self._counters(t, ev_tags[t])
+                if on_step is not None:
+                    on_step(t)
+            return
+        # the side streams must see the inputs produced on the main stream
         start = torch.cuda.Event()
         start.record(self.main)
-        self.side.wait_event(start)
-        if self.pipelined:
-            with torch.cuda.stream(self.side):
-                self._prepare(first_step, batches[0], 0, ev_tags[0], ev_ready[0], None, None)
+        self.tag.wait_event(start)
+        self.move.wait_event(start)
+        overflow = {}
+        self._lookup(0, first_step, batches[0], ev_tags[0], None)
+        self._move(0, ev_tags[0], ev_ready[0], None)
+        overflow[0] = self._counters(0, ev_tags[0])
+        if K > 1:
+            self._lookup(1, first_step + 1, batches[1], ev_tags[1], None)
         for t in range(K):
-            ctx = t & 1
             idx, off, _ = batches[t]
-            N = idx.numel()
-            if not self.pipelined:
-                self._prepare(first_step + t, batches[t], ctx, ev_tags[t], ev_ready[t], None, None)
-            else:
-                self.main.wait_event(ev_ready[t])
-            m.forward(idx, off, N, out=out, stream=self.main, ctx=ctx)
-            m.backward(idx, off, N, grads[t], stream=self.main, ctx=ctx)
+            self.main.wait_event(ev_ready[t])
+            m.forward(idx, off, idx.numel(), out=out, stream=self.main, ctx=t & 1)
+            m.backward(idx, off, idx.numel(), grads[t], stream=self.main, ctx=t & 1)
             ev_bwd[t].record(self.main)
-            ev_tags[t].synchronize()                     # counters of batch t are on the host
-            cnt = self.host_counters[ctx].numpy().copy()
-            self.history.append(cnt)
-            overflow_t = bool(cnt[:, 9].sum() > 0)
-            if self.pipelined and t + 1 < K:
-                with torch.cuda.stream(self.side):
-                    self._prepare(first_step + t + 1, batches[t + 1], (t + 1) & 1, ev_tags[t + 1], ev_ready[t + 1],
-                                  ev_bwd[t - 1] if t >= 1 else None, ev_bwd[t] if overflow_t else None)
+            if t + 1 < K:
+                overflow[t + 1] = self._counters(t + 1, ev_tags[t + 1])
+                self._move(t + 1, ev_tags[t + 1], ev_ready[t + 1], ev_bwd[t] if overflow[t] else None)
+            if t + 2 < K:
+                # context (t+2) mod 2 is the one batch t is using: wait for its backward
+                self._lookup(t + 2, first_step + t + 2, batches[t + 2], ev_tags[t + 2], ev_bwd[t])
             if on_step is not None:
                 on_step(t)
-        self.main.wait_stream(self.side)
+        self.main.wait_stream(self.tag)
+        self.main.wait_stream(self.move)

@@ -174,10 +174,12 @@ def test_cached_training_matches_oracle_and_is_transparent(dtype, frac, lock):
     model.close()
 
 
-def test_gpu_cached_run_equals_gpu_uncached_run_bitwise():
-    """Transparency on the GPU alone: cached and uncached training give identical bits."""
-    rows, dims = [5000, 2500], [128, 128]
-    spec = custom_spec(rows, dims, 128, wl.FP16, [8, 12], [1.05, 1.1], seed=33)
+@pytest.mark.parametrize("dim,dtype", [(128, wl.FP16), (8, wl.FP16), (1024, wl.FP32)])
+def test_gpu_cached_run_equals_gpu_uncached_run_bitwise(dim, dtype):
+    """Transparency on the GPU alone: cached and uncached training give identical bits (rows of
+    256 B, of 16 B and of 4 KB go through the bulk-copy fetch)."""
+    rows, dims = [5000, 2500], [dim, dim]
+    spec = custom_spec(rows, dims, 128, dtype, [8, 12], [1.05, 1.1], seed=33)
     W0 = wl.all_weights_numpy(spec)
     plain = DeviceModel(spec, weights=W0)
     import copy
@@ -197,6 +199,7 @@ def test_gpu_cached_run_equals_gpu_uncached_run_bitwise():
         plain.backward(d_idx, d_off, N, grad)
     cached.flush()
     torch.cuda.synchronize()
-    assert (cached.weights_numpy().view(np.uint16) == plain.weights_numpy().view(np.uint16)).all()
+    assert all(c.status() == 0 for c in cached.caches)
+    assert (cached.weights_numpy().view(np.uint8) == plain.weights_numpy().view(np.uint8)).all()
     assert torch.equal(cached.momentum, plain.momentum)
     plain.close(); cached.close()

@@ -36,7 +36,7 @@ class ListCache:
         miss, evict, overflow = [], [], 0
         for s in sorted(by_set):
             order = sorted(self.sets[s], key=lambda e: (e[2], e[0]))
-            cands = [e for e in order if e[2] < step - self.lock]
+            cands = [e for e in order if e[1] == -1 or e[2] < step - self.lock]
             todo = [k for k in by_set[s] if k not in hits]
             for j, k in enumerate(todo):
                 if j < len(cands):
@@ -157,6 +157,15 @@ def test_lock_window_protects_rows_of_batches_in_flight():
         assert not (set(res["evict_keys"].tolist()) & prev), "evicted a row of the batch in flight"
         placed = {int(k) for k, s in zip(keys, res["slot_of_lookup"]) if s >= 0}
         prev = placed
+    c.close()
+
+
+def test_free_ways_are_usable_from_the_first_step_whatever_the_lock_depth():
+    """Section 5.5.2: a missed index takes a free slot when there is one; eviction (and with it the
+    lock window) only matters once the set is full."""
+    c = oracle.Cache(2, 4, 4, wl.FP32, 0, 3, with_data=False)
+    res = c.lookup_insert(np.arange(6, dtype=np.int64), 0)
+    assert res["counters"]["overflow"] == 0 and res["counters"]["inserted"] == 6 and res["counters"]["evicted"] == 0
     c.close()
 
 
