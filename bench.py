@@ -442,7 +442,7 @@ def run_cached(args, rank: int, world: int, local_rank: int):
     torch.cuda.synchronize(dev)
     sampler.mark(False)
     # diagnostics on the last batch, GPU otherwise idle: lookups that bypass the cache, forward alone
-    last_ctx = (K - 1) & 1
+    last_ctx = (K - 1) % DeviceModel.N_CTX
     n_last = batches[K - 1][0].numel()
     bypass = int((model.ctx[last_ctx]["slot"][:n_last] < 0).sum().item())
     out_d = torch.empty((spec.batch, spec.total_dim), dtype=torch.float32, device=dev)

@@ -239,6 +239,8 @@ int mts_linearize_keys(const mts_tables* tables, int32_t t_begin, int32_t t_end,
  * order of the misses that displaced them).  list_capacity >= number of distinct keys is always
  * enough; entries beyond the capacity are dropped while MTS_CNT_INSERTED / MTS_CNT_EVICTED
  * keep counting, so a counter above list_capacity tells the caller that a list was cut.
+ * overflow_keys (nullable, device int64 [list_capacity]): the keys counted in MTS_CNT_OVERFLOW, in no
+ * particular order (see mts_cache_refetch_overflowed).
  * counters: device int64 [MTS_NUM_COUNTERS], overwritten.  `step` must not decrease between calls.
  * workspace: at least mts_cache_workspace_bytes(cache, N) bytes, 256-byte aligned.
  * Errors: INVALID_ARG, WORKSPACE, CUDA. */
@@ -246,8 +248,8 @@ size_t mts_cache_workspace_bytes(const mts_cache* cache, int64_t N);
 int mts_cache_lookup_insert(mts_cache* cache, const int64_t* keys, int64_t N, int64_t step,
                             int32_t* slot_of_lookup, int64_t* miss_keys, int32_t* miss_slots,
                             int64_t* evict_keys, int32_t* evict_slots, uint8_t* evict_dirty,
-                            int64_t list_capacity, int64_t* counters, void* workspace,
-                            size_t workspace_bytes, void* stream);
+                            int64_t* overflow_keys, int64_t list_capacity, int64_t* counters,
+                            void* workspace, size_t workspace_bytes, void* stream);
 
 /* Data movement for one lookup_insert result (Sections 5.5.3, 5.5.4): first the rows of dirty
  * victims are saved, slot -> evict_staging[k] (k = position in the evict list), then every
@@ -262,6 +264,15 @@ int mts_cache_prefetch_misses(mts_cache* cache, const void* host_rows_mapped, co
 int mts_cache_writeback_evicted(mts_cache* cache, void* host_rows_mapped, const int64_t* evict_keys,
                                 const uint8_t* evict_dirty, int64_t list_capacity,
                                 const int64_t* counters, const void* evict_staging, void* stream);
+
+/* Support for running the data movement of batch t+1 while batch t still trains (Section 5.7).
+ * A key that overflowed in batch t is read and updated in the host tier by batch t's forward and
+ * backward; if batch t+1 places that key, mts_cache_prefetch_misses(t+1) may have copied the host
+ * row before batch t's update reached it.  Call this after batch t's backward with batch t's
+ * overflow list and counters: every listed key that is resident now gets its row copied from the
+ * host tier again.  A no-op when the steps run one after the other. */
+int mts_cache_refetch_overflowed(mts_cache* cache, const void* host_rows_mapped, const int64_t* overflow_keys,
+                                 int64_t list_capacity, const int64_t* counters, void* stream);
 
 /* Writes every dirty resident row to the host tier and clears its dirty byte. */
 int mts_cache_flush(mts_cache* cache, void* host_rows_mapped, void* stream);

@@ -31,7 +31,7 @@ EXPORTS = (
     "mts_tbe_backward_rowwise_adagrad_static",
     "mts_cache_create", "mts_cache_destroy", "mts_cache_status", "mts_cache_data", "mts_cache_dirty",
     "mts_linearize_keys", "mts_cache_workspace_bytes", "mts_cache_lookup_insert",
-    "mts_cache_prefetch_misses", "mts_cache_writeback_evicted", "mts_cache_flush",
+    "mts_cache_prefetch_misses", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
     "mts_cache_export_state",
 )
 
@@ -93,7 +93,8 @@ def lib():
         L.mts_linearize_keys.argtypes = [vp, i32, i32, i32, vp, vp, i64, i64, vp, vp]
         L.mts_cache_workspace_bytes.restype = sz
         L.mts_cache_workspace_bytes.argtypes = [vp, i64]
-        L.mts_cache_lookup_insert.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
+        L.mts_cache_lookup_insert.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
+        L.mts_cache_refetch_overflowed.argtypes = [vp, vp, vp, i64, vp, vp]
         L.mts_cache_prefetch_misses.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.mts_cache_writeback_evicted.argtypes = [vp, vp, vp, vp, i64, vp, vp, vp]
         L.mts_cache_flush.argtypes = [vp, vp, vp]
@@ -282,11 +283,17 @@ def cache_workspace_bytes(cache: Cache, N: int) -> int:
 
 def cache_lookup_insert(cache: Cache, keys, N: int, step: int, slot_of_lookup, miss_keys, miss_slots, evict_keys,
                         evict_slots, evict_dirty, list_capacity: int, counters, workspace, workspace_bytes: int,
-                        stream=None) -> None:
+                        stream=None, overflow_keys=None) -> None:
     _check(lib().mts_cache_lookup_insert(cache.handle, _ptr(keys), N, step, _ptr(slot_of_lookup), _ptr(miss_keys),
                                          _ptr(miss_slots), _ptr(evict_keys), _ptr(evict_slots), _ptr(evict_dirty),
-                                         list_capacity, _ptr(counters), _ptr(workspace), workspace_bytes,
-                                         _stream(stream)))
+                                         _ptr(overflow_keys), list_capacity, _ptr(counters), _ptr(workspace),
+                                         workspace_bytes, _stream(stream)))
+
+
+def cache_refetch_overflowed(cache: Cache, host_rows_mapped, overflow_keys, list_capacity: int, counters,
+                             stream=None) -> None:
+    _check(lib().mts_cache_refetch_overflowed(cache.handle, _ptr(host_rows_mapped), _ptr(overflow_keys),
+                                              list_capacity, _ptr(counters), _stream(stream)))
 
 
 def cache_prefetch_misses(cache: Cache, host_rows_mapped, miss_keys, miss_slots, evict_slots, evict_dirty,

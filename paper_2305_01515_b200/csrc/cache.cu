@@ -47,9 +47,11 @@ __global__ void cache_init_state(uint32_t* tags, int32_t* ts, uint32_t* freq, ui
 }
 
 __global__ void cache_prepare_keys(const int64_t* __restrict__ keys, int64_t n, uint32_t* __restrict__ k32,
-                                   uint32_t* __restrict__ pos, int64_t* __restrict__ counters) {
+                                   uint32_t* __restrict__ pos, int64_t* __restrict__ counters,
+                                   uint32_t* __restrict__ overflow_cursor) {
   const int64_t i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i0 < MTS_NUM_COUNTERS) counters[i0] = i0 == MTS_CNT_LOOKUPS ? n : 0;
+  if (i0 == 0) *overflow_cursor = 0u;
   for (int64_t i = i0; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     k32[i] = (uint32_t)keys[i];
     pos[i] = (uint32_t)i;
@@ -291,7 +293,8 @@ cache_write_lists(const uint8_t* __restrict__ member_flag, const uint32_t* __res
                   const uint32_t* __restrict__ base_evict, int64_t capacity,
                   int64_t* __restrict__ miss_keys, int32_t* __restrict__ miss_slots,
                   int64_t* __restrict__ evict_keys, int32_t* __restrict__ evict_slots,
-                  uint8_t* __restrict__ evict_dirty) {
+                  uint8_t* __restrict__ evict_dirty, int64_t* __restrict__ overflow_keys,
+                  uint32_t* __restrict__ overflow_cursor) {
   __shared__ uint32_t sh[9];
   const int64_t n = *n_unique;
   const int64_t per = list_per_block(n, gridDim.x);
@@ -299,6 +302,11 @@ cache_write_lists(const uint8_t* __restrict__ member_flag, const uint32_t* __res
   uint32_t bm = base_miss[blockIdx.x], be = base_evict[blockIdx.x];
   for (int64_t t0 = begin; t0 < end; t0 += CACHE_THREADS) {
     const int64_t j = t0 + threadIdx.x;
+    if (overflow_keys != nullptr && j < end && member_flag[j] == 2) {
+      // the overflow list is a set: its order is not specified
+      const uint32_t at = atomicAdd(overflow_cursor, 1u);
+      if ((int64_t)at < capacity) overflow_keys[at] = (int64_t)ukey[member_uidx[j]];
+    }
     const bool placed = j < end && member_flag[j] == 1;
     const bool ev = placed && member_old_key[j] != FREE_TAG;
     uint32_t ta, tb;
@@ -471,6 +479,29 @@ cache_fetch_misses_bulk(char* __restrict__ data, int row_bytes, const char* __re
   }
 }
 
+// One warp per key of an overflow list: if the key is resident now, copy its host row into its
+// slot again (the copy made when it was placed may predate an update applied to the host row).
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_refetch_resident(char* __restrict__ data, int row_bytes, const char* __restrict__ host_rows,
+                       const int64_t* __restrict__ keys, const int64_t* __restrict__ counters, int64_t capacity,
+                       const uint32_t* __restrict__ tags, uint64_t S) {
+  const int64_t n = list_len(counters, MTS_CNT_OVERFLOW, capacity);
+  const int lane = threadIdx.x & 31;
+  const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t k = warp0; k < n; k += nwarps) {
+    const uint32_t key = (uint32_t)keys[k];
+    const int64_t slot0 = (int64_t)set_of_key(key, S) * 32;
+    const uint32_t hit = __ballot_sync(0xffffffffu, tags[slot0 + lane] == key);
+    if (hit) {
+      const char* src = host_rows + (int64_t)key * row_bytes;
+      char* dst = data + (slot0 + __ffs(hit) - 1) * row_bytes;
+      for (int c = lane * 16; c < row_bytes; c += 32 * 16)
+        *reinterpret_cast<uint4*>(dst + c) = *reinterpret_cast<const uint4*>(src + c);
+    }
+  }
+}
+
 __global__ void __launch_bounds__(CACHE_THREADS)
 cache_write_victims(char* __restrict__ host_rows, int row_bytes, const int64_t* __restrict__ evict_keys,
                     const uint8_t* __restrict__ evict_dirty, const int64_t* __restrict__ counters,
@@ -508,7 +539,7 @@ __global__ void cache_export(const uint32_t* __restrict__ tags, const int32_t* _
 struct CacheLayout {
   size_t keys_a, keys_b, vals_a, vals_b, uniq_idx, seg_start, ukey, mult, set_a, set_b, sval_a, sval_b,
       sseg_start, slot_of_uniq, member_flag, member_old_key, member_old_dirty, member_slot, hist, scan, cnt_miss,
-      cnt_evict, n_unique, n_sets, total;
+      cnt_evict, n_unique, n_sets, ovf_cursor, total;
 };
 
 static CacheLayout cache_layout(int64_t N) {
@@ -526,7 +557,7 @@ static CacheLayout cache_layout(int64_t N) {
   L.hist = take(sort_hist_words() * 4);
   L.scan = take(scan_scratch_words() * 4);
   L.cnt_miss = take(LIST_BLOCKS * 4); L.cnt_evict = take(LIST_BLOCKS * 4);
-  L.n_unique = take(256); L.n_sets = take(256);
+  L.n_unique = take(256); L.n_sets = take(256); L.ovf_cursor = take(256);
   L.total = off;
   return L;
 }
@@ -642,8 +673,8 @@ extern "C" size_t mts_cache_workspace_bytes(const mts_cache* c, int64_t N) {
 extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_t N, int64_t step,
                                        int32_t* slot_of_lookup, int64_t* miss_keys, int32_t* miss_slots,
                                        int64_t* evict_keys, int32_t* evict_slots, uint8_t* evict_dirty,
-                                       int64_t list_capacity, int64_t* counters, void* workspace,
-                                       size_t workspace_bytes, void* stream) {
+                                       int64_t* overflow_keys, int64_t list_capacity, int64_t* counters,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
   if (!c || !counters || N < 0 || list_capacity < 0 || step < 0 || step >= (1ll << 31) - 1)
     return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert: bad argument");
   if (N > 0 && (!keys || !slot_of_lookup))
@@ -662,7 +693,7 @@ extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_
   const int grid = c->sm_count * 8;
   {
     LaunchScope scope(K_CACHE_PREPARE, s);
-    cache_prepare_keys<<<grid, 256, 0, s>>>(keys, N, U32(L.keys_a), U32(L.vals_a), counters);
+    cache_prepare_keys<<<grid, 256, 0, s>>>(keys, N, U32(L.keys_a), U32(L.vals_a), counters, U32(L.ovf_cursor));
   }
   int rc = check_launch("cache_prepare_keys");
   if (rc != MTS_OK) return rc;
@@ -722,7 +753,7 @@ extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_
     cache_write_lists<<<G, CACHE_THREADS, 0, s>>>(member_flag, U32(L.member_old_key), member_old_dirty, member_slot, su,
                                                   U32(L.ukey), n_unique, U32(L.cnt_miss), U32(L.cnt_evict),
                                                   list_capacity, miss_keys, miss_slots, evict_keys, evict_slots,
-                                                  evict_dirty);
+                                                  evict_dirty, overflow_keys, U32(L.ovf_cursor));
   }
   {
     LaunchScope scope(K_CACHE_SCATTER_SLOTS, s);
@@ -778,6 +809,21 @@ extern "C" int mts_cache_writeback_evicted(mts_cache* c, void* host_rows_mapped,
         static_cast<const char*>(evict_staging));
   }
   return check_launch("cache_write_victims");
+}
+
+extern "C" int mts_cache_refetch_overflowed(mts_cache* c, const void* host_rows_mapped, const int64_t* overflow_keys,
+                                            int64_t list_capacity, const int64_t* counters, void* stream) {
+  if (!c || !host_rows_mapped || !counters || list_capacity < 0 || (list_capacity > 0 && !overflow_keys))
+    return set_error(MTS_ERR_INVALID_ARG, "cache_refetch_overflowed: null argument");
+  if ((uintptr_t)host_rows_mapped & 15) return set_error(MTS_ERR_ALIGNMENT, "cache_refetch_overflowed: host buffer alignment");
+  if (list_capacity == 0) return MTS_OK;
+  {
+    LaunchScope scope(K_CACHE_FETCH_MISSES, static_cast<cudaStream_t>(stream));
+    cache_refetch_resident<<<c->sm_count, CACHE_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
+        c->data, c->row_bytes, static_cast<const char*>(host_rows_mapped), overflow_keys, counters, list_capacity,
+        c->tags, (uint64_t)c->S);
+  }
+  return check_launch("cache_refetch_resident");
 }
 
 extern "C" int mts_cache_flush(mts_cache* c, void* host_rows_mapped, void* stream) {

@@ -79,15 +79,21 @@ class DeviceModel:
         self.cache_ws_bytes = max([mb.cache_workspace_bytes(c, max_lookups) for c in self.caches] + [256])
         self.cache_ws = torch.empty(self.cache_ws_bytes, dtype=torch.uint8, device=self.device)
         if self.cached:
-            # two batch contexts, so that the cache calls of batch t+1 can run while batch t trains
-            self.ctx = [self._new_context(max_lookups) for _ in range(2)]
+            # three batch contexts: batch t trains while the rows of batch t+1 move and the tags of
+            # batch t+2 are looked up; the victim staging buffer is only used inside one data
+            # movement call sequence, so one per cache serves all contexts
+            esz = 4 if self.spec.dtype == wl.FP32 else 2
+            self.staging = [torch.empty(min(max_lookups, c.num_sets * c.ways) * c.dim * esz, dtype=torch.uint8,
+                                        device=self.device) for c in self.caches]
+            self.ctx = [self._new_context(max_lookups) for _ in range(self.N_CTX)]
             self.cur = 0
+
+    N_CTX = 3
 
     def _new_context(self, n: int):
         dev = self.device
-        esz = 4 if self.spec.dtype == wl.FP32 else 2
         lists = []
-        for c in self.caches:
+        for g, c in enumerate(self.caches):
             cap = min(n, c.num_sets * c.ways)        # a call can place at most one row per slot
             lists.append(dict(
                 miss_keys=torch.empty(cap, dtype=torch.int64, device=dev),
@@ -95,8 +101,9 @@ class DeviceModel:
                 evict_keys=torch.empty(cap, dtype=torch.int64, device=dev),
                 evict_slots=torch.empty(cap, dtype=torch.int32, device=dev),
                 evict_dirty=torch.empty(cap, dtype=torch.uint8, device=dev),
+                overflow_keys=torch.empty(cap, dtype=torch.int64, device=dev),
                 counters=torch.zeros(mb.NUM_COUNTERS, dtype=torch.int64, device=dev),
-                staging=torch.empty(cap * c.dim * esz, dtype=torch.uint8, device=dev),
+                staging=self.staging[g],
                 capacity=cap))
         return dict(slot=torch.full((n,), -1, dtype=torch.int32, device=dev),
                     keys=torch.empty(n, dtype=torch.int64, device=dev), lists=lists)
@@ -156,7 +163,7 @@ class DeviceModel:
             mb.cache_lookup_insert(c, keys if n else None, n, step, cx["slot"][begin:begin + n] if n else None,
                                    L["miss_keys"], L["miss_slots"], L["evict_keys"], L["evict_slots"],
                                    L["evict_dirty"], L["capacity"], L["counters"], self.cache_ws, self.cache_ws_bytes,
-                                   stream)
+                                   stream, overflow_keys=L["overflow_keys"])
 
     def cache_move(self, stream=None, ctx: Optional[int] = None) -> None:
         """Data path of one batch: save dirty victims, pull missed rows from the host tier, write victims back."""
@@ -168,6 +175,14 @@ class DeviceModel:
                                      L["capacity"], L["counters"], L["staging"], stream)
             mb.cache_writeback_evicted(c, hp, L["evict_keys"], L["evict_dirty"], L["capacity"], L["counters"],
                                        L["staging"], stream)
+
+    def cache_refetch(self, prev_ctx: int, stream=None) -> None:
+        """After the backward of the batch in context `prev_ctx`: refresh rows that overflowed there
+        and were placed by the next batch."""
+        for g, c in enumerate(self.caches):
+            L = self.ctx[prev_ctx]["lists"][g]
+            mb.cache_refetch_overflowed(c, self.host_rows_ptr(g), L["overflow_keys"], L["capacity"], L["counters"],
+                                        stream)
 
     def cache_step(self, indices, offsets, offsets_host: np.ndarray, step: int, stream=None,
                    do_prefetch: bool = True, ctx: Optional[int] = None) -> None:

@@ -16,8 +16,10 @@ and the dirty bytes of its victims only; forward/backward write none of the firs
 dirty bytes of their own batch's slots.  The data movement of batch t+1 touches victim slots (trained
 at t-1 or earlier, complete because the tag step waited for backward(t-1)) and the slots of missed
 rows, which no batch in flight uses.  One hazard is left: a row that found no evictable way in batch
-t (it is read and updated in host memory directly) and is fetched from host memory for batch t+1.
-When batch t reported such overflow, the data movement of batch t+1 waits for backward(t).
+t (it is read and updated in host memory directly) and is fetched from host memory for batch t+1,
+possibly before backward(t) has updated it.  When batch t reported such overflow, the data movement
+of batch t+1 still runs at once, and after backward(t) the rows of batch t's overflow list that are
+resident by then are copied from host memory again (mts_cache_refetch_overflowed).
 """
 from __future__ import annotations
 
@@ -40,12 +42,13 @@ class CachedTrainer:
         self.tag = torch.cuda.Stream(self.dev) if pipelined else self.main
         self.move = torch.cuda.Stream(self.dev) if pipelined else self.main
         n_c = len(model.caches)
-        self.host_counters = [torch.zeros((n_c, mb.NUM_COUNTERS), dtype=torch.int64).pin_memory() for _ in range(2)]
+        self.host_counters = [torch.zeros((n_c, mb.NUM_COUNTERS), dtype=torch.int64).pin_memory()
+                              for _ in range(DeviceModel.N_CTX)]
         self.history: List[np.ndarray] = []           # per batch [n_caches, NUM_COUNTERS]
 
     def _lookup(self, t, step, batch, ev_tags, wait_event):
-        """Tag path of batch t on the tag stream (into context t mod 2)."""
-        m, s, ctx = self.m, self.tag, t & 1
+        """Tag path of batch t on the tag stream (into context t mod 3)."""
+        m, s, ctx = self.m, self.tag, t % DeviceModel.N_CTX
         if wait_event is not None:
             s.wait_event(wait_event)
         m.cache_lookup(batch[0], batch[1], batch[2], step, stream=s, ctx=ctx)
@@ -54,20 +57,29 @@ class CachedTrainer:
                 self.host_counters[ctx][g].copy_(m.ctx[ctx]["lists"][g]["counters"], non_blocking=True)
         ev_tags.record(s)
 
-    def _move(self, t, ev_tags, ev_ready, wait_event):
-        """Data path of batch t on the move stream."""
+    def _move(self, t, ev_tags, ev_ready, prev_overflow, prev_bwd):
+        """Data path of batch t on the move stream.  prev_overflow: number of rows of batch t-1 that
+        found no way (0 = none), prev_bwd: event after batch t-1's backward."""
         s = self.move
         s.wait_event(ev_tags)
-        if wait_event is not None:
-            s.wait_event(wait_event)
-        self.m.cache_move(stream=s, ctx=t & 1)
+        refetch = False
+        if prev_overflow:
+            cap = min(L["capacity"] for L in self.m.ctx[(t - 1) % DeviceModel.N_CTX]["lists"])
+            if prev_overflow <= cap:
+                refetch = True                       # move now, repair the few stale rows afterwards
+            else:
+                s.wait_event(prev_bwd)               # the list was cut: wait for the backward first
+        self.m.cache_move(stream=s, ctx=t % DeviceModel.N_CTX)
+        if refetch:
+            s.wait_event(prev_bwd)
+            self.m.cache_refetch((t - 1) % DeviceModel.N_CTX, stream=s)
         ev_ready.record(s)
 
-    def _counters(self, t, ev_tags) -> bool:
+    def _counters(self, t, ev_tags) -> int:
         ev_tags.synchronize()                        # counters of batch t are on the host
-        cnt = self.host_counters[t & 1].numpy().copy()
+        cnt = self.host_counters[t % DeviceModel.N_CTX].numpy().copy()
         self.history.append(cnt)
-        return bool(cnt[:, mb.COUNTER_NAMES.index("overflow")].sum() > 0)
+        return int(cnt[:, mb.COUNTER_NAMES.index("overflow")].max())
 
     def run(self, batches, grads, out: Optional[torch.Tensor] = None,
             on_step: Optional[Callable[[int], None]] = None, first_step: int = 0) -> None:
@@ -85,9 +97,9 @@ class CachedTrainer:
             for t in range(K):
                 idx, off, _ = batches[t]
                 self._lookup(t, first_step + t, batches[t], ev_tags[t], None)
-                self._move(t, ev_tags[t], ev_ready[t], None)
-                m.forward(idx, off, idx.numel(), out=out, stream=self.main, ctx=t & 1)
-                m.backward(idx, off, idx.numel(), grads[t], stream=self.main, ctx=t & 1)
+                self._move(t, ev_tags[t], ev_ready[t], 0, None)
+                m.forward(idx, off, idx.numel(), out=out, stream=self.main, ctx=t % DeviceModel.N_CTX)
+                m.backward(idx, off, idx.numel(), grads[t], stream=self.main, ctx=t % DeviceModel.N_CTX)
                 self._counters(t, ev_tags[t])
                 if on_step is not None:
                     on_step(t)
@@ -99,21 +111,21 @@ class CachedTrainer:
         self.move.wait_event(start)
         overflow = {}
         self._lookup(0, first_step, batches[0], ev_tags[0], None)
-        self._move(0, ev_tags[0], ev_ready[0], None)
+        self._move(0, ev_tags[0], ev_ready[0], 0, None)
         overflow[0] = self._counters(0, ev_tags[0])
         if K > 1:
             self._lookup(1, first_step + 1, batches[1], ev_tags[1], None)
         for t in range(K):
             idx, off, _ = batches[t]
             self.main.wait_event(ev_ready[t])
-            m.forward(idx, off, idx.numel(), out=out, stream=self.main, ctx=t & 1)
-            m.backward(idx, off, idx.numel(), grads[t], stream=self.main, ctx=t & 1)
+            m.forward(idx, off, idx.numel(), out=out, stream=self.main, ctx=t % DeviceModel.N_CTX)
+            m.backward(idx, off, idx.numel(), grads[t], stream=self.main, ctx=t % DeviceModel.N_CTX)
             ev_bwd[t].record(self.main)
             if t + 1 < K:
                 overflow[t + 1] = self._counters(t + 1, ev_tags[t + 1])
-                self._move(t + 1, ev_tags[t + 1], ev_ready[t + 1], ev_bwd[t] if overflow[t] else None)
+                self._move(t + 1, ev_tags[t + 1], ev_ready[t + 1], overflow[t], ev_bwd[t])
             if t + 2 < K:
-                # context (t+2) mod 2 is the one batch t is using: wait for its backward
+                # the tag step of batch t+2 may evict rows of batch t: wait for its backward
                 self._lookup(t + 2, first_step + t + 2, batches[t + 2], ev_tags[t + 2], ev_bwd[t])
             if on_step is not None:
                 on_step(t)

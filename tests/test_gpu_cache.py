@@ -23,6 +23,7 @@ class GpuCache:
         self.ek = torch.empty(cap, dtype=torch.int64, device=d); self.es = torch.empty(cap, dtype=torch.int32, device=d)
         self.ed = torch.empty(cap, dtype=torch.uint8, device=d)
         self.cnt = torch.empty(mb.NUM_COUNTERS, dtype=torch.int64, device=d)
+        self.ok = torch.empty(cap, dtype=torch.int64, device=d)
         self.wsb = mb.cache_workspace_bytes(self.c, cap)
         self.ws = torch.empty(self.wsb, dtype=torch.uint8, device=d)
         self.n = S * 32
@@ -30,10 +31,11 @@ class GpuCache:
     def lookup_insert(self, keys, step):
         N = len(keys)
         mb.cache_lookup_insert(self.c, to_dev(keys) if N else None, N, step, self.slot, self.mk, self.ms, self.ek,
-                               self.es, self.ed, self.cap, self.cnt, self.ws, self.wsb)
+                               self.es, self.ed, self.cap, self.cnt, self.ws, self.wsb, overflow_keys=self.ok)
         torch.cuda.synchronize()
         cnt = dict(zip(mb.COUNTER_NAMES, self.cnt.cpu().tolist()))
         nm, ne = cnt["inserted"], cnt["evicted"]
+        self.overflow_keys = np.sort(self.ok[:cnt["overflow"]].cpu().numpy())
         return dict(slot_of_lookup=self.slot[:N].cpu().numpy(), miss_keys=self.mk[:nm].cpu().numpy(),
                     miss_slots=self.ms[:nm].cpu().numpy(), evict_keys=self.ek[:ne].cpu().numpy(),
                     evict_slots=self.es[:ne].cpu().numpy(), evict_dirty=self.ed[:ne].cpu().numpy(), counters=cnt)
@@ -68,6 +70,7 @@ def test_tag_path_matches_oracle_bit_for_bit(S, lock, policy, universe):
         res = g.lookup_insert(keys, step)
         ref = o.lookup_insert(keys, step)
         _compare(res, ref)
+        np.testing.assert_array_equal(g.overflow_keys, np.unique(keys[ref["slot_of_lookup"] < 0]))
         # the backward pass would dirty the batch's slots: mark every second placed slot on both sides
         sl = np.unique(ref["slot_of_lookup"][ref["slot_of_lookup"] >= 0])[::2]
         if len(sl):
