@@ -501,8 +501,45 @@ def run_cached(args, rank: int, world: int, local_rank: int):
                      "frac": t_roof / t_meas, "traffic": None, "peak_source": peak_src},
         "clocks": clocks, "gpu_launches": int(launches), "e2e": None, "kernels": kernels,
     }
-    print(json.dumps(line), flush=True)
     model.close()
+    if getattr(args, "_collect", None) is not None:
+        args._collect.append(line)
+    else:
+        print(json.dumps(line), flush=True)
+
+
+def run_sweep(args, rank: int, world: int, local_rank: int):
+    """Configuration 5: one-factor sweeps around the centre point (batch 16K, pooling 50, Zipf 1.0,
+    cache 10%) plus the four extreme corners.  Prints one JSON line per point (hit rate, lookups/s,
+    roofline fraction); not the default bench line."""
+    import copy
+
+    centre = dict(batch=16384, pooling=50, alpha=1.0, cache_fraction=0.10)
+    points = [dict(centre)]
+    for b in (1024, 4096, 65536):
+        points.append(dict(centre, batch=b))
+    for L in (1, 10, 200):
+        points.append(dict(centre, pooling=L))
+    for a in (0.6, 0.8, 1.2, 1.4):
+        points.append(dict(centre, alpha=a))
+    for c in (0.01, 0.05, 0.25, 0.50):
+        points.append(dict(centre, cache_fraction=c))
+    points += [dict(batch=1024, pooling=1, alpha=0.6, cache_fraction=0.01),
+               dict(batch=65536, pooling=200, alpha=1.4, cache_fraction=0.50),
+               dict(batch=1024, pooling=200, alpha=1.4, cache_fraction=0.01),
+               dict(batch=65536, pooling=1, alpha=0.6, cache_fraction=0.50)]
+    for p in points:
+        a = copy.copy(args)
+        a.workload = "cfg5"
+        a.batch, a.pooling, a.alpha, a.cache_fraction = p["batch"], p["pooling"], p["alpha"], p["cache_fraction"]
+        a._collect = []
+        run_cached(a, rank, world, local_rank)
+        j = a._collect[0]
+        print(json.dumps({"point": p, "lookups_per_sec": j["value"], "ms_per_step": j["ms_per_step"],
+                          "hit_rate_per_lookup": j["hit_rate_per_lookup"], "unique_hit_rate": j["unique_hit_rate"],
+                          "overflow_rows": j["overflow_rows"], "roofline_frac": j["roofline"]["frac"],
+                          "bound": j["roofline"]["bound"], "miss_gb_per_step": j["host_link"]["miss_gb_per_step"],
+                          "achieved_h2d_gbs": j["host_link"]["achieved_h2d_gbs"]}), flush=True)
 
 
 def main():
@@ -535,6 +572,9 @@ def main():
         return
     if world == 1 and args.gpus > 1:
         raise SystemExit("launch with torch.distributed.run for --gpus > 1")
+    if args.workload == "cfg5-sweep":
+        run_sweep(args, rank, world, local_rank)
+        return
     if args.workload in ("cfg4", "cfg5"):
         if world > 1:
             raise SystemExit("cached workloads are single-GPU bench lines")

@@ -40,7 +40,8 @@ class CachedTrainer:
         self.dev = model.device
         self.main = torch.cuda.current_stream(self.dev)
         self.tag = torch.cuda.Stream(self.dev) if pipelined else self.main
-        self.move = torch.cuda.Stream(self.dev) if pipelined else self.main
+        # the data movement needs few thread blocks but must not queue behind the training kernels' blocks
+        self.move = torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main
         n_c = len(model.caches)
         self.host_counters = [torch.zeros((n_c, mb.NUM_COUNTERS), dtype=torch.int64).pin_memory()
                               for _ in range(DeviceModel.N_CTX)]

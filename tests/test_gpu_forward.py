@@ -93,3 +93,57 @@ def test_config2_full_size_sampled_bags():
         got = out[bs][:, spec.out_offset[t]:spec.out_offset[t + 1]]
         assert_close_mag(got, ref, mag, FWD_RTOL[spec.dtype], f"table {t}")
     m.close()
+
+
+def test_config3_full_size_sampled_bags_and_rows():
+    """Full configuration 3 (64 heterogeneous tables, 17 GB) as bench.py runs it: the oracle
+    recomputes a sample of bags (forward) and of rows (backward) from the counter-based weights."""
+    spec = wl.config3()
+    idx, off = wl.gen_batch(spec, 0)
+    grad = wl.gen_grad(spec, 0)
+    m = DeviceModel(spec)
+    d_idx, d_off = to_dev(idx), to_dev(off)
+    out = m.forward(d_idx, d_off, len(idx)).cpu().numpy()
+    m.backward(d_idx, d_off, len(idx), to_dev(grad))
+    torch.cuda.synchronize()
+    assert m.tables.status() == 0
+    rng = np.random.default_rng(3)
+    B = spec.batch
+    picked = [int(np.argmax(spec.dims == d)) for d in (64, 128, 256)] + [spec.T - 1]
+    for t in picked:
+        D = int(spec.dims[t])
+        # forward on 48 sampled bags
+        bs = np.sort(rng.choice(B, 48, replace=False))
+        rows_needed = np.unique(np.concatenate([idx[off[t * B + b]:off[t * B + b + 1]] for b in bs] + [np.zeros(1, np.int64)]))
+        Wsub = wl.weights_numpy(spec, t, rows_needed).reshape(-1)
+        sub_idx = np.concatenate([np.searchsorted(rows_needed, idx[off[t * B + b]:off[t * B + b + 1]]) for b in bs])
+        lens = np.array([off[t * B + b + 1] - off[t * B + b] for b in bs])
+        sub_off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+        ref, mag = oracle.tbe_forward(spec.dtype, [D], [0], [0], Wsub, len(bs), sub_idx, sub_off, 0, want_mag=True)
+        assert_close_mag(out[bs][:, spec.out_offset[t]:spec.out_offset[t + 1]], ref, mag, FWD_RTOL[spec.dtype], f"fwd table {t}")
+        # backward on sampled rows: the hottest, some touched once, some untouched
+        seg = idx[off[t * B]:off[(t + 1) * B]]
+        counts = np.bincount(seg, minlength=int(spec.rows[t]))
+        groups = [np.argsort(counts)[-2:]]
+        for sel in (counts == 1, counts > 1, counts == 0):
+            cand = np.nonzero(sel)[0]
+            if len(cand):
+                groups.append(rng.choice(cand, min(20, len(cand)), replace=False))
+        sample = np.unique(np.concatenate(groups))
+        keep = np.isin(seg, sample)
+        bag_of = np.repeat(np.arange(B), np.diff(off[t * B:(t + 1) * B + 1]))
+        sub_idx = np.searchsorted(sample, seg[keep])
+        sub_off = np.concatenate([[0], np.cumsum(np.bincount(bag_of[keep], minlength=B))]).astype(np.int64)
+        Wsub = wl.weights_numpy(spec, t, sample).reshape(-1)
+        W_before = Wsub.astype(np.float64)
+        msub = np.zeros(len(sample), np.float32)
+        smag = np.zeros(Wsub.size, np.float64)
+        g = np.ascontiguousarray(grad[:, spec.out_offset[t]:spec.out_offset[t + 1]])
+        oracle.tbe_backward_rowwise_adagrad(spec.dtype, [D], [0], [0], [0, len(sample)], Wsub, msub, B, sub_idx, sub_off,
+                                            g, spec.lr, spec.eps, step_mag=smag)
+        base = int(spec.weight_offset[t])
+        got_w = m.dev_weights[base:base + int(spec.rows[t]) * D].view(-1, D)[to_dev(sample)].cpu().numpy().reshape(-1)
+        got_m = m.momentum[int(spec.row_offset[t]) + to_dev(sample)].cpu().numpy()
+        assert_close_mag(got_w, Wsub, np.abs(W_before) + smag, FWD_RTOL[spec.dtype], f"bwd table {t} weights")
+        assert_close_mag(got_m, msub, msub, 1e-5, f"bwd table {t} momentum")
+    m.close()
