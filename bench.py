@@ -409,7 +409,7 @@ def run_cached(args, rank: int, world: int, local_rank: int):
                           cache_fraction=args.cache_fraction, n_batches=args.warmup + args.steps)
         spec.reuse_prob, spec.reuse_window = 0.0, 0
     t_setup = time.time()
-    model = DeviceModel(spec, device=dev, lock_depth=1)
+    model = DeviceModel(spec, device=dev, lock_depth=args.lock_depth)
     h2d_gbs, d2h_gbs = host_link_bandwidth(dev)
     stream = wl.BatchStream(spec)
     K = args.warmup + args.steps
@@ -486,7 +486,7 @@ def run_cached(args, rank: int, world: int, local_rank: int):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": spec.name, "note": spec.note, "tables": spec.T, "rows_total": int(spec.row_offset[-1]),
                    "host_weight_gb": spec.weight_bytes / 1e9, "cache_fraction": spec.cache_fraction, "batch": B,
-                   "lookups_per_step": lookups / args.steps, "schedule": "sequential" if args.sequential else "pipelined",
+                   "lookups_per_step": lookups / args.steps, "schedule": "sequential" if args.sequential else "pipelined", "lock_depth": args.lock_depth,
                    "l2": "inputs larger than L2 (host tier and caches are GBs)", "setup_seconds": setup_s},
         "samples_per_sec": B * args.steps / t_meas, "hit_rate_per_lookup": hit,
         "unique_hit_rate": float(hist[:, :, 4].sum()) / max(float(hist[:, :, 1].sum()), 1.0),
@@ -558,6 +558,8 @@ def main():
     ap.add_argument("--alpha", type=float, default=1.0, help="cfg5: Zipf exponent")
     ap.add_argument("--cache-fraction", type=float, default=0.10, help="cfg5: cache slots / rows")
     ap.add_argument("--sequential", action="store_true", help="cached workloads: no side stream")
+    ap.add_argument("--lock-depth", type=int, default=2,
+                    help="cached workloads: batches a stamped way stays unevictable (Section 5.7 invariant)")
     ap.add_argument("--trace", action="store_true",
                     help="cached workloads: CUDA events around every launch of the run (perturbs the timing)")
     ap.add_argument("--tables", type=int, default=0,

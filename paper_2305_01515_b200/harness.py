@@ -23,6 +23,7 @@ class DeviceModel:
     def __init__(self, spec: wl.ModelSpec, device="cuda:0", max_lookups: int = 0, weights: Optional[np.ndarray] = None,
                  lock_depth: int = 0, policy: int = mb.POLICY_LRU, cache_sets: Optional[List[int]] = None):
         self.spec = spec
+        self.lock_depth = lock_depth
         self.device = torch.device(device)
         self.tdtype = torch.float32 if spec.dtype == wl.FP32 else torch.float16
         n_elem = int(spec.weight_offset[-1])

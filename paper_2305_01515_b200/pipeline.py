@@ -9,9 +9,10 @@ lookups).  Three streams, ordered by events only:
 so the host-link traffic of the next batch and the tag work of the one after it overlap the
 training of the current batch.
 
-Why this is safe with lock_depth >= 1.  The tag step of batch t+2 waits for backward(t); it may only
-take ways stamped at t or earlier, i.e. rows whose batches have trained, and never a way of batch
-t+1 (stamped t+1), which is still waiting to train.  Its decisions read and write tags, timestamps
+Why this is safe with lock_depth >= 1.  The tag step of batch t+2 may only take ways stamped before
+t+2-lock_depth; it waits for the backward of the newest such batch (batch t for lock_depth 1, batch
+t-1 for lock_depth 2, which takes the tag step off the critical path), so it only evicts rows whose
+batches have trained, and never a way of a batch that is still waiting to train.  Its decisions read and write tags, timestamps
 and the dirty bytes of its victims only; forward/backward write none of the first two and only the
 dirty bytes of their own batch's slots.  The data movement of batch t+1 touches victim slots (trained
 at t-1 or earlier, complete because the tag step waited for backward(t-1)) and the slots of missed
@@ -39,20 +40,38 @@ class CachedTrainer:
         self.pipelined = pipelined
         self.dev = model.device
         self.main = torch.cuda.current_stream(self.dev)
-        self.tag = torch.cuda.Stream(self.dev) if pipelined else self.main
+        self.tag = torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main
         # the data movement needs few thread blocks but must not queue behind the training kernels' blocks
         self.move = torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main
         n_c = len(model.caches)
         self.host_counters = [torch.zeros((n_c, mb.NUM_COUNTERS), dtype=torch.int64).pin_memory()
                               for _ in range(DeviceModel.N_CTX)]
         self.history: List[np.ndarray] = []           # per batch [n_caches, NUM_COUNTERS]
+        self.record_timeline = False                  # set to True to time every phase with events
+        self._marks = []
+
+    def _mark(self, name, t, stream):
+        if self.record_timeline:
+            e = torch.cuda.Event(enable_timing=True)
+            e.record(stream)
+            self._marks.append((name, t, e))
+
+    def timeline(self):
+        """[(phase, batch, ms since the first mark)] after a run with record_timeline = True."""
+        if not self._marks:
+            return []
+        torch.cuda.synchronize(self.dev)
+        base = self._marks[0][2]
+        return [(n, t, base.elapsed_time(e)) for n, t, e in self._marks]
 
     def _lookup(self, t, step, batch, ev_tags, wait_event):
         """Tag path of batch t on the tag stream (into context t mod 3)."""
         m, s, ctx = self.m, self.tag, t % DeviceModel.N_CTX
         if wait_event is not None:
             s.wait_event(wait_event)
+        self._mark("tag_begin", t, s)
         m.cache_lookup(batch[0], batch[1], batch[2], step, stream=s, ctx=ctx)
+        self._mark("tag_end", t, s)
         with torch.cuda.stream(s):
             for g in range(len(m.caches)):
                 self.host_counters[ctx][g].copy_(m.ctx[ctx]["lists"][g]["counters"], non_blocking=True)
@@ -70,7 +89,9 @@ class CachedTrainer:
                 refetch = True                       # move now, repair the few stale rows afterwards
             else:
                 s.wait_event(prev_bwd)               # the list was cut: wait for the backward first
+        self._mark("move_begin", t, s)
         self.m.cache_move(stream=s, ctx=t % DeviceModel.N_CTX)
+        self._mark("move_end", t, s)
         if refetch:
             s.wait_event(prev_bwd)
             self.m.cache_refetch((t - 1) % DeviceModel.N_CTX, stream=s)
@@ -119,15 +140,22 @@ class CachedTrainer:
         for t in range(K):
             idx, off, _ = batches[t]
             self.main.wait_event(ev_ready[t])
+            self._mark("fwd_begin", t, self.main)
             m.forward(idx, off, idx.numel(), out=out, stream=self.main, ctx=t % DeviceModel.N_CTX)
+            self._mark("fwd_end", t, self.main)
             m.backward(idx, off, idx.numel(), grads[t], stream=self.main, ctx=t % DeviceModel.N_CTX)
+            self._mark("bwd_end", t, self.main)
             ev_bwd[t].record(self.main)
             if t + 1 < K:
                 overflow[t + 1] = self._counters(t + 1, ev_tags[t + 1])
                 self._move(t + 1, ev_tags[t + 1], ev_ready[t + 1], overflow[t], ev_bwd[t])
             if t + 2 < K:
-                # the tag step of batch t+2 may evict rows of batch t: wait for its backward
-                self._lookup(t + 2, first_step + t + 2, batches[t + 2], ev_tags[t + 2], ev_bwd[t])
+                # the tag step of batch t+2 may evict rows stamped before t+2-lock_depth: the backward
+                # of the last such batch must be over (with lock_depth 1 that is batch t, with 2 batch
+                # t-1); the context it writes was last used by batch t-1
+                last = min(t, t + 1 - m.lock_depth)
+                self._lookup(t + 2, first_step + t + 2, batches[t + 2], ev_tags[t + 2],
+                             ev_bwd[last] if last >= 0 else None)
             if on_step is not None:
                 on_step(t)
         self.main.wait_stream(self.tag)

@@ -16,8 +16,9 @@ from helpers import custom_spec, to_dev
 pytestmark = pytest.mark.gpu
 
 
+@pytest.mark.parametrize("lock", [1, 2])
 @pytest.mark.parametrize("frac", [0.2, 0.004])       # roomy cache; cache smaller than a batch (overflow path)
-def test_pipelined_equals_sequential_and_oracle_tags(frac):
+def test_pipelined_equals_sequential_and_oracle_tags(frac, lock):
     rows, dims = [20000, 9000, 4000, 12000], [64, 64, 128, 128]
     spec = custom_spec(rows, dims, 256, wl.FP16, [8, 12, 20, 5], [1.05, 0.9, 1.2, 1.0], seed=77)
     spec.cached = True
@@ -30,7 +31,7 @@ def test_pipelined_equals_sequential_and_oracle_tags(frac):
     W0 = wl.all_weights_numpy(spec)
     results = []
     for pipelined in (False, True):
-        m = DeviceModel(spec, weights=W0, lock_depth=1)
+        m = DeviceModel(spec, weights=W0, lock_depth=lock)
         m.reserve(max(len(b[0]) for b in host_batches))
         batches = [(to_dev(i), to_dev(o), o) for i, o in host_batches]
         tr = CachedTrainer(m, pipelined=pipelined)
@@ -49,7 +50,7 @@ def test_pipelined_equals_sequential_and_oracle_tags(frac):
     overflow = 0
     for g, (dim, t0, t1) in enumerate(groups):
         rows_g = int(spec.row_offset[t1] - spec.row_offset[t0])
-        oc = oracle.Cache(wl.cache_sets_for(rows_g, frac), 32, dim, spec.dtype, 0, 1, with_data=False)
+        oc = oracle.Cache(wl.cache_sets_for(rows_g, frac), 32, dim, spec.dtype, 0, lock, with_data=False)
         for k, (idx, off) in enumerate(host_batches):
             keys = np.concatenate([spec.row_offset[t] - spec.row_offset[t0] + idx[off[t * B]:off[(t + 1) * B]]
                                    for t in range(t0, t1)])
