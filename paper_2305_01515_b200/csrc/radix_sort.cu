@@ -109,7 +109,10 @@ scan_histogram(uint32_t* __restrict__ hist, uint32_t* __restrict__ totals, int G
   if (threadIdx.x == 0) totals[blockIdx.x] = total;
 }
 
-__global__ void __launch_bounds__(SORT_THREADS)
+#ifndef MTS_SORT_MINBLK
+#define MTS_SORT_MINBLK 3
+#endif
+__global__ void __launch_bounds__(SORT_THREADS, MTS_SORT_MINBLK)
 scatter_by_digit(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
                  uint32_t* __restrict__ keys_out, uint32_t* __restrict__ vals_out, int64_t n_max,
                  const uint32_t* __restrict__ n_dev, int shift, uint32_t mask,
