@@ -292,6 +292,48 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
   }
 }
 
+// Rows with very many lookups span hundreds of chunks.  One warp per aligned group of
+// COMBINE_GROUP consecutive chunks: when every chunk of the group starts inside one row that began
+// before the group, the group's head partials are added up (in chunk order) into one partial, so
+// that the owner of the row adds one vector per group instead of COMBINE_GROUP.
+constexpr int COMBINE_GROUP = 32;
+
+template <int NV>
+__global__ void __launch_bounds__(BWD_WARPS * 32)
+combine_groups(const uint32_t* __restrict__ keys, int64_t n, const float* __restrict__ partial_head,
+               float* __restrict__ partial_group) {
+  constexpr int PSTRIDE = NV * 128;
+  const int lane = threadIdx.x & 31;
+  const int64_t grp = (int64_t)blockIdx.x * BWD_WARPS + (threadIdx.x >> 5);
+  const int64_t c0 = grp * COMBINE_GROUP;
+  const int64_t p0 = c0 * BWD_CHUNK;
+  if (p0 == 0 || p0 + (int64_t)(COMBINE_GROUP - 1) * BWD_CHUNK >= n) return;
+  const uint32_t key = keys[p0 - 1];
+  // the last chunk of the group still starts inside the row <=> all of them do (keys ascend)
+  if (keys[p0 + (int64_t)(COMBINE_GROUP - 1) * BWD_CHUNK] != key) return;
+  float4 acc[NV];
+#pragma unroll
+  for (int q = 0; q < NV; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+  constexpr int U = 4;
+  for (int c = 0; c < COMBINE_GROUP; c += U) {
+    float4 v[U][NV];
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+      for (int q = 0; q < NV; ++q)
+        v[u][q] = *reinterpret_cast<const float4*>(partial_head + (c0 + c + u) * PSTRIDE + (q * 32 + lane) * 4);
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+      for (int q = 0; q < NV; ++q) {
+        acc[q].x += v[u][q].x; acc[q].y += v[u][q].y; acc[q].z += v[u][q].z; acc[q].w += v[u][q].w;
+      }
+  }
+#pragma unroll
+  for (int q = 0; q < NV; ++q)
+    *reinterpret_cast<float4*>(partial_group + grp * PSTRIDE + (q * 32 + lane) * 4) = acc[q];
+}
+
 // One warp per chunk.  The chunk owns a row iff the row's lookups start in it and run past
 // its end; the owner adds tail[c] + head[c+1] + ... in chunk order and applies the update.
 template <bool FP16, int NV>
@@ -300,7 +342,7 @@ combine_partials(const TableMeta* __restrict__ meta, int T, const uint32_t* __re
                  const uint32_t* __restrict__ pos, int64_t n, float lr, float eps,
                  const int32_t* __restrict__ slot_of_lookup, CachePtrs caches, char* dev_w, char* host_w,
                  float* __restrict__ momentum, const float* __restrict__ partial_head,
-                 const float* __restrict__ partial_tail) {
+                 const float* __restrict__ partial_tail, const float* __restrict__ partial_group) {
   constexpr int EB = FP16 ? 2 : 4;
   constexpr int PSTRIDE = NV * 128;
   const int lane = threadIdx.x & 31;
@@ -326,24 +368,44 @@ combine_partials(const TableMeta* __restrict__ meta, int T, const uint32_t* __re
 #pragma unroll
   for (int q = 0; q < NV; ++q)
     acc[q] = *reinterpret_cast<const float4*>(partial_tail + chunk * PSTRIDE + (q * 32 + lane) * 4);
+  // chunks chunk+1 .. chunk+nc carry the row's pieces; whole aligned groups of them were added up
+  // by combine_groups.  The order (single chunks up to the first group border, groups, single
+  // chunks again) depends only on the chunk numbers.
   constexpr int U = 4;
-  for (int64_t c = 1; c <= nc; c += U) {
-    float4 v[U][NV];
+  int64_t c = chunk + 1;
+  const int64_t c_end = chunk + nc;            // inclusive
+  while (c <= c_end) {
+    if ((c % COMBINE_GROUP) == 0 && c + COMBINE_GROUP - 1 <= c_end) {
+      const int64_t grp = c / COMBINE_GROUP;
 #pragma unroll
-    for (int u = 0; u < U; ++u)
-#pragma unroll
-      for (int q = 0; q < NV; ++q)
-        v[u][q] = (c + u <= nc)
-                      ? *reinterpret_cast<const float4*>(partial_head + (chunk + c + u) * PSTRIDE + (q * 32 + lane) * 4)
-                      : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-    for (int u = 0; u < U; ++u)
-      if (c + u <= nc) {
-#pragma unroll
-        for (int q = 0; q < NV; ++q) {
-          acc[q].x += v[u][q].x; acc[q].y += v[u][q].y; acc[q].z += v[u][q].z; acc[q].w += v[u][q].w;
-        }
+      for (int q = 0; q < NV; ++q) {
+        const float4 v = *reinterpret_cast<const float4*>(partial_group + grp * PSTRIDE + (q * 32 + lane) * 4);
+        acc[q].x += v.x; acc[q].y += v.y; acc[q].z += v.z; acc[q].w += v.w;
       }
+      c += COMBINE_GROUP;
+      continue;
+    }
+    // single chunks up to the next group border (or the end), U loads in flight
+    const int64_t stop = min(c_end, (c / COMBINE_GROUP + 1) * COMBINE_GROUP - 1);
+    for (; c <= stop; c += U) {
+      float4 v[U][NV];
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+#pragma unroll
+        for (int q = 0; q < NV; ++q)
+          v[u][q] = (c + u <= stop)
+                        ? *reinterpret_cast<const float4*>(partial_head + (c + u) * PSTRIDE + (q * 32 + lane) * 4)
+                        : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+        if (c + u <= stop) {
+#pragma unroll
+          for (int q = 0; q < NV; ++q) {
+            acc[q].x += v[u][q].x; acc[q].y += v[u][q].y; acc[q].z += v[u][q].z; acc[q].w += v[u][q].w;
+          }
+        }
+    }
+    c = stop + 1;
   }
   const int t = table_of_key(meta, T, (int64_t)key);
   const TableMeta m = meta[t];
@@ -363,7 +425,7 @@ __global__ void export_unique(const uint32_t* __restrict__ keys, const uint32_t*
 }
 
 struct BwdLayout {
-  size_t keys_a, keys_b, vals_a, vals_b, bag_of_pos, hist, scan, seg_start, n_unique, head, tail, total;
+  size_t keys_a, keys_b, vals_a, vals_b, bag_of_pos, hist, scan, seg_start, n_unique, head, tail, group, total;
 };
 
 static BwdLayout bwd_layout(const mts_tables* h, int64_t N) {
@@ -382,6 +444,7 @@ static BwdLayout bwd_layout(const mts_tables* h, int64_t N) {
   const size_t chunks = (size_t)ceil_div((int64_t)n, BWD_CHUNK);
   L.head = take(chunks * nvp * 128 * 4);
   L.tail = take(chunks * nvp * 128 * 4);
+  L.group = take((chunks / COMBINE_GROUP + 1) * nvp * 128 * 4);
   L.total = off;
   return L;
 }
@@ -391,7 +454,7 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
                            const uint32_t* bag_of_pos, int64_t N, const int64_t* offsets, int32_t pooling_mode,
                            const float* grad, int64_t grad_stride, float lr, float eps,
                            const int32_t* slot_of_lookup, const CachePtrs& caches, float* head, float* tail,
-                           cudaStream_t s) {
+                           float* group, cudaStream_t s) {
   const int64_t chunks = ceil_div(N, BWD_CHUNK);
   const unsigned grid = (unsigned)ceil_div(chunks, BWD_WARPS);
   {
@@ -405,11 +468,16 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
           h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
           static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail);
   }
+  if (chunks >= 2 * COMBINE_GROUP) {
+    LaunchScope scope(K_COMBINE_PARTIALS, s);
+    combine_groups<NV><<<(unsigned)ceil_div(ceil_div(chunks, COMBINE_GROUP), BWD_WARPS), BWD_WARPS * 32, 0, s>>>(
+        keys, N, head, group);
+  }
   {
     LaunchScope scope(K_COMBINE_PARTIALS, s);
     combine_partials<FP16, NV><<<grid, BWD_WARPS * 32, 0, s>>>(
         h->d_meta, h->T, keys, pos, N, lr, eps, slot_of_lookup, caches, static_cast<char*>(h->dev_weights),
-        static_cast<char*>(h->host_weights), h->momentum, head, tail);
+        static_cast<char*>(h->host_weights), h->momentum, head, tail, group);
   }
   return check_launch("reduce_chunks / combine_partials");
 }
@@ -492,9 +560,10 @@ extern "C" int mts_tbe_backward_rowwise_adagrad(
   }
   float* head = reinterpret_cast<float*>(ws + L.head);
   float* tail = reinterpret_cast<float*>(ws + L.tail);
+  float* group = reinterpret_cast<float*>(ws + L.group);
   const int nv = (h->max_dim + 127) / 128;
   const bool fp16 = h->dtype == MTS_DTYPE_FP16;
-#define MTS_BWD(F, V, G) return launch_backward<F, V, G>(h, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad_out, grad_stride, lr, eps, slot_of_lookup, caches, head, tail, s)
+#define MTS_BWD(F, V, G) return launch_backward<F, V, G>(h, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad_out, grad_stride, lr, eps, slot_of_lookup, caches, head, tail, group, s)
   if (fp16) {
     if (nv <= 1) MTS_BWD(true, 1, MTS_BWD_GROUP1);
     if (nv <= 2) MTS_BWD(true, 2, 4);
