@@ -1,5 +1,5 @@
 // Pooled multi-table embedding lookup (Section 2.1.1 of the paper: an embedding operator
-// selects rows of a table and pools them).  One warp per bag (table t, sample b); a row of
+// selects rows of a table and pools them).  One warp per bag (table t, sample b) at a time; a row of
 // vec16 16-byte chunks is read by a group of G = pow2(vec16) lanes, so 32 / G rows are in
 // flight per load instruction and UNROLL of those instructions are issued back to back.
 // Accumulation in fp32 registers, one 16-byte store per lane group member at the end.
@@ -7,11 +7,25 @@
 
 namespace mts {
 
+#ifndef MTS_FWD_UNROLL
+#define MTS_FWD_UNROLL 4         // load instructions issued back to back per lane
+#endif
+#ifndef MTS_FWD_MINBLK
+#define MTS_FWD_MINBLK 4         // resident blocks per SM the register allocation is bounded for
+#endif
+#ifndef MTS_FWD_BAGS
+#define MTS_FWD_BAGS 4           // consecutive bags one warp walks through
+#endif
 constexpr int FWD_WARPS = 8;
-constexpr int FWD_UNROLL = 4;
+constexpr int FWD_UNROLL = MTS_FWD_UNROLL;
+constexpr int FWD_BAGS = MTS_FWD_BAGS;
+static_assert(FWD_BAGS >= 1 && FWD_BAGS <= 30, "a warp keeps the offsets of its bags in its lanes");
 
+// A warp walks FWD_BAGS consecutive bags.  Their offsets are read with one load, and the first 32
+// indices of the next bag are requested before the rows of the current bag, so that a bag costs
+// about one memory round trip (its rows) instead of three (offsets, indices, rows).
 template <bool FP16, int NV>
-__global__ void __launch_bounds__(FWD_WARPS * 32)
+__global__ void __launch_bounds__(FWD_WARPS * 32, (NV == 1 ? MTS_FWD_MINBLK : 1))
 tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B,
                    const int64_t* __restrict__ indices, const int64_t* __restrict__ offsets,
                    const int32_t* __restrict__ slot_of_lookup, CachePtrs caches,
@@ -21,84 +35,114 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
   constexpr int EPC = FP16 ? 8 : 4;       // elements per 16-byte chunk
   constexpr int EB = FP16 ? 2 : 4;
   const int lane = threadIdx.x & 31;
-  const int64_t bag = (int64_t)blockIdx.x * FWD_WARPS + (threadIdx.x >> 5);
-  if (bag >= n_bags) return;
-  const int32_t t = (int32_t)(bag / B);
-  const int32_t b = (int32_t)(bag - (int64_t)t * B);
-  const TableMeta m = meta[t];
-  const int vec16 = m.vec16;
-  // lanes per row: smallest power of two >= vec16, at most 32
-  int logG = 0;
-  while ((1 << logG) < vec16 && logG < 5) ++logG;
-  const int G = 1 << logG;
-  const int R = 32 >> logG;               // rows per load instruction
-  const int sub = lane >> logG;
-  const int cl = lane & (G - 1);
-  const int64_t i0 = offsets[bag], i1 = offsets[bag + 1];
-  const int64_t row_bytes = (int64_t)m.dim * EB;
-  const char* table_base = (m.cache_id < 0 ? dev_w : host_w) + m.weight_offset * EB;
-  const char* cache_base = m.cache_id >= 0 ? static_cast<const char*>(caches.data[m.cache_id]) : nullptr;
-
-  float acc[NV][EPC];
-#pragma unroll
-  for (int v = 0; v < NV; ++v)
-#pragma unroll
-    for (int k = 0; k < EPC; ++k) acc[v][k] = 0.f;
-
-  for (int64_t base = i0; base < i1; base += 32) {
-    const int cnt = (int)min((int64_t)32, i1 - base);
-    const char* my_ptr = table_base;
-    if (lane < cnt) {
-      int64_t idx = clamp_index(indices[base + lane], m.rows, status);
-      my_ptr = table_base + idx * row_bytes;
-      if (cache_base != nullptr) {
-        int32_t s = slot_of_lookup[base + lane];
-        if (s >= 0) my_ptr = cache_base + (int64_t)s * row_bytes;
-      }
-    }
-    for (int r = 0; r < cnt; r += R * FWD_UNROLL) {
-      uint4 v[FWD_UNROLL][NV];
-#pragma unroll
-      for (int u = 0; u < FWD_UNROLL; ++u) {
-        const int j = r + u * R + sub;
-        const unsigned long long p =
-            __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_ptr, j & 31);
-        const bool valid = j < cnt;
-#pragma unroll
-        for (int q = 0; q < NV; ++q) {
-          const int c = cl + q * 32;
-          if (valid && c < vec16) v[u][q] = ld_nc_16(reinterpret_cast<const char*>(p) + (int64_t)c * 16);
-          else v[u][q] = make_uint4(0u, 0u, 0u, 0u);
-        }
-      }
-#pragma unroll
-      for (int u = 0; u < FWD_UNROLL; ++u)
-#pragma unroll
-        for (int q = 0; q < NV; ++q) {
-          if (FP16) add_half8(acc[q], v[u][q]);
-          else add_float4(acc[q], v[u][q]);
-        }
+  const int64_t bag0 = ((int64_t)blockIdx.x * FWD_WARPS + (threadIdx.x >> 5)) * FWD_BAGS;
+  if (bag0 >= n_bags) return;
+  const int nb = (int)min((int64_t)FWD_BAGS, n_bags - bag0);
+  // lane k holds the start of bag k of this warp, lane nb the end of the last one
+  const int64_t my_off = offsets[bag0 + min(lane, nb)];
+  int64_t i1 = __shfl_sync(0xffffffffu, my_off, 0);
+  // first indices (and cache slots) of the first bag
+  int64_t pf_idx = 0;
+  int32_t pf_slot = -1;
+  {
+    const int64_t e = __shfl_sync(0xffffffffu, my_off, 1);
+    if (i1 + lane < e) {
+      pf_idx = indices[i1 + lane];
+      if (meta[bag0 / B].cache_id >= 0) pf_slot = slot_of_lookup[i1 + lane];
     }
   }
-  // fold the row groups of the warp together
-  for (int o = G; o < 32; o <<= 1) {
+
+  for (int k = 0; k < nb; ++k) {
+    const int64_t bag = bag0 + k;
+    const int32_t t = (int32_t)(bag / B);
+    const int32_t b = (int32_t)(bag - (int64_t)t * B);
+    const TableMeta m = meta[t];
+    const int vec16 = m.vec16;
+    // lanes per row: smallest power of two >= vec16, at most 32
+    int logG = 0;
+    while ((1 << logG) < vec16 && logG < 5) ++logG;
+    const int G = 1 << logG;
+    const int R = 32 >> logG;               // rows per load instruction
+    const int sub = lane >> logG;
+    const int cl = lane & (G - 1);
+    const int64_t i0 = i1;
+    i1 = __shfl_sync(0xffffffffu, my_off, k + 1);
+    const int64_t row_bytes = (int64_t)m.dim * EB;
+    const char* table_base = (m.cache_id < 0 ? dev_w : host_w) + m.weight_offset * EB;
+    const char* cache_base = m.cache_id >= 0 ? static_cast<const char*>(caches.data[m.cache_id]) : nullptr;
+    const int64_t cur_idx = pf_idx;
+    const int32_t cur_slot = pf_slot;
+    if (k + 1 < nb) {
+      const int64_t e = __shfl_sync(0xffffffffu, my_off, k + 2);
+      pf_slot = -1;
+      if (i1 + lane < e) {
+        pf_idx = indices[i1 + lane];
+        if (meta[(bag + 1) / B].cache_id >= 0) pf_slot = slot_of_lookup[i1 + lane];
+      }
+    }
+
+    float acc[NV][EPC];
 #pragma unroll
-    for (int q = 0; q < NV; ++q)
+    for (int v = 0; v < NV; ++v)
 #pragma unroll
-      for (int k = 0; k < EPC; ++k) acc[q][k] += __shfl_xor_sync(0xffffffffu, acc[q][k], o);
-  }
-  if (sub == 0) {
-    float scale = 1.f;
-    if (pooling_mode == MTS_POOL_MEAN && i1 > i0) scale = 1.f / (float)(i1 - i0);
-    float* o = out + (int64_t)b * out_stride + m.out_offset;
+      for (int e = 0; e < EPC; ++e) acc[v][e] = 0.f;
+
+    for (int64_t base = i0; base < i1; base += 32) {
+      const int cnt = (int)min((int64_t)32, i1 - base);
+      const char* my_ptr = table_base;
+      if (lane < cnt) {
+        const bool first = base == i0;
+        const int64_t idx = clamp_index(first ? cur_idx : indices[base + lane], m.rows, status);
+        my_ptr = table_base + idx * row_bytes;
+        if (cache_base != nullptr) {
+          const int32_t s = first ? cur_slot : slot_of_lookup[base + lane];
+          if (s >= 0) my_ptr = cache_base + (int64_t)s * row_bytes;
+        }
+      }
+      for (int r = 0; r < cnt; r += R * FWD_UNROLL) {
+        uint4 v[FWD_UNROLL][NV];
 #pragma unroll
-    for (int q = 0; q < NV; ++q) {
-      const int c = cl + q * 32;
-      if (c < vec16) {
-        float4* dst = reinterpret_cast<float4*>(o + c * EPC);
-        dst[0] = make_float4(acc[q][0] * scale, acc[q][1] * scale, acc[q][2] * scale, acc[q][3] * scale);
-        if (FP16)
-          dst[1] = make_float4(acc[q][4] * scale, acc[q][5] * scale, acc[q][6] * scale, acc[q][7] * scale);
+        for (int u = 0; u < FWD_UNROLL; ++u) {
+          const int j = r + u * R + sub;
+          const unsigned long long p =
+              __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_ptr, j & 31);
+          const bool valid = j < cnt;
+#pragma unroll
+          for (int q = 0; q < NV; ++q) {
+            const int c = cl + q * 32;
+            if (valid && c < vec16) v[u][q] = ld_nc_16(reinterpret_cast<const char*>(p) + (int64_t)c * 16);
+            else v[u][q] = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < FWD_UNROLL; ++u)
+#pragma unroll
+          for (int q = 0; q < NV; ++q) {
+            if (FP16) add_half8(acc[q], v[u][q]);
+            else add_float4(acc[q], v[u][q]);
+          }
+      }
+    }
+    // fold the row groups of the warp together
+    for (int o = G; o < 32; o <<= 1) {
+#pragma unroll
+      for (int q = 0; q < NV; ++q)
+#pragma unroll
+        for (int e = 0; e < EPC; ++e) acc[q][e] += __shfl_xor_sync(0xffffffffu, acc[q][e], o);
+    }
+    if (sub == 0) {
+      float scale = 1.f;
+      if (pooling_mode == MTS_POOL_MEAN && i1 > i0) scale = 1.f / (float)(i1 - i0);
+      float* o = out + (int64_t)b * out_stride + m.out_offset;
+#pragma unroll
+      for (int q = 0; q < NV; ++q) {
+        const int c = cl + q * 32;
+        if (c < vec16) {
+          float4* dst = reinterpret_cast<float4*>(o + c * EPC);
+          dst[0] = make_float4(acc[q][0] * scale, acc[q][1] * scale, acc[q][2] * scale, acc[q][3] * scale);
+          if (FP16)
+            dst[1] = make_float4(acc[q][4] * scale, acc[q][5] * scale, acc[q][6] * scale, acc[q][7] * scale);
+        }
       }
     }
   }
@@ -109,7 +153,7 @@ static int launch_forward(const mts_tables* h, int32_t B, const int64_t* indices
                           int32_t pooling_mode, const int32_t* slot_of_lookup, const CachePtrs& caches,
                           float* out, int64_t out_stride, cudaStream_t stream) {
   const int64_t n_bags = (int64_t)h->T * B;
-  const int64_t grid = ceil_div(n_bags, FWD_WARPS);
+  const int64_t grid = ceil_div(n_bags, (int64_t)FWD_WARPS * FWD_BAGS);
   {
     LaunchScope scope(K_FORWARD, stream);
     tbe_forward_kernel<FP16, NV><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
