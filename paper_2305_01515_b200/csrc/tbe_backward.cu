@@ -25,11 +25,27 @@ namespace mts {
 #ifndef MTS_BWD_GROUP1
 #define MTS_BWD_GROUP1 4        // lookups whose loads are issued together when a row fits one warp pass
 #endif
+#ifndef MTS_BWD_USE_LEAN
+#define MTS_BWD_USE_LEAN 1      // rows of up to 128 columns take reduce_chunks_lean
+#endif
+#ifndef MTS_BWD_LEAN_WARPS
+#define MTS_BWD_LEAN_WARPS 4
+#endif
+#ifndef MTS_BWD_LEAN_MINBLK
+#define MTS_BWD_LEAN_MINBLK 16  // resident blocks per SM reduce_chunks_lean is bounded for (32 registers)
+#endif
+#ifndef MTS_BWD_GROUP2
+#define MTS_BWD_GROUP2 1        // the same for rows of 129..256 columns
+#endif
+#ifndef MTS_BWD_MINBLK2
+#define MTS_BWD_MINBLK2 10      // resident blocks per SM for those rows
+#endif
 #ifndef MTS_BWD_MINBLK
 #define MTS_BWD_MINBLK 8        // resident blocks per SM the register allocation is bounded for
 #endif
 constexpr int BWD_CHUNK = MTS_BWD_CHUNK;
 constexpr int BWD_WARPS = 4;
+constexpr int LEAN_WARPS = MTS_BWD_LEAN_WARPS;   // warps per block of reduce_chunks_lean
 constexpr int LIN_GROUP = 8;     // lanes per bag in linearize_lookups
 
 __global__ void __launch_bounds__(256)
@@ -90,19 +106,23 @@ __device__ __forceinline__ RowTarget row_target(const TableMeta& m, int64_t key,
 }
 
 // Row-wise Adagrad on one row held across the warp: lane owns columns (q*32 + lane)*4 .. +3.
-// m += mean(g^2); W -= lr * g / (sqrt(m) + eps).
+// m += mean(g^2); W -= lr * g / (sqrt(m) + eps).  inv_dim = __frcp_rn(dim), hoisted by the callers.
 template <bool FP16, int NV>
 __device__ __forceinline__ void adagrad_row(const float4 (&g)[NV], const uint4 (&wraw)[NV], float m_old,
-                                            int dim, float lr, float eps, char* wptr, float* mom_ptr,
-                                            uint8_t* dirty) {
+                                            int dim, float inv_dim, float lr, float eps, char* wptr,
+                                            float* mom_ptr, uint8_t* dirty) {
   const int lane = threadIdx.x & 31;
   float sq = 0.f;
 #pragma unroll
   for (int q = 0; q < NV; ++q) sq += g[q].x * g[q].x + g[q].y * g[q].y + g[q].z * g[q].z + g[q].w * g[q].w;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-  const float m_new = m_old + sq * __frcp_rn((float)dim);
-  const float step = __fdividef(lr, __fsqrt_rn(m_new) + eps);
+  const float m_new = m_old + sq * inv_dim;
+  // approximate square root and division: their relative error (a few 2^-23) only scales the
+  // step, far inside the tolerance of the update; the state m itself is exact fp32 arithmetic
+  float root;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(root) : "f"(m_new));
+  const float step = __fdividef(lr, root + eps);
 #pragma unroll
   for (int q = 0; q < NV; ++q) {
     const int d = (q * 32 + lane) * 4;
@@ -153,13 +173,14 @@ __device__ __forceinline__ void load_row(uint4 (&wraw)[NV], const char* wptr, in
 // loads of a whole group (gradient slices, and row + Adagrad state where a row ends) are issued
 // before the first one is used.
 template <bool FP16, int NV, int GROUP, bool MEAN>
-__global__ void __launch_bounds__(BWD_WARPS * 32, (NV == 1 ? MTS_BWD_MINBLK : 1))
+__global__ void __launch_bounds__(BWD_WARPS * 32, (NV == 1 ? MTS_BWD_MINBLK : NV == 2 ? MTS_BWD_MINBLK2 : 1))
 reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
               const uint32_t* __restrict__ keys, const uint32_t* __restrict__ pos,
               const uint32_t* __restrict__ bag_of_pos, int64_t n,
               const int64_t* __restrict__ offsets,
               const float* __restrict__ grad, int64_t grad_stride, float lr, float eps,
-              const int32_t* __restrict__ slot_of_lookup, CachePtrs caches, char* dev_w, char* host_w,
+              const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches, char* dev_w,
+                   char* host_w,
               float* __restrict__ momentum, float* __restrict__ partial_head,
               float* __restrict__ partial_tail) {
   constexpr int EB = FP16 ? 2 : 4;
@@ -272,7 +293,7 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
               const uint4 d = s_desc[wib][j];
               const int dim = uniform ? dim0 : (int)s_aux[wib][j].x;
               char* wp = reinterpret_cast<char*>((uintptr_t)d.z | ((uintptr_t)d.w << 32));
-              adagrad_row<FP16, NV>(acc, w[u], mo[u], dim, lr, eps, wp, momentum + d.y,
+              adagrad_row<FP16, NV>(acc, w[u], mo[u], dim, __frcp_rn((float)dim), lr, eps, wp, momentum + d.y,
                                     any_dirty ? s_dirty[wib][j] : nullptr);
             }
             seen_end = true;
@@ -289,6 +310,129 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
 #pragma unroll
     for (int q = 0; q < NV; ++q)
       *reinterpret_cast<float4*>(dst + chunk * PSTRIDE + (q * 32 + lane) * 4) = acc[q];
+  }
+}
+
+// ---- reduce_chunks_lean: the same walk for rows of up to 128 columns (one 16-byte piece per lane).
+// The walk is bound by instruction issue and by the latency of dependent instructions, not by
+// bytes in flight, so this form keeps one lookup in flight per warp, fits 32 registers and runs 64
+// warps per SM; a row's loads (gradient slice, and row + state where the row ends) are issued
+// together.  Same summation order and arithmetic as reduce_chunks.
+template <bool FP16, bool MEAN>
+__global__ void __launch_bounds__(LEAN_WARPS * 32, MTS_BWD_LEAN_MINBLK)
+reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
+                   const uint32_t* __restrict__ keys, const uint32_t* __restrict__ pos,
+                   const uint32_t* __restrict__ bag_of_pos, int64_t n,
+                   const int64_t* __restrict__ offsets,
+                   const float* __restrict__ grad, int64_t grad_stride, float lr, float eps,
+                   const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches, char* dev_w,
+                   char* host_w,
+                   float* __restrict__ momentum, float* __restrict__ partial_head,
+                   float* __restrict__ partial_tail) {
+  constexpr int EB = FP16 ? 2 : 4;
+  constexpr int PSTRIDE = 128;
+  __shared__ uint4 s_desc[LEAN_WARPS][32];      // {gradient float offset, key, row address lo, hi}
+  __shared__ uint2 s_aux[LEAN_WARPS][32];       // {dim, mean-pooling scale bits}
+  __shared__ uint8_t* s_dirty[LEAN_WARPS][32];
+  const int lane = threadIdx.x & 31;
+  const int wib = threadIdx.x >> 5;
+  const int64_t chunk = (int64_t)blockIdx.x * LEAN_WARPS + wib;
+  const int64_t p0 = chunk * BWD_CHUNK;
+  if (p0 >= n) return;
+  const int len = (int)min((int64_t)BWD_CHUNK, n - p0);
+  // a row that started in an earlier chunk: its piece here goes to combine_partials
+  bool open_head = p0 > 0 && keys[p0 - 1] == keys[p0];
+  const float* grad_lane = grad + lane * 4;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  bool last_is_end = true;
+
+  for (int k0 = 0; k0 < len; k0 += 32) {
+    const int cnt = min(32, len - k0);
+    bool my_end = false;
+    bool my_dirty = false;
+    int my_dim = 0;
+    if (lane < cnt) {
+      const int64_t p = p0 + k0 + lane;
+      const uint32_t key = keys[p];
+      my_end = (p + 1 >= n) || keys[p + 1] != key;
+      const uint32_t ps = pos[p];
+      const uint32_t bag = bag_of_pos[ps];
+      const int t = (int)(bag / (uint32_t)B);
+      const int b = (int)(bag - (uint32_t)t * (uint32_t)B);
+      const TableMeta m = meta[t];
+      my_dim = m.dim;
+      uint4 d;
+      d.x = (uint32_t)((int64_t)b * grad_stride + m.out_offset);
+      d.y = key;
+      d.z = 0u; d.w = 0u;
+      uint8_t* dirty = nullptr;
+      if (my_end) {
+        const RowTarget rt = row_target(m, (int64_t)key, ps, EB, slot_of_lookup, caches, dev_w, host_w);
+        d.z = (uint32_t)(uintptr_t)rt.w;
+        d.w = (uint32_t)((uintptr_t)rt.w >> 32);
+        dirty = rt.dirty;
+      }
+      s_desc[wib][lane] = d;
+      if (MEAN) {
+        uint2 a;
+        a.x = (uint32_t)m.dim;
+        a.y = __float_as_uint(1.f / (float)(offsets[bag + 1] - offsets[bag]));
+        s_aux[wib][lane] = a;
+      } else {
+        s_aux[wib][lane].x = (uint32_t)m.dim;
+      }
+      s_dirty[wib][lane] = dirty;
+      my_dirty = dirty != nullptr;
+    }
+    __syncwarp();                                                  // staged descriptions visible to the warp
+    const uint32_t ends = __ballot_sync(0xffffffffu, my_end);
+    const bool any_dirty = __any_sync(0xffffffffu, my_dirty);
+    // one dim for the whole batch unless it straddles tables of different width
+    const int dim0 = __shfl_sync(0xffffffffu, my_dim, 0);
+    const bool uniform = __all_sync(0xffffffffu, lane >= cnt || my_dim == dim0);
+    if (k0 + 32 >= len) last_is_end = (ends >> (cnt - 1)) & 1u;
+    const float inv_dim0 = __frcp_rn((float)dim0);
+
+    for (int j = 0; j < cnt; ++j) {
+      const uint4 d = s_desc[wib][j];
+      const int dim = uniform ? dim0 : (int)s_aux[wib][j].x;
+      const bool col = lane * 4 < dim;
+      float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (col) g = __ldg(reinterpret_cast<const float4*>(grad_lane + d.x));
+      const bool is_end = (ends >> j) & 1u;
+      uint4 w[1];
+      float m_old = 0.f;
+      char* wp = nullptr;
+      if (is_end && !open_head) {
+        wp = reinterpret_cast<char*>((uintptr_t)d.z | ((uintptr_t)d.w << 32));
+        load_row<FP16, 1>(w, wp, dim);
+        m_old = momentum[d.y];
+      }
+      if (MEAN) {
+        const float sc = __uint_as_float(s_aux[wib][j].y);
+        acc.x = fmaf(sc, g.x, acc.x); acc.y = fmaf(sc, g.y, acc.y);
+        acc.z = fmaf(sc, g.z, acc.z); acc.w = fmaf(sc, g.w, acc.w);
+      } else {
+        acc.x += g.x; acc.y += g.y; acc.z += g.z; acc.w += g.w;
+      }
+      if (is_end) {
+        if (open_head) {
+          *reinterpret_cast<float4*>(partial_head + chunk * PSTRIDE + lane * 4) = acc;
+          open_head = false;
+        } else {
+          float4 a1[1] = {acc};
+          adagrad_row<FP16, 1>(a1, w, m_old, dim, uniform ? inv_dim0 : __frcp_rn((float)dim), lr, eps, wp,
+                               momentum + d.y, any_dirty ? s_dirty[wib][j] : nullptr);
+        }
+        acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    __syncwarp();      // the next batch overwrites the staged descriptions
+  }
+  if (!last_is_end) {
+    // open_head still set: the whole chunk lies inside a row that started earlier
+    float* dst = open_head ? partial_head : partial_tail;
+    *reinterpret_cast<float4*>(dst + chunk * PSTRIDE + lane * 4) = acc;
   }
 }
 
@@ -340,7 +484,8 @@ template <bool FP16, int NV>
 __global__ void __launch_bounds__(BWD_WARPS * 32)
 combine_partials(const TableMeta* __restrict__ meta, int T, const uint32_t* __restrict__ keys,
                  const uint32_t* __restrict__ pos, int64_t n, float lr, float eps,
-                 const int32_t* __restrict__ slot_of_lookup, CachePtrs caches, char* dev_w, char* host_w,
+                 const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches, char* dev_w,
+                   char* host_w,
                  float* __restrict__ momentum, const float* __restrict__ partial_head,
                  const float* __restrict__ partial_tail, const float* __restrict__ partial_group) {
   constexpr int EB = FP16 ? 2 : 4;
@@ -412,7 +557,7 @@ combine_partials(const TableMeta* __restrict__ meta, int T, const uint32_t* __re
   const RowTarget rt = row_target(m, (int64_t)key, pos[pe - 1], EB, slot_of_lookup, caches, dev_w, host_w);
   uint4 w[NV];
   load_row<FP16, NV>(w, rt.w, m.dim);
-  adagrad_row<FP16, NV>(acc, w, momentum[key], m.dim, lr, eps, rt.w, momentum + key, rt.dirty);
+  adagrad_row<FP16, NV>(acc, w, momentum[key], m.dim, __frcp_rn((float)m.dim), lr, eps, rt.w, momentum + key, rt.dirty);
 }
 
 __global__ void export_unique(const uint32_t* __restrict__ keys, const uint32_t* __restrict__ seg_start,
@@ -457,7 +602,18 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
                            float* group, cudaStream_t s) {
   const int64_t chunks = ceil_div(N, BWD_CHUNK);
   const unsigned grid = (unsigned)ceil_div(chunks, BWD_WARPS);
-  {
+  if constexpr (NV == 1 && MTS_BWD_USE_LEAN) {
+    LaunchScope scope(K_REDUCE_CHUNKS, s);
+    const unsigned lean_grid = (unsigned)ceil_div(chunks, LEAN_WARPS);
+    if (pooling_mode == MTS_POOL_MEAN)
+      reduce_chunks_lean<FP16, true><<<lean_grid, LEAN_WARPS * 32, 0, s>>>(
+          h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
+          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail);
+    else
+      reduce_chunks_lean<FP16, false><<<lean_grid, LEAN_WARPS * 32, 0, s>>>(
+          h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
+          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail);
+  } else {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
     if (pooling_mode == MTS_POOL_MEAN)
       reduce_chunks<FP16, NV, GROUP, true><<<grid, BWD_WARPS * 32, 0, s>>>(
@@ -566,12 +722,12 @@ extern "C" int mts_tbe_backward_rowwise_adagrad(
 #define MTS_BWD(F, V, G) return launch_backward<F, V, G>(h, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad_out, grad_stride, lr, eps, slot_of_lookup, caches, head, tail, group, s)
   if (fp16) {
     if (nv <= 1) MTS_BWD(true, 1, MTS_BWD_GROUP1);
-    if (nv <= 2) MTS_BWD(true, 2, 4);
+    if (nv <= 2) MTS_BWD(true, 2, MTS_BWD_GROUP2);
     if (nv <= 4) MTS_BWD(true, 4, 2);
     MTS_BWD(true, 8, 1);
   } else {
     if (nv <= 1) MTS_BWD(false, 1, MTS_BWD_GROUP1);
-    if (nv <= 2) MTS_BWD(false, 2, 4);
+    if (nv <= 2) MTS_BWD(false, 2, MTS_BWD_GROUP2);
     if (nv <= 4) MTS_BWD(false, 4, 2);
     MTS_BWD(false, 8, 1);
   }
