@@ -229,10 +229,33 @@ def run_native(args, rank: int, world: int, local_rank: int):
     out = torch.empty((B, TD), dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream(dev)
 
+    # One training step.  The index-only half of the backward (ordering the lookups by row) does not
+    # need the gradient, so it runs on a second stream beside the forward pass; the gradient half
+    # follows the forward pass on the main stream.
+    side = torch.cuda.Stream(dev)
+    ev_fork, ev_sorted = torch.cuda.Event(), torch.cuda.Event()
+
+    def train_step(i, o, g, out_t, mid=None):
+        n = i.numel()
+        if args.sequential:
+            model.forward(i, o, n, out=out_t, stream=stream)
+            if mid is not None:
+                mid.record(stream)
+            model.backward(i, o, n, g, stream=stream)
+            return
+        ev_fork.record(stream)                 # after the previous step's use of the workspace
+        side.wait_event(ev_fork)
+        model.backward_sort(i, o, n, stream=side)
+        ev_sorted.record(side)
+        model.forward(i, o, n, out=out_t, stream=stream)
+        if mid is not None:
+            mid.record(stream)
+        stream.wait_event(ev_sorted)
+        model.backward_apply(o, n, g, stream=stream)
+
     def step(k):
         i, o, g = devb[k % R]
-        model.forward(i, o, i.numel(), out=out, stream=stream)
-        model.backward(i, o, i.numel(), g, stream=stream)
+        train_step(i, o, g, out)
 
     def barrier():
         if world > 1:
@@ -254,9 +277,7 @@ def run_native(args, rank: int, world: int, local_rank: int):
     ev[0].record(stream)
     for k in range(args.steps):
         i, o, g = devb[k % R]
-        model.forward(i, o, i.numel(), out=out, stream=stream)
-        ev[2 * k + 1].record(stream)
-        model.backward(i, o, i.numel(), g, stream=stream)
+        train_step(i, o, g, out, mid=ev[2 * k + 1])
         ev[2 * k + 2].record(stream)
     torch.cuda.synchronize(dev)
     sampler.mark(False)
@@ -302,8 +323,7 @@ def run_native(args, rank: int, world: int, local_rank: int):
             stream.wait_event(ev_in[k])
             if k >= 2:
                 stream.wait_event(ev_out[k - 2])            # the output buffer has been read back
-            model.forward(di, do_, n, out=d_out[k & 1], stream=stream)
-            model.backward(di, do_, n, dg, stream=stream)
+            train_step(di[:n], do_, dg, d_out[k & 1])
             ev_cmp[k].record(stream)
             with torch.cuda.stream(s_out):
                 s_out.wait_event(ev_cmp[k])
@@ -369,6 +389,7 @@ def run_native(args, rank: int, world: int, local_rank: int):
             "config": {"workload": spec.name, "tables": spec.T, "rows_per_table": int(spec.rows[0]),
                        "dim": int(spec.dims[0]), "storage": "fp16" if spec.dtype == wl.FP16 else "fp32",
                        "batch": B, "lookups_per_step": n_avg, "parallelism": f"{world} replica(s), own batches",
+                       "schedule": "sequential" if args.sequential else "backward's sort on a second stream beside the forward",
                        "l2": f"inputs larger than L2: {spec.weight_bytes / 1e9:.2f} GB of weights, {R} batches rotate"},
             "samples_per_sec": world * B / (ms_step * 1e-3),
             "forward_ms": fwd_ms, "backward_ms": bwd_ms,
@@ -578,7 +599,7 @@ def main():
     ap.add_argument("--pooling", type=int, default=50, help="cfg5: lookups per bag")
     ap.add_argument("--alpha", type=float, default=1.0, help="cfg5: Zipf exponent")
     ap.add_argument("--cache-fraction", type=float, default=0.10, help="cfg5: cache slots / rows")
-    ap.add_argument("--sequential", action="store_true", help="cached workloads: no side stream")
+    ap.add_argument("--sequential", action="store_true", help="one stream only (no sort beside the forward, no cache pipeline)")
     ap.add_argument("--lock-depth", type=int, default=2,
                     help="cached workloads: batches a stamped way stays unevictable (Section 5.7 invariant)")
     ap.add_argument("--trace", action="store_true",

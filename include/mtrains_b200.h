@@ -164,6 +164,25 @@ int mts_tbe_backward_rowwise_adagrad(const mts_tables* tables, int32_t B, const 
                                      void* workspace, size_t workspace_bytes,
                                      int64_t* uniq_rows_out, int64_t* n_unique_out, void* stream);
 
+/* The same backward in two calls, for callers that schedule the two halves themselves.
+ * mts_tbe_backward_sort needs only the batch's indices: it writes into the workspace the lookups
+ * ordered by row (and, if asked, the distinct rows), so it can run before the gradient exists,
+ * for instance on another stream while the forward pass of the same batch runs (the paper's
+ * pipeline likewise works on a batch's indices ahead of its training step, Section 5.7).
+ * mts_tbe_backward_apply sums the gradients per row and applies the optimizer (Section 5.9); it
+ * must be ordered after the matching mts_tbe_backward_sort (same stream, or an event), with the
+ * same tables, B, offsets, N and workspace, whose contents nothing else may touch in between.
+ * mts_tbe_backward_rowwise_adagrad is exactly sort followed by apply on one stream; arguments
+ * and errors are the same as there. */
+int mts_tbe_backward_sort(const mts_tables* tables, int32_t B, const int64_t* indices,
+                          const int64_t* offsets, int64_t N, void* workspace, size_t workspace_bytes,
+                          int64_t* uniq_rows_out, int64_t* n_unique_out, void* stream);
+int mts_tbe_backward_apply(const mts_tables* tables, int32_t B, const int64_t* offsets, int64_t N,
+                           int32_t pooling_mode, const float* grad_out, int64_t grad_stride, float lr,
+                           float eps, const int32_t* slot_of_lookup, void* const* host_cache_data,
+                           uint8_t* const* host_cache_dirty, int32_t n_caches, void* workspace,
+                           size_t workspace_bytes, void* stream);
+
 /* Backward without a workspace argument and without any allocation (the paper has no
  * counterpart; this exists for callers of this library that cannot allocate device memory).
  * Such callers are, for example, a training or serving loop embedded in a framework that

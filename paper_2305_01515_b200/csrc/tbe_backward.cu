@@ -648,32 +648,43 @@ extern "C" size_t mts_tbe_backward_workspace_bytes(const mts_tables* h, int32_t 
   return bwd_layout(h, N).total;
 }
 
-extern "C" int mts_tbe_backward_rowwise_adagrad(
-    const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets, int64_t N,
-    int32_t pooling_mode, const float* grad_out, int64_t grad_stride, float lr, float eps,
-    const int32_t* slot_of_lookup, void* const* host_cache_data, uint8_t* const* host_cache_dirty,
-    int32_t n_caches, void* workspace, size_t workspace_bytes, int64_t* uniq_rows_out,
-    int64_t* n_unique_out, void* stream) {
-  if (!h || !offsets || !grad_out || B < 1 || N < 0 || (N > 0 && !indices))
-    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward: null argument or bad size");
-  if (pooling_mode != MTS_POOL_SUM && pooling_mode != MTS_POOL_MEAN)
-    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward: pooling mode %d", pooling_mode);
-  if ((uniq_rows_out == nullptr) != (n_unique_out == nullptr))
-    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward: pass both uniq_rows_out and n_unique_out or neither");
-  if (grad_stride < h->total_dim || (grad_stride & 3) || ((uintptr_t)grad_out & 15))
-    return set_error(MTS_ERR_ALIGNMENT, "tbe_backward: grad_out must be 16-byte aligned, grad_stride >= %d and a multiple of 4",
-                     h->total_dim);
-  if (N >= (1ll << 32) - BWD_CHUNK || (int64_t)h->T * B >= (1ll << 32) || (int64_t)B * grad_stride >= (1ll << 32))
-    return set_error(MTS_ERR_UNSUPPORTED,
-                     "tbe_backward: lookup positions, bag ids and grad_out element offsets must fit 32 bits");
-  const BwdLayout L = bwd_layout(h, N);
+namespace {
+
+int key_bits_of(const mts_tables* h) {
+  int key_bits = 1;
+  while (key_bits < 32 && (1ll << key_bits) < h->total_rows) ++key_bits;
+  return key_bits;
+}
+
+// which of the two buffer pairs holds the sorted lookups after radix_sort_pairs
+bool sorted_in_b(const mts_tables* h, int64_t N) {
+  return N > 1 && (((key_bits_of(h) + 7) / 8) & 1) != 0;
+}
+
+int check_backward_common(const mts_tables* h, int32_t B, const int64_t* offsets, int64_t N, void* workspace,
+                          size_t workspace_bytes, const BwdLayout& L, const char* who) {
+  if (!h || !offsets || B < 1 || N < 0) return set_error(MTS_ERR_INVALID_ARG, "%s: null argument or bad size", who);
+  if (N >= (1ll << 32) - BWD_CHUNK || (int64_t)h->T * B >= (1ll << 32))
+    return set_error(MTS_ERR_UNSUPPORTED, "%s: lookup positions and bag ids must fit 32 bits", who);
   if (!workspace || ((uintptr_t)workspace & 255))
-    return set_error(MTS_ERR_ALIGNMENT, "tbe_backward: workspace must be non-null and 256-byte aligned");
+    return set_error(MTS_ERR_ALIGNMENT, "%s: workspace must be non-null and 256-byte aligned", who);
   if (workspace_bytes < L.total)
-    return set_error(MTS_ERR_WORKSPACE, "tbe_backward: workspace of %zu bytes, %zu needed", workspace_bytes, L.total);
-  CachePtrs caches;
-  int rc = fill_cache_ptrs(h, host_cache_data, host_cache_dirty, n_caches, slot_of_lookup, &caches);
+    return set_error(MTS_ERR_WORKSPACE, "%s: workspace of %zu bytes, %zu needed", who, workspace_bytes, L.total);
+  return MTS_OK;
+}
+
+}  // namespace
+
+extern "C" int mts_tbe_backward_sort(const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets,
+                                     int64_t N, void* workspace, size_t workspace_bytes, int64_t* uniq_rows_out,
+                                     int64_t* n_unique_out, void* stream) {
+  if (!h) return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_sort: null tables");
+  const BwdLayout L = bwd_layout(h, N > 0 ? N : 0);
+  int rc = check_backward_common(h, B, offsets, N, workspace, workspace_bytes, L, "tbe_backward_sort");
   if (rc != MTS_OK) return rc;
+  if (N > 0 && !indices) return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_sort: null indices");
+  if ((uniq_rows_out == nullptr) != (n_unique_out == nullptr))
+    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_sort: pass both uniq_rows_out and n_unique_out or neither");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   char* ws = static_cast<char*>(workspace);
   if (N == 0) {
@@ -696,12 +707,11 @@ extern "C" int mts_tbe_backward_rowwise_adagrad(
     rc = check_launch("linearize_lookups");
     if (rc != MTS_OK) return rc;
   }
-  int key_bits = 1;
-  while (key_bits < 32 && (1ll << key_bits) < h->total_rows) ++key_bits;
   uint32_t *keys = nullptr, *pos = nullptr;
-  rc = radix_sort_pairs(keys_a, vals_a, keys_b, vals_b, N, nullptr, key_bits, reinterpret_cast<uint32_t*>(ws + L.hist), &keys,
-                        &pos, s);
+  rc = radix_sort_pairs(keys_a, vals_a, keys_b, vals_b, N, nullptr, key_bits_of(h), reinterpret_cast<uint32_t*>(ws + L.hist),
+                        &keys, &pos, s);
   if (rc != MTS_OK) return rc;
+  if ((keys == keys_b) != sorted_in_b(h, N)) return set_error(MTS_ERR_CUDA, "tbe_backward_sort: unexpected result buffer");
   if (uniq_rows_out) {
     uint32_t* seg_start = reinterpret_cast<uint32_t*>(ws + L.seg_start);
     uint32_t* n_unique = reinterpret_cast<uint32_t*>(ws + L.n_unique);
@@ -714,6 +724,36 @@ extern "C" int mts_tbe_backward_rowwise_adagrad(
     rc = check_launch("export_unique");
     if (rc != MTS_OK) return rc;
   }
+  return MTS_OK;
+}
+
+extern "C" int mts_tbe_backward_apply(const mts_tables* h, int32_t B, const int64_t* offsets, int64_t N,
+                                      int32_t pooling_mode, const float* grad_out, int64_t grad_stride, float lr,
+                                      float eps, const int32_t* slot_of_lookup, void* const* host_cache_data,
+                                      uint8_t* const* host_cache_dirty, int32_t n_caches, void* workspace,
+                                      size_t workspace_bytes, void* stream) {
+  if (!h) return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_apply: null tables");
+  const BwdLayout L = bwd_layout(h, N > 0 ? N : 0);
+  int rc = check_backward_common(h, B, offsets, N, workspace, workspace_bytes, L, "tbe_backward_apply");
+  if (rc != MTS_OK) return rc;
+  if (!grad_out) return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_apply: null grad_out");
+  if (pooling_mode != MTS_POOL_SUM && pooling_mode != MTS_POOL_MEAN)
+    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_apply: pooling mode %d", pooling_mode);
+  if (grad_stride < h->total_dim || (grad_stride & 3) || ((uintptr_t)grad_out & 15))
+    return set_error(MTS_ERR_ALIGNMENT,
+                     "tbe_backward_apply: grad_out must be 16-byte aligned, grad_stride >= %d and a multiple of 4", h->total_dim);
+  if ((int64_t)B * grad_stride >= (1ll << 32))
+    return set_error(MTS_ERR_UNSUPPORTED, "tbe_backward_apply: grad_out element offsets must fit 32 bits");
+  CachePtrs caches;
+  rc = fill_cache_ptrs(h, host_cache_data, host_cache_dirty, n_caches, slot_of_lookup, &caches);
+  if (rc != MTS_OK) return rc;
+  if (N == 0) return MTS_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  const bool in_b = sorted_in_b(h, N);
+  const uint32_t* keys = reinterpret_cast<const uint32_t*>(ws + (in_b ? L.keys_b : L.keys_a));
+  const uint32_t* pos = reinterpret_cast<const uint32_t*>(ws + (in_b ? L.vals_b : L.vals_a));
+  const uint32_t* bag_of_pos = reinterpret_cast<const uint32_t*>(ws + L.bag_of_pos);
   float* head = reinterpret_cast<float*>(ws + L.head);
   float* tail = reinterpret_cast<float*>(ws + L.tail);
   float* group = reinterpret_cast<float*>(ws + L.group);
@@ -732,6 +772,33 @@ extern "C" int mts_tbe_backward_rowwise_adagrad(
     MTS_BWD(false, 8, 1);
   }
 #undef MTS_BWD
+}
+
+extern "C" int mts_tbe_backward_rowwise_adagrad(
+    const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets, int64_t N,
+    int32_t pooling_mode, const float* grad_out, int64_t grad_stride, float lr, float eps,
+    const int32_t* slot_of_lookup, void* const* host_cache_data, uint8_t* const* host_cache_dirty,
+    int32_t n_caches, void* workspace, size_t workspace_bytes, int64_t* uniq_rows_out,
+    int64_t* n_unique_out, void* stream) {
+  // every argument is checked before the first launch
+  if (!h || !offsets || !grad_out || B < 1 || N < 0 || (N > 0 && !indices))
+    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward: null argument or bad size");
+  if (pooling_mode != MTS_POOL_SUM && pooling_mode != MTS_POOL_MEAN)
+    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward: pooling mode %d", pooling_mode);
+  if (grad_stride < h->total_dim || (grad_stride & 3) || ((uintptr_t)grad_out & 15))
+    return set_error(MTS_ERR_ALIGNMENT, "tbe_backward: grad_out must be 16-byte aligned, grad_stride >= %d and a multiple of 4",
+                     h->total_dim);
+  if ((int64_t)B * grad_stride >= (1ll << 32))
+    return set_error(MTS_ERR_UNSUPPORTED, "tbe_backward: grad_out element offsets must fit 32 bits");
+  {
+    CachePtrs caches;
+    int rc = fill_cache_ptrs(h, host_cache_data, host_cache_dirty, n_caches, slot_of_lookup, &caches);
+    if (rc != MTS_OK) return rc;
+  }
+  int rc = mts_tbe_backward_sort(h, B, indices, offsets, N, workspace, workspace_bytes, uniq_rows_out, n_unique_out, stream);
+  if (rc != MTS_OK) return rc;
+  return mts_tbe_backward_apply(h, B, offsets, N, pooling_mode, grad_out, grad_stride, lr, eps, slot_of_lookup,
+                                host_cache_data, host_cache_dirty, n_caches, workspace, workspace_bytes, stream);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -138,6 +138,21 @@ class DeviceModel:
             slot, self.cache_data, self.cache_dirty, self.workspace,
             self.ws_bytes, uniq_rows_out, n_unique_out, stream)
 
+    def backward_sort(self, indices, offsets, N: int, uniq_rows_out=None, n_unique_out=None, stream=None) -> None:
+        """Index-only half of the backward; may run on another stream than the forward pass."""
+        self.reserve(N)
+        mb.tbe_backward_sort(self.tables, self.spec.batch, indices, offsets, N, self.workspace, self.ws_bytes,
+                             uniq_rows_out, n_unique_out, stream)
+
+    def backward_apply(self, offsets, N: int, grad_out, lr: Optional[float] = None, eps: Optional[float] = None,
+                       pooling_mode: int = mb.POOL_SUM, stream=None, ctx: Optional[int] = None) -> None:
+        """Gradient half of the backward, after backward_sort of the same batch."""
+        slot = self.ctx[self.cur if ctx is None else ctx]["slot"] if self.cached else None
+        mb.tbe_backward_apply(
+            self.tables, self.spec.batch, offsets, N, pooling_mode, grad_out, grad_out.shape[1],
+            self.spec.lr if lr is None else lr, self.spec.eps if eps is None else eps,
+            slot, self.cache_data, self.cache_dirty, self.workspace, self.ws_bytes, stream)
+
     def group_range(self, g: int, offsets_host: np.ndarray):
         """Lookup range [begin, begin + n) of cache group g in one batch (host-side CSR)."""
         _, t0, t1 = self.groups[g]

@@ -176,3 +176,44 @@ def test_config2_full_size_sampled_rows():
         assert_close_mag(got_w, Wsub, mag, FWD_RTOL[spec.dtype], f"table {t} weights")
         assert_close_mag(got_m, msub, msub, 1e-5, f"table {t} momentum")
     m.close()
+
+
+@pytest.mark.gpu
+def test_backward_in_two_calls_matches_one_call():
+    """mts_tbe_backward_sort on a second stream + mts_tbe_backward_apply give the bits of the one-call backward."""
+    import torch
+    from paper_2305_01515_b200 import workload as wl
+    from paper_2305_01515_b200.harness import DeviceModel
+    spec = wl.config1()
+    dev = torch.device("cuda:0")
+    idx_h, off_h = wl.gen_batch(spec, 0)[:2]
+    grad_h = wl.gen_grad(spec, 0)
+    idx, off = torch.from_numpy(idx_h).to(dev), torch.from_numpy(off_h).to(dev)
+    grad = torch.from_numpy(grad_h).to(dev)
+    n = idx.numel()
+    results = []
+    for split in (False, True):
+        m = DeviceModel(spec, dev)
+        main = torch.cuda.current_stream(dev)
+        for _ in range(2):                          # two steps: the second reuses the workspace
+            if split:
+                side = torch.cuda.Stream(dev)
+                fork, done = torch.cuda.Event(), torch.cuda.Event()
+                fork.record(main)
+                side.wait_event(fork)
+                uniq = torch.empty(n, dtype=torch.int64, device=dev)
+                nuniq = torch.zeros(1, dtype=torch.int64, device=dev)
+                m.backward_sort(idx, off, n, uniq_rows_out=uniq, n_unique_out=nuniq, stream=side)
+                done.record(side)
+                main.wait_event(done)
+                m.backward_apply(off, n, grad, stream=main)
+            else:
+                uniq = torch.empty(n, dtype=torch.int64, device=dev)
+                nuniq = torch.zeros(1, dtype=torch.int64, device=dev)
+                m.backward(idx, off, n, grad, uniq_rows_out=uniq, n_unique_out=nuniq, stream=main)
+        torch.cuda.synchronize(dev)
+        k = int(nuniq.item())
+        results.append((m.dev_weights.clone(), m.momentum.clone(), uniq[:k].clone()))
+    assert torch.equal(results[0][0], results[1][0])
+    assert torch.equal(results[0][1], results[1][1])
+    assert torch.equal(results[0][2], results[1][2])
