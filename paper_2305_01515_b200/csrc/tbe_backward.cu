@@ -31,6 +31,9 @@ namespace mts {
 #ifndef MTS_BWD_LEAN_WARPS
 #define MTS_BWD_LEAN_WARPS 4
 #endif
+#ifndef MTS_BWD_LEAN_RUN
+#define MTS_BWD_LEAN_RUN 6      // gradient loads issued together inside a run of lookups of one row
+#endif
 #ifndef MTS_BWD_LEAN_MINBLK
 #define MTS_BWD_LEAN_MINBLK 16  // resident blocks per SM reduce_chunks_lean is bounded for (32 registers)
 #endif
@@ -45,6 +48,7 @@ namespace mts {
 #endif
 constexpr int BWD_CHUNK = MTS_BWD_CHUNK;
 constexpr int BWD_WARPS = 4;
+constexpr int LEAN_RUN = MTS_BWD_LEAN_RUN;
 constexpr int LEAN_WARPS = MTS_BWD_LEAN_WARPS;   // warps per block of reduce_chunks_lean
 constexpr int LIN_GROUP = 8;     // lanes per bag in linearize_lookups
 
@@ -393,38 +397,56 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
     if (k0 + 32 >= len) last_is_end = (ends >> (cnt - 1)) & 1u;
     const float inv_dim0 = __frcp_rn((float)dim0);
 
-    for (int j = 0; j < cnt; ++j) {
-      const uint4 d = s_desc[wib][j];
-      const int dim = uniform ? dim0 : (int)s_aux[wib][j].x;
-      const bool col = lane * 4 < dim;
-      float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (col) g = __ldg(reinterpret_cast<const float4*>(grad_lane + d.x));
-      const bool is_end = (ends >> j) & 1u;
-      uint4 w[1];
-      float m_old = 0.f;
-      char* wp = nullptr;
-      if (is_end && !open_head) {
-        wp = reinterpret_cast<char*>((uintptr_t)d.z | ((uintptr_t)d.w << 32));
-        load_row<FP16, 1>(w, wp, dim);
-        m_old = momentum[d.y];
-      }
+    // walk the 32 lookups run by run: the lookups before the next "last of its row" are only
+    // summed (no test per lookup), then that lookup closes its row
+    auto add_scaled = [&](const float4& g, int jj) {
       if (MEAN) {
-        const float sc = __uint_as_float(s_aux[wib][j].y);
+        const float sc = __uint_as_float(s_aux[wib][jj].y);
         acc.x = fmaf(sc, g.x, acc.x); acc.y = fmaf(sc, g.y, acc.y);
         acc.z = fmaf(sc, g.z, acc.z); acc.w = fmaf(sc, g.w, acc.w);
       } else {
         acc.x += g.x; acc.y += g.y; acc.z += g.z; acc.w += g.w;
       }
-      if (is_end) {
+    };
+    auto load_grad = [&](int jj) {
+      const int dim = uniform ? dim0 : (int)s_aux[wib][jj].x;
+      float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (lane * 4 < dim) g = __ldg(reinterpret_cast<const float4*>(grad_lane + s_desc[wib][jj].x));
+      return g;
+    };
+    int j = 0;
+    while (j < cnt) {
+      const uint32_t rest = ends >> j;
+      const int e = rest ? j + __ffs(rest) - 1 : cnt;              // next lookup that ends a row (or none)
+      for (; j + LEAN_RUN <= e; j += LEAN_RUN) {
+        float4 g[LEAN_RUN];
+#pragma unroll
+        for (int u = 0; u < LEAN_RUN; ++u) g[u] = load_grad(j + u);
+#pragma unroll
+        for (int u = 0; u < LEAN_RUN; ++u) add_scaled(g[u], j + u);
+      }
+      for (; j < e; ++j) add_scaled(load_grad(j), j);
+      if (e < cnt) {
+        const uint4 d = s_desc[wib][e];
+        const int dim = uniform ? dim0 : (int)s_aux[wib][e].x;
+        float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (lane * 4 < dim) g = __ldg(reinterpret_cast<const float4*>(grad_lane + d.x));
         if (open_head) {
+          add_scaled(g, e);
           *reinterpret_cast<float4*>(partial_head + chunk * PSTRIDE + lane * 4) = acc;
           open_head = false;
         } else {
+          uint4 w[1];
+          char* wp = reinterpret_cast<char*>((uintptr_t)d.z | ((uintptr_t)d.w << 32));
+          load_row<FP16, 1>(w, wp, dim);
+          const float m_old = momentum[d.y];
+          add_scaled(g, e);
           float4 a1[1] = {acc};
           adagrad_row<FP16, 1>(a1, w, m_old, dim, uniform ? inv_dim0 : __frcp_rn((float)dim), lr, eps, wp,
-                               momentum + d.y, any_dirty ? s_dirty[wib][j] : nullptr);
+                               momentum + d.y, any_dirty ? s_dirty[wib][e] : nullptr);
         }
         acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        j = e + 1;
       }
     }
     __syncwarp();      // the next batch overwrites the staged descriptions
