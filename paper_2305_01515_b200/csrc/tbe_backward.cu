@@ -14,6 +14,7 @@
 // The summation tree depends only on the sorted order and CHUNK, so two runs give the same
 // bits.  No thread ever writes a word another thread of the same launch writes.
 #include <mutex>
+#include <type_traits>
 
 #include "common.cuh"
 
@@ -32,7 +33,7 @@ namespace mts {
 #define MTS_BWD_LEAN_WARPS 4
 #endif
 #ifndef MTS_BWD_LEAN_RUN
-#define MTS_BWD_LEAN_RUN 6      // gradient loads issued together inside a run of lookups of one row
+#define MTS_BWD_LEAN_RUN 4      // gradient loads issued together inside a run of lookups of one row
 #endif
 #ifndef MTS_BWD_LEAN_MINBLK
 #define MTS_BWD_LEAN_MINBLK 16  // resident blocks per SM reduce_chunks_lean is bounded for (32 registers)
@@ -398,7 +399,10 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
     const float inv_dim0 = __frcp_rn((float)dim0);
 
     // walk the 32 lookups run by run: the lookups before the next "last of its row" are only
-    // summed (no test per lookup), then that lookup closes its row
+    // summed (no test per lookup), then that lookup closes its row.  `full` = every row of the
+    // batch has 128 columns: all lanes take part and the width is a constant.
+    auto walk = [&](auto full) {
+    constexpr bool FULL = decltype(full)::value;
     auto add_scaled = [&](const float4& g, int jj) {
       if (MEAN) {
         const float sc = __uint_as_float(s_aux[wib][jj].y);
@@ -409,9 +413,9 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
       }
     };
     auto load_grad = [&](int jj) {
-      const int dim = uniform ? dim0 : (int)s_aux[wib][jj].x;
+      const int dim = FULL ? 128 : uniform ? dim0 : (int)s_aux[wib][jj].x;
       float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (lane * 4 < dim) g = __ldg(reinterpret_cast<const float4*>(grad_lane + s_desc[wib][jj].x));
+      if (FULL || lane * 4 < dim) g = __ldg(reinterpret_cast<const float4*>(grad_lane + s_desc[wib][jj].x));
       return g;
     };
     int j = 0;
@@ -428,9 +432,9 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
       for (; j < e; ++j) add_scaled(load_grad(j), j);
       if (e < cnt) {
         const uint4 d = s_desc[wib][e];
-        const int dim = uniform ? dim0 : (int)s_aux[wib][e].x;
+        const int dim = FULL ? 128 : uniform ? dim0 : (int)s_aux[wib][e].x;
         float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (lane * 4 < dim) g = __ldg(reinterpret_cast<const float4*>(grad_lane + d.x));
+        if (FULL || lane * 4 < dim) g = __ldg(reinterpret_cast<const float4*>(grad_lane + d.x));
         if (open_head) {
           add_scaled(g, e);
           *reinterpret_cast<float4*>(partial_head + chunk * PSTRIDE + lane * 4) = acc;
@@ -442,13 +446,16 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
           const float m_old = momentum[d.y];
           add_scaled(g, e);
           float4 a1[1] = {acc};
-          adagrad_row<FP16, 1>(a1, w, m_old, dim, uniform ? inv_dim0 : __frcp_rn((float)dim), lr, eps, wp,
+          adagrad_row<FP16, 1>(a1, w, m_old, dim, FULL ? 0.0078125f : uniform ? inv_dim0 : __frcp_rn((float)dim), lr, eps, wp,
                                momentum + d.y, any_dirty ? s_dirty[wib][e] : nullptr);
         }
         acc = make_float4(0.f, 0.f, 0.f, 0.f);
         j = e + 1;
       }
     }
+    };
+    if (uniform && dim0 == 128) walk(std::true_type{});
+    else walk(std::false_type{});
     __syncwarp();      // the next batch overwrites the staged descriptions
   }
   if (!last_is_end) {
