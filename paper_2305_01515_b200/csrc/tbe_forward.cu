@@ -3,6 +3,8 @@
 // vec16 16-byte chunks is read by a group of G = pow2(vec16) lanes, so 32 / G rows are in
 // flight per load instruction and UNROLL of those instructions are issued back to back.
 // Accumulation in fp32 registers, one 16-byte store per lane group member at the end.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace mts {
@@ -28,7 +30,7 @@ template <bool FP16, int NV>
 __global__ void __launch_bounds__(FWD_WARPS * 32, (NV == 1 ? MTS_FWD_MINBLK : 1))
 tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B,
                    const int64_t* __restrict__ indices, const int64_t* __restrict__ offsets,
-                   const int32_t* __restrict__ slot_of_lookup, CachePtrs caches,
+                   const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches,
                    const char* __restrict__ dev_w, const char* __restrict__ host_w,
                    int32_t pooling_mode, float* __restrict__ out, int64_t out_stride,
                    int32_t* status) {
@@ -99,29 +101,36 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
           if (s >= 0) my_ptr = cache_base + (int64_t)s * row_bytes;
         }
       }
-      for (int r = 0; r < cnt; r += R * FWD_UNROLL) {
-        uint4 v[FWD_UNROLL][NV];
+      // `whole` = the row is exactly G pieces wide (a power of two, at most 32): every lane of a
+      // group has a piece, no column test
+      auto rows = [&](auto whole) {
+        constexpr bool WHOLE = decltype(whole)::value;
+        for (int r = 0; r < cnt; r += R * FWD_UNROLL) {
+          uint4 v[FWD_UNROLL][NV];
 #pragma unroll
-        for (int u = 0; u < FWD_UNROLL; ++u) {
-          const int j = r + u * R + sub;
-          const unsigned long long p =
-              __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_ptr, j & 31);
-          const bool valid = j < cnt;
+          for (int u = 0; u < FWD_UNROLL; ++u) {
+            const int j = r + u * R + sub;
+            const unsigned long long p =
+                __shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)my_ptr, j & 31);
+            const bool valid = j < cnt;
 #pragma unroll
-          for (int q = 0; q < NV; ++q) {
-            const int c = cl + q * 32;
-            if (valid && c < vec16) v[u][q] = ld_nc_16(reinterpret_cast<const char*>(p) + (int64_t)c * 16);
-            else v[u][q] = make_uint4(0u, 0u, 0u, 0u);
+            for (int q = 0; q < (WHOLE ? 1 : NV); ++q) {
+              const int c = cl + q * 32;
+              if (valid && (WHOLE || c < vec16)) v[u][q] = ld_nc_16(reinterpret_cast<const char*>(p) + (int64_t)c * 16);
+              else v[u][q] = make_uint4(0u, 0u, 0u, 0u);
+            }
           }
+#pragma unroll
+          for (int u = 0; u < FWD_UNROLL; ++u)
+#pragma unroll
+            for (int q = 0; q < (WHOLE ? 1 : NV); ++q) {
+              if (FP16) add_half8(acc[q], v[u][q]);
+              else add_float4(acc[q], v[u][q]);
+            }
         }
-#pragma unroll
-        for (int u = 0; u < FWD_UNROLL; ++u)
-#pragma unroll
-          for (int q = 0; q < NV; ++q) {
-            if (FP16) add_half8(acc[q], v[u][q]);
-            else add_float4(acc[q], v[u][q]);
-          }
-      }
+      };
+      if (vec16 == G) rows(std::true_type{});
+      else rows(std::false_type{});
     }
     // fold the row groups of the warp together
     for (int o = G; o < 32; o <<= 1) {
