@@ -232,7 +232,7 @@ def run_native(args, rank: int, world: int, local_rank: int):
     # One training step.  The index-only half of the backward (ordering the lookups by row) does not
     # need the gradient, so it runs on a second stream beside the forward pass; the gradient half
     # follows the forward pass on the main stream.
-    side = torch.cuda.Stream(dev)
+    side = torch.cuda.Stream(dev, priority=-1)   # its small grids get SM slots at once, beside the forward's blocks
     ev_fork, ev_sorted = torch.cuda.Event(), torch.cuda.Event()
 
     def train_step(i, o, g, out_t, mid=None):
