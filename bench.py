@@ -235,9 +235,9 @@ def run_native(args, rank: int, world: int, local_rank: int):
     side = torch.cuda.Stream(dev, priority=-1)   # its small grids get SM slots at once, beside the forward's blocks
     ev_fork, ev_sorted = torch.cuda.Event(), torch.cuda.Event()
 
-    def train_step(i, o, g, out_t, mid=None):
+    def train_step(i, o, g, out_t, mid=None, sequential=args.sequential):
         n = i.numel()
-        if args.sequential:
+        if sequential:
             model.forward(i, o, n, out=out_t, stream=stream)
             if mid is not None:
                 mid.record(stream)
@@ -288,10 +288,12 @@ def run_native(args, rank: int, world: int, local_rank: int):
     bwd_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(args.steps)) / args.steps
     clocks = sampler.stop()
 
-    # per-kernel device times over the same K steps, bracketed by CUDA events on the launch stream
+    # per-kernel device times over the same K steps, bracketed by CUDA events on the launch stream;
+    # one stream here, so that no kernel's time includes another stream's kernels running beside it
     mb.trace_enable(True)
     for k in range(args.steps):
-        step(k)
+        i, o, g = devb[k % R]
+        train_step(i, o, g, out, sequential=True)
     trace = mb.trace_report()
     mb.trace_enable(False)
 
@@ -364,8 +366,8 @@ def run_native(args, rank: int, world: int, local_rank: int):
         # profiles/ncu_full_cfg2_8tables_top_kernels.md (1.967 M lookups per launch there); DRAM traffic
         # grows with the lookups processed, so a launch's traffic is this figure times its lookups.
         # Set an entry to None when its kernel changes after the capture.
-        ncu_dram_bytes_per_lookup = {"reduce_chunks": (214.897664e6 + 158.551552e6) / 1.9667e6,
-                                     "tbe_forward_kernel": (149.063168e6 + 26.262272e6) / 1.9667e6}
+        ncu_dram_bytes_per_lookup = {"reduce_chunks": (233.486848e6 + 111.202048e6) / 1.967755e6,
+                                     "tbe_forward_kernel": (148.992768e6 + 21.388032e6) / 1.967755e6}
         top = max(trace.items(), key=lambda kv: kv[1][0]) if trace else (None, (0.0, 0))
         kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps} for k, v in trace.items()}
         roof = None
@@ -379,7 +381,7 @@ def run_native(args, rank: int, world: int, local_rank: int):
                     "traffic_source": "ncu capture on 8 of 26 tables, scaled by lookups per launch",
                     "peak_source": peak_src,
                     "algorithmic_bytes_per_launch": alg[top[0]], "avg_launch_ms": avg_ms,
-                    "timing": "CUDA events around every launch, separate pass of the same K steps"}
+                    "timing": "CUDA events around every launch, separate single-stream pass of the same K steps"}
         step_bytes = 2.0 * n_avg * per_lookup
         ms_step = ms_total / args.steps
         line = {

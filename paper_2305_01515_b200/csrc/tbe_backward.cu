@@ -13,6 +13,7 @@
 //                          chunk order and applies the update
 // The summation tree depends only on the sorted order and CHUNK, so two runs give the same
 // bits.  No thread ever writes a word another thread of the same launch writes.
+#include <algorithm>
 #include <mutex>
 #include <type_traits>
 
@@ -333,7 +334,7 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
                    const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches, char* dev_w,
                    char* host_w,
                    float* __restrict__ momentum, float* __restrict__ partial_head,
-                   float* __restrict__ partial_tail) {
+                   float* __restrict__ partial_tail, uint32_t* __restrict__ next_chunk) {
   constexpr int EB = FP16 ? 2 : 4;
   constexpr int PSTRIDE = 128;
   __shared__ uint4 s_desc[LEAN_WARPS][32];      // {gradient float offset, key, row address lo, hi}
@@ -341,13 +342,18 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
   __shared__ uint8_t* s_dirty[LEAN_WARPS][32];
   const int lane = threadIdx.x & 31;
   const int wib = threadIdx.x >> 5;
-  const int64_t chunk = (int64_t)blockIdx.x * LEAN_WARPS + wib;
+  const float* grad_lane = grad + lane * 4;
+  // Chunks differ a lot in cost (a chunk inside one hot row is a plain sum, a chunk of rows seen
+  // once is 128 updates), so a warp takes its next chunk from a counter instead of a fixed share.
+  for (;;) {
+  uint32_t taken = 0;
+  if (lane == 0) taken = atomicAdd(next_chunk, 1u);
+  const int64_t chunk = (int64_t)__shfl_sync(0xffffffffu, taken, 0);
   const int64_t p0 = chunk * BWD_CHUNK;
   if (p0 >= n) return;
   const int len = (int)min((int64_t)BWD_CHUNK, n - p0);
   // a row that started in an earlier chunk: its piece here goes to combine_partials
   bool open_head = p0 > 0 && keys[p0 - 1] == keys[p0];
-  const float* grad_lane = grad + lane * 4;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   bool last_is_end = true;
 
@@ -462,6 +468,7 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
     // open_head still set: the whole chunk lies inside a row that started earlier
     float* dst = open_head ? partial_head : partial_tail;
     *reinterpret_cast<float4*>(dst + chunk * PSTRIDE + lane * 4) = acc;
+  }
   }
 }
 
@@ -599,7 +606,7 @@ __global__ void export_unique(const uint32_t* __restrict__ keys, const uint32_t*
 }
 
 struct BwdLayout {
-  size_t keys_a, keys_b, vals_a, vals_b, bag_of_pos, hist, scan, seg_start, n_unique, head, tail, group, total;
+  size_t keys_a, keys_b, vals_a, vals_b, bag_of_pos, hist, scan, seg_start, n_unique, next_chunk, head, tail, group, total;
 };
 
 static BwdLayout bwd_layout(const mts_tables* h, int64_t N) {
@@ -613,6 +620,7 @@ static BwdLayout bwd_layout(const mts_tables* h, int64_t N) {
   L.scan = take(scan_scratch_words() * 4);
   L.seg_start = take((n + 1) * 4);
   L.n_unique = take(256);
+  L.next_chunk = take(256);
   const int nv = (h->max_dim + 127) / 128;
   const int nvp = nv <= 1 ? 1 : nv <= 2 ? 2 : nv <= 4 ? 4 : 8;
   const size_t chunks = (size_t)ceil_div((int64_t)n, BWD_CHUNK);
@@ -628,20 +636,23 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
                            const uint32_t* bag_of_pos, int64_t N, const int64_t* offsets, int32_t pooling_mode,
                            const float* grad, int64_t grad_stride, float lr, float eps,
                            const int32_t* slot_of_lookup, const CachePtrs& caches, float* head, float* tail,
-                           float* group, cudaStream_t s) {
+                           float* group, uint32_t* next_chunk, cudaStream_t s) {
   const int64_t chunks = ceil_div(N, BWD_CHUNK);
   const unsigned grid = (unsigned)ceil_div(chunks, BWD_WARPS);
   if constexpr (NV == 1 && MTS_BWD_USE_LEAN) {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
-    const unsigned lean_grid = (unsigned)ceil_div(chunks, LEAN_WARPS);
+    // as many blocks as fit on the device at once (or fewer); the warps share out the chunks
+    const unsigned lean_grid =
+        (unsigned)std::min<int64_t>(ceil_div(chunks, LEAN_WARPS), (int64_t)h->sm_count * MTS_BWD_LEAN_MINBLK);
+    if (cudaMemsetAsync(next_chunk, 0, sizeof(uint32_t), s) != cudaSuccess) return check_launch("memset(next_chunk)");
     if (pooling_mode == MTS_POOL_MEAN)
       reduce_chunks_lean<FP16, true><<<lean_grid, LEAN_WARPS * 32, 0, s>>>(
           h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
-          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail);
+          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail, next_chunk);
     else
       reduce_chunks_lean<FP16, false><<<lean_grid, LEAN_WARPS * 32, 0, s>>>(
           h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
-          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail);
+          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail, next_chunk);
   } else {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
     if (pooling_mode == MTS_POOL_MEAN)
@@ -788,7 +799,7 @@ extern "C" int mts_tbe_backward_apply(const mts_tables* h, int32_t B, const int6
   float* group = reinterpret_cast<float*>(ws + L.group);
   const int nv = (h->max_dim + 127) / 128;
   const bool fp16 = h->dtype == MTS_DTYPE_FP16;
-#define MTS_BWD(F, V, G) return launch_backward<F, V, G>(h, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad_out, grad_stride, lr, eps, slot_of_lookup, caches, head, tail, group, s)
+#define MTS_BWD(F, V, G) return launch_backward<F, V, G>(h, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad_out, grad_stride, lr, eps, slot_of_lookup, caches, head, tail, group, reinterpret_cast<uint32_t*>(ws + L.next_chunk), s)
   if (fp16) {
     if (nv <= 1) MTS_BWD(true, 1, MTS_BWD_GROUP1);
     if (nv <= 2) MTS_BWD(true, 2, MTS_BWD_GROUP2);
