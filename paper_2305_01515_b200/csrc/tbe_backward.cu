@@ -188,7 +188,7 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
               const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches, char* dev_w,
                    char* host_w,
               float* __restrict__ momentum, float* __restrict__ partial_head,
-              float* __restrict__ partial_tail) {
+              float* __restrict__ partial_tail, uint32_t* __restrict__ next_chunk) {
   constexpr int EB = FP16 ? 2 : 4;
   constexpr int PSTRIDE = NV * 128;
   __shared__ uint4 s_desc[BWD_WARPS][32];      // {gradient float offset, key, row address lo, hi}
@@ -196,7 +196,11 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
   __shared__ uint8_t* s_dirty[BWD_WARPS][32];
   const int lane = threadIdx.x & 31;
   const int wib = threadIdx.x >> 5;
-  const int64_t chunk = (int64_t)blockIdx.x * BWD_WARPS + wib;
+  // a warp takes its next chunk from a counter: chunk costs differ a lot (see reduce_chunks_lean)
+  for (;;) {
+  uint32_t taken = 0;
+  if (lane == 0) taken = atomicAdd(next_chunk, 1u);
+  const int64_t chunk = (int64_t)__shfl_sync(0xffffffffu, taken, 0);
   const int64_t p0 = chunk * BWD_CHUNK;
   if (p0 >= n) return;
   const int64_t p1 = min(n, p0 + BWD_CHUNK);
@@ -316,6 +320,7 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
 #pragma unroll
     for (int q = 0; q < NV; ++q)
       *reinterpret_cast<float4*>(dst + chunk * PSTRIDE + (q * 32 + lane) * 4) = acc[q];
+  }
   }
 }
 
@@ -655,14 +660,17 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
           static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail, next_chunk);
   } else {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
+    constexpr int resident = NV == 1 ? MTS_BWD_MINBLK : NV == 2 ? MTS_BWD_MINBLK2 : 2;
+    const unsigned dyn_grid = (unsigned)std::min<int64_t>(grid, (int64_t)h->sm_count * resident);
+    if (cudaMemsetAsync(next_chunk, 0, sizeof(uint32_t), s) != cudaSuccess) return check_launch("memset(next_chunk)");
     if (pooling_mode == MTS_POOL_MEAN)
-      reduce_chunks<FP16, NV, GROUP, true><<<grid, BWD_WARPS * 32, 0, s>>>(
+      reduce_chunks<FP16, NV, GROUP, true><<<dyn_grid, BWD_WARPS * 32, 0, s>>>(
           h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
-          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail);
+          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail, next_chunk);
     else
-      reduce_chunks<FP16, NV, GROUP, false><<<grid, BWD_WARPS * 32, 0, s>>>(
+      reduce_chunks<FP16, NV, GROUP, false><<<dyn_grid, BWD_WARPS * 32, 0, s>>>(
           h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
-          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail);
+          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail, next_chunk);
   }
   if (chunks >= 2 * COMBINE_GROUP) {
     LaunchScope scope(K_COMBINE_PARTIALS, s);

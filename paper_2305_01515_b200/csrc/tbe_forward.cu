@@ -13,12 +13,15 @@ namespace mts {
 #define MTS_FWD_UNROLL 4         // load instructions issued back to back per lane
 #endif
 #ifndef MTS_FWD_MINBLK
-#define MTS_FWD_MINBLK 4         // resident blocks per SM the register allocation is bounded for
+#define MTS_FWD_MINBLK 8         // resident blocks per SM the register allocation is bounded for
 #endif
 #ifndef MTS_FWD_BAGS
 #define MTS_FWD_BAGS 4           // consecutive bags one warp walks through
 #endif
-constexpr int FWD_WARPS = 8;
+#ifndef MTS_FWD_WARPS
+#define MTS_FWD_WARPS 4
+#endif
+constexpr int FWD_WARPS = MTS_FWD_WARPS;
 constexpr int FWD_UNROLL = MTS_FWD_UNROLL;
 constexpr int FWD_BAGS = MTS_FWD_BAGS;
 static_assert(FWD_BAGS >= 1 && FWD_BAGS <= 30, "a warp keeps the offsets of its bags in its lanes");
