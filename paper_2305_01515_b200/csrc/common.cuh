@@ -124,6 +124,19 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // (*keys_out, *vals_out), which point at either the a or the b buffers.
 // hist: scratch of sort_hist_words() uint32.
 size_t sort_hist_words();
+// Segments of a segmented sort: segment t = positions [offsets[t*stride], offsets[(t+1)*stride]),
+// digits taken from key - meta[t].row_offset.
+struct SortSegments {
+  const int64_t* offsets;    // device
+  int32_t stride;
+  const TableMeta* meta;     // device
+};
+size_t sort_hist_words_segmented(int64_t n, int T);
+// Sorts every segment on its own by the low key_bits of (key - base of its segment); same buffers and
+// result convention as radix_sort_pairs, hist: sort_hist_words_segmented(n, T) uint32.
+int radix_sort_pairs_segmented(uint32_t* keys_a, uint32_t* vals_a, uint32_t* keys_b, uint32_t* vals_b, int64_t n,
+                               int T, const SortSegments& seg, int key_bits, uint32_t* hist, uint32_t** keys_out,
+                               uint32_t** vals_out, cudaStream_t stream);
 // n_max is the host-known element count or an upper bound of it; when n_dev is not null the
 // kernels use min(*n_dev, n_max) (a device-resident count) instead.
 int radix_sort_pairs(uint32_t* keys_a, uint32_t* vals_a, uint32_t* keys_b, uint32_t* vals_b,

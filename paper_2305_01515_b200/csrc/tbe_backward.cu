@@ -621,7 +621,7 @@ static BwdLayout bwd_layout(const mts_tables* h, int64_t N) {
   const size_t n = (size_t)(N > 0 ? N : 1);
   L.keys_a = take(n * 4); L.keys_b = take(n * 4); L.vals_a = take(n * 4); L.vals_b = take(n * 4);
   L.bag_of_pos = take(n * 4);
-  L.hist = take(sort_hist_words() * 4);
+  L.hist = take(std::max(sort_hist_words(), sort_hist_words_segmented((int64_t)n, h->T)) * 4);
   L.scan = take(scan_scratch_words() * 4);
   L.seg_start = take((n + 1) * 4);
   L.n_unique = take(256);
@@ -698,15 +698,32 @@ extern "C" size_t mts_tbe_backward_workspace_bytes(const mts_tables* h, int32_t 
 
 namespace {
 
-int key_bits_of(const mts_tables* h) {
-  int key_bits = 1;
-  while (key_bits < 32 && (1ll << key_bits) < h->total_rows) ++key_bits;
-  return key_bits;
+int bits_for(int64_t values) {
+  int bits = 1;
+  while (bits < 32 && (1ll << bits) < values) ++bits;
+  return bits;
 }
 
-// which of the two buffer pairs holds the sorted lookups after radix_sort_pairs
+// How the lookups are sorted by row.  They arrive grouped by table, so each table's lookups can be
+// sorted on their own on the bits of the row index inside the table; that is used when it saves a
+// pass over sorting the linear row ids of all tables together.
+struct SortPlan {
+  bool segmented;
+  int key_bits;
+  int passes() const { return (key_bits + 7) / 8; }
+};
+
+SortPlan sort_plan(const mts_tables* h) {
+  int64_t max_rows = 1;
+  for (const auto& m : h->h_meta) max_rows = std::max<int64_t>(max_rows, m.rows);
+  const int all_bits = bits_for(h->total_rows), table_bits = bits_for(max_rows);
+  if (h->T > 1 && (table_bits + 7) / 8 < (all_bits + 7) / 8) return {true, table_bits};
+  return {false, all_bits};
+}
+
+// which of the two buffer pairs holds the sorted lookups after the sort
 bool sorted_in_b(const mts_tables* h, int64_t N) {
-  return N > 1 && (((key_bits_of(h) + 7) / 8) & 1) != 0;
+  return N > 1 && (sort_plan(h).passes() & 1) != 0;
 }
 
 int check_backward_common(const mts_tables* h, int32_t B, const int64_t* offsets, int64_t N, void* workspace,
@@ -756,8 +773,15 @@ extern "C" int mts_tbe_backward_sort(const mts_tables* h, int32_t B, const int64
     if (rc != MTS_OK) return rc;
   }
   uint32_t *keys = nullptr, *pos = nullptr;
-  rc = radix_sort_pairs(keys_a, vals_a, keys_b, vals_b, N, nullptr, key_bits_of(h), reinterpret_cast<uint32_t*>(ws + L.hist),
-                        &keys, &pos, s);
+  const SortPlan plan = sort_plan(h);
+  if (plan.segmented) {
+    const SortSegments seg{offsets, B, h->d_meta};
+    rc = radix_sort_pairs_segmented(keys_a, vals_a, keys_b, vals_b, N, h->T, seg, plan.key_bits,
+                                    reinterpret_cast<uint32_t*>(ws + L.hist), &keys, &pos, s);
+  } else {
+    rc = radix_sort_pairs(keys_a, vals_a, keys_b, vals_b, N, nullptr, plan.key_bits,
+                          reinterpret_cast<uint32_t*>(ws + L.hist), &keys, &pos, s);
+  }
   if (rc != MTS_OK) return rc;
   if ((keys == keys_b) != sorted_in_b(h, N)) return set_error(MTS_ERR_CUDA, "tbe_backward_sort: unexpected result buffer");
   if (uniq_rows_out) {

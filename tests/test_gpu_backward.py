@@ -217,3 +217,14 @@ def test_backward_in_two_calls_matches_one_call():
     assert torch.equal(results[0][0], results[1][0])
     assert torch.equal(results[0][1], results[1][1])
     assert torch.equal(results[0][2], results[1][2])
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("rows,pool,B", [
+    ([250, 200, 256, 100, 255], [7, 0.02, 30, 3, 12], 257),          # 1 pass per table instead of 2; a nearly empty table
+    ([60000, 65536, 40000], [40, 25, 33], 600),                      # 2 passes instead of 3; several tiles per table
+])
+def test_tables_sorted_separately(rows, pool, B):
+    """Table sets for which the lookups of each table are sorted on their own (fewer digit passes)."""
+    spec = custom_spec(rows, [64] * len(rows), B, wl.FP16, pool, [1.1] * len(rows), seed=5)
+    _run_steps(spec, n_steps=2)
