@@ -18,7 +18,10 @@ namespace mts {
 
 constexpr int SORT_THREADS = 256;
 constexpr int SORT_WARPS = SORT_THREADS / 32;
-constexpr int SORT_ITEMS = 16;
+#ifndef MTS_SORT_ITEMS
+#define MTS_SORT_ITEMS 16
+#endif
+constexpr int SORT_ITEMS = MTS_SORT_ITEMS;
 constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;   // 4096 pairs
 constexpr int SORT_BINS = 256;
 constexpr int SORT_MAX_BLOCKS = 1024;
