@@ -360,7 +360,7 @@ def run_native(args, rank: int, world: int, local_rank: int):
             sum(spec.tables[t].pooling for t in range(spec.T))
         alg = {
             "tbe_forward_kernel": n_avg * (per_lookup + 8) + 8 * (spec.T * B + 1) + 4.0 * B * TD,
-            "reduce_chunks": n_avg * (per_lookup + 12),
+            "reduce_chunks": n_avg * (per_lookup + 8),      # row-equivalent + sorted key and bag id
         }
         # dram__bytes_read + dram__bytes_write per lookup from the ncu capture summarised in
         # profiles/ncu_full_cfg2_8tables_top_kernels.md (1.967 M lookups per launch there); DRAM traffic

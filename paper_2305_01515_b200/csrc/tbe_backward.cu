@@ -2,8 +2,8 @@
 // optimizer with few states per row; Section 5.9: aggregate, optimize, write rows back).
 //
 // Steps, all on the caller's stream, no host synchronisation:
-//   1. linearize_lookups : key = linear row id of every lookup, value = its position,
-//                          bag_of_pos[position] = bag id
+//   1. linearize_lookups : key = linear row id of every lookup, value = its position and
+//                          bag_of_pos[position] = bag id (value = bag id when no table is cached)
 //   2. radix_sort_pairs  : stable sort by key; equal rows keep ascending position
 //   3. reduce_chunks     : one warp per CHUNK consecutive sorted lookups.  Gradients of a row
 //                          are summed in sorted order; a row whose lookups lie inside the
@@ -70,8 +70,12 @@ linearize_lookups(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B,
   for (int64_t i = offsets[bag] + sub; i < i1; i += LIN_GROUP) {
     const int64_t idx = clamp_index(indices[i], rows, status);
     keys[i] = (uint32_t)(roff + idx);
-    vals[i] = (uint32_t)i;
-    bag_of_pos[i] = (uint32_t)bag;
+    if (bag_of_pos != nullptr) {
+      vals[i] = (uint32_t)i;
+      bag_of_pos[i] = (uint32_t)bag;
+    } else {
+      vals[i] = (uint32_t)bag;       // no cached table: nothing needs the position, the bag id travels with the key
+    }
   }
 }
 
@@ -221,7 +225,7 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
       const uint32_t key = keys[p];
       my_end = (p + 1 >= n) || keys[p + 1] != key;
       const uint32_t ps = pos[p];
-      const uint32_t bag = bag_of_pos[ps];
+      const uint32_t bag = bag_of_pos != nullptr ? bag_of_pos[ps] : ps;
       const int t = (int)(bag / (uint32_t)B);
       const int b = (int)(bag - (uint32_t)t * (uint32_t)B);
       const TableMeta m = meta[t];
@@ -372,7 +376,7 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
       const uint32_t key = keys[p];
       my_end = (p + 1 >= n) || keys[p + 1] != key;
       const uint32_t ps = pos[p];
-      const uint32_t bag = bag_of_pos[ps];
+      const uint32_t bag = bag_of_pos != nullptr ? bag_of_pos[ps] : ps;
       const int t = (int)(bag / (uint32_t)B);
       const int b = (int)(bag - (uint32_t)t * (uint32_t)B);
       const TableMeta m = meta[t];
@@ -760,7 +764,8 @@ extern "C" int mts_tbe_backward_sort(const mts_tables* h, int32_t B, const int64
   uint32_t* keys_b = reinterpret_cast<uint32_t*>(ws + L.keys_b);
   uint32_t* vals_a = reinterpret_cast<uint32_t*>(ws + L.vals_a);
   uint32_t* vals_b = reinterpret_cast<uint32_t*>(ws + L.vals_b);
-  uint32_t* bag_of_pos = reinterpret_cast<uint32_t*>(ws + L.bag_of_pos);
+  // positions are only needed to find a lookup's cache slot; without cached tables the sorted value is the bag id
+  uint32_t* bag_of_pos = h->any_cached ? reinterpret_cast<uint32_t*>(ws + L.bag_of_pos) : nullptr;
   const int64_t n_bags = (int64_t)h->T * B;
   {
     const int64_t threads = n_bags * LIN_GROUP;
@@ -825,7 +830,7 @@ extern "C" int mts_tbe_backward_apply(const mts_tables* h, int32_t B, const int6
   const bool in_b = sorted_in_b(h, N);
   const uint32_t* keys = reinterpret_cast<const uint32_t*>(ws + (in_b ? L.keys_b : L.keys_a));
   const uint32_t* pos = reinterpret_cast<const uint32_t*>(ws + (in_b ? L.vals_b : L.vals_a));
-  const uint32_t* bag_of_pos = reinterpret_cast<const uint32_t*>(ws + L.bag_of_pos);
+  const uint32_t* bag_of_pos = h->any_cached ? reinterpret_cast<const uint32_t*>(ws + L.bag_of_pos) : nullptr;
   float* head = reinterpret_cast<float*>(ws + L.head);
   float* tail = reinterpret_cast<float*>(ws + L.tail);
   float* group = reinterpret_cast<float*>(ws + L.group);
