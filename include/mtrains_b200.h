@@ -183,6 +183,24 @@ int mts_tbe_backward_apply(const mts_tables* tables, int32_t B, const int64_t* o
                            uint8_t* const* host_cache_dirty, int32_t n_caches, void* workspace,
                            size_t workspace_bytes, void* stream);
 
+/* The same forward and gradient half of the backward with fp16 tensors on the dense side (the
+ * paper's operators pool rows into an output that the dense network consumes, Section 2.1.1; it
+ * does not fix that output's type).  out_f16 / grad_out_f16: device, IEEE binary16, [B, out_stride]
+ * and [B, grad_stride] in elements, 16-byte aligned, strides multiples of 4.  The pooled sum is
+ * accumulated in fp32 and rounded to nearest even once; the gradient is converted exactly to fp32
+ * and everything after that is the arithmetic of the fp32 entry points.  Halves the bytes of the
+ * output and, in the backward, of the gradient slices read once per lookup.  Other arguments,
+ * ordering rules (mts_tbe_backward_sort first) and errors as for the fp32 entry points. */
+int mts_tbe_forward_f16(const mts_tables* tables, int32_t B, const int64_t* indices,
+                        const int64_t* offsets, int64_t N, int32_t pooling_mode,
+                        const int32_t* slot_of_lookup, void* const* host_cache_data, int32_t n_caches,
+                        void* out_f16, int64_t out_stride, void* stream);
+int mts_tbe_backward_apply_f16(const mts_tables* tables, int32_t B, const int64_t* offsets, int64_t N,
+                               int32_t pooling_mode, const void* grad_out_f16, int64_t grad_stride,
+                               float lr, float eps, const int32_t* slot_of_lookup,
+                               void* const* host_cache_data, uint8_t* const* host_cache_dirty,
+                               int32_t n_caches, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Backward without a workspace argument and without any allocation (the paper has no
  * counterpart; this exists for callers of this library that cannot allocate device memory).
  * Such callers are, for example, a training or serving loop embedded in a framework that

@@ -29,6 +29,7 @@ EXPORTS = (
     "mts_trace_kernel_name", "mts_trace_report", "mts_tables_create", "mts_tables_destroy", "mts_tables_status",
     "mts_tbe_forward", "mts_tbe_backward_workspace_bytes", "mts_tbe_backward_rowwise_adagrad",
     "mts_tbe_backward_rowwise_adagrad_static", "mts_tbe_backward_sort", "mts_tbe_backward_apply",
+    "mts_tbe_forward_f16", "mts_tbe_backward_apply_f16",
     "mts_cache_create", "mts_cache_destroy", "mts_cache_status", "mts_cache_data", "mts_cache_dirty",
     "mts_linearize_keys", "mts_cache_workspace_bytes", "mts_cache_lookup_insert",
     "mts_cache_prefetch_misses", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
@@ -86,6 +87,8 @@ def lib():
         L.mts_tbe_backward_sort.argtypes = [vp, i32, vp, vp, i64, vp, sz, vp, vp, vp]
         L.mts_tbe_backward_apply.argtypes = [vp, i32, vp, i64, i32, vp, i64, f32, f32, vp, C.POINTER(vp),
                                              C.POINTER(vp), i32, vp, sz, vp]
+        L.mts_tbe_forward_f16.argtypes = L.mts_tbe_forward.argtypes
+        L.mts_tbe_backward_apply_f16.argtypes = L.mts_tbe_backward_apply.argtypes
         L.mts_cache_create.argtypes = [C.POINTER(vp), i64, i64, i32, i32, i32, i32, i32]
         L.mts_cache_destroy.argtypes = [vp]
         L.mts_cache_status.argtypes = [vp, C.POINTER(i32), vp]
@@ -201,9 +204,11 @@ def tables_create(dtype, rows, dim, weight_offset, cache_id, dev_weights, host_w
 
 
 def tbe_forward(tables: Tables, B: int, indices, offsets, N: int, pooling_mode: int, slot_of_lookup,
-                cache_data: Optional[Sequence], out, out_stride: int, stream=None) -> None:
+                cache_data: Optional[Sequence], out, out_stride: int, stream=None, f16: bool = False) -> None:
+    """f16: `out` holds IEEE binary16 (mts_tbe_forward_f16), else fp32."""
     n_caches = len(cache_data) if cache_data is not None else 0
-    _check(lib().mts_tbe_forward(tables.handle, B, _ptr(indices), _ptr(offsets), N, pooling_mode,
+    fn = lib().mts_tbe_forward_f16 if f16 else lib().mts_tbe_forward
+    _check(fn(tables.handle, B, _ptr(indices), _ptr(offsets), N, pooling_mode,
                                  _ptr(slot_of_lookup), _ptr_array(cache_data, n_caches), n_caches, _ptr(out),
                                  out_stride, _stream(stream)))
 
@@ -232,10 +237,13 @@ def tbe_backward_sort(tables: Tables, B: int, indices, offsets, N: int, workspac
 
 def tbe_backward_apply(tables: Tables, B: int, offsets, N: int, pooling_mode: int, grad_out, grad_stride: int,
                        lr: float, eps: float, slot_of_lookup, cache_data: Optional[Sequence],
-                       cache_dirty: Optional[Sequence], workspace, workspace_bytes: int, stream=None) -> None:
-    """Second half: per-row gradient sums and the optimizer, on the workspace tbe_backward_sort left."""
+                       cache_dirty: Optional[Sequence], workspace, workspace_bytes: int, stream=None,
+                       f16: bool = False) -> None:
+    """Second half: per-row gradient sums and the optimizer, on the workspace tbe_backward_sort left.
+    f16: `grad_out` holds IEEE binary16 (mts_tbe_backward_apply_f16), else fp32."""
     n_caches = len(cache_data) if cache_data is not None else 0
-    _check(lib().mts_tbe_backward_apply(
+    fn = lib().mts_tbe_backward_apply_f16 if f16 else lib().mts_tbe_backward_apply
+    _check(fn(
         tables.handle, B, _ptr(offsets), N, pooling_mode, _ptr(grad_out), grad_stride, lr, eps,
         _ptr(slot_of_lookup), _ptr_array(cache_data, n_caches), _ptr_array(cache_dirty, n_caches), n_caches,
         _ptr(workspace), workspace_bytes, _stream(stream)))

@@ -115,6 +115,18 @@ __device__ __forceinline__ RowTarget row_target(const TableMeta& m, int64_t key,
   return r;
 }
 
+// Four consecutive values of the upstream gradient starting at element `elem` (fp32, or fp16 when GH).
+template <bool GH>
+__device__ __forceinline__ float4 load_grad4(const void* __restrict__ grad, int64_t elem) {
+  if (GH) {
+    const uint2 v = __ldg(reinterpret_cast<const uint2*>(static_cast<const __half*>(grad) + elem));
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&v.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+  }
+  return __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(grad) + elem));
+}
+
 // Row-wise Adagrad on one row held across the warp: lane owns columns (q*32 + lane)*4 .. +3.
 // m += mean(g^2); W -= lr * g / (sqrt(m) + eps).  inv_dim = __frcp_rn(dim), hoisted by the callers.
 template <bool FP16, int NV>
@@ -182,13 +194,13 @@ __device__ __forceinline__ void load_row(uint4 (&wraw)[NV], const char* wptr, in
 // result in shared memory; then the warp walks the 32 lookups in order, GROUP at a time: the
 // loads of a whole group (gradient slices, and row + Adagrad state where a row ends) are issued
 // before the first one is used.
-template <bool FP16, int NV, int GROUP, bool MEAN>
+template <bool FP16, int NV, int GROUP, bool MEAN, bool GH>
 __global__ void __launch_bounds__(BWD_WARPS * 32, (NV == 1 ? MTS_BWD_MINBLK : NV == 2 ? MTS_BWD_MINBLK2 : 1))
 reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
               const uint32_t* __restrict__ keys, const uint32_t* __restrict__ pos,
               const uint32_t* __restrict__ bag_of_pos, int64_t n,
               const int64_t* __restrict__ offsets,
-              const float* __restrict__ grad, int64_t grad_stride, float lr, float eps,
+              const void* __restrict__ grad, int64_t grad_stride, float lr, float eps,
               const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches, char* dev_w,
                    char* host_w,
               float* __restrict__ momentum, float* __restrict__ partial_head,
@@ -267,11 +279,11 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
         if (j < cnt) {
           const uint4 d = s_desc[wib][j];
           const int dim = uniform ? dim0 : (int)s_aux[wib][j].x;
-          const float* gp = grad + d.x;
+          const int64_t gp = d.x;
 #pragma unroll
           for (int q = 0; q < NV; ++q) {
             const int c = (q * 32 + lane) * 4;
-            g[u][q] = c < dim ? __ldg(reinterpret_cast<const float4*>(gp + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            g[u][q] = c < dim ? load_grad4<GH>(grad, gp + c) : make_float4(0.f, 0.f, 0.f, 0.f);
           }
           if ((ends >> j) & 1u) {
             const char* wp = reinterpret_cast<const char*>((uintptr_t)d.z | ((uintptr_t)d.w << 32));
@@ -333,13 +345,13 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
 // bytes in flight, so this form keeps one lookup in flight per warp, fits 32 registers and runs 64
 // warps per SM; a row's loads (gradient slice, and row + state where the row ends) are issued
 // together.  Same summation order and arithmetic as reduce_chunks.
-template <bool FP16, bool MEAN>
+template <bool FP16, bool MEAN, bool GH>
 __global__ void __launch_bounds__(LEAN_WARPS * 32, MTS_BWD_LEAN_MINBLK)
 reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
                    const uint32_t* __restrict__ keys, const uint32_t* __restrict__ pos,
                    const uint32_t* __restrict__ bag_of_pos, int64_t n,
                    const int64_t* __restrict__ offsets,
-                   const float* __restrict__ grad, int64_t grad_stride, float lr, float eps,
+                   const void* __restrict__ grad, int64_t grad_stride, float lr, float eps,
                    const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches, char* dev_w,
                    char* host_w,
                    float* __restrict__ momentum, float* __restrict__ partial_head,
@@ -351,7 +363,7 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
   __shared__ uint8_t* s_dirty[LEAN_WARPS][32];
   const int lane = threadIdx.x & 31;
   const int wib = threadIdx.x >> 5;
-  const float* grad_lane = grad + lane * 4;
+  const int64_t lane_elem = lane * 4;
   // Chunks differ a lot in cost (a chunk inside one hot row is a plain sum, a chunk of rows seen
   // once is 128 updates), so a warp takes its next chunk from a counter instead of a fixed share.
   for (;;) {
@@ -430,7 +442,7 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
     auto load_grad = [&](int jj) {
       const int dim = FULL ? 128 : uniform ? dim0 : (int)s_aux[wib][jj].x;
       float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (FULL || lane * 4 < dim) g = __ldg(reinterpret_cast<const float4*>(grad_lane + s_desc[wib][jj].x));
+      if (FULL || lane * 4 < dim) g = load_grad4<GH>(grad, lane_elem + s_desc[wib][jj].x);
       return g;
     };
     int j = 0;
@@ -449,7 +461,7 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
         const uint4 d = s_desc[wib][e];
         const int dim = FULL ? 128 : uniform ? dim0 : (int)s_aux[wib][e].x;
         float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (FULL || lane * 4 < dim) g = __ldg(reinterpret_cast<const float4*>(grad_lane + d.x));
+        if (FULL || lane * 4 < dim) g = load_grad4<GH>(grad, lane_elem + d.x);
         if (open_head) {
           add_scaled(g, e);
           *reinterpret_cast<float4*>(partial_head + chunk * PSTRIDE + lane * 4) = acc;
@@ -643,11 +655,28 @@ static BwdLayout bwd_layout(const mts_tables* h, int64_t N) {
 template <bool FP16, int NV, int GROUP>
 static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys, const uint32_t* pos,
                            const uint32_t* bag_of_pos, int64_t N, const int64_t* offsets, int32_t pooling_mode,
-                           const float* grad, int64_t grad_stride, float lr, float eps,
+                           const void* grad, bool grad_half, int64_t grad_stride, float lr, float eps,
                            const int32_t* slot_of_lookup, const CachePtrs& caches, float* head, float* tail,
                            float* group, uint32_t* next_chunk, cudaStream_t s) {
   const int64_t chunks = ceil_div(N, BWD_CHUNK);
   const unsigned grid = (unsigned)ceil_div(chunks, BWD_WARPS);
+  // the reduce kernels exist for fp32 and for fp16 upstream gradients
+#define COMMA ,
+#define MTS_LAUNCH_GH(KERNEL, TARGS, GRID, THREADS)                                                                  \
+  do {                                                                                                               \
+    if (grad_half)                                                                                                   \
+      KERNEL<TARGS, true><<<GRID, THREADS, 0, s>>>(h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad,     \
+                                                    grad_stride, lr, eps, slot_of_lookup, caches,                    \
+                                                    static_cast<char*>(h->dev_weights),                              \
+                                                    static_cast<char*>(h->host_weights), h->momentum, head, tail,    \
+                                                    next_chunk);                                                     \
+    else                                                                                                             \
+      KERNEL<TARGS, false><<<GRID, THREADS, 0, s>>>(h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad,    \
+                                                     grad_stride, lr, eps, slot_of_lookup, caches,                   \
+                                                     static_cast<char*>(h->dev_weights),                             \
+                                                     static_cast<char*>(h->host_weights), h->momentum, head, tail,   \
+                                                     next_chunk);                                                    \
+  } while (0)
   if constexpr (NV == 1 && MTS_BWD_USE_LEAN) {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
     // as many blocks as fit on the device at once (or fewer); the warps share out the chunks
@@ -655,26 +684,18 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
         (unsigned)std::min<int64_t>(ceil_div(chunks, LEAN_WARPS), (int64_t)h->sm_count * MTS_BWD_LEAN_MINBLK);
     if (cudaMemsetAsync(next_chunk, 0, sizeof(uint32_t), s) != cudaSuccess) return check_launch("memset(next_chunk)");
     if (pooling_mode == MTS_POOL_MEAN)
-      reduce_chunks_lean<FP16, true><<<lean_grid, LEAN_WARPS * 32, 0, s>>>(
-          h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
-          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail, next_chunk);
+      MTS_LAUNCH_GH(reduce_chunks_lean, FP16 COMMA true, lean_grid, LEAN_WARPS * 32);
     else
-      reduce_chunks_lean<FP16, false><<<lean_grid, LEAN_WARPS * 32, 0, s>>>(
-          h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
-          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail, next_chunk);
+      MTS_LAUNCH_GH(reduce_chunks_lean, FP16 COMMA false, lean_grid, LEAN_WARPS * 32);
   } else {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
     constexpr int resident = NV == 1 ? MTS_BWD_MINBLK : NV == 2 ? MTS_BWD_MINBLK2 : 2;
     const unsigned dyn_grid = (unsigned)std::min<int64_t>(grid, (int64_t)h->sm_count * resident);
     if (cudaMemsetAsync(next_chunk, 0, sizeof(uint32_t), s) != cudaSuccess) return check_launch("memset(next_chunk)");
     if (pooling_mode == MTS_POOL_MEAN)
-      reduce_chunks<FP16, NV, GROUP, true><<<dyn_grid, BWD_WARPS * 32, 0, s>>>(
-          h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
-          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail, next_chunk);
+      MTS_LAUNCH_GH(reduce_chunks, FP16 COMMA NV COMMA GROUP COMMA true, dyn_grid, BWD_WARPS * 32);
     else
-      reduce_chunks<FP16, NV, GROUP, false><<<dyn_grid, BWD_WARPS * 32, 0, s>>>(
-          h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup, caches,
-          static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, head, tail, next_chunk);
+      MTS_LAUNCH_GH(reduce_chunks, FP16 COMMA NV COMMA GROUP COMMA false, dyn_grid, BWD_WARPS * 32);
   }
   if (chunks >= 2 * COMBINE_GROUP) {
     LaunchScope scope(K_COMBINE_PARTIALS, s);
@@ -687,6 +708,8 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
         h->d_meta, h->T, keys, pos, N, lr, eps, slot_of_lookup, caches, static_cast<char*>(h->dev_weights),
         static_cast<char*>(h->host_weights), h->momentum, head, tail, group);
   }
+#undef MTS_LAUNCH_GH
+#undef COMMA
   return check_launch("reduce_chunks / combine_partials");
 }
 
@@ -804,11 +827,11 @@ extern "C" int mts_tbe_backward_sort(const mts_tables* h, int32_t B, const int64
   return MTS_OK;
 }
 
-extern "C" int mts_tbe_backward_apply(const mts_tables* h, int32_t B, const int64_t* offsets, int64_t N,
-                                      int32_t pooling_mode, const float* grad_out, int64_t grad_stride, float lr,
-                                      float eps, const int32_t* slot_of_lookup, void* const* host_cache_data,
-                                      uint8_t* const* host_cache_dirty, int32_t n_caches, void* workspace,
-                                      size_t workspace_bytes, void* stream) {
+namespace {
+int backward_apply(const mts_tables* h, int32_t B, const int64_t* offsets, int64_t N, int32_t pooling_mode,
+                   const void* grad_out, bool grad_half, int64_t grad_stride, float lr, float eps,
+                   const int32_t* slot_of_lookup, void* const* host_cache_data, uint8_t* const* host_cache_dirty,
+                   int32_t n_caches, void* workspace, size_t workspace_bytes, void* stream) {
   if (!h) return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_apply: null tables");
   const BwdLayout L = bwd_layout(h, N > 0 ? N : 0);
   int rc = check_backward_common(h, B, offsets, N, workspace, workspace_bytes, L, "tbe_backward_apply");
@@ -836,7 +859,7 @@ extern "C" int mts_tbe_backward_apply(const mts_tables* h, int32_t B, const int6
   float* group = reinterpret_cast<float*>(ws + L.group);
   const int nv = (h->max_dim + 127) / 128;
   const bool fp16 = h->dtype == MTS_DTYPE_FP16;
-#define MTS_BWD(F, V, G) return launch_backward<F, V, G>(h, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad_out, grad_stride, lr, eps, slot_of_lookup, caches, head, tail, group, reinterpret_cast<uint32_t*>(ws + L.next_chunk), s)
+#define MTS_BWD(F, V, G) return launch_backward<F, V, G>(h, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad_out, grad_half, grad_stride, lr, eps, slot_of_lookup, caches, head, tail, group, reinterpret_cast<uint32_t*>(ws + L.next_chunk), s)
   if (fp16) {
     if (nv <= 1) MTS_BWD(true, 1, MTS_BWD_GROUP1);
     if (nv <= 2) MTS_BWD(true, 2, MTS_BWD_GROUP2);
@@ -849,6 +872,25 @@ extern "C" int mts_tbe_backward_apply(const mts_tables* h, int32_t B, const int6
     MTS_BWD(false, 8, 1);
   }
 #undef MTS_BWD
+}
+}  // namespace
+
+extern "C" int mts_tbe_backward_apply(const mts_tables* h, int32_t B, const int64_t* offsets, int64_t N,
+                                      int32_t pooling_mode, const float* grad_out, int64_t grad_stride, float lr,
+                                      float eps, const int32_t* slot_of_lookup, void* const* host_cache_data,
+                                      uint8_t* const* host_cache_dirty, int32_t n_caches, void* workspace,
+                                      size_t workspace_bytes, void* stream) {
+  return backward_apply(h, B, offsets, N, pooling_mode, grad_out, false, grad_stride, lr, eps, slot_of_lookup,
+                        host_cache_data, host_cache_dirty, n_caches, workspace, workspace_bytes, stream);
+}
+
+extern "C" int mts_tbe_backward_apply_f16(const mts_tables* h, int32_t B, const int64_t* offsets, int64_t N,
+                                          int32_t pooling_mode, const void* grad_out_f16, int64_t grad_stride,
+                                          float lr, float eps, const int32_t* slot_of_lookup,
+                                          void* const* host_cache_data, uint8_t* const* host_cache_dirty,
+                                          int32_t n_caches, void* workspace, size_t workspace_bytes, void* stream) {
+  return backward_apply(h, B, offsets, N, pooling_mode, grad_out_f16, true, grad_stride, lr, eps, slot_of_lookup,
+                        host_cache_data, host_cache_dirty, n_caches, workspace, workspace_bytes, stream);
 }
 
 extern "C" int mts_tbe_backward_rowwise_adagrad(

@@ -35,7 +35,7 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
                    const int64_t* __restrict__ indices, const int64_t* __restrict__ offsets,
                    const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches,
                    const char* __restrict__ dev_w, const char* __restrict__ host_w,
-                   int32_t pooling_mode, float* __restrict__ out, int64_t out_stride,
+                   int32_t pooling_mode, void* __restrict__ out, bool out_half, int64_t out_stride,
                    int32_t* status) {
   constexpr int EPC = FP16 ? 8 : 4;       // elements per 16-byte chunk
   constexpr int EB = FP16 ? 2 : 4;
@@ -145,15 +145,34 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
     if (sub == 0) {
       float scale = 1.f;
       if (pooling_mode == MTS_POOL_MEAN && i1 > i0) scale = 1.f / (float)(i1 - i0);
-      float* o = out + (int64_t)b * out_stride + m.out_offset;
+      const int64_t o = (int64_t)b * out_stride + m.out_offset;     // element offset of the bag's slice
 #pragma unroll
       for (int q = 0; q < NV; ++q) {
         const int c = cl + q * 32;
         if (c < vec16) {
-          float4* dst = reinterpret_cast<float4*>(o + c * EPC);
-          dst[0] = make_float4(acc[q][0] * scale, acc[q][1] * scale, acc[q][2] * scale, acc[q][3] * scale);
-          if (FP16)
-            dst[1] = make_float4(acc[q][4] * scale, acc[q][5] * scale, acc[q][6] * scale, acc[q][7] * scale);
+          if (out_half) {
+            // pooled sums rounded to fp16 (round to nearest even), EPC values = EPC * 2 bytes
+            __half2 h01 = __floats2half2_rn(acc[q][0] * scale, acc[q][1] * scale);
+            __half2 h23 = __floats2half2_rn(acc[q][2] * scale, acc[q][3] * scale);
+            uint2 lo;
+            lo.x = *reinterpret_cast<uint32_t*>(&h01);
+            lo.y = *reinterpret_cast<uint32_t*>(&h23);
+            __half* dst = static_cast<__half*>(out) + o + c * EPC;
+            *reinterpret_cast<uint2*>(dst) = lo;
+            if (FP16) {
+              __half2 h45 = __floats2half2_rn(acc[q][4] * scale, acc[q][5] * scale);
+              __half2 h67 = __floats2half2_rn(acc[q][6] * scale, acc[q][7] * scale);
+              uint2 hi;
+              hi.x = *reinterpret_cast<uint32_t*>(&h45);
+              hi.y = *reinterpret_cast<uint32_t*>(&h67);
+              *reinterpret_cast<uint2*>(dst + 4) = hi;
+            }
+          } else {
+            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(out) + o + c * EPC);
+            dst[0] = make_float4(acc[q][0] * scale, acc[q][1] * scale, acc[q][2] * scale, acc[q][3] * scale);
+            if (FP16)
+              dst[1] = make_float4(acc[q][4] * scale, acc[q][5] * scale, acc[q][6] * scale, acc[q][7] * scale);
+          }
         }
       }
     }
@@ -163,7 +182,7 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
 template <bool FP16, int NV>
 static int launch_forward(const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets,
                           int32_t pooling_mode, const int32_t* slot_of_lookup, const CachePtrs& caches,
-                          float* out, int64_t out_stride, cudaStream_t stream) {
+                          void* out, bool out_half, int64_t out_stride, cudaStream_t stream) {
   const int64_t n_bags = (int64_t)h->T * B;
   const int64_t grid = ceil_div(n_bags, (int64_t)FWD_WARPS * FWD_BAGS);
   {
@@ -171,7 +190,7 @@ static int launch_forward(const mts_tables* h, int32_t B, const int64_t* indices
     tbe_forward_kernel<FP16, NV><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
         h->d_meta, n_bags, B, indices, offsets, slot_of_lookup, caches,
         static_cast<const char*>(h->dev_weights), static_cast<const char*>(h->host_weights), pooling_mode,
-        out, out_stride, h->d_status);
+        out, out_half, out_stride, h->d_status);
   }
   return check_launch("tbe_forward_kernel");
 }
@@ -197,10 +216,10 @@ int fill_cache_ptrs(const mts_tables* h, void* const* host_cache_data, uint8_t* 
 
 using namespace mts;
 
-extern "C" int mts_tbe_forward(const mts_tables* h, int32_t B, const int64_t* indices,
-                               const int64_t* offsets, int64_t N, int32_t pooling_mode,
-                               const int32_t* slot_of_lookup, void* const* host_cache_data,
-                               int32_t n_caches, float* out, int64_t out_stride, void* stream) {
+namespace {
+int forward_any(const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets, int64_t N,
+                int32_t pooling_mode, const int32_t* slot_of_lookup, void* const* host_cache_data, int32_t n_caches,
+                void* out, bool out_half, int64_t out_stride, void* stream) {
   if (!h || !offsets || !out || B < 1 || N < 0 || (N > 0 && !indices))
     return set_error(MTS_ERR_INVALID_ARG, "tbe_forward: null argument or bad size");
   if (pooling_mode != MTS_POOL_SUM && pooling_mode != MTS_POOL_MEAN)
@@ -217,7 +236,7 @@ extern "C" int mts_tbe_forward(const mts_tables* h, int32_t B, const int64_t* in
   const int max_vec = h->max_dim * h->elem_bytes / 16;
   const int nv = max_vec <= 32 ? 1 : max_vec <= 64 ? 2 : max_vec <= 128 ? 4 : 8;
   const bool fp16 = h->dtype == MTS_DTYPE_FP16;
-#define MTS_FWD(F, V) return launch_forward<F, V>(h, B, indices, offsets, pooling_mode, slot_of_lookup, caches, out, out_stride, s)
+#define MTS_FWD(F, V) return launch_forward<F, V>(h, B, indices, offsets, pooling_mode, slot_of_lookup, caches, out, out_half, out_stride, s)
   if (fp16) {
     if (nv == 1) MTS_FWD(true, 1);
     if (nv == 2) MTS_FWD(true, 2);
@@ -229,4 +248,21 @@ extern "C" int mts_tbe_forward(const mts_tables* h, int32_t B, const int64_t* in
     MTS_FWD(false, 8);
   }
 #undef MTS_FWD
+}
+}  // namespace
+
+extern "C" int mts_tbe_forward(const mts_tables* h, int32_t B, const int64_t* indices,
+                               const int64_t* offsets, int64_t N, int32_t pooling_mode,
+                               const int32_t* slot_of_lookup, void* const* host_cache_data,
+                               int32_t n_caches, float* out, int64_t out_stride, void* stream) {
+  return forward_any(h, B, indices, offsets, N, pooling_mode, slot_of_lookup, host_cache_data, n_caches, out, false,
+                     out_stride, stream);
+}
+
+extern "C" int mts_tbe_forward_f16(const mts_tables* h, int32_t B, const int64_t* indices,
+                                   const int64_t* offsets, int64_t N, int32_t pooling_mode,
+                                   const int32_t* slot_of_lookup, void* const* host_cache_data,
+                                   int32_t n_caches, void* out_f16, int64_t out_stride, void* stream) {
+  return forward_any(h, B, indices, offsets, N, pooling_mode, slot_of_lookup, host_cache_data, n_caches, out_f16, true,
+                     out_stride, stream);
 }

@@ -124,13 +124,17 @@ class DeviceModel:
             out = torch.empty((self.spec.batch, self.spec.total_dim), dtype=torch.float32, device=self.device)
         slot = self.ctx[self.cur if ctx is None else ctx]["slot"] if self.cached else None
         mb.tbe_forward(self.tables, self.spec.batch, indices, offsets, N, pooling_mode, slot, self.cache_data, out,
-                       out.shape[1], stream)
+                       out.shape[1], stream, f16=out.dtype == torch.float16)
         return out
 
     def backward(self, indices, offsets, N: int, grad_out, lr: Optional[float] = None, eps: Optional[float] = None,
                  pooling_mode: int = mb.POOL_SUM, uniq_rows_out=None, n_unique_out=None, stream=None,
                  ctx: Optional[int] = None) -> None:
         self.reserve(N)
+        if grad_out.dtype == torch.float16:      # fp16 gradients: the two-call form
+            self.backward_sort(indices, offsets, N, uniq_rows_out, n_unique_out, stream)
+            self.backward_apply(offsets, N, grad_out, lr, eps, pooling_mode, stream, ctx)
+            return
         slot = self.ctx[self.cur if ctx is None else ctx]["slot"] if self.cached else None
         mb.tbe_backward_rowwise_adagrad(
             self.tables, self.spec.batch, indices, offsets, N, pooling_mode, grad_out, grad_out.shape[1],
@@ -151,7 +155,8 @@ class DeviceModel:
         mb.tbe_backward_apply(
             self.tables, self.spec.batch, offsets, N, pooling_mode, grad_out, grad_out.shape[1],
             self.spec.lr if lr is None else lr, self.spec.eps if eps is None else eps,
-            slot, self.cache_data, self.cache_dirty, self.workspace, self.ws_bytes, stream)
+            slot, self.cache_data, self.cache_dirty, self.workspace, self.ws_bytes, stream,
+            f16=grad_out.dtype == torch.float16)
 
     def group_range(self, g: int, offsets_host: np.ndarray):
         """Lookup range [begin, begin + n) of cache group g in one batch (host-side CSR)."""

@@ -16,8 +16,10 @@ def _weights_f64(spec, W):
     return W.astype(np.float64)
 
 
-def _run_steps(spec, n_steps=2, mode=0, batches=None, lr=None):
-    """n_steps train steps on GPU and oracle; compares weights, momentum and unique rows."""
+def _run_steps(spec, n_steps=2, mode=0, batches=None, lr=None, grad_f16=False):
+    """n_steps train steps on GPU and oracle; compares weights, momentum and unique rows.
+    grad_f16: the upstream gradient is rounded to binary16 first; the oracle gets those values in fp32 (the
+    conversion is exact), the GPU gets the binary16 tensor (mts_tbe_backward_apply_f16)."""
     lr = spec.lr if lr is None else lr
     W0 = wl.all_weights_numpy(spec)
     W_ref = W0.copy()
@@ -26,6 +28,8 @@ def _run_steps(spec, n_steps=2, mode=0, batches=None, lr=None):
     for k in range(n_steps):
         idx, off = batches[k] if batches is not None else wl.gen_batch(spec, k)
         grad = wl.gen_grad(spec, k)
+        if grad_f16:
+            grad = grad.astype(np.float16).astype(np.float32)
         N = len(idx)
         W_before = W_ref.copy()
         m_before = m_ref.copy()
@@ -35,7 +39,8 @@ def _run_steps(spec, n_steps=2, mode=0, batches=None, lr=None):
                                                        step_mag=step_mag)
         uniq = torch.full((max(N, 1),), -1, dtype=torch.int64, device="cuda:0")
         nu = torch.full((1,), -1, dtype=torch.int64, device="cuda:0")
-        model.backward(to_dev(idx), to_dev(off), N, to_dev(grad), lr=lr, pooling_mode=mode,
+        grad_dev = to_dev(grad).to(torch.float16) if grad_f16 else to_dev(grad)
+        model.backward(to_dev(idx), to_dev(off), N, grad_dev, lr=lr, pooling_mode=mode,
                        uniq_rows_out=uniq, n_unique_out=nu)
         torch.cuda.synchronize()
         assert model.tables.status() == 0
@@ -228,3 +233,19 @@ def test_tables_sorted_separately(rows, pool, B):
     """Table sets for which the lookups of each table are sorted on their own (fewer digit passes)."""
     spec = custom_spec(rows, [64] * len(rows), B, wl.FP16, pool, [1.1] * len(rows), seed=5)
     _run_steps(spec, n_steps=2)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", [wl.FP32, wl.FP16])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_fp16_gradient(dtype, mode):
+    """Upstream gradient in binary16: every column-group width, long and short rows, sum and mean."""
+    dims = [8, 64, 128, 200, 256, 512] if dtype == wl.FP16 else [4, 64, 128, 100, 256, 512]
+    spec = custom_spec([3, 5000, 20000, 7, 777, 129], dims, 193, dtype, [40, 30, 20, 90, 33, 2],
+                       [0, 1.3, 0.9, 0, 1.2, 0], seed=12)
+    _run_steps(spec, n_steps=2, mode=mode, grad_f16=True)
+
+
+@pytest.mark.gpu
+def test_fp16_gradient_rows_of_128_columns():
+    _run_steps(wl.config2(row_scale=0.02, batch=256), n_steps=2, grad_f16=True)

@@ -147,3 +147,29 @@ def test_config3_full_size_sampled_bags_and_rows():
         assert_close_mag(got_w, Wsub, np.abs(W_before) + smag, FWD_RTOL[spec.dtype], f"bwd table {t} weights")
         assert_close_mag(got_m, msub, msub, 1e-5, f"bwd table {t} momentum")
     m.close()
+
+
+@pytest.mark.parametrize("dtype", [wl.FP32, wl.FP16])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_fp16_output(dtype, mode):
+    """mts_tbe_forward_f16: the pooled sum is accumulated in fp32 and rounded once to binary16.  Against the
+    oracle's fp64 sums: the fp32 tolerance of the sum plus half a binary16 ulp of the rounded value."""
+    dims = [8, 64, 128, 200, 256, 512] if dtype == wl.FP16 else [4, 64, 128, 100, 256, 512]
+    spec = custom_spec([50, 5000, 20000, 300, 777, 129], dims, 97, dtype, [0.7, 70, 20, 5, 33, 2],
+                       [0, 1.05, 0.9, 0, 1.3, 0], seed=4)
+    W = wl.all_weights_numpy(spec)
+    idx, off = wl.gen_batch(spec, 0)
+    ref, mag = oracle.tbe_forward(*oracle_args(spec), W, spec.batch, idx, off, mode, want_mag=True)
+    m = DeviceModel(spec, weights=W)
+    out = torch.full((spec.batch, spec.total_dim), float("nan"), dtype=torch.float16, device="cuda:0")
+    m.forward(to_dev(idx), to_dev(off), len(idx), out=out, pooling_mode=mode)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy().astype(np.float64)
+    ref = np.asarray(ref, np.float64).reshape(got.shape)
+    mag = np.asarray(mag, np.float64).reshape(got.shape)
+    # binary16: 11 significant bits -> half an ulp is at most 2^-11 relative (normal range; the values here
+    # are far above the subnormal range or exactly 0)
+    bound = FWD_RTOL[spec.dtype] * (np.abs(ref) + mag) + 2.0 ** -11 * np.abs(ref) + 2.0 ** -25
+    assert np.isfinite(got).all()
+    assert (np.abs(got - ref) <= bound).all(), float(np.max(np.abs(got - ref) - bound))
+    m.close()
