@@ -216,17 +216,20 @@ def run_native(args, rank: int, world: int, local_rank: int):
     spec = make_spec(args.workload, rank, args.tables)
     model = DeviceModel(spec, device=dev)
     R = args.rotate
+    io_t = torch.float16 if args.io_dtype == "f16" else torch.float32     # pooled output and its gradient
+    io_b = 2 if args.io_dtype == "f16" else 4
     host, devb = [], []
     for k in range(R):
         idx, off = wl.gen_batch(spec, k)
         grad = wl.gen_grad(spec, k)
-        h = (torch.from_numpy(idx).pin_memory(), torch.from_numpy(off).pin_memory(), torch.from_numpy(grad).pin_memory())
+        h = (torch.from_numpy(idx).pin_memory(), torch.from_numpy(off).pin_memory(),
+             torch.from_numpy(grad).to(io_t).pin_memory())
         host.append(h)
         devb.append(tuple(x.to(dev) for x in h))
     n_max = max(len(h[0]) for h in host)
     model.reserve(n_max)
     B, TD = spec.batch, spec.total_dim
-    out = torch.empty((B, TD), dtype=torch.float32, device=dev)
+    out = torch.empty((B, TD), dtype=io_t, device=dev)
     stream = torch.cuda.current_stream(dev)
 
     # One training step.  The index-only half of the backward (ordering the lookups by row) does not
@@ -301,10 +304,10 @@ def run_native(args, rank: int, world: int, local_rank: int):
     # pooled output back to pinned host memory.  Copies run on their own streams (input copy of
     # step k+1 and output copy of step k-1 overlap the kernels of step k; two buffers each way).
     s_in, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
-    h_out = [torch.empty((B, TD), dtype=torch.float32).pin_memory() for _ in range(2)]
+    h_out = [torch.empty((B, TD), dtype=io_t).pin_memory() for _ in range(2)]
     d_in = [(torch.empty(n_max, dtype=torch.int64, device=dev), torch.empty(spec.T * B + 1, dtype=torch.int64, device=dev),
-             torch.empty((B, TD), dtype=torch.float32, device=dev)) for _ in range(2)]
-    d_out = [torch.empty((B, TD), dtype=torch.float32, device=dev) for _ in range(2)]
+             torch.empty((B, TD), dtype=io_t, device=dev)) for _ in range(2)]
+    d_out = [torch.empty((B, TD), dtype=io_t, device=dev) for _ in range(2)]
 
     def e2e_run(n_steps):
         ev_in = [torch.cuda.Event() for _ in range(n_steps)]
@@ -331,8 +334,8 @@ def run_native(args, rank: int, world: int, local_rank: int):
                 s_out.wait_event(ev_cmp[k])
                 h_out[k & 1].copy_(d_out[k & 1], non_blocking=True)
                 ev_out[k].record(s_out)
-            h2d_b += n * 8 + ho.numel() * 8 + hg.numel() * 4
-            d2h_b += h_out[0].numel() * 4
+            h2d_b += n * 8 + ho.numel() * 8 + hg.numel() * io_b
+            d2h_b += h_out[0].numel() * io_b
         stream.wait_stream(s_out)
         stream.wait_stream(s_in)
         return h2d_b, d2h_b
@@ -359,7 +362,7 @@ def run_native(args, rank: int, world: int, local_rank: int):
         per_lookup = sum(float(spec.tables[t].dim) * eb * spec.tables[t].pooling for t in range(spec.T)) / \
             sum(spec.tables[t].pooling for t in range(spec.T))
         alg = {
-            "tbe_forward_kernel": n_avg * (per_lookup + 8) + 8 * (spec.T * B + 1) + 4.0 * B * TD,
+            "tbe_forward_kernel": n_avg * (per_lookup + 8) + 8 * (spec.T * B + 1) + float(io_b) * B * TD,
             "reduce_chunks": n_avg * (per_lookup + 8),      # row-equivalent + sorted key and bag id
         }
         # dram__bytes_read + dram__bytes_write per lookup from the ncu capture summarised in
@@ -377,7 +380,8 @@ def run_native(args, rank: int, world: int, local_rank: int):
             roof = {"kernel": top[0], "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
                     "frac": ach / peak,
                     "traffic": (ncu_dram_bytes_per_lookup[top[0]] * n_avg
-                                if spec.name == "cfg2" and ncu_dram_bytes_per_lookup.get(top[0]) else None),
+                                if spec.name == "cfg2" and args.io_dtype == "f32" and ncu_dram_bytes_per_lookup.get(top[0])
+                                else None),
                     "traffic_source": "ncu capture on 8 of 26 tables, scaled by lookups per launch",
                     "peak_source": peak_src,
                     "algorithmic_bytes_per_launch": alg[top[0]], "avg_launch_ms": avg_ms,
@@ -391,6 +395,7 @@ def run_native(args, rank: int, world: int, local_rank: int):
             "config": {"workload": spec.name, "tables": spec.T, "rows_per_table": int(spec.rows[0]),
                        "dim": int(spec.dims[0]), "storage": "fp16" if spec.dtype == wl.FP16 else "fp32",
                        "batch": B, "lookups_per_step": n_avg, "parallelism": f"{world} replica(s), own batches",
+                       "io_dtype": args.io_dtype,
                        "schedule": "sequential" if args.sequential else "backward's sort on a second stream beside the forward",
                        "l2": f"inputs larger than L2: {spec.weight_bytes / 1e9:.2f} GB of weights, {R} batches rotate"},
             "samples_per_sec": world * B / (ms_step * 1e-3),
@@ -601,6 +606,8 @@ def main():
     ap.add_argument("--pooling", type=int, default=50, help="cfg5: lookups per bag")
     ap.add_argument("--alpha", type=float, default=1.0, help="cfg5: Zipf exponent")
     ap.add_argument("--cache-fraction", type=float, default=0.10, help="cfg5: cache slots / rows")
+    ap.add_argument("--io-dtype", default="f32", choices=["f32", "f16"],
+                    help="type of the pooled output and of its gradient (uncached workloads); the headline metric is f32")
     ap.add_argument("--sequential", action="store_true", help="one stream only (no sort beside the forward, no cache pipeline)")
     ap.add_argument("--lock-depth", type=int, default=2,
                     help="cached workloads: batches a stamped way stays unevictable (Section 5.7 invariant)")

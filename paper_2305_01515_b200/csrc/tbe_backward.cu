@@ -127,6 +127,46 @@ __device__ __forceinline__ float4 load_grad4(const void* __restrict__ grad, int6
   return __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(grad) + elem));
 }
 
+// A lane's four gradient values as loaded: fp32, or fp16 left packed so that the sum can use the
+// mixed-precision add (no conversion instructions).
+template <bool GH>
+struct GradPiece {
+  float4 f;
+  uint2 h;
+};
+template <bool GH>
+__device__ __forceinline__ GradPiece<GH> load_piece(const void* __restrict__ grad, int64_t elem, bool valid) {
+  GradPiece<GH> p;
+  if (GH) {
+    p.h = make_uint2(0u, 0u);
+    if (valid) p.h = __ldg(reinterpret_cast<const uint2*>(static_cast<const __half*>(grad) + elem));
+  } else {
+    p.f = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (valid) p.f = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(grad) + elem));
+  }
+  return p;
+}
+template <bool GH>
+__device__ __forceinline__ void add_piece(float4& acc, const GradPiece<GH>& p) {
+  if (GH) {
+    add_half2(acc.x, acc.y, p.h.x);
+    add_half2(acc.z, acc.w, p.h.y);
+  } else {
+    acc.x += p.f.x; acc.y += p.f.y; acc.z += p.f.z; acc.w += p.f.w;
+  }
+}
+template <bool GH>
+__device__ __forceinline__ void fma_piece(float4& acc, float sc, const GradPiece<GH>& p) {
+  float4 g = p.f;
+  if (GH) {
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&p.h.x));
+    const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&p.h.y));
+    g = make_float4(a.x, a.y, b.x, b.y);
+  }
+  acc.x = fmaf(sc, g.x, acc.x); acc.y = fmaf(sc, g.y, acc.y);
+  acc.z = fmaf(sc, g.z, acc.z); acc.w = fmaf(sc, g.w, acc.w);
+}
+
 // Row-wise Adagrad on one row held across the warp: lane owns columns (q*32 + lane)*4 .. +3.
 // m += mean(g^2); W -= lr * g / (sqrt(m) + eps).  inv_dim = __frcp_rn(dim), hoisted by the callers.
 template <bool FP16, int NV>
@@ -430,27 +470,20 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
     // batch has 128 columns: all lanes take part and the width is a constant.
     auto walk = [&](auto full) {
     constexpr bool FULL = decltype(full)::value;
-    auto add_scaled = [&](const float4& g, int jj) {
-      if (MEAN) {
-        const float sc = __uint_as_float(s_aux[wib][jj].y);
-        acc.x = fmaf(sc, g.x, acc.x); acc.y = fmaf(sc, g.y, acc.y);
-        acc.z = fmaf(sc, g.z, acc.z); acc.w = fmaf(sc, g.w, acc.w);
-      } else {
-        acc.x += g.x; acc.y += g.y; acc.z += g.z; acc.w += g.w;
-      }
+    auto add_scaled = [&](const GradPiece<GH>& g, int jj) {
+      if (MEAN) fma_piece<GH>(acc, __uint_as_float(s_aux[wib][jj].y), g);
+      else add_piece<GH>(acc, g);
     };
     auto load_grad = [&](int jj) {
       const int dim = FULL ? 128 : uniform ? dim0 : (int)s_aux[wib][jj].x;
-      float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (FULL || lane * 4 < dim) g = load_grad4<GH>(grad, lane_elem + s_desc[wib][jj].x);
-      return g;
+      return load_piece<GH>(grad, lane_elem + s_desc[wib][jj].x, FULL || lane * 4 < dim);
     };
     int j = 0;
     while (j < cnt) {
       const uint32_t rest = ends >> j;
       const int e = rest ? j + __ffs(rest) - 1 : cnt;              // next lookup that ends a row (or none)
       for (; j + LEAN_RUN <= e; j += LEAN_RUN) {
-        float4 g[LEAN_RUN];
+        GradPiece<GH> g[LEAN_RUN];
 #pragma unroll
         for (int u = 0; u < LEAN_RUN; ++u) g[u] = load_grad(j + u);
 #pragma unroll
@@ -460,8 +493,7 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
       if (e < cnt) {
         const uint4 d = s_desc[wib][e];
         const int dim = FULL ? 128 : uniform ? dim0 : (int)s_aux[wib][e].x;
-        float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (FULL || lane * 4 < dim) g = load_grad4<GH>(grad, lane_elem + d.x);
+        const GradPiece<GH> g = load_piece<GH>(grad, lane_elem + d.x, FULL || lane * 4 < dim);
         if (open_head) {
           add_scaled(g, e);
           *reinterpret_cast<float4*>(partial_head + chunk * PSTRIDE + lane * 4) = acc;
