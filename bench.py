@@ -66,7 +66,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100", "-i",
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50", "-i",
                  str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -594,8 +594,8 @@ def run_sweep(args, rank: int, world: int, local_rank: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=None, help="timed steps (default: 100 for cfg1/cfg2, 8 otherwise)")
+    ap.add_argument("--warmup", type=int, default=None, help="warm-up steps (default: 10 for cfg1/cfg2, 8 otherwise)")
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--rotate", type=int, default=4, help="distinct batches that take turns")
@@ -616,6 +616,11 @@ def main():
     ap.add_argument("--tables", type=int, default=0,
                     help="cfg2 only: fewer tables (a small case for profiler captures; not a bench line)")
     args = ap.parse_args()
+    light = args.workload in ("cfg1", "cfg2") and args.impl == "native"     # a step takes about a millisecond
+    if args.steps is None:
+        args.steps = 100 if light else (3 if args.impl == "reference" else 8)
+    if args.warmup is None:
+        args.warmup = 10 if light else (1 if args.impl == "reference" else 8)
     args.warmup = max(args.warmup, 3) if args.impl == "native" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
