@@ -365,8 +365,8 @@ def run_native(args, rank: int, world: int, local_rank: int):
             "tbe_forward_kernel": n_avg * (per_lookup + 8) + 8 * (spec.T * B + 1) + float(io_b) * B * TD,
             "reduce_chunks": n_avg * (per_lookup + 8),      # row-equivalent + sorted key and bag id
         }
-        # dram__bytes_read + dram__bytes_write per lookup from the ncu capture summarised in
-        # under profiles/ (8 of the 26 tables, 1.967 M lookups per launch there); DRAM traffic
+        # dram__bytes_read + dram__bytes_write per lookup from the ncu capture summarised under
+        # profiles/ (8 of the 26 tables, 1.967 M lookups per launch there); DRAM traffic
         # grows with the lookups processed, so a launch's traffic is this figure times its lookups.
         # Set an entry to None when its kernel changes after the capture.
         ncu_dram_bytes_per_lookup = {"reduce_chunks": (221.659392e6 + 110.100480e6) / 1.967755e6,
