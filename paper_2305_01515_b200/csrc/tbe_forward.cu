@@ -46,6 +46,9 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
   // lane k holds the start of bag k of this warp, lane nb the end of the last one
   const int64_t my_off = offsets[bag0 + min(lane, nb)];
   int64_t i1 = __shfl_sync(0xffffffffu, my_off, 0);
+  // table and sample of the warp's first bag; the following bags step from there (no division per bag)
+  int32_t t = (int32_t)(bag0 / B);
+  int32_t b = (int32_t)(bag0 - (int64_t)t * B);
   // first indices (and cache slots) of the first bag
   int64_t pf_idx = 0;
   int32_t pf_slot = -1;
@@ -53,14 +56,12 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
     const int64_t e = __shfl_sync(0xffffffffu, my_off, 1);
     if (i1 + lane < e) {
       pf_idx = indices[i1 + lane];
-      if (meta[bag0 / B].cache_id >= 0) pf_slot = slot_of_lookup[i1 + lane];
+      if (meta[t].cache_id >= 0) pf_slot = slot_of_lookup[i1 + lane];
     }
   }
 
-  for (int k = 0; k < nb; ++k) {
-    const int64_t bag = bag0 + k;
-    const int32_t t = (int32_t)(bag / B);
-    const int32_t b = (int32_t)(bag - (int64_t)t * B);
+  for (int k = 0; k < nb; ++k, ++b) {
+    if (b == B) { b = 0; ++t; }
     const TableMeta m = meta[t];
     const int vec16 = m.vec16;
     // lanes per row: smallest power of two >= vec16, at most 32
@@ -82,7 +83,7 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
       pf_slot = -1;
       if (i1 + lane < e) {
         pf_idx = indices[i1 + lane];
-        if (meta[(bag + 1) / B].cache_id >= 0) pf_slot = slot_of_lookup[i1 + lane];
+        if (meta[b + 1 == B ? t + 1 : t].cache_id >= 0) pf_slot = slot_of_lookup[i1 + lane];
       }
     }
 
