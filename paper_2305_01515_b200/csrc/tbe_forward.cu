@@ -49,6 +49,8 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
   // table and sample of the warp's first bag; the following bags step from there (no division per bag)
   int32_t t = (int32_t)(bag0 / B);
   int32_t b = (int32_t)(bag0 - (int64_t)t * B);
+  // per-table values, refreshed only when the walk crosses into the next table
+  TableMeta m = meta[t];
   // first indices (and cache slots) of the first bag
   int64_t pf_idx = 0;
   int32_t pf_slot = -1;
@@ -56,26 +58,34 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
     const int64_t e = __shfl_sync(0xffffffffu, my_off, 1);
     if (i1 + lane < e) {
       pf_idx = indices[i1 + lane];
-      if (meta[t].cache_id >= 0) pf_slot = slot_of_lookup[i1 + lane];
+      if (m.cache_id >= 0) pf_slot = slot_of_lookup[i1 + lane];
     }
   }
 
+  int32_t t_cur = -1;
+  int vec16 = 0, logG = 0, G = 1, R = 32, sub = 0, cl = 0;
+  int64_t row_bytes = 0;
+  const char* table_base = nullptr;
+  const char* cache_base = nullptr;
   for (int k = 0; k < nb; ++k, ++b) {
     if (b == B) { b = 0; ++t; }
-    const TableMeta m = meta[t];
-    const int vec16 = m.vec16;
-    // lanes per row: smallest power of two >= vec16, at most 32
-    int logG = 0;
-    while ((1 << logG) < vec16 && logG < 5) ++logG;
-    const int G = 1 << logG;
-    const int R = 32 >> logG;               // rows per load instruction
-    const int sub = lane >> logG;
-    const int cl = lane & (G - 1);
+    if (t != t_cur) {
+      t_cur = t;
+      m = meta[t];
+      vec16 = m.vec16;
+      // lanes per row: smallest power of two >= vec16, at most 32
+      logG = 0;
+      while ((1 << logG) < vec16 && logG < 5) ++logG;
+      G = 1 << logG;
+      R = 32 >> logG;               // rows per load instruction
+      sub = lane >> logG;
+      cl = lane & (G - 1);
+      row_bytes = (int64_t)m.dim * EB;
+      table_base = (m.cache_id < 0 ? dev_w : host_w) + m.weight_offset * EB;
+      cache_base = m.cache_id >= 0 ? static_cast<const char*>(caches.data[m.cache_id]) : nullptr;
+    }
     const int64_t i0 = i1;
     i1 = __shfl_sync(0xffffffffu, my_off, k + 1);
-    const int64_t row_bytes = (int64_t)m.dim * EB;
-    const char* table_base = (m.cache_id < 0 ? dev_w : host_w) + m.weight_offset * EB;
-    const char* cache_base = m.cache_id >= 0 ? static_cast<const char*>(caches.data[m.cache_id]) : nullptr;
     const int64_t cur_idx = pf_idx;
     const int32_t cur_slot = pf_slot;
     if (k + 1 < nb) {
@@ -83,7 +93,8 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
       pf_slot = -1;
       if (i1 + lane < e) {
         pf_idx = indices[i1 + lane];
-        if (meta[b + 1 == B ? t + 1 : t].cache_id >= 0) pf_slot = slot_of_lookup[i1 + lane];
+        const int32_t next_cache = b + 1 == B ? meta[t + 1].cache_id : m.cache_id;
+        if (next_cache >= 0) pf_slot = slot_of_lookup[i1 + lane];
       }
     }
 
@@ -196,6 +207,160 @@ static int launch_forward(const mts_tables* h, int32_t B, const int64_t* indices
   return check_launch("tbe_forward_kernel");
 }
 
+// ---- tbe_forward_lean: the same walk when no table sits behind a cache and a row is at most 32
+// 16-byte pieces.  The walk is bound by latency and instruction issue, not by bytes in flight, so this
+// form trades loads in flight per warp for resident warps: positions and row numbers are 32-bit, there
+// is no cache-slot path, and the register allocation is bounded for MTS_FWD_LEAN_MINBLK blocks per SM.
+// Same summation order and arithmetic as tbe_forward_kernel (bit-identical results).
+#ifndef MTS_FWD_LEAN
+#define MTS_FWD_LEAN 1
+#endif
+#ifndef MTS_FWD_LEAN_MINBLK
+#define MTS_FWD_LEAN_MINBLK 16    // 64 warps per SM: 32 registers a thread
+#endif
+#ifndef MTS_FWD_LEAN_UNROLL
+#define MTS_FWD_LEAN_UNROLL 1    // load instructions issued back to back per lane
+#endif
+constexpr int LEAN_UNROLL = MTS_FWD_LEAN_UNROLL;
+
+template <bool FP16>
+__global__ void __launch_bounds__(FWD_WARPS * 32, MTS_FWD_LEAN_MINBLK)
+tbe_forward_lean(const TableMeta* __restrict__ meta, int32_t n_bags, int32_t B,
+                 const int64_t* __restrict__ indices, const int64_t* __restrict__ offsets,
+                 const char* __restrict__ dev_w, int32_t pooling_mode, void* __restrict__ out, bool out_half,
+                 int64_t out_stride, int32_t* status) {
+  constexpr int EPC = FP16 ? 8 : 4;       // elements per 16-byte chunk
+  constexpr int EB = FP16 ? 2 : 4;
+  const int lane = threadIdx.x & 31;
+  const int32_t bag0 = (int32_t)((blockIdx.x * FWD_WARPS + (threadIdx.x >> 5)) * FWD_BAGS);
+  if (bag0 >= n_bags) return;
+  const int nb = min(FWD_BAGS, n_bags - bag0);
+  // lane k holds the start of bag k of this warp, lane nb the end of the last one
+  const uint32_t my_off = (uint32_t)offsets[bag0 + min(lane, nb)];
+  uint32_t i1 = __shfl_sync(0xffffffffu, my_off, 0);
+  int32_t t = (int32_t)((uint32_t)bag0 / (uint32_t)B);
+  int32_t b = bag0 - t * B;
+  // first indices of the first bag
+  int64_t pf_idx = 0;
+  {
+    const uint32_t e = __shfl_sync(0xffffffffu, my_off, 1);
+    if (i1 + lane < e) pf_idx = indices[i1 + lane];
+  }
+  // per-table values, refreshed only when the walk crosses into the next table
+  int32_t t_cur = -1;
+  int vec16 = 0, logG = 0, row_bytes = 0, out_offset = 0;
+  uint32_t rows = 0;
+  const char* lane_base = nullptr;        // the lane's 16-byte piece of row 0
+  for (int k = 0; k < nb; ++k, ++b) {
+    if (b == B) { b = 0; ++t; }
+    if (t != t_cur) {
+      t_cur = t;
+      const TableMeta m = meta[t];
+      vec16 = m.vec16;
+      logG = 0;
+      while ((1 << logG) < vec16) ++logG;   // lanes per row: smallest power of two >= vec16 (vec16 <= 32 here)
+      row_bytes = m.dim * EB;
+      rows = (uint32_t)m.rows;
+      out_offset = m.out_offset;
+      lane_base = dev_w + m.weight_offset * EB + (lane & ((1 << logG) - 1)) * 16;
+    }
+    const int R = 32 >> logG;               // rows per load instruction
+    const int sub = lane >> logG;
+    const int cl = lane & ((1 << logG) - 1);
+    const uint32_t i0 = i1;
+    i1 = __shfl_sync(0xffffffffu, my_off, k + 1);
+    const int64_t cur_idx = pf_idx;
+    if (k + 1 < nb) {
+      const uint32_t e = __shfl_sync(0xffffffffu, my_off, k + 2);
+      if (i1 + lane < e) pf_idx = indices[i1 + lane];
+    }
+
+    float acc[EPC];
+#pragma unroll
+    for (int e = 0; e < EPC; ++e) acc[e] = 0.f;
+
+    for (uint32_t base = i0; base < i1; base += 32) {
+      const int cnt = (int)min(32u, i1 - base);
+      uint32_t my_row = 0;
+      if (lane < cnt) {
+        int64_t idx = base == i0 ? cur_idx : indices[base + lane];
+        if (idx < 0 || idx >= (int64_t)rows) {
+          atomicOr(status, STATUS_INDEX_CLAMPED);
+          idx = idx < 0 ? 0 : (int64_t)rows - 1;
+        }
+        my_row = (uint32_t)idx;
+      }
+      auto walk = [&](auto whole) {
+        constexpr bool WHOLE = decltype(whole)::value;
+        for (int r = 0; r < cnt; r += R * LEAN_UNROLL) {
+          uint4 v[LEAN_UNROLL];
+#pragma unroll
+          for (int u = 0; u < LEAN_UNROLL; ++u) {
+            const int j = r + u * R + sub;
+            const uint32_t row = __shfl_sync(0xffffffffu, my_row, j & 31);
+            if (j < cnt && (WHOLE || cl < vec16)) v[u] = ld_nc_16(lane_base + (int64_t)row * row_bytes);
+            else v[u] = make_uint4(0u, 0u, 0u, 0u);
+          }
+#pragma unroll
+          for (int u = 0; u < LEAN_UNROLL; ++u) {
+            if (FP16) add_half8(acc, v[u]);
+            else add_float4(acc, v[u]);
+          }
+        }
+      };
+      if (vec16 == (1 << logG)) walk(std::true_type{});
+      else walk(std::false_type{});
+    }
+    // fold the row groups of the warp together
+    for (int o = 1 << logG; o < 32; o <<= 1) {
+#pragma unroll
+      for (int e = 0; e < EPC; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+    }
+    if (sub == 0 && cl < vec16) {
+      float scale = 1.f;
+      if (pooling_mode == MTS_POOL_MEAN && i1 > i0) scale = 1.f / (float)(i1 - i0);
+      const int64_t o = (int64_t)b * out_stride + out_offset + cl * EPC;     // first element of the lane's piece
+      if (out_half) {
+        // pooled sums rounded to fp16 (round to nearest even)
+        __half2 h01 = __floats2half2_rn(acc[0] * scale, acc[1] * scale);
+        __half2 h23 = __floats2half2_rn(acc[2] * scale, acc[3] * scale);
+        uint2 lo;
+        lo.x = *reinterpret_cast<uint32_t*>(&h01);
+        lo.y = *reinterpret_cast<uint32_t*>(&h23);
+        __half* dst = static_cast<__half*>(out) + o;
+        *reinterpret_cast<uint2*>(dst) = lo;
+        if (FP16) {
+          __half2 h45 = __floats2half2_rn(acc[4] * scale, acc[5] * scale);
+          __half2 h67 = __floats2half2_rn(acc[6] * scale, acc[7] * scale);
+          uint2 hi;
+          hi.x = *reinterpret_cast<uint32_t*>(&h45);
+          hi.y = *reinterpret_cast<uint32_t*>(&h67);
+          *reinterpret_cast<uint2*>(dst + 4) = hi;
+        }
+      } else {
+        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(out) + o);
+        dst[0] = make_float4(acc[0] * scale, acc[1] * scale, acc[2] * scale, acc[3] * scale);
+        if (FP16) dst[1] = make_float4(acc[4] * scale, acc[5] * scale, acc[6] * scale, acc[7] * scale);
+      }
+    }
+  }
+}
+
+template <bool FP16>
+static int launch_forward_lean(const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets,
+                               int32_t pooling_mode, void* out, bool out_half, int64_t out_stride,
+                               cudaStream_t stream) {
+  const int64_t n_bags = (int64_t)h->T * B;
+  const int64_t grid = ceil_div(n_bags, (int64_t)FWD_WARPS * FWD_BAGS);
+  {
+    LaunchScope scope(K_FORWARD, stream);
+    tbe_forward_lean<FP16><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
+        h->d_meta, (int32_t)n_bags, B, indices, offsets, static_cast<const char*>(h->dev_weights), pooling_mode, out,
+        out_half, out_stride, h->d_status);
+  }
+  return check_launch("tbe_forward_lean");
+}
+
 int fill_cache_ptrs(const mts_tables* h, void* const* host_cache_data, uint8_t* const* host_cache_dirty,
                     int32_t n_caches, const int32_t* slot_of_lookup, CachePtrs* out) {
   for (int c = 0; c < MTS_MAX_CACHES; ++c) { out->data[c] = nullptr; out->dirty[c] = nullptr; }
@@ -237,6 +402,13 @@ int forward_any(const mts_tables* h, int32_t B, const int64_t* indices, const in
   const int max_vec = h->max_dim * h->elem_bytes / 16;
   const int nv = max_vec <= 32 ? 1 : max_vec <= 64 ? 2 : max_vec <= 128 ? 4 : 8;
   const bool fp16 = h->dtype == MTS_DTYPE_FP16;
+#if MTS_FWD_LEAN
+  // positions and bag numbers fit 32 bits (row numbers always do), no cached table, rows of at most 32 pieces
+  if (!h->any_cached && nv == 1 && N < (1ll << 31) && (int64_t)h->T * B < (1ll << 31) - FWD_WARPS * FWD_BAGS) {
+    if (fp16) return launch_forward_lean<true>(h, B, indices, offsets, pooling_mode, out, out_half, out_stride, s);
+    return launch_forward_lean<false>(h, B, indices, offsets, pooling_mode, out, out_half, out_stride, s);
+  }
+#endif
 #define MTS_FWD(F, V) return launch_forward<F, V>(h, B, indices, offsets, pooling_mode, slot_of_lookup, caches, out, out_half, out_stride, s)
   if (fp16) {
     if (nv == 1) MTS_FWD(true, 1);
