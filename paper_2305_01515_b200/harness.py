@@ -188,14 +188,21 @@ class DeviceModel:
 
     def cache_move(self, stream=None, ctx: Optional[int] = None) -> None:
         """Data path of one batch: save dirty victims, pull missed rows from the host tier, write victims back."""
-        cx = self.ctx[self.cur if ctx is None else ctx]
-        for g, c in enumerate(self.caches):
-            L = cx["lists"][g]
-            hp = self.host_rows_ptr(g)
-            mb.cache_prefetch_misses(c, hp, L["miss_keys"], L["miss_slots"], L["evict_slots"], L["evict_dirty"],
-                                     L["capacity"], L["counters"], L["staging"], stream)
-            mb.cache_writeback_evicted(c, hp, L["evict_keys"], L["evict_dirty"], L["capacity"], L["counters"],
-                                       L["staging"], stream)
+        for g in range(len(self.caches)):
+            self.cache_fetch(g, stream, ctx)
+            self.cache_writeback(g, stream, ctx)
+
+    def cache_fetch(self, g: int, stream=None, ctx: Optional[int] = None) -> None:
+        """Cache g: dirty victims into the staging buffer, then the missed rows from the host tier into their slots."""
+        L = self.ctx[self.cur if ctx is None else ctx]["lists"][g]
+        mb.cache_prefetch_misses(self.caches[g], self.host_rows_ptr(g), L["miss_keys"], L["miss_slots"],
+                                 L["evict_slots"], L["evict_dirty"], L["capacity"], L["counters"], L["staging"], stream)
+
+    def cache_writeback(self, g: int, stream=None, ctx: Optional[int] = None) -> None:
+        """Cache g: the staged dirty victims back to the host tier (after cache_fetch of the same batch)."""
+        L = self.ctx[self.cur if ctx is None else ctx]["lists"][g]
+        mb.cache_writeback_evicted(self.caches[g], self.host_rows_ptr(g), L["evict_keys"], L["evict_dirty"],
+                                   L["capacity"], L["counters"], L["staging"], stream)
 
     def cache_refetch(self, prev_ctx: int, stream=None) -> None:
         """After the backward of the batch in context `prev_ctx`: refresh rows that overflowed there

@@ -1,10 +1,11 @@
 """Schedule of the cached train step (Section 5.7 of the paper: prefetch into the cache ahead of
 training; Section 6.1: cache kernels on their own streams, synchronised with the next batch's
-lookups).  Three streams, ordered by events only:
+lookups).  Streams, ordered by events only:
 
-    main : forward(t), backward(t)
-    move : save victims / fetch missed rows / write victims back for batch t+1   (host link)
-    tag  : tag lookup and replacement for batch t+2                              (HBM, small)
+    main    : forward(t), backward(t)
+    move[g] : cache g: save victims / fetch missed rows / write victims back for batch t+1   (host link)
+    fix     : repair of rows that overflowed in batch t and were placed in batch t+1 (after backward(t))
+    tag     : tag lookup and replacement for batch t+2                              (HBM, small)
 
 so the host-link traffic of the next batch and the tag work of the one after it overlap the
 training of the current batch.
@@ -41,9 +42,11 @@ class CachedTrainer:
         self.dev = model.device
         self.main = torch.cuda.current_stream(self.dev)
         self.tag = torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main
-        # the data movement needs few thread blocks but must not queue behind the training kernels' blocks
-        self.move = torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main
+        # the data movement needs few thread blocks but must not queue behind the training kernels' blocks;
+        # one stream per cache, so that the caches' row fetches share the host link instead of taking turns
         n_c = len(model.caches)
+        self.moves = [torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main for _ in range(n_c)]
+        self.fix = torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main
         self.host_counters = [torch.zeros((n_c, mb.NUM_COUNTERS), dtype=torch.int64).pin_memory()
                               for _ in range(DeviceModel.N_CTX)]
         self.history: List[np.ndarray] = []           # per batch [n_caches, NUM_COUNTERS]
@@ -78,23 +81,40 @@ class CachedTrainer:
         ev_tags.record(s)
 
     def _move(self, t, ev_tags, ev_ready, prev_overflow, prev_bwd):
-        """Data path of batch t on the move stream.  prev_overflow: number of rows of batch t-1 that
-        found no way (0 = none), prev_bwd: event after batch t-1's backward."""
-        s = self.move
-        s.wait_event(ev_tags)
-        refetch = False
+        """Data path of batch t, each cache on its own move stream.  prev_overflow: number of rows of
+        batch t-1 that found no way (0 = none), prev_bwd: event after batch t-1's backward."""
+        ctx = t % DeviceModel.N_CTX
+        refetch = wait_bwd = False
         if prev_overflow:
             cap = min(L["capacity"] for L in self.m.ctx[(t - 1) % DeviceModel.N_CTX]["lists"])
             if prev_overflow <= cap:
                 refetch = True                       # move now, repair the few stale rows afterwards
             else:
-                s.wait_event(prev_bwd)               # the list was cut: wait for the backward first
-        self._mark("move_begin", t, s)
-        self.m.cache_move(stream=s, ctx=t % DeviceModel.N_CTX)
-        self._mark("move_end", t, s)
+                wait_bwd = True                      # the list was cut: wait for the backward first
+        ends = []
+        for g, s in enumerate(self.moves):
+            s.wait_event(ev_tags)
+            if wait_bwd:
+                s.wait_event(prev_bwd)
+            self._mark(f"move{g}_begin", t, s)
+            # fetch, then write back, in stream order: the next batch's fetch of this cache, which may
+            # miss a row written back now, comes after it on the same stream
+            self.m.cache_fetch(g, stream=s, ctx=ctx)
+            self.m.cache_writeback(g, stream=s, ctx=ctx)
+            self._mark(f"move{g}_end", t, s)
+            e = torch.cuda.Event()
+            e.record(s)
+            ends.append(e)
+        # the repair of stale rows waits for the previous backward; on its own stream it does not hold
+        # up the next batch's data movement
+        s = self.fix
+        for e in ends:
+            s.wait_event(e)
         if refetch:
             s.wait_event(prev_bwd)
+            self._mark("refetch_begin", t, s)
             self.m.cache_refetch((t - 1) % DeviceModel.N_CTX, stream=s)
+        self._mark("ready", t, s)
         ev_ready.record(s)
 
     def _counters(self, t, ev_tags) -> int:
@@ -130,7 +150,8 @@ class CachedTrainer:
         start = torch.cuda.Event()
         start.record(self.main)
         self.tag.wait_event(start)
-        self.move.wait_event(start)
+        for s in self.moves + [self.fix]:
+            s.wait_event(start)
         overflow = {}
         self._lookup(0, first_step, batches[0], ev_tags[0], None)
         self._move(0, ev_tags[0], ev_ready[0], 0, None)
@@ -159,4 +180,5 @@ class CachedTrainer:
             if on_step is not None:
                 on_step(t)
         self.main.wait_stream(self.tag)
-        self.main.wait_stream(self.move)
+        for s in self.moves + [self.fix]:
+            self.main.wait_stream(s)
