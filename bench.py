@@ -369,8 +369,8 @@ def run_native(args, rank: int, world: int, local_rank: int):
         # profiles/ (8 of the 26 tables, 1.967 M lookups per launch there); DRAM traffic
         # grows with the lookups processed, so a launch's traffic is this figure times its lookups.
         # Set an entry to None when its kernel changes after the capture.
-        ncu_dram_bytes_per_lookup = {"reduce_chunks": (221.659392e6 + 110.100480e6) / 1.967755e6,
-                                     "tbe_forward_kernel": (148.988928e6 + 21.364992e6) / 1.967755e6}
+        ncu_dram_bytes_per_lookup = {"reduce_chunks": (221.632256e6 + 110.179584e6) / 1.967755e6,
+                                     "tbe_forward_kernel": (152.497152e6 + 27.390464e6) / 1.967755e6}
         top = max(trace.items(), key=lambda kv: kv[1][0]) if trace else (None, (0.0, 0))
         kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps} for k, v in trace.items()}
         roof = None
