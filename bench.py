@@ -470,7 +470,7 @@ def run_cached(args, rank: int, world: int, local_rank: int):
     grads = [torch.from_numpy(wl.gen_grad(spec, k)).to(dev) for k in range(R)]
     glist = [grads[k % R] for k in range(K)]
     setup_s = time.time() - t_setup
-    trainer = CachedTrainer(model, pipelined=not args.sequential)
+    trainer = CachedTrainer(model, pipelined=not args.sequential, host_gather=args.fetch == "host")
     main = torch.cuda.current_stream(dev)
     marks = {}
 
@@ -536,6 +536,7 @@ def run_cached(args, rank: int, world: int, local_rank: int):
         "config": {"workload": spec.name, "note": spec.note, "tables": spec.T, "rows_total": int(spec.row_offset[-1]),
                    "host_weight_gb": spec.weight_bytes / 1e9, "cache_fraction": spec.cache_fraction, "batch": B,
                    "lookups_per_step": lookups / args.steps, "schedule": "sequential" if args.sequential else "pipelined", "lock_depth": args.lock_depth,
+                   "missed_rows": "gathered by host threads, copy engine" if args.fetch == "host" else "read by a kernel over the host link",
                    "l2": "inputs larger than L2 (host tier and caches are GBs)", "setup_seconds": setup_s},
         "samples_per_sec": B * args.steps / t_meas, "hit_rate_per_lookup": hit,
         "unique_hit_rate": float(hist[:, :, 4].sum()) / max(float(hist[:, :, 1].sum()), 1.0),
@@ -608,6 +609,9 @@ def main():
     ap.add_argument("--cache-fraction", type=float, default=0.10, help="cfg5: cache slots / rows")
     ap.add_argument("--io-dtype", default="f32", choices=["f32", "f16"],
                     help="type of the pooled output and of its gradient (uncached workloads); the headline metric is f32")
+    ap.add_argument("--fetch", default="sm", choices=["sm", "host"],
+                    help="cached workloads: missed rows read over the host link by a kernel (sm), or gathered by host "
+                         "threads into a pinned buffer and moved by the copy engine (host)")
     ap.add_argument("--sequential", action="store_true", help="one stream only (no sort beside the forward, no cache pipeline)")
     ap.add_argument("--lock-depth", type=int, default=2,
                     help="cached workloads: batches a stamped way stays unevictable (Section 5.7 invariant)")

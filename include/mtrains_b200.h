@@ -297,6 +297,23 @@ int mts_cache_prefetch_misses(mts_cache* cache, const void* host_rows_mapped, co
                               const uint8_t* evict_dirty, int64_t list_capacity,
                               const int64_t* counters, void* evict_staging, void* stream);
 
+/* The same data movement with the missed rows arriving through the copy engine instead of being read
+ * from host memory by the kernels (Sections 5.5.3, 5.5.4; the paper's own lower tier is read by host
+ * threads as well).  Rows read by SMs over the host link are slow (small requests) and slow down every
+ * kernel that shares the GPU with them; a contiguous copy is neither.  Three steps, the middle one the
+ * caller's: (1) mts_host_gather_rows, on the host: host_out[k] = host_rows[host_keys[k]] for k < n, with
+ * `threads` host threads (plain memory, no GPU call; host_keys is a HOST copy of the first n entries of
+ * the miss list; blocks until done; the rows must not be written meanwhile); (2) one contiguous copy of
+ * host_out to a device buffer `fetched`; (3) mts_cache_place_fetched, on `stream` after that copy: saves
+ * the dirty victims like mts_cache_prefetch_misses, then fetched[k] -> slot miss_slots[k] for every k
+ * below min(MTS_CNT_INSERTED, list_capacity).  fetched: device [>= that many rows, dim], 16-byte aligned.
+ * Errors: INVALID_ARG, ALIGNMENT, CUDA. */
+int mts_host_gather_rows(const void* host_rows, const int64_t* host_keys, int64_t n, int64_t row_bytes,
+                         void* host_out, int32_t threads);
+int mts_cache_place_fetched(mts_cache* cache, const void* fetched, const int32_t* miss_slots,
+                            const int32_t* evict_slots, const uint8_t* evict_dirty, int64_t list_capacity,
+                            const int64_t* counters, void* evict_staging, void* stream);
+
 /* Evicted dirty rows go back to the host tier: evict_staging[k] -> host row evict_keys[k]. */
 int mts_cache_writeback_evicted(mts_cache* cache, void* host_rows_mapped, const int64_t* evict_keys,
                                 const uint8_t* evict_dirty, int64_t list_capacity,
@@ -306,10 +323,14 @@ int mts_cache_writeback_evicted(mts_cache* cache, void* host_rows_mapped, const 
  * A key that overflowed in batch t is read and updated in the host tier by batch t's forward and
  * backward; if batch t+1 places that key, mts_cache_prefetch_misses(t+1) may have copied the host
  * row before batch t's update reached it.  Call this after batch t's backward with batch t's
- * overflow list and counters: every listed key that is resident now gets its row copied from the
- * host tier again.  A no-op when the steps run one after the other. */
+ * overflow list and counters: every listed key that is resident now, in a way stamped `placed_step`
+ * (the `step` of batch t+1's lookup_insert; -1 = any stamp), gets its row copied from the host tier
+ * again.  The stamp keeps the call away from a key that a tag step running further ahead (batch t+2)
+ * has placed meanwhile: that slot still holds its victim's row until batch t+2's data movement.
+ * A no-op when the steps run one after the other. */
 int mts_cache_refetch_overflowed(mts_cache* cache, const void* host_rows_mapped, const int64_t* overflow_keys,
-                                 int64_t list_capacity, const int64_t* counters, void* stream);
+                                 int64_t list_capacity, const int64_t* counters, int64_t placed_step,
+                                 void* stream);
 
 /* Writes every dirty resident row to the host tier and clears its dirty byte. */
 int mts_cache_flush(mts_cache* cache, void* host_rows_mapped, void* stream);

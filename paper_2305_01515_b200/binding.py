@@ -32,7 +32,7 @@ EXPORTS = (
     "mts_tbe_forward_f16", "mts_tbe_backward_apply_f16",
     "mts_cache_create", "mts_cache_destroy", "mts_cache_status", "mts_cache_data", "mts_cache_dirty",
     "mts_linearize_keys", "mts_cache_workspace_bytes", "mts_cache_lookup_insert",
-    "mts_cache_prefetch_misses", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
+    "mts_cache_prefetch_misses", "mts_host_gather_rows", "mts_cache_place_fetched", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
     "mts_cache_export_state",
 )
 
@@ -100,9 +100,11 @@ def lib():
         L.mts_cache_workspace_bytes.restype = sz
         L.mts_cache_workspace_bytes.argtypes = [vp, i64]
         L.mts_cache_lookup_insert.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
-        L.mts_cache_refetch_overflowed.argtypes = [vp, vp, vp, i64, vp, vp]
+        L.mts_cache_refetch_overflowed.argtypes = [vp, vp, vp, i64, vp, i64, vp]
         L.mts_cache_prefetch_misses.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.mts_cache_writeback_evicted.argtypes = [vp, vp, vp, vp, i64, vp, vp, vp]
+        L.mts_host_gather_rows.argtypes = [vp, vp, i64, i64, vp, i32]
+        L.mts_cache_place_fetched.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.mts_cache_flush.argtypes = [vp, vp, vp]
         L.mts_cache_export_state.argtypes = [vp, vp, vp, vp, vp, vp]
         for name in EXPORTS:
@@ -320,9 +322,9 @@ def cache_lookup_insert(cache: Cache, keys, N: int, step: int, slot_of_lookup, m
 
 
 def cache_refetch_overflowed(cache: Cache, host_rows_mapped, overflow_keys, list_capacity: int, counters,
-                             stream=None) -> None:
+                             placed_step: int = -1, stream=None) -> None:
     _check(lib().mts_cache_refetch_overflowed(cache.handle, _ptr(host_rows_mapped), _ptr(overflow_keys),
-                                              list_capacity, _ptr(counters), _stream(stream)))
+                                              list_capacity, _ptr(counters), placed_step, _stream(stream)))
 
 
 def cache_prefetch_misses(cache: Cache, host_rows_mapped, miss_keys, miss_slots, evict_slots, evict_dirty,
@@ -330,6 +332,20 @@ def cache_prefetch_misses(cache: Cache, host_rows_mapped, miss_keys, miss_slots,
     _check(lib().mts_cache_prefetch_misses(cache.handle, _ptr(host_rows_mapped), _ptr(miss_keys), _ptr(miss_slots),
                                            _ptr(evict_slots), _ptr(evict_dirty), list_capacity, _ptr(counters),
                                            _ptr(evict_staging), _stream(stream)))
+
+
+def host_gather_rows(host_rows_ptr: int, host_keys, n: int, row_bytes: int, host_out, threads: int) -> None:
+    """host_keys: host int64 array (numpy); host_rows_ptr / host_out: host addresses (pinned buffers)."""
+    assert host_keys.dtype.itemsize == 8 and host_keys.flags.c_contiguous and len(host_keys) >= n
+    _check(lib().mts_host_gather_rows(int(host_rows_ptr), int(host_keys.ctypes.data), n, row_bytes,
+                                      _ptr(host_out), threads))
+
+
+def cache_place_fetched(cache: Cache, fetched, miss_slots, evict_slots, evict_dirty, list_capacity: int, counters,
+                        evict_staging, stream=None) -> None:
+    _check(lib().mts_cache_place_fetched(cache.handle, _ptr(fetched), _ptr(miss_slots), _ptr(evict_slots),
+                                         _ptr(evict_dirty), list_capacity, _ptr(counters), _ptr(evict_staging),
+                                         _stream(stream)))
 
 
 def cache_writeback_evicted(cache: Cache, host_rows_mapped, evict_keys, evict_dirty, list_capacity: int, counters,

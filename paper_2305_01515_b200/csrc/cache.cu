@@ -12,6 +12,8 @@
 // Every decision is a pure function of the cache state and the batch, so the slots, lists and
 // counters are reproducible bit for bit.
 #include <algorithm>
+#include <cstring>
+#include <thread>
 
 #include "common.cuh"
 
@@ -400,6 +402,16 @@ cache_fetch_misses(char* __restrict__ data, int row_bytes, const char* __restric
             [&](int64_t k) { return data + (int64_t)miss_slots[k] * row_bytes; });
 }
 
+// Missed rows that arrived in list order through a contiguous copy: fetched[k] -> slot miss_slots[k].
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_place_fetched(char* __restrict__ data, int row_bytes, const char* __restrict__ fetched,
+                    const int32_t* __restrict__ miss_slots, const int64_t* __restrict__ counters, int64_t capacity) {
+  const int64_t n = list_len(counters, MTS_CNT_INSERTED, capacity);
+  copy_rows(n, row_bytes / 16,
+            [&](int64_t k) { return fetched + k * row_bytes; },
+            [&](int64_t k) { return data + (int64_t)miss_slots[k] * row_bytes; });
+}
+
 // ---- missed rows through the bulk-copy engine (TMA, non-tensor form) ------------------------
 // Plain 16-byte loads from mapped host memory top out far below the host link's bandwidth (the
 // requests that reach the link are small).  Here one warp per block asks the bulk-copy engine for
@@ -484,7 +496,8 @@ cache_fetch_misses_bulk(char* __restrict__ data, int row_bytes, const char* __re
 __global__ void __launch_bounds__(CACHE_THREADS)
 cache_refetch_resident(char* __restrict__ data, int row_bytes, const char* __restrict__ host_rows,
                        const int64_t* __restrict__ keys, const int64_t* __restrict__ counters, int64_t capacity,
-                       const uint32_t* __restrict__ tags, uint64_t S) {
+                       const uint32_t* __restrict__ tags, const int32_t* __restrict__ ts, int64_t placed_step,
+                       uint64_t S) {
   const int64_t n = list_len(counters, MTS_CNT_OVERFLOW, capacity);
   const int lane = threadIdx.x & 31;
   const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -492,7 +505,10 @@ cache_refetch_resident(char* __restrict__ data, int row_bytes, const char* __res
   for (int64_t k = warp0; k < n; k += nwarps) {
     const uint32_t key = (uint32_t)keys[k];
     const int64_t slot0 = (int64_t)set_of_key(key, S) * 32;
-    const uint32_t hit = __ballot_sync(0xffffffffu, tags[slot0 + lane] == key);
+    // only a way stamped by the batch named in placed_step: a later tag step may have placed the key
+    // already, in a slot whose victim has not been saved yet and whose own fetch is still to come
+    const uint32_t hit = __ballot_sync(0xffffffffu, tags[slot0 + lane] == key &&
+                                                        (placed_step < 0 || (int64_t)ts[slot0 + lane] == placed_step));
     if (hit) {
       const char* src = host_rows + (int64_t)key * row_bytes;
       char* dst = data + (slot0 + __ffs(hit) - 1) * row_bytes;
@@ -793,6 +809,58 @@ extern "C" int mts_cache_prefetch_misses(mts_cache* c, const void* host_rows_map
   return check_launch("cache_save_victims / cache_fetch_misses");
 }
 
+extern "C" int mts_host_gather_rows(const void* host_rows, const int64_t* host_keys, int64_t n, int64_t row_bytes,
+                                    void* host_out, int32_t threads) {
+  if (n < 0 || row_bytes < 1 || (n > 0 && (!host_rows || !host_keys || !host_out)))
+    return set_error(MTS_ERR_INVALID_ARG, "host_gather_rows: null argument or bad size");
+  if (n == 0) return MTS_OK;
+  const char* src = static_cast<const char*>(host_rows);
+  char* dst = static_cast<char*>(host_out);
+  const size_t rb = (size_t)row_bytes;
+  auto work = [=](int64_t k0, int64_t k1) {
+    constexpr int64_t AHEAD = 16;        // rows requested ahead of the copy: the reads are random DRAM accesses
+    for (int64_t k = k0; k < k1; ++k) {
+      if (k + AHEAD < k1) {
+        const char* ahead = src + (size_t)host_keys[k + AHEAD] * rb;
+        for (size_t b = 0; b < rb; b += 64) __builtin_prefetch(ahead + b, 0, 0);
+      }
+      memcpy(dst + (size_t)k * rb, src + (size_t)host_keys[k] * rb, rb);
+    }
+  };
+  const int64_t nt = std::max<int64_t>(1, std::min<int64_t>(threads, (n + 1023) / 1024));
+  if (nt == 1) { work(0, n); return MTS_OK; }
+  std::vector<std::thread> pool;
+  const int64_t per = (n + nt - 1) / nt;
+  for (int64_t i = 1; i < nt; ++i) pool.emplace_back(work, std::min(n, i * per), std::min(n, (i + 1) * per));
+  work(0, std::min(n, per));
+  for (auto& t : pool) t.join();
+  return MTS_OK;
+}
+
+extern "C" int mts_cache_place_fetched(mts_cache* c, const void* fetched, const int32_t* miss_slots,
+                                       const int32_t* evict_slots, const uint8_t* evict_dirty, int64_t list_capacity,
+                                       const int64_t* counters, void* evict_staging, void* stream) {
+  if (!c || !counters || list_capacity < 0 ||
+      (list_capacity > 0 && (!fetched || !miss_slots || !evict_slots || !evict_dirty || !evict_staging)))
+    return set_error(MTS_ERR_INVALID_ARG, "cache_place_fetched: null argument");
+  if (((uintptr_t)fetched | (uintptr_t)evict_staging) & 15)
+    return set_error(MTS_ERR_ALIGNMENT, "cache_place_fetched: buffers must be 16-byte aligned");
+  if (list_capacity == 0) return MTS_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int grid = c->sm_count * 8;
+  {
+    LaunchScope scope(K_CACHE_SAVE_VICTIMS, s);
+    cache_save_victims<<<grid, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, evict_slots, evict_dirty, counters,
+                                                      list_capacity, static_cast<char*>(evict_staging));
+  }
+  {
+    LaunchScope scope(K_CACHE_FETCH_MISSES, s);
+    cache_place_fetched<<<grid, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, static_cast<const char*>(fetched),
+                                                       miss_slots, counters, list_capacity);
+  }
+  return check_launch("cache_save_victims / cache_place_fetched");
+}
+
 extern "C" int mts_cache_writeback_evicted(mts_cache* c, void* host_rows_mapped, const int64_t* evict_keys,
                                            const uint8_t* evict_dirty, int64_t list_capacity,
                                            const int64_t* counters, const void* evict_staging, void* stream) {
@@ -812,7 +880,8 @@ extern "C" int mts_cache_writeback_evicted(mts_cache* c, void* host_rows_mapped,
 }
 
 extern "C" int mts_cache_refetch_overflowed(mts_cache* c, const void* host_rows_mapped, const int64_t* overflow_keys,
-                                            int64_t list_capacity, const int64_t* counters, void* stream) {
+                                            int64_t list_capacity, const int64_t* counters, int64_t placed_step,
+                                            void* stream) {
   if (!c || !host_rows_mapped || !counters || list_capacity < 0 || (list_capacity > 0 && !overflow_keys))
     return set_error(MTS_ERR_INVALID_ARG, "cache_refetch_overflowed: null argument");
   if ((uintptr_t)host_rows_mapped & 15) return set_error(MTS_ERR_ALIGNMENT, "cache_refetch_overflowed: host buffer alignment");
@@ -821,7 +890,7 @@ extern "C" int mts_cache_refetch_overflowed(mts_cache* c, const void* host_rows_
     LaunchScope scope(K_CACHE_FETCH_MISSES, static_cast<cudaStream_t>(stream));
     cache_refetch_resident<<<c->sm_count, CACHE_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
         c->data, c->row_bytes, static_cast<const char*>(host_rows_mapped), overflow_keys, counters, list_capacity,
-        c->tags, (uint64_t)c->S);
+        c->tags, c->ts, placed_step, (uint64_t)c->S);
   }
   return check_launch("cache_refetch_resident");
 }

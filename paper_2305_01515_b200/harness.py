@@ -198,19 +198,61 @@ class DeviceModel:
         mb.cache_prefetch_misses(self.caches[g], self.host_rows_ptr(g), L["miss_keys"], L["miss_slots"],
                                  L["evict_slots"], L["evict_dirty"], L["capacity"], L["counters"], L["staging"], stream)
 
+    # ---- missed rows gathered by host threads and moved by the copy engine
+    FETCH_STAGE_BYTES = 192 << 20        # per cache and batch context; larger miss lists take cache_fetch
+
+    def enable_host_gather(self, threads: Optional[int] = None) -> None:
+        """Pinned host buffers (keys and gathered rows, per cache and batch context) and one device
+        buffer per cache for the copy-engine path of the missed rows."""
+        import os
+        esz = 4 if self.spec.dtype == wl.FP32 else 2
+        self.gather_threads = threads or os.cpu_count() or 1
+        self.fetch_rows = [max(1, min(self.ctx[0]["lists"][g]["capacity"], self.FETCH_STAGE_BYTES // (c.dim * esz)))
+                           for g, c in enumerate(self.caches)]
+        self.fetch_dev = [torch.empty(r * c.dim * esz, dtype=torch.uint8, device=self.device)
+                          for r, c in zip(self.fetch_rows, self.caches)]
+        self.fetch_host = [[torch.empty(r * c.dim * esz, dtype=torch.uint8).pin_memory()
+                            for r, c in zip(self.fetch_rows, self.caches)] for _ in range(self.N_CTX)]
+        self.fetch_keys = [[torch.empty(r, dtype=torch.int64).pin_memory() for r in self.fetch_rows]
+                           for _ in range(self.N_CTX)]
+
+    def cache_fetch_via_host(self, g: int, n_miss: int, copy_stream, stream, ctx: int) -> bool:
+        """Cache g, copy-engine path: the first n_miss keys of the miss list come to the host on
+        `copy_stream` (the caller made it wait for the tag step), host threads gather the rows, one
+        contiguous copy and the placing kernel follow on `stream`.  Blocks the calling thread for the key
+        copy and the gather.  Returns False (nothing done) when the list does not fit the buffers."""
+        if n_miss > self.fetch_rows[g]:
+            return False
+        L = self.ctx[ctx]["lists"][g]
+        c = self.caches[g]
+        esz = 4 if self.spec.dtype == wl.FP32 else 2
+        rb = c.dim * esz
+        if n_miss > 0:
+            keys_h = self.fetch_keys[ctx][g]
+            with torch.cuda.stream(copy_stream):
+                keys_h[:n_miss].copy_(L["miss_keys"][:n_miss], non_blocking=True)
+            copy_stream.synchronize()
+            rows_h = self.fetch_host[ctx][g]
+            mb.host_gather_rows(self.host_rows_ptr(g), keys_h.numpy(), n_miss, rb, rows_h, self.gather_threads)
+            with torch.cuda.stream(stream):
+                self.fetch_dev[g][:n_miss * rb].copy_(rows_h[:n_miss * rb], non_blocking=True)
+        mb.cache_place_fetched(c, self.fetch_dev[g], L["miss_slots"], L["evict_slots"], L["evict_dirty"],
+                               L["capacity"], L["counters"], L["staging"], stream)
+        return True
+
     def cache_writeback(self, g: int, stream=None, ctx: Optional[int] = None) -> None:
         """Cache g: the staged dirty victims back to the host tier (after cache_fetch of the same batch)."""
         L = self.ctx[self.cur if ctx is None else ctx]["lists"][g]
         mb.cache_writeback_evicted(self.caches[g], self.host_rows_ptr(g), L["evict_keys"], L["evict_dirty"],
                                    L["capacity"], L["counters"], L["staging"], stream)
 
-    def cache_refetch(self, prev_ctx: int, stream=None) -> None:
+    def cache_refetch(self, prev_ctx: int, placed_step: int = -1, stream=None) -> None:
         """After the backward of the batch in context `prev_ctx`: refresh rows that overflowed there
-        and were placed by the next batch."""
+        and were placed by the next batch (the one whose lookup had step `placed_step`)."""
         for g, c in enumerate(self.caches):
             L = self.ctx[prev_ctx]["lists"][g]
             mb.cache_refetch_overflowed(c, self.host_rows_ptr(g), L["overflow_keys"], L["capacity"], L["counters"],
-                                        stream)
+                                        placed_step, stream)
 
     def cache_step(self, indices, offsets, offsets_host: np.ndarray, step: int, stream=None,
                    do_prefetch: bool = True, ctx: Optional[int] = None) -> None:

@@ -35,9 +35,15 @@ from .harness import DeviceModel
 
 
 class CachedTrainer:
-    def __init__(self, model: DeviceModel, pipelined: bool = True):
+    def __init__(self, model: DeviceModel, pipelined: bool = True, host_gather: bool = False):
+        """host_gather: missed rows are gathered by host threads into a pinned buffer and moved by the
+        copy engine, instead of being read over the host link by a kernel."""
         assert model.cached
         self.m = model
+        self.host_gather = host_gather
+        if host_gather:
+            model.enable_host_gather()
+        self._ev_prev_ready = None
         self.pipelined = pipelined
         self.dev = model.device
         self.main = torch.cuda.current_stream(self.dev)
@@ -47,6 +53,7 @@ class CachedTrainer:
         n_c = len(model.caches)
         self.moves = [torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main for _ in range(n_c)]
         self.fix = torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main
+        self.copy = torch.cuda.Stream(self.dev, priority=-1)       # miss keys to the host (host_gather)
         self.host_counters = [torch.zeros((n_c, mb.NUM_COUNTERS), dtype=torch.int64).pin_memory()
                               for _ in range(DeviceModel.N_CTX)]
         self.history: List[np.ndarray] = []           # per batch [n_caches, NUM_COUNTERS]
@@ -99,7 +106,21 @@ class CachedTrainer:
             self._mark(f"move{g}_begin", t, s)
             # fetch, then write back, in stream order: the next batch's fetch of this cache, which may
             # miss a row written back now, comes after it on the same stream
-            self.m.cache_fetch(g, stream=s, ctx=ctx)
+            done = False
+            if self.host_gather:
+                # the host reads the rows itself: the tag step of this batch is over (its counters are on
+                # the host), and every write-back of earlier batches has reached host memory (the
+                # previous batch's data movement is over)
+                if g == 0:
+                    ev_tags.synchronize()
+                    if self._ev_prev_ready is not None:
+                        self._ev_prev_ready.synchronize()
+                    if wait_bwd:
+                        prev_bwd.synchronize()
+                n_miss = int(self.host_counters[ctx][g][mb.COUNTER_NAMES.index("inserted")])
+                done = self.m.cache_fetch_via_host(g, n_miss, self.copy, s, ctx)
+            if not done:
+                self.m.cache_fetch(g, stream=s, ctx=ctx)
             self.m.cache_writeback(g, stream=s, ctx=ctx)
             self._mark(f"move{g}_end", t, s)
             e = torch.cuda.Event()
@@ -113,9 +134,10 @@ class CachedTrainer:
         if refetch:
             s.wait_event(prev_bwd)
             self._mark("refetch_begin", t, s)
-            self.m.cache_refetch((t - 1) % DeviceModel.N_CTX, stream=s)
+            self.m.cache_refetch((t - 1) % DeviceModel.N_CTX, placed_step=self._first_step + t, stream=s)
         self._mark("ready", t, s)
         ev_ready.record(s)
+        self._ev_prev_ready = ev_ready
 
     def _counters(self, t, ev_tags) -> int:
         ev_tags.synchronize()                        # counters of batch t are on the host
@@ -130,6 +152,7 @@ class CachedTrainer:
         K = len(batches)
         if K == 0:
             return
+        self._first_step = first_step
         ev_tags = [torch.cuda.Event() for _ in range(K)]
         ev_ready = [torch.cuda.Event() for _ in range(K)]
         ev_bwd = [torch.cuda.Event() for _ in range(K)]
@@ -169,6 +192,13 @@ class CachedTrainer:
             ev_bwd[t].record(self.main)
             if t + 1 < K:
                 overflow[t + 1] = self._counters(t + 1, ev_tags[t + 1])
+                if t >= 1:
+                    # a row that overflowed in batch t-1 (updated in host memory by its backward) and is
+                    # placed only now is fetched from host memory: after that backward
+                    for s in self.moves:
+                        s.wait_event(ev_bwd[t - 1])
+                    if self.host_gather:
+                        ev_bwd[t - 1].synchronize()
                 self._move(t + 1, ev_tags[t + 1], ev_ready[t + 1], overflow[t], ev_bwd[t])
             if t + 2 < K:
                 # the tag step of batch t+2 may evict rows stamped before t+2-lock_depth: the backward

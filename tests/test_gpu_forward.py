@@ -42,6 +42,20 @@ def test_mixed_dims_and_ragged_bags(dtype, mode):
     _run_and_compare(spec, mode=mode)
 
 
+@pytest.mark.parametrize("dtype", [wl.FP32, wl.FP16])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_rows_of_at_most_one_warp_pass(dtype, mode):
+    """No row wider than 32 16-byte chunks and no cached table: the launch takes the kernel specialised
+    for that case.  Every lane-group width from 1 to 32 chunks (whole powers of two and not), a table
+    change inside a warp's run of bags (batch 97 is no multiple of the bags per warp), empty bags and
+    bags of several 32-lookup tiles with a ragged tail."""
+    dims = [8, 16, 24, 64, 128, 200, 256, 104] if dtype == wl.FP16 else [4, 8, 12, 64, 128, 100, 32, 52]
+    rows = [50, 1000, 37, 5000, 20000, 300, 777, 129]
+    pool = [0.7, 3, 40, 70, 20, 5, 33, 2]
+    spec = custom_spec(rows, dims, 97, dtype, pool, [0, 1.1, 0, 1.05, 0.9, 0, 1.3, 0], seed=4)
+    _run_and_compare(spec, mode=mode)
+
+
 def test_dim_1024_fp32_and_fp16():
     for dtype in (wl.FP32, wl.FP16):
         _run_and_compare(custom_spec([300, 40], [1024, 64], 33, dtype, [6, 2], seed=5))
