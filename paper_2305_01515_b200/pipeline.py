@@ -190,6 +190,14 @@ class CachedTrainer:
             m.backward(idx, off, idx.numel(), grads[t], stream=self.main, ctx=t % DeviceModel.N_CTX)
             self._mark("bwd_end", t, self.main)
             ev_bwd[t].record(self.main)
+            if t + 2 < K:
+                # the tag step of batch t+2 may evict rows stamped before t+2-lock_depth: the backward
+                # of the last such batch must be over (with lock_depth 1 that is batch t, with 2 batch
+                # t-1); the context it writes was last used by batch t-1.  Enqueued before the data movement
+                # of batch t+1, whose host part (counters, row gather) blocks this thread
+                last = min(t, t + 1 - m.lock_depth)
+                self._lookup(t + 2, first_step + t + 2, batches[t + 2], ev_tags[t + 2],
+                             ev_bwd[last] if last >= 0 else None)
             if t + 1 < K:
                 overflow[t + 1] = self._counters(t + 1, ev_tags[t + 1])
                 if t >= 1:
@@ -200,13 +208,6 @@ class CachedTrainer:
                     if self.host_gather:
                         ev_bwd[t - 1].synchronize()
                 self._move(t + 1, ev_tags[t + 1], ev_ready[t + 1], overflow[t], ev_bwd[t])
-            if t + 2 < K:
-                # the tag step of batch t+2 may evict rows stamped before t+2-lock_depth: the backward
-                # of the last such batch must be over (with lock_depth 1 that is batch t, with 2 batch
-                # t-1); the context it writes was last used by batch t-1
-                last = min(t, t + 1 - m.lock_depth)
-                self._lookup(t + 2, first_step + t + 2, batches[t + 2], ev_tags[t + 2],
-                             ev_bwd[last] if last >= 0 else None)
             if on_step is not None:
                 on_step(t)
         self.main.wait_stream(self.tag)
