@@ -20,8 +20,12 @@ at t-1 or earlier, complete because the tag step waited for backward(t-1)) and t
 rows, which no batch in flight uses.  One hazard is left: a row that found no evictable way in batch
 t (it is read and updated in host memory directly) and is fetched from host memory for batch t+1,
 possibly before backward(t) has updated it.  When batch t reported such overflow, the data movement
-of batch t+1 still runs at once, and after backward(t) the rows of batch t's overflow list that are
-resident by then are copied from host memory again (mts_cache_refetch_overflowed).
+of batch t+1 still runs at once, and after backward(t) the rows of batch t's overflow list that batch
+t+1 placed are copied from host memory again (mts_cache_refetch_overflowed with placed_step = the step
+of batch t+1: the tag step of batch t+2 may already have placed other keys of that list, in slots that
+hold their victims' rows until batch t+2's data movement, and those must not be touched).  A row that
+overflowed in batch t-1 and is first placed by batch t+1 is covered by ordering: the data movement of
+batch t+1 waits for backward(t-1).
 """
 from __future__ import annotations
 
