@@ -216,7 +216,7 @@ class DeviceModel:
         self.fetch_keys = [[torch.empty(r, dtype=torch.int64).pin_memory() for r in self.fetch_rows]
                            for _ in range(self.N_CTX)]
 
-    def cache_fetch_via_host(self, g: int, n_miss: int, copy_stream, stream, ctx: int) -> bool:
+    def cache_fetch_via_host(self, g: int, n_miss: int, copy_stream, stream, ctx: int, mark=None) -> bool:
         """Cache g, copy-engine path: the first n_miss keys of the miss list come to the host on
         `copy_stream` (the caller made it wait for the tag step), host threads gather the rows, one
         contiguous copy and the placing kernel follow on `stream`.  Blocks the calling thread for the key
@@ -235,7 +235,11 @@ class DeviceModel:
             rows_h = self.fetch_host[ctx][g]
             mb.host_gather_rows(self.host_rows_ptr(g), keys_h.numpy(), n_miss, rb, rows_h, self.gather_threads)
             with torch.cuda.stream(stream):
+                if mark is not None:
+                    mark(f"copy{g}_begin")
                 self.fetch_dev[g][:n_miss * rb].copy_(rows_h[:n_miss * rb], non_blocking=True)
+                if mark is not None:
+                    mark(f"copy{g}_end")
         mb.cache_place_fetched(c, self.fetch_dev[g], L["miss_slots"], L["evict_slots"], L["evict_dirty"],
                                L["capacity"], L["counters"], L["staging"], stream)
         return True

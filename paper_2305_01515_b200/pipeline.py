@@ -122,9 +122,11 @@ class CachedTrainer:
                     if wait_bwd:
                         prev_bwd.synchronize()
                 n_miss = int(self.host_counters[ctx][g][mb.COUNTER_NAMES.index("inserted")])
-                done = self.m.cache_fetch_via_host(g, n_miss, self.copy, s, ctx)
+                done = self.m.cache_fetch_via_host(g, n_miss, self.copy, s, ctx,
+                                                   mark=(lambda name, s=s: self._mark(name, t, s)) if self.record_timeline else None)
             if not done:
                 self.m.cache_fetch(g, stream=s, ctx=ctx)
+            self._mark(f"placed{g}", t, s)
             self.m.cache_writeback(g, stream=s, ctx=ctx)
             self._mark(f"move{g}_end", t, s)
             e = torch.cuda.Event()
