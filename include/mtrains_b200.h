@@ -243,13 +243,15 @@ typedef struct mts_cache mts_cache;
  * lock_depth: a way stamped at step >= step - lock_depth is not evictable (Section 5.7: a
  * prefetched row is not evicted before its batch has trained).  Synchronous.
  * Errors: INVALID_ARG (num_sets < 1 or num_sets*32 >= 2^31, key_space >= 2^32 - 1, ways != 32),
- * ALIGNMENT, CUDA. */
+ * UNSUPPORTED (dim > 1024), ALIGNMENT, CUDA. */
 int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_space, int32_t ways, int32_t dim,
                      int32_t dtype, int32_t policy, int32_t lock_depth);
 int mts_cache_destroy(mts_cache* cache);
 /* Reads and clears the cache's sticky device status word; synchronises `stream`.  Bit 0: a
  * bounded wait for a bulk copy of missed rows ran out (the kernel gave up instead of hanging; the
- * rows of that call are incomplete) — also reported as MTS_ERR_TIMEOUT. */
+ * rows of that call are incomplete) — also reported as MTS_ERR_TIMEOUT.  Bit 1: a key outside
+ * [0, key_space) was passed to mts_cache_lookup_insert; it was clamped into the range (the call
+ * stays memory-safe, its result for that lookup is the clamped key's). */
 int mts_cache_status(mts_cache* cache, int32_t* host_status, void* stream);
 void* mts_cache_data(mts_cache* cache);        /* device [num_sets*32, dim] */
 uint8_t* mts_cache_dirty(mts_cache* cache);    /* device [num_sets*32] */

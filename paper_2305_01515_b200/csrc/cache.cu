@@ -36,6 +36,8 @@ namespace mts {
 
 constexpr uint32_t FREE_TAG = 0xffffffffu;
 constexpr int CACHE_THREADS = 256;
+constexpr int CACHE_STATUS_FETCH_TIMEOUT = 1;   // a bounded wait on a bulk copy ran out
+constexpr int CACHE_STATUS_KEY_RANGE = 2;       // a key outside [0, key_space) was clamped
 
 __device__ __forceinline__ uint32_t set_of_key(uint32_t key, uint64_t S) {
   const uint64_t x = (uint64_t)key * 0x9E3779B97F4A7C15ull;
@@ -48,14 +50,22 @@ __global__ void cache_init_state(uint32_t* tags, int32_t* ts, uint32_t* freq, ui
   }
 }
 
-__global__ void cache_prepare_keys(const int64_t* __restrict__ keys, int64_t n, uint32_t* __restrict__ k32,
-                                   uint32_t* __restrict__ pos, int64_t* __restrict__ counters,
-                                   uint32_t* __restrict__ overflow_cursor) {
+// A key outside [0, key_space) is clamped into the range (never sorted or probed as it is: the
+// sort only looks at the bits of key_space) and raises status bit 1.
+__global__ void cache_prepare_keys(const int64_t* __restrict__ keys, int64_t n, int64_t key_space,
+                                   uint32_t* __restrict__ k32, uint32_t* __restrict__ pos,
+                                   int64_t* __restrict__ counters, uint32_t* __restrict__ overflow_cursor,
+                                   int32_t* __restrict__ status) {
   const int64_t i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i0 < MTS_NUM_COUNTERS) counters[i0] = i0 == MTS_CNT_LOOKUPS ? n : 0;
   if (i0 == 0) *overflow_cursor = 0u;
   for (int64_t i = i0; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-    k32[i] = (uint32_t)keys[i];
+    int64_t k = keys[i];
+    if (k < 0 || k >= key_space) {
+      atomicOr(status, CACHE_STATUS_KEY_RANGE);
+      k = k < 0 ? 0 : key_space - 1;
+    }
+    k32[i] = (uint32_t)k;
     pos[i] = (uint32_t)i;
   }
 }
@@ -476,7 +486,7 @@ cache_fetch_misses_bulk(char* __restrict__ data, int row_bytes, const char* __re
     }
     bool ok = mbar_wait_bounded(bar, parity, FETCH_WAIT_LIMIT);
     if (!__syncthreads_and(ok)) {
-      if (threadIdx.x == 0) atomicOr(status, 1);
+      if (threadIdx.x == 0) atomicOr(status, CACHE_STATUS_FETCH_TIMEOUT);
       mbar_wait_bounded(bar, parity, FETCH_WAIT_LIMIT);
       return;
     }
@@ -594,6 +604,7 @@ extern "C" int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_s
   if (dtype != MTS_DTYPE_FP32 && dtype != MTS_DTYPE_FP16) return set_error(MTS_ERR_INVALID_ARG, "cache_create: dtype");
   if (policy != MTS_POLICY_LRU && policy != MTS_POLICY_LFU) return set_error(MTS_ERR_INVALID_ARG, "cache_create: policy");
   if (lock_depth < 0 || dim < 1) return set_error(MTS_ERR_INVALID_ARG, "cache_create: lock_depth / dim");
+  if (dim > 1024) return set_error(MTS_ERR_UNSUPPORTED, "cache_create: dim %d above 1024", dim);
   const int eb = dtype == MTS_DTYPE_FP32 ? 4 : 2;
   if ((dim * eb) % 16) return set_error(MTS_ERR_ALIGNMENT, "cache_create: row bytes %d not a multiple of 16", dim * eb);
   mts_cache* c = new mts_cache();
@@ -709,7 +720,8 @@ extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_
   const int grid = c->sm_count * 8;
   {
     LaunchScope scope(K_CACHE_PREPARE, s);
-    cache_prepare_keys<<<grid, 256, 0, s>>>(keys, N, U32(L.keys_a), U32(L.vals_a), counters, U32(L.ovf_cursor));
+    cache_prepare_keys<<<grid, 256, 0, s>>>(keys, N, c->key_space, U32(L.keys_a), U32(L.vals_a), counters,
+                                            U32(L.ovf_cursor), c->d_status);
   }
   int rc = check_launch("cache_prepare_keys");
   if (rc != MTS_OK) return rc;
@@ -871,7 +883,7 @@ extern "C" int mts_cache_writeback_evicted(mts_cache* c, void* host_rows_mapped,
     return set_error(MTS_ERR_ALIGNMENT, "cache_writeback_evicted: buffers must be 16-byte aligned");
   if (list_capacity == 0) return MTS_OK;
   {
-    LaunchScope scope(K_CACHE_WRITE_VICTIMS, nullptr);
+    LaunchScope scope(K_CACHE_WRITE_VICTIMS, static_cast<cudaStream_t>(stream));
     cache_write_victims<<<c->sm_count * 8, CACHE_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<char*>(host_rows_mapped), c->row_bytes, evict_keys, evict_dirty, counters, list_capacity,
         static_cast<const char*>(evict_staging));
@@ -901,12 +913,12 @@ extern "C" int mts_cache_flush(mts_cache* c, void* host_rows_mapped, void* strea
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int64_t n = c->S * MTS_CACHE_WAYS;
   {
-    LaunchScope scope(K_CACHE_FLUSH, nullptr);
+    LaunchScope scope(K_CACHE_FLUSH, s);
     cache_flush_rows<<<c->sm_count * 8, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, c->tags, c->dirty, n,
                                                                static_cast<char*>(host_rows_mapped));
   }
   {
-    LaunchScope scope(K_CACHE_FLUSH, nullptr);
+    LaunchScope scope(K_CACHE_FLUSH, s);
     cache_clear_dirty<<<c->sm_count * 4, 256, 0, s>>>(c->dirty, n);
   }
   return check_launch("cache_flush");
@@ -916,7 +928,7 @@ extern "C" int mts_cache_export_state(mts_cache* c, int64_t* tags, int64_t* time
                                       uint8_t* dirty, void* stream) {
   if (!c) return set_error(MTS_ERR_INVALID_ARG, "cache_export_state: null cache");
   {
-    LaunchScope scope(K_OTHER, nullptr);
+    LaunchScope scope(K_OTHER, static_cast<cudaStream_t>(stream));
     cache_export<<<c->sm_count * 4, 256, 0, static_cast<cudaStream_t>(stream)>>>(
         c->tags, c->ts, c->freq, c->dirty, c->S * MTS_CACHE_WAYS, tags, timestamps, counts, dirty);
   }

@@ -850,7 +850,7 @@ extern "C" int mts_tbe_backward_sort(const mts_tables* h, int32_t B, const int64
     rc = unique_segments(keys, N, nullptr, seg_start, nullptr, n_unique, reinterpret_cast<uint32_t*>(ws + L.scan), s);
     if (rc != MTS_OK) return rc;
     {
-      LaunchScope scope(K_UNIQUE, nullptr);
+      LaunchScope scope(K_UNIQUE, s);
       export_unique<<<h->sm_count * 4, 256, 0, s>>>(keys, seg_start, n_unique, uniq_rows_out, n_unique_out);
     }
     rc = check_launch("export_unique");

@@ -202,6 +202,9 @@ class CachedTrainer:
                 # t-1); the context it writes was last used by batch t-1.  Enqueued before the data movement
                 # of batch t+1, whose host part (counters, row gather) blocks this thread
                 last = min(t, t + 1 - m.lock_depth)
+                # it rewrites the context of batch t-1, whose overflow list and counters the repair step
+                # inside the data movement of batch t still reads: after that
+                self.tag.wait_event(ev_ready[t])
                 self._lookup(t + 2, first_step + t + 2, batches[t + 2], ev_tags[t + 2],
                              ev_bwd[last] if last >= 0 else None)
             if t + 1 < K:

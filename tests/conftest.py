@@ -35,3 +35,23 @@ def _built_libraries():
     if shutil.which("nvcc") or os.path.exists("/usr/local/cuda/bin/nvcc"):
         build.build_library()
     yield
+
+
+def pytest_terminal_summary(terminalreporter, exitstatus, config):
+    """Floating-point parity actually observed: the plain max|diff| / max|ref| of every tolerance check,
+    and the share of its per-element bound rtol * (|ref| + mag) the worst element used."""
+    try:
+        from helpers import PARITY_LOG
+    except ImportError:
+        return
+    if not PARITY_LOG:
+        return
+    worst = {}
+    for what, plain, used, rtol, n in PARITY_LOG:
+        key = (what.rstrip("0123456789 ").strip() or "(unnamed)", rtol)
+        w = worst.setdefault(key, [0.0, 0.0, 0, 0])
+        w[0], w[1], w[2], w[3] = max(w[0], plain), max(w[1], used), w[2] + 1, w[3] + n
+    terminalreporter.write_line("floating-point parity (worst over the checks of a kind):")
+    terminalreporter.write_line("  kind | rtol | checks | elements | max|diff|/max|ref| | worst |diff|/bound")
+    for (what, rtol), (plain, used, checks, n) in sorted(worst.items()):
+        terminalreporter.write_line(f"  {what} | {rtol:g} | {checks} | {n} | {plain:.3e} | {used:.3f}")

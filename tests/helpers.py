@@ -17,12 +17,21 @@ def storage_dtype(spec):
     return np.float32 if spec.dtype == wl.FP32 else np.float16
 
 
+PARITY_LOG = []     # (what, plain max|diff| / max|ref|, largest |diff| / bound, rtol, elements); printed at session end
+
+
 def assert_close_mag(got, ref, mag, rtol, what=""):
-    """|got - ref| <= rtol * (|ref| + mag), element by element."""
+    """|got - ref| <= rtol * (|ref| + mag), element by element.  Also records the plain
+    max|diff| / max|ref| and how much of the bound the worst element used."""
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)
     bound = rtol * (np.abs(ref) + np.asarray(mag, dtype=np.float64))
     err = np.abs(got - ref)
+    if err.size:
+        with np.errstate(divide="ignore", invalid="ignore"):
+            used = np.where(bound > 0, err / bound, np.where(err > 0, np.inf, 0.0))
+        PARITY_LOG.append((what, float(err.max() / max(np.abs(ref).max(), 1e-300)), float(used.max()), rtol,
+                           int(err.size)))
     bad = err > bound
     if bad.any():
         k = np.argmax(err - bound)

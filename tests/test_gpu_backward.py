@@ -16,18 +16,19 @@ def _weights_f64(spec, W):
     return W.astype(np.float64)
 
 
-def _run_steps(spec, n_steps=2, mode=0, batches=None, lr=None, grad_f16=False):
+def _run_steps(spec, n_steps=2, mode=0, batches=None, lr=None, grad_f16=False, m0=None, grad_fn=None):
     """n_steps train steps on GPU and oracle; compares weights, momentum and unique rows.
     grad_f16: the upstream gradient is rounded to binary16 first; the oracle gets those values in fp32 (the
     conversion is exact), the GPU gets the binary16 tensor (mts_tbe_backward_apply_f16)."""
     lr = spec.lr if lr is None else lr
     W0 = wl.all_weights_numpy(spec)
     W_ref = W0.copy()
-    m_ref = np.zeros(int(spec.row_offset[-1]), np.float32)
+    m_ref = np.zeros(int(spec.row_offset[-1]), np.float32) if m0 is None else m0.astype(np.float32).copy()
     model = DeviceModel(spec, weights=W0)
+    model.momentum.copy_(torch.from_numpy(m_ref))
     for k in range(n_steps):
         idx, off = batches[k] if batches is not None else wl.gen_batch(spec, k)
-        grad = wl.gen_grad(spec, k)
+        grad = wl.gen_grad(spec, k) if grad_fn is None else grad_fn(k)
         if grad_f16:
             grad = grad.astype(np.float16).astype(np.float32)
         N = len(idx)
@@ -102,6 +103,31 @@ def test_lookup_counts_around_chunk_and_tile_borders():
     for n in (1, 127, 128, 129, 4095, 4096, 4097):
         spec = custom_spec([50], [64], 1, wl.FP32, [n], bag_dist="fixed", seed=n)
         _run_steps(spec, n_steps=1)
+
+
+def test_zero_gradient_leaves_weights_and_state_alone():
+    """All-zero upstream gradient on fresh state: m stays 0, the step size is lr / eps times a zero gradient."""
+    for dtype in (wl.FP32, wl.FP16):
+        spec = custom_spec([40, 3000], [64, 256], 33, dtype, [6, 20], [0, 1.1], seed=8)
+        zero = lambda k: np.zeros((spec.batch, spec.total_dim), np.float32)
+        _run_steps(spec, n_steps=2, grad_fn=zero)
+        # zero gradient for one table only, and for single columns
+        def partly(k):
+            g = wl.gen_grad(spec, k)
+            g[:, :64] = 0.0
+            g[:, 64::7] = 0.0
+            return g
+        _run_steps(spec, n_steps=2, grad_fn=partly)
+
+
+def test_step_on_rows_whose_state_is_already_large_or_tiny():
+    """Adagrad state far from its initial value: 1e6 (tiny steps), 1e-12 (steps near lr * g / eps scale)
+    and a mix, two steps each."""
+    spec = custom_spec([500, 2000], [128, 64], 64, wl.FP32, [10, 15], [1.05, 0.9], seed=9)
+    n = int(spec.row_offset[-1])
+    rng = np.random.default_rng(3)
+    for m0 in (np.full(n, 1e6), np.full(n, 1e-12), 10.0 ** rng.uniform(-10, 6, n)):
+        _run_steps(spec, n_steps=2, m0=m0)
 
 
 def test_empty_batch_is_a_no_op():

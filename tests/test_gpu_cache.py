@@ -171,7 +171,7 @@ def test_cached_training_matches_oracle_and_is_transparent(dtype, frac, lock):
     np.testing.assert_array_equal(W_host.view(np.uint8), W_plain.view(np.uint8))      # transparency (oracle)
     np.testing.assert_array_equal(m_o, m_plain)
     if frac < 0.05:
-        assert total_overflow >= 0
+        assert total_overflow > 0          # the small cache really sent rows around the cache
     for oc in ocaches:
         oc.close()
     model.close()

@@ -12,14 +12,19 @@ from helpers import small_spec
 
 class ListCache:
     """Naive per-set simulation with python lists; same contract, different construction:
-    each set is a list of [way, key, stamp, dirty] kept sorted by (stamp, way)."""
+    each set is a list of [way, key, stamp, dirty, count]; victims are taken in (stamp, way) order
+    for LRU and in (count, stamp, way) order for LFU, where count = lookups of the key while it has
+    been resident (every occurrence in a batch counts), starting at the inserting batch's lookups."""
 
-    def __init__(self, S, ways, lock_depth=0):
-        self.S, self.ways, self.lock = S, ways, lock_depth
-        self.sets = [[[w, -1, -1, 0] for w in range(ways)] for _ in range(S)]
+    def __init__(self, S, ways, lock_depth=0, policy=0):
+        self.S, self.ways, self.lock, self.policy = S, ways, lock_depth, policy
+        self.sets = [[[w, -1, -1, 0, 0] for w in range(ways)] for _ in range(S)]
 
     def step(self, keys, step):
         uniq = sorted(set(int(k) for k in keys))
+        times = {}
+        for k in keys:
+            times[int(k)] = times.get(int(k), 0) + 1
         by_set = {}
         for k in uniq:
             by_set.setdefault(oracle.cache_set_of(k, self.S), []).append(k)
@@ -33,9 +38,13 @@ class ListCache:
             for e in self.sets[s]:
                 if e[1] in hits and e[1] in ks:
                     e[2] = step
+                    e[4] += times[e[1]]
         miss, evict, overflow = [], [], 0
         for s in sorted(by_set):
-            order = sorted(self.sets[s], key=lambda e: (e[2], e[0]))
+            if self.policy == 1:
+                order = sorted(self.sets[s], key=lambda e: (e[4], e[2], e[0]))
+            else:
+                order = sorted(self.sets[s], key=lambda e: (e[2], e[0]))
             cands = [e for e in order if e[1] == -1 or e[2] < step - self.lock]
             todo = [k for k in by_set[s] if k not in hits]
             for j, k in enumerate(todo):
@@ -43,7 +52,7 @@ class ListCache:
                     e = cands[j]
                     if e[1] != -1:
                         evict.append((e[1], s * self.ways + e[0], e[3]))
-                    e[1], e[2], e[3] = k, step, 0
+                    e[1], e[2], e[3], e[4] = k, step, 0, times[k]
                     slot[k] = s * self.ways + e[0]
                     miss.append((k, slot[k]))
                 else:
@@ -63,11 +72,14 @@ def _check_invariants(c, S, ways):
     assert (tags >= 0).sum() <= S * ways
 
 
+@pytest.mark.parametrize("policy", [0, 1])
 @pytest.mark.parametrize("S,ways,lock", [(1, 4, 0), (5, 4, 0), (7, 32, 1), (3, 2, 1), (16, 8, 2)])
-def test_lookup_insert_vs_list_simulation(S, ways, lock):
+def test_lookup_insert_vs_list_simulation(S, ways, lock, policy):
+    """LRU and LFU against the list simulation; the Zipf keys repeat inside a batch (multiplicities
+    up to dozens) and small universes give many equal counts, so count ties are frequent."""
     rng = np.random.default_rng(S * 100 + ways)
-    c = oracle.Cache(S, ways, 4, wl.FP32, 0, lock, with_data=False)
-    ref = ListCache(S, ways, lock)
+    c = oracle.Cache(S, ways, 4, wl.FP32, policy, lock, with_data=False)
+    ref = ListCache(S, ways, lock, policy)
     occupancy = 0
     for step in range(40):
         n = int(rng.integers(0, 3 * S * ways // 2 + 2))
@@ -89,6 +101,10 @@ def test_lookup_insert_vs_list_simulation(S, ways, lock):
         occupancy += cnt["inserted"] - cnt["evicted"]
         assert occupancy == int((c.tags >= 0).sum())
         _check_invariants(c, S, ways)
+        for s_i in range(S):
+            for e in ref.sets[s_i]:
+                if e[1] >= 0:
+                    assert int(c.freq[s_i][e[0]]) == e[4], "use count"
         # mark the slots of every second distinct key dirty on both sides
         for k in sorted(set(keys.tolist()))[::2]:
             sl = slot[k]
@@ -194,6 +210,61 @@ def test_lfu_keeps_frequent_rows():
         c.lookup_insert(np.array([7], np.int64), step)
     c.lookup_insert(np.array([8], np.int64), 5)
     assert c.lookup_insert(np.array([9], np.int64), 6)["evict_keys"].tolist() == [7]
+    c.close()
+
+
+def _one_set(policy, ways=2, lock=0):
+    return oracle.Cache(1, ways, 4, wl.FP32, policy, lock, with_data=False)
+
+
+def test_lfu_counts_lookups_not_distinct_keys():
+    """Key 7 is looked up three times in one batch, key 8 once in each of two batches: by lookups 8 is
+    the less used (2 < 3) and is evicted; counting batches (or distinct keys) would evict 7."""
+    c = _one_set(1)
+    c.lookup_insert(np.array([7, 7, 7], np.int64), 0)
+    c.lookup_insert(np.array([8], np.int64), 1)
+    c.lookup_insert(np.array([8], np.int64), 2)
+    assert c.freq[0].tolist() == [3, 2]
+    res = c.lookup_insert(np.array([9], np.int64), 3)
+    assert res["evict_keys"].tolist() == [8]
+    c.close()
+
+
+def test_lfu_count_ties_fall_back_to_timestamp_then_way():
+    c = _one_set(1, ways=3)
+    c.lookup_insert(np.array([1, 2, 3], np.int64), 0)       # ways 0, 1, 2 (ascending key), counts 1, 1, 1
+    c.lookup_insert(np.array([1], np.int64), 1)             # key 1: count 2
+    c.lookup_insert(np.array([3], np.int64), 2)             # key 3: count 2, newer than key 1
+    c.lookup_insert(np.array([2], np.int64), 3)             # key 2: count 2, newest
+    res = c.lookup_insert(np.array([10], np.int64), 4)      # all counts equal: the oldest stamp goes
+    assert res["evict_keys"].tolist() == [1]
+    c.close()
+    c = _one_set(1, ways=3)
+    c.lookup_insert(np.array([1, 2, 3], np.int64), 0)       # same count, same stamp: lowest way first
+    res = c.lookup_insert(np.array([10, 11], np.int64), 1)
+    assert res["evict_keys"].tolist() == [1, 2] and res["evict_slots"].tolist() == [0, 1]
+    c.close()
+
+
+def test_lfu_count_restarts_when_a_key_is_inserted_again():
+    c = _one_set(1)
+    for step in range(6):
+        c.lookup_insert(np.array([7], np.int64), step)                       # key 7: count 6
+    c.lookup_insert(np.array([8, 8], np.int64), 6)                          # key 8: count 2
+    assert c.lookup_insert(np.array([9, 9, 9], np.int64), 7)["evict_keys"].tolist() == [8]   # key 9: count 3
+    assert c.lookup_insert(np.array([8, 8, 8, 8], np.int64), 8)["evict_keys"].tolist() == [9]
+    assert sorted(c.freq[0].tolist()) == [4, 6]               # key 8 starts again at this batch's 4 lookups
+    c.close()
+
+
+def test_lfu_lock_window_overrides_the_count():
+    """A rarely used row stamped inside the lock window is not a candidate; the frequently used one goes."""
+    c = _one_set(1, lock=1)
+    for step in range(4):
+        c.lookup_insert(np.array([7, 7], np.int64), step)                    # key 7: count 8, stamp 3
+    c.lookup_insert(np.array([8], np.int64), 4)                             # key 8: count 1, stamp 4
+    res = c.lookup_insert(np.array([9], np.int64), 5)                       # 8 is locked (4 >= 5 - 1)
+    assert res["evict_keys"].tolist() == [7]
     c.close()
 
 
