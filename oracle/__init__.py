@@ -197,16 +197,18 @@ class Cache:
         except Exception:
             pass
 
-    def lookup_insert(self, keys, step: int):
+    def lookup_insert(self, keys, step: int, list_capacity: Optional[int] = None):
+        """list_capacity: entries the miss list may hold (default: no limit)."""
         keys = _i64(keys)
         N = len(keys)
         cap = max(N, 1)
+        list_capacity = cap if list_capacity is None else int(list_capacity)
         slot = np.full(cap, -1, dtype=np.int32)
         mk = np.zeros(cap, np.int64); msl = np.zeros(cap, np.int32)
         ek = np.zeros(cap, np.int64); esl = np.zeros(cap, np.int32); ed = np.zeros(cap, np.uint8)
         cnt = np.zeros(NCOUNTERS, np.int64)
         lib().orc_cache_lookup_insert(self._h, _p(keys), C.c_int64(N), C.c_int64(step), _p(slot),
-                                      _p(mk), _p(msl), _p(ek), _p(esl), _p(ed), _p(cnt))
+                                      _p(mk), _p(msl), _p(ek), _p(esl), _p(ed), C.c_int64(list_capacity), _p(cnt))
         nm, ne = int(cnt[6]), int(cnt[7])
         return dict(slot_of_lookup=slot[:N], miss_keys=mk[:nm], miss_slots=msl[:nm],
                     evict_keys=ek[:ne], evict_slots=esl[:ne], evict_dirty=ed[:ne],

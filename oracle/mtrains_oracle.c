@@ -341,14 +341,16 @@ static int64_t find_way(const orc_cache* c, int64_t set, int64_t key) {
  *     step - lock_depth (free ways have ts = -1, so they are taken first).  Candidates are ordered by (ts, way) for LRU and by
  *     (count, ts, way) for LFU; the k-th missing key takes the k-th candidate.  A victim
  *     with a valid tag is appended to the evict list with its dirty byte, which is then
- *     cleared.  Misses beyond the candidates are not inserted: slot -1 (overflow).
+ *     cleared.  Misses beyond the candidates are not inserted: slot -1 (overflow).  The miss
+ *     list holds at most list_capacity entries: once it is full, every further missing key is
+ *     treated like one without a candidate (not inserted, slot -1, counted as overflow).
  *  4. slot = set * ways + way.  miss list order: (set, key).
- * slot_of_lookup[i] receives the slot of keys[i] (or -1).  Lists need capacity >= the
- * number of distinct keys.  Returns the number of distinct keys. */
+ * slot_of_lookup[i] receives the slot of keys[i] (or -1).  The lists hold list_capacity entries
+ * (the number of distinct keys is always enough).  Returns the number of distinct keys. */
 int64_t orc_cache_lookup_insert(orc_cache* c, const int64_t* keys, int64_t N, int64_t step,
                                 int32_t* slot_of_lookup, int64_t* miss_keys, int32_t* miss_slots,
                                 int64_t* evict_keys, int32_t* evict_slots, uint8_t* evict_dirty,
-                                int64_t* counters) {
+                                int64_t list_capacity, int64_t* counters) {
     for (int k = 0; k < ORC_NCOUNTERS; ++k) counters[k] = 0;
     counters[0] = N;
     if (N == 0) return 0;
@@ -414,7 +416,7 @@ int64_t orc_cache_lookup_insert(orc_cache* c, const int64_t* keys, int64_t N, in
         for (int64_t k = a; k < z; ++k) {
             int64_t key = ms[k].key;
             int64_t slot = -1;
-            if (k - a < nc) {
+            if (k - a < nc && n_miss < list_capacity) {
                 slot = set * c->ways + cand[k - a];
                 if (c->tag[slot] != -1) {
                     evict_keys[n_evict] = c->tag[slot];

@@ -20,7 +20,7 @@ class ListCache:
         self.S, self.ways, self.lock, self.policy = S, ways, lock_depth, policy
         self.sets = [[[w, -1, -1, 0, 0] for w in range(ways)] for _ in range(S)]
 
-    def step(self, keys, step):
+    def step(self, keys, step, capacity=None):
         uniq = sorted(set(int(k) for k in keys))
         times = {}
         for k in keys:
@@ -48,7 +48,7 @@ class ListCache:
             cands = [e for e in order if e[1] == -1 or e[2] < step - self.lock]
             todo = [k for k in by_set[s] if k not in hits]
             for j, k in enumerate(todo):
-                if j < len(cands):
+                if j < len(cands) and (capacity is None or len(miss) < capacity):
                     e = cands[j]
                     if e[1] != -1:
                         evict.append((e[1], s * self.ways + e[0], e[3]))
@@ -114,6 +114,45 @@ def test_lookup_insert_vs_list_simulation(S, ways, lock, policy):
                     if e[0] == sl % ways:
                         e[3] = 1
     c.close()
+
+
+@pytest.mark.parametrize("policy", [0, 1])
+def test_full_miss_list_turns_further_misses_into_overflow(policy):
+    """A miss list of `capacity` entries: the first `capacity` placements (in set, key order) stand, every
+    later missing key is not inserted and its would-be victim keeps its way.  Checked against the list
+    simulation, and against the unlimited call when the capacity is not reached."""
+    S, ways = 6, 4
+    rng = np.random.default_rng(11 + policy)
+    c = oracle.Cache(S, ways, 4, wl.FP32, policy, 1, with_data=False)
+    twin = oracle.Cache(S, ways, 4, wl.FP32, policy, 1, with_data=False)      # same calls, generous capacity
+    ref = ListCache(S, ways, 1, policy)
+    cut = whole = 0
+    for step in range(30):
+        keys = (rng.zipf(1.3, 40) % 150).astype(np.int64)
+        cap = int(rng.integers(0, 12))
+        # the same call without a limit, on a copy of the state
+        twin.tags[:], twin.ts[:], twin.freq[:], twin.dirty[:] = c.tags, c.ts, c.freq, c.dirty
+        free = twin.lookup_insert(keys, step)
+        res = c.lookup_insert(keys, step, list_capacity=cap)
+        slot, miss, evict, overflow, n_hit, n_uhit = ref.step(keys, step, capacity=cap)
+        cnt = res["counters"]
+        assert cnt["inserted"] == len(miss) <= cap and cnt["evicted"] == len(evict) and cnt["overflow"] == overflow
+        assert cnt["unique_misses"] == cnt["inserted"] + cnt["overflow"]
+        assert [slot[int(k)] for k in keys] == res["slot_of_lookup"].tolist()
+        assert miss == list(zip(res["miss_keys"].tolist(), res["miss_slots"].tolist()))
+        assert [(k, s) for k, s, _ in evict] == list(zip(res["evict_keys"].tolist(), res["evict_slots"].tolist()))
+        _check_invariants(c, S, ways)
+        if free["counters"]["inserted"] <= cap:          # the limit was not reached: nothing may differ
+            whole += 1
+            assert free["counters"] == cnt
+            assert (free["slot_of_lookup"] == res["slot_of_lookup"]).all()
+            assert (twin.tags == c.tags).all() and (twin.ts == c.ts).all() and (twin.freq == c.freq).all()
+        else:
+            cut += 1
+            # the placements that fit are the first ones of the unlimited call
+            assert free["miss_keys"][:cap].tolist() == res["miss_keys"].tolist()
+    assert cut > 5 and whole > 2
+    c.close(); twin.close()
 
 
 def test_textbook_fully_associative_lru():
