@@ -201,6 +201,26 @@ int mts_tbe_backward_apply_f16(const mts_tables* tables, int32_t B, const int64_
                                void* const* host_cache_data, uint8_t* const* host_cache_dirty,
                                int32_t n_caches, void* workspace, size_t workspace_bytes, void* stream);
 
+/* The gradient half of the backward on lookups that are already ordered by row (Section 5.9; the
+ * cache's tag lookup, Section 5.5.1, orders a batch's requests by row for its own purposes, and the
+ * backward of the same batch can reuse that order instead of sorting again).
+ *   sorted_rows[p]   : linear row id (row_offset[t] + index) of the p-th lookup in ascending row order,
+ *   sorted_pos[p]    : that lookup's position in `indices`; equal rows in ascending position,
+ *   bag_of_lookup[i] : bag id t*B + b of the lookup at position i,
+ * all device uint32 [N], covering every lookup of the batch — as written by
+ * mts_cache_lookup_insert_tables calls that together cover all tables (every table cached).  The
+ * arrays are trusted: rows outside the tables or an order that is not ascending give undefined
+ * results.  grad_dtype: MTS_DTYPE_FP32 (float) or MTS_DTYPE_FP16 (binary16) gradient.  The
+ * workspace is the one of mts_tbe_backward_workspace_bytes; mts_tbe_backward_sort is not needed.
+ * Same arithmetic, summation order and errors as mts_tbe_backward_apply. */
+int mts_tbe_backward_apply_presorted(const mts_tables* tables, int32_t B, const int64_t* offsets, int64_t N,
+                                     int32_t pooling_mode, const void* grad_out, int32_t grad_dtype,
+                                     int64_t grad_stride, float lr, float eps, const uint32_t* sorted_rows,
+                                     const uint32_t* sorted_pos, const uint32_t* bag_of_lookup,
+                                     const int32_t* slot_of_lookup, void* const* host_cache_data,
+                                     uint8_t* const* host_cache_dirty, int32_t n_caches, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+
 /* Backward without a workspace argument and without any allocation (the paper has no
  * counterpart; this exists for callers of this library that cannot allocate device memory).
  * Such callers are, for example, a training or serving loop embedded in a framework that
@@ -251,7 +271,8 @@ int mts_cache_destroy(mts_cache* cache);
  * bounded wait for a bulk copy of missed rows ran out (the kernel gave up instead of hanging; the
  * rows of that call are incomplete) — also reported as MTS_ERR_TIMEOUT.  Bit 1: a key outside
  * [0, key_space) was passed to mts_cache_lookup_insert; it was clamped into the range (the call
- * stays memory-safe, its result for that lookup is the clamped key's). */
+ * stays memory-safe, its result for that lookup is the clamped key's).  Bit 2: a miss list was
+ * full and later missing keys were not inserted (see mts_cache_lookup_insert). */
 int mts_cache_status(mts_cache* cache, int32_t* host_status, void* stream);
 void* mts_cache_data(mts_cache* cache);        /* device [num_sets*32, dim] */
 uint8_t* mts_cache_dirty(mts_cache* cache);    /* device [num_sets*32] */
@@ -276,8 +297,10 @@ int mts_linearize_keys(const mts_tables* tables, int32_t t_begin, int32_t t_end,
  *  4. slot = set * 32 + way; slot_of_lookup[i] = slot of keys[i].
  * miss list {key, slot} is ordered by (set, key); evict list {old key, slot, dirty} by (set,
  * order of the misses that displaced them).  list_capacity >= number of distinct keys is always
- * enough; entries beyond the capacity are dropped while MTS_CNT_INSERTED / MTS_CNT_EVICTED
- * keep counting, so a counter above list_capacity tells the caller that a list was cut.
+ * enough.  When the miss list is full, every further missing key is treated like one without an
+ * evictable way: it is not inserted (slot -1), its victim keeps its way, and it is counted in
+ * MTS_CNT_OVERFLOW and listed in overflow_keys; bit 2 of mts_cache_status records that this
+ * happened.  MTS_CNT_INSERTED and MTS_CNT_EVICTED are the lengths of the lists.
  * overflow_keys (nullable, device int64 [list_capacity]): the keys counted in MTS_CNT_OVERFLOW, in no
  * particular order (see mts_cache_refetch_overflowed).
  * counters: device int64 [MTS_NUM_COUNTERS], overwritten.  `step` must not decrease between calls.
@@ -289,6 +312,30 @@ int mts_cache_lookup_insert(mts_cache* cache, const int64_t* keys, int64_t N, in
                             int64_t* evict_keys, int32_t* evict_slots, uint8_t* evict_dirty,
                             int64_t* overflow_keys, int64_t list_capacity, int64_t* counters,
                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* The same tag/state lookup and replacement, fed from a batch's sparse input instead of a key
+ * array (Sections 5.5.1, 5.5.2 and the per-table metadata of Section 5.8): the lookups of tables
+ * [t_begin, t_end) — one cache's table group, whose rows must add up to the cache's key_space — are
+ * positions [lookup_begin, lookup_begin + n) = [offsets[t_begin*B], offsets[t_end*B]) of `indices`;
+ * the key of a lookup is its row id relative to the group.  Differences from mts_cache_lookup_insert:
+ *   - slot_of_lookup is the batch-wide array (int32 [>= lookup_begin + n]); the call writes the
+ *     entries of its own lookups, slot_of_lookup[i] for position i;
+ *   - the overflow list has a capacity of its own (overflow_capacity; n is always enough);
+ *   - sorted_rows_out, sorted_pos_out, bag_of_lookup_out (all NULL, or the first two, or all three;
+ *     batch-wide device uint32 arrays): entries [lookup_begin, lookup_begin + n) receive the group's
+ *     lookups ordered by row — linear row id row_offset[t] + index ascending, equal rows in ascending
+ *     position — and their positions; bag_of_lookup_out[i] = t*B + b for the positions of the group.
+ *     Calls for all groups of a batch fill the arrays mts_tbe_backward_apply_presorted consumes.
+ * An index outside [0, rows[t]) is clamped and raises bit 0 of mts_tables_status. */
+int mts_cache_lookup_insert_tables(mts_cache* cache, const mts_tables* tables, int32_t t_begin, int32_t t_end,
+                                   int32_t B, const int64_t* indices, const int64_t* offsets,
+                                   int64_t lookup_begin, int64_t n, int64_t step, int32_t* slot_of_lookup,
+                                   int64_t* miss_keys, int32_t* miss_slots, int64_t* evict_keys,
+                                   int32_t* evict_slots, uint8_t* evict_dirty, int64_t list_capacity,
+                                   int64_t* overflow_keys, int64_t overflow_capacity, int64_t* counters,
+                                   uint32_t* sorted_rows_out, uint32_t* sorted_pos_out,
+                                   uint32_t* bag_of_lookup_out, void* workspace, size_t workspace_bytes,
+                                   void* stream);
 
 /* Data movement for one lookup_insert result (Sections 5.5.3, 5.5.4): first the rows of dirty
  * victims are saved, slot -> evict_staging[k] (k = position in the evict list), then every
@@ -321,15 +368,17 @@ int mts_cache_writeback_evicted(mts_cache* cache, void* host_rows_mapped, const 
                                 const uint8_t* evict_dirty, int64_t list_capacity,
                                 const int64_t* counters, const void* evict_staging, void* stream);
 
-/* Support for running the data movement of batch t+1 while batch t still trains (Section 5.7).
- * A key that overflowed in batch t is read and updated in the host tier by batch t's forward and
- * backward; if batch t+1 places that key, mts_cache_prefetch_misses(t+1) may have copied the host
- * row before batch t's update reached it.  Call this after batch t's backward with batch t's
- * overflow list and counters: every listed key that is resident now, in a way stamped `placed_step`
- * (the `step` of batch t+1's lookup_insert; -1 = any stamp), gets its row copied from the host tier
- * again.  The stamp keeps the call away from a key that a tag step running further ahead (batch t+2)
- * has placed meanwhile: that slot still holds its victim's row until batch t+2's data movement.
- * A no-op when the steps run one after the other. */
+/* Support for running the data movement of a batch while earlier batches still train (Section 5.7).
+ * A key that overflowed in batch u is read and updated in the host tier by batch u's forward and
+ * backward; if a later batch t inserts that key and its data movement runs before batch u's backward,
+ * the copy it takes of the host row is stale.  Call this after batch u's backward and batch t's data
+ * movement with batch u's overflow list and counters: every listed key whose row was inserted by the
+ * lookup_insert call with step `placed_step` (batch t's; -1 = whichever call inserted it) gets its row
+ * copied from the host tier again.  The cache remembers the step at which each resident row was inserted,
+ * apart from its timestamp, so the call leaves alone both a row inserted earlier (it has been updated in
+ * its slot since, the host copy is the older one) and a key that a tag step running further ahead has
+ * inserted meanwhile (that slot still holds its victim's row until that batch's data movement).
+ * list_capacity: capacity of the overflow list.  A no-op when the steps run one after the other. */
 int mts_cache_refetch_overflowed(mts_cache* cache, const void* host_rows_mapped, const int64_t* overflow_keys,
                                  int64_t list_capacity, const int64_t* counters, int64_t placed_step,
                                  void* stream);

@@ -31,7 +31,8 @@ EXPORTS = (
     "mts_tbe_backward_rowwise_adagrad_static", "mts_tbe_backward_sort", "mts_tbe_backward_apply",
     "mts_tbe_forward_f16", "mts_tbe_backward_apply_f16",
     "mts_cache_create", "mts_cache_destroy", "mts_cache_status", "mts_cache_data", "mts_cache_dirty",
-    "mts_linearize_keys", "mts_cache_workspace_bytes", "mts_cache_lookup_insert",
+    "mts_linearize_keys", "mts_cache_workspace_bytes", "mts_cache_lookup_insert", "mts_cache_lookup_insert_tables",
+    "mts_tbe_backward_apply_presorted",
     "mts_cache_prefetch_misses", "mts_host_gather_rows", "mts_cache_place_fetched", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
     "mts_cache_export_state",
 )
@@ -100,6 +101,10 @@ def lib():
         L.mts_cache_workspace_bytes.restype = sz
         L.mts_cache_workspace_bytes.argtypes = [vp, i64]
         L.mts_cache_lookup_insert.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
+        L.mts_cache_lookup_insert_tables.argtypes = [vp, vp, i32, i32, i32, vp, vp, i64, i64, i64, vp, vp, vp, vp, vp, vp,
+                                                     i64, vp, i64, vp, vp, vp, vp, vp, sz, vp]
+        L.mts_tbe_backward_apply_presorted.argtypes = [vp, i32, vp, i64, i32, vp, i32, i64, f32, f32, vp, vp, vp, vp,
+                                                       C.POINTER(vp), C.POINTER(vp), i32, vp, sz, vp]
         L.mts_cache_refetch_overflowed.argtypes = [vp, vp, vp, i64, vp, i64, vp]
         L.mts_cache_prefetch_misses.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.mts_cache_writeback_evicted.argtypes = [vp, vp, vp, vp, i64, vp, vp, vp]
@@ -251,6 +256,19 @@ def tbe_backward_apply(tables: Tables, B: int, offsets, N: int, pooling_mode: in
         _ptr(workspace), workspace_bytes, _stream(stream)))
 
 
+def tbe_backward_apply_presorted(tables: Tables, B: int, offsets, N: int, pooling_mode: int, grad_out,
+                                 grad_stride: int, lr: float, eps: float, sorted_rows, sorted_pos, bag_of_lookup,
+                                 slot_of_lookup, cache_data: Optional[Sequence], cache_dirty: Optional[Sequence],
+                                 workspace, workspace_bytes: int, stream=None, f16: bool = False) -> None:
+    """Gradient half of the backward on lookups already ordered by row (mts_cache_lookup_insert_tables)."""
+    n_caches = len(cache_data) if cache_data is not None else 0
+    _check(lib().mts_tbe_backward_apply_presorted(
+        tables.handle, B, _ptr(offsets), N, pooling_mode, _ptr(grad_out), DTYPE_FP16 if f16 else DTYPE_FP32,
+        grad_stride, lr, eps, _ptr(sorted_rows), _ptr(sorted_pos), _ptr(bag_of_lookup), _ptr(slot_of_lookup),
+        _ptr_array(cache_data, n_caches), _ptr_array(cache_dirty, n_caches), n_caches, _ptr(workspace),
+        workspace_bytes, _stream(stream)))
+
+
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -319,6 +337,21 @@ def cache_lookup_insert(cache: Cache, keys, N: int, step: int, slot_of_lookup, m
                                          _ptr(miss_slots), _ptr(evict_keys), _ptr(evict_slots), _ptr(evict_dirty),
                                          _ptr(overflow_keys), list_capacity, _ptr(counters), _ptr(workspace),
                                          workspace_bytes, _stream(stream)))
+
+
+def cache_lookup_insert_tables(cache: Cache, tables: Tables, t_begin: int, t_end: int, B: int, indices, offsets,
+                               lookup_begin: int, n: int, step: int, slot_of_lookup, miss_keys, miss_slots,
+                               evict_keys, evict_slots, evict_dirty, list_capacity: int, overflow_keys,
+                               overflow_capacity: int, counters, workspace, workspace_bytes: int, stream=None,
+                               sorted_rows_out=None, sorted_pos_out=None, bag_of_lookup_out=None) -> None:
+    """Tag lookup of one cache fed from the batch's sparse input; slot_of_lookup and the three optional
+    outputs are batch-wide arrays."""
+    _check(lib().mts_cache_lookup_insert_tables(
+        cache.handle, tables.handle, t_begin, t_end, B, _ptr(indices), _ptr(offsets), lookup_begin, n, step,
+        _ptr(slot_of_lookup), _ptr(miss_keys), _ptr(miss_slots), _ptr(evict_keys), _ptr(evict_slots),
+        _ptr(evict_dirty), list_capacity, _ptr(overflow_keys), overflow_capacity, _ptr(counters),
+        _ptr(sorted_rows_out), _ptr(sorted_pos_out), _ptr(bag_of_lookup_out), _ptr(workspace), workspace_bytes,
+        _stream(stream)))
 
 
 def cache_refetch_overflowed(cache: Cache, host_rows_mapped, overflow_keys, list_capacity: int, counters,

@@ -26,6 +26,7 @@ struct mts_cache {
   int32_t sm_count = 148;
   uint32_t* tags = nullptr;      // [S*32]  0xffffffff = free
   int32_t* ts = nullptr;         // [S*32]  -1 = free
+  int32_t* placed = nullptr;     // [S*32]  step at which the way's current row was inserted (-1 = free)
   uint32_t* freq = nullptr;      // [S*32]
   uint8_t* dirty = nullptr;      // [S*32]
   char* data = nullptr;          // [S*32, row_bytes]
@@ -38,15 +39,16 @@ constexpr uint32_t FREE_TAG = 0xffffffffu;
 constexpr int CACHE_THREADS = 256;
 constexpr int CACHE_STATUS_FETCH_TIMEOUT = 1;   // a bounded wait on a bulk copy ran out
 constexpr int CACHE_STATUS_KEY_RANGE = 2;       // a key outside [0, key_space) was clamped
+constexpr int CACHE_STATUS_LIST_CUT = 4;        // more placements than list_capacity: the surplus was not inserted
 
 __device__ __forceinline__ uint32_t set_of_key(uint32_t key, uint64_t S) {
   const uint64_t x = (uint64_t)key * 0x9E3779B97F4A7C15ull;
   return (uint32_t)__umul64hi(x, S);
 }
 
-__global__ void cache_init_state(uint32_t* tags, int32_t* ts, uint32_t* freq, uint8_t* dirty, int64_t n) {
+__global__ void cache_init_state(uint32_t* tags, int32_t* ts, int32_t* placed, uint32_t* freq, uint8_t* dirty, int64_t n) {
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
-    tags[i] = FREE_TAG; ts[i] = -1; freq[i] = 0; dirty[i] = 0;
+    tags[i] = FREE_TAG; ts[i] = -1; placed[i] = -1; freq[i] = 0; dirty[i] = 0;
   }
 }
 
@@ -70,9 +72,39 @@ __global__ void cache_prepare_keys(const int64_t* __restrict__ keys, int64_t n, 
   }
 }
 
+// The same preparation straight from a batch's sparse input, for the lookups of the tables
+// [t_begin, t_end) (8 lanes per bag): the sort key is the linear row id row_offset[t] + index, the
+// value the lookup's position in the batch; bag_of_lookup (nullable) receives every lookup's bag id.
+__global__ void cache_prepare_from_indices(const TableMeta* __restrict__ meta, int32_t t_begin, int64_t n_bags,
+                                           int32_t B, const int64_t* __restrict__ indices,
+                                           const int64_t* __restrict__ offsets, int64_t lookup_begin, int64_t n,
+                                           uint32_t* __restrict__ k32, uint32_t* __restrict__ pos,
+                                           uint32_t* __restrict__ bag_of_lookup, int64_t* __restrict__ counters,
+                                           uint32_t* __restrict__ overflow_cursor, int32_t* __restrict__ status) {
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (gid < MTS_NUM_COUNTERS) counters[gid] = gid == MTS_CNT_LOOKUPS ? n : 0;
+  if (gid == 0) *overflow_cursor = 0u;
+  const int64_t gb = gid / 8;
+  if (gb >= n_bags) return;
+  const int sub = (int)(gid % 8);
+  const int64_t bag = (int64_t)t_begin * B + gb;
+  const int32_t t = (int32_t)(bag / B);
+  const int64_t rows = meta[t].rows;
+  const int64_t roff = meta[t].row_offset;
+  const int64_t i1 = offsets[bag + 1];
+  for (int64_t i = offsets[bag] + sub; i < i1; i += 8) {
+    const int64_t o = i - lookup_begin;
+    if (o >= 0 && o < n) {
+      k32[o] = (uint32_t)(roff + clamp_index(indices[i], rows, status));
+      pos[o] = (uint32_t)i;
+      if (bag_of_lookup != nullptr) bag_of_lookup[i] = (uint32_t)bag;
+    }
+  }
+}
+
 // Distinct key u: its value, multiplicity and set.  Entries u >= U of the sort input are not
 // touched: the second sort runs on the device-side count U.
-__global__ void cache_describe_unique(const uint32_t* __restrict__ sorted_keys,
+__global__ void cache_describe_unique(const uint32_t* __restrict__ sorted_keys, uint32_t key_base,
                                       const uint32_t* __restrict__ seg_start,
                                       const uint32_t* __restrict__ n_unique, uint64_t S,
                                       uint32_t* __restrict__ ukey, uint32_t* __restrict__ mult,
@@ -80,7 +112,7 @@ __global__ void cache_describe_unique(const uint32_t* __restrict__ sorted_keys,
   const uint32_t U = *n_unique;
   for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < U; u += (int64_t)gridDim.x * blockDim.x) {
     const uint32_t s0 = seg_start[u];
-    const uint32_t k = sorted_keys[s0];
+    const uint32_t k = sorted_keys[s0] - key_base;
     ukey[u] = k;
     mult[u] = seg_start[u + 1] - s0;
     set_keys[u] = set_of_key(k, S);
@@ -94,10 +126,13 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
                     const uint32_t* __restrict__ member_uidx,     // distinct-key index of member j
                     const uint32_t* __restrict__ sseg_start, const uint32_t* __restrict__ n_sets,
                     const uint32_t* __restrict__ ukey, const uint32_t* __restrict__ mult,
-                    uint32_t* __restrict__ tags, int32_t* __restrict__ ts, uint32_t* __restrict__ freq,
+                    uint32_t* __restrict__ tags, int32_t* __restrict__ ts, int32_t* __restrict__ placed_at,
+                    uint32_t* __restrict__ freq,
                     uint8_t* __restrict__ dirty, int32_t step, int32_t lock_depth, int32_t policy,
                     int32_t* __restrict__ slot_of_uniq, uint8_t* __restrict__ member_flag,
                     uint32_t* __restrict__ member_old_key, uint8_t* __restrict__ member_old_dirty,
+                    int32_t* __restrict__ member_old_ts, uint32_t* __restrict__ member_old_freq,
+                    int32_t* __restrict__ member_old_placed,
                     int32_t* __restrict__ member_slot, unsigned long long* __restrict__ counters) {
   const int lane = threadIdx.x & 31;
   const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -111,6 +146,7 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
     uint32_t tag = tags[slot0 + lane];
     int32_t stamp = ts[slot0 + lane];
     uint32_t cnt = freq[slot0 + lane];
+    int32_t plc = placed_at[slot0 + lane];
     bool touched = false;
     // pass 1: probe every member against the state before the call, refresh the hits
     for (uint32_t jb = j0; jb < j1; jb += 32) {
@@ -168,6 +204,8 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
       int32_t my_slot = -1;
       uint32_t my_old = FREE_TAG;
       uint8_t my_old_dirty = 0;
+      int32_t my_old_ts = -1, my_old_placed = -1;
+      uint32_t my_old_freq = 0;
       for (int q = 0; q < m; ++q) {
         if (!((miss_mask >> q) & 1u)) continue;
         const uint32_t kq = __shfl_sync(0xffffffffu, k, q);
@@ -177,15 +215,23 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
           const int way = __ffs(sel) - 1;
           uint32_t old_tag = 0;
           uint8_t old_dirty = 0;
+          int32_t old_ts = -1, old_placed = -1;
+          uint32_t old_freq = 0;
           if (lane == way) {
-            old_tag = tag;
+            old_tag = tag; old_ts = stamp; old_freq = cnt; old_placed = plc;
             if (!dirty_loaded) { dirty_reg = dirty[slot0 + lane]; dirty_loaded = true; }
             old_dirty = tag != FREE_TAG ? dirty_reg : 0;
-            tag = kq; stamp = step; cnt = mq; dirty_reg = 0; touched = true;
+            tag = kq; stamp = step; cnt = mq; plc = step; dirty_reg = 0; touched = true;
           }
           old_tag = __shfl_sync(0xffffffffu, old_tag, way);
+          old_placed = __shfl_sync(0xffffffffu, old_placed, way);
           old_dirty = (uint8_t)__shfl_sync(0xffffffffu, (uint32_t)old_dirty, way);
-          if (lane == q) { my_flag = 1; my_slot = (int32_t)(slot0 + way); my_old = old_tag; my_old_dirty = old_dirty; }
+          old_ts = __shfl_sync(0xffffffffu, old_ts, way);
+          old_freq = __shfl_sync(0xffffffffu, old_freq, way);
+          if (lane == q) {
+            my_flag = 1; my_slot = (int32_t)(slot0 + way); my_old = old_tag; my_old_dirty = old_dirty;
+            my_old_ts = old_ts; my_old_freq = old_freq; my_old_placed = old_placed;
+          }
           if (old_tag != FREE_TAG && old_dirty) c_dirty += 1;
           ++placed;
         } else {
@@ -198,12 +244,16 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
         member_slot[j] = my_slot;
         member_old_key[j] = my_old;
         member_old_dirty[j] = my_old_dirty;
+        member_old_ts[j] = my_old_ts;
+        member_old_freq[j] = my_old_freq;
+        member_old_placed[j] = my_old_placed;
       }
       if (j < j1) slot_of_uniq[u] = (fl == 0) ? my_slot : member_slot[j];
     }
     if (touched) {
       tags[slot0 + lane] = tag;
       ts[slot0 + lane] = stamp;
+      placed_at[slot0 + lane] = plc;
       freq[slot0 + lane] = cnt;
       if (dirty_loaded) dirty[slot0 + lane] = dirty_reg;
     }
@@ -273,7 +323,8 @@ cache_count_lists(const uint8_t* __restrict__ member_flag, const uint32_t* __res
 
 __global__ void __launch_bounds__(CACHE_THREADS)
 cache_scan_lists(uint32_t* __restrict__ cnt_miss, uint32_t* __restrict__ cnt_evict, int G,
-                 const uint32_t* __restrict__ n_unique, int64_t n_lookups, int64_t* __restrict__ counters) {
+                 const uint32_t* __restrict__ n_unique, int64_t n_lookups, int64_t capacity,
+                 int64_t* __restrict__ counters, int32_t* __restrict__ status) {
   __shared__ uint32_t sh[9];
   constexpr int PER = LIST_BLOCKS / CACHE_THREADS;
   const int j0 = threadIdx.x * PER;
@@ -287,7 +338,16 @@ cache_scan_lists(uint32_t* __restrict__ cnt_miss, uint32_t* __restrict__ cnt_evi
     uint32_t ex = block_scan_256(s, sh, &total);
 #pragma unroll
     for (int k = 0; k < PER; ++k) { if (j0 + k < G) cnt[j0 + k] = ex; ex += v[k]; }
-    if (threadIdx.x == 0) counters[which == 0 ? MTS_CNT_INSERTED : MTS_CNT_EVICTED] = (int64_t)total;
+    // more placements than list entries: the surplus is undone by cache_write_lists, which also sets
+    // the number of evictions that remain
+    if (threadIdx.x == 0) {
+      if (which == 0) {
+        counters[MTS_CNT_INSERTED] = min((int64_t)total, capacity);
+        if ((int64_t)total > capacity) atomicOr(status, CACHE_STATUS_LIST_CUT);
+      } else {
+        counters[MTS_CNT_EVICTED] = capacity > 0 ? (int64_t)total : 0;
+      }
+    }
   }
   if (threadIdx.x == 0) {
     const int64_t U = *n_unique;
@@ -297,16 +357,25 @@ cache_scan_lists(uint32_t* __restrict__ cnt_miss, uint32_t* __restrict__ cnt_evi
   }
 }
 
+// Writes the lists.  A placement whose list position is beyond the capacity cannot be carried out by the
+// data movement, so it is undone here: the way gets its old tag, timestamp, count and dirty byte back,
+// the key is not inserted (slot -1) and joins the overflow list.  Inside a set the surplus placements are
+// the last ones, so the earlier ones stand as they are.
 __global__ void __launch_bounds__(CACHE_THREADS)
-cache_write_lists(const uint8_t* __restrict__ member_flag, const uint32_t* __restrict__ member_old_key,
-                  const uint8_t* __restrict__ member_old_dirty, const int32_t* __restrict__ member_slot,
+cache_write_lists(uint8_t* __restrict__ member_flag, const uint32_t* __restrict__ member_old_key,
+                  const uint8_t* __restrict__ member_old_dirty, const int32_t* __restrict__ member_old_ts,
+                  const uint32_t* __restrict__ member_old_freq, const int32_t* __restrict__ member_old_placed,
+                  const int32_t* __restrict__ member_slot,
                   const uint32_t* __restrict__ member_uidx, const uint32_t* __restrict__ ukey,
                   const uint32_t* __restrict__ n_unique, const uint32_t* __restrict__ base_miss,
                   const uint32_t* __restrict__ base_evict, int64_t capacity,
                   int64_t* __restrict__ miss_keys, int32_t* __restrict__ miss_slots,
                   int64_t* __restrict__ evict_keys, int32_t* __restrict__ evict_slots,
                   uint8_t* __restrict__ evict_dirty, int64_t* __restrict__ overflow_keys,
-                  uint32_t* __restrict__ overflow_cursor) {
+                  int64_t overflow_capacity, uint32_t* __restrict__ overflow_cursor,
+                  uint32_t* __restrict__ tags, int32_t* __restrict__ ts, int32_t* __restrict__ placed_at,
+                  uint32_t* __restrict__ freq, uint8_t* __restrict__ dirty, int32_t* __restrict__ slot_of_uniq,
+                  unsigned long long* __restrict__ counters) {
   __shared__ uint32_t sh[9];
   const int64_t n = *n_unique;
   const int64_t per = list_per_block(n, gridDim.x);
@@ -314,24 +383,42 @@ cache_write_lists(const uint8_t* __restrict__ member_flag, const uint32_t* __res
   uint32_t bm = base_miss[blockIdx.x], be = base_evict[blockIdx.x];
   for (int64_t t0 = begin; t0 < end; t0 += CACHE_THREADS) {
     const int64_t j = t0 + threadIdx.x;
-    if (overflow_keys != nullptr && j < end && member_flag[j] == 2) {
-      // the overflow list is a set: its order is not specified
-      const uint32_t at = atomicAdd(overflow_cursor, 1u);
-      if ((int64_t)at < capacity) overflow_keys[at] = (int64_t)ukey[member_uidx[j]];
-    }
+    bool overflowed = j < end && member_flag[j] == 2;
     const bool placed = j < end && member_flag[j] == 1;
     const bool ev = placed && member_old_key[j] != FREE_TAG;
     uint32_t ta, tb;
     const uint32_t pa = block_scan_256(placed ? 1u : 0u, sh, &ta);
     const uint32_t pb = block_scan_256(ev ? 1u : 0u, sh, &tb);
-    if (placed && (int64_t)(bm + pa) < capacity) {
-      miss_keys[bm + pa] = (int64_t)ukey[member_uidx[j]];
-      miss_slots[bm + pa] = member_slot[j];
+    if (placed) {
+      const int64_t at = (int64_t)bm + pa;
+      if (at < capacity) {
+        miss_keys[at] = (int64_t)ukey[member_uidx[j]];
+        miss_slots[at] = member_slot[j];
+        if (ev) {                                  // its position is at most `at`: inside the capacity too
+          evict_keys[be + pb] = (int64_t)member_old_key[j];
+          evict_slots[be + pb] = member_slot[j];
+          evict_dirty[be + pb] = member_old_dirty[j];
+        }
+        // the last placement that fits fixes the length of the evict list
+        if (at == capacity - 1) counters[MTS_CNT_EVICTED] = (unsigned long long)(be + pb + (ev ? 1u : 0u));
+      } else {
+        const int32_t slot = member_slot[j];
+        tags[slot] = member_old_key[j];
+        ts[slot] = member_old_ts[j];
+        placed_at[slot] = member_old_placed[j];
+        freq[slot] = member_old_freq[j];
+        dirty[slot] = member_old_dirty[j];
+        slot_of_uniq[member_uidx[j]] = -1;
+        member_flag[j] = 2;
+        overflowed = true;
+        atomicAdd(&counters[MTS_CNT_OVERFLOW], 1ull);
+        if (ev && member_old_dirty[j]) atomicAdd(&counters[MTS_CNT_EVICTED_DIRTY], ~0ull);     // minus one
+      }
     }
-    if (ev && (int64_t)(be + pb) < capacity) {
-      evict_keys[be + pb] = (int64_t)member_old_key[j];
-      evict_slots[be + pb] = member_slot[j];
-      evict_dirty[be + pb] = member_old_dirty[j];
+    if (overflow_keys != nullptr && overflowed) {
+      // the overflow list is a set: its order is not specified
+      const uint32_t at = atomicAdd(overflow_cursor, 1u);
+      if ((int64_t)at < overflow_capacity) overflow_keys[at] = (int64_t)ukey[member_uidx[j]];
     }
     bm += ta;
     be += tb;
@@ -506,7 +593,7 @@ cache_fetch_misses_bulk(char* __restrict__ data, int row_bytes, const char* __re
 __global__ void __launch_bounds__(CACHE_THREADS)
 cache_refetch_resident(char* __restrict__ data, int row_bytes, const char* __restrict__ host_rows,
                        const int64_t* __restrict__ keys, const int64_t* __restrict__ counters, int64_t capacity,
-                       const uint32_t* __restrict__ tags, const int32_t* __restrict__ ts, int64_t placed_step,
+                       const uint32_t* __restrict__ tags, const int32_t* __restrict__ placed_at, int64_t placed_step,
                        uint64_t S) {
   const int64_t n = list_len(counters, MTS_CNT_OVERFLOW, capacity);
   const int lane = threadIdx.x & 31;
@@ -515,10 +602,12 @@ cache_refetch_resident(char* __restrict__ data, int row_bytes, const char* __res
   for (int64_t k = warp0; k < n; k += nwarps) {
     const uint32_t key = (uint32_t)keys[k];
     const int64_t slot0 = (int64_t)set_of_key(key, S) * 32;
-    // only a way stamped by the batch named in placed_step: a later tag step may have placed the key
-    // already, in a slot whose victim has not been saved yet and whose own fetch is still to come
+    // only a row inserted by the batch named in placed_step.  A row inserted earlier has been updated in
+    // its slot since (the host copy is the stale one); a later tag step may have inserted the key meanwhile,
+    // in a slot whose victim has not been saved yet and whose own fetch is still to come.  The step of the
+    // insertion is kept apart from the timestamp, which later hits refresh.
     const uint32_t hit = __ballot_sync(0xffffffffu, tags[slot0 + lane] == key &&
-                                                        (placed_step < 0 || (int64_t)ts[slot0 + lane] == placed_step));
+                                                        (placed_step < 0 || (int64_t)placed_at[slot0 + lane] == placed_step));
     if (hit) {
       const char* src = host_rows + (int64_t)key * row_bytes;
       char* dst = data + (slot0 + __ffs(hit) - 1) * row_bytes;
@@ -564,11 +653,18 @@ __global__ void cache_export(const uint32_t* __restrict__ tags, const int32_t* _
 
 struct CacheLayout {
   size_t keys_a, keys_b, vals_a, vals_b, uniq_idx, seg_start, ukey, mult, set_a, set_b, sval_a, sval_b,
-      sseg_start, slot_of_uniq, member_flag, member_old_key, member_old_dirty, member_slot, hist, scan, cnt_miss,
+      sseg_start, slot_of_uniq, member_flag, member_old_key, member_old_dirty, member_old_ts, member_old_freq,
+      member_old_placed, member_slot, hist, scan, cnt_miss,
       cnt_evict, n_unique, n_sets, ovf_cursor, total;
 };
 
-static CacheLayout cache_layout(int64_t N) {
+static int bits_of(int64_t values) {
+  int bits = 1;
+  while (bits < 32 && (1ll << bits) < values) ++bits;
+  return bits;
+}
+
+static CacheLayout cache_layout(const mts_cache* c, int64_t N) {
   CacheLayout L;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
@@ -580,7 +676,8 @@ static CacheLayout cache_layout(int64_t N) {
   L.sseg_start = take((n + 1) * 4);
   L.slot_of_uniq = take(n * 4);
   L.member_flag = take(n); L.member_old_key = take(n * 4); L.member_old_dirty = take(n); L.member_slot = take(n * 4);
-  L.hist = take(sort_hist_words() * 4);
+  L.member_old_ts = take(n * 4); L.member_old_freq = take(n * 4); L.member_old_placed = take(n * 4);
+  L.hist = take(std::max(sort_hist_words((int64_t)n, bits_of(c->key_space)), sort_hist_words((int64_t)n, bits_of(c->S))) * 4);
   L.scan = take(scan_scratch_words() * 4);
   L.cnt_miss = take(LIST_BLOCKS * 4); L.cnt_evict = take(LIST_BLOCKS * 4);
   L.n_unique = take(256); L.n_sets = take(256); L.ovf_cursor = take(256);
@@ -617,6 +714,7 @@ extern "C" int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_s
   if (rc == MTS_OK && sms > 0) c->sm_count = sms;
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->tags, n * 4), "cudaMalloc(tags)");
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->ts, n * 4), "cudaMalloc(timestamps)");
+  if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->placed, n * 4), "cudaMalloc(insertion steps)");
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->freq, n * 4), "cudaMalloc(counts)");
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->dirty, n), "cudaMalloc(dirty)");
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->data, (size_t)n * c->row_bytes), "cudaMalloc(cache rows)");
@@ -625,7 +723,7 @@ extern "C" int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_s
   if (rc == MTS_OK) {
     {
       LaunchScope scope(K_OTHER, nullptr);
-      cache_init_state<<<c->sm_count * 4, 256>>>(c->tags, c->ts, c->freq, c->dirty, n);
+      cache_init_state<<<c->sm_count * 4, 256>>>(c->tags, c->ts, c->placed, c->freq, c->dirty, n);
     }
     rc = check_launch("cache_init_state");
   }
@@ -638,7 +736,7 @@ extern "C" int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_s
 
 extern "C" int mts_cache_destroy(mts_cache* c) {
   if (!c) return MTS_OK;
-  cudaFree(c->tags); cudaFree(c->ts); cudaFree(c->freq); cudaFree(c->dirty); cudaFree(c->data); cudaFree(c->d_status);
+  cudaFree(c->tags); cudaFree(c->ts); cudaFree(c->placed); cudaFree(c->freq); cudaFree(c->dirty); cudaFree(c->data); cudaFree(c->d_status);
   delete c;
   return MTS_OK;
 }
@@ -694,22 +792,36 @@ extern "C" int mts_linearize_keys(const mts_tables* h, int32_t t_begin, int32_t 
 
 extern "C" size_t mts_cache_workspace_bytes(const mts_cache* c, int64_t N) {
   if (!c || N < 0) return 0;
-  return cache_layout(N).total;
+  return cache_layout(c, N).total;
 }
 
-extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_t N, int64_t step,
-                                       int32_t* slot_of_lookup, int64_t* miss_keys, int32_t* miss_slots,
-                                       int64_t* evict_keys, int32_t* evict_slots, uint8_t* evict_dirty,
-                                       int64_t* overflow_keys, int64_t list_capacity, int64_t* counters,
-                                       void* workspace, size_t workspace_bytes, void* stream) {
-  if (!c || !counters || N < 0 || list_capacity < 0 || step < 0 || step >= (1ll << 31) - 1)
+namespace {
+
+// Where the keys of a lookup_insert call come from: an array of keys relative to the cache's table
+// group, or the sparse input of a batch (tables [t_begin, t_end) of `tables`).
+struct KeySource {
+  const int64_t* keys = nullptr;
+  const mts_tables* tables = nullptr;
+  int32_t t_begin = 0, t_end = 0, B = 0;
+  const int64_t* indices = nullptr;
+  const int64_t* offsets = nullptr;
+  int64_t lookup_begin = 0;
+  uint32_t* sorted_rows_out = nullptr;     // batch-wide arrays; this call fills [lookup_begin, lookup_begin + N)
+  uint32_t* sorted_pos_out = nullptr;
+  uint32_t* bag_of_lookup_out = nullptr;
+};
+
+int lookup_insert_impl(mts_cache* c, const KeySource& src, int64_t N, int64_t step, int32_t* slot_of_lookup,
+                       int64_t* miss_keys, int32_t* miss_slots, int64_t* evict_keys, int32_t* evict_slots,
+                       uint8_t* evict_dirty, int64_t* overflow_keys, int64_t list_capacity, int64_t overflow_capacity,
+                       int64_t* counters, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!c || !counters || N < 0 || list_capacity < 0 || overflow_capacity < 0 || step < 0 || step >= (1ll << 31) - 1)
     return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert: bad argument");
-  if (N > 0 && (!keys || !slot_of_lookup))
-    return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert: null keys / slot_of_lookup");
+  if (N > 0 && !slot_of_lookup) return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert: null slot_of_lookup");
   if (list_capacity > 0 && (!miss_keys || !miss_slots || !evict_keys || !evict_slots || !evict_dirty))
     return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert: null list buffer");
   if (N >= (1ll << 32) - 1) return set_error(MTS_ERR_UNSUPPORTED, "cache_lookup_insert: N must fit 32 bits");
-  const CacheLayout L = cache_layout(N);
+  const CacheLayout L = cache_layout(c, N);
   if (!workspace || ((uintptr_t)workspace & 255))
     return set_error(MTS_ERR_ALIGNMENT, "cache_lookup_insert: workspace must be non-null and 256-byte aligned");
   if (workspace_bytes < L.total)
@@ -718,37 +830,59 @@ extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_
   char* ws = static_cast<char*>(workspace);
   auto U32 = [&](size_t off) { return reinterpret_cast<uint32_t*>(ws + off); };
   const int grid = c->sm_count * 8;
-  {
-    LaunchScope scope(K_CACHE_PREPARE, s);
-    cache_prepare_keys<<<grid, 256, 0, s>>>(keys, N, c->key_space, U32(L.keys_a), U32(L.vals_a), counters,
-                                            U32(L.ovf_cursor), c->d_status);
+  const int key_bits = bits_of(c->key_space);
+  // The sort alternates between two buffer pairs.  When the caller wants the sorted lookups, its
+  // arrays are the pair the last pass writes into, so that exporting them costs nothing.
+  uint32_t *keys_a = U32(L.keys_a), *vals_a = U32(L.vals_a), *keys_b = U32(L.keys_b), *vals_b = U32(L.vals_b);
+  uint32_t key_base = 0u;
+  if (src.tables != nullptr) {
+    key_base = (uint32_t)src.tables->h_meta[src.t_begin].row_offset;
+    if (src.sorted_rows_out != nullptr) {
+      const bool result_in_a = N <= 1 || (sort_passes(key_bits) & 1) == 0;
+      (result_in_a ? keys_a : keys_b) = src.sorted_rows_out + src.lookup_begin;
+      (result_in_a ? vals_a : vals_b) = src.sorted_pos_out + src.lookup_begin;
+    }
   }
-  int rc = check_launch("cache_prepare_keys");
+  int rc;
+  if (src.tables == nullptr) {
+    if (N > 0 && !src.keys) return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert: null keys");
+    {
+      LaunchScope scope(K_CACHE_PREPARE, s);
+      cache_prepare_keys<<<grid, 256, 0, s>>>(src.keys, N, c->key_space, keys_a, vals_a, counters, U32(L.ovf_cursor),
+                                              c->d_status);
+    }
+    rc = check_launch("cache_prepare_keys");
+  } else {
+    const int64_t n_bags = (int64_t)(src.t_end - src.t_begin) * src.B;
+    {
+      LaunchScope scope(K_CACHE_PREPARE, s);
+      cache_prepare_from_indices<<<(unsigned)ceil_div(std::max<int64_t>(n_bags * 8, MTS_NUM_COUNTERS), 256), 256, 0, s>>>(
+          src.tables->d_meta, src.t_begin, n_bags, src.B, src.indices, src.offsets, src.lookup_begin, N, keys_a, vals_a,
+          src.bag_of_lookup_out, counters, U32(L.ovf_cursor), src.tables->d_status);
+    }
+    rc = check_launch("cache_prepare_from_indices");
+  }
   if (rc != MTS_OK) return rc;
   uint32_t* n_unique = U32(L.n_unique);
   uint32_t* n_sets = U32(L.n_sets);
   if (N == 0) {
     return MTS_OK;   // counters already written: all zero
   }
-  int key_bits = 1;
-  while (key_bits < 32 && (1ll << key_bits) < c->key_space) ++key_bits;
   uint32_t *sk = nullptr, *sp = nullptr;
-  rc = radix_sort_pairs(U32(L.keys_a), U32(L.vals_a), U32(L.keys_b), U32(L.vals_b), N, nullptr, key_bits,
-                        U32(L.hist), &sk, &sp, s);
+  rc = radix_sort_pairs(keys_a, vals_a, keys_b, vals_b, N, nullptr, key_bits, key_base, U32(L.hist), &sk, &sp, s);
   if (rc != MTS_OK) return rc;
   rc = unique_segments(sk, N, nullptr, U32(L.seg_start), U32(L.uniq_idx), n_unique, U32(L.scan), s);
   if (rc != MTS_OK) return rc;
   {
     LaunchScope scope(K_CACHE_DESCRIBE, s);
-    cache_describe_unique<<<grid, 256, 0, s>>>(sk, U32(L.seg_start), n_unique, (uint64_t)c->S, U32(L.ukey),
+    cache_describe_unique<<<grid, 256, 0, s>>>(sk, key_base, U32(L.seg_start), n_unique, (uint64_t)c->S, U32(L.ukey),
                                                U32(L.mult), U32(L.set_a), U32(L.sval_a));
   }
   rc = check_launch("cache_describe_unique");
   if (rc != MTS_OK) return rc;
-  int set_bits = 0;
-  while ((1ll << set_bits) < c->S) ++set_bits;
+  const int set_bits = c->S > 1 ? bits_of(c->S) : 0;
   uint32_t *ss = nullptr, *su = nullptr;
-  rc = radix_sort_pairs(U32(L.set_a), U32(L.sval_a), U32(L.set_b), U32(L.sval_b), N, n_unique, set_bits,
+  rc = radix_sort_pairs(U32(L.set_a), U32(L.sval_a), U32(L.set_b), U32(L.sval_b), N, n_unique, set_bits, 0u,
                         U32(L.hist), &ss, &su, s);
   if (rc != MTS_OK) return rc;
   rc = unique_segments(ss, N, n_unique, U32(L.sseg_start), nullptr, n_sets, U32(L.scan), s);
@@ -760,8 +894,10 @@ extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_
   {
     LaunchScope scope(K_CACHE_PROBE_REPLACE, s);
     cache_probe_replace<<<grid, CACHE_THREADS, 0, s>>>(
-        ss, su, U32(L.sseg_start), n_sets, U32(L.ukey), U32(L.mult), c->tags, c->ts, c->freq, c->dirty, (int32_t)step,
-        c->lock_depth, c->policy, slot_of_uniq, member_flag, U32(L.member_old_key), member_old_dirty, member_slot,
+        ss, su, U32(L.sseg_start), n_sets, U32(L.ukey), U32(L.mult), c->tags, c->ts, c->placed, c->freq, c->dirty, (int32_t)step,
+        c->lock_depth, c->policy, slot_of_uniq, member_flag, U32(L.member_old_key), member_old_dirty,
+        reinterpret_cast<int32_t*>(ws + L.member_old_ts), U32(L.member_old_freq),
+        reinterpret_cast<int32_t*>(ws + L.member_old_placed), member_slot,
         reinterpret_cast<unsigned long long*>(counters));
   }
   rc = check_launch("cache_probe_replace");
@@ -774,20 +910,66 @@ extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_
   }
   {
     LaunchScope scope(K_CACHE_LISTS, s);
-    cache_scan_lists<<<1, CACHE_THREADS, 0, s>>>(U32(L.cnt_miss), U32(L.cnt_evict), G, n_unique, N, counters);
+    cache_scan_lists<<<1, CACHE_THREADS, 0, s>>>(U32(L.cnt_miss), U32(L.cnt_evict), G, n_unique, N, list_capacity,
+                                                 counters, c->d_status);
   }
   {
     LaunchScope scope(K_CACHE_LISTS, s);
-    cache_write_lists<<<G, CACHE_THREADS, 0, s>>>(member_flag, U32(L.member_old_key), member_old_dirty, member_slot, su,
-                                                  U32(L.ukey), n_unique, U32(L.cnt_miss), U32(L.cnt_evict),
-                                                  list_capacity, miss_keys, miss_slots, evict_keys, evict_slots,
-                                                  evict_dirty, overflow_keys, U32(L.ovf_cursor));
+    cache_write_lists<<<G, CACHE_THREADS, 0, s>>>(
+        member_flag, U32(L.member_old_key), member_old_dirty, reinterpret_cast<int32_t*>(ws + L.member_old_ts),
+        U32(L.member_old_freq), reinterpret_cast<int32_t*>(ws + L.member_old_placed), member_slot, su, U32(L.ukey), n_unique, U32(L.cnt_miss), U32(L.cnt_evict), list_capacity,
+        miss_keys, miss_slots, evict_keys, evict_slots, evict_dirty, overflow_keys, overflow_capacity, U32(L.ovf_cursor),
+        c->tags, c->ts, c->placed, c->freq, c->dirty, slot_of_uniq, reinterpret_cast<unsigned long long*>(counters));
   }
   {
+    // positions are relative to the key array, or batch positions when the keys came from a batch's
+    // sparse input (slot_of_lookup is then the batch-wide array)
     LaunchScope scope(K_CACHE_SCATTER_SLOTS, s);
     cache_scatter_slots<<<grid, 256, 0, s>>>(sp, U32(L.uniq_idx), slot_of_uniq, N, slot_of_lookup);
   }
   return check_launch("cache lists / scatter");
+}
+
+}  // namespace
+
+extern "C" int mts_cache_lookup_insert(mts_cache* c, const int64_t* keys, int64_t N, int64_t step,
+                                       int32_t* slot_of_lookup, int64_t* miss_keys, int32_t* miss_slots,
+                                       int64_t* evict_keys, int32_t* evict_slots, uint8_t* evict_dirty,
+                                       int64_t* overflow_keys, int64_t list_capacity, int64_t* counters,
+                                       void* workspace, size_t workspace_bytes, void* stream) {
+  KeySource src;
+  src.keys = keys;
+  return lookup_insert_impl(c, src, N, step, slot_of_lookup, miss_keys, miss_slots, evict_keys, evict_slots, evict_dirty,
+                            overflow_keys, list_capacity, list_capacity, counters, workspace, workspace_bytes, stream);
+}
+
+extern "C" int mts_cache_lookup_insert_tables(mts_cache* c, const mts_tables* h, int32_t t_begin, int32_t t_end,
+                                              int32_t B, const int64_t* indices, const int64_t* offsets,
+                                              int64_t lookup_begin, int64_t n, int64_t step, int32_t* slot_of_lookup,
+                                              int64_t* miss_keys, int32_t* miss_slots, int64_t* evict_keys,
+                                              int32_t* evict_slots, uint8_t* evict_dirty, int64_t list_capacity,
+                                              int64_t* overflow_keys, int64_t overflow_capacity, int64_t* counters,
+                                              uint32_t* sorted_rows_out, uint32_t* sorted_pos_out,
+                                              uint32_t* bag_of_lookup_out, void* workspace, size_t workspace_bytes,
+                                              void* stream) {
+  if (!c || !h || !offsets || B < 1 || t_begin < 0 || t_end > h->T || t_begin >= t_end || n < 0 || lookup_begin < 0 ||
+      (n > 0 && !indices))
+    return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert_tables: bad argument");
+  if (h->h_meta[t_end - 1].row_offset + h->h_meta[t_end - 1].rows - h->h_meta[t_begin].row_offset != c->key_space)
+    return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert_tables: tables [%d, %d) hold %lld rows, the cache was created for %lld",
+                     t_begin, t_end,
+                     (long long)(h->h_meta[t_end - 1].row_offset + h->h_meta[t_end - 1].rows - h->h_meta[t_begin].row_offset),
+                     (long long)c->key_space);
+  if ((sorted_rows_out == nullptr) != (sorted_pos_out == nullptr) || (bag_of_lookup_out != nullptr && !sorted_rows_out))
+    return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert_tables: pass sorted_rows_out, sorted_pos_out (and bag_of_lookup_out) together");
+  if (lookup_begin + n >= (1ll << 32) - 1 || (int64_t)h->T * B >= (1ll << 32))
+    return set_error(MTS_ERR_UNSUPPORTED, "cache_lookup_insert_tables: lookup positions and bag ids must fit 32 bits");
+  KeySource src;
+  src.tables = h; src.t_begin = t_begin; src.t_end = t_end; src.B = B;
+  src.indices = indices; src.offsets = offsets; src.lookup_begin = lookup_begin;
+  src.sorted_rows_out = sorted_rows_out; src.sorted_pos_out = sorted_pos_out; src.bag_of_lookup_out = bag_of_lookup_out;
+  return lookup_insert_impl(c, src, n, step, slot_of_lookup, miss_keys, miss_slots, evict_keys, evict_slots, evict_dirty,
+                            overflow_keys, list_capacity, overflow_capacity, counters, workspace, workspace_bytes, stream);
 }
 
 extern "C" int mts_cache_prefetch_misses(mts_cache* c, const void* host_rows_mapped, const int64_t* miss_keys,
@@ -902,7 +1084,7 @@ extern "C" int mts_cache_refetch_overflowed(mts_cache* c, const void* host_rows_
     LaunchScope scope(K_CACHE_FETCH_MISSES, static_cast<cudaStream_t>(stream));
     cache_refetch_resident<<<c->sm_count, CACHE_THREADS, 0, static_cast<cudaStream_t>(stream)>>>(
         c->data, c->row_bytes, static_cast<const char*>(host_rows_mapped), overflow_keys, counters, list_capacity,
-        c->tags, c->ts, placed_step, (uint64_t)c->S);
+        c->tags, c->placed, placed_step, (uint64_t)c->S);
   }
   return check_launch("cache_refetch_resident");
 }

@@ -119,28 +119,34 @@ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // ----------------------------------------------------------------------------- sorting (radix_sort.cu)
-// Stable LSD radix sort of (key, value) pairs on the low `key_bits` bits of the keys.
+// Stable LSD radix sort of (key, value) pairs on the low `key_bits` bits of key - key_base.
 // keys_a/vals_a hold the input; *_b are same-sized scratch.  The sorted result ends in
 // (*keys_out, *vals_out), which point at either the a or the b buffers.
-// hist: scratch of sort_hist_words() uint32.
-size_t sort_hist_words();
+// hist: scratch of sort_hist_words(n_max, key_bits) uint32.
+size_t sort_hist_words(int64_t n_max, int key_bits);
+// Pass plan of the sort: the fewest passes of at most SORT_MAX_DIGIT_BITS bits, the key bits split
+// evenly over them.
+constexpr int SORT_MAX_DIGIT_BITS = 11;
+inline int sort_passes(int key_bits) { return key_bits <= 8 ? 1 : (key_bits + SORT_MAX_DIGIT_BITS - 1) / SORT_MAX_DIGIT_BITS; }
+inline int sort_digit_bits(int key_bits) { const int p = sort_passes(key_bits); return (key_bits + p - 1) / p; }
 // Segments of a segmented sort: segment t = positions [offsets[t*stride], offsets[(t+1)*stride]),
-// digits taken from key - meta[t].row_offset.
+// digits taken from key - meta[t].row_offset.  An unsegmented sort takes its digits from key - base.
 struct SortSegments {
   const int64_t* offsets;    // device
   int32_t stride;
   const TableMeta* meta;     // device
+  uint32_t base;
 };
-size_t sort_hist_words_segmented(int64_t n, int T);
+size_t sort_hist_words_segmented(int64_t n, int T, int key_bits);
 // Sorts every segment on its own by the low key_bits of (key - base of its segment); same buffers and
-// result convention as radix_sort_pairs, hist: sort_hist_words_segmented(n, T) uint32.
+// result convention as radix_sort_pairs, hist: sort_hist_words_segmented(n, T, key_bits) uint32.
 int radix_sort_pairs_segmented(uint32_t* keys_a, uint32_t* vals_a, uint32_t* keys_b, uint32_t* vals_b, int64_t n,
                                int T, const SortSegments& seg, int key_bits, uint32_t* hist, uint32_t** keys_out,
                                uint32_t** vals_out, cudaStream_t stream);
 // n_max is the host-known element count or an upper bound of it; when n_dev is not null the
 // kernels use min(*n_dev, n_max) (a device-resident count) instead.
 int radix_sort_pairs(uint32_t* keys_a, uint32_t* vals_a, uint32_t* keys_b, uint32_t* vals_b,
-                     int64_t n_max, const uint32_t* n_dev, int key_bits, uint32_t* hist,
+                     int64_t n_max, const uint32_t* n_dev, int key_bits, uint32_t key_base, uint32_t* hist,
                      uint32_t** keys_out, uint32_t** vals_out, cudaStream_t stream);
 
 // Distinct keys of an ascending key array.  Writes seg_start[u] = first position of the u-th

@@ -3,6 +3,8 @@
 // Section 5.9; cache: the grouping of requests in Section 5.5.1).  Stability is what makes
 // the backward deterministic: equal keys keep their input order.
 //
+// Digits are 8 to 11 bits wide: the key bits are split evenly over the fewest passes of at most 11
+// bits (20 bits: two passes of 10; 24: three of 8; 27: three of 9).
 // One pass = three kernels over G blocks, block b owning a contiguous range of tiles:
 //   digit_histogram  : hist[d][b] = occurrences of digit d in block b's range
 //   scan_histogram   : per digit, exclusive prefix over blocks (+ digit totals)
@@ -18,12 +20,8 @@ namespace mts {
 
 constexpr int SORT_THREADS = 256;
 constexpr int SORT_WARPS = SORT_THREADS / 32;
-#ifndef MTS_SORT_ITEMS
-#define MTS_SORT_ITEMS 16
-#endif
-constexpr int SORT_ITEMS = MTS_SORT_ITEMS;
+constexpr int SORT_ITEMS = 16;
 constexpr int SORT_TILE = SORT_THREADS * SORT_ITEMS;   // 4096 pairs
-constexpr int SORT_BINS = 256;
 constexpr int SORT_MAX_BLOCKS = 1024;
 
 // Element count of a launch: the host bound, or the smaller device-resident count when the
@@ -39,39 +37,46 @@ __device__ __forceinline__ int64_t tiles_per_block_of(int64_t n, int G) {
   return (ntiles + G - 1) / G;
 }
 
-size_t sort_hist_words() { return (size_t)SORT_BINS * SORT_MAX_BLOCKS + SORT_BINS; }
+static int sort_bins(int key_bits) { return 1 << std::max(8, sort_digit_bits(key_bits)); }
+size_t sort_hist_words(int64_t n, int key_bits) {
+  const int64_t G = std::min<int64_t>(std::max<int64_t>(ceil_div(n, SORT_TILE), 1), SORT_MAX_BLOCKS);
+  return (size_t)sort_bins(key_bits) * (size_t)(G + 1);
+}
 
 // Segmented sort: the input is a sequence of T segments (the lookups of a batch arrive grouped by
 // table) and each segment is sorted on its own, on the digits of key - base[t].  Keys of different
 // tables never have to be compared, so only the bits of the largest table's row index are sorted
-// (20 instead of 25 bits for 26 tables of a million rows: 3 passes instead of 4).
-#ifndef MTS_SORT_SEG_TILES
-#define MTS_SORT_SEG_TILES 4
-#endif
+// (20 instead of 25 bits for 26 tables of a million rows), and a table whose row index has no bit
+// left in a pass is only copied in that pass.
+constexpr int SORT_SEG_TILES = 4;
 int sort_segment_blocks(int64_t n, int T) {
   const int64_t avg_tiles = (n / (T > 0 ? T : 1) + SORT_TILE - 1) / SORT_TILE;
   int64_t g = 1;
-  while (g * MTS_SORT_SEG_TILES < 2 * avg_tiles) g <<= 1;   // about MTS_SORT_SEG_TILES / 2 .. MTS_SORT_SEG_TILES tiles per block for an average table
+  while (g * SORT_SEG_TILES < 2 * avg_tiles) g <<= 1;   // about SORT_SEG_TILES / 2 .. SORT_SEG_TILES tiles per block for an average table
   const int64_t cap = std::max<int64_t>(64, SORT_MAX_BLOCKS / (T > 0 ? T : 1));
   return (int)std::min<int64_t>(std::min<int64_t>(g, cap), SORT_MAX_BLOCKS);
 }
-size_t sort_hist_words_segmented(int64_t n, int T) {
-  return (size_t)T * SORT_BINS * sort_segment_blocks(n, T) + (size_t)T * SORT_BINS;
+size_t sort_hist_words_segmented(int64_t n, int T, int key_bits) {
+  return (size_t)T * sort_bins(key_bits) * (size_t)(sort_segment_blocks(n, T) + 1);
 }
 
-// Bounds and key base of the segment a block works on (the whole input when SEG is false).
+// Bounds and key base of the segment a block works on (the whole input when SEG is false), and
+// whether every digit of the segment is zero from bit `shift` on (then the pass only copies it).
 template <bool SEG>
 __device__ __forceinline__ void segment_of_block(const SortSegments& seg, int64_t n_max, const uint32_t* n_dev,
-                                                 int64_t* seg_begin, int64_t* n, uint32_t* base) {
+                                                 int shift, int64_t* seg_begin, int64_t* n, uint32_t* base,
+                                                 bool* exhausted) {
   if (SEG) {
     const int t = blockIdx.y;
     *seg_begin = seg.offsets[(int64_t)t * seg.stride];
     *n = seg.offsets[(int64_t)(t + 1) * seg.stride] - *seg_begin;
     *base = (uint32_t)seg.meta[t].row_offset;
+    *exhausted = ((uint64_t)(seg.meta[t].rows - 1) >> shift) == 0;
   } else {
     *seg_begin = 0;
     *n = effective_n(n_max, n_dev);
-    *base = 0u;
+    *base = seg.base;
+    *exhausted = false;
   }
 }
 size_t scan_scratch_words() { return SORT_MAX_BLOCKS + 8; }
@@ -106,30 +111,40 @@ __device__ __forceinline__ uint32_t block_exclusive_scan_256(uint32_t v, uint32_
   return res;
 }
 
-template <bool SEG>
+// hist[(segment * BINS + digit) * G + block]
+template <int BITS, bool SEG>
 __global__ void __launch_bounds__(SORT_THREADS)
 digit_histogram(const uint32_t* __restrict__ keys, int64_t n_max, const uint32_t* __restrict__ n_dev,
                 int shift, uint32_t mask, uint32_t* __restrict__ hist, int G, SortSegments seg) {
-  __shared__ uint32_t h[SORT_BINS];
-  h[threadIdx.x] = 0;
-  __syncthreads();
+  constexpr int BINS = 1 << BITS;
+  __shared__ uint32_t h[BINS];
   int64_t seg_begin, n;
   uint32_t base;
-  segment_of_block<SEG>(seg, n_max, n_dev, &seg_begin, &n, &base);
+  bool exhausted;
+  segment_of_block<SEG>(seg, n_max, n_dev, shift, &seg_begin, &n, &base, &exhausted);
   const int64_t tiles_per_block = tiles_per_block_of(n, G);
   const int64_t begin = (int64_t)blockIdx.x * tiles_per_block * SORT_TILE;
   const int64_t end = min(n, begin + tiles_per_block * SORT_TILE);
+  if (exhausted) {
+    // every digit is zero: the count of digit 0 is the size of the block's range
+    for (int d = threadIdx.x; d < BINS; d += SORT_THREADS)
+      hist[((size_t)blockIdx.y * BINS + d) * G + blockIdx.x] = d == 0 ? (uint32_t)max((int64_t)0, end - begin) : 0u;
+    return;
+  }
+  for (int d = threadIdx.x; d < BINS; d += SORT_THREADS) h[d] = 0;
+  __syncthreads();
   for (int64_t i = begin + threadIdx.x; i < end; i += SORT_THREADS)
     atomicAdd(&h[((keys[seg_begin + i] - base) >> shift) & mask], 1u);
   __syncthreads();
-  hist[((size_t)blockIdx.y * SORT_BINS + threadIdx.x) * G + blockIdx.x] = h[threadIdx.x];
+  for (int d = threadIdx.x; d < BINS; d += SORT_THREADS)
+    hist[((size_t)blockIdx.y * BINS + d) * G + blockIdx.x] = h[d];
 }
 
 // Block (d, segment): exclusive prefix over the G per-block counts of digit d, in place; totals = sum.
 __global__ void __launch_bounds__(SORT_THREADS)
 scan_histogram(uint32_t* __restrict__ hist, uint32_t* __restrict__ totals, int G) {
   __shared__ uint32_t sh[SORT_WARPS + 1];
-  uint32_t* row = hist + ((size_t)blockIdx.y * SORT_BINS + blockIdx.x) * G;
+  uint32_t* row = hist + ((size_t)blockIdx.y * gridDim.x + blockIdx.x) * G;
   const int per = (G + SORT_THREADS - 1) / SORT_THREADS;      // <= 4
   const int j0 = threadIdx.x * per;
   uint32_t v[SORT_MAX_BLOCKS / SORT_THREADS];
@@ -146,14 +161,14 @@ scan_histogram(uint32_t* __restrict__ hist, uint32_t* __restrict__ totals, int G
     if (k < per && j0 + k < G) row[j0 + k] = ex;
     ex += v[k];
   }
-  if (threadIdx.x == 0) totals[blockIdx.y * SORT_BINS + blockIdx.x] = total;
+  if (threadIdx.x == 0) totals[blockIdx.y * gridDim.x + blockIdx.x] = total;
 }
 
 // The same scan for short rows (segmented sort: few blocks per segment): one warp per (digit, segment).
 __global__ void __launch_bounds__(SORT_THREADS)
 scan_histogram_rows(uint32_t* __restrict__ hist, uint32_t* __restrict__ totals, int G, int n_rows) {
   const int lane = threadIdx.x & 31;
-  const int r = blockIdx.x * SORT_WARPS + (threadIdx.x >> 5);     // r = segment * SORT_BINS + digit
+  const int r = blockIdx.x * SORT_WARPS + (threadIdx.x >> 5);     // r = segment * BINS + digit
   if (r >= n_rows) return;
   uint32_t* row = hist + (size_t)r * G;
   uint32_t carry = 0;
@@ -172,36 +187,62 @@ scan_histogram_rows(uint32_t* __restrict__ hist, uint32_t* __restrict__ totals, 
   if (lane == 0) totals[r] = carry;
 }
 
-#ifndef MTS_SORT_MINBLK
-#define MTS_SORT_MINBLK 3
-#endif
-template <bool SEG>
-__global__ void __launch_bounds__(SORT_THREADS, MTS_SORT_MINBLK)
+// Shared memory of scatter_by_digit<BITS>: the tile (keys, values), per-warp digit counts (16 bits: a
+// warp holds 512 elements), the digit offsets inside the tile and in the output.
+template <int BITS>
+constexpr size_t scatter_smem_bytes() {
+  return (size_t)SORT_TILE * 8 + (size_t)SORT_WARPS * (1 << BITS) * 2 + (size_t)(1 << BITS) * 8 + 64;
+}
+
+template <int BITS, bool SEG>
+__global__ void __launch_bounds__(SORT_THREADS, 3)
 scatter_by_digit(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
                  uint32_t* __restrict__ keys_out, uint32_t* __restrict__ vals_out, int64_t n_max,
                  const uint32_t* __restrict__ n_dev, int shift, uint32_t mask,
                  const uint32_t* __restrict__ hist, const uint32_t* __restrict__ totals, int G, SortSegments seg) {
-  __shared__ uint32_t s_key[SORT_TILE];
-  __shared__ uint32_t s_val[SORT_TILE];
-  __shared__ uint32_t warp_cnt[SORT_WARPS][SORT_BINS];
-  __shared__ uint32_t s_off[SORT_BINS];     // first shared-memory position of a digit in the tile
-  __shared__ uint32_t s_goff[SORT_BINS];    // global position of this block's next element of a digit
-  __shared__ uint32_t sh[SORT_WARPS + 1];
+  constexpr int BINS = 1 << BITS;
+  constexpr int DPT = BINS / SORT_THREADS;      // digits per thread: thread tid owns digits tid*DPT .. tid*DPT + DPT-1
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint32_t* s_key = reinterpret_cast<uint32_t*>(smem_raw);
+  uint32_t* s_val = s_key + SORT_TILE;
+  uint32_t* s_off = s_val + SORT_TILE;          // first shared-memory position of a digit in the tile
+  uint32_t* s_goff = s_off + BINS;              // global position of this block's next element of a digit
+  uint32_t* sh = s_goff + BINS;                 // 9 words (+ padding to 16)
+  uint16_t* warp_cnt = reinterpret_cast<uint16_t*>(sh + 16);    // [SORT_WARPS][BINS]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t lt_mask = (1u << lane) - 1u;
   int64_t seg_begin, n;
   uint32_t base;
-  segment_of_block<SEG>(seg, n_max, n_dev, &seg_begin, &n, &base);
+  bool exhausted;
+  segment_of_block<SEG>(seg, n_max, n_dev, shift, &seg_begin, &n, &base, &exhausted);
   const int64_t tiles_per_block = tiles_per_block_of(n, G);
   keys_in += seg_begin; vals_in += seg_begin; keys_out += seg_begin; vals_out += seg_begin;
-
-  // where this block's elements of digit `tid` start in the (segment's) output
-  uint32_t dummy;
-  uint32_t digit_base = block_exclusive_scan_256(totals[blockIdx.y * SORT_BINS + tid], sh, &dummy);
-  uint32_t goff = digit_base + hist[((size_t)blockIdx.y * SORT_BINS + tid) * G + blockIdx.x];
-
   const int64_t begin = (int64_t)blockIdx.x * tiles_per_block * SORT_TILE;
   const int64_t end = min(n, begin + tiles_per_block * SORT_TILE);
+  if (exhausted) {
+    // no bit of this segment's keys is left: the pass keeps the order, copy the block's range
+    for (int64_t i = begin + tid; i < end; i += SORT_THREADS) {
+      keys_out[i] = keys_in[i];
+      vals_out[i] = vals_in[i];
+    }
+    return;
+  }
+
+  // where this block's elements of the thread's digits start in the (segment's) output
+  uint32_t goff[DPT];
+  {
+    uint32_t tot[DPT], sum = 0;
+#pragma unroll
+    for (int k = 0; k < DPT; ++k) { tot[k] = totals[blockIdx.y * BINS + tid * DPT + k]; sum += tot[k]; }
+    uint32_t dummy;
+    uint32_t digit_base = block_exclusive_scan_256(sum, sh, &dummy);
+#pragma unroll
+    for (int k = 0; k < DPT; ++k) {
+      goff[k] = digit_base + hist[((size_t)blockIdx.y * BINS + tid * DPT + k) * G + blockIdx.x];
+      digit_base += tot[k];
+    }
+  }
+
   for (int64_t tile = begin; tile < end; tile += SORT_TILE) {
     const int tile_n = (int)min((int64_t)SORT_TILE, end - tile);
     uint32_t key[SORT_ITEMS], val[SORT_ITEMS];
@@ -218,9 +259,13 @@ scatter_by_digit(const uint32_t* __restrict__ keys_in, const uint32_t* __restric
       const int li = warp * (32 * SORT_ITEMS) + j * 32 + lane;
       return li < tile_n ? ((key[j] - base) >> shift) & mask : mask;
     };
+    {
+      uint32_t* wc32 = reinterpret_cast<uint32_t*>(warp_cnt + warp * BINS);
 #pragma unroll
-    for (int k = 0; k < SORT_BINS / 32; ++k) warp_cnt[warp][lane + 32 * k] = 0;
-    s_goff[tid] = goff;
+      for (int k = 0; k < BINS / 64; ++k) wc32[lane + 32 * k] = 0u;
+    }
+#pragma unroll
+    for (int k = 0; k < DPT; ++k) s_goff[tid * DPT + k] = goff[k];
     __syncwarp();
 #pragma unroll
     for (int j = 0; j < SORT_ITEMS; ++j) {
@@ -229,30 +274,38 @@ scatter_by_digit(const uint32_t* __restrict__ keys_in, const uint32_t* __restric
       const int leader = __ffs(peers) - 1;
       uint32_t basec = 0;
       if (lane == leader) {
-        basec = warp_cnt[warp][d];
-        warp_cnt[warp][d] = basec + __popc(peers);
+        basec = warp_cnt[warp * BINS + d];
+        warp_cnt[warp * BINS + d] = (uint16_t)(basec + __popc(peers));
       }
       basec = __shfl_sync(0xffffffffu, basec, leader);
       rank[j] = (uint16_t)(basec + __popc(peers & lt_mask));
       __syncwarp();
     }
     __syncthreads();
-    // digit `tid`: prefix over warps, then over digits
-    uint32_t run = 0;
+    // the thread's digits: prefix over warps, then over digits
+    uint32_t run[DPT], sum = 0;
 #pragma unroll
-    for (int w = 0; w < SORT_WARPS; ++w) {
-      uint32_t c = warp_cnt[w][tid];
-      warp_cnt[w][tid] = run;
-      run += c;
+    for (int k = 0; k < DPT; ++k) {
+      const int d = tid * DPT + k;
+      uint32_t r = 0;
+#pragma unroll
+      for (int w = 0; w < SORT_WARPS; ++w) {
+        const uint32_t c = warp_cnt[w * BINS + d];
+        warp_cnt[w * BINS + d] = (uint16_t)r;
+        r += c;
+      }
+      run[k] = r;
+      sum += r;
     }
     uint32_t tot;
-    uint32_t off = block_exclusive_scan_256(run, sh, &tot);
-    s_off[tid] = off;
+    uint32_t off = block_exclusive_scan_256(sum, sh, &tot);
+#pragma unroll
+    for (int k = 0; k < DPT; ++k) { s_off[tid * DPT + k] = off; off += run[k]; }
     __syncthreads();
 #pragma unroll
     for (int j = 0; j < SORT_ITEMS; ++j) {
       const uint32_t d = digit_of(j);
-      const uint32_t p = s_off[d] + warp_cnt[warp][d] + rank[j];
+      const uint32_t p = s_off[d] + warp_cnt[warp * BINS + d] + rank[j];
       s_key[p] = key[j];
       s_val[p] = val[j];
     }
@@ -265,49 +318,96 @@ scatter_by_digit(const uint32_t* __restrict__ keys_in, const uint32_t* __restric
       keys_out[g] = k;
       vals_out[g] = s_val[i];
     }
-    uint32_t mine = run;
-    if ((uint32_t)tid == mask) mine -= (uint32_t)(SORT_TILE - tile_n);
-    goff += mine;
+#pragma unroll
+    for (int k = 0; k < DPT; ++k) {
+      uint32_t mine = run[k];
+      if ((uint32_t)(tid * DPT + k) == mask) mine -= (uint32_t)(SORT_TILE - tile_n);
+      goff[k] += mine;
+    }
     __syncthreads();
   }
 }
 
-int radix_sort_pairs(uint32_t* keys_a, uint32_t* vals_a, uint32_t* keys_b, uint32_t* vals_b,
-                     int64_t n_max, const uint32_t* n_dev, int key_bits, uint32_t* hist,
-                     uint32_t** keys_out, uint32_t** vals_out, cudaStream_t stream) {
-  *keys_out = keys_a;
-  *vals_out = vals_a;
-  if (n_max <= 1 || key_bits <= 0) return MTS_OK;
-  const int64_t ntiles = ceil_div(n_max, SORT_TILE);
-  const int G = (int)std::min<int64_t>(ntiles, SORT_MAX_BLOCKS);
-  uint32_t* totals = hist + (size_t)SORT_BINS * SORT_MAX_BLOCKS;
-  const int passes = (key_bits + 7) / 8;
+namespace {
+
+template <int BITS, bool SEG>
+int launch_pass(const uint32_t* ki, const uint32_t* vi, uint32_t* ko, uint32_t* vo, int64_t n_max,
+                const uint32_t* n_dev, int shift, uint32_t mask, uint32_t* hist, uint32_t* totals, int G, int T,
+                const SortSegments& seg, cudaStream_t stream) {
+  constexpr int BINS = 1 << BITS;
+  constexpr size_t SMEM = scatter_smem_bytes<BITS>();
+  static bool attr_set[64] = {};                         // per device: the opt-in for more than 48 KB
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return set_error(MTS_ERR_CUDA, "sort: cudaGetDevice");
+  if (!attr_set[dev]) {
+    int rc = check_cuda(cudaFuncSetAttribute(scatter_by_digit<BITS, SEG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)SMEM), "cudaFuncSetAttribute(scatter_by_digit)");
+    if (rc != MTS_OK) return rc;
+    attr_set[dev] = true;
+  }
+  const dim3 grid((unsigned)G, SEG ? (unsigned)T : 1u);
+  {
+    LaunchScope scope(K_SORT_HISTOGRAM, stream);
+    digit_histogram<BITS, SEG><<<grid, SORT_THREADS, 0, stream>>>(ki, n_max, n_dev, shift, mask, hist, G, seg);
+  }
+  {
+    LaunchScope scope(K_SORT_SCAN, stream);
+    const int n_rows = (SEG ? T : 1) * BINS;
+    if (G <= 64)
+      scan_histogram_rows<<<(unsigned)ceil_div(n_rows, SORT_WARPS), SORT_THREADS, 0, stream>>>(hist, totals, G, n_rows);
+    else
+      scan_histogram<<<dim3(BINS, SEG ? (unsigned)T : 1u), SORT_THREADS, 0, stream>>>(hist, totals, G);
+  }
+  {
+    LaunchScope scope(K_SORT_SCATTER, stream);
+    scatter_by_digit<BITS, SEG><<<grid, SORT_THREADS, SMEM, stream>>>(ki, vi, ko, vo, n_max, n_dev, shift, mask, hist,
+                                                                     totals, G, seg);
+  }
+  return MTS_OK;
+}
+
+template <bool SEG>
+int run_passes(uint32_t* keys_a, uint32_t* vals_a, uint32_t* keys_b, uint32_t* vals_b, int64_t n_max,
+               const uint32_t* n_dev, int key_bits, uint32_t* hist, int G, int T, const SortSegments& seg,
+               uint32_t** keys_out, uint32_t** vals_out, cudaStream_t stream) {
+  const int passes = sort_passes(key_bits), width = sort_digit_bits(key_bits);
+  const int bins_bits = width <= 8 ? 8 : width;          // the kernels exist for 8 to SORT_MAX_DIGIT_BITS bits
+  uint32_t* totals = hist + (size_t)(SEG ? T : 1) * (1u << bins_bits) * G;
   uint32_t *ki = keys_a, *vi = vals_a, *ko = keys_b, *vo = vals_b;
   for (int p = 0; p < passes; ++p) {
-    const int shift = 8 * p;
-    const int bits = min(8, key_bits - shift);
+    const int shift = width * p;
+    const int bits = std::min(width, key_bits - shift);
     const uint32_t mask = (1u << bits) - 1u;
-    const SortSegments none{nullptr, 0, nullptr};
-    {
-      LaunchScope scope(K_SORT_HISTOGRAM, stream);
-      digit_histogram<false><<<G, SORT_THREADS, 0, stream>>>(ki, n_max, n_dev, shift, mask, hist, G, none);
+    int rc;
+    switch (bins_bits) {
+      case 8: rc = launch_pass<8, SEG>(ki, vi, ko, vo, n_max, n_dev, shift, mask, hist, totals, G, T, seg, stream); break;
+      case 9: rc = launch_pass<9, SEG>(ki, vi, ko, vo, n_max, n_dev, shift, mask, hist, totals, G, T, seg, stream); break;
+      case 10: rc = launch_pass<10, SEG>(ki, vi, ko, vo, n_max, n_dev, shift, mask, hist, totals, G, T, seg, stream); break;
+      default: rc = launch_pass<11, SEG>(ki, vi, ko, vo, n_max, n_dev, shift, mask, hist, totals, G, T, seg, stream); break;
     }
-    {
-      LaunchScope scope(K_SORT_SCAN, stream);
-      scan_histogram<<<SORT_BINS, SORT_THREADS, 0, stream>>>(hist, totals, G);
-    }
-    {
-      LaunchScope scope(K_SORT_SCATTER, stream);
-      scatter_by_digit<false><<<G, SORT_THREADS, 0, stream>>>(ki, vi, ko, vo, n_max, n_dev, shift, mask, hist, totals, G,
-                                                               none);
-    }
+    if (rc != MTS_OK) return rc;
     uint32_t* t;
     t = ki; ki = ko; ko = t;
     t = vi; vi = vo; vo = t;
   }
   *keys_out = ki;
   *vals_out = vi;
-  return check_launch("radix_sort_pairs");
+  return check_launch("radix sort passes");
+}
+
+}  // namespace
+
+int radix_sort_pairs(uint32_t* keys_a, uint32_t* vals_a, uint32_t* keys_b, uint32_t* vals_b,
+                     int64_t n_max, const uint32_t* n_dev, int key_bits, uint32_t key_base, uint32_t* hist,
+                     uint32_t** keys_out, uint32_t** vals_out, cudaStream_t stream) {
+  *keys_out = keys_a;
+  *vals_out = vals_a;
+  if (n_max <= 1 || key_bits <= 0) return MTS_OK;
+  const int64_t ntiles = ceil_div(n_max, SORT_TILE);
+  const int G = (int)std::min<int64_t>(ntiles, SORT_MAX_BLOCKS);
+  const SortSegments none{nullptr, 0, nullptr, key_base};
+  return run_passes<false>(keys_a, vals_a, keys_b, vals_b, n_max, n_dev, key_bits, hist, G, 1, none, keys_out, vals_out,
+                           stream);
 }
 
 int radix_sort_pairs_segmented(uint32_t* keys_a, uint32_t* vals_a, uint32_t* keys_b, uint32_t* vals_b, int64_t n,
@@ -317,35 +417,8 @@ int radix_sort_pairs_segmented(uint32_t* keys_a, uint32_t* vals_a, uint32_t* key
   *vals_out = vals_a;
   if (n <= 1 || key_bits <= 0 || T <= 0) return MTS_OK;
   const int G = sort_segment_blocks(n, T);
-  uint32_t* totals = hist + (size_t)T * SORT_BINS * G;
-  const int passes = (key_bits + 7) / 8;
-  const dim3 grid((unsigned)G, (unsigned)T);
-  uint32_t *ki = keys_a, *vi = vals_a, *ko = keys_b, *vo = vals_b;
-  for (int p = 0; p < passes; ++p) {
-    const int shift = 8 * p;
-    const int bits = min(8, key_bits - shift);
-    const uint32_t mask = (1u << bits) - 1u;
-    {
-      LaunchScope scope(K_SORT_HISTOGRAM, stream);
-      digit_histogram<true><<<grid, SORT_THREADS, 0, stream>>>(ki, n, nullptr, shift, mask, hist, G, seg);
-    }
-    {
-      LaunchScope scope(K_SORT_SCAN, stream);
-      const int n_rows = T * SORT_BINS;
-      scan_histogram_rows<<<(unsigned)ceil_div(n_rows, SORT_WARPS), SORT_THREADS, 0, stream>>>(hist, totals, G, n_rows);
-    }
-    {
-      LaunchScope scope(K_SORT_SCATTER, stream);
-      scatter_by_digit<true><<<grid, SORT_THREADS, 0, stream>>>(ki, vi, ko, vo, n, nullptr, shift, mask, hist, totals, G,
-                                                               seg);
-    }
-    uint32_t* t;
-    t = ki; ki = ko; ko = t;
-    t = vi; vi = vo; vo = t;
-  }
-  *keys_out = ki;
-  *vals_out = vi;
-  return check_launch("radix_sort_pairs_segmented");
+  return run_passes<true>(keys_a, vals_a, keys_b, vals_b, n, nullptr, key_bits, hist, G, T, seg, keys_out, vals_out,
+                          stream);
 }
 
 // ------------------------------------------------------------------------------------ distinct keys

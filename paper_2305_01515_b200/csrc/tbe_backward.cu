@@ -658,6 +658,46 @@ __global__ void export_unique(const uint32_t* __restrict__ keys, const uint32_t*
   if (blockIdx.x == 0 && threadIdx.x == 0) *n_unique_out = (int64_t)U;
 }
 
+namespace {
+
+int bits_for(int64_t values) {
+  int bits = 1;
+  while (bits < 32 && (1ll << bits) < values) ++bits;
+  return bits;
+}
+
+// How the lookups are sorted by row.  They arrive grouped by table, so each table's lookups can be
+// sorted on their own on the bits of the row index inside the table; that is used when it saves a
+// pass over sorting the linear row ids of all tables together.
+struct SortPlan {
+  bool segmented;
+  int key_bits;
+  int passes() const { return sort_passes(key_bits); }
+};
+
+SortPlan sort_plan(const mts_tables* h) {
+  int64_t max_rows = 1;
+  for (const auto& m : h->h_meta) max_rows = std::max<int64_t>(max_rows, m.rows);
+  int64_t min_rows = max_rows;
+  for (const auto& m : h->h_meta) min_rows = std::min<int64_t>(min_rows, m.rows);
+  const int all_bits = bits_for(h->total_rows), table_bits = bits_for(max_rows);
+  if (h->T > 1) {
+    if (sort_passes(table_bits) < sort_passes(all_bits)) return {true, table_bits};
+    // as many passes, but the smaller tables have no bit left in the last one and are only copied there
+    if (sort_passes(table_bits) == sort_passes(all_bits) && sort_passes(table_bits) > 1 &&
+        bits_for(min_rows) <= sort_digit_bits(table_bits) * (sort_passes(table_bits) - 1))
+      return {true, table_bits};
+  }
+  return {false, all_bits};
+}
+
+// which of the two buffer pairs holds the sorted lookups after the sort
+bool sorted_in_b(const mts_tables* h, int64_t N) {
+  return N > 1 && (sort_plan(h).passes() & 1) != 0;
+}
+
+}  // namespace
+
 struct BwdLayout {
   size_t keys_a, keys_b, vals_a, vals_b, bag_of_pos, hist, scan, seg_start, n_unique, next_chunk, head, tail, group, total;
 };
@@ -669,7 +709,9 @@ static BwdLayout bwd_layout(const mts_tables* h, int64_t N) {
   const size_t n = (size_t)(N > 0 ? N : 1);
   L.keys_a = take(n * 4); L.keys_b = take(n * 4); L.vals_a = take(n * 4); L.vals_b = take(n * 4);
   L.bag_of_pos = take(n * 4);
-  L.hist = take(std::max(sort_hist_words(), sort_hist_words_segmented((int64_t)n, h->T)) * 4);
+  const SortPlan plan = sort_plan(h);
+  L.hist = take((plan.segmented ? sort_hist_words_segmented((int64_t)n, h->T, plan.key_bits)
+                                : sort_hist_words((int64_t)n, plan.key_bits)) * 4);
   L.scan = take(scan_scratch_words() * 4);
   L.seg_start = take((n + 1) * 4);
   L.n_unique = take(256);
@@ -757,34 +799,6 @@ extern "C" size_t mts_tbe_backward_workspace_bytes(const mts_tables* h, int32_t 
 
 namespace {
 
-int bits_for(int64_t values) {
-  int bits = 1;
-  while (bits < 32 && (1ll << bits) < values) ++bits;
-  return bits;
-}
-
-// How the lookups are sorted by row.  They arrive grouped by table, so each table's lookups can be
-// sorted on their own on the bits of the row index inside the table; that is used when it saves a
-// pass over sorting the linear row ids of all tables together.
-struct SortPlan {
-  bool segmented;
-  int key_bits;
-  int passes() const { return (key_bits + 7) / 8; }
-};
-
-SortPlan sort_plan(const mts_tables* h) {
-  int64_t max_rows = 1;
-  for (const auto& m : h->h_meta) max_rows = std::max<int64_t>(max_rows, m.rows);
-  const int all_bits = bits_for(h->total_rows), table_bits = bits_for(max_rows);
-  if (h->T > 1 && (table_bits + 7) / 8 < (all_bits + 7) / 8) return {true, table_bits};
-  return {false, all_bits};
-}
-
-// which of the two buffer pairs holds the sorted lookups after the sort
-bool sorted_in_b(const mts_tables* h, int64_t N) {
-  return N > 1 && (sort_plan(h).passes() & 1) != 0;
-}
-
 int check_backward_common(const mts_tables* h, int32_t B, const int64_t* offsets, int64_t N, void* workspace,
                           size_t workspace_bytes, const BwdLayout& L, const char* who) {
   if (!h || !offsets || B < 1 || N < 0) return set_error(MTS_ERR_INVALID_ARG, "%s: null argument or bad size", who);
@@ -835,11 +849,11 @@ extern "C" int mts_tbe_backward_sort(const mts_tables* h, int32_t B, const int64
   uint32_t *keys = nullptr, *pos = nullptr;
   const SortPlan plan = sort_plan(h);
   if (plan.segmented) {
-    const SortSegments seg{offsets, B, h->d_meta};
+    const SortSegments seg{offsets, B, h->d_meta, 0u};
     rc = radix_sort_pairs_segmented(keys_a, vals_a, keys_b, vals_b, N, h->T, seg, plan.key_bits,
                                     reinterpret_cast<uint32_t*>(ws + L.hist), &keys, &pos, s);
   } else {
-    rc = radix_sort_pairs(keys_a, vals_a, keys_b, vals_b, N, nullptr, plan.key_bits,
+    rc = radix_sort_pairs(keys_a, vals_a, keys_b, vals_b, N, nullptr, plan.key_bits, 0u,
                           reinterpret_cast<uint32_t*>(ws + L.hist), &keys, &pos, s);
   }
   if (rc != MTS_OK) return rc;
@@ -860,10 +874,13 @@ extern "C" int mts_tbe_backward_sort(const mts_tables* h, int32_t B, const int64
 }
 
 namespace {
+// sorted_rows / sorted_pos / bag_of_lookup: null = the arrays mts_tbe_backward_sort left in the workspace
 int backward_apply(const mts_tables* h, int32_t B, const int64_t* offsets, int64_t N, int32_t pooling_mode,
                    const void* grad_out, bool grad_half, int64_t grad_stride, float lr, float eps,
                    const int32_t* slot_of_lookup, void* const* host_cache_data, uint8_t* const* host_cache_dirty,
-                   int32_t n_caches, void* workspace, size_t workspace_bytes, void* stream) {
+                   int32_t n_caches, void* workspace, size_t workspace_bytes, void* stream,
+                   const uint32_t* sorted_rows = nullptr, const uint32_t* sorted_pos = nullptr,
+                   const uint32_t* bag_of_lookup = nullptr) {
   if (!h) return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_apply: null tables");
   const BwdLayout L = bwd_layout(h, N > 0 ? N : 0);
   int rc = check_backward_common(h, B, offsets, N, workspace, workspace_bytes, L, "tbe_backward_apply");
@@ -886,6 +903,11 @@ int backward_apply(const mts_tables* h, int32_t B, const int64_t* offsets, int64
   const uint32_t* keys = reinterpret_cast<const uint32_t*>(ws + (in_b ? L.keys_b : L.keys_a));
   const uint32_t* pos = reinterpret_cast<const uint32_t*>(ws + (in_b ? L.vals_b : L.vals_a));
   const uint32_t* bag_of_pos = h->any_cached ? reinterpret_cast<const uint32_t*>(ws + L.bag_of_pos) : nullptr;
+  if (sorted_rows != nullptr) {
+    keys = sorted_rows;
+    pos = sorted_pos;
+    bag_of_pos = bag_of_lookup;
+  }
   float* head = reinterpret_cast<float*>(ws + L.head);
   float* tail = reinterpret_cast<float*>(ws + L.tail);
   float* group = reinterpret_cast<float*>(ws + L.group);
@@ -923,6 +945,23 @@ extern "C" int mts_tbe_backward_apply_f16(const mts_tables* h, int32_t B, const 
                                           int32_t n_caches, void* workspace, size_t workspace_bytes, void* stream) {
   return backward_apply(h, B, offsets, N, pooling_mode, grad_out_f16, true, grad_stride, lr, eps, slot_of_lookup,
                         host_cache_data, host_cache_dirty, n_caches, workspace, workspace_bytes, stream);
+}
+
+extern "C" int mts_tbe_backward_apply_presorted(const mts_tables* h, int32_t B, const int64_t* offsets, int64_t N,
+                                                int32_t pooling_mode, const void* grad_out, int32_t grad_dtype,
+                                                int64_t grad_stride, float lr, float eps,
+                                                const uint32_t* sorted_rows, const uint32_t* sorted_pos,
+                                                const uint32_t* bag_of_lookup, const int32_t* slot_of_lookup,
+                                                void* const* host_cache_data, uint8_t* const* host_cache_dirty,
+                                                int32_t n_caches, void* workspace, size_t workspace_bytes,
+                                                void* stream) {
+  if (grad_dtype != MTS_DTYPE_FP32 && grad_dtype != MTS_DTYPE_FP16)
+    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_apply_presorted: grad_dtype %d", grad_dtype);
+  if (N > 0 && (!sorted_rows || !sorted_pos || !bag_of_lookup))
+    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_apply_presorted: null sorted_rows / sorted_pos / bag_of_lookup");
+  return backward_apply(h, B, offsets, N, pooling_mode, grad_out, grad_dtype == MTS_DTYPE_FP16, grad_stride, lr, eps,
+                        slot_of_lookup, host_cache_data, host_cache_dirty, n_caches, workspace, workspace_bytes, stream,
+                        sorted_rows, sorted_pos, bag_of_lookup);
 }
 
 extern "C" int mts_tbe_backward_rowwise_adagrad(

@@ -4,7 +4,8 @@ Nothing here computes anything on its own; every step is a call into libmtrains_
 """
 from __future__ import annotations
 
-from typing import List, Optional
+import os
+from typing import List, Optional, Sequence
 
 import numpy as np
 import torch
@@ -16,42 +17,57 @@ from . import workload as wl
 class DeviceModel:
     """Weights, optimizer state and scratch of one ModelSpec on one GPU.
 
-    Uncached specs keep all tables in one flat HBM buffer.  Cached specs keep them in one flat
-    pinned host buffer (device-visible through unified addressing) behind one cache per
-    embedding dim."""
+    Tables are either HBM resident (one flat device buffer) or host resident (one flat pinned host
+    buffer, device-visible through unified addressing) behind one cache per embedding dim.  By default
+    an uncached spec keeps every table in HBM and a cached spec every table in the host tier;
+    `host_tables` (one bool per table) mixes the two in one model."""
+
+    N_CTX = 4        # batch contexts: batch t trains, the rows of t+1 move, the tags of t+2 are looked
+    #                  up, and the overflow list of t-1 is still needed to repair rows after batch t
 
     def __init__(self, spec: wl.ModelSpec, device="cuda:0", max_lookups: int = 0, weights: Optional[np.ndarray] = None,
-                 lock_depth: int = 0, policy: int = mb.POLICY_LRU, cache_sets: Optional[List[int]] = None):
+                 lock_depth: int = 0, policy: int = mb.POLICY_LRU, cache_sets: Optional[List[int]] = None,
+                 host_tables: Optional[Sequence[bool]] = None):
         self.spec = spec
         self.lock_depth = lock_depth
         self.device = torch.device(device)
         self.tdtype = torch.float32 if spec.dtype == wl.FP32 else torch.float16
         n_elem = int(spec.weight_offset[-1])
-        self.cached = spec.cached
-        if self.cached:
-            self.host_weights = torch.empty(n_elem, dtype=self.tdtype, pin_memory=True)
-            self.dev_weights = None
-            store = self.host_weights
-        else:
-            self.dev_weights = torch.empty(n_elem, dtype=self.tdtype, device=self.device)
-            self.host_weights = None
-            store = self.dev_weights
-        if weights is not None:
-            store.copy_(torch.from_numpy(weights))
-        else:
-            for t in range(spec.T):
-                a, b = int(spec.weight_offset[t]), int(spec.weight_offset[t + 1])
-                dst = store[a:b].view(-1, int(spec.dims[t]))
-                step = 1 << 22
-                for r0 in range(0, int(spec.rows[t]), step):
-                    r1 = min(r0 + step, int(spec.rows[t]))
-                    dst[r0:r1].copy_(wl.weights_torch(spec, t, self.device, r0, r1))
+        if host_tables is None:
+            host_tables = [bool(spec.cached)] * spec.T
+        self.host_tables = [bool(x) for x in host_tables]
+        self.cached = any(self.host_tables)
+        self.all_cached = all(self.host_tables)
+        self.host_weights = torch.empty(n_elem, dtype=self.tdtype, pin_memory=True) if self.cached else None
+        self.dev_weights = None if self.all_cached else torch.empty(n_elem, dtype=self.tdtype, device=self.device)
+        for t in range(spec.T):
+            a, b = int(spec.weight_offset[t]), int(spec.weight_offset[t + 1])
+            store = self.host_weights if self.host_tables[t] else self.dev_weights
+            if weights is not None:
+                store[a:b].copy_(torch.from_numpy(weights[a:b]))
+                continue
+            dst = store[a:b].view(-1, int(spec.dims[t]))
+            step = 1 << 22
+            for r0 in range(0, int(spec.rows[t]), step):
+                r1 = min(r0 + step, int(spec.rows[t]))
+                dst[r0:r1].copy_(wl.weights_torch(spec, t, self.device, r0, r1))
         self.momentum = torch.zeros(int(spec.row_offset[-1]), dtype=torch.float32, device=self.device)
         self.caches: List[mb.Cache] = []
-        self.groups = spec.dim_groups() if self.cached else []
+        # one cache per run of consecutive host-tier tables of one dim
+        self.groups = []
+        t = 0
+        while t < spec.T:
+            if not self.host_tables[t]:
+                t += 1
+                continue
+            t1 = t
+            while t1 < spec.T and self.host_tables[t1] and spec.dims[t1] == spec.dims[t]:
+                t1 += 1
+            self.groups.append((int(spec.dims[t]), t, t1))
+            t = t1
         cache_id = None
         if self.cached:
-            cache_id = np.zeros(spec.T, np.int32)
+            cache_id = np.full(spec.T, -1, np.int32)
             for g, (dim, t0, t1) in enumerate(self.groups):
                 cache_id[t0:t1] = g
                 rows_g = int(spec.row_offset[t1] - spec.row_offset[t0])
@@ -64,6 +80,7 @@ class DeviceModel:
         self.max_lookups = 0
         self.workspace = None
         self.ws_bytes = 0
+        self.fetch_rows = None
         if max_lookups:
             self.reserve(max_lookups)
 
@@ -80,16 +97,13 @@ class DeviceModel:
         self.cache_ws_bytes = max([mb.cache_workspace_bytes(c, max_lookups) for c in self.caches] + [256])
         self.cache_ws = torch.empty(self.cache_ws_bytes, dtype=torch.uint8, device=self.device)
         if self.cached:
-            # three batch contexts: batch t trains while the rows of batch t+1 move and the tags of
-            # batch t+2 are looked up; the victim staging buffer is only used inside one data
-            # movement call sequence, so one per cache serves all contexts
+            # the victim staging buffer is only used inside one data movement call sequence, so one per
+            # cache serves all batch contexts
             esz = 4 if self.spec.dtype == wl.FP32 else 2
             self.staging = [torch.empty(min(max_lookups, c.num_sets * c.ways) * c.dim * esz, dtype=torch.uint8,
                                         device=self.device) for c in self.caches]
             self.ctx = [self._new_context(max_lookups) for _ in range(self.N_CTX)]
             self.cur = 0
-
-    N_CTX = 3
 
     def _new_context(self, n: int):
         dev = self.device
@@ -102,12 +116,16 @@ class DeviceModel:
                 evict_keys=torch.empty(cap, dtype=torch.int64, device=dev),
                 evict_slots=torch.empty(cap, dtype=torch.int32, device=dev),
                 evict_dirty=torch.empty(cap, dtype=torch.uint8, device=dev),
-                overflow_keys=torch.empty(cap, dtype=torch.int64, device=dev),
+                overflow_keys=torch.empty(n, dtype=torch.int64, device=dev),      # never cut: n distinct keys at most
+                overflow_capacity=n,
                 counters=torch.zeros(mb.NUM_COUNTERS, dtype=torch.int64, device=dev),
                 staging=self.staging[g],
                 capacity=cap))
+        # the lookups ordered by row (uint32 bit patterns), written by the tag step and reused by the backward
         return dict(slot=torch.full((n,), -1, dtype=torch.int32, device=dev),
-                    keys=torch.empty(n, dtype=torch.int64, device=dev), lists=lists)
+                    sorted_rows=torch.empty(n, dtype=torch.int32, device=dev),
+                    sorted_pos=torch.empty(n, dtype=torch.int32, device=dev),
+                    bag_of_lookup=torch.empty(n, dtype=torch.int32, device=dev), lists=lists)
 
     @property
     def slot_of_lookup(self):
@@ -117,30 +135,42 @@ class DeviceModel:
     def lists(self):
         return self.ctx[self.cur]["lists"]
 
+    def _ctx(self, ctx: Optional[int]):
+        return self.ctx[self.cur if ctx is None else ctx]
+
     # ------------------------------------------------------------------ steps of the path
     def forward(self, indices, offsets, N: int, out=None, pooling_mode: int = mb.POOL_SUM, stream=None,
                 ctx: Optional[int] = None):
         if out is None:
             out = torch.empty((self.spec.batch, self.spec.total_dim), dtype=torch.float32, device=self.device)
-        slot = self.ctx[self.cur if ctx is None else ctx]["slot"] if self.cached else None
+        slot = self._ctx(ctx)["slot"] if self.cached else None
         mb.tbe_forward(self.tables, self.spec.batch, indices, offsets, N, pooling_mode, slot, self.cache_data, out,
                        out.shape[1], stream, f16=out.dtype == torch.float16)
         return out
 
     def backward(self, indices, offsets, N: int, grad_out, lr: Optional[float] = None, eps: Optional[float] = None,
                  pooling_mode: int = mb.POOL_SUM, uniq_rows_out=None, n_unique_out=None, stream=None,
-                 ctx: Optional[int] = None) -> None:
+                 ctx: Optional[int] = None, reuse_tag_order: bool = True) -> None:
+        """reuse_tag_order: when every table is cached, the backward takes the lookups ordered by row from
+        the tag step of the same batch instead of sorting them again."""
         self.reserve(N)
+        lr = self.spec.lr if lr is None else lr
+        eps = self.spec.eps if eps is None else eps
+        if self.all_cached and reuse_tag_order and uniq_rows_out is None:
+            cx = self._ctx(ctx)
+            mb.tbe_backward_apply_presorted(
+                self.tables, self.spec.batch, offsets, N, pooling_mode, grad_out, grad_out.shape[1], lr, eps,
+                cx["sorted_rows"], cx["sorted_pos"], cx["bag_of_lookup"], cx["slot"], self.cache_data,
+                self.cache_dirty, self.workspace, self.ws_bytes, stream, f16=grad_out.dtype == torch.float16)
+            return
         if grad_out.dtype == torch.float16:      # fp16 gradients: the two-call form
             self.backward_sort(indices, offsets, N, uniq_rows_out, n_unique_out, stream)
             self.backward_apply(offsets, N, grad_out, lr, eps, pooling_mode, stream, ctx)
             return
-        slot = self.ctx[self.cur if ctx is None else ctx]["slot"] if self.cached else None
+        slot = self._ctx(ctx)["slot"] if self.cached else None
         mb.tbe_backward_rowwise_adagrad(
-            self.tables, self.spec.batch, indices, offsets, N, pooling_mode, grad_out, grad_out.shape[1],
-            self.spec.lr if lr is None else lr, self.spec.eps if eps is None else eps,
-            slot, self.cache_data, self.cache_dirty, self.workspace,
-            self.ws_bytes, uniq_rows_out, n_unique_out, stream)
+            self.tables, self.spec.batch, indices, offsets, N, pooling_mode, grad_out, grad_out.shape[1], lr, eps,
+            slot, self.cache_data, self.cache_dirty, self.workspace, self.ws_bytes, uniq_rows_out, n_unique_out, stream)
 
     def backward_sort(self, indices, offsets, N: int, uniq_rows_out=None, n_unique_out=None, stream=None) -> None:
         """Index-only half of the backward; may run on another stream than the forward pass."""
@@ -151,7 +181,7 @@ class DeviceModel:
     def backward_apply(self, offsets, N: int, grad_out, lr: Optional[float] = None, eps: Optional[float] = None,
                        pooling_mode: int = mb.POOL_SUM, stream=None, ctx: Optional[int] = None) -> None:
         """Gradient half of the backward, after backward_sort of the same batch."""
-        slot = self.ctx[self.cur if ctx is None else ctx]["slot"] if self.cached else None
+        slot = self._ctx(ctx)["slot"] if self.cached else None
         mb.tbe_backward_apply(
             self.tables, self.spec.batch, offsets, N, pooling_mode, grad_out, grad_out.shape[1],
             self.spec.lr if lr is None else lr, self.spec.eps if eps is None else eps,
@@ -172,19 +202,20 @@ class DeviceModel:
 
     def cache_lookup(self, indices, offsets, offsets_host: np.ndarray, step: int, stream=None,
                      ctx: Optional[int] = None) -> None:
-        """Tag path of one batch: keys, lookup_insert of every cache (slots, miss and evict lists)."""
+        """Tag path of one batch: lookup_insert of every cache (slots, miss / evict / overflow lists, and the
+        batch's lookups ordered by row for the backward)."""
         B = self.spec.batch
-        cx = self.ctx[self.cur if ctx is None else ctx]
+        cx = self._ctx(ctx)
         for g, c in enumerate(self.caches):
             _, t0, t1 = self.groups[g]
             begin, n = self.group_range(g, offsets_host)
             L = cx["lists"][g]
-            keys = cx["keys"][begin:begin + n]
-            mb.linearize_keys(self.tables, t0, t1, B, indices, offsets, begin, n, keys if n else None, stream)
-            mb.cache_lookup_insert(c, keys if n else None, n, step, cx["slot"][begin:begin + n] if n else None,
-                                   L["miss_keys"], L["miss_slots"], L["evict_keys"], L["evict_slots"],
-                                   L["evict_dirty"], L["capacity"], L["counters"], self.cache_ws, self.cache_ws_bytes,
-                                   stream, overflow_keys=L["overflow_keys"])
+            mb.cache_lookup_insert_tables(
+                c, self.tables, t0, t1, B, indices, offsets, begin, n, step, cx["slot"], L["miss_keys"],
+                L["miss_slots"], L["evict_keys"], L["evict_slots"], L["evict_dirty"], L["capacity"],
+                L["overflow_keys"], L["overflow_capacity"], L["counters"], self.cache_ws, self.cache_ws_bytes, stream,
+                sorted_rows_out=cx["sorted_rows"], sorted_pos_out=cx["sorted_pos"],
+                bag_of_lookup_out=cx["bag_of_lookup"])
 
     def cache_move(self, stream=None, ctx: Optional[int] = None) -> None:
         """Data path of one batch: save dirty victims, pull missed rows from the host tier, write victims back."""
@@ -194,7 +225,7 @@ class DeviceModel:
 
     def cache_fetch(self, g: int, stream=None, ctx: Optional[int] = None) -> None:
         """Cache g: dirty victims into the staging buffer, then the missed rows from the host tier into their slots."""
-        L = self.ctx[self.cur if ctx is None else ctx]["lists"][g]
+        L = self._ctx(ctx)["lists"][g]
         mb.cache_prefetch_misses(self.caches[g], self.host_rows_ptr(g), L["miss_keys"], L["miss_slots"],
                                  L["evict_slots"], L["evict_dirty"], L["capacity"], L["counters"], L["staging"], stream)
 
@@ -204,7 +235,8 @@ class DeviceModel:
     def enable_host_gather(self, threads: Optional[int] = None) -> None:
         """Pinned host buffers (keys and gathered rows, per cache and batch context) and one device
         buffer per cache for the copy-engine path of the missed rows."""
-        import os
+        if self.fetch_rows is not None:
+            return
         esz = 4 if self.spec.dtype == wl.FP32 else 2
         self.gather_threads = threads or os.cpu_count() or 1
         self.fetch_rows = [max(1, min(self.ctx[0]["lists"][g]["capacity"], self.FETCH_STAGE_BYTES // (c.dim * esz)))
@@ -218,7 +250,7 @@ class DeviceModel:
 
     def cache_fetch_via_host(self, g: int, n_miss: int, copy_stream, stream, ctx: int, mark=None) -> bool:
         """Cache g, copy-engine path: the first n_miss keys of the miss list come to the host on
-        `copy_stream` (the caller made it wait for the tag step), host threads gather the rows, one
+        `copy_stream` (the caller made sure the tag step is over), host threads gather the rows, one
         contiguous copy and the placing kernel follow on `stream`.  Blocks the calling thread for the key
         copy and the gather.  Returns False (nothing done) when the list does not fit the buffers."""
         if n_miss > self.fetch_rows[g]:
@@ -246,17 +278,17 @@ class DeviceModel:
 
     def cache_writeback(self, g: int, stream=None, ctx: Optional[int] = None) -> None:
         """Cache g: the staged dirty victims back to the host tier (after cache_fetch of the same batch)."""
-        L = self.ctx[self.cur if ctx is None else ctx]["lists"][g]
+        L = self._ctx(ctx)["lists"][g]
         mb.cache_writeback_evicted(self.caches[g], self.host_rows_ptr(g), L["evict_keys"], L["evict_dirty"],
                                    L["capacity"], L["counters"], L["staging"], stream)
 
     def cache_refetch(self, prev_ctx: int, placed_step: int = -1, stream=None) -> None:
         """After the backward of the batch in context `prev_ctx`: refresh rows that overflowed there
-        and were placed by the next batch (the one whose lookup had step `placed_step`)."""
+        and were placed by the batch whose lookup had step `placed_step`."""
         for g, c in enumerate(self.caches):
             L = self.ctx[prev_ctx]["lists"][g]
-            mb.cache_refetch_overflowed(c, self.host_rows_ptr(g), L["overflow_keys"], L["capacity"], L["counters"],
-                                        placed_step, stream)
+            mb.cache_refetch_overflowed(c, self.host_rows_ptr(g), L["overflow_keys"], L["overflow_capacity"],
+                                        L["counters"], placed_step, stream)
 
     def cache_step(self, indices, offsets, offsets_host: np.ndarray, step: int, stream=None,
                    do_prefetch: bool = True, ctx: Optional[int] = None) -> None:
@@ -270,9 +302,18 @@ class DeviceModel:
             mb.cache_flush(c, self.host_rows_ptr(g), stream)
 
     def weights_numpy(self) -> np.ndarray:
+        """All tables back to back, each from the memory that holds it (host-tier tables: call flush first)."""
         torch.cuda.synchronize(self.device)
-        src = self.host_weights if self.cached else self.dev_weights
-        return src.cpu().numpy().copy()
+        if not self.cached:
+            return self.dev_weights.cpu().numpy().copy()
+        out = self.host_weights.numpy().copy()
+        if not self.all_cached:
+            dev = self.dev_weights.cpu().numpy()
+            for t in range(self.spec.T):
+                if not self.host_tables[t]:
+                    a, b = int(self.spec.weight_offset[t]), int(self.spec.weight_offset[t + 1])
+                    out[a:b] = dev[a:b]
+        return out
 
     def close(self) -> None:
         self.tables.destroy()

@@ -4,31 +4,44 @@ lookups).  Streams, ordered by events only:
 
     main    : forward(t), backward(t)
     move[g] : cache g: save victims / fetch missed rows / write victims back for batch t+1   (host link)
-    fix     : repair of rows that overflowed in batch t and were placed in batch t+1 (after backward(t))
+    fix     : repair of rows that overflowed in batches t and t-1 and were placed by batch t+1
     tag     : tag lookup and replacement for batch t+2                              (HBM, small)
 
 so the host-link traffic of the next batch and the tag work of the one after it overlap the
-training of the current batch.
+training of the current batch.  With lock_depth 2 the side streams run up to two batches ahead of
+the training; the launching thread never waits for the device.
 
-Why this is safe with lock_depth >= 1.  The tag step of batch t+2 may only take ways stamped before
-t+2-lock_depth; it waits for the backward of the newest such batch (batch t for lock_depth 1, batch
-t-1 for lock_depth 2, which takes the tag step off the critical path), so it only evicts rows whose
-batches have trained, and never a way of a batch that is still waiting to train.  Its decisions read and write tags, timestamps
-and the dirty bytes of its victims only; forward/backward write none of the first two and only the
-dirty bytes of their own batch's slots.  The data movement of batch t+1 touches victim slots (trained
-at t-1 or earlier, complete because the tag step waited for backward(t-1)) and the slots of missed
-rows, which no batch in flight uses.  One hazard is left: a row that found no evictable way in batch
-t (it is read and updated in host memory directly) and is fetched from host memory for batch t+1,
-possibly before backward(t) has updated it.  When batch t reported such overflow, the data movement
-of batch t+1 still runs at once, and after backward(t) the rows of batch t's overflow list that batch
-t+1 placed are copied from host memory again (mts_cache_refetch_overflowed with placed_step = the step
-of batch t+1: the tag step of batch t+2 may already have placed other keys of that list, in slots that
-hold their victims' rows until batch t+2's data movement, and those must not be touched).  A row that
-overflowed in batch t-1 and is first placed by batch t+1 is covered by ordering: the data movement of
-batch t+1 waits for backward(t-1).
+Why this is safe with lock_depth >= 1.  The tag step of batch t may only take ways stamped before
+t - lock_depth; it waits for the backward of the newest such batch (t - 1 - lock_depth), so it only
+evicts rows whose batches have trained and never a way of a batch that is still waiting to train.
+Its decisions read and write tags, timestamps and the dirty bytes of its victims only;
+forward/backward write none of the first two and only the dirty bytes of their own batch's slots.
+The data movement of batch t touches victim slots (complete, because the tag step waited for their
+batches) and the slots of missed rows, which no batch in flight uses; a cache's movements follow
+one another on one stream, so a row written back by one batch is in host memory before a later
+batch fetches it.
+
+Rows that found no evictable way ("overflow": read and updated in host memory directly) need one
+more rule.  Batch t's data movement may run before the backward passes of batches t-1 ... t-lock_depth
+have updated such rows in host memory; if batch t places one of them, its copy in the cache can be
+stale.  After the backward of batch t-1 (and the data movement of batch t), the keys of the overflow
+lists of batches t-1 ... t-lock_depth that are resident in a way stamped t are therefore copied from
+host memory again (mts_cache_refetch_overflowed with placed_step = t; the stamp keeps the repair away
+from keys that a tag step running further ahead has placed in slots that still hold their victims'
+rows).  Older overflowed rows need nothing: the tag step of batch t already waited for their backward.
+
+Batch contexts (DeviceModel.N_CTX = 4): the tag step of batch t+2 rewrites the context batch t-2
+used, whose overflow list the repair before batch t still reads, so it also waits for that repair.
+
+With host_gather the missed rows do not cross the host link at the request of SMs (small reads that
+slow every kernel beside them): a worker thread reads the miss list, gathers the rows with the host's
+threads into a pinned buffer and enqueues one contiguous copy and the placing kernel.  The worker runs
+ahead of the launching thread; host-side flags tell each side which events the other has recorded.
 """
 from __future__ import annotations
 
+import queue
+import threading
 from typing import Callable, List, Optional
 
 import numpy as np
@@ -43,32 +56,40 @@ class CachedTrainer:
         """host_gather: missed rows are gathered by host threads into a pinned buffer and moved by the
         copy engine, instead of being read over the host link by a kernel."""
         assert model.cached
+        # the side streams run two batches ahead and keep two overflow lists alive: lock depths 1 and 2
+        assert not pipelined or 1 <= model.lock_depth <= 2, "the pipelined schedule needs lock_depth 1 or 2"
         self.m = model
         self.host_gather = host_gather
         if host_gather:
             model.enable_host_gather()
-        self._ev_prev_ready = None
         self.pipelined = pipelined
         self.dev = model.device
         self.main = torch.cuda.current_stream(self.dev)
         self.tag = torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main
         # the data movement needs few thread blocks but must not queue behind the training kernels' blocks;
-        # one stream per cache, so that the caches' row fetches share the host link instead of taking turns
+        # one stream per cache, so that the caches' row traffic shares the host link instead of taking turns
         n_c = len(model.caches)
         self.moves = [torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main for _ in range(n_c)]
         self.fix = torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main
         self.copy = torch.cuda.Stream(self.dev, priority=-1)       # miss keys to the host (host_gather)
-        self.host_counters = [torch.zeros((n_c, mb.NUM_COUNTERS), dtype=torch.int64).pin_memory()
-                              for _ in range(DeviceModel.N_CTX)]
-        self.history: List[np.ndarray] = []           # per batch [n_caches, NUM_COUNTERS]
+        self.history: List[np.ndarray] = []           # per batch [n_caches, NUM_COUNTERS], filled when run() returns
         self.record_timeline = False                  # set to True to time every phase with events
         self._marks = []
+        self._mark_lock = threading.Lock()
+        self.debug_delay_cycles = 0                   # > 0: the move and repair streams idle that long before their work
+
+    def _delay(self, stream):
+        """Test aid: hold a side stream back so that the training and the tag step run far ahead of it."""
+        if self.debug_delay_cycles > 0:
+            with torch.cuda.stream(stream):
+                torch.cuda._sleep(int(self.debug_delay_cycles))
 
     def _mark(self, name, t, stream):
         if self.record_timeline:
             e = torch.cuda.Event(enable_timing=True)
             e.record(stream)
-            self._marks.append((name, t, e))
+            with self._mark_lock:
+                self._marks.append((name, t, e))
 
     def timeline(self):
         """[(phase, batch, ms since the first mark)] after a run with record_timeline = True."""
@@ -78,147 +99,184 @@ class CachedTrainer:
         base = self._marks[0][2]
         return [(n, t, base.elapsed_time(e)) for n, t, e in self._marks]
 
-    def _lookup(self, t, step, batch, ev_tags, wait_event):
-        """Tag path of batch t on the tag stream (into context t mod 3)."""
+    # ------------------------------------------------------------------ the three phases of a batch
+    def _lookup(self, t, batch):
+        """Tag path of batch t on the tag stream (into context t mod N_CTX); its counters go to row t of the
+        pinned history buffer."""
         m, s, ctx = self.m, self.tag, t % DeviceModel.N_CTX
-        if wait_event is not None:
-            s.wait_event(wait_event)
+        if self.pipelined:
+            if t - 2 >= 0:
+                s.wait_event(self.ev_ready[t - 2])              # the repair that still read this context's lists
+            last = t - 1 - m.lock_depth                         # newest batch whose rows may be evicted now
+            if last >= 0:
+                s.wait_event(self.ev_bwd[last])
         self._mark("tag_begin", t, s)
-        m.cache_lookup(batch[0], batch[1], batch[2], step, stream=s, ctx=ctx)
+        m.cache_lookup(batch[0], batch[1], batch[2], self._first_step + t, stream=s, ctx=ctx)
         self._mark("tag_end", t, s)
         with torch.cuda.stream(s):
             for g in range(len(m.caches)):
-                self.host_counters[ctx][g].copy_(m.ctx[ctx]["lists"][g]["counters"], non_blocking=True)
-        ev_tags.record(s)
+                self._host_counters[t, g].copy_(m.ctx[ctx]["lists"][g]["counters"], non_blocking=True)
+        self.ev_tags[t].record(s)
 
-    def _move(self, t, ev_tags, ev_ready, prev_overflow, prev_bwd):
-        """Data path of batch t, each cache on its own move stream.  prev_overflow: number of rows of
-        batch t-1 that found no way (0 = none), prev_bwd: event after batch t-1's backward."""
-        ctx = t % DeviceModel.N_CTX
-        refetch = wait_bwd = False
-        if prev_overflow:
-            cap = min(L["capacity"] for L in self.m.ctx[(t - 1) % DeviceModel.N_CTX]["lists"])
-            if prev_overflow <= cap:
-                refetch = True                       # move now, repair the few stale rows afterwards
-            else:
-                wait_bwd = True                      # the list was cut: wait for the backward first
-        ends = []
-        for g, s in enumerate(self.moves):
-            s.wait_event(ev_tags)
-            if wait_bwd:
-                s.wait_event(prev_bwd)
-            self._mark(f"move{g}_begin", t, s)
-            # fetch, then write back, in stream order: the next batch's fetch of this cache, which may
-            # miss a row written back now, comes after it on the same stream
-            done = False
-            if self.host_gather:
-                # the host reads the rows itself: the tag step of this batch is over (its counters are on
-                # the host), and every write-back of earlier batches has reached host memory (the
-                # previous batch's data movement is over)
-                if g == 0:
-                    ev_tags.synchronize()
-                    if self._ev_prev_ready is not None:
-                        self._ev_prev_ready.synchronize()
-                    if wait_bwd:
-                        prev_bwd.synchronize()
-                n_miss = int(self.host_counters[ctx][g][mb.COUNTER_NAMES.index("inserted")])
-                done = self.m.cache_fetch_via_host(g, n_miss, self.copy, s, ctx,
-                                                   mark=(lambda name, s=s: self._mark(name, t, s)) if self.record_timeline else None)
-            if not done:
-                self.m.cache_fetch(g, stream=s, ctx=ctx)
-            self._mark(f"placed{g}", t, s)
-            self.m.cache_writeback(g, stream=s, ctx=ctx)
-            self._mark(f"move{g}_end", t, s)
-            e = torch.cuda.Event()
-            e.record(s)
-            ends.append(e)
-        # the repair of stale rows waits for the previous backward; on its own stream it does not hold
-        # up the next batch's data movement
+    def _move_cache(self, t, g, via_host):
+        """Data path of batch t for cache g on its move stream: fetch, then write back, in stream order (the
+        next batch's fetch of this cache, which may miss a row written back now, follows on the same stream)."""
+        s, ctx = self.moves[g], t % DeviceModel.N_CTX
+        s.wait_event(self.ev_tags[t])
+        self._delay(s)
+        self._mark(f"move{g}_begin", t, s)
+        done = False
+        if via_host:
+            # the host reads the rows itself: the tag step of this batch is over (its counters are on the
+            # host) and this cache's write-backs of earlier batches have reached host memory
+            self.ev_tags[t].synchronize()
+            if t > 0:
+                self.ev_moved[t - 1][g].synchronize()
+            n_miss = int(self._host_counters[t, g, mb.COUNTER_NAMES.index("inserted")])
+            done = self.m.cache_fetch_via_host(
+                g, n_miss, self.copy, s, ctx,
+                mark=(lambda name, s=s: self._mark(name, t, s)) if self.record_timeline else None)
+        if not done:
+            self.m.cache_fetch(g, stream=s, ctx=ctx)
+        self._mark(f"placed{g}", t, s)
+        self.m.cache_writeback(g, stream=s, ctx=ctx)
+        self._mark(f"move{g}_end", t, s)
+        self.ev_moved[t][g].record(s)
+
+    def _finish_move(self, t):
+        """After the data movement of batch t: repair the rows that overflowed in the batches whose backward may
+        have run after their copy was taken, then batch t is ready to train."""
         s = self.fix
-        for e in ends:
+        for e in self.ev_moved[t]:
             s.wait_event(e)
-        if refetch:
-            s.wait_event(prev_bwd)
+        if self.pipelined and t >= 1:
+            s.wait_event(self.ev_bwd[t - 1])
+            self._delay(s)
             self._mark("refetch_begin", t, s)
-            self.m.cache_refetch((t - 1) % DeviceModel.N_CTX, placed_step=self._first_step + t, stream=s)
+            for k in range(1, self.m.lock_depth + 1):
+                if t - k >= 0:
+                    self.m.cache_refetch((t - k) % DeviceModel.N_CTX, placed_step=self._first_step + t, stream=s)
         self._mark("ready", t, s)
-        ev_ready.record(s)
-        self._ev_prev_ready = ev_ready
+        self.ev_ready[t].record(s)
 
-    def _counters(self, t, ev_tags) -> int:
-        ev_tags.synchronize()                        # counters of batch t are on the host
-        cnt = self.host_counters[t % DeviceModel.N_CTX].numpy().copy()
-        self.history.append(cnt)
-        return int(cnt[:, mb.COUNTER_NAMES.index("overflow")].max())
+    def _move(self, t):
+        for g in range(len(self.moves)):
+            self._move_cache(t, g, self.host_gather)
+        self._finish_move(t)
+
+    # ------------------------------------------------------------------ worker thread (host_gather, pipelined)
+    def _worker(self):
+        try:
+            torch.cuda.set_device(self.dev)
+            while True:
+                t = self._jobs.get()
+                if t is None:
+                    return
+                for g in range(len(self.moves)):
+                    self._move_cache(t, g, True)
+                if t >= 1:
+                    self._bwd_recorded[t - 1].wait()            # the repair waits for that event on the device
+                self._finish_move(t)
+                self._ready_recorded[t].set()
+        except BaseException as e:                              # surface the failure in the launching thread
+            self._worker_error = e
+            for f in self._ready_recorded:
+                f.set()
+
+    def _wait_ready_recorded(self, t):
+        if self._thread is not None:
+            self._ready_recorded[t].wait()
+            if self._worker_error is not None:
+                raise self._worker_error
 
     def run(self, batches, grads, out: Optional[torch.Tensor] = None,
-            on_step: Optional[Callable[[int], None]] = None, first_step: int = 0) -> None:
-        """Train on `batches` = [(indices_dev, offsets_dev, offsets_host)], `grads` = [grad_out_dev]."""
+            on_step: Optional[Callable[[int], None]] = None, first_step: int = 0,
+            after_backward: Optional[Callable[[int], None]] = None) -> None:
+        """Train on `batches` = [(indices_dev, offsets_dev, offsets_host)], `grads` = [grad_out_dev].
+        after_backward(t) is called when batch t's backward has been enqueued and before any later work that
+        may reuse its context; on_step(t) at the end of iteration t."""
         m = self.m
         K = len(batches)
         if K == 0:
             return
         self._first_step = first_step
-        ev_tags = [torch.cuda.Event() for _ in range(K)]
-        ev_ready = [torch.cuda.Event() for _ in range(K)]
-        ev_bwd = [torch.cuda.Event() for _ in range(K)]
+        n_c = len(m.caches)
+        self.ev_tags = [torch.cuda.Event() for _ in range(K)]
+        self.ev_ready = [torch.cuda.Event() for _ in range(K)]
+        self.ev_bwd = [torch.cuda.Event() for _ in range(K)]
+        self.ev_moved = [[torch.cuda.Event() for _ in range(n_c)] for _ in range(K)]
+        self._host_counters = torch.zeros((K, n_c, mb.NUM_COUNTERS), dtype=torch.int64).pin_memory()
+        self._thread = None
+        self._worker_error = None
         if out is None:
             out = torch.empty((m.spec.batch, m.spec.total_dim), dtype=torch.float32, device=self.dev)
+
+        def train(t):
+            idx, off, _ = batches[t]
+            ctx = t % DeviceModel.N_CTX
+            self._mark("fwd_begin", t, self.main)
+            m.forward(idx, off, idx.numel(), out=out, stream=self.main, ctx=ctx)
+            self._mark("fwd_end", t, self.main)
+            m.backward(idx, off, idx.numel(), grads[t], stream=self.main, ctx=ctx)
+            self._mark("bwd_end", t, self.main)
+            if after_backward is not None:
+                after_backward(t)
+
         if not self.pipelined:
             for t in range(K):
-                idx, off, _ = batches[t]
-                self._lookup(t, first_step + t, batches[t], ev_tags[t], None)
-                self._move(t, ev_tags[t], ev_ready[t], 0, None)
-                m.forward(idx, off, idx.numel(), out=out, stream=self.main, ctx=t % DeviceModel.N_CTX)
-                m.backward(idx, off, idx.numel(), grads[t], stream=self.main, ctx=t % DeviceModel.N_CTX)
-                self._counters(t, ev_tags[t])
+                self._lookup(t, batches[t])
+                self._move(t)
+                train(t)
                 if on_step is not None:
                     on_step(t)
+            torch.cuda.synchronize(self.dev)
+            self.history.extend(self._host_counters.numpy().copy())
             return
+
         # the side streams must see the inputs produced on the main stream
         start = torch.cuda.Event()
         start.record(self.main)
-        self.tag.wait_event(start)
-        for s in self.moves + [self.fix]:
+        for s in [self.tag, self.fix, self.copy] + self.moves:
             s.wait_event(start)
-        overflow = {}
-        self._lookup(0, first_step, batches[0], ev_tags[0], None)
-        self._move(0, ev_tags[0], ev_ready[0], 0, None)
-        overflow[0] = self._counters(0, ev_tags[0])
-        if K > 1:
-            self._lookup(1, first_step + 1, batches[1], ev_tags[1], None)
-        for t in range(K):
-            idx, off, _ = batches[t]
-            self.main.wait_event(ev_ready[t])
-            self._mark("fwd_begin", t, self.main)
-            m.forward(idx, off, idx.numel(), out=out, stream=self.main, ctx=t % DeviceModel.N_CTX)
-            self._mark("fwd_end", t, self.main)
-            m.backward(idx, off, idx.numel(), grads[t], stream=self.main, ctx=t % DeviceModel.N_CTX)
-            self._mark("bwd_end", t, self.main)
-            ev_bwd[t].record(self.main)
-            if t + 2 < K:
-                # the tag step of batch t+2 may evict rows stamped before t+2-lock_depth: the backward
-                # of the last such batch must be over (with lock_depth 1 that is batch t, with 2 batch
-                # t-1); the context it writes was last used by batch t-1.  Enqueued before the data movement
-                # of batch t+1, whose host part (counters, row gather) blocks this thread
-                last = min(t, t + 1 - m.lock_depth)
-                # it rewrites the context of batch t-1, whose overflow list and counters the repair step
-                # inside the data movement of batch t still reads: after that
-                self.tag.wait_event(ev_ready[t])
-                self._lookup(t + 2, first_step + t + 2, batches[t + 2], ev_tags[t + 2],
-                             ev_bwd[last] if last >= 0 else None)
-            if t + 1 < K:
-                overflow[t + 1] = self._counters(t + 1, ev_tags[t + 1])
-                if t >= 1:
-                    # a row that overflowed in batch t-1 (updated in host memory by its backward) and is
-                    # placed only now is fetched from host memory: after that backward
-                    for s in self.moves:
-                        s.wait_event(ev_bwd[t - 1])
-                    if self.host_gather:
-                        ev_bwd[t - 1].synchronize()
-                self._move(t + 1, ev_tags[t + 1], ev_ready[t + 1], overflow[t], ev_bwd[t])
-            if on_step is not None:
-                on_step(t)
-        self.main.wait_stream(self.tag)
-        for s in self.moves + [self.fix]:
+        if self.host_gather:
+            self._jobs: "queue.Queue" = queue.Queue()
+            self._ready_recorded = [threading.Event() for _ in range(K)]
+            self._bwd_recorded = [threading.Event() for _ in range(K)]
+            self._thread = threading.Thread(target=self._worker, daemon=True)
+            self._thread.start()
+
+        def move(t):
+            if self._thread is not None:
+                self._jobs.put(t)          # ev_tags[t] has been recorded by this thread already
+            else:
+                self._move(t)
+
+        try:
+            self._lookup(0, batches[0])
+            move(0)
+            if K > 1:
+                self._lookup(1, batches[1])
+            for t in range(K):
+                self._wait_ready_recorded(t)
+                self.main.wait_event(self.ev_ready[t])
+                train(t)
+                self.ev_bwd[t].record(self.main)
+                if self._thread is not None:
+                    self._bwd_recorded[t].set()
+                if t + 1 < K:
+                    move(t + 1)
+                if t + 2 < K:
+                    self._lookup(t + 2, batches[t + 2])
+                if on_step is not None:
+                    on_step(t)
+        finally:
+            if self._thread is not None:
+                for f in self._bwd_recorded:       # on an error in this thread: do not leave the worker waiting
+                    f.set()
+                self._jobs.put(None)
+                self._thread.join()
+                self._thread = None
+        for s in [self.tag, self.fix, self.copy] + self.moves:
             self.main.wait_stream(s)
+        torch.cuda.synchronize(self.dev)
+        self.history.extend(self._host_counters.numpy().copy())

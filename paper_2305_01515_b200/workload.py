@@ -238,37 +238,58 @@ def bag_lengths(spec: ModelSpec, tab: TableSpec, rng: np.random.Generator) -> np
 class BatchStream:
     """Consecutive batches of one model; keeps the per-table history temporal reuse needs.
 
-    Batch k uses `default_rng([seed, k])`, so batch k of a stream is reproducible only as
-    part of the stream when reuse is on (it copies indices of earlier batches)."""
+    Table t of batch k draws from `default_rng([seed, 7919, k, t])`, so the tables of a batch are independent
+    of one another (large batches are generated by a few threads, with the same result) and batch k of a
+    stream is reproducible only as part of the stream when reuse is on (it copies indices of earlier batches)."""
+
+    PARALLEL_FROM = 2_000_000       # expected lookups per batch from which the tables are drawn by threads
 
     def __init__(self, spec: ModelSpec):
         self.spec = spec
         self.k = 0
         self.history: List[List[np.ndarray]] = []   # last `reuse_window` batches, per table
+        expected = spec.batch * sum(t.pooling for t in spec.tables)
+        self._pool = None
+        if expected >= self.PARALLEL_FROM and spec.T > 1:
+            from concurrent.futures import ThreadPoolExecutor
+            self._pool = ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1, spec.T))
+
+    def _table(self, t: int):
+        spec, tab = self.spec, self.spec.tables[t]
+        rng = np.random.default_rng([spec.seed, 7919, self.k, t])
+        lens = bag_lengths(spec, tab, rng)
+        n = int(lens.sum())
+        idx = draw_rows(tab, rng, n)
+        if spec.reuse_prob > 0.0 and self.history:
+            parts = [h[t] for h in self.history]
+            size = sum(p.size for p in parts)
+            if size:
+                reuse = rng.random(n) < spec.reuse_prob
+                pick = rng.integers(0, size, size=n)
+                # index `pick` of the previous batches' indices laid end to end, oldest first
+                ends = np.cumsum([p.size for p in parts])
+                which = np.searchsorted(ends, pick, side="right")
+                old = np.empty(n, dtype=np.int64)
+                for j, p in enumerate(parts):
+                    sel = which == j
+                    if sel.any():
+                        old[sel] = p[pick[sel] - (ends[j] - p.size)]
+                idx = np.where(reuse, old, idx)
+        return idx, lens
 
     def next(self):
         spec = self.spec
-        rng = np.random.default_rng([spec.seed, 7919, self.k])
-        idx_parts, len_parts, per_table = [], [], []
-        for t, tab in enumerate(spec.tables):
-            lens = bag_lengths(spec, tab, rng)
-            n = int(lens.sum())
-            idx = draw_rows(tab, rng, n)
-            if spec.reuse_prob > 0.0 and self.history:
-                pool = np.concatenate([h[t] for h in self.history])
-                if pool.size:
-                    reuse = rng.random(n) < spec.reuse_prob
-                    pick = rng.integers(0, pool.size, size=n)
-                    idx = np.where(reuse, pool[pick], idx)
-            idx_parts.append(idx)
-            len_parts.append(lens)
-            per_table.append(idx)
+        if self._pool is not None:
+            res = list(self._pool.map(self._table, range(spec.T)))
+        else:
+            res = [self._table(t) for t in range(spec.T)]
+        per_table = [r[0] for r in res]
         if spec.reuse_window > 0:
             self.history.append(per_table)
             if len(self.history) > spec.reuse_window:
                 self.history.pop(0)
-        indices = np.concatenate(idx_parts).astype(np.int64) if idx_parts else np.zeros(0, np.int64)
-        lens = np.concatenate(len_parts)
+        indices = np.concatenate(per_table).astype(np.int64) if per_table else np.zeros(0, np.int64)
+        lens = np.concatenate([r[1] for r in res])
         offsets = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
         self.k += 1
         return indices, offsets
@@ -329,6 +350,9 @@ def config3(seed: int = 0, row_scale: float = 1.0, batch: int = 16384, tables: i
     anti-correlated with size, Zipf 0.8-1.3, fp16, batch 16384, all in HBM."""
     rng = np.random.default_rng([seed, 3])
     return ModelSpec("cfg3", _hetero_tables(rng, tables, row_scale), FP16, batch, "poisson", seed=seed)
+
+
+BENCH_CFG4_BUDGET_GB = 20.0     # HBM budget bench.py runs configuration 4 at (80 GB of host rows)
 
 
 def config4(seed: int = 0, hbm_budget_gb: Optional[float] = None, batch: int = 16384,

@@ -45,3 +45,34 @@ def test_reference_arm_prints_one_line_on_rank_zero_only():
     assert line["impl"] == "reference" and line["unit"] == "lookups/s" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["value"] == line["value"]
+
+
+def test_profiler_traffic_record_is_dropped_when_the_kernel_source_changes(tmp_path, monkeypatch):
+    import bench
+
+    files = ["tbe_backward.cu", "common.cuh"]
+    rec = {"reduce_chunks": {"workload": "cfg2", "dram_bytes_per_lookup": 168.5, "source_files": files,
+                             "source_sha256": bench.kernel_source_hash(files), "capture": "test"}}
+    path = tmp_path / "traffic.json"
+    path.write_text(json.dumps(rec))
+    monkeypatch.setattr(bench, "TRAFFIC_FILE", str(path))
+    assert bench.ncu_traffic_per_lookup("reduce_chunks", "cfg2")[0] == 168.5
+    assert bench.ncu_traffic_per_lookup("reduce_chunks", "cfg3")[0] is None          # another workload
+    assert bench.ncu_traffic_per_lookup("tbe_forward_kernel", "cfg2")[0] is None     # no record
+    rec["reduce_chunks"]["source_sha256"] = "0" * 64                                 # the kernel changed since
+    path.write_text(json.dumps(rec))
+    assert bench.ncu_traffic_per_lookup("reduce_chunks", "cfg2")[0] is None
+
+
+def test_every_workload_has_a_spec_for_both_arms():
+    import argparse
+
+    import bench
+
+    a = argparse.Namespace(tables=0, budget_gb=0.01, warmup=1, steps=1, rows=1000, batch=8, pooling=3, alpha=1.0,
+                           cache_fraction=0.1)
+    for name, cached in (("cfg1", False), ("cfg2", False), ("cfg3", False), ("cfg4", True), ("cfg5", True)):
+        spec = bench.make_spec(name, 0, a)
+        assert spec.name == name and spec.cached == cached
+    f = bench.fractions(4000.0, 6547.2)
+    assert abs(f["frac_of_measured"] - 4000.0 / 6547.2) < 1e-12 and abs(f["frac_of_nominal"] - 0.5) < 1e-12

@@ -254,11 +254,38 @@ def test_backward_in_two_calls_matches_one_call():
 @pytest.mark.parametrize("rows,pool,B", [
     ([250, 200, 256, 100, 255], [7, 0.02, 30, 3, 12], 257),          # 1 pass per table instead of 2; a nearly empty table
     ([60000, 65536, 40000], [40, 25, 33], 600),                      # 2 passes instead of 3; several tiles per table
+    ([200, 70000, 3, 131072], [30, 25, 9, 20], 700),                 # 17 bits: two passes of 9; tables 0 and 2 have no bit left in the second
+    ([1 << 20, 1000, 1 << 18, 5], [30, 40, 20, 3], 900),             # 20 bits: two passes of 10; table 1 is only copied in the second
+    ([3 << 20, 900000], [35, 30], 1500),                             # 22 bits: two passes of 11
 ])
 def test_tables_sorted_separately(rows, pool, B):
     """Table sets for which the lookups of each table are sorted on their own (fewer digit passes)."""
-    spec = custom_spec(rows, [64] * len(rows), B, wl.FP16, pool, [1.1] * len(rows), seed=5)
+    spec = custom_spec(rows, [8 if max(rows) > 200000 else 64] * len(rows), B, wl.FP16, pool, [1.1] * len(rows), seed=5)
     _run_steps(spec, n_steps=2)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("rows", [[100_000_000], [1_200_000_000], [900_000_000, 3_000_000_000]])
+def test_unsegmented_sort_of_wide_row_ids(rows):
+    """Row ids of 27, 31 and 32 bits in one sort (three passes of 9, 11 and 11 bits): the distinct rows of the
+    batch are compared with numpy's; the tables themselves are never allocated (sort only)."""
+    spec = custom_spec(rows, [8] * len(rows), 500, wl.FP16, [40] * len(rows), [0.9] * len(rows), seed=6)
+    idx, off = wl.gen_batch(spec, 0)
+    N = len(idx)
+    dummy = torch.zeros(64, dtype=torch.float16, device="cuda:0")
+    mom = torch.zeros(1, dtype=torch.float32, device="cuda:0")
+    tables = mb.tables_create(spec.dtype, spec.rows, spec.dims, spec.weight_offset[:-1], None, dummy, None, mom)
+    wsb = mb.tbe_backward_workspace_bytes(tables, spec.batch, N)
+    ws = torch.empty(wsb, dtype=torch.uint8, device="cuda:0")
+    uniq = torch.full((N,), -1, dtype=torch.int64, device="cuda:0")
+    nu = torch.zeros(1, dtype=torch.int64, device="cuda:0")
+    mb.tbe_backward_sort(tables, spec.batch, to_dev(idx), to_dev(off), N, ws, wsb, uniq, nu)
+    torch.cuda.synchronize()
+    lin = np.concatenate([spec.row_offset[t] + idx[off[t * spec.batch]:off[(t + 1) * spec.batch]] for t in range(spec.T)])
+    ref = np.unique(lin)
+    assert int(nu.item()) == len(ref)
+    np.testing.assert_array_equal(uniq[:len(ref)].cpu().numpy(), ref)
+    tables.destroy()
 
 
 @pytest.mark.gpu

@@ -28,14 +28,15 @@ class GpuCache:
         self.ws = torch.empty(self.wsb, dtype=torch.uint8, device=d)
         self.n = S * 32
 
-    def lookup_insert(self, keys, step):
+    def lookup_insert(self, keys, step, list_capacity=None):
         N = len(keys)
         mb.cache_lookup_insert(self.c, to_dev(keys) if N else None, N, step, self.slot, self.mk, self.ms, self.ek,
-                               self.es, self.ed, self.cap, self.cnt, self.ws, self.wsb, overflow_keys=self.ok)
+                               self.es, self.ed, self.cap if list_capacity is None else list_capacity, self.cnt,
+                               self.ws, self.wsb, overflow_keys=self.ok)
         torch.cuda.synchronize()
         cnt = dict(zip(mb.COUNTER_NAMES, self.cnt.cpu().tolist()))
         nm, ne = cnt["inserted"], cnt["evicted"]
-        self.overflow_keys = np.sort(self.ok[:cnt["overflow"]].cpu().numpy())
+        self.overflow_keys = np.sort(self.ok[:min(cnt["overflow"], self.cap if list_capacity is None else list_capacity)].cpu().numpy())
         return dict(slot_of_lookup=self.slot[:N].cpu().numpy(), miss_keys=self.mk[:nm].cpu().numpy(),
                     miss_slots=self.ms[:nm].cpu().numpy(), evict_keys=self.ek[:ne].cpu().numpy(),
                     evict_slots=self.es[:ne].cpu().numpy(), evict_dirty=self.ed[:ne].cpu().numpy(), counters=cnt)
@@ -84,6 +85,78 @@ def test_tag_path_matches_oracle_bit_for_bit(S, lock, policy, universe):
         np.testing.assert_array_equal(fr, o.freq.reshape(-1))
         np.testing.assert_array_equal(dirty, o.dirty)
     o.close()
+    g.c.destroy()
+
+
+def _scattered_keys(rng, n, universe):
+    """Skewed keys spread over the whole key range (every digit of the sort sees many values)."""
+    hot = rng.zipf(1.15, n).astype(np.uint64)
+    spread = (hot * np.uint64(0x9E3779B97F4A7C15) >> np.uint64(11)) % np.uint64(universe)
+    fresh = rng.integers(0, universe, n).astype(np.uint64)
+    return np.where(rng.random(n) < 0.8, spread, fresh).astype(np.int64)
+
+
+@pytest.mark.parametrize("S,universe,cap", [(300, 1 << 20, 60000), (5000, 3 << 20, 60000), (1, 131072, 60000),
+                                            (70000, 100_000_000, 400000), (1 << 17, 1_000_000_000, 60000),
+                                            (2500, (1 << 32) - 2, 300000), (64, 500, 60000)])
+def test_tag_path_wide_keys_and_set_counts(S, universe, cap):
+    """Key ranges of 9 to 32 bits and set counts of 0 to 17 bits: every digit width and pass count of the
+    key sort and of the sort by set (one pass of 8 or 9 bits, two of 7 to 11, three of 9 to 11)."""
+    rng = np.random.default_rng(S % 1000 + universe % 1000)
+    g = GpuCache(S, universe, 8, wl.FP16, 0, 1, cap)
+    o = oracle.Cache(S, 32, 8, wl.FP16, 0, 1, with_data=False)
+    for step in range(6):
+        n = int(rng.integers(cap // 2, cap))
+        keys = _scattered_keys(rng, n, universe)
+        res = g.lookup_insert(keys, step)
+        ref = o.lookup_insert(keys, step)
+        _compare(res, ref)
+        np.testing.assert_array_equal(g.overflow_keys, np.unique(keys[ref["slot_of_lookup"] < 0]))
+    tags, ts, fr, dirty = g.state()
+    np.testing.assert_array_equal(tags, o.tags.reshape(-1))
+    np.testing.assert_array_equal(ts, o.ts.reshape(-1))
+    assert g.c.status() == 0
+    o.close()
+    g.c.destroy()
+
+
+@pytest.mark.parametrize("policy", [0, 1])
+def test_full_miss_list_is_served_as_overflow(policy):
+    """list_capacity smaller than the placements of a call: the surplus keys are not inserted (slot -1), their
+    victims keep their ways, counters / lists / state equal the oracle's, and the status word says so."""
+    S, universe, cap = 40, 30000, 8000
+    rng = np.random.default_rng(5 + policy)
+    g = GpuCache(S, universe, 64, wl.FP16, policy, 1, cap)
+    o = oracle.Cache(S, 32, 64, wl.FP16, policy, 1, with_data=False)
+    twin = oracle.Cache(S, 32, 64, wl.FP16, policy, 1, with_data=False)
+    cut_calls = 0
+    for step in range(12):
+        keys = _scattered_keys(rng, int(rng.integers(2000, cap)), universe)
+        limit = int(rng.choice([0, 1, 7, 200, 255, 256, 257, 600, cap]))
+        # what the call would place without a limit (on a copy of the oracle's state)
+        twin.tags[:], twin.ts[:], twin.freq[:], twin.dirty[:] = o.tags, o.ts, o.freq, o.dirty
+        wanted = twin.lookup_insert(keys, step)["counters"]["inserted"]
+        res = g.lookup_insert(keys, step, list_capacity=limit)
+        ref = o.lookup_insert(keys, step, list_capacity=limit)
+        _compare(res, ref)
+        assert res["counters"]["inserted"] == min(wanted, limit)
+        if res["counters"]["overflow"] <= limit:           # the overflow list shares the capacity in this entry point
+            np.testing.assert_array_equal(g.overflow_keys, np.unique(keys[ref["slot_of_lookup"] < 0]))
+        status = g.c.status()
+        assert (status & 4 != 0) == (wanted > limit), (status, wanted, limit)
+        cut_calls += 1 if status & 4 else 0
+        sl = np.unique(ref["slot_of_lookup"][ref["slot_of_lookup"] >= 0])[::2]
+        if len(sl):
+            o.dirty[sl] = 1
+            dirty_t = as_tensor(g.c.dirty_ptr, g.n, torch.uint8)
+            dirty_t[to_dev(sl.astype(np.int64))] = torch.ones(len(sl), dtype=torch.uint8, device="cuda:0")
+        tags, ts, fr, dirty = g.state()
+        np.testing.assert_array_equal(tags, o.tags.reshape(-1))
+        np.testing.assert_array_equal(ts, o.ts.reshape(-1))
+        np.testing.assert_array_equal(fr, o.freq.reshape(-1))
+        np.testing.assert_array_equal(dirty, o.dirty)
+    assert cut_calls >= 4
+    o.close(); twin.close()
     g.c.destroy()
 
 

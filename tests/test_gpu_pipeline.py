@@ -65,3 +65,39 @@ def test_pipelined_equals_sequential_and_oracle_tags(frac, lock):
         oc.close()
     if frac < 0.01:
         assert overflow > 0
+
+
+@pytest.mark.parametrize("host_gather", [False, True])
+def test_overflow_repair_survives_slow_side_streams(host_gather):
+    """Lock depth 2, a cache much smaller than a batch (rows overflow in every batch) and move / repair
+    streams that idle for about a millisecond before each piece of work, so that the tag step two batches
+    ahead and the training run as far ahead of them as the events allow: the result must still equal the
+    sequential run bit for bit (the overflow lists stay intact until their repair has read them)."""
+    rows, dims = [20000, 9000, 4000, 12000], [64, 64, 128, 128]
+    spec = custom_spec(rows, dims, 256, wl.FP16, [8, 12, 20, 5], [1.05, 0.9, 1.2, 1.0], seed=78)
+    spec.cached = True
+    spec.cache_fraction = 0.004
+    spec.reuse_prob, spec.reuse_window = 0.7, 4
+    stream = wl.BatchStream(spec)
+    K = 12
+    host_batches = [stream.next() for _ in range(K)]
+    grads = [to_dev(wl.gen_grad(spec, k)) for k in range(K)]
+    W0 = wl.all_weights_numpy(spec)
+    results = []
+    for pipelined, delay in ((False, 0), (True, 2_000_000), (True, 0)):
+        m = DeviceModel(spec, weights=W0, lock_depth=2)
+        m.reserve(max(len(b[0]) for b in host_batches))
+        batches = [(to_dev(i), to_dev(o), o) for i, o in host_batches]
+        tr = CachedTrainer(m, pipelined=pipelined, host_gather=host_gather)
+        tr.debug_delay_cycles = delay
+        tr.run(batches, grads)
+        m.flush()
+        torch.cuda.synchronize()
+        results.append((m.weights_numpy(), m.momentum.cpu().numpy(), np.stack(tr.history)))
+        m.close()
+    Wa, ma, ha = results[0]
+    assert ha[:, :, mb.COUNTER_NAMES.index("overflow")].sum() > 100
+    for Wx, mx, hx in results[1:]:
+        assert (ha == hx).all()
+        assert (Wa.view(np.uint16) == Wx.view(np.uint16)).all()
+        assert (ma.view(np.uint32) == mx.view(np.uint32)).all()
