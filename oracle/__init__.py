@@ -19,6 +19,10 @@ _SRC = os.path.join(_HERE, "mtrains_oracle.c")
 _LIB = os.path.join(_HERE, "libmtrains_oracle.so")
 
 NCOUNTERS = 10
+NCOUNTERS2 = 20
+COUNTER_NAMES2 = ("lookups", "unique", "hit_lookups", "miss_lookups", "unique_hits", "unique_misses", "inserted",
+                  "evicted", "evicted_dirty", "overflow", "l2_hit_lookups", "l2_unique_hits", "promoted", "demoted",
+                  "l2_evicted", "l2_evicted_dirty", "l2_bypass", "l2_bypass_dirty", "l2_dropped", "l2_dropped_dirty")
 COUNTER_NAMES = ("lookups", "unique", "hit_lookups", "miss_lookups", "unique_hits",
                  "unique_misses", "inserted", "evicted", "evicted_dirty", "overflow")
 
@@ -47,6 +51,7 @@ def lib():
         _lib.orc_cache_create.restype = C.c_void_p
         _lib.orc_cache_lookup_insert.restype = C.c_int64
         _lib.orc_cache_flush.restype = C.c_int64
+        _lib.orc_cache2_lookup_insert.restype = C.c_int64
         for name in ("orc_cache_tags", "orc_cache_ts", "orc_cache_freq", "orc_cache_dirty",
                      "orc_cache_data"):
             getattr(_lib, name).restype = C.c_void_p
@@ -229,3 +234,45 @@ class Cache:
 
     def flush(self, host: np.ndarray) -> int:
         return int(lib().orc_cache_flush(self._h, _p(host)))
+
+
+class Cache2:
+    """Two-level exclusive cache of the oracle: `l1` and `l2` are Cache objects of one row shape."""
+
+    def __init__(self, l1: Cache, l2: Cache):
+        assert l1.dim == l2.dim and l1.dtype == l2.dtype
+        self.l1, self.l2 = l1, l2
+
+    def lookup_insert(self, keys, step: int):
+        keys = _i64(keys)
+        N = len(keys)
+        cap = max(N, 1)
+        slot = np.full(cap, -1, dtype=np.int32)
+        fk = np.zeros(cap, np.int64); fs = np.zeros(cap, np.int32); fsrc = np.zeros(cap, np.int32)
+        e1k = np.zeros(cap, np.int64); e1s = np.zeros(cap, np.int32); e1d = np.zeros(cap, np.uint8)
+        e1dst = np.zeros(cap, np.int32)
+        e2k = np.zeros(cap, np.int64); e2s = np.zeros(cap, np.int32); e2d = np.zeros(cap, np.uint8)
+        dk = np.zeros(cap, np.int64); ds = np.zeros(cap, np.int32); dd = np.zeros(cap, np.uint8)
+        cnt = np.zeros(NCOUNTERS2, np.int64)
+        lib().orc_cache2_lookup_insert(self.l1._h, self.l2._h, _p(keys), C.c_int64(N), C.c_int64(step), _p(slot),
+                                       _p(fk), _p(fs), _p(fsrc), _p(e1k), _p(e1s), _p(e1d), _p(e1dst),
+                                       _p(e2k), _p(e2s), _p(e2d), _p(dk), _p(ds), _p(dd), _p(cnt))
+        c = dict(zip(COUNTER_NAMES2, (int(x) for x in cnt)))
+        nf, n1, n2, nd = c["inserted"], c["evicted"], c["l2_evicted"], c["l2_dropped"]
+        return dict(slot_of_lookup=slot[:N], fetch_keys=fk[:nf], fetch_slots=fs[:nf], fetch_src=fsrc[:nf],
+                    ev1_keys=e1k[:n1], ev1_slots=e1s[:n1], ev1_dirty=e1d[:n1], ev1_dst=e1dst[:n1],
+                    ev2_keys=e2k[:n2], ev2_slots=e2s[:n2], ev2_dirty=e2d[:n2],
+                    drop_keys=dk[:nd], drop_slots=ds[:nd], drop_dirty=dd[:nd], counters=c)
+
+    def move(self, store: np.ndarray, res) -> None:
+        """Data movement of one lookup_insert result between the two levels and the backing store."""
+        lib().orc_cache2_move(
+            self.l1._h, self.l2._h, _p(store), _p(res["fetch_keys"]), _p(res["fetch_slots"]), _p(res["fetch_src"]),
+            C.c_int64(len(res["fetch_keys"])), _p(res["ev1_keys"]), _p(res["ev1_slots"]), _p(res["ev1_dirty"]),
+            _p(res["ev1_dst"]), C.c_int64(len(res["ev1_keys"])), _p(res["ev2_keys"]), _p(res["ev2_slots"]),
+            _p(res["ev2_dirty"]), C.c_int64(len(res["ev2_keys"])), _p(res["drop_keys"]), _p(res["drop_slots"]),
+            _p(res["drop_dirty"]), C.c_int64(len(res["drop_keys"])))
+
+    def flush(self, store: np.ndarray) -> int:
+        """Every dirty row of either level goes to the store (a row is in one level only)."""
+        return self.l1.flush(store) + self.l2.flush(store)

@@ -18,13 +18,18 @@
  *     fetched rows and eviction of LRU rows back to the lower tier
  *   - prefetch invariant (a prefetched row is not evicted before its batch  Section 5.7
  *     trained), expressed as a lock window on timestamps
+ *   - two cache levels, exclusive, over a backing store: promotion of       Section 5.3.2,
+ *     second-level hits and fetched rows, demotion of first-level LRU rows,  Section 5.5.4
+ *     eviction of second-level LRU rows to the store
  *
  * Floating point: all sums and the optimizer step are evaluated in double precision and
  * rounded once to the storage type (fp32, or IEEE binary16 with round-to-nearest-even).
  *
  * Parity pins (tests/, CPU only): brute-force per-bag loops, torch embedding_bag, a
  * hand-worked Adagrad step, torch.optim.Adagrad for D = 1, a list-based LRU simulation,
- * cache invariants and cached-vs-uncached transparency.  The paper prints no worked
+ * cache invariants and cached-vs-uncached transparency; the two-level cache against the
+ * one-level cache (its first level decides identically), a list simulation of the second
+ * level, the exclusivity invariant and transparency.  The paper prints no worked
  * numeric example for this path, so no pin comes from a printed value:
  * parity unpinned against paper-printed values; pinned against definitions only.
  */
@@ -483,6 +488,243 @@ int64_t orc_cache_flush(orc_cache* c, void* host) {
             c->dirty[s] = 0; ++n;
         }
     return n;
+}
+
+/* ------------------------------------------------------------------ two-level exclusive cache */
+
+/* Two cache levels over a backing store (Section 5.3.2: a two-level exclusive cache, the faster
+ * memory as the first level; Section 5.5.4: both levels are looked up, first-level misses that
+ * hit the second level and rows fetched from the lowest tier are promoted to the first level,
+ * first-level LRU rows are evicted to the second level, second-level LRU rows back to the
+ * lowest tier).  Exclusive: a row is in at most one level.  Both levels are orc_cache objects.
+ *
+ * lookup_insert2(keys, step):
+ *  1. Every distinct key is probed in both levels (state before the call).
+ *  2. + 3. The first level is handled exactly like a one-level cache (orc_cache_lookup_insert):
+ *     hits are refreshed, the missing keys of a set take its evictable ways, victims go to the
+ *     first-level evict list, keys beyond the evictable ways are not inserted (slot -1, served
+ *     from the backing store).  Whether a key that misses the first level sits in the second
+ *     level makes no difference to these decisions; it only says where its row comes from:
+ *     fetch_src = its second-level slot, or -1 = the backing store.  A promoted row keeps the
+ *     dirty byte it had in the second level.
+ *  4. Every second-level hit leaves the second level (its way becomes free): it was promoted, or
+ *     it found no first-level way and is served from the backing store in this batch, in which
+ *     case it is listed in the drop list {key, slot, dirty} so that a dirty row is written to
+ *     the store first.
+ *  5. The first-level victims are inserted into the second level: grouped by second-level set
+ *     (ascending), ascending key inside a set, the k-th takes the set's k-th evictable way (free
+ *     ways, then ways with ts < step - lock_depth of the second level, ordered like first-level
+ *     candidates).  The inserted entry keeps the timestamp, use count and dirty byte it had in
+ *     the first level.  A second-level victim with a valid tag goes to the second-level evict list
+ *     {key, slot, dirty}.  ev1_dst = the second-level slot, or -1 when the set had no evictable
+ *     way left: that victim goes to the backing store directly.
+ * Lists: fetch {key, first-level slot, src} in (first-level set, key) order; ev1 {key, slot,
+ * dirty, dst} in the order of the one-level evict list; ev2 in (second-level set, key of the
+ * displacing row) order; drop in (first-level set, key) order.
+ * counters[0..9] as for one level (hits and misses of the first level), then
+ * 10 l2_hit_lookups, 11 l2_unique_hits, 12 promoted, 13 demoted, 14 l2_evicted,
+ * 15 l2_evicted_dirty, 16 l2_bypass, 17 l2_bypass_dirty, 18 l2_dropped, 19 l2_dropped_dirty. */
+#define ORC_NCOUNTERS2 20
+
+typedef struct { int64_t set; int64_t key; int64_t idx; } orc_demote;
+
+static int demote_cmp(const void* a, const void* b) {
+    const orc_demote* x = (const orc_demote*)a; const orc_demote* y = (const orc_demote*)b;
+    if (x->set != y->set) return x->set < y->set ? -1 : 1;
+    return x->key < y->key ? -1 : (x->key > y->key ? 1 : 0);
+}
+
+/* candidate ways of one set in eviction order; returns their number */
+static int32_t ordered_candidates(const orc_cache* c, int64_t set, int64_t step, int32_t* cand) {
+    int32_t nc = 0;
+    for (int32_t w = 0; w < c->ways; ++w)
+        if (c->tag[set * c->ways + w] == -1 || c->ts[set * c->ways + w] < step - c->lock_depth) cand[nc++] = w;
+    for (int32_t x = 1; x < nc; ++x) {
+        int32_t w = cand[x]; int32_t y = x - 1;
+        while (y >= 0) {
+            int64_t sa = set * c->ways + cand[y], sb = set * c->ways + w;
+            int before;
+            if (c->policy == 1 && c->freq[sa] != c->freq[sb]) before = c->freq[sa] < c->freq[sb];
+            else if (c->ts[sa] != c->ts[sb]) before = c->ts[sa] < c->ts[sb];
+            else before = cand[y] < w;
+            if (before) break;
+            cand[y + 1] = cand[y]; --y;
+        }
+        cand[y + 1] = w;
+    }
+    return nc;
+}
+
+int64_t orc_cache2_lookup_insert(orc_cache* l1, orc_cache* l2, const int64_t* keys, int64_t N, int64_t step,
+                                 int32_t* slot_of_lookup,
+                                 int64_t* fetch_keys, int32_t* fetch_slots, int32_t* fetch_src,
+                                 int64_t* ev1_keys, int32_t* ev1_slots, uint8_t* ev1_dirty, int32_t* ev1_dst,
+                                 int64_t* ev2_keys, int32_t* ev2_slots, uint8_t* ev2_dirty,
+                                 int64_t* drop_keys, int32_t* drop_slots, uint8_t* drop_dirty,
+                                 int64_t* counters) {
+    for (int k = 0; k < ORC_NCOUNTERS2; ++k) counters[k] = 0;
+    counters[0] = N;
+    if (N == 0) return 0;
+    int64_t* sorted = (int64_t*)malloc((size_t)N * sizeof(int64_t));
+    memcpy(sorted, keys, (size_t)N * sizeof(int64_t));
+    qsort(sorted, (size_t)N, sizeof(int64_t), i64_cmp);
+    orc_setkey* uq = (orc_setkey*)malloc((size_t)N * sizeof(orc_setkey));
+    int64_t* mult = (int64_t*)malloc((size_t)N * sizeof(int64_t));
+    int64_t U = 0;
+    for (int64_t i = 0; i < N; ++i) {
+        if (i == 0 || sorted[i] != sorted[i - 1]) {
+            uq[U].key = sorted[i]; uq[U].set = orc_cache_set_of(sorted[i], l1->S); uq[U].u = U;
+            mult[U] = 0; ++U;
+        }
+        ++mult[U - 1];
+    }
+    counters[1] = U;
+    /* step 1: probe both levels against the state before the call */
+    int64_t* slot_of_uniq = (int64_t*)malloc((size_t)U * sizeof(int64_t));
+    int64_t* l2slot_of_uniq = (int64_t*)malloc((size_t)U * sizeof(int64_t));
+    for (int64_t u = 0; u < U; ++u) {
+        int64_t w = find_way(l1, uq[u].set, uq[u].key);
+        l2slot_of_uniq[u] = -1;
+        if (w >= 0) {
+            slot_of_uniq[u] = uq[u].set * l1->ways + w;
+            counters[2] += mult[u]; counters[4] += 1;
+        } else {
+            slot_of_uniq[u] = -2;
+            counters[3] += mult[u]; counters[5] += 1;
+            int64_t set2 = orc_cache_set_of(uq[u].key, l2->S);
+            int64_t w2 = find_way(l2, set2, uq[u].key);
+            if (w2 >= 0) {
+                l2slot_of_uniq[u] = set2 * l2->ways + w2;
+                counters[10] += mult[u]; counters[11] += 1;
+            }
+        }
+    }
+    /* step 2: refresh first-level hits */
+    for (int64_t u = 0; u < U; ++u)
+        if (slot_of_uniq[u] >= 0) {
+            l1->ts[slot_of_uniq[u]] = step;
+            l1->freq[slot_of_uniq[u]] += mult[u];
+        }
+    /* step 3: first-level placement, set by set */
+    orc_setkey* ms = (orc_setkey*)malloc((size_t)U * sizeof(orc_setkey));
+    int64_t M = 0;
+    for (int64_t u = 0; u < U; ++u) if (slot_of_uniq[u] == -2) ms[M++] = uq[u];
+    qsort(ms, (size_t)M, sizeof(orc_setkey), setkey_cmp);
+    int64_t n_fetch = 0, n_ev1 = 0, n_ev2 = 0, n_drop = 0;
+    int64_t* ev1_ts = (int64_t*)malloc((size_t)(U + 1) * sizeof(int64_t));
+    int64_t* ev1_freq = (int64_t*)malloc((size_t)(U + 1) * sizeof(int64_t));
+    int32_t* cand = (int32_t*)malloc((size_t)(l1->ways > l2->ways ? l1->ways : l2->ways) * sizeof(int32_t));
+    for (int64_t a = 0; a < M;) {
+        int64_t z = a;
+        while (z < M && ms[z].set == ms[a].set) ++z;
+        int64_t set = ms[a].set;
+        int32_t nc = ordered_candidates(l1, set, step, cand);
+        for (int64_t k = a; k < z; ++k) {
+            int64_t key = ms[k].key, u = ms[k].u;
+            int64_t slot = -1;
+            if (k - a < nc) {
+                slot = set * l1->ways + cand[k - a];
+                if (l1->tag[slot] != -1) {
+                    ev1_keys[n_ev1] = l1->tag[slot]; ev1_slots[n_ev1] = (int32_t)slot;
+                    ev1_dirty[n_ev1] = l1->dirty[slot];
+                    ev1_ts[n_ev1] = l1->ts[slot]; ev1_freq[n_ev1] = l1->freq[slot];
+                    counters[7] += 1; counters[8] += l1->dirty[slot] ? 1 : 0;
+                    ++n_ev1;
+                }
+                l1->tag[slot] = key; l1->ts[slot] = step; l1->freq[slot] = mult[u];
+                l1->dirty[slot] = l2slot_of_uniq[u] >= 0 ? l2->dirty[l2slot_of_uniq[u]] : 0;
+                fetch_keys[n_fetch] = key; fetch_slots[n_fetch] = (int32_t)slot;
+                fetch_src[n_fetch] = (int32_t)l2slot_of_uniq[u]; ++n_fetch;
+                counters[6] += 1;
+                if (l2slot_of_uniq[u] >= 0) counters[12] += 1;
+            } else {
+                counters[9] += 1;
+                if (l2slot_of_uniq[u] >= 0) {
+                    drop_keys[n_drop] = key; drop_slots[n_drop] = (int32_t)l2slot_of_uniq[u];
+                    drop_dirty[n_drop] = l2->dirty[l2slot_of_uniq[u]];
+                    counters[18] += 1; counters[19] += l2->dirty[l2slot_of_uniq[u]] ? 1 : 0;
+                    ++n_drop;
+                }
+            }
+            slot_of_uniq[u] = slot;
+        }
+        a = z;
+    }
+    /* step 4: every second-level hit leaves the second level */
+    for (int64_t u = 0; u < U; ++u)
+        if (l2slot_of_uniq[u] >= 0) {
+            int64_t s2 = l2slot_of_uniq[u];
+            l2->tag[s2] = -1; l2->ts[s2] = -1; l2->freq[s2] = 0; l2->dirty[s2] = 0;
+        }
+    /* step 5: first-level victims into the second level */
+    orc_demote* dm = (orc_demote*)malloc((size_t)(n_ev1 + 1) * sizeof(orc_demote));
+    for (int64_t k = 0; k < n_ev1; ++k) {
+        dm[k].key = ev1_keys[k]; dm[k].set = orc_cache_set_of(ev1_keys[k], l2->S); dm[k].idx = k;
+    }
+    qsort(dm, (size_t)n_ev1, sizeof(orc_demote), demote_cmp);
+    for (int64_t a = 0; a < n_ev1;) {
+        int64_t z = a;
+        while (z < n_ev1 && dm[z].set == dm[a].set) ++z;
+        int64_t set = dm[a].set;
+        int32_t nc = ordered_candidates(l2, set, step, cand);
+        for (int64_t k = a; k < z; ++k) {
+            int64_t e = dm[k].idx;
+            if (k - a < nc) {
+                int64_t s2 = set * l2->ways + cand[k - a];
+                if (l2->tag[s2] != -1) {
+                    ev2_keys[n_ev2] = l2->tag[s2]; ev2_slots[n_ev2] = (int32_t)s2; ev2_dirty[n_ev2] = l2->dirty[s2];
+                    counters[14] += 1; counters[15] += l2->dirty[s2] ? 1 : 0;
+                    ++n_ev2;
+                }
+                l2->tag[s2] = dm[k].key; l2->ts[s2] = ev1_ts[e]; l2->freq[s2] = ev1_freq[e];
+                l2->dirty[s2] = ev1_dirty[e];
+                ev1_dst[e] = (int32_t)s2;
+                counters[13] += 1;
+            } else {
+                ev1_dst[e] = -1;
+                counters[16] += 1; counters[17] += ev1_dirty[e] ? 1 : 0;
+            }
+        }
+        a = z;
+    }
+    for (int64_t i = 0; i < N; ++i) {
+        int64_t lo = 0, hi = U;
+        while (lo < hi) { int64_t mid = (lo + hi) / 2; if (uq[mid].key < keys[i]) lo = mid + 1; else hi = mid; }
+        slot_of_lookup[i] = (int32_t)slot_of_uniq[lo];
+    }
+    free(dm); free(cand); free(ev1_freq); free(ev1_ts); free(ms); free(l2slot_of_uniq); free(slot_of_uniq);
+    free(mult); free(uq); free(sorted);
+    return U;
+}
+
+/* Data movement for one lookup_insert2 result (Section 5.5.4), in an order that never reads a
+ * slot after it was overwritten: second-level rows that leave for the store (victims and dropped
+ * hits, when dirty); the rows to be fetched are read (from their second-level slot or from the
+ * store); first-level victims move to their second-level slot, or to the store when they have
+ * none and are dirty; the fetched rows enter their first-level slots. */
+void orc_cache2_move(orc_cache* l1, orc_cache* l2, void* store,
+                     const int64_t* fetch_keys, const int32_t* fetch_slots, const int32_t* fetch_src, int64_t n_fetch,
+                     const int64_t* ev1_keys, const int32_t* ev1_slots, const uint8_t* ev1_dirty,
+                     const int32_t* ev1_dst, int64_t n_ev1,
+                     const int64_t* ev2_keys, const int32_t* ev2_slots, const uint8_t* ev2_dirty, int64_t n_ev2,
+                     const int64_t* drop_keys, const int32_t* drop_slots, const uint8_t* drop_dirty, int64_t n_drop) {
+    size_t rb = (size_t)l1->dim * (l1->dtype == ORC_FP32 ? 4 : 2);
+    char* d1 = (char*)l1->data; char* d2 = (char*)l2->data; char* st = (char*)store;
+    for (int64_t k = 0; k < n_ev2; ++k)
+        if (ev2_dirty[k]) memcpy(st + (size_t)ev2_keys[k] * rb, d2 + (size_t)ev2_slots[k] * rb, rb);
+    for (int64_t k = 0; k < n_drop; ++k)
+        if (drop_dirty[k]) memcpy(st + (size_t)drop_keys[k] * rb, d2 + (size_t)drop_slots[k] * rb, rb);
+    char* tmp = (char*)malloc((size_t)(n_fetch > 0 ? n_fetch : 1) * rb);
+    for (int64_t k = 0; k < n_fetch; ++k)
+        memcpy(tmp + (size_t)k * rb,
+               fetch_src[k] >= 0 ? d2 + (size_t)fetch_src[k] * rb : st + (size_t)fetch_keys[k] * rb, rb);
+    for (int64_t k = 0; k < n_ev1; ++k) {
+        if (ev1_dst[k] >= 0) memcpy(d2 + (size_t)ev1_dst[k] * rb, d1 + (size_t)ev1_slots[k] * rb, rb);
+        else if (ev1_dirty[k]) memcpy(st + (size_t)ev1_keys[k] * rb, d1 + (size_t)ev1_slots[k] * rb, rb);
+    }
+    for (int64_t k = 0; k < n_fetch; ++k)
+        memcpy(d1 + (size_t)fetch_slots[k] * rb, tmp + (size_t)k * rb, rb);
+    free(tmp);
 }
 
 /* ------------------------------------------------------------------ analytical models */

@@ -21,6 +21,9 @@ class ListCache:
         self.sets = [[[w, -1, -1, 0, 0] for w in range(ways)] for _ in range(S)]
 
     def step(self, keys, step, capacity=None):
+        import copy
+        self.prev_sets = copy.deepcopy(self.sets)                    # state before the call
+        self.prev_resident = {e[1] for s in self.sets for e in s if e[1] >= 0}
         uniq = sorted(set(int(k) for k in keys))
         times = {}
         for k in keys:
