@@ -67,6 +67,22 @@ enum {
   MTS_CNT_OVERFLOW = 9       /* distinct missing keys that found no evictable way */
 };
 
+/* Counter block of the two-level cache (mts_cache2_lookup_insert): entries 0..9 are the counters above
+ * for the first level, then: */
+#define MTS_NUM_COUNTERS2 20
+enum {
+  MTS_CNT2_L2_HIT_LOOKUPS = 10,   /* lookups that missed the first level and hit the second */
+  MTS_CNT2_L2_UNIQUE_HITS = 11,
+  MTS_CNT2_PROMOTED = 12,         /* second-level hits inserted into the first level */
+  MTS_CNT2_DEMOTED = 13,          /* first-level victims inserted into the second level */
+  MTS_CNT2_L2_EVICTED = 14,       /* length of the second-level evict list */
+  MTS_CNT2_L2_EVICTED_DIRTY = 15,
+  MTS_CNT2_L2_BYPASS = 16,        /* first-level victims that found no second-level way (go to the store) */
+  MTS_CNT2_L2_BYPASS_DIRTY = 17,
+  MTS_CNT2_L2_DROPPED = 18,       /* second-level hits that found no first-level way (length of the drop list) */
+  MTS_CNT2_L2_DROPPED_DIRTY = 19
+};
+
 const char* mts_last_error_string(void);
 
 /* ---------------------------------------------------------------------------------------
@@ -336,6 +352,66 @@ int mts_cache_lookup_insert_tables(mts_cache* cache, const mts_tables* tables, i
                                    uint32_t* sorted_rows_out, uint32_t* sorted_pos_out,
                                    uint32_t* bag_of_lookup_out, void* workspace, size_t workspace_bytes,
                                    void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Two cache levels, exclusive (Section 5.3.2: the faster memory is the first level, the larger one the
+ * second, a row is in at most one of them; Section 5.5.4: both levels are looked up; first-level
+ * misses that hit the second level and rows fetched from the lowest tier are promoted to the first
+ * level; first-level LRU rows are evicted to the second level, second-level LRU rows to the lowest
+ * tier).  Here the first level is a cache in HBM (mts_cache_create), the second level keeps its rows in
+ * pinned host memory and its tags and states in HBM (mts_cache_create_host_level), and the lowest tier
+ * ("store") is a device-visible host buffer of all rows, row `key` at element key * dim.
+ * ------------------------------------------------------------------------------------- */
+
+/* A cache level whose rows live in caller-owned pinned, mapped host memory: host_rows_mapped is the
+ * device-visible address of [num_sets*32, dim] elements, 16-byte aligned; it must outlive the handle.
+ * Other arguments and errors as for mts_cache_create. */
+int mts_cache_create_host_level(mts_cache** out, int64_t num_sets, int64_t key_space, int32_t ways, int32_t dim,
+                                int32_t dtype, int32_t policy, int32_t lock_depth, void* host_rows_mapped);
+
+/* Tag/state lookup and replacement of both levels for one batch at time `step`:
+ *  1. every distinct key is probed in both levels (state before the call);
+ *  2. the first level is handled exactly as by mts_cache_lookup_insert (hits refreshed, missing keys take
+ *     the evictable ways of their set, victims go to the first-level evict list, keys beyond the evictable
+ *     ways get slot -1 and are served from the store); whether a key that misses the first level sits in
+ *     the second level only says where its row comes from: fetch_src[k] = its second-level slot, or -1 =
+ *     the store, for entry k of the fetch list {fetch_keys, fetch_slots} (the miss list of the first
+ *     level); a promoted row keeps the dirty byte it had in the second level;
+ *  3. every second-level hit leaves the second level: promoted, or — when it found no first-level way —
+ *     listed in the drop list {key, second-level slot, dirty} (no particular order) so that the data
+ *     movement writes a dirty row to the store before the batch reads it there;
+ *  4. the first-level victims are inserted into the second level: per second-level set in ascending key
+ *     order they take the set's evictable ways (free ways, then ways with timestamp < step - lock_depth of
+ *     the second level, in (timestamp, way) order [LFU: (count, timestamp, way)]) and keep the timestamp,
+ *     use count and dirty byte they had in the first level; ev1_dst[k] = second-level slot of entry k of
+ *     the first-level evict list {ev1_keys, ev1_slots, ev1_dirty}, or -1 = no way left, the row goes to the
+ *     store; displaced second-level rows form the second-level evict list {ev2_keys, ev2_slots, ev2_dirty}
+ *     in (second-level set, key of the displacing row) order.
+ * All lists are device arrays of list_capacity entries (the number of distinct keys is always enough);
+ * counters2: device int64 [MTS_NUM_COUNTERS2].  The two levels must have the same dim, dtype and
+ * key_space.  workspace: mts_cache2_workspace_bytes(l1, l2, N, list_capacity) bytes, 256-byte aligned.
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, CUDA. */
+size_t mts_cache2_workspace_bytes(const mts_cache* l1, const mts_cache* l2, int64_t N, int64_t list_capacity);
+int mts_cache2_lookup_insert(mts_cache* l1, mts_cache* l2, const int64_t* keys, int64_t N, int64_t step,
+                             int32_t* slot_of_lookup, int64_t* fetch_keys, int32_t* fetch_slots, int32_t* fetch_src,
+                             int64_t* ev1_keys, int32_t* ev1_slots, uint8_t* ev1_dirty, int32_t* ev1_dst,
+                             int64_t* ev2_keys, int32_t* ev2_slots, uint8_t* ev2_dirty, int64_t* drop_keys,
+                             int32_t* drop_slots, uint8_t* drop_dirty, int64_t list_capacity, int64_t* counters2,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Data movement for one mts_cache2_lookup_insert result (Section 5.5.4), in an order that never reads a slot
+ * after it was overwritten: dirty rows of the second-level evict list and of the drop list go to the store;
+ * the rows of the fetch list are collected in fetch_staging (device, [list_capacity, dim]) from their
+ * second-level slot or from the store; the first-level victims move to their second-level slot, or to the
+ * store when they have none and are dirty; the collected rows enter their first-level slots.  All on
+ * `stream`; list lengths are read from counters2 on the device.  mts_cache_flush on each level writes the
+ * dirty rows of that level to the store. */
+int mts_cache2_move(mts_cache* l1, mts_cache* l2, void* host_store_mapped, const int64_t* fetch_keys,
+                    const int32_t* fetch_slots, const int32_t* fetch_src, const int64_t* ev1_keys,
+                    const int32_t* ev1_slots, const uint8_t* ev1_dirty, const int32_t* ev1_dst,
+                    const int64_t* ev2_keys, const int32_t* ev2_slots, const uint8_t* ev2_dirty,
+                    const int64_t* drop_keys, const int32_t* drop_slots, const uint8_t* drop_dirty,
+                    int64_t list_capacity, const int64_t* counters2, void* fetch_staging, void* stream);
 
 /* Data movement for one lookup_insert result (Sections 5.5.3, 5.5.4): first the rows of dirty
  * victims are saved, slot -> evict_staging[k] (k = position in the evict list), then every

@@ -20,7 +20,10 @@ ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CAPACITY, ERR_CUDA, ERR_TIMEO
 DTYPE_FP32, DTYPE_FP16 = 0, 1
 POOL_SUM, POOL_MEAN = 0, 1
 POLICY_LRU, POLICY_LFU = 0, 1
-MAX_CACHES, CACHE_WAYS, NUM_COUNTERS = 8, 32, 10
+MAX_CACHES, CACHE_WAYS, NUM_COUNTERS, NUM_COUNTERS2 = 8, 32, 10, 20
+COUNTER_NAMES2 = ("lookups", "unique", "hit_lookups", "miss_lookups", "unique_hits", "unique_misses", "inserted",
+                  "evicted", "evicted_dirty", "overflow", "l2_hit_lookups", "l2_unique_hits", "promoted", "demoted",
+                  "l2_evicted", "l2_evicted_dirty", "l2_bypass", "l2_bypass_dirty", "l2_dropped", "l2_dropped_dirty")
 COUNTER_NAMES = ("lookups", "unique", "hit_lookups", "miss_lookups", "unique_hits",
                  "unique_misses", "inserted", "evicted", "evicted_dirty", "overflow")
 
@@ -32,7 +35,8 @@ EXPORTS = (
     "mts_tbe_forward_f16", "mts_tbe_backward_apply_f16",
     "mts_cache_create", "mts_cache_destroy", "mts_cache_status", "mts_cache_data", "mts_cache_dirty",
     "mts_linearize_keys", "mts_cache_workspace_bytes", "mts_cache_lookup_insert", "mts_cache_lookup_insert_tables",
-    "mts_tbe_backward_apply_presorted",
+    "mts_tbe_backward_apply_presorted", "mts_cache_create_host_level", "mts_cache2_workspace_bytes",
+    "mts_cache2_lookup_insert", "mts_cache2_move",
     "mts_cache_prefetch_misses", "mts_host_gather_rows", "mts_cache_place_fetched", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
     "mts_cache_export_state",
 )
@@ -105,6 +109,11 @@ def lib():
                                                      i64, vp, i64, vp, vp, vp, vp, vp, sz, vp]
         L.mts_tbe_backward_apply_presorted.argtypes = [vp, i32, vp, i64, i32, vp, i32, i64, f32, f32, vp, vp, vp, vp,
                                                        C.POINTER(vp), C.POINTER(vp), i32, vp, sz, vp]
+        L.mts_cache_create_host_level.argtypes = [C.POINTER(vp), i64, i64, i32, i32, i32, i32, i32, vp]
+        L.mts_cache2_workspace_bytes.restype = sz
+        L.mts_cache2_workspace_bytes.argtypes = [vp, vp, i64, i64]
+        L.mts_cache2_lookup_insert.argtypes = [vp, vp, vp, i64, i64] + [vp] * 14 + [i64, vp, vp, sz, vp]
+        L.mts_cache2_move.argtypes = [vp, vp, vp] + [vp] * 13 + [i64, vp, vp, vp]
         L.mts_cache_refetch_overflowed.argtypes = [vp, vp, vp, i64, vp, i64, vp]
         L.mts_cache_prefetch_misses.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.mts_cache_writeback_evicted.argtypes = [vp, vp, vp, vp, i64, vp, vp, vp]
@@ -291,9 +300,16 @@ class Cache:
     """Handle returned by mts_cache_create."""
 
     def __init__(self, num_sets: int, key_space: int, dim: int, dtype: int, policy: int = POLICY_LRU,
-                 lock_depth: int = 0, ways: int = CACHE_WAYS):
+                 lock_depth: int = 0, ways: int = CACHE_WAYS, host_rows=None):
+        """host_rows: pinned host tensor (or address) that holds the rows of this level (a second level);
+        None = the rows live in HBM, allocated by the library."""
         h = C.c_void_p()
-        _check(lib().mts_cache_create(C.byref(h), num_sets, key_space, ways, dim, dtype, policy, lock_depth))
+        if host_rows is None:
+            _check(lib().mts_cache_create(C.byref(h), num_sets, key_space, ways, dim, dtype, policy, lock_depth))
+        else:
+            _check(lib().mts_cache_create_host_level(C.byref(h), num_sets, key_space, ways, dim, dtype, policy,
+                                                     lock_depth, _ptr(host_rows)))
+        self._host_rows = host_rows            # keep the storage alive
         self.handle = h
         self.num_sets, self.ways, self.dim, self.dtype = num_sets, ways, dim, dtype
         self.data_ptr = int(lib().mts_cache_data(h))
@@ -352,6 +368,32 @@ def cache_lookup_insert_tables(cache: Cache, tables: Tables, t_begin: int, t_end
         _ptr(evict_dirty), list_capacity, _ptr(overflow_keys), overflow_capacity, _ptr(counters),
         _ptr(sorted_rows_out), _ptr(sorted_pos_out), _ptr(bag_of_lookup_out), _ptr(workspace), workspace_bytes,
         _stream(stream)))
+
+
+def cache2_workspace_bytes(l1: Cache, l2: Cache, N: int, list_capacity: int) -> int:
+    return int(lib().mts_cache2_workspace_bytes(l1.handle, l2.handle, N, list_capacity))
+
+
+def cache2_lookup_insert(l1: Cache, l2: Cache, keys, N: int, step: int, slot_of_lookup, lists: dict, list_capacity: int,
+                         counters2, workspace, workspace_bytes: int, stream=None) -> None:
+    """lists: the thirteen list arrays by name (fetch_keys, fetch_slots, fetch_src, ev1_keys, ev1_slots, ev1_dirty,
+    ev1_dst, ev2_keys, ev2_slots, ev2_dirty, drop_keys, drop_slots, drop_dirty)."""
+    L = lists
+    _check(lib().mts_cache2_lookup_insert(
+        l1.handle, l2.handle, _ptr(keys), N, step, _ptr(slot_of_lookup), _ptr(L["fetch_keys"]), _ptr(L["fetch_slots"]),
+        _ptr(L["fetch_src"]), _ptr(L["ev1_keys"]), _ptr(L["ev1_slots"]), _ptr(L["ev1_dirty"]), _ptr(L["ev1_dst"]),
+        _ptr(L["ev2_keys"]), _ptr(L["ev2_slots"]), _ptr(L["ev2_dirty"]), _ptr(L["drop_keys"]), _ptr(L["drop_slots"]),
+        _ptr(L["drop_dirty"]), list_capacity, _ptr(counters2), _ptr(workspace), workspace_bytes, _stream(stream)))
+
+
+def cache2_move(l1: Cache, l2: Cache, host_store_mapped, lists: dict, list_capacity: int, counters2, fetch_staging,
+                stream=None) -> None:
+    L = lists
+    _check(lib().mts_cache2_move(
+        l1.handle, l2.handle, _ptr(host_store_mapped), _ptr(L["fetch_keys"]), _ptr(L["fetch_slots"]), _ptr(L["fetch_src"]),
+        _ptr(L["ev1_keys"]), _ptr(L["ev1_slots"]), _ptr(L["ev1_dirty"]), _ptr(L["ev1_dst"]), _ptr(L["ev2_keys"]),
+        _ptr(L["ev2_slots"]), _ptr(L["ev2_dirty"]), _ptr(L["drop_keys"]), _ptr(L["drop_slots"]), _ptr(L["drop_dirty"]),
+        list_capacity, _ptr(counters2), _ptr(fetch_staging), _stream(stream)))
 
 
 def cache_refetch_overflowed(cache: Cache, host_rows_mapped, overflow_keys, list_capacity: int, counters,

@@ -29,7 +29,8 @@ struct mts_cache {
   int32_t* placed = nullptr;     // [S*32]  step at which the way's current row was inserted (-1 = free)
   uint32_t* freq = nullptr;      // [S*32]
   uint8_t* dirty = nullptr;      // [S*32]
-  char* data = nullptr;          // [S*32, row_bytes]
+  char* data = nullptr;          // [S*32, row_bytes]  HBM, or pinned host memory of the caller (a second level)
+  bool owns_data = true;
   int32_t* d_status = nullptr;   // sticky status bits (bit 0: a bounded wait on a bulk copy ran out)
 };
 
@@ -54,10 +55,12 @@ __global__ void cache_init_state(uint32_t* tags, int32_t* ts, int32_t* placed, u
 
 // A key outside [0, key_space) is clamped into the range (never sorted or probed as it is: the
 // sort only looks at the bits of key_space) and raises status bit 1.
-__global__ void cache_prepare_keys(const int64_t* __restrict__ keys, int64_t n, int64_t key_space,
+__global__ void cache_prepare_keys(const int64_t* __restrict__ keys, int64_t n, const uint32_t* __restrict__ n_dev,
+                                   int64_t key_space,
                                    uint32_t* __restrict__ k32, uint32_t* __restrict__ pos,
                                    int64_t* __restrict__ counters, uint32_t* __restrict__ overflow_cursor,
                                    int32_t* __restrict__ status) {
+  if (n_dev != nullptr) n = min(n, (int64_t)*n_dev);      // the number of keys is only known on the device
   const int64_t i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i0 < MTS_NUM_COUNTERS) counters[i0] = i0 == MTS_CNT_LOOKUPS ? n : 0;
   if (i0 == 0) *overflow_cursor = 0u;
@@ -102,21 +105,219 @@ __global__ void cache_prepare_from_indices(const TableMeta* __restrict__ meta, i
   }
 }
 
-// Distinct key u: its value, multiplicity and set.  Entries u >= U of the sort input are not
-// touched: the second sort runs on the device-side count U.
-__global__ void cache_describe_unique(const uint32_t* __restrict__ sorted_keys, uint32_t key_base,
-                                      const uint32_t* __restrict__ seg_start,
-                                      const uint32_t* __restrict__ n_unique, uint64_t S,
-                                      uint32_t* __restrict__ ukey, uint32_t* __restrict__ mult,
-                                      uint32_t* __restrict__ set_keys, uint32_t* __restrict__ set_vals) {
-  const uint32_t U = *n_unique;
-  for (int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; u < U; u += (int64_t)gridDim.x * blockDim.x) {
-    const uint32_t s0 = seg_start[u];
-    const uint32_t k = sorted_keys[s0] - key_base;
-    ukey[u] = k;
-    mult[u] = seg_start[u + 1] - s0;
-    set_keys[u] = set_of_key(k, S);
-    set_vals[u] = (uint32_t)u;
+// Exclusive scan of one value per thread over a 256-thread block (`sh`: 9 words of shared memory).
+__device__ __forceinline__ uint32_t block_scan_256(uint32_t v, uint32_t* sh, uint32_t* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += y;
+  }
+  if (lane == 31) sh[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t w = lane < 8 ? sh[lane] : 0u;
+    uint32_t winc = w;
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) {
+      uint32_t y = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += y;
+    }
+    if (lane < 8) sh[lane] = winc - w;
+    if (lane == 7) sh[8] = winc;
+  }
+  __syncthreads();
+  const uint32_t res = sh[warp] + inc - v;
+  *total = sh[8];
+  __syncthreads();
+  return res;
+}
+
+// Rows that are inserted with a history instead of as fresh rows (first-level victims entering a second
+// level): timestamp, use count and dirty byte per entry of the source list; all null = fresh rows.
+struct InsertAttrs {
+  const int32_t* ts = nullptr;
+  const uint32_t* freq = nullptr;
+  const uint8_t* dirty = nullptr;
+};
+
+// The second level as the first level's tag step sees it.
+struct SecondLevel {
+  uint32_t* tags = nullptr;
+  int32_t* ts = nullptr;
+  int32_t* placed = nullptr;
+  uint32_t* freq = nullptr;
+  uint8_t* dirty = nullptr;
+  uint64_t S = 0;
+};
+
+// Probe of every distinct key against the state before the call, 32 keys per warp at a time: each lane
+// describes one key (value, multiplicity, set), then the warp walks the 32 keys and compares the 32 tags of
+// each key's set (lane = way).  A hit is refreshed here (timestamp, use count) and gets its slot; a key
+// that misses is only flagged.  Block b owns a contiguous range of keys and counts its misses, so that
+// the misses can be compacted in key order afterwards.  Entries u >= U are not touched.
+constexpr int PROBE_BLOCKS = 1024;
+
+__device__ __forceinline__ int64_t probe_per_block(int64_t n, int G) {
+  const int64_t per = (n + G - 1) / G;
+  return (per + CACHE_THREADS - 1) / CACHE_THREADS * CACHE_THREADS;
+}
+
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_probe_hits(const uint32_t* __restrict__ sorted_keys, uint32_t key_base,
+                 const uint32_t* __restrict__ seg_start, const uint32_t* __restrict__ n_unique, uint64_t S,
+                 const uint32_t* __restrict__ tags, int32_t* __restrict__ ts, uint32_t* __restrict__ freq,
+                 int32_t step, uint32_t* __restrict__ ukey, uint32_t* __restrict__ mult,
+                 int32_t* __restrict__ slot_of_uniq, uint8_t* __restrict__ missed,
+                 uint32_t* __restrict__ cnt_missed, unsigned long long* __restrict__ counters,
+                 const uint32_t* __restrict__ sorted_pos, InsertAttrs attrs, int32_t* __restrict__ ins_ts,
+                 uint8_t* __restrict__ ins_dirty) {
+  __shared__ uint32_t sh[9];
+  const int lane = threadIdx.x & 31;
+  const int64_t U = *n_unique;
+  const int64_t per = probe_per_block(U, gridDim.x);
+  const int64_t begin = (int64_t)blockIdx.x * per, end = min(U, begin + per);
+  unsigned long long c_hit_lookups = 0, c_uhits = 0;
+  uint32_t my_missed = 0;
+  for (int64_t base = begin + (threadIdx.x & ~31); base < end; base += CACHE_THREADS) {
+    const int64_t u = base + lane;
+    const bool valid = u < end;
+    uint32_t k = 0, mu = 0, set = 0;
+    if (valid) {
+      const uint32_t s0 = seg_start[u];
+      k = sorted_keys[s0] - key_base;
+      mu = seg_start[u + 1] - s0;
+      set = set_of_key(k, S);
+      if (attrs.ts != nullptr) {
+        // a row that arrives with a history: the entry it came from (position in the source list)
+        const uint32_t e = sorted_pos[s0];
+        mu = attrs.freq[e];
+        ins_ts[u] = attrs.ts[e];
+        ins_dirty[u] = attrs.dirty[e];
+      }
+      ukey[u] = k;
+      mult[u] = mu;
+    }
+    const int m = (int)min((int64_t)32, end - base);
+    int32_t my_slot = -1;
+#pragma unroll 8
+    for (int q = 0; q < 32; ++q) {
+      if (q < m) {
+        const uint32_t kq = __shfl_sync(0xffffffffu, k, q);
+        const uint32_t sq = __shfl_sync(0xffffffffu, set, q);
+        const uint32_t tag = tags[(int64_t)sq * 32 + lane];
+        const uint32_t hit = __ballot_sync(0xffffffffu, tag == kq);      // a free way holds no valid key
+        if (hit && lane == q) my_slot = (int32_t)((int64_t)sq * 32 + __ffs(hit) - 1);
+      }
+    }
+    if (valid) {
+      if (my_slot >= 0) {
+        ts[my_slot] = step;
+        freq[my_slot] += mu;
+        c_hit_lookups += mu;
+        c_uhits += 1;
+        slot_of_uniq[u] = my_slot;
+        missed[u] = 0;
+      } else {
+        missed[u] = 1;
+        my_missed += 1;
+      }
+    }
+  }
+  uint32_t total;
+  block_scan_256(my_missed, sh, &total);
+  if (threadIdx.x == 0) cnt_missed[blockIdx.x] = total;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    c_hit_lookups += __shfl_xor_sync(0xffffffffu, c_hit_lookups, o);
+    c_uhits += __shfl_xor_sync(0xffffffffu, c_uhits, o);
+  }
+  if (lane == 0) {
+    if (c_hit_lookups) atomicAdd(&counters[MTS_CNT_HIT_LOOKUPS], c_hit_lookups);
+    if (c_uhits) atomicAdd(&counters[MTS_CNT_UNIQUE_HITS], c_uhits);
+  }
+}
+
+// Exclusive prefix over the blocks' miss counts (in place); *n_missed = their sum.
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_scan_missed(uint32_t* __restrict__ cnt_missed, int G, uint32_t* __restrict__ n_missed) {
+  __shared__ uint32_t sh[9];
+  constexpr int PER = PROBE_BLOCKS / CACHE_THREADS;
+  const int j0 = threadIdx.x * PER;
+  uint32_t v[PER];
+  uint32_t s = 0;
+#pragma unroll
+  for (int k = 0; k < PER; ++k) { v[k] = j0 + k < G ? cnt_missed[j0 + k] : 0u; s += v[k]; }
+  uint32_t total;
+  uint32_t ex = block_scan_256(s, sh, &total);
+#pragma unroll
+  for (int k = 0; k < PER; ++k) { if (j0 + k < G) cnt_missed[j0 + k] = ex; ex += v[k]; }
+  if (threadIdx.x == 0) *n_missed = total;
+}
+
+// The missing keys in ascending key order: (set, index among the distinct keys), the input of the sort by set.
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_compact_missed(const uint8_t* __restrict__ missed, const uint32_t* __restrict__ ukey,
+                     const uint32_t* __restrict__ n_unique, uint64_t S, const uint32_t* __restrict__ base_missed,
+                     uint32_t* __restrict__ set_keys, uint32_t* __restrict__ set_vals) {
+  __shared__ uint32_t sh[9];
+  const int64_t U = *n_unique;
+  const int64_t per = probe_per_block(U, gridDim.x);
+  const int64_t begin = (int64_t)blockIdx.x * per, end = min(U, begin + per);
+  uint32_t at = base_missed[blockIdx.x];
+  for (int64_t t0 = begin; t0 < end; t0 += CACHE_THREADS) {
+    const int64_t u = t0 + threadIdx.x;
+    const bool miss = u < end && missed[u] != 0;
+    uint32_t total;
+    const uint32_t p = block_scan_256(miss ? 1u : 0u, sh, &total);
+    if (miss) {
+      set_keys[at + p] = set_of_key(ukey[u], S);
+      set_vals[at + p] = (uint32_t)u;
+    }
+    at += total;
+  }
+}
+
+// Second level: where does every key that missed the first level sit there (slot, or -1)?  Read only; 32 of
+// the compacted misses per warp at a time, lane = way in the walk.
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_probe_second_level(const uint32_t* __restrict__ miss_uidx, const uint32_t* __restrict__ n_missed,
+                         const uint32_t* __restrict__ ukey, const uint32_t* __restrict__ mult, SecondLevel l2,
+                         int32_t* __restrict__ l2slot_of_uniq, unsigned long long* __restrict__ counters2) {
+  const int lane = threadIdx.x & 31;
+  const int64_t M = *n_missed;
+  const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  unsigned long long c_lookups = 0, c_keys = 0;
+  for (int64_t base = warp0 * 32; base < M; base += nwarps * 32) {
+    const int64_t j = base + lane;
+    uint32_t u = 0, k = 0, set = 0;
+    if (j < M) { u = miss_uidx[j]; k = ukey[u]; set = set_of_key(k, l2.S); }
+    const int m = (int)min((int64_t)32, M - base);
+    int32_t my_slot = -1;
+#pragma unroll 8
+    for (int q = 0; q < 32; ++q) {
+      if (q < m) {
+        const uint32_t kq = __shfl_sync(0xffffffffu, k, q);
+        const uint32_t sq = __shfl_sync(0xffffffffu, set, q);
+        const uint32_t hit = __ballot_sync(0xffffffffu, l2.tags[(int64_t)sq * 32 + lane] == kq);
+        if (hit && lane == q) my_slot = (int32_t)((int64_t)sq * 32 + __ffs(hit) - 1);
+      }
+    }
+    if (j < M) {
+      l2slot_of_uniq[u] = my_slot;
+      if (my_slot >= 0) { c_lookups += mult[u]; c_keys += 1; }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    c_lookups += __shfl_xor_sync(0xffffffffu, c_lookups, o);
+    c_keys += __shfl_xor_sync(0xffffffffu, c_keys, o);
+  }
+  if (lane == 0) {
+    if (c_lookups) atomicAdd(&counters2[MTS_CNT2_L2_HIT_LOOKUPS], c_lookups);
+    if (c_keys) atomicAdd(&counters2[MTS_CNT2_L2_UNIQUE_HITS], c_keys);
   }
 }
 
@@ -133,12 +334,14 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
                     uint32_t* __restrict__ member_old_key, uint8_t* __restrict__ member_old_dirty,
                     int32_t* __restrict__ member_old_ts, uint32_t* __restrict__ member_old_freq,
                     int32_t* __restrict__ member_old_placed,
-                    int32_t* __restrict__ member_slot, unsigned long long* __restrict__ counters) {
+                    int32_t* __restrict__ member_slot, unsigned long long* __restrict__ counters,
+                    const int32_t* __restrict__ ins_ts, const uint8_t* __restrict__ ins_dirty,
+                    unsigned long long* __restrict__ overflow_dirty_count) {
   const int lane = threadIdx.x & 31;
   const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   const uint32_t NS = *n_sets;
-  unsigned long long c_hit_lookups = 0, c_uhits = 0, c_dirty = 0, c_overflow = 0;
+  unsigned long long c_hit_lookups = 0, c_uhits = 0, c_dirty = 0, c_overflow = 0, c_overflow_dirty = 0;
   for (int64_t si = warp0; si < NS; si += nwarps) {
     const uint32_t j0 = sseg_start[si], j1 = sseg_start[si + 1];
     const uint32_t set = set_sorted[j0];
@@ -197,7 +400,12 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
       const uint32_t j = jb + lane;
       uint32_t u = 0, k = 0, mu = 0;
       uint8_t fl = 3;
-      if (j < j1) { u = member_uidx[j]; k = ukey[u]; mu = mult[u]; fl = member_flag[j]; }
+      int32_t its = step;              // state a placed row starts with: fresh, or the history it arrives with
+      uint32_t idr = 0;
+      if (j < j1) {
+        u = member_uidx[j]; k = ukey[u]; mu = mult[u]; fl = member_flag[j];
+        if (ins_ts != nullptr) { its = ins_ts[u]; idr = ins_dirty[u]; }
+      }
       const int m = (int)min(32u, j1 - jb);
       const uint32_t miss_mask = __ballot_sync(0xffffffffu, j < j1 && fl == 0);
       uint8_t my_flag = fl;
@@ -210,6 +418,8 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
         if (!((miss_mask >> q) & 1u)) continue;
         const uint32_t kq = __shfl_sync(0xffffffffu, k, q);
         const uint32_t mq = __shfl_sync(0xffffffffu, mu, q);
+        const int32_t tsq = __shfl_sync(0xffffffffu, its, q);
+        const uint32_t drq = __shfl_sync(0xffffffffu, idr, q);
         if (placed < ncand) {
           const uint32_t sel = __ballot_sync(0xffffffffu, cand && rank == placed);
           const int way = __ffs(sel) - 1;
@@ -221,7 +431,7 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
             old_tag = tag; old_ts = stamp; old_freq = cnt; old_placed = plc;
             if (!dirty_loaded) { dirty_reg = dirty[slot0 + lane]; dirty_loaded = true; }
             old_dirty = tag != FREE_TAG ? dirty_reg : 0;
-            tag = kq; stamp = step; cnt = mq; plc = step; dirty_reg = 0; touched = true;
+            tag = kq; stamp = tsq; cnt = mq; plc = step; dirty_reg = (uint8_t)drq; touched = true;
           }
           old_tag = __shfl_sync(0xffffffffu, old_tag, way);
           old_placed = __shfl_sync(0xffffffffu, old_placed, way);
@@ -237,6 +447,7 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
         } else {
           if (lane == q) { my_flag = 2; my_slot = -1; }
           c_overflow += 1;
+          c_overflow_dirty += drq ? 1 : 0;
         }
       }
       if (j < j1 && fl == 0) {
@@ -263,39 +474,12 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
     if (c_uhits) atomicAdd(&counters[MTS_CNT_UNIQUE_HITS], c_uhits);
     if (c_dirty) atomicAdd(&counters[MTS_CNT_EVICTED_DIRTY], c_dirty);
     if (c_overflow) atomicAdd(&counters[MTS_CNT_OVERFLOW], c_overflow);
+    if (c_overflow_dirty && overflow_dirty_count != nullptr) atomicAdd(overflow_dirty_count, c_overflow_dirty);
   }
 }
 
 // Ordered compaction of the members flagged "placed" (miss list) and of those whose victim
 // held a row (evict list): count per block, scan the block counts, write.
-__device__ __forceinline__ uint32_t block_scan_256(uint32_t v, uint32_t* sh, uint32_t* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  uint32_t inc = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += y;
-  }
-  if (lane == 31) sh[warp] = inc;
-  __syncthreads();
-  if (warp == 0) {
-    uint32_t w = lane < 8 ? sh[lane] : 0u;
-    uint32_t winc = w;
-#pragma unroll
-    for (int o = 1; o < 8; o <<= 1) {
-      uint32_t y = __shfl_up_sync(0xffffffffu, winc, o);
-      if (lane >= o) winc += y;
-    }
-    if (lane < 8) sh[lane] = winc - w;
-    if (lane == 7) sh[8] = winc;
-  }
-  __syncthreads();
-  const uint32_t res = sh[warp] + inc - v;
-  *total = sh[8];
-  __syncthreads();
-  return res;
-}
-
 constexpr int LIST_BLOCKS = 1024;
 
 __device__ __forceinline__ int64_t list_per_block(int64_t n, int G) {
@@ -357,6 +541,20 @@ cache_scan_lists(uint32_t* __restrict__ cnt_miss, uint32_t* __restrict__ cnt_evi
   }
 }
 
+// What the first level's list pass does for a second level behind it (all null when there is none).
+struct TwoLevelLists {
+  const int32_t* l2slot_of_uniq = nullptr;     // second-level slot of every key that missed the first level, or -1
+  SecondLevel l2;
+  int32_t* fetch_src = nullptr;                // per miss-list entry: second-level slot of the row, or -1 = store
+  int64_t* drop_keys = nullptr;
+  int32_t* drop_slots = nullptr;
+  uint8_t* drop_dirty = nullptr;
+  uint32_t* drop_cursor = nullptr;
+  int32_t* ev1_ts = nullptr;                   // per evict-list entry: timestamp and use count of the victim
+  uint32_t* ev1_freq = nullptr;
+  unsigned long long* counters2 = nullptr;
+};
+
 // Writes the lists.  A placement whose list position is beyond the capacity cannot be carried out by the
 // data movement, so it is undone here: the way gets its old tag, timestamp, count and dirty byte back,
 // the key is not inserted (slot -1) and joins the overflow list.  Inside a set the surplus placements are
@@ -375,7 +573,7 @@ cache_write_lists(uint8_t* __restrict__ member_flag, const uint32_t* __restrict_
                   int64_t overflow_capacity, uint32_t* __restrict__ overflow_cursor,
                   uint32_t* __restrict__ tags, int32_t* __restrict__ ts, int32_t* __restrict__ placed_at,
                   uint32_t* __restrict__ freq, uint8_t* __restrict__ dirty, int32_t* __restrict__ slot_of_uniq,
-                  unsigned long long* __restrict__ counters) {
+                  unsigned long long* __restrict__ counters, TwoLevelLists two) {
   __shared__ uint32_t sh[9];
   const int64_t n = *n_unique;
   const int64_t per = list_per_block(n, gridDim.x);
@@ -398,6 +596,21 @@ cache_write_lists(uint8_t* __restrict__ member_flag, const uint32_t* __restrict_
           evict_keys[be + pb] = (int64_t)member_old_key[j];
           evict_slots[be + pb] = member_slot[j];
           evict_dirty[be + pb] = member_old_dirty[j];
+          if (two.ev1_ts != nullptr) {             // the history the victim takes along to the second level
+            two.ev1_ts[be + pb] = member_old_ts[j];
+            two.ev1_freq[be + pb] = member_old_freq[j];
+          }
+        }
+        if (two.l2slot_of_uniq != nullptr) {
+          // where the row comes from: its second-level slot (the row is promoted: it leaves the second level
+          // and keeps its dirty byte), or -1 = the backing store
+          const int32_t s2 = two.l2slot_of_uniq[member_uidx[j]];
+          two.fetch_src[at] = s2;
+          if (s2 >= 0) {
+            dirty[member_slot[j]] = two.l2.dirty[s2];
+            two.l2.tags[s2] = FREE_TAG; two.l2.ts[s2] = -1; two.l2.placed[s2] = -1; two.l2.freq[s2] = 0; two.l2.dirty[s2] = 0;
+            atomicAdd(&two.counters2[MTS_CNT2_PROMOTED], 1ull);
+          }
         }
         // the last placement that fits fixes the length of the evict list
         if (at == capacity - 1) counters[MTS_CNT_EVICTED] = (unsigned long long)(be + pb + (ev ? 1u : 0u));
@@ -420,6 +633,23 @@ cache_write_lists(uint8_t* __restrict__ member_flag, const uint32_t* __restrict_
       const uint32_t at = atomicAdd(overflow_cursor, 1u);
       if ((int64_t)at < overflow_capacity) overflow_keys[at] = (int64_t)ukey[member_uidx[j]];
     }
+    if (two.l2slot_of_uniq != nullptr && overflowed) {
+      // a second-level hit without a first-level way is served from the backing store in this batch: it
+      // leaves the second level (dirty rows are written to the store by the data movement: drop list)
+      const int32_t s2 = two.l2slot_of_uniq[member_uidx[j]];
+      if (s2 >= 0) {
+        const uint32_t at = atomicAdd(two.drop_cursor, 1u);
+        const uint8_t d = two.l2.dirty[s2];
+        if ((int64_t)at < capacity) {
+          two.drop_keys[at] = (int64_t)ukey[member_uidx[j]];
+          two.drop_slots[at] = s2;
+          two.drop_dirty[at] = d;
+        }
+        two.l2.tags[s2] = FREE_TAG; two.l2.ts[s2] = -1; two.l2.placed[s2] = -1; two.l2.freq[s2] = 0; two.l2.dirty[s2] = 0;
+        atomicAdd(&two.counters2[MTS_CNT2_L2_DROPPED], 1ull);
+        if (d) atomicAdd(&two.counters2[MTS_CNT2_L2_DROPPED_DIRTY], 1ull);
+      }
+    }
     bm += ta;
     be += tb;
   }
@@ -427,7 +657,8 @@ cache_write_lists(uint8_t* __restrict__ member_flag, const uint32_t* __restrict_
 
 __global__ void cache_scatter_slots(const uint32_t* __restrict__ sorted_pos, const uint32_t* __restrict__ uniq_idx,
                                     const int32_t* __restrict__ slot_of_uniq, int64_t n,
-                                    int32_t* __restrict__ slot_of_lookup) {
+                                    const uint32_t* __restrict__ n_dev, int32_t* __restrict__ slot_of_lookup) {
+  if (n_dev != nullptr) n = min(n, (int64_t)*n_dev);
   for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += (int64_t)gridDim.x * blockDim.x)
     slot_of_lookup[sorted_pos[p]] = slot_of_uniq[uniq_idx[p]];
 }
@@ -655,7 +886,8 @@ struct CacheLayout {
   size_t keys_a, keys_b, vals_a, vals_b, uniq_idx, seg_start, ukey, mult, set_a, set_b, sval_a, sval_b,
       sseg_start, slot_of_uniq, member_flag, member_old_key, member_old_dirty, member_old_ts, member_old_freq,
       member_old_placed, member_slot, hist, scan, cnt_miss,
-      cnt_evict, n_unique, n_sets, ovf_cursor, total;
+      cnt_evict, n_unique, n_sets, ovf_cursor, missed, cnt_missed, n_missed, ins_ts, ins_dirty, l2slot_of_uniq,
+      drop_cursor, total;
 };
 
 static int bits_of(int64_t values) {
@@ -681,6 +913,8 @@ static CacheLayout cache_layout(const mts_cache* c, int64_t N) {
   L.scan = take(scan_scratch_words() * 4);
   L.cnt_miss = take(LIST_BLOCKS * 4); L.cnt_evict = take(LIST_BLOCKS * 4);
   L.n_unique = take(256); L.n_sets = take(256); L.ovf_cursor = take(256);
+  L.missed = take(n); L.cnt_missed = take(PROBE_BLOCKS * 4); L.n_missed = take(256);
+  L.ins_ts = take(n * 4); L.ins_dirty = take(n); L.l2slot_of_uniq = take(n * 4); L.drop_cursor = take(256);
   L.total = off;
   return L;
 }
@@ -689,8 +923,10 @@ static CacheLayout cache_layout(const mts_cache* c, int64_t N) {
 
 using namespace mts;
 
-extern "C" int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_space, int32_t ways, int32_t dim,
-                                int32_t dtype, int32_t policy, int32_t lock_depth) {
+extern "C" int mts_cache_destroy(mts_cache* c);
+
+static int cache_create_impl(mts_cache** out, int64_t num_sets, int64_t key_space, int32_t ways, int32_t dim,
+                             int32_t dtype, int32_t policy, int32_t lock_depth, void* external_rows) {
   if (!out) return set_error(MTS_ERR_INVALID_ARG, "cache_create: null out");
   *out = nullptr;
   if (ways != MTS_CACHE_WAYS) return set_error(MTS_ERR_INVALID_ARG, "cache_create: ways must be %d", MTS_CACHE_WAYS);
@@ -717,7 +953,12 @@ extern "C" int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_s
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->placed, n * 4), "cudaMalloc(insertion steps)");
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->freq, n * 4), "cudaMalloc(counts)");
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->dirty, n), "cudaMalloc(dirty)");
-  if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->data, (size_t)n * c->row_bytes), "cudaMalloc(cache rows)");
+  if (external_rows != nullptr) {
+    c->data = static_cast<char*>(external_rows);
+    c->owns_data = false;
+  } else if (rc == MTS_OK) {
+    rc = check_cuda(cudaMalloc(&c->data, (size_t)n * c->row_bytes), "cudaMalloc(cache rows)");
+  }
   if (rc == MTS_OK) rc = check_cuda(cudaMalloc(&c->d_status, 256), "cudaMalloc(cache status)");
   if (rc == MTS_OK) rc = check_cuda(cudaMemset(c->d_status, 0, 256), "cudaMemset(cache status)");
   if (rc == MTS_OK) {
@@ -727,16 +968,31 @@ extern "C" int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_s
     }
     rc = check_launch("cache_init_state");
   }
-  if (rc == MTS_OK) rc = check_cuda(cudaMemset(c->data, 0, (size_t)n * c->row_bytes), "cudaMemset(cache rows)");
+  if (rc == MTS_OK && c->owns_data) rc = check_cuda(cudaMemset(c->data, 0, (size_t)n * c->row_bytes), "cudaMemset(cache rows)");
   if (rc == MTS_OK) rc = check_cuda(cudaDeviceSynchronize(), "cache_create sync");
   if (rc != MTS_OK) { mts_cache_destroy(c); return rc; }
   *out = c;
   return MTS_OK;
 }
 
+extern "C" int mts_cache_create(mts_cache** out, int64_t num_sets, int64_t key_space, int32_t ways, int32_t dim,
+                                int32_t dtype, int32_t policy, int32_t lock_depth) {
+  return cache_create_impl(out, num_sets, key_space, ways, dim, dtype, policy, lock_depth, nullptr);
+}
+
+extern "C" int mts_cache_create_host_level(mts_cache** out, int64_t num_sets, int64_t key_space, int32_t ways,
+                                           int32_t dim, int32_t dtype, int32_t policy, int32_t lock_depth,
+                                           void* host_rows_mapped) {
+  if (!host_rows_mapped) return set_error(MTS_ERR_INVALID_ARG, "cache_create_host_level: null row storage");
+  if ((uintptr_t)host_rows_mapped & 15) return set_error(MTS_ERR_ALIGNMENT, "cache_create_host_level: row storage must be 16-byte aligned");
+  return cache_create_impl(out, num_sets, key_space, ways, dim, dtype, policy, lock_depth, host_rows_mapped);
+}
+
 extern "C" int mts_cache_destroy(mts_cache* c) {
   if (!c) return MTS_OK;
-  cudaFree(c->tags); cudaFree(c->ts); cudaFree(c->placed); cudaFree(c->freq); cudaFree(c->dirty); cudaFree(c->data); cudaFree(c->d_status);
+  cudaFree(c->tags); cudaFree(c->ts); cudaFree(c->placed); cudaFree(c->freq); cudaFree(c->dirty);
+  if (c->owns_data) cudaFree(c->data);
+  cudaFree(c->d_status);
   delete c;
   return MTS_OK;
 }
@@ -811,10 +1067,15 @@ struct KeySource {
   uint32_t* bag_of_lookup_out = nullptr;
 };
 
+// n_dev (nullable): device-resident number of keys, N is then its upper bound.  attrs: the keys are rows that
+// arrive with a history (see InsertAttrs; indexed by position in `src.keys`).  two (nullable): a second level
+// behind this cache; its l2slot_of_uniq and drop_cursor are taken from the workspace here.
 int lookup_insert_impl(mts_cache* c, const KeySource& src, int64_t N, int64_t step, int32_t* slot_of_lookup,
                        int64_t* miss_keys, int32_t* miss_slots, int64_t* evict_keys, int32_t* evict_slots,
                        uint8_t* evict_dirty, int64_t* overflow_keys, int64_t list_capacity, int64_t overflow_capacity,
-                       int64_t* counters, void* workspace, size_t workspace_bytes, void* stream) {
+                       int64_t* counters, void* workspace, size_t workspace_bytes, void* stream,
+                       const uint32_t* n_dev = nullptr, InsertAttrs attrs = InsertAttrs(),
+                       TwoLevelLists* two = nullptr, unsigned long long* overflow_dirty_count = nullptr) {
   if (!c || !counters || N < 0 || list_capacity < 0 || overflow_capacity < 0 || step < 0 || step >= (1ll << 31) - 1)
     return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert: bad argument");
   if (N > 0 && !slot_of_lookup) return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert: null slot_of_lookup");
@@ -848,8 +1109,8 @@ int lookup_insert_impl(mts_cache* c, const KeySource& src, int64_t N, int64_t st
     if (N > 0 && !src.keys) return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert: null keys");
     {
       LaunchScope scope(K_CACHE_PREPARE, s);
-      cache_prepare_keys<<<grid, 256, 0, s>>>(src.keys, N, c->key_space, keys_a, vals_a, counters, U32(L.ovf_cursor),
-                                              c->d_status);
+      cache_prepare_keys<<<grid, 256, 0, s>>>(src.keys, N, n_dev, c->key_space, keys_a, vals_a, counters,
+                                              U32(L.ovf_cursor), c->d_status);
     }
     rc = check_launch("cache_prepare_keys");
   } else {
@@ -869,25 +1130,55 @@ int lookup_insert_impl(mts_cache* c, const KeySource& src, int64_t N, int64_t st
     return MTS_OK;   // counters already written: all zero
   }
   uint32_t *sk = nullptr, *sp = nullptr;
-  rc = radix_sort_pairs(keys_a, vals_a, keys_b, vals_b, N, nullptr, key_bits, key_base, U32(L.hist), &sk, &sp, s);
+  rc = radix_sort_pairs(keys_a, vals_a, keys_b, vals_b, N, n_dev, key_bits, key_base, U32(L.hist), &sk, &sp, s);
   if (rc != MTS_OK) return rc;
-  rc = unique_segments(sk, N, nullptr, U32(L.seg_start), U32(L.uniq_idx), n_unique, U32(L.scan), s);
+  rc = unique_segments(sk, N, n_dev, U32(L.seg_start), U32(L.uniq_idx), n_unique, U32(L.scan), s);
   if (rc != MTS_OK) return rc;
+  // hits are found and refreshed key by key; only the missing keys are grouped by set for the replacement
+  int32_t* slot_of_uniq = reinterpret_cast<int32_t*>(ws + L.slot_of_uniq);
+  uint8_t* missed = reinterpret_cast<uint8_t*>(ws + L.missed);
+  uint32_t* n_missed = U32(L.n_missed);
+  const int PG = (int)std::min<int64_t>((int64_t)PROBE_BLOCKS, ceil_div(N, CACHE_THREADS * 4));
   {
     LaunchScope scope(K_CACHE_DESCRIBE, s);
-    cache_describe_unique<<<grid, 256, 0, s>>>(sk, key_base, U32(L.seg_start), n_unique, (uint64_t)c->S, U32(L.ukey),
-                                               U32(L.mult), U32(L.set_a), U32(L.sval_a));
+    cache_probe_hits<<<PG, CACHE_THREADS, 0, s>>>(sk, key_base, U32(L.seg_start), n_unique, (uint64_t)c->S, c->tags, c->ts,
+                                                  c->freq, (int32_t)step, U32(L.ukey), U32(L.mult), slot_of_uniq, missed,
+                                                  U32(L.cnt_missed), reinterpret_cast<unsigned long long*>(counters), sp,
+                                                  attrs, reinterpret_cast<int32_t*>(ws + L.ins_ts),
+                                                  reinterpret_cast<uint8_t*>(ws + L.ins_dirty));
   }
-  rc = check_launch("cache_describe_unique");
+  {
+    LaunchScope scope(K_CACHE_DESCRIBE, s);
+    cache_scan_missed<<<1, CACHE_THREADS, 0, s>>>(U32(L.cnt_missed), PG, n_missed);
+  }
+  {
+    LaunchScope scope(K_CACHE_DESCRIBE, s);
+    cache_compact_missed<<<PG, CACHE_THREADS, 0, s>>>(missed, U32(L.ukey), n_unique, (uint64_t)c->S, U32(L.cnt_missed),
+                                                      U32(L.set_a), U32(L.sval_a));
+  }
+  TwoLevelLists lists2;
+  if (two != nullptr) {
+    // where the keys that missed this level sit in the second one (before the sort by set reuses the buffers)
+    two->l2slot_of_uniq = reinterpret_cast<int32_t*>(ws + L.l2slot_of_uniq);
+    two->drop_cursor = U32(L.drop_cursor);
+    if (cudaMemsetAsync(two->drop_cursor, 0, sizeof(uint32_t), s) != cudaSuccess) return check_launch("memset(drop cursor)");
+    {
+      LaunchScope scope(K_CACHE_DESCRIBE, s);
+      cache_probe_second_level<<<grid, CACHE_THREADS, 0, s>>>(U32(L.sval_a), n_missed, U32(L.ukey), U32(L.mult), two->l2,
+                                                              reinterpret_cast<int32_t*>(ws + L.l2slot_of_uniq),
+                                                              two->counters2);
+    }
+    lists2 = *two;
+  }
+  rc = check_launch("cache_probe_hits / cache_compact_missed");
   if (rc != MTS_OK) return rc;
   const int set_bits = c->S > 1 ? bits_of(c->S) : 0;
   uint32_t *ss = nullptr, *su = nullptr;
-  rc = radix_sort_pairs(U32(L.set_a), U32(L.sval_a), U32(L.set_b), U32(L.sval_b), N, n_unique, set_bits, 0u,
+  rc = radix_sort_pairs(U32(L.set_a), U32(L.sval_a), U32(L.set_b), U32(L.sval_b), N, n_missed, set_bits, 0u,
                         U32(L.hist), &ss, &su, s);
   if (rc != MTS_OK) return rc;
-  rc = unique_segments(ss, N, n_unique, U32(L.sseg_start), nullptr, n_sets, U32(L.scan), s);
+  rc = unique_segments(ss, N, n_missed, U32(L.sseg_start), nullptr, n_sets, U32(L.scan), s);
   if (rc != MTS_OK) return rc;
-  int32_t* slot_of_uniq = reinterpret_cast<int32_t*>(ws + L.slot_of_uniq);
   uint8_t* member_flag = reinterpret_cast<uint8_t*>(ws + L.member_flag);
   uint8_t* member_old_dirty = reinterpret_cast<uint8_t*>(ws + L.member_old_dirty);
   int32_t* member_slot = reinterpret_cast<int32_t*>(ws + L.member_slot);
@@ -898,14 +1189,16 @@ int lookup_insert_impl(mts_cache* c, const KeySource& src, int64_t N, int64_t st
         c->lock_depth, c->policy, slot_of_uniq, member_flag, U32(L.member_old_key), member_old_dirty,
         reinterpret_cast<int32_t*>(ws + L.member_old_ts), U32(L.member_old_freq),
         reinterpret_cast<int32_t*>(ws + L.member_old_placed), member_slot,
-        reinterpret_cast<unsigned long long*>(counters));
+        reinterpret_cast<unsigned long long*>(counters),
+        attrs.ts != nullptr ? reinterpret_cast<const int32_t*>(ws + L.ins_ts) : nullptr,
+        attrs.ts != nullptr ? reinterpret_cast<const uint8_t*>(ws + L.ins_dirty) : nullptr, overflow_dirty_count);
   }
   rc = check_launch("cache_probe_replace");
   if (rc != MTS_OK) return rc;
   const int G = (int)std::min<int64_t>((int64_t)LIST_BLOCKS, ceil_div(N, CACHE_THREADS * 4));
   {
     LaunchScope scope(K_CACHE_LISTS, s);
-    cache_count_lists<<<G, CACHE_THREADS, 0, s>>>(member_flag, U32(L.member_old_key), n_unique, U32(L.cnt_miss),
+    cache_count_lists<<<G, CACHE_THREADS, 0, s>>>(member_flag, U32(L.member_old_key), n_missed, U32(L.cnt_miss),
                                                   U32(L.cnt_evict));
   }
   {
@@ -917,15 +1210,15 @@ int lookup_insert_impl(mts_cache* c, const KeySource& src, int64_t N, int64_t st
     LaunchScope scope(K_CACHE_LISTS, s);
     cache_write_lists<<<G, CACHE_THREADS, 0, s>>>(
         member_flag, U32(L.member_old_key), member_old_dirty, reinterpret_cast<int32_t*>(ws + L.member_old_ts),
-        U32(L.member_old_freq), reinterpret_cast<int32_t*>(ws + L.member_old_placed), member_slot, su, U32(L.ukey), n_unique, U32(L.cnt_miss), U32(L.cnt_evict), list_capacity,
+        U32(L.member_old_freq), reinterpret_cast<int32_t*>(ws + L.member_old_placed), member_slot, su, U32(L.ukey), n_missed, U32(L.cnt_miss), U32(L.cnt_evict), list_capacity,
         miss_keys, miss_slots, evict_keys, evict_slots, evict_dirty, overflow_keys, overflow_capacity, U32(L.ovf_cursor),
-        c->tags, c->ts, c->placed, c->freq, c->dirty, slot_of_uniq, reinterpret_cast<unsigned long long*>(counters));
+        c->tags, c->ts, c->placed, c->freq, c->dirty, slot_of_uniq, reinterpret_cast<unsigned long long*>(counters), lists2);
   }
   {
     // positions are relative to the key array, or batch positions when the keys came from a batch's
     // sparse input (slot_of_lookup is then the batch-wide array)
     LaunchScope scope(K_CACHE_SCATTER_SLOTS, s);
-    cache_scatter_slots<<<grid, 256, 0, s>>>(sp, U32(L.uniq_idx), slot_of_uniq, N, slot_of_lookup);
+    cache_scatter_slots<<<grid, 256, 0, s>>>(sp, U32(L.uniq_idx), slot_of_uniq, N, n_dev, slot_of_lookup);
   }
   return check_launch("cache lists / scatter");
 }
@@ -970,6 +1263,203 @@ extern "C" int mts_cache_lookup_insert_tables(mts_cache* c, const mts_tables* h,
   src.sorted_rows_out = sorted_rows_out; src.sorted_pos_out = sorted_pos_out; src.bag_of_lookup_out = bag_of_lookup_out;
   return lookup_insert_impl(c, src, n, step, slot_of_lookup, miss_keys, miss_slots, evict_keys, evict_slots, evict_dirty,
                             overflow_keys, list_capacity, overflow_capacity, counters, workspace, workspace_bytes, stream);
+}
+
+// ------------------------------------------------------------------------------------ two cache levels
+namespace mts {
+
+// counters2[0..9] come from the first level's pass; the second level's pass counted into a scratch block.
+__global__ void cache2_finish_counters(const int64_t* __restrict__ l2_counters,
+                                       const unsigned long long* __restrict__ bypass_dirty,
+                                       int64_t* __restrict__ counters2) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) {
+    counters2[MTS_CNT2_DEMOTED] = l2_counters[MTS_CNT_INSERTED];
+    counters2[MTS_CNT2_L2_EVICTED] = l2_counters[MTS_CNT_EVICTED];
+    counters2[MTS_CNT2_L2_EVICTED_DIRTY] = l2_counters[MTS_CNT_EVICTED_DIRTY];
+    counters2[MTS_CNT2_L2_BYPASS] = l2_counters[MTS_CNT_OVERFLOW];
+    counters2[MTS_CNT2_L2_BYPASS_DIRTY] = (int64_t)*bypass_dirty;
+  }
+}
+
+__global__ void cache2_begin(int64_t* __restrict__ counters2, unsigned long long* __restrict__ bypass_dirty) {
+  if (blockIdx.x == 0 && threadIdx.x < MTS_NUM_COUNTERS2 - MTS_NUM_COUNTERS) counters2[MTS_NUM_COUNTERS + threadIdx.x] = 0;
+  if (blockIdx.x == 0 && threadIdx.x == 0) *bypass_dirty = 0ull;
+}
+
+// number of first-level victims as the 32-bit device count the second level's pass takes
+__global__ void cache2_victim_count(const int64_t* __restrict__ counters, int64_t capacity, uint32_t* __restrict__ n_out) {
+  if (blockIdx.x == 0 && threadIdx.x == 0) *n_out = (uint32_t)list_len(counters, MTS_CNT_EVICTED, capacity);
+}
+
+// rows that leave the second level for the store (its victims, and hits that found no first-level way)
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache2_rows_to_store(const char* __restrict__ l2_rows, int row_bytes, const int64_t* __restrict__ keys,
+                     const int32_t* __restrict__ slots, const uint8_t* __restrict__ dirty,
+                     const int64_t* __restrict__ counters2, int which, int64_t capacity, char* __restrict__ store) {
+  const int64_t n = list_len(counters2, which, capacity);
+  copy_rows(n, row_bytes / 16,
+            [&](int64_t k) { return dirty[k] ? l2_rows + (int64_t)slots[k] * row_bytes : nullptr; },
+            [&](int64_t k) { return store + keys[k] * row_bytes; });
+}
+
+// the rows to be inserted into the first level, from their second-level slot or from the store, in list order
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache2_gather_fetch(const char* __restrict__ l2_rows, const char* __restrict__ store, int row_bytes,
+                    const int64_t* __restrict__ fetch_keys, const int32_t* __restrict__ fetch_src,
+                    const int64_t* __restrict__ counters2, int64_t capacity, char* __restrict__ fetched) {
+  const int64_t n = list_len(counters2, MTS_CNT_INSERTED, capacity);
+  copy_rows(n, row_bytes / 16,
+            [&](int64_t k) { return fetch_src[k] >= 0 ? l2_rows + (int64_t)fetch_src[k] * row_bytes : store + fetch_keys[k] * row_bytes; },
+            [&](int64_t k) { return fetched + k * row_bytes; });
+}
+
+// first-level victims to their second-level slot, or to the store when they have none and are dirty
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache2_demote(const char* __restrict__ l1_rows, int row_bytes, const int64_t* __restrict__ ev1_keys,
+              const int32_t* __restrict__ ev1_slots, const uint8_t* __restrict__ ev1_dirty,
+              const int32_t* __restrict__ ev1_dst, const int64_t* __restrict__ counters2, int64_t capacity,
+              char* __restrict__ l2_rows, char* __restrict__ store) {
+  const int64_t n = list_len(counters2, MTS_CNT_EVICTED, capacity);
+  copy_rows(n, row_bytes / 16,
+            [&](int64_t k) { return l1_rows + (int64_t)ev1_slots[k] * row_bytes; },
+            [&](int64_t k) -> char* {
+              if (ev1_dst[k] >= 0) return l2_rows + (int64_t)ev1_dst[k] * row_bytes;
+              return ev1_dirty[k] ? store + ev1_keys[k] * row_bytes : nullptr;
+            });
+}
+
+struct Cache2Layout { size_t first, second, ev1_ts, ev1_freq, miss2_keys, miss2_slots, l2_counters, n_victims, bypass_dirty, total; };
+
+static Cache2Layout cache2_layout(const mts_cache* l1, const mts_cache* l2, int64_t N, int64_t list_capacity) {
+  Cache2Layout L;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t cap = (size_t)(list_capacity > 0 ? list_capacity : 1);
+  L.first = take(cache_layout(l1, N).total);
+  L.second = take(cache_layout(l2, list_capacity).total);
+  L.ev1_ts = take(cap * 4); L.ev1_freq = take(cap * 4);
+  L.miss2_keys = take(cap * 8); L.miss2_slots = take(cap * 4);
+  L.l2_counters = take(MTS_NUM_COUNTERS * 8); L.n_victims = take(256); L.bypass_dirty = take(256);
+  L.total = off;
+  return L;
+}
+
+}  // namespace mts
+
+extern "C" size_t mts_cache2_workspace_bytes(const mts_cache* l1, const mts_cache* l2, int64_t N, int64_t list_capacity) {
+  if (!l1 || !l2 || N < 0 || list_capacity < 0) return 0;
+  return cache2_layout(l1, l2, N, list_capacity).total;
+}
+
+extern "C" int mts_cache2_lookup_insert(mts_cache* l1, mts_cache* l2, const int64_t* keys, int64_t N, int64_t step,
+                                        int32_t* slot_of_lookup, int64_t* fetch_keys, int32_t* fetch_slots,
+                                        int32_t* fetch_src, int64_t* ev1_keys, int32_t* ev1_slots, uint8_t* ev1_dirty,
+                                        int32_t* ev1_dst, int64_t* ev2_keys, int32_t* ev2_slots, uint8_t* ev2_dirty,
+                                        int64_t* drop_keys, int32_t* drop_slots, uint8_t* drop_dirty,
+                                        int64_t list_capacity, int64_t* counters2, void* workspace,
+                                        size_t workspace_bytes, void* stream) {
+  if (!l1 || !l2 || !counters2 || N < 0 || list_capacity < 1)
+    return set_error(MTS_ERR_INVALID_ARG, "cache2_lookup_insert: bad argument");
+  if (l1->row_bytes != l2->row_bytes || l1->key_space != l2->key_space || l1->dtype != l2->dtype)
+    return set_error(MTS_ERR_INVALID_ARG, "cache2_lookup_insert: the two levels must hold the same rows (dim, dtype, key_space)");
+  if (!fetch_src || !ev1_dst || !ev2_keys || !ev2_slots || !ev2_dirty || !drop_keys || !drop_slots || !drop_dirty)
+    return set_error(MTS_ERR_INVALID_ARG, "cache2_lookup_insert: null list buffer");
+  const Cache2Layout L = cache2_layout(l1, l2, N, list_capacity);
+  if (!workspace || ((uintptr_t)workspace & 255))
+    return set_error(MTS_ERR_ALIGNMENT, "cache2_lookup_insert: workspace must be non-null and 256-byte aligned");
+  if (workspace_bytes < L.total)
+    return set_error(MTS_ERR_WORKSPACE, "cache2_lookup_insert: workspace of %zu bytes, %zu needed", workspace_bytes, L.total);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  char* ws = static_cast<char*>(workspace);
+  unsigned long long* bypass_dirty = reinterpret_cast<unsigned long long*>(ws + L.bypass_dirty);
+  int64_t* l2_counters = reinterpret_cast<int64_t*>(ws + L.l2_counters);
+  uint32_t* n_victims = reinterpret_cast<uint32_t*>(ws + L.n_victims);
+  {
+    LaunchScope scope(K_CACHE_PREPARE, s);
+    cache2_begin<<<1, 32, 0, s>>>(counters2, bypass_dirty);
+  }
+  // first level: exactly the one-level pass; its list pass also resolves the second-level hits
+  TwoLevelLists two;
+  two.l2.tags = l2->tags; two.l2.ts = l2->ts; two.l2.placed = l2->placed; two.l2.freq = l2->freq; two.l2.dirty = l2->dirty;
+  two.l2.S = (uint64_t)l2->S;
+  two.fetch_src = fetch_src;
+  two.drop_keys = drop_keys; two.drop_slots = drop_slots; two.drop_dirty = drop_dirty;
+  two.ev1_ts = reinterpret_cast<int32_t*>(ws + L.ev1_ts);
+  two.ev1_freq = reinterpret_cast<uint32_t*>(ws + L.ev1_freq);
+  two.counters2 = reinterpret_cast<unsigned long long*>(counters2);
+  KeySource src;
+  src.keys = keys;
+  int rc = lookup_insert_impl(l1, src, N, step, slot_of_lookup, fetch_keys, fetch_slots, ev1_keys, ev1_slots, ev1_dirty,
+                              nullptr, list_capacity, 0, counters2, ws + L.first, cache_layout(l1, N).total, stream, nullptr,
+                              InsertAttrs(), &two);
+  if (rc != MTS_OK) return rc;
+  if (N == 0) {
+    return check_cuda(cudaMemsetAsync(counters2 + MTS_NUM_COUNTERS, 0, (MTS_NUM_COUNTERS2 - MTS_NUM_COUNTERS) * sizeof(int64_t), s),
+                      "memset(counters2)");
+  }
+  // second level: the first level's victims enter with their timestamp, use count and dirty byte
+  {
+    LaunchScope scope(K_CACHE_PREPARE, s);
+    cache2_victim_count<<<1, 32, 0, s>>>(counters2, list_capacity, n_victims);
+  }
+  InsertAttrs attrs;
+  attrs.ts = two.ev1_ts; attrs.freq = two.ev1_freq; attrs.dirty = ev1_dirty;
+  KeySource victims;
+  victims.keys = ev1_keys;
+  rc = lookup_insert_impl(l2, victims, list_capacity, step, ev1_dst, reinterpret_cast<int64_t*>(ws + L.miss2_keys),
+                          reinterpret_cast<int32_t*>(ws + L.miss2_slots), ev2_keys, ev2_slots, ev2_dirty, nullptr,
+                          list_capacity, 0, l2_counters, ws + L.second, cache_layout(l2, list_capacity).total, stream,
+                          n_victims, attrs, nullptr, bypass_dirty);
+  if (rc != MTS_OK) return rc;
+  {
+    LaunchScope scope(K_CACHE_LISTS, s);
+    cache2_finish_counters<<<1, 32, 0, s>>>(l2_counters, bypass_dirty, counters2);
+  }
+  return check_launch("cache2_lookup_insert");
+}
+
+extern "C" int mts_cache2_move(mts_cache* l1, mts_cache* l2, void* host_store_mapped, const int64_t* fetch_keys,
+                               const int32_t* fetch_slots, const int32_t* fetch_src, const int64_t* ev1_keys,
+                               const int32_t* ev1_slots, const uint8_t* ev1_dirty, const int32_t* ev1_dst,
+                               const int64_t* ev2_keys, const int32_t* ev2_slots, const uint8_t* ev2_dirty,
+                               const int64_t* drop_keys, const int32_t* drop_slots, const uint8_t* drop_dirty,
+                               int64_t list_capacity, const int64_t* counters2, void* fetch_staging, void* stream) {
+  if (!l1 || !l2 || !host_store_mapped || !counters2 || list_capacity < 1 || !fetch_staging || !fetch_keys || !fetch_slots ||
+      !fetch_src || !ev1_keys || !ev1_slots || !ev1_dirty || !ev1_dst || !ev2_keys || !ev2_slots || !ev2_dirty || !drop_keys ||
+      !drop_slots || !drop_dirty)
+    return set_error(MTS_ERR_INVALID_ARG, "cache2_move: null argument");
+  if (((uintptr_t)host_store_mapped | (uintptr_t)fetch_staging) & 15)
+    return set_error(MTS_ERR_ALIGNMENT, "cache2_move: buffers must be 16-byte aligned");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int grid = l1->sm_count * 8;
+  const int rb = l1->row_bytes;
+  char* store = static_cast<char*>(host_store_mapped);
+  {
+    LaunchScope scope(K_CACHE_WRITE_VICTIMS, s);
+    cache2_rows_to_store<<<grid, CACHE_THREADS, 0, s>>>(l2->data, rb, ev2_keys, ev2_slots, ev2_dirty, counters2,
+                                                        MTS_CNT2_L2_EVICTED, list_capacity, store);
+  }
+  {
+    LaunchScope scope(K_CACHE_WRITE_VICTIMS, s);
+    cache2_rows_to_store<<<grid, CACHE_THREADS, 0, s>>>(l2->data, rb, drop_keys, drop_slots, drop_dirty, counters2,
+                                                        MTS_CNT2_L2_DROPPED, list_capacity, store);
+  }
+  {
+    LaunchScope scope(K_CACHE_FETCH_MISSES, s);
+    cache2_gather_fetch<<<grid, CACHE_THREADS, 0, s>>>(l2->data, store, rb, fetch_keys, fetch_src, counters2, list_capacity,
+                                                       static_cast<char*>(fetch_staging));
+  }
+  {
+    LaunchScope scope(K_CACHE_SAVE_VICTIMS, s);
+    cache2_demote<<<grid, CACHE_THREADS, 0, s>>>(l1->data, rb, ev1_keys, ev1_slots, ev1_dirty, ev1_dst, counters2,
+                                                 list_capacity, l2->data, store);
+  }
+  {
+    LaunchScope scope(K_CACHE_FETCH_MISSES, s);
+    cache_place_fetched<<<grid, CACHE_THREADS, 0, s>>>(l1->data, rb, static_cast<const char*>(fetch_staging), fetch_slots,
+                                                       counters2, list_capacity);
+  }
+  return check_launch("cache2_move");
 }
 
 extern "C" int mts_cache_prefetch_misses(mts_cache* c, const void* host_rows_mapped, const int64_t* miss_keys,

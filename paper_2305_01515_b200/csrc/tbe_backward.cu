@@ -754,8 +754,12 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
   if constexpr (NV == 1 && MTS_BWD_USE_LEAN) {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
     // as many blocks as fit on the device at once (or fewer); the warps share out the chunks
-    const unsigned lean_grid =
-        (unsigned)std::min<int64_t>(ceil_div(chunks, LEAN_WARPS), (int64_t)h->sm_count * MTS_BWD_LEAN_MINBLK);
+    // With cached tables the step shares the GPU with the cache's tag lookup and data movement on other
+    // streams: blocks that stay until the last chunk would keep every warp slot for the whole kernel and
+    // hold those streams back, so there the grid covers the chunks and a block leaves after one round.
+    const unsigned lean_grid = h->any_cached
+        ? (unsigned)ceil_div(chunks, LEAN_WARPS)
+        : (unsigned)std::min<int64_t>(ceil_div(chunks, LEAN_WARPS), (int64_t)h->sm_count * MTS_BWD_LEAN_MINBLK);
     if (cudaMemsetAsync(next_chunk, 0, sizeof(uint32_t), s) != cudaSuccess) return check_launch("memset(next_chunk)");
     if (pooling_mode == MTS_POOL_MEAN)
       MTS_LAUNCH_GH(reduce_chunks_lean, FP16 COMMA true, lean_grid, LEAN_WARPS * 32);
@@ -764,7 +768,7 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
   } else {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
     constexpr int resident = NV == 1 ? MTS_BWD_MINBLK : NV == 2 ? MTS_BWD_MINBLK2 : 2;
-    const unsigned dyn_grid = (unsigned)std::min<int64_t>(grid, (int64_t)h->sm_count * resident);
+    const unsigned dyn_grid = h->any_cached ? grid : (unsigned)std::min<int64_t>(grid, (int64_t)h->sm_count * resident);
     if (cudaMemsetAsync(next_chunk, 0, sizeof(uint32_t), s) != cudaSuccess) return check_launch("memset(next_chunk)");
     if (pooling_mode == MTS_POOL_MEAN)
       MTS_LAUNCH_GH(reduce_chunks, FP16 COMMA NV COMMA GROUP COMMA true, dyn_grid, BWD_WARPS * 32);

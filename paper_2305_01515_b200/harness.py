@@ -22,8 +22,9 @@ class DeviceModel:
     an uncached spec keeps every table in HBM and a cached spec every table in the host tier;
     `host_tables` (one bool per table) mixes the two in one model."""
 
-    N_CTX = 4        # batch contexts: batch t trains, the rows of t+1 move, the tags of t+2 are looked
-    #                  up, and the overflow list of t-1 is still needed to repair rows after batch t
+    N_CTX = 6        # batch contexts: batch t trains, the rows of t+1 move, the tags of t+2 are looked up, the
+    #                  overflow lists of t-1 and t-2 are still needed for repairs; two more so that the tag step
+    #                  never has to wait for the repair that last read the context it rewrites
 
     def __init__(self, spec: wl.ModelSpec, device="cuda:0", max_lookups: int = 0, weights: Optional[np.ndarray] = None,
                  lock_depth: int = 0, policy: int = mb.POLICY_LRU, cache_sets: Optional[List[int]] = None,
@@ -238,7 +239,8 @@ class DeviceModel:
         if self.fetch_rows is not None:
             return
         esz = 4 if self.spec.dtype == wl.FP32 else 2
-        self.gather_threads = threads or os.cpu_count() or 1
+        # the caches gather side by side (one worker each): share the cores out
+        self.gather_threads = threads or max(1, (os.cpu_count() or 1) // max(1, len(self.caches)))
         self.fetch_rows = [max(1, min(self.ctx[0]["lists"][g]["capacity"], self.FETCH_STAGE_BYTES // (c.dim * esz)))
                            for g, c in enumerate(self.caches)]
         self.fetch_dev = [torch.empty(r * c.dim * esz, dtype=torch.uint8, device=self.device)

@@ -30,13 +30,15 @@ host memory again (mts_cache_refetch_overflowed with placed_step = t; the stamp 
 from keys that a tag step running further ahead has placed in slots that still hold their victims'
 rows).  Older overflowed rows need nothing: the tag step of batch t already waited for their backward.
 
-Batch contexts (DeviceModel.N_CTX = 4): the tag step of batch t+2 rewrites the context batch t-2
-used, whose overflow list the repair before batch t still reads, so it also waits for that repair.
+Batch contexts (DeviceModel.N_CTX = 6): the tag step of batch t rewrites the context batch t-6 used,
+whose overflow list the repair before batch t-4 was the last to read, so it also waits for that repair
+(long over in practice: the contexts are many so that this wait never holds the tag step back).
 
 With host_gather the missed rows do not cross the host link at the request of SMs (small reads that
-slow every kernel beside them): a worker thread reads the miss list, gathers the rows with the host's
-threads into a pinned buffer and enqueues one contiguous copy and the placing kernel.  The worker runs
-ahead of the launching thread; host-side flags tell each side which events the other has recorded.
+slow every kernel beside them): one worker thread per cache reads the miss list, gathers the rows with
+the host's threads into a pinned buffer and enqueues one contiguous copy and the placing kernel; one more
+thread enqueues the repair once all caches of a batch have moved.  The workers run ahead of the launching
+thread; host-side flags tell each side which events the other has recorded.
 """
 from __future__ import annotations
 
@@ -71,7 +73,7 @@ class CachedTrainer:
         n_c = len(model.caches)
         self.moves = [torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main for _ in range(n_c)]
         self.fix = torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main
-        self.copy = torch.cuda.Stream(self.dev, priority=-1)       # miss keys to the host (host_gather)
+        self.copies = [torch.cuda.Stream(self.dev, priority=-1) for _ in range(n_c)]    # miss keys to the host (host_gather)
         self.history: List[np.ndarray] = []           # per batch [n_caches, NUM_COUNTERS], filled when run() returns
         self.record_timeline = False                  # set to True to time every phase with events
         self._marks = []
@@ -105,8 +107,8 @@ class CachedTrainer:
         pinned history buffer."""
         m, s, ctx = self.m, self.tag, t % DeviceModel.N_CTX
         if self.pipelined:
-            if t - 2 >= 0:
-                s.wait_event(self.ev_ready[t - 2])              # the repair that still read this context's lists
+            if t - DeviceModel.N_CTX + 2 >= 0:                  # the last repair that read this context's lists
+                s.wait_event(self.ev_ready[t - DeviceModel.N_CTX + 2])
             last = t - 1 - m.lock_depth                         # newest batch whose rows may be evicted now
             if last >= 0:
                 s.wait_event(self.ev_bwd[last])
@@ -134,7 +136,7 @@ class CachedTrainer:
                 self.ev_moved[t - 1][g].synchronize()
             n_miss = int(self._host_counters[t, g, mb.COUNTER_NAMES.index("inserted")])
             done = self.m.cache_fetch_via_host(
-                g, n_miss, self.copy, s, ctx,
+                g, n_miss, self.copies[g], s, ctx,
                 mark=(lambda name, s=s: self._mark(name, t, s)) if self.record_timeline else None)
         if not done:
             self.m.cache_fetch(g, stream=s, ctx=ctx)
@@ -164,27 +166,47 @@ class CachedTrainer:
             self._move_cache(t, g, self.host_gather)
         self._finish_move(t)
 
-    # ------------------------------------------------------------------ worker thread (host_gather, pipelined)
-    def _worker(self):
+    # ------------------------------------------------------------------ worker threads (host_gather, pipelined)
+    def _fail(self, e):
+        self._worker_error = e
+        for f in self._ready_recorded:
+            f.set()
+        for row in self._moved_recorded:
+            for f in row:
+                f.set()
+
+    def _cache_worker(self, g):
+        """Batch after batch, the data path of cache g."""
         try:
             torch.cuda.set_device(self.dev)
             while True:
-                t = self._jobs.get()
+                t = self._jobs[g].get()
                 if t is None:
                     return
-                for g in range(len(self.moves)):
-                    self._move_cache(t, g, True)
+                self._move_cache(t, g, True)
+                self._moved_recorded[t][g].set()
+        except BaseException as e:                              # surface the failure in the launching thread
+            self._fail(e)
+
+    def _finisher(self, K):
+        """Batch after batch: once every cache has enqueued its data path and the launching thread has recorded
+        the previous backward, enqueue the repair and the batch's ready event."""
+        try:
+            torch.cuda.set_device(self.dev)
+            for t in range(K):
+                for f in self._moved_recorded[t]:
+                    f.wait()
                 if t >= 1:
                     self._bwd_recorded[t - 1].wait()            # the repair waits for that event on the device
+                if self._stop.is_set() or self._worker_error is not None:
+                    return
                 self._finish_move(t)
                 self._ready_recorded[t].set()
-        except BaseException as e:                              # surface the failure in the launching thread
-            self._worker_error = e
-            for f in self._ready_recorded:
-                f.set()
+        except BaseException as e:
+            self._fail(e)
 
     def _wait_ready_recorded(self, t):
-        if self._thread is not None:
+        if self._threads:
             self._ready_recorded[t].wait()
             if self._worker_error is not None:
                 raise self._worker_error
@@ -206,7 +228,7 @@ class CachedTrainer:
         self.ev_bwd = [torch.cuda.Event() for _ in range(K)]
         self.ev_moved = [[torch.cuda.Event() for _ in range(n_c)] for _ in range(K)]
         self._host_counters = torch.zeros((K, n_c, mb.NUM_COUNTERS), dtype=torch.int64).pin_memory()
-        self._thread = None
+        self._threads = []
         self._worker_error = None
         if out is None:
             out = torch.empty((m.spec.batch, m.spec.total_dim), dtype=torch.float32, device=self.dev)
@@ -236,18 +258,23 @@ class CachedTrainer:
         # the side streams must see the inputs produced on the main stream
         start = torch.cuda.Event()
         start.record(self.main)
-        for s in [self.tag, self.fix, self.copy] + self.moves:
+        for s in [self.tag, self.fix] + self.copies + self.moves:
             s.wait_event(start)
         if self.host_gather:
-            self._jobs: "queue.Queue" = queue.Queue()
+            self._jobs = [queue.Queue() for _ in range(n_c)]
             self._ready_recorded = [threading.Event() for _ in range(K)]
             self._bwd_recorded = [threading.Event() for _ in range(K)]
-            self._thread = threading.Thread(target=self._worker, daemon=True)
-            self._thread.start()
+            self._moved_recorded = [[threading.Event() for _ in range(n_c)] for _ in range(K)]
+            self._stop = threading.Event()
+            self._threads = [threading.Thread(target=self._cache_worker, args=(g,), daemon=True) for g in range(n_c)]
+            self._threads.append(threading.Thread(target=self._finisher, args=(K,), daemon=True))
+            for th in self._threads:
+                th.start()
 
         def move(t):
-            if self._thread is not None:
-                self._jobs.put(t)          # ev_tags[t] has been recorded by this thread already
+            if self._threads:
+                for q in self._jobs:
+                    q.put(t)               # ev_tags[t] has been recorded by this thread already
             else:
                 self._move(t)
 
@@ -261,7 +288,7 @@ class CachedTrainer:
                 self.main.wait_event(self.ev_ready[t])
                 train(t)
                 self.ev_bwd[t].record(self.main)
-                if self._thread is not None:
+                if self._threads:
                     self._bwd_recorded[t].set()
                 if t + 1 < K:
                     move(t + 1)
@@ -270,13 +297,20 @@ class CachedTrainer:
                 if on_step is not None:
                     on_step(t)
         finally:
-            if self._thread is not None:
-                for f in self._bwd_recorded:       # on an error in this thread: do not leave the worker waiting
+            if self._threads:
+                if any(not f.is_set() for f in self._ready_recorded):      # an error in this thread: release the others
+                    self._stop.set()
+                for f in self._bwd_recorded:
                     f.set()
-                self._jobs.put(None)
-                self._thread.join()
-                self._thread = None
-        for s in [self.tag, self.fix, self.copy] + self.moves:
+                for q in self._jobs:
+                    q.put(None)
+                for row in self._moved_recorded:
+                    for f in row:
+                        f.set()
+                for th in self._threads:
+                    th.join()
+                self._threads = []
+        for s in [self.tag, self.fix] + self.copies + self.moves:
             self.main.wait_stream(s)
         torch.cuda.synchronize(self.dev)
         self.history.extend(self._host_counters.numpy().copy())

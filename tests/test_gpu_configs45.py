@@ -55,7 +55,8 @@ def test_config4_structure_200_batches_pipelined():
     stream = wl.BatchStream(spec)
     host_batches = [stream.next() for _ in range(K)]
     n_max = max(len(b[0]) for b in host_batches)
-    grads = [to_dev(wl.gen_grad(spec, k)) for k in range(4)]
+    grads_h = [wl.gen_grad(spec, k) for k in range(4)]
+    grads = [to_dev(g) for g in grads_h]
     glist = [grads[k % 4] for k in range(K)]
     batches = [(to_dev(i), to_dev(o), o) for i, o in host_batches]
     groups = spec.dim_groups()
@@ -165,7 +166,7 @@ def test_config4_structure_200_batches_pipelined():
                 bag_of = np.repeat(np.arange(B), lens)
                 sub_idx = np.searchsorted(sample, seg[keep])
                 sub_off = np.concatenate([[0], np.cumsum(np.bincount(bag_of[keep], minlength=B))]).astype(np.int64)
-                gk = np.ascontiguousarray(wl.gen_grad(spec, k % 4)[:, spec.out_offset[t]:spec.out_offset[t + 1]])
+                gk = np.ascontiguousarray(grads_h[k % 4][:, spec.out_offset[t]:spec.out_offset[t + 1]])
                 smag = np.zeros(Wsub.size, np.float64)
                 W_before = np.abs(Wsub.astype(np.float64))
                 oracle.tbe_backward_rowwise_adagrad(spec.dtype, [dim], [0], [0], [0, len(sample)], Wsub, msub, B, sub_idx,
