@@ -533,7 +533,10 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
 
     t_setup = time.time()
     policy = mb.POLICY_LFU if args.policy == "lfu" else mb.POLICY_LRU
-    model = DeviceModel(spec, device=dev, lock_depth=args.lock_depth, policy=policy)
+    two_level = args.l2_fraction > 0.0
+    if two_level:        # two cache levels run the sequential schedule with kernel data movement
+        args.sequential, args.fetch, args.lock_depth = True, "sm", 0
+    model = DeviceModel(spec, device=dev, lock_depth=args.lock_depth, policy=policy, l2_fraction=args.l2_fraction)
     h2d_gbs, d2h_gbs = host_link_bandwidth(dev)
     stream = wl.BatchStream(spec)
     K = warmup + steps
@@ -634,6 +637,17 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
                      "traffic": None, "peak_source": peak_src},
         "clocks": clocks, "gpu_launches": int(launches), "kernels": kernels,
     }
+    if two_level:
+        l2_hits = float(hist[:, :, 10].sum())
+        rec["two_level"] = {"l2_fraction": args.l2_fraction, "l1_hit_rate_per_lookup": hit,
+                            "l2_hit_rate_per_lookup": l2_hits / max(lookups, 1.0),
+                            "store_rate_per_lookup": 1.0 - hit - l2_hits / max(lookups, 1.0),
+                            "promoted_rows_per_step": float(hist[:, :, 12].sum()) / steps,
+                            "demoted_rows_per_step": float(hist[:, :, 13].sum()) / steps,
+                            "l2_evicted_rows_per_step": float(hist[:, :, 14].sum()) / steps,
+                            "l2_bypass_rows_per_step": float(hist[:, :, 16].sum()) / steps,
+                            "l2_dropped_rows_per_step": float(hist[:, :, 18].sum()) / steps,
+                            "schedule": "sequential, rows moved by kernels"}
     model.close()
     del model, trainer, batches, grads, glist
     torch.cuda.empty_cache()
@@ -706,6 +720,9 @@ def main():
     ap.add_argument("--pooling", type=int, default=50, help="cfg5: lookups per bag")
     ap.add_argument("--alpha", type=float, default=1.0, help="cfg5: Zipf exponent")
     ap.add_argument("--cache-fraction", type=float, default=0.10, help="cfg5: cache slots / rows")
+    ap.add_argument("--l2-fraction", type=float, default=0.0,
+                    help="cached workloads: share of the rows a second, exclusive cache level in pinned host memory holds "
+                         "(Section 5.3.2); 0 = one level")
     ap.add_argument("--policy", default="lru", choices=["lru", "lfu"], help="cached workloads: replacement policy (Section 5.5.2)")
     ap.add_argument("--io-dtype", default="f32", choices=["f32", "f16"],
                     help="type of the pooled output and of its gradient (uncached workloads); the headline metric is f32")

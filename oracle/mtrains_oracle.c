@@ -144,9 +144,11 @@ static inline void row_location(int t, int64_t i, int64_t idx, const int32_t* di
 
 /* Pooled lookup.  For every table t and sample b:
  *   out[b, out_offset[t] + d] = sum over the bag's lookups i of W_t[indices[i], d]
- * (mean pooling divides by the bag length; an empty bag gives 0).  A row id that occurs
- * twice in a bag counts twice.  offsets is CSR over bag id t*B + b.
- * mag (nullable, same layout as out, double) receives sum |W| for error bounds. */
+ * (pooling_mode 0; mode 1, mean pooling, divides by the bag length; mode 2, max pooling, takes
+ * the largest of the bag's values in every column instead of their sum; an empty bag gives 0 in
+ * every mode).  A row id that occurs twice in a bag counts twice.  offsets is CSR over bag id
+ * t*B + b.  mag (nullable, same layout as out, double) receives sum |W| (max pooling: the
+ * largest |W|) for error bounds. */
 void orc_tbe_forward(int32_t T, int32_t dtype, const int32_t* dim, const int32_t* out_offset,
                      const int64_t* weight_offset, const void* weights, int32_t B,
                      const int64_t* indices, const int64_t* offsets, int32_t pooling_mode,
@@ -165,8 +167,13 @@ void orc_tbe_forward(int32_t T, int32_t dtype, const int32_t* dim, const int32_t
                     row_location(t, i, indices[i], dim, weight_offset, (void*)weights,
                                  slot_of_lookup, cache_data, &base, &e0, &slot);
                     double w = load_elem(base, dtype, e0 + d);
-                    acc += w;
-                    am += fabs(w);
+                    if (pooling_mode == 2) {
+                        if (i == i0 || w > acc) acc = w;
+                        if (fabs(w) > am) am = fabs(w);
+                    } else {
+                        acc += w;
+                        am += fabs(w);
+                    }
                 }
                 if (pooling_mode == 1 && i1 > i0) { acc /= (double)(i1 - i0); am /= (double)(i1 - i0); }
                 out[(int64_t)b * out_stride + out_offset[t] + d] = (float)acc;

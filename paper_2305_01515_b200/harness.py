@@ -28,9 +28,13 @@ class DeviceModel:
 
     def __init__(self, spec: wl.ModelSpec, device="cuda:0", max_lookups: int = 0, weights: Optional[np.ndarray] = None,
                  lock_depth: int = 0, policy: int = mb.POLICY_LRU, cache_sets: Optional[List[int]] = None,
-                 host_tables: Optional[Sequence[bool]] = None):
+                 host_tables: Optional[Sequence[bool]] = None, l2_fraction: float = 0.0):
+        """l2_fraction > 0: every cache gets a second, exclusive level in pinned host memory holding that share
+        of its table group's rows (two-level hierarchy; sequential schedule only)."""
         self.spec = spec
         self.lock_depth = lock_depth
+        self.l2_fraction = float(l2_fraction)
+        self.l2: List[mb.Cache] = []
         self.device = torch.device(device)
         self.tdtype = torch.float32 if spec.dtype == wl.FP32 else torch.float16
         n_elem = int(spec.weight_offset[-1])
@@ -74,6 +78,11 @@ class DeviceModel:
                 rows_g = int(spec.row_offset[t1] - spec.row_offset[t0])
                 sets = cache_sets[g] if cache_sets is not None else wl.cache_sets_for(rows_g, spec.cache_fraction)
                 self.caches.append(mb.cache_create(sets, rows_g, dim, spec.dtype, policy, lock_depth))
+                if self.l2_fraction > 0.0:
+                    sets2 = wl.cache_sets_for(rows_g, self.l2_fraction)
+                    esz = 4 if spec.dtype == wl.FP32 else 2
+                    rows2 = torch.zeros(sets2 * 32 * dim * esz, dtype=torch.uint8).pin_memory()
+                    self.l2.append(mb.Cache(sets2, rows_g, dim, spec.dtype, policy, lock_depth, host_rows=rows2))
         self.tables = mb.tables_create(spec.dtype, spec.rows, spec.dims, spec.weight_offset[:-1], cache_id,
                                        self.dev_weights, self.host_weights, self.momentum)
         self.cache_data = [c.data_ptr for c in self.caches] if self.cached else None
@@ -96,6 +105,11 @@ class DeviceModel:
         self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=self.device)
         # the cache calls may run on a side stream while backward runs: scratch of their own
         self.cache_ws_bytes = max([mb.cache_workspace_bytes(c, max_lookups) for c in self.caches] + [256])
+        if self.l2:
+            self.cache_ws_bytes = max(mb.cache2_workspace_bytes(a, b, max_lookups, max_lookups) for a, b in zip(self.caches, self.l2))
+            esz = 4 if self.spec.dtype == wl.FP32 else 2
+            self.fetch_staging2 = torch.empty(max_lookups * max(c.dim for c in self.caches) * esz, dtype=torch.uint8,
+                                              device=self.device)
         self.cache_ws = torch.empty(self.cache_ws_bytes, dtype=torch.uint8, device=self.device)
         if self.cached:
             # the victim staging buffer is only used inside one data movement call sequence, so one per
@@ -122,6 +136,22 @@ class DeviceModel:
                 counters=torch.zeros(mb.NUM_COUNTERS, dtype=torch.int64, device=dev),
                 staging=self.staging[g],
                 capacity=cap))
+        if self.l2:
+            # two levels: the lists of mts_cache2_lookup_insert, a key array, a staging buffer for the rows
+            # on their way into the first level; the first ten counters are the one-level counters
+            esz = 4 if self.spec.dtype == wl.FP32 else 2
+            for g, (c, L) in enumerate(zip(self.caches, lists)):
+                cap = L["capacity"] = n
+                two = {name: torch.zeros(cap, dtype=t, device=dev) for name, t in (
+                    ("fetch_keys", torch.int64), ("fetch_slots", torch.int32), ("fetch_src", torch.int32),
+                    ("ev1_keys", torch.int64), ("ev1_slots", torch.int32), ("ev1_dirty", torch.uint8),
+                    ("ev1_dst", torch.int32), ("ev2_keys", torch.int64), ("ev2_slots", torch.int32),
+                    ("ev2_dirty", torch.uint8), ("drop_keys", torch.int64), ("drop_slots", torch.int32),
+                    ("drop_dirty", torch.uint8))}
+                L["two"] = two
+                L["counters2"] = torch.zeros(mb.NUM_COUNTERS2, dtype=torch.int64, device=dev)
+                L["counters"] = L["counters2"][:mb.NUM_COUNTERS]
+                L["keys"] = torch.empty(n, dtype=torch.int64, device=dev)
         # the lookups ordered by row (uint32 bit patterns), written by the tag step and reused by the backward
         return dict(slot=torch.full((n,), -1, dtype=torch.int32, device=dev),
                     sorted_rows=torch.empty(n, dtype=torch.int32, device=dev),
@@ -157,7 +187,7 @@ class DeviceModel:
         self.reserve(N)
         lr = self.spec.lr if lr is None else lr
         eps = self.spec.eps if eps is None else eps
-        if self.all_cached and reuse_tag_order and uniq_rows_out is None:
+        if self.all_cached and reuse_tag_order and uniq_rows_out is None and not self.l2:
             cx = self._ctx(ctx)
             mb.tbe_backward_apply_presorted(
                 self.tables, self.spec.batch, offsets, N, pooling_mode, grad_out, grad_out.shape[1], lr, eps,
@@ -211,6 +241,13 @@ class DeviceModel:
             _, t0, t1 = self.groups[g]
             begin, n = self.group_range(g, offsets_host)
             L = cx["lists"][g]
+            if self.l2:
+                keys = L["keys"][:n]
+                mb.linearize_keys(self.tables, t0, t1, B, indices, offsets, begin, n, keys if n else None, stream)
+                mb.cache2_lookup_insert(c, self.l2[g], keys if n else None, n, step,
+                                        cx["slot"][begin:begin + n] if n else None, L["two"], L["capacity"],
+                                        L["counters2"], self.cache_ws, self.cache_ws_bytes, stream)
+                continue
             mb.cache_lookup_insert_tables(
                 c, self.tables, t0, t1, B, indices, offsets, begin, n, step, cx["slot"], L["miss_keys"],
                 L["miss_slots"], L["evict_keys"], L["evict_slots"], L["evict_dirty"], L["capacity"],
@@ -227,6 +264,11 @@ class DeviceModel:
     def cache_fetch(self, g: int, stream=None, ctx: Optional[int] = None) -> None:
         """Cache g: dirty victims into the staging buffer, then the missed rows from the host tier into their slots."""
         L = self._ctx(ctx)["lists"][g]
+        if self.l2:
+            # two levels: the whole data movement between the levels and the store is one call
+            mb.cache2_move(self.caches[g], self.l2[g], self.host_rows_ptr(g), L["two"], L["capacity"], L["counters2"],
+                           self.fetch_staging2, stream)
+            return
         mb.cache_prefetch_misses(self.caches[g], self.host_rows_ptr(g), L["miss_keys"], L["miss_slots"],
                                  L["evict_slots"], L["evict_dirty"], L["capacity"], L["counters"], L["staging"], stream)
 
@@ -281,6 +323,8 @@ class DeviceModel:
     def cache_writeback(self, g: int, stream=None, ctx: Optional[int] = None) -> None:
         """Cache g: the staged dirty victims back to the host tier (after cache_fetch of the same batch)."""
         L = self._ctx(ctx)["lists"][g]
+        if self.l2:
+            return                               # part of the two-level data movement
         mb.cache_writeback_evicted(self.caches[g], self.host_rows_ptr(g), L["evict_keys"], L["evict_dirty"],
                                    L["capacity"], L["counters"], L["staging"], stream)
 
@@ -302,6 +346,8 @@ class DeviceModel:
     def flush(self, stream=None) -> None:
         for g, c in enumerate(self.caches):
             mb.cache_flush(c, self.host_rows_ptr(g), stream)
+            if self.l2:
+                mb.cache_flush(self.l2[g], self.host_rows_ptr(g), stream)
 
     def weights_numpy(self) -> np.ndarray:
         """All tables back to back, each from the memory that holds it (host-tier tables: call flush first)."""
@@ -319,5 +365,5 @@ class DeviceModel:
 
     def close(self) -> None:
         self.tables.destroy()
-        for c in self.caches:
+        for c in self.caches + self.l2:
             c.destroy()

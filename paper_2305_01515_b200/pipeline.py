@@ -60,6 +60,7 @@ class CachedTrainer:
         assert model.cached
         # the side streams run two batches ahead and keep two overflow lists alive: lock depths 1 and 2
         assert not pipelined or 1 <= model.lock_depth <= 2, "the pipelined schedule needs lock_depth 1 or 2"
+        assert not (model.l2 and (pipelined or host_gather)), "two cache levels: sequential schedule, kernel data movement"
         self.m = model
         self.host_gather = host_gather
         if host_gather:
@@ -117,7 +118,8 @@ class CachedTrainer:
         self._mark("tag_end", t, s)
         with torch.cuda.stream(s):
             for g in range(len(m.caches)):
-                self._host_counters[t, g].copy_(m.ctx[ctx]["lists"][g]["counters"], non_blocking=True)
+                L = m.ctx[ctx]["lists"][g]
+                self._host_counters[t, g].copy_(L["counters2"] if m.l2 else L["counters"], non_blocking=True)
         self.ev_tags[t].record(s)
 
     def _move_cache(self, t, g, via_host):
@@ -227,7 +229,8 @@ class CachedTrainer:
         self.ev_ready = [torch.cuda.Event() for _ in range(K)]
         self.ev_bwd = [torch.cuda.Event() for _ in range(K)]
         self.ev_moved = [[torch.cuda.Event() for _ in range(n_c)] for _ in range(K)]
-        self._host_counters = torch.zeros((K, n_c, mb.NUM_COUNTERS), dtype=torch.int64).pin_memory()
+        n_cnt = mb.NUM_COUNTERS2 if m.l2 else mb.NUM_COUNTERS
+        self._host_counters = torch.zeros((K, n_c, n_cnt), dtype=torch.int64).pin_memory()
         self._threads = []
         self._worker_error = None
         if out is None:

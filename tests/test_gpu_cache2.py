@@ -207,3 +207,43 @@ def test_training_through_two_levels_matches_oracle_and_uncached_run(dtype, S1, 
         assert tot["overflow"] > 0
     assert g.l1.status() == 0 and g.l2.status() == 0 and tables.status() == 0
     o1.close(); o2.close(); g.close(); tables.destroy()
+
+
+def test_two_level_model_equals_uncached_model_bitwise():
+    """Several table groups (two dims), each behind its own pair of levels, through the trainer's sequential
+    schedule: after the flush the host rows and the states equal the all-HBM run bit for bit, and rows really
+    travelled between the levels."""
+    import copy
+
+    from paper_2305_01515_b200.harness import DeviceModel
+    from paper_2305_01515_b200.pipeline import CachedTrainer
+
+    rows, dims = [20000, 9000, 4000, 12000], [64, 64, 128, 128]
+    spec = custom_spec(rows, dims, 256, wl.FP16, [8, 12, 20, 5], [1.05, 0.9, 1.2, 1.0], seed=79)
+    spec.reuse_prob, spec.reuse_window = 0.6, 4
+    stream = wl.BatchStream(spec)
+    K = 12
+    host_batches = [stream.next() for _ in range(K)]
+    grads = [to_dev(wl.gen_grad(spec, k)) for k in range(K)]
+    W0 = wl.all_weights_numpy(spec)
+    n_max = max(len(b[0]) for b in host_batches)
+    plain = DeviceModel(spec, weights=W0, max_lookups=n_max)
+    batches = [(to_dev(i), to_dev(o), o) for i, o in host_batches]
+    for k in range(K):
+        i, o, _ = batches[k]
+        plain.backward(i, o, i.numel(), grads[k])
+    cspec = copy.deepcopy(spec); cspec.cached = True; cspec.cache_fraction = 0.02
+    m = DeviceModel(cspec, weights=W0, lock_depth=0, l2_fraction=0.05, max_lookups=n_max)
+    tr = CachedTrainer(m, pipelined=False)
+    tr.run(batches, grads)
+    m.flush()
+    torch.cuda.synchronize()
+    hist = np.stack(tr.history)
+    assert hist.shape == (K, 2, mb.NUM_COUNTERS2)
+    names = mb.COUNTER_NAMES2
+    assert hist[:, :, names.index("promoted")].sum() > 50 and hist[:, :, names.index("demoted")].sum() > 500
+    assert hist[:, :, names.index("l2_evicted_dirty")].sum() > 0
+    assert (m.weights_numpy().view(np.uint16) == plain.weights_numpy().view(np.uint16)).all()
+    assert torch.equal(m.momentum, plain.momentum)
+    assert all(c.status() == 0 for c in m.caches + m.l2)
+    m.close(); plain.close()

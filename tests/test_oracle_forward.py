@@ -20,7 +20,7 @@ def _oracle_fwd(spec, W, idx, off, mode=0, **kw):
 
 
 @pytest.mark.parametrize("dtype", [wl.FP32, wl.FP16])
-@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("mode", [0, 1, 2])
 def test_forward_vs_python_loops(dtype, mode):
     """Brute force on a tiny input: explicit loops over bags, rows and columns."""
     spec = small_spec(dtype=dtype)
@@ -35,18 +35,19 @@ def test_forward_vs_python_loops(dtype, mode):
             for d in range(D):
                 s = 0.0
                 for i in range(lo, hi):
-                    s += float(W[base + int(idx[i]) * D + d])
+                    w = float(W[base + int(idx[i]) * D + d])
+                    s = (w if i == lo else max(s, w)) if mode == 2 else s + w
                 if mode == 1 and hi > lo:
                     s /= (hi - lo)
                 assert out[b, spec.out_offset[t] + d] == np.float32(s)
 
 
-@pytest.mark.parametrize("mode", ["sum", "mean"])
+@pytest.mark.parametrize("mode", ["sum", "mean", "max"])
 def test_forward_vs_torch_embedding_bag(mode):
     """Special case that is a library routine: per table, torch's embedding_bag in fp64."""
     spec = small_spec(T=3, rows=(50, 31, 17), dims=(16, 8, 32), B=9, pooling=4.0, dtype=wl.FP16, seed=3)
     W, idx, off = _problem(spec)
-    out = _oracle_fwd(spec, W, idx, off, 0 if mode == "sum" else 1)
+    out = _oracle_fwd(spec, W, idx, off, {"sum": 0, "mean": 1, "max": 2}[mode])
     B = spec.batch
     for t in range(spec.T):
         D = int(spec.dims[t])
@@ -134,3 +135,18 @@ def test_half_conversion_matches_numpy():
         ref = xs.astype(np.float16).view(np.uint16)
     for x, r in zip(xs, ref):
         assert oracle.double_to_half(x) == int(r), x
+
+
+def test_max_pooling_closed_forms():
+    """Max pooling (Section 2.1.1 names sum, mean and max): an all-negative table keeps its sign (the maximum
+    is not started from 0), a bag of one row is that row, an empty bag gives 0, a repeated row changes nothing."""
+    spec = small_spec(T=1, rows=(6,), dims=(4,), B=4, dtype=wl.FP32)
+    W = -(np.arange(24, dtype=np.float32) + 1.0)                       # row r = -(4r+1 .. 4r+4)
+    idx = np.array([2, 5, 2, 3, 0, 0, 1], np.int64)
+    off = np.array([0, 3, 4, 4, 7], np.int64)                          # bags: [2,5,2], [3], [], [0,0,1]
+    out, mag = _oracle_fwd(spec, W, idx, off, 2, want_mag=True)
+    np.testing.assert_array_equal(out[0], W.reshape(6, 4)[2])
+    np.testing.assert_array_equal(out[1], W.reshape(6, 4)[3])
+    np.testing.assert_array_equal(out[2], np.zeros(4, np.float32))
+    np.testing.assert_array_equal(out[3], W.reshape(6, 4)[0])
+    np.testing.assert_array_equal(mag[0], np.abs(W.reshape(6, 4)[5]))    # largest magnitude seen in the bag
