@@ -45,6 +45,7 @@ extern "C" {
 
 #define MTS_POOL_SUM 0
 #define MTS_POOL_MEAN 1
+#define MTS_POOL_MAX 2          /* forward only */
 
 #define MTS_POLICY_LRU 0
 #define MTS_POLICY_LFU 1
@@ -139,10 +140,12 @@ int mts_tables_status(mts_tables* tables, int32_t* host_status, void* stream);
 
 /* ---------------------------------------------------------------------------------------
  * Forward: pooled lookup (Section 2.1.1: an embedding operator selects rows of a table and
- * pools them by sum, mean or max; sum and mean are provided).
+ * pools them by sum, mean or max).
  *   out[b, out_offset[t] + d] = sum over the lookups i of bag (t, b) of W_t[indices[i], d]
- * accumulated in fp32; MTS_POOL_MEAN divides by the bag length; an empty bag gives 0; an id
- * that occurs twice in a bag counts twice.
+ * accumulated in fp32; MTS_POOL_MEAN divides by the bag length; MTS_POOL_MAX takes the largest of
+ * the bag's values in every column instead of their sum (forward only: the backward entry points
+ * take sum and mean); an empty bag gives 0 in every mode; an id that occurs twice in a bag counts
+ * twice.
  * slot_of_lookup (int32 [N], may be NULL when no table is cached): for a lookup of a cached
  * table, the cache slot holding its row, or -1 = read the row from the host tier directly.
  * host_cache_data: host array [n_caches] of device pointers to each cache's row storage.
@@ -211,6 +214,12 @@ int mts_tbe_forward_f16(const mts_tables* tables, int32_t B, const int64_t* indi
                         const int64_t* offsets, int64_t N, int32_t pooling_mode,
                         const int32_t* slot_of_lookup, void* const* host_cache_data, int32_t n_caches,
                         void* out_f16, int64_t out_stride, void* stream);
+/* The forward with a bfloat16 output (round to nearest even once, from the fp32 pooled value); layout and
+ * alignment rules as for mts_tbe_forward_f16. */
+int mts_tbe_forward_bf16(const mts_tables* tables, int32_t B, const int64_t* indices,
+                         const int64_t* offsets, int64_t N, int32_t pooling_mode,
+                         const int32_t* slot_of_lookup, void* const* host_cache_data, int32_t n_caches,
+                         void* out_bf16, int64_t out_stride, void* stream);
 int mts_tbe_backward_apply_f16(const mts_tables* tables, int32_t B, const int64_t* offsets, int64_t N,
                                int32_t pooling_mode, const void* grad_out_f16, int64_t grad_stride,
                                float lr, float eps, const int32_t* slot_of_lookup,
@@ -466,6 +475,23 @@ int mts_cache_flush(mts_cache* cache, void* host_rows_mapped, void* stream);
  * and dirty bytes to caller buffers (device); any pointer may be NULL. */
 int mts_cache_export_state(mts_cache* cache, int64_t* tags, int64_t* timestamps, int64_t* counts,
                            uint8_t* dirty, void* stream);
+
+/* The inverse of mts_cache_export_state, for resuming a run (the paper keeps the cache's tags and states in
+ * HBM, Section 5.6, and has no checkpoint format of its own): sets tags (-1 = free way), timestamps, use
+ * counts and dirty bytes from device arrays of num_sets*32 entries and fills the slot of every resident tag
+ * with its row from the host tier.  The rows themselves are not part of the exported state, so export after
+ * mts_cache_flush: then every row of the host tier is current and every dirty byte 0.  The step of the next
+ * mts_cache_lookup_insert must be larger than every imported timestamp.
+ * Errors: INVALID_ARG, ALIGNMENT, CUDA. */
+int mts_cache_import_state(mts_cache* cache, const int64_t* tags, const int64_t* timestamps, const int64_t* counts,
+                           const uint8_t* dirty, const void* host_rows_mapped, void* stream);
+
+/* How many times mts_cache_prefetch_misses polls for a tile of missed rows before it gives up (default and
+ * maximum 2^22; the paper has no counterpart).  When the polls run out the kernel raises bit 0 of
+ * mts_cache_status, waits (bounded by the maximum) until its copies in flight have landed and returns; the
+ * rows of that call are incomplete, the call can simply be repeated.  0 makes every call give up at once:
+ * for testing the error path without hanging anything. */
+int mts_cache_set_fetch_wait_limit(mts_cache* cache, int64_t polls);
 
 #ifdef __cplusplus
 }

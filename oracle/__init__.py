@@ -52,6 +52,7 @@ def lib():
         _lib.orc_cache_lookup_insert.restype = C.c_int64
         _lib.orc_cache_flush.restype = C.c_int64
         _lib.orc_cache2_lookup_insert.restype = C.c_int64
+        _lib.orc_place_tables.restype = C.c_double
         for name in ("orc_cache_tags", "orc_cache_ts", "orc_cache_freq", "orc_cache_dirty",
                      "orc_cache_data"):
             getattr(_lib, name).restype = C.c_void_p
@@ -97,6 +98,19 @@ def double_to_half(x: float) -> int:
 
 def cache_set_of(key: int, S: int) -> int:
     return int(lib().orc_cache_set_of(C.c_int64(int(key)), C.c_int64(int(S))))
+
+
+def place_tables(size_bytes, bytes_per_sample, fast_capacity_bytes: int, bw_fast: float, bw_slow: float):
+    """Brute-force placement of T <= 24 tables over a fast and a slow memory (Eq. 6, one GPU).
+    Returns (placement int32 [T]: 0 fast / 1 slow, minimal time per sample)."""
+    size_bytes = _i64(size_bytes)
+    cost = np.ascontiguousarray(bytes_per_sample, dtype=np.float64)
+    T = len(size_bytes)
+    assert T <= 24
+    out = np.zeros(T, np.int32)
+    t = lib().orc_place_tables(C.c_int32(T), _p(size_bytes), _p(cost), C.c_int64(int(fast_capacity_bytes)),
+                               C.c_double(bw_fast), C.c_double(bw_slow), _p(out))
+    return out, float(t)
 
 
 def eq3_bandwidth(qps, T, D, p, L) -> float:

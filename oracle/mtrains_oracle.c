@@ -18,6 +18,7 @@
  *     fetched rows and eviction of LRU rows back to the lower tier
  *   - prefetch invariant (a prefetched row is not evicted before its batch  Section 5.7
  *     trained), expressed as a lock window on timestamps
+ *   - table placement over two memories by the lookup-time objective        Section 5.6, Eq. 6
  *   - two cache levels, exclusive, over a backing store: promotion of       Section 5.3.2,
  *     second-level hits and fetched rows, demotion of first-level LRU rows,  Section 5.5.4
  *     eviction of second-level LRU rows to the store
@@ -732,6 +733,32 @@ void orc_cache2_move(orc_cache* l1, orc_cache* l2, void* store,
     for (int64_t k = 0; k < n_fetch; ++k)
         memcpy(d1 + (size_t)fetch_slots[k] * rb, tmp + (size_t)k * rb, rb);
     free(tmp);
+}
+
+/* ------------------------------------------------------------------ table placement */
+
+/* Table placement over two memories of one GPU (Section 5.6, Eq. 6): each table goes to exactly one
+ * memory, the tables of the fast memory must fit its capacity, and the lookup time
+ *   time = sum over tables of (D * L * p) / BW of the table's memory
+ * is minimal (Eq. 6 with one GPU, where the maximum over GPUs is the single term).  bytes_per_sample[t]
+ * = D_t * L_t * p.  Brute force over all 2^T assignments (T <= 24).  placement[t] = 0 fast memory, 1 slow
+ * memory.  Returns the minimal time per sample (seconds when the bandwidths are bytes per second). */
+double orc_place_tables(int32_t T, const int64_t* size_bytes, const double* bytes_per_sample,
+                        int64_t fast_capacity_bytes, double bw_fast, double bw_slow, int32_t* placement) {
+    double best = -1.0;
+    uint32_t best_mask = 0;
+    for (uint32_t mask = 0; mask < (1u << T); ++mask) {       /* bit t set = table t in the fast memory */
+        int64_t used = 0;
+        double time = 0.0;
+        for (int32_t t = 0; t < T; ++t) {
+            if ((mask >> t) & 1u) { used += size_bytes[t]; time += bytes_per_sample[t] / bw_fast; }
+            else time += bytes_per_sample[t] / bw_slow;
+        }
+        if (used > fast_capacity_bytes) continue;
+        if (best < 0.0 || time < best) { best = time; best_mask = mask; }
+    }
+    for (int32_t t = 0; t < T; ++t) placement[t] = ((best_mask >> t) & 1u) ? 0 : 1;
+    return best;
 }
 
 /* ------------------------------------------------------------------ analytical models */

@@ -18,7 +18,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CAPACITY, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = (
     -1, -2, -3, -4, -5, -6, -7)
 DTYPE_FP32, DTYPE_FP16 = 0, 1
-POOL_SUM, POOL_MEAN = 0, 1
+POOL_SUM, POOL_MEAN, POOL_MAX = 0, 1, 2
 POLICY_LRU, POLICY_LFU = 0, 1
 MAX_CACHES, CACHE_WAYS, NUM_COUNTERS, NUM_COUNTERS2 = 8, 32, 10, 20
 COUNTER_NAMES2 = ("lookups", "unique", "hit_lookups", "miss_lookups", "unique_hits", "unique_misses", "inserted",
@@ -32,11 +32,11 @@ EXPORTS = (
     "mts_trace_kernel_name", "mts_trace_report", "mts_tables_create", "mts_tables_destroy", "mts_tables_status",
     "mts_tbe_forward", "mts_tbe_backward_workspace_bytes", "mts_tbe_backward_rowwise_adagrad",
     "mts_tbe_backward_rowwise_adagrad_static", "mts_tbe_backward_sort", "mts_tbe_backward_apply",
-    "mts_tbe_forward_f16", "mts_tbe_backward_apply_f16",
+    "mts_tbe_forward_f16", "mts_tbe_forward_bf16", "mts_tbe_backward_apply_f16",
     "mts_cache_create", "mts_cache_destroy", "mts_cache_status", "mts_cache_data", "mts_cache_dirty",
     "mts_linearize_keys", "mts_cache_workspace_bytes", "mts_cache_lookup_insert", "mts_cache_lookup_insert_tables",
     "mts_tbe_backward_apply_presorted", "mts_cache_create_host_level", "mts_cache2_workspace_bytes",
-    "mts_cache2_lookup_insert", "mts_cache2_move",
+    "mts_cache2_lookup_insert", "mts_cache2_move", "mts_cache_import_state", "mts_cache_set_fetch_wait_limit",
     "mts_cache_prefetch_misses", "mts_host_gather_rows", "mts_cache_place_fetched", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
     "mts_cache_export_state",
 )
@@ -93,6 +93,7 @@ def lib():
         L.mts_tbe_backward_apply.argtypes = [vp, i32, vp, i64, i32, vp, i64, f32, f32, vp, C.POINTER(vp),
                                              C.POINTER(vp), i32, vp, sz, vp]
         L.mts_tbe_forward_f16.argtypes = L.mts_tbe_forward.argtypes
+        L.mts_tbe_forward_bf16.argtypes = L.mts_tbe_forward.argtypes
         L.mts_tbe_backward_apply_f16.argtypes = L.mts_tbe_backward_apply.argtypes
         L.mts_cache_create.argtypes = [C.POINTER(vp), i64, i64, i32, i32, i32, i32, i32]
         L.mts_cache_destroy.argtypes = [vp]
@@ -121,6 +122,8 @@ def lib():
         L.mts_cache_place_fetched.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.mts_cache_flush.argtypes = [vp, vp, vp]
         L.mts_cache_export_state.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.mts_cache_import_state.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+        L.mts_cache_set_fetch_wait_limit.argtypes = [vp, i64]
         for name in EXPORTS:
             getattr(L, name)            # raises AttributeError when a declared symbol is missing
         _lib = L
@@ -220,10 +223,11 @@ def tables_create(dtype, rows, dim, weight_offset, cache_id, dev_weights, host_w
 
 
 def tbe_forward(tables: Tables, B: int, indices, offsets, N: int, pooling_mode: int, slot_of_lookup,
-                cache_data: Optional[Sequence], out, out_stride: int, stream=None, f16: bool = False) -> None:
-    """f16: `out` holds IEEE binary16 (mts_tbe_forward_f16), else fp32."""
+                cache_data: Optional[Sequence], out, out_stride: int, stream=None, f16: bool = False,
+                bf16: bool = False) -> None:
+    """f16 / bf16: `out` holds IEEE binary16 / bfloat16 (mts_tbe_forward_f16 / _bf16), else fp32."""
     n_caches = len(cache_data) if cache_data is not None else 0
-    fn = lib().mts_tbe_forward_f16 if f16 else lib().mts_tbe_forward
+    fn = lib().mts_tbe_forward_bf16 if bf16 else lib().mts_tbe_forward_f16 if f16 else lib().mts_tbe_forward
     _check(fn(tables.handle, B, _ptr(indices), _ptr(offsets), N, pooling_mode,
                                  _ptr(slot_of_lookup), _ptr_array(cache_data, n_caches), n_caches, _ptr(out),
                                  out_stride, _stream(stream)))
@@ -432,6 +436,15 @@ def cache_writeback_evicted(cache: Cache, host_rows_mapped, evict_keys, evict_di
 
 def cache_flush(cache: Cache, host_rows_mapped, stream=None) -> None:
     _check(lib().mts_cache_flush(cache.handle, _ptr(host_rows_mapped), _stream(stream)))
+
+
+def cache_import_state(cache: Cache, tags, timestamps, counts, dirty, host_rows_mapped, stream=None) -> None:
+    _check(lib().mts_cache_import_state(cache.handle, _ptr(tags), _ptr(timestamps), _ptr(counts), _ptr(dirty),
+                                        _ptr(host_rows_mapped), _stream(stream)))
+
+
+def cache_set_fetch_wait_limit(cache: Cache, polls: int) -> None:
+    _check(lib().mts_cache_set_fetch_wait_limit(cache.handle, polls))
 
 
 def cache_export_state(cache: Cache, tags, timestamps, counts, dirty, stream=None) -> None:

@@ -31,6 +31,7 @@ struct mts_cache {
   uint8_t* dirty = nullptr;      // [S*32]
   char* data = nullptr;          // [S*32, row_bytes]  HBM, or pinned host memory of the caller (a second level)
   bool owns_data = true;
+  uint32_t fetch_wait_limit = 1u << 22;   // polls the bulk-copy fetch waits for a tile before it gives up
   int32_t* d_status = nullptr;   // sticky status bits (bit 0: a bounded wait on a bulk copy ran out)
 };
 
@@ -770,7 +771,8 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 __global__ void __launch_bounds__(FETCH_THREADS)
 cache_fetch_misses_bulk(char* __restrict__ data, int row_bytes, const char* __restrict__ host_rows,
                         const int64_t* __restrict__ miss_keys, const int32_t* __restrict__ miss_slots,
-                        const int64_t* __restrict__ counters, int64_t capacity, int32_t* status) {
+                        const int64_t* __restrict__ counters, int64_t capacity, int32_t* status,
+                        uint32_t wait_limit) {
   __shared__ __align__(128) unsigned char tile[FETCH_TILE_BYTES];
   __shared__ __align__(8) unsigned long long bar_storage;
   const int64_t n = list_len(counters, MTS_CNT_INSERTED, capacity);
@@ -802,8 +804,10 @@ cache_fetch_misses_bulk(char* __restrict__ data, int row_bytes, const char* __re
                      : "memory");
       }
     }
-    bool ok = mbar_wait_bounded(bar, parity, FETCH_WAIT_LIMIT);
+    bool ok = mbar_wait_bounded(bar, parity, wait_limit);
     if (!__syncthreads_and(ok)) {
+      // give up on this call: say so, but leave only when the copies in flight have landed (bounded as
+      // well), so that nothing writes into this block's shared memory after it is gone
       if (threadIdx.x == 0) atomicOr(status, CACHE_STATUS_FETCH_TIMEOUT);
       mbar_wait_bounded(bar, parity, FETCH_WAIT_LIMIT);
       return;
@@ -1487,7 +1491,7 @@ extern "C" int mts_cache_prefetch_misses(mts_cache* c, const void* host_rows_map
 #else
     cache_fetch_misses_bulk<<<MTS_FETCH_BLOCKS, FETCH_THREADS, 0, s>>>(
         c->data, c->row_bytes, static_cast<const char*>(host_rows_mapped), miss_keys, miss_slots, counters,
-        list_capacity, c->d_status);
+        list_capacity, c->d_status, c->fetch_wait_limit);
 #endif
   }
   return check_launch("cache_save_victims / cache_fetch_misses");
@@ -1594,6 +1598,55 @@ extern "C" int mts_cache_flush(mts_cache* c, void* host_rows_mapped, void* strea
     cache_clear_dirty<<<c->sm_count * 4, 256, 0, s>>>(c->dirty, n);
   }
   return check_launch("cache_flush");
+}
+
+namespace mts {
+__global__ void cache_import(const int64_t* __restrict__ i_tags, const int64_t* __restrict__ i_ts,
+                             const int64_t* __restrict__ i_freq, const uint8_t* __restrict__ i_dirty, int64_t n,
+                             uint32_t* tags, int32_t* ts, int32_t* placed, uint32_t* freq, uint8_t* dirty) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const bool free_way = i_tags[i] < 0;
+    tags[i] = free_way ? FREE_TAG : (uint32_t)i_tags[i];
+    ts[i] = free_way ? -1 : (int32_t)i_ts[i];
+    placed[i] = ts[i];            // inserted no later than its last use: never equal to a later call's step
+    freq[i] = free_way ? 0u : (uint32_t)i_freq[i];
+    dirty[i] = free_way ? 0 : i_dirty[i];
+  }
+}
+
+__global__ void __launch_bounds__(CACHE_THREADS)
+cache_refill_rows(char* __restrict__ data, int row_bytes, const uint32_t* __restrict__ tags, int64_t n_slots,
+                  const char* __restrict__ host_rows) {
+  copy_rows(n_slots, row_bytes / 16,
+            [&](int64_t s) { return tags[s] != FREE_TAG ? host_rows + (int64_t)tags[s] * row_bytes : nullptr; },
+            [&](int64_t s) { return data + s * row_bytes; });
+}
+}  // namespace mts
+
+extern "C" int mts_cache_import_state(mts_cache* c, const int64_t* tags, const int64_t* timestamps, const int64_t* counts,
+                                      const uint8_t* dirty, const void* host_rows_mapped, void* stream) {
+  if (!c || !tags || !timestamps || !counts || !dirty || !host_rows_mapped)
+    return set_error(MTS_ERR_INVALID_ARG, "cache_import_state: null argument");
+  if ((uintptr_t)host_rows_mapped & 15) return set_error(MTS_ERR_ALIGNMENT, "cache_import_state: host buffer alignment");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int64_t n = c->S * MTS_CACHE_WAYS;
+  {
+    LaunchScope scope(K_OTHER, s);
+    cache_import<<<c->sm_count * 4, 256, 0, s>>>(tags, timestamps, counts, dirty, n, c->tags, c->ts, c->placed, c->freq,
+                                                 c->dirty);
+  }
+  {
+    LaunchScope scope(K_CACHE_FETCH_MISSES, s);
+    cache_refill_rows<<<c->sm_count * 8, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, c->tags, n,
+                                                                static_cast<const char*>(host_rows_mapped));
+  }
+  return check_launch("cache_import_state");
+}
+
+extern "C" int mts_cache_set_fetch_wait_limit(mts_cache* c, int64_t polls) {
+  if (!c || polls < 0 || polls > (1ll << 22)) return set_error(MTS_ERR_INVALID_ARG, "cache_set_fetch_wait_limit: 0 .. 2^22 polls");
+  c->fetch_wait_limit = (uint32_t)polls;
+  return MTS_OK;
 }
 
 extern "C" int mts_cache_export_state(mts_cache* c, int64_t* tags, int64_t* timestamps, int64_t* counts,

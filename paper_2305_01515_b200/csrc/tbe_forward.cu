@@ -5,6 +5,8 @@
 // Accumulation in fp32 registers, one 16-byte store per lane group member at the end.
 #include <type_traits>
 
+#include <cuda_bf16.h>
+
 #include "common.cuh"
 
 namespace mts {
@@ -26,19 +28,67 @@ constexpr int FWD_UNROLL = MTS_FWD_UNROLL;
 constexpr int FWD_BAGS = MTS_FWD_BAGS;
 static_assert(FWD_BAGS >= 1 && FWD_BAGS <= 30, "a warp keeps the offsets of its bags in its lanes");
 
+// Pooled values leave as fp32, IEEE binary16 or bfloat16 (round to nearest even).
+enum OutKind { OUT_F32 = 0, OUT_F16 = 1, OUT_BF16 = 2 };
+
+// One lane's EPC consecutive pooled values (already scaled) to element offset `o` of `out`.
+template <int EPC>
+__device__ __forceinline__ void store_pooled(void* __restrict__ out, int out_kind, int64_t o, const float (&v)[EPC]) {
+  if (out_kind == OUT_F32) {
+    float4* dst = reinterpret_cast<float4*>(static_cast<float*>(out) + o);
+    dst[0] = make_float4(v[0], v[1], v[2], v[3]);
+    if (EPC == 8) dst[1] = make_float4(v[4], v[5], v[6], v[7]);
+    return;
+  }
+  uint32_t w[EPC / 2];
+#pragma unroll
+  for (int e = 0; e < EPC / 2; ++e) {
+    if (out_kind == OUT_F16) {
+      __half2 h = __floats2half2_rn(v[2 * e], v[2 * e + 1]);
+      w[e] = *reinterpret_cast<uint32_t*>(&h);
+    } else {
+      __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+      w[e] = *reinterpret_cast<uint32_t*>(&h);
+    }
+  }
+  uint16_t* dst = static_cast<uint16_t*>(out) + o;
+  *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);
+  if (EPC == 8) *reinterpret_cast<uint2*>(dst + 4) = make_uint2(w[2], w[3]);
+}
+
+// max pooling: acc = max(acc, value) per column; a piece that is not loaded is filled with -infinity
+__device__ __forceinline__ void max_half8(float* acc, const uint4& v) {
+  const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float2 f = __half22float2(h[e]);
+    acc[2 * e] = fmaxf(acc[2 * e], f.x);
+    acc[2 * e + 1] = fmaxf(acc[2 * e + 1], f.y);
+  }
+}
+__device__ __forceinline__ void max_float4(float* acc, const uint4& v) {
+  acc[0] = fmaxf(acc[0], __uint_as_float(v.x));
+  acc[1] = fmaxf(acc[1], __uint_as_float(v.y));
+  acc[2] = fmaxf(acc[2], __uint_as_float(v.z));
+  acc[3] = fmaxf(acc[3], __uint_as_float(v.w));
+}
+
 // A warp walks FWD_BAGS consecutive bags.  Their offsets are read with one load, and the first 32
 // indices of the next bag are requested before the rows of the current bag, so that a bag costs
 // about one memory round trip (its rows) instead of three (offsets, indices, rows).
-template <bool FP16, int NV>
+template <bool FP16, int NV, bool MAXP>
 __global__ void __launch_bounds__(FWD_WARPS * 32, (NV == 1 ? MTS_FWD_MINBLK : 1))
 tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B,
                    const int64_t* __restrict__ indices, const int64_t* __restrict__ offsets,
                    const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches,
                    const char* __restrict__ dev_w, const char* __restrict__ host_w,
-                   int32_t pooling_mode, void* __restrict__ out, bool out_half, int64_t out_stride,
+                   int32_t pooling_mode, void* __restrict__ out, int out_kind, int64_t out_stride,
                    int32_t* status) {
   constexpr int EPC = FP16 ? 8 : 4;       // elements per 16-byte chunk
   constexpr int EB = FP16 ? 2 : 4;
+  // what an accumulator starts from and a piece that is not loaded holds: 0, or -infinity for max pooling
+  const float acc0 = MAXP ? __uint_as_float(0xff800000u) : 0.f;
+  const uint32_t pad = MAXP ? (FP16 ? 0xfc00fc00u : 0xff800000u) : 0u;
   const int lane = threadIdx.x & 31;
   const int64_t bag0 = ((int64_t)blockIdx.x * FWD_WARPS + (threadIdx.x >> 5)) * FWD_BAGS;
   if (bag0 >= n_bags) return;
@@ -102,7 +152,7 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
 #pragma unroll
     for (int v = 0; v < NV; ++v)
 #pragma unroll
-      for (int e = 0; e < EPC; ++e) acc[v][e] = 0.f;
+      for (int e = 0; e < EPC; ++e) acc[v][e] = acc0;
 
     for (int64_t base = i0; base < i1; base += 32) {
       const int cnt = (int)min((int64_t)32, i1 - base);
@@ -132,15 +182,20 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
             for (int q = 0; q < (WHOLE ? 1 : NV); ++q) {
               const int c = cl + q * 32;
               if (valid && (WHOLE || c < vec16)) v[u][q] = ld_nc_16(reinterpret_cast<const char*>(p) + (int64_t)c * 16);
-              else v[u][q] = make_uint4(0u, 0u, 0u, 0u);
+              else v[u][q] = make_uint4(pad, pad, pad, pad);
             }
           }
 #pragma unroll
           for (int u = 0; u < FWD_UNROLL; ++u)
 #pragma unroll
             for (int q = 0; q < (WHOLE ? 1 : NV); ++q) {
-              if (FP16) add_half8(acc[q], v[u][q]);
-              else add_float4(acc[q], v[u][q]);
+              if (MAXP) {
+                if (FP16) max_half8(acc[q], v[u][q]);
+                else max_float4(acc[q], v[u][q]);
+              } else {
+                if (FP16) add_half8(acc[q], v[u][q]);
+                else add_float4(acc[q], v[u][q]);
+              }
             }
         }
       };
@@ -152,7 +207,10 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
 #pragma unroll
       for (int q = 0; q < NV; ++q)
 #pragma unroll
-        for (int e = 0; e < EPC; ++e) acc[q][e] += __shfl_xor_sync(0xffffffffu, acc[q][e], o);
+        for (int e = 0; e < EPC; ++e) {
+          const float other = __shfl_xor_sync(0xffffffffu, acc[q][e], o);
+          acc[q][e] = MAXP ? fmaxf(acc[q][e], other) : acc[q][e] + other;
+        }
     }
     if (sub == 0) {
       float scale = 1.f;
@@ -162,29 +220,10 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
       for (int q = 0; q < NV; ++q) {
         const int c = cl + q * 32;
         if (c < vec16) {
-          if (out_half) {
-            // pooled sums rounded to fp16 (round to nearest even), EPC values = EPC * 2 bytes
-            __half2 h01 = __floats2half2_rn(acc[q][0] * scale, acc[q][1] * scale);
-            __half2 h23 = __floats2half2_rn(acc[q][2] * scale, acc[q][3] * scale);
-            uint2 lo;
-            lo.x = *reinterpret_cast<uint32_t*>(&h01);
-            lo.y = *reinterpret_cast<uint32_t*>(&h23);
-            __half* dst = static_cast<__half*>(out) + o + c * EPC;
-            *reinterpret_cast<uint2*>(dst) = lo;
-            if (FP16) {
-              __half2 h45 = __floats2half2_rn(acc[q][4] * scale, acc[q][5] * scale);
-              __half2 h67 = __floats2half2_rn(acc[q][6] * scale, acc[q][7] * scale);
-              uint2 hi;
-              hi.x = *reinterpret_cast<uint32_t*>(&h45);
-              hi.y = *reinterpret_cast<uint32_t*>(&h67);
-              *reinterpret_cast<uint2*>(dst + 4) = hi;
-            }
-          } else {
-            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(out) + o + c * EPC);
-            dst[0] = make_float4(acc[q][0] * scale, acc[q][1] * scale, acc[q][2] * scale, acc[q][3] * scale);
-            if (FP16)
-              dst[1] = make_float4(acc[q][4] * scale, acc[q][5] * scale, acc[q][6] * scale, acc[q][7] * scale);
-          }
+          float r[EPC];
+#pragma unroll
+          for (int e = 0; e < EPC; ++e) r[e] = MAXP ? (i1 > i0 ? acc[q][e] : 0.f) : acc[q][e] * scale;
+          store_pooled<EPC>(out, out_kind, o + c * EPC, r);
         }
       }
     }
@@ -194,15 +233,21 @@ tbe_forward_kernel(const TableMeta* __restrict__ meta, int64_t n_bags, int32_t B
 template <bool FP16, int NV>
 static int launch_forward(const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets,
                           int32_t pooling_mode, const int32_t* slot_of_lookup, const CachePtrs& caches,
-                          void* out, bool out_half, int64_t out_stride, cudaStream_t stream) {
+                          void* out, int out_kind, int64_t out_stride, cudaStream_t stream) {
   const int64_t n_bags = (int64_t)h->T * B;
   const int64_t grid = ceil_div(n_bags, (int64_t)FWD_WARPS * FWD_BAGS);
   {
     LaunchScope scope(K_FORWARD, stream);
-    tbe_forward_kernel<FP16, NV><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
-        h->d_meta, n_bags, B, indices, offsets, slot_of_lookup, caches,
-        static_cast<const char*>(h->dev_weights), static_cast<const char*>(h->host_weights), pooling_mode,
-        out, out_half, out_stride, h->d_status);
+    if (pooling_mode == MTS_POOL_MAX)
+      tbe_forward_kernel<FP16, NV, true><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
+          h->d_meta, n_bags, B, indices, offsets, slot_of_lookup, caches,
+          static_cast<const char*>(h->dev_weights), static_cast<const char*>(h->host_weights), pooling_mode,
+          out, out_kind, out_stride, h->d_status);
+    else
+      tbe_forward_kernel<FP16, NV, false><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
+          h->d_meta, n_bags, B, indices, offsets, slot_of_lookup, caches,
+          static_cast<const char*>(h->dev_weights), static_cast<const char*>(h->host_weights), pooling_mode,
+          out, out_kind, out_stride, h->d_status);
   }
   return check_launch("tbe_forward_kernel");
 }
@@ -227,7 +272,7 @@ template <bool FP16>
 __global__ void __launch_bounds__(FWD_WARPS * 32, MTS_FWD_LEAN_MINBLK)
 tbe_forward_lean(const TableMeta* __restrict__ meta, int32_t n_bags, int32_t B,
                  const int64_t* __restrict__ indices, const int64_t* __restrict__ offsets,
-                 const char* __restrict__ dev_w, int32_t pooling_mode, void* __restrict__ out, bool out_half,
+                 const char* __restrict__ dev_w, int32_t pooling_mode, void* __restrict__ out, int out_kind,
                  int64_t out_stride, int32_t* status) {
   constexpr int EPC = FP16 ? 8 : 4;       // elements per 16-byte chunk
   constexpr int EB = FP16 ? 2 : 4;
@@ -320,35 +365,17 @@ tbe_forward_lean(const TableMeta* __restrict__ meta, int32_t n_bags, int32_t B,
       float scale = 1.f;
       if (pooling_mode == MTS_POOL_MEAN && i1 > i0) scale = 1.f / (float)(i1 - i0);
       const int64_t o = (int64_t)b * out_stride + out_offset + cl * EPC;     // first element of the lane's piece
-      if (out_half) {
-        // pooled sums rounded to fp16 (round to nearest even)
-        __half2 h01 = __floats2half2_rn(acc[0] * scale, acc[1] * scale);
-        __half2 h23 = __floats2half2_rn(acc[2] * scale, acc[3] * scale);
-        uint2 lo;
-        lo.x = *reinterpret_cast<uint32_t*>(&h01);
-        lo.y = *reinterpret_cast<uint32_t*>(&h23);
-        __half* dst = static_cast<__half*>(out) + o;
-        *reinterpret_cast<uint2*>(dst) = lo;
-        if (FP16) {
-          __half2 h45 = __floats2half2_rn(acc[4] * scale, acc[5] * scale);
-          __half2 h67 = __floats2half2_rn(acc[6] * scale, acc[7] * scale);
-          uint2 hi;
-          hi.x = *reinterpret_cast<uint32_t*>(&h45);
-          hi.y = *reinterpret_cast<uint32_t*>(&h67);
-          *reinterpret_cast<uint2*>(dst + 4) = hi;
-        }
-      } else {
-        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(out) + o);
-        dst[0] = make_float4(acc[0] * scale, acc[1] * scale, acc[2] * scale, acc[3] * scale);
-        if (FP16) dst[1] = make_float4(acc[4] * scale, acc[5] * scale, acc[6] * scale, acc[7] * scale);
-      }
+      float r[EPC];
+#pragma unroll
+      for (int e = 0; e < EPC; ++e) r[e] = acc[e] * scale;
+      store_pooled<EPC>(out, out_kind, o, r);
     }
   }
 }
 
 template <bool FP16>
 static int launch_forward_lean(const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets,
-                               int32_t pooling_mode, void* out, bool out_half, int64_t out_stride,
+                               int32_t pooling_mode, void* out, int out_kind, int64_t out_stride,
                                cudaStream_t stream) {
   const int64_t n_bags = (int64_t)h->T * B;
   const int64_t grid = ceil_div(n_bags, (int64_t)FWD_WARPS * FWD_BAGS);
@@ -356,7 +383,7 @@ static int launch_forward_lean(const mts_tables* h, int32_t B, const int64_t* in
     LaunchScope scope(K_FORWARD, stream);
     tbe_forward_lean<FP16><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
         h->d_meta, (int32_t)n_bags, B, indices, offsets, static_cast<const char*>(h->dev_weights), pooling_mode, out,
-        out_half, out_stride, h->d_status);
+        out_kind, out_stride, h->d_status);
   }
   return check_launch("tbe_forward_lean");
 }
@@ -385,10 +412,10 @@ using namespace mts;
 namespace {
 int forward_any(const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets, int64_t N,
                 int32_t pooling_mode, const int32_t* slot_of_lookup, void* const* host_cache_data, int32_t n_caches,
-                void* out, bool out_half, int64_t out_stride, void* stream) {
+                void* out, int out_kind, int64_t out_stride, void* stream) {
   if (!h || !offsets || !out || B < 1 || N < 0 || (N > 0 && !indices))
     return set_error(MTS_ERR_INVALID_ARG, "tbe_forward: null argument or bad size");
-  if (pooling_mode != MTS_POOL_SUM && pooling_mode != MTS_POOL_MEAN)
+  if (pooling_mode != MTS_POOL_SUM && pooling_mode != MTS_POOL_MEAN && pooling_mode != MTS_POOL_MAX)
     return set_error(MTS_ERR_INVALID_ARG, "tbe_forward: pooling mode %d", pooling_mode);
   if (out_stride < h->total_dim || (out_stride & 3) || ((uintptr_t)out & 15))
     return set_error(MTS_ERR_ALIGNMENT, "tbe_forward: out must be 16-byte aligned, out_stride >= %d and a multiple of 4",
@@ -404,12 +431,13 @@ int forward_any(const mts_tables* h, int32_t B, const int64_t* indices, const in
   const bool fp16 = h->dtype == MTS_DTYPE_FP16;
 #if MTS_FWD_LEAN
   // positions and bag numbers fit 32 bits (row numbers always do), no cached table, rows of at most 32 pieces
-  if (!h->any_cached && nv == 1 && N < (1ll << 31) && (int64_t)h->T * B < (1ll << 31) - FWD_WARPS * FWD_BAGS) {
-    if (fp16) return launch_forward_lean<true>(h, B, indices, offsets, pooling_mode, out, out_half, out_stride, s);
-    return launch_forward_lean<false>(h, B, indices, offsets, pooling_mode, out, out_half, out_stride, s);
+  if (!h->any_cached && nv == 1 && pooling_mode != MTS_POOL_MAX && N < (1ll << 31) &&
+      (int64_t)h->T * B < (1ll << 31) - FWD_WARPS * FWD_BAGS) {
+    if (fp16) return launch_forward_lean<true>(h, B, indices, offsets, pooling_mode, out, out_kind, out_stride, s);
+    return launch_forward_lean<false>(h, B, indices, offsets, pooling_mode, out, out_kind, out_stride, s);
   }
 #endif
-#define MTS_FWD(F, V) return launch_forward<F, V>(h, B, indices, offsets, pooling_mode, slot_of_lookup, caches, out, out_half, out_stride, s)
+#define MTS_FWD(F, V) return launch_forward<F, V>(h, B, indices, offsets, pooling_mode, slot_of_lookup, caches, out, out_kind, out_stride, s)
   if (fp16) {
     if (nv == 1) MTS_FWD(true, 1);
     if (nv == 2) MTS_FWD(true, 2);
@@ -428,7 +456,7 @@ extern "C" int mts_tbe_forward(const mts_tables* h, int32_t B, const int64_t* in
                                const int64_t* offsets, int64_t N, int32_t pooling_mode,
                                const int32_t* slot_of_lookup, void* const* host_cache_data,
                                int32_t n_caches, float* out, int64_t out_stride, void* stream) {
-  return forward_any(h, B, indices, offsets, N, pooling_mode, slot_of_lookup, host_cache_data, n_caches, out, false,
+  return forward_any(h, B, indices, offsets, N, pooling_mode, slot_of_lookup, host_cache_data, n_caches, out, OUT_F32,
                      out_stride, stream);
 }
 
@@ -436,6 +464,14 @@ extern "C" int mts_tbe_forward_f16(const mts_tables* h, int32_t B, const int64_t
                                    const int64_t* offsets, int64_t N, int32_t pooling_mode,
                                    const int32_t* slot_of_lookup, void* const* host_cache_data,
                                    int32_t n_caches, void* out_f16, int64_t out_stride, void* stream) {
-  return forward_any(h, B, indices, offsets, N, pooling_mode, slot_of_lookup, host_cache_data, n_caches, out_f16, true,
+  return forward_any(h, B, indices, offsets, N, pooling_mode, slot_of_lookup, host_cache_data, n_caches, out_f16, OUT_F16,
+                     out_stride, stream);
+}
+
+extern "C" int mts_tbe_forward_bf16(const mts_tables* h, int32_t B, const int64_t* indices,
+                                    const int64_t* offsets, int64_t N, int32_t pooling_mode,
+                                    const int32_t* slot_of_lookup, void* const* host_cache_data,
+                                    int32_t n_caches, void* out_bf16, int64_t out_stride, void* stream) {
+  return forward_any(h, B, indices, offsets, N, pooling_mode, slot_of_lookup, host_cache_data, n_caches, out_bf16, OUT_BF16,
                      out_stride, stream);
 }

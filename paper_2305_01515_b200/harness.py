@@ -176,7 +176,7 @@ class DeviceModel:
             out = torch.empty((self.spec.batch, self.spec.total_dim), dtype=torch.float32, device=self.device)
         slot = self._ctx(ctx)["slot"] if self.cached else None
         mb.tbe_forward(self.tables, self.spec.batch, indices, offsets, N, pooling_mode, slot, self.cache_data, out,
-                       out.shape[1], stream, f16=out.dtype == torch.float16)
+                       out.shape[1], stream, f16=out.dtype == torch.float16, bf16=out.dtype == torch.bfloat16)
         return out
 
     def backward(self, indices, offsets, N: int, grad_out, lr: Optional[float] = None, eps: Optional[float] = None,

@@ -2,14 +2,16 @@
 training; Section 6.1: cache kernels on their own streams, synchronised with the next batch's
 lookups).  Streams, ordered by events only:
 
-    main    : forward(t), backward(t)
-    move[g] : cache g: save victims / fetch missed rows / write victims back for batch t+1   (host link)
+    main    : forward(t), backward(t), tag lookup and replacement for batch t + lock_depth + 1
+    move[g] : cache g: save victims / fetch missed rows / write victims back for the batches ahead  (host link)
     fix     : repair of rows that overflowed in batches t and t-1 and were placed by batch t+1
-    tag     : tag lookup and replacement for batch t+2                              (HBM, small)
 
-so the host-link traffic of the next batch and the tag work of the one after it overlap the
-training of the current batch.  With lock_depth 2 the side streams run up to two batches ahead of
-the training; the launching thread never waits for the device.
+so the host-link traffic of the batches ahead overlaps the training of the current batch; the launching
+thread never waits for the device.  The tag step is a train of some forty kernels that each fill the GPU;
+measured beside the training kernels on a stream of its own (tag_on_main = False: two batches ahead) it
+took three to four times as long as alone and became the longest stage, so by default it runs between
+the training steps, where both run at their own speed, and gives the data movement lock_depth batches of
+time instead of one.
 
 Why this is safe with lock_depth >= 1.  The tag step of batch t may only take ways stamped before
 t - lock_depth; it waits for the backward of the newest such batch (t - 1 - lock_depth), so it only
@@ -54,9 +56,11 @@ from .harness import DeviceModel
 
 
 class CachedTrainer:
-    def __init__(self, model: DeviceModel, pipelined: bool = True, host_gather: bool = False):
+    def __init__(self, model: DeviceModel, pipelined: bool = True, host_gather: bool = False, tag_on_main: bool = True):
         """host_gather: missed rows are gathered by host threads into a pinned buffer and moved by the
-        copy engine, instead of being read over the host link by a kernel."""
+        copy engine, instead of being read over the host link by a kernel.
+        tag_on_main: the tag step of batch t + lock_depth + 1 follows the backward of batch t on the training
+        stream, instead of running two batches ahead on a stream of its own (see the module docstring)."""
         assert model.cached
         # the side streams run two batches ahead and keep two overflow lists alive: lock depths 1 and 2
         assert not pipelined or 1 <= model.lock_depth <= 2, "the pipelined schedule needs lock_depth 1 or 2"
@@ -68,7 +72,8 @@ class CachedTrainer:
         self.pipelined = pipelined
         self.dev = model.device
         self.main = torch.cuda.current_stream(self.dev)
-        self.tag = torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main
+        self.tag_on_main = tag_on_main
+        self.tag = torch.cuda.Stream(self.dev, priority=-1) if (pipelined and not tag_on_main) else self.main
         # the data movement needs few thread blocks but must not queue behind the training kernels' blocks;
         # one stream per cache, so that the caches' row traffic shares the host link instead of taking turns
         n_c = len(model.caches)
@@ -274,18 +279,28 @@ class CachedTrainer:
             for th in self._threads:
                 th.start()
 
-        def move(t):
+        def start_move(t):
+            """The data path of batch t, as soon as its tag step is enqueued."""
             if self._threads:
                 for q in self._jobs:
                     q.put(t)               # ev_tags[t] has been recorded by this thread already
             else:
-                self._move(t)
+                for g in range(n_c):
+                    self._move_cache(t, g, False)
 
+        def finish_move(t):
+            """The repair and the ready event of batch t; needs the event of the backward of batch t-1."""
+            if not self._threads:          # with worker threads the finisher thread does this
+                self._finish_move(t)
+
+        # batches the tag step runs ahead of the training: it may evict rows of batches up to its own minus
+        # lock_depth + 1, and those must have trained
+        ahead = m.lock_depth + 1 if self.tag_on_main else 2
         try:
-            self._lookup(0, batches[0])
-            move(0)
-            if K > 1:
-                self._lookup(1, batches[1])
+            for t in range(min(ahead, K)):
+                self._lookup(t, batches[t])
+                start_move(t)
+            finish_move(0)
             for t in range(K):
                 self._wait_ready_recorded(t)
                 self.main.wait_event(self.ev_ready[t])
@@ -294,9 +309,10 @@ class CachedTrainer:
                 if self._threads:
                     self._bwd_recorded[t].set()
                 if t + 1 < K:
-                    move(t + 1)
-                if t + 2 < K:
-                    self._lookup(t + 2, batches[t + 2])
+                    finish_move(t + 1)
+                if t + ahead < K:
+                    self._lookup(t + ahead, batches[t + ahead])
+                    start_move(t + ahead)
                 if on_step is not None:
                     on_step(t)
         finally:

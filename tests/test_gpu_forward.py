@@ -187,3 +187,62 @@ def test_fp16_output(dtype, mode):
     assert np.isfinite(got).all()
     assert (np.abs(got - ref) <= bound).all(), float(np.max(np.abs(got - ref) - bound))
     m.close()
+
+
+@pytest.mark.parametrize("dtype", [wl.FP32, wl.FP16])
+def test_max_pooling_is_exact(dtype):
+    """Max pooling selects stored values, so the fp32 output equals the oracle's bit for bit: every lane-group
+    width, empty bags (0), bags of one row, negative-only bags, bags longer than a 32-lookup tile."""
+    dims = [8, 16, 24, 64, 128, 200, 256, 512] if dtype == wl.FP16 else [4, 8, 12, 64, 128, 100, 256, 512]
+    rows = [50, 1000, 37, 5000, 20000, 300, 777, 129]
+    spec = custom_spec(rows, dims, 97, dtype, [0.7, 3, 40, 70, 20, 5, 33, 2], [0, 1.1, 0, 1.05, 0.9, 0, 1.3, 0], seed=13)
+    W = wl.all_weights_numpy(spec)
+    W[: int(spec.weight_offset[1])] = -np.abs(W[: int(spec.weight_offset[1])]) - 0.25      # table 0: all negative
+    idx, off = wl.gen_batch(spec, 0)
+    ref = oracle.tbe_forward(*oracle_args(spec), W, spec.batch, idx, off, 2)
+    m = DeviceModel(spec, weights=W)
+    out = torch.full((spec.batch, spec.total_dim), float("nan"), dtype=torch.float32, device="cuda:0")
+    m.forward(to_dev(idx), to_dev(off), len(idx), out=out, pooling_mode=mb.POOL_MAX)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(out.cpu().numpy().view(np.uint32), ref.view(np.uint32))
+    lens = np.diff(off)
+    assert (lens == 0).any() and (lens == 1).any() and (lens > 40).any()
+    m.close()
+    # the 32-piece kernel family too (no wide row in the model)
+    spec2 = custom_spec(rows[:5], dims[:5], 97, dtype, [0.7, 3, 40, 70, 20], [0, 1.1, 0, 1.05, 0.9], seed=14)
+    W2 = wl.all_weights_numpy(spec2)
+    idx2, off2 = wl.gen_batch(spec2, 0)
+    ref2 = oracle.tbe_forward(*oracle_args(spec2), W2, spec2.batch, idx2, off2, 2)
+    m2 = DeviceModel(spec2, weights=W2)
+    out2 = m2.forward(to_dev(idx2), to_dev(off2), len(idx2), pooling_mode=mb.POOL_MAX)
+    np.testing.assert_array_equal(out2.cpu().numpy().view(np.uint32), ref2.view(np.uint32))
+    m2.close()
+
+
+@pytest.mark.parametrize("dtype", [wl.FP32, wl.FP16])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_bf16_output(dtype, mode):
+    """mts_tbe_forward_bf16: the fp32 pooled value rounded once to bfloat16 (8 significant bits: half an ulp is
+    at most 2^-8 relative), both kernel families."""
+    for dims in ([8, 64, 128, 200, 256, 512] if dtype == wl.FP16 else [4, 64, 128, 100, 256, 512],
+                 [8, 64, 128, 200] if dtype == wl.FP16 else [4, 64, 128, 100]):
+        n = len(dims)
+        spec = custom_spec([50, 5000, 20000, 300, 777, 129][:n], dims, 97, dtype, [0.7, 70, 20, 5, 33, 2][:n],
+                           [0, 1.05, 0.9, 0, 1.3, 0][:n], seed=4)
+        W = wl.all_weights_numpy(spec)
+        idx, off = wl.gen_batch(spec, 0)
+        ref, mag = oracle.tbe_forward(*oracle_args(spec), W, spec.batch, idx, off, mode, want_mag=True)
+        m = DeviceModel(spec, weights=W)
+        out = torch.full((spec.batch, spec.total_dim), float("nan"), dtype=torch.bfloat16, device="cuda:0")
+        m.forward(to_dev(idx), to_dev(off), len(idx), out=out, pooling_mode=mode)
+        torch.cuda.synchronize()
+        got = out.float().cpu().numpy().astype(np.float64)
+        ref = np.asarray(ref, np.float64).reshape(got.shape)
+        mag = np.asarray(mag, np.float64).reshape(got.shape)
+        bound = FWD_RTOL[spec.dtype] * (np.abs(ref) + mag) + 2.0 ** -8 * np.abs(ref) + 2.0 ** -40
+        assert np.isfinite(got).all()
+        assert (np.abs(got - ref) <= bound).all(), float(np.max(np.abs(got - ref) - bound))
+        # and it is the fp32 output rounded to nearest even, bit for bit
+        out32 = m.forward(to_dev(idx), to_dev(off), len(idx), pooling_mode=mode)
+        assert torch.equal(out32.to(torch.bfloat16), out)
+        m.close()

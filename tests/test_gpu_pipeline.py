@@ -32,11 +32,13 @@ def test_pipelined_equals_sequential_and_oracle_tags(frac, lock):
     results = []
     # sequential with the kernels fetching the missed rows; pipelined the same way; pipelined and
     # sequential with the rows gathered by host threads and moved by the copy engine
-    for pipelined, host_gather in ((False, False), (True, False), (True, True), (False, True)):
+    # ... and both places of the tag step: between the training steps, or on a stream of its own
+    for pipelined, host_gather, tag_on_main in ((False, False, True), (True, False, True), (True, True, True),
+                                                (False, True, True), (True, False, False), (True, True, False)):
         m = DeviceModel(spec, weights=W0, lock_depth=lock)
         m.reserve(max(len(b[0]) for b in host_batches))
         batches = [(to_dev(i), to_dev(o), o) for i, o in host_batches]
-        tr = CachedTrainer(m, pipelined=pipelined, host_gather=host_gather)
+        tr = CachedTrainer(m, pipelined=pipelined, host_gather=host_gather, tag_on_main=tag_on_main)
         tr.run(batches, grads)
         m.flush()
         torch.cuda.synchronize()
@@ -84,11 +86,12 @@ def test_overflow_repair_survives_slow_side_streams(host_gather):
     grads = [to_dev(wl.gen_grad(spec, k)) for k in range(K)]
     W0 = wl.all_weights_numpy(spec)
     results = []
-    for pipelined, delay in ((False, 0), (True, 2_000_000), (True, 0)):
+    for pipelined, delay, tag_on_main in ((False, 0, True), (True, 2_000_000, True), (True, 0, True),
+                                          (True, 2_000_000, False)):
         m = DeviceModel(spec, weights=W0, lock_depth=2)
         m.reserve(max(len(b[0]) for b in host_batches))
         batches = [(to_dev(i), to_dev(o), o) for i, o in host_batches]
-        tr = CachedTrainer(m, pipelined=pipelined, host_gather=host_gather)
+        tr = CachedTrainer(m, pipelined=pipelined, host_gather=host_gather, tag_on_main=tag_on_main)
         tr.debug_delay_cycles = delay
         tr.run(batches, grads)
         m.flush()
