@@ -476,6 +476,19 @@ int mts_cache_flush(mts_cache* cache, void* host_rows_mapped, void* stream);
 int mts_cache_export_state(mts_cache* cache, int64_t* tags, int64_t* timestamps, int64_t* counts,
                            uint8_t* dirty, void* stream);
 
+/* ---------------------------------------------------------------------------------------
+ * Table placement (Section 5.6, Eq. 6).  Chooses for every table the memory that holds it — HBM
+ * (placement 0, cache id -1 in mts_table_desc) or the host tier behind a cache (placement 1) — so that
+ * each table is in one memory, the HBM tables fit hbm_budget_bytes, and the lookup time per sample
+ *   sum over tables of host_bytes_per_sample[t] / (bw_hbm or bw_host),  bytes_per_sample = D * L * p,
+ * is minimal (Eq. 6 for one GPU).  Exact (branch and bound) unless the search meets its node limit, in
+ * which case the best placement found is returned and *optimal_out is 0.  All pointers are HOST pointers;
+ * time_out and optimal_out may be NULL; bandwidths in bytes per second.  No GPU call.
+ * Errors: INVALID_ARG. */
+int mts_place_tables(int32_t T, const int64_t* host_size_bytes, const double* host_bytes_per_sample,
+                     int64_t hbm_budget_bytes, double bw_hbm, double bw_host, int32_t* host_placement_out,
+                     double* time_out, int32_t* optimal_out);
+
 /* The inverse of mts_cache_export_state, for resuming a run (the paper keeps the cache's tags and states in
  * HBM, Section 5.6, and has no checkpoint format of its own): sets tags (-1 = free way), timestamps, use
  * counts and dirty bytes from device arrays of num_sets*32 entries and fills the slot of every resident tag

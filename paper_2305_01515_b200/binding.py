@@ -37,6 +37,7 @@ EXPORTS = (
     "mts_linearize_keys", "mts_cache_workspace_bytes", "mts_cache_lookup_insert", "mts_cache_lookup_insert_tables",
     "mts_tbe_backward_apply_presorted", "mts_cache_create_host_level", "mts_cache2_workspace_bytes",
     "mts_cache2_lookup_insert", "mts_cache2_move", "mts_cache_import_state", "mts_cache_set_fetch_wait_limit",
+    "mts_place_tables",
     "mts_cache_prefetch_misses", "mts_host_gather_rows", "mts_cache_place_fetched", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
     "mts_cache_export_state",
 )
@@ -124,6 +125,8 @@ def lib():
         L.mts_cache_export_state.argtypes = [vp, vp, vp, vp, vp, vp]
         L.mts_cache_import_state.argtypes = [vp, vp, vp, vp, vp, vp, vp]
         L.mts_cache_set_fetch_wait_limit.argtypes = [vp, i64]
+        L.mts_place_tables.argtypes = [i32, C.POINTER(i64), C.POINTER(C.c_double), i64, C.c_double, C.c_double,
+                                       C.POINTER(i32), C.POINTER(C.c_double), C.POINTER(i32)]
         for name in EXPORTS:
             getattr(L, name)            # raises AttributeError when a declared symbol is missing
         _lib = L
@@ -436,6 +439,18 @@ def cache_writeback_evicted(cache: Cache, host_rows_mapped, evict_keys, evict_di
 
 def cache_flush(cache: Cache, host_rows_mapped, stream=None) -> None:
     _check(lib().mts_cache_flush(cache.handle, _ptr(host_rows_mapped), _stream(stream)))
+
+
+def place_tables(size_bytes, bytes_per_sample, hbm_budget_bytes: int, bw_hbm: float, bw_host: float):
+    """mts_place_tables on host sequences: ([placement per table: 0 HBM / 1 host tier], time per sample, optimal)."""
+    T = len(size_bytes)
+    sz = (C.c_int64 * T)(*[int(x) for x in size_bytes])
+    cost = (C.c_double * T)(*[float(x) for x in bytes_per_sample])
+    out = (C.c_int32 * T)()
+    t, opt = C.c_double(0.0), C.c_int32(0)
+    _check(lib().mts_place_tables(T, sz, cost, int(hbm_budget_bytes), float(bw_hbm), float(bw_host), out,
+                                  C.byref(t), C.byref(opt)))
+    return list(out), float(t.value), bool(opt.value)
 
 
 def cache_import_state(cache: Cache, tags, timestamps, counts, dirty, host_rows_mapped, stream=None) -> None:
