@@ -522,6 +522,29 @@ def host_link_bandwidth(dev, nbytes: int = 1 << 30):
     return res[0], res[1]
 
 
+def host_gather_rates(model, n_rows: int = 200_000):
+    """GB/s of mts_host_gather_rows on random rows of every cache's table group (host threads only)."""
+    import torch
+
+    from paper_2305_01515_b200 import binding as mb
+
+    rng = np.random.default_rng(0)
+    rates = {}
+    for g, c in enumerate(model.caches):
+        _, t0, t1 = model.groups[g]
+        rows_g = int(model.spec.row_offset[t1] - model.spec.row_offset[t0])
+        rb = c.dim * model.spec.elem_bytes
+        n = min(n_rows, model.fetch_rows[g])
+        keys = torch.from_numpy(rng.integers(0, rows_g, n).astype(np.int64))
+        best = 1e9
+        for _ in range(3):
+            t0_ = time.perf_counter()
+            mb.host_gather_rows(model.host_rows_ptr(g), keys.numpy(), n, rb, model.fetch_host[0][g], model.gather_threads)
+            best = min(best, time.perf_counter() - t0_)
+        rates[str(c.dim)] = n * rb / best / 1e9
+    return rates
+
+
 def measure_cached(args, spec, dev, steps: int, warmup: int):
     """Configurations 4 and 5: rows in pinned host memory behind HBM caches, pipelined train step.  `warmup`
     batches bring the caches to their steady state, the next `steps` batches are timed.  Returns the record."""
@@ -548,7 +571,10 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
     grads = [torch.from_numpy(wl.gen_grad(spec, k)).to(dev) for k in range(R)]
     glist = [grads[k % R] for k in range(K)]
     setup_s = time.time() - t_setup
-    trainer = CachedTrainer(model, pipelined=not args.sequential, host_gather=args.fetch == "host")
+    trainer = CachedTrainer(model, pipelined=not args.sequential, host_gather=args.fetch == "host",
+                            tag_on_main=not args.tag_stream)
+    trainer.record_timeline = args.timeline
+    gather_gbs = host_gather_rates(model) if args.fetch == "host" else None
     main = torch.cuda.current_stream(dev)
     marks = {}
 
@@ -637,6 +663,14 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
                      "traffic": None, "peak_source": peak_src},
         "clocks": clocks, "gpu_launches": int(launches), "kernels": kernels,
     }
+    if gather_gbs is not None:
+        rec["host_link"]["host_gather_gbs_by_dim"] = gather_gbs
+    if args.timeline:
+        # device time of every phase of the last batches, ms since the first mark (perturbs the run a little)
+        by_batch = {}
+        for name, t, ms_at in trainer.timeline():
+            by_batch.setdefault(t, {})[name] = round(ms_at, 2)
+        rec["timeline_ms"] = {str(t): dict(sorted(by_batch[t].items(), key=lambda kv: kv[1])) for t in sorted(by_batch)[-4:]}
     if two_level:
         l2_hits = float(hist[:, :, 10].sum())
         rec["two_level"] = {"l2_fraction": args.l2_fraction, "l1_hit_rate_per_lookup": hit,
@@ -732,6 +766,11 @@ def main():
     ap.add_argument("--sequential", action="store_true", help="one stream only (no sort beside the forward, no cache pipeline)")
     ap.add_argument("--lock-depth", type=int, default=2,
                     help="cached workloads: batches a stamped way stays unevictable (Section 5.7 invariant)")
+    ap.add_argument("--timeline", action="store_true",
+                    help="cached workloads: add the device timeline of the last batches (events on every stream) to the line")
+    ap.add_argument("--tag-stream", action="store_true",
+                    help="cached workloads: the tag step on a stream of its own, two batches ahead, instead of between the "
+                         "training steps")
     ap.add_argument("--trace", action="store_true",
                     help="cached workloads: CUDA events around every launch of the run (perturbs the timing)")
     ap.add_argument("--tables", type=int, default=0,

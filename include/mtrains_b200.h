@@ -229,10 +229,12 @@ int mts_tbe_backward_apply_f16(const mts_tables* tables, int32_t B, const int64_
 /* The gradient half of the backward on lookups that are already ordered by row (Section 5.9; the
  * cache's tag lookup, Section 5.5.1, orders a batch's requests by row for its own purposes, and the
  * backward of the same batch can reuse that order instead of sorting again).
- *   sorted_rows[p]   : linear row id (row_offset[t] + index) of the p-th lookup in ascending row order,
- *   sorted_pos[p]    : that lookup's position in `indices`; equal rows in ascending position,
- *   bag_of_lookup[i] : bag id t*B + b of the lookup at position i,
- * all device uint32 [N], covering every lookup of the batch — as written by
+ *   sorted_rows[p] : linear row id (row_offset[t] + index) of the p-th lookup in ascending row order,
+ *                    equal rows in ascending position in the batch,
+ *   sorted_bag[p]  : that lookup's bag id t*B + b,
+ *   sorted_slot[p] : its cache slot, or -1 = the row is updated in the host tier (ignored for tables that
+ *                    live in HBM),
+ * all device arrays of N entries covering every lookup of the batch — as written by
  * mts_cache_lookup_insert_tables calls that together cover all tables (every table cached).  The
  * arrays are trusted: rows outside the tables or an order that is not ascending give undefined
  * results.  grad_dtype: MTS_DTYPE_FP32 (float) or MTS_DTYPE_FP16 (binary16) gradient.  The
@@ -241,10 +243,9 @@ int mts_tbe_backward_apply_f16(const mts_tables* tables, int32_t B, const int64_
 int mts_tbe_backward_apply_presorted(const mts_tables* tables, int32_t B, const int64_t* offsets, int64_t N,
                                      int32_t pooling_mode, const void* grad_out, int32_t grad_dtype,
                                      int64_t grad_stride, float lr, float eps, const uint32_t* sorted_rows,
-                                     const uint32_t* sorted_pos, const uint32_t* bag_of_lookup,
-                                     const int32_t* slot_of_lookup, void* const* host_cache_data,
-                                     uint8_t* const* host_cache_dirty, int32_t n_caches, void* workspace,
-                                     size_t workspace_bytes, void* stream);
+                                     const uint32_t* sorted_bag, const int32_t* sorted_slot,
+                                     void* const* host_cache_data, uint8_t* const* host_cache_dirty,
+                                     int32_t n_caches, void* workspace, size_t workspace_bytes, void* stream);
 
 /* Backward without a workspace argument and without any allocation (the paper has no
  * counterpart; this exists for callers of this library that cannot allocate device memory).
@@ -346,11 +347,11 @@ int mts_cache_lookup_insert(mts_cache* cache, const int64_t* keys, int64_t N, in
  *   - slot_of_lookup is the batch-wide array (int32 [>= lookup_begin + n]); the call writes the
  *     entries of its own lookups, slot_of_lookup[i] for position i;
  *   - the overflow list has a capacity of its own (overflow_capacity; n is always enough);
- *   - sorted_rows_out, sorted_pos_out, bag_of_lookup_out (all NULL, or the first two, or all three;
- *     batch-wide device uint32 arrays): entries [lookup_begin, lookup_begin + n) receive the group's
- *     lookups ordered by row — linear row id row_offset[t] + index ascending, equal rows in ascending
- *     position — and their positions; bag_of_lookup_out[i] = t*B + b for the positions of the group.
- *     Calls for all groups of a batch fill the arrays mts_tbe_backward_apply_presorted consumes.
+ *   - sorted_rows_out, sorted_bag_out, sorted_slot_out (all NULL or all three; batch-wide device arrays):
+ *     entries [lookup_begin, lookup_begin + n) receive the group's lookups ordered by row — linear row id
+ *     row_offset[t] + index ascending, equal rows in ascending position — with the bag id t*B + b and the
+ *     cache slot (or -1) of each.  Calls for all groups of a batch fill the arrays
+ *     mts_tbe_backward_apply_presorted consumes.
  * An index outside [0, rows[t]) is clamped and raises bit 0 of mts_tables_status. */
 int mts_cache_lookup_insert_tables(mts_cache* cache, const mts_tables* tables, int32_t t_begin, int32_t t_end,
                                    int32_t B, const int64_t* indices, const int64_t* offsets,
@@ -358,8 +359,8 @@ int mts_cache_lookup_insert_tables(mts_cache* cache, const mts_tables* tables, i
                                    int64_t* miss_keys, int32_t* miss_slots, int64_t* evict_keys,
                                    int32_t* evict_slots, uint8_t* evict_dirty, int64_t list_capacity,
                                    int64_t* overflow_keys, int64_t overflow_capacity, int64_t* counters,
-                                   uint32_t* sorted_rows_out, uint32_t* sorted_pos_out,
-                                   uint32_t* bag_of_lookup_out, void* workspace, size_t workspace_bytes,
+                                   uint32_t* sorted_rows_out, uint32_t* sorted_bag_out,
+                                   int32_t* sorted_slot_out, void* workspace, size_t workspace_bytes,
                                    void* stream);
 
 /* ---------------------------------------------------------------------------------------
@@ -444,6 +445,13 @@ int mts_cache_prefetch_misses(mts_cache* cache, const void* host_rows_mapped, co
  * Errors: INVALID_ARG, ALIGNMENT, CUDA. */
 int mts_host_gather_rows(const void* host_rows, const int64_t* host_keys, int64_t n, int64_t row_bytes,
                          void* host_out, int32_t threads);
+/* The write-back the same way (Section 5.5.4: evicted rows go back to the lower tier): after
+ * mts_cache_place_fetched the dirty victims sit in evict_staging in list order; the caller copies the first
+ * MTS_CNT_EVICTED rows of it, with evict_keys and evict_dirty, to host buffers (one contiguous copy each) and
+ * calls this on the host: host_rows[host_keys[k]] = host_in[k] for every k < n with host_mask[k] != 0
+ * (host_mask NULL = all), with `threads` host threads.  Plain memory, no GPU call; blocks until done. */
+int mts_host_scatter_rows(void* host_rows, const int64_t* host_keys, const uint8_t* host_mask, int64_t n,
+                          int64_t row_bytes, const void* host_in, int32_t threads);
 int mts_cache_place_fetched(mts_cache* cache, const void* fetched, const int32_t* miss_slots,
                             const int32_t* evict_slots, const uint8_t* evict_dirty, int64_t list_capacity,
                             const int64_t* counters, void* evict_staging, void* stream);

@@ -38,7 +38,7 @@ EXPORTS = (
     "mts_tbe_backward_apply_presorted", "mts_cache_create_host_level", "mts_cache2_workspace_bytes",
     "mts_cache2_lookup_insert", "mts_cache2_move", "mts_cache_import_state", "mts_cache_set_fetch_wait_limit",
     "mts_place_tables",
-    "mts_cache_prefetch_misses", "mts_host_gather_rows", "mts_cache_place_fetched", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
+    "mts_cache_prefetch_misses", "mts_host_gather_rows", "mts_host_scatter_rows", "mts_cache_place_fetched", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
     "mts_cache_export_state",
 )
 
@@ -109,7 +109,7 @@ def lib():
         L.mts_cache_lookup_insert.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, i64, vp, vp, sz, vp]
         L.mts_cache_lookup_insert_tables.argtypes = [vp, vp, i32, i32, i32, vp, vp, i64, i64, i64, vp, vp, vp, vp, vp, vp,
                                                      i64, vp, i64, vp, vp, vp, vp, vp, sz, vp]
-        L.mts_tbe_backward_apply_presorted.argtypes = [vp, i32, vp, i64, i32, vp, i32, i64, f32, f32, vp, vp, vp, vp,
+        L.mts_tbe_backward_apply_presorted.argtypes = [vp, i32, vp, i64, i32, vp, i32, i64, f32, f32, vp, vp, vp,
                                                        C.POINTER(vp), C.POINTER(vp), i32, vp, sz, vp]
         L.mts_cache_create_host_level.argtypes = [C.POINTER(vp), i64, i64, i32, i32, i32, i32, i32, vp]
         L.mts_cache2_workspace_bytes.restype = sz
@@ -120,6 +120,7 @@ def lib():
         L.mts_cache_prefetch_misses.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.mts_cache_writeback_evicted.argtypes = [vp, vp, vp, vp, i64, vp, vp, vp]
         L.mts_host_gather_rows.argtypes = [vp, vp, i64, i64, vp, i32]
+        L.mts_host_scatter_rows.argtypes = [vp, vp, vp, i64, i64, vp, i32]
         L.mts_cache_place_fetched.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.mts_cache_flush.argtypes = [vp, vp, vp]
         L.mts_cache_export_state.argtypes = [vp, vp, vp, vp, vp, vp]
@@ -273,14 +274,14 @@ def tbe_backward_apply(tables: Tables, B: int, offsets, N: int, pooling_mode: in
 
 
 def tbe_backward_apply_presorted(tables: Tables, B: int, offsets, N: int, pooling_mode: int, grad_out,
-                                 grad_stride: int, lr: float, eps: float, sorted_rows, sorted_pos, bag_of_lookup,
-                                 slot_of_lookup, cache_data: Optional[Sequence], cache_dirty: Optional[Sequence],
+                                 grad_stride: int, lr: float, eps: float, sorted_rows, sorted_bag, sorted_slot,
+                                 cache_data: Optional[Sequence], cache_dirty: Optional[Sequence],
                                  workspace, workspace_bytes: int, stream=None, f16: bool = False) -> None:
     """Gradient half of the backward on lookups already ordered by row (mts_cache_lookup_insert_tables)."""
     n_caches = len(cache_data) if cache_data is not None else 0
     _check(lib().mts_tbe_backward_apply_presorted(
         tables.handle, B, _ptr(offsets), N, pooling_mode, _ptr(grad_out), DTYPE_FP16 if f16 else DTYPE_FP32,
-        grad_stride, lr, eps, _ptr(sorted_rows), _ptr(sorted_pos), _ptr(bag_of_lookup), _ptr(slot_of_lookup),
+        grad_stride, lr, eps, _ptr(sorted_rows), _ptr(sorted_bag), _ptr(sorted_slot),
         _ptr_array(cache_data, n_caches), _ptr_array(cache_dirty, n_caches), n_caches, _ptr(workspace),
         workspace_bytes, _stream(stream)))
 
@@ -366,14 +367,14 @@ def cache_lookup_insert_tables(cache: Cache, tables: Tables, t_begin: int, t_end
                                lookup_begin: int, n: int, step: int, slot_of_lookup, miss_keys, miss_slots,
                                evict_keys, evict_slots, evict_dirty, list_capacity: int, overflow_keys,
                                overflow_capacity: int, counters, workspace, workspace_bytes: int, stream=None,
-                               sorted_rows_out=None, sorted_pos_out=None, bag_of_lookup_out=None) -> None:
+                               sorted_rows_out=None, sorted_bag_out=None, sorted_slot_out=None) -> None:
     """Tag lookup of one cache fed from the batch's sparse input; slot_of_lookup and the three optional
     outputs are batch-wide arrays."""
     _check(lib().mts_cache_lookup_insert_tables(
         cache.handle, tables.handle, t_begin, t_end, B, _ptr(indices), _ptr(offsets), lookup_begin, n, step,
         _ptr(slot_of_lookup), _ptr(miss_keys), _ptr(miss_slots), _ptr(evict_keys), _ptr(evict_slots),
         _ptr(evict_dirty), list_capacity, _ptr(overflow_keys), overflow_capacity, _ptr(counters),
-        _ptr(sorted_rows_out), _ptr(sorted_pos_out), _ptr(bag_of_lookup_out), _ptr(workspace), workspace_bytes,
+        _ptr(sorted_rows_out), _ptr(sorted_bag_out), _ptr(sorted_slot_out), _ptr(workspace), workspace_bytes,
         _stream(stream)))
 
 
@@ -421,6 +422,14 @@ def host_gather_rows(host_rows_ptr: int, host_keys, n: int, row_bytes: int, host
     assert host_keys.dtype.itemsize == 8 and host_keys.flags.c_contiguous and len(host_keys) >= n
     _check(lib().mts_host_gather_rows(int(host_rows_ptr), int(host_keys.ctypes.data), n, row_bytes,
                                       _ptr(host_out), threads))
+
+
+def host_scatter_rows(host_rows_ptr: int, host_keys, host_mask, n: int, row_bytes: int, host_in, threads: int) -> None:
+    """host_keys int64 / host_mask uint8 (or None): host numpy arrays; host_rows_ptr / host_in: host addresses."""
+    assert host_keys.dtype.itemsize == 8 and host_keys.flags.c_contiguous and len(host_keys) >= n
+    _check(lib().mts_host_scatter_rows(int(host_rows_ptr), int(host_keys.ctypes.data),
+                                       None if host_mask is None else int(host_mask.ctypes.data), n, row_bytes,
+                                       _ptr(host_in), threads))
 
 
 def cache_place_fetched(cache: Cache, fetched, miss_slots, evict_slots, evict_dirty, list_capacity: int, counters,

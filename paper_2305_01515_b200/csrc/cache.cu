@@ -78,7 +78,8 @@ __global__ void cache_prepare_keys(const int64_t* __restrict__ keys, int64_t n, 
 
 // The same preparation straight from a batch's sparse input, for the lookups of the tables
 // [t_begin, t_end) (8 lanes per bag): the sort key is the linear row id row_offset[t] + index, the
-// value the lookup's position in the batch; bag_of_lookup (nullable) receives every lookup's bag id.
+// value the lookup's position in the batch; bag_of_lookup (nullable, indexed by position - lookup_begin)
+// receives every lookup's bag id.
 __global__ void cache_prepare_from_indices(const TableMeta* __restrict__ meta, int32_t t_begin, int64_t n_bags,
                                            int32_t B, const int64_t* __restrict__ indices,
                                            const int64_t* __restrict__ offsets, int64_t lookup_begin, int64_t n,
@@ -101,7 +102,7 @@ __global__ void cache_prepare_from_indices(const TableMeta* __restrict__ meta, i
     if (o >= 0 && o < n) {
       k32[o] = (uint32_t)(roff + clamp_index(indices[i], rows, status));
       pos[o] = (uint32_t)i;
-      if (bag_of_lookup != nullptr) bag_of_lookup[i] = (uint32_t)bag;
+      if (bag_of_lookup != nullptr) bag_of_lookup[o] = (uint32_t)bag;
     }
   }
 }
@@ -658,10 +659,20 @@ cache_write_lists(uint8_t* __restrict__ member_flag, const uint32_t* __restrict_
 
 __global__ void cache_scatter_slots(const uint32_t* __restrict__ sorted_pos, const uint32_t* __restrict__ uniq_idx,
                                     const int32_t* __restrict__ slot_of_uniq, int64_t n,
-                                    const uint32_t* __restrict__ n_dev, int32_t* __restrict__ slot_of_lookup) {
+                                    const uint32_t* __restrict__ n_dev, int32_t* __restrict__ slot_of_lookup,
+                                    const uint32_t* __restrict__ bag_of_lookup, int64_t pos_base,
+                                    uint32_t* __restrict__ sorted_bag, int32_t* __restrict__ sorted_slot) {
   if (n_dev != nullptr) n = min(n, (int64_t)*n_dev);
-  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += (int64_t)gridDim.x * blockDim.x)
-    slot_of_lookup[sorted_pos[p]] = slot_of_uniq[uniq_idx[p]];
+  for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += (int64_t)gridDim.x * blockDim.x) {
+    const uint32_t ps = sorted_pos[p];
+    const int32_t slot = slot_of_uniq[uniq_idx[p]];
+    slot_of_lookup[ps] = slot;
+    if (sorted_bag != nullptr) {
+      // for the backward of the same batch: bag and slot of every lookup in the order of the sorted rows
+      sorted_bag[p] = bag_of_lookup[ps - pos_base];
+      sorted_slot[p] = slot;
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------ data movement
@@ -891,7 +902,7 @@ struct CacheLayout {
       sseg_start, slot_of_uniq, member_flag, member_old_key, member_old_dirty, member_old_ts, member_old_freq,
       member_old_placed, member_slot, hist, scan, cnt_miss,
       cnt_evict, n_unique, n_sets, ovf_cursor, missed, cnt_missed, n_missed, ins_ts, ins_dirty, l2slot_of_uniq,
-      drop_cursor, total;
+      drop_cursor, bag_of_lookup, total;
 };
 
 static int bits_of(int64_t values) {
@@ -919,6 +930,7 @@ static CacheLayout cache_layout(const mts_cache* c, int64_t N) {
   L.n_unique = take(256); L.n_sets = take(256); L.ovf_cursor = take(256);
   L.missed = take(n); L.cnt_missed = take(PROBE_BLOCKS * 4); L.n_missed = take(256);
   L.ins_ts = take(n * 4); L.ins_dirty = take(n); L.l2slot_of_uniq = take(n * 4); L.drop_cursor = take(256);
+  L.bag_of_lookup = take(n * 4);
   L.total = off;
   return L;
 }
@@ -1067,8 +1079,8 @@ struct KeySource {
   const int64_t* offsets = nullptr;
   int64_t lookup_begin = 0;
   uint32_t* sorted_rows_out = nullptr;     // batch-wide arrays; this call fills [lookup_begin, lookup_begin + N)
-  uint32_t* sorted_pos_out = nullptr;
-  uint32_t* bag_of_lookup_out = nullptr;
+  uint32_t* sorted_bag_out = nullptr;
+  int32_t* sorted_slot_out = nullptr;
 };
 
 // n_dev (nullable): device-resident number of keys, N is then its upper bound.  attrs: the keys are rows that
@@ -1105,7 +1117,6 @@ int lookup_insert_impl(mts_cache* c, const KeySource& src, int64_t N, int64_t st
     if (src.sorted_rows_out != nullptr) {
       const bool result_in_a = N <= 1 || (sort_passes(key_bits) & 1) == 0;
       (result_in_a ? keys_a : keys_b) = src.sorted_rows_out + src.lookup_begin;
-      (result_in_a ? vals_a : vals_b) = src.sorted_pos_out + src.lookup_begin;
     }
   }
   int rc;
@@ -1123,7 +1134,8 @@ int lookup_insert_impl(mts_cache* c, const KeySource& src, int64_t N, int64_t st
       LaunchScope scope(K_CACHE_PREPARE, s);
       cache_prepare_from_indices<<<(unsigned)ceil_div(std::max<int64_t>(n_bags * 8, MTS_NUM_COUNTERS), 256), 256, 0, s>>>(
           src.tables->d_meta, src.t_begin, n_bags, src.B, src.indices, src.offsets, src.lookup_begin, N, keys_a, vals_a,
-          src.bag_of_lookup_out, counters, U32(L.ovf_cursor), src.tables->d_status);
+          src.sorted_rows_out != nullptr ? U32(L.bag_of_lookup) : nullptr, counters, U32(L.ovf_cursor),
+          src.tables->d_status);
     }
     rc = check_launch("cache_prepare_from_indices");
   }
@@ -1222,7 +1234,11 @@ int lookup_insert_impl(mts_cache* c, const KeySource& src, int64_t N, int64_t st
     // positions are relative to the key array, or batch positions when the keys came from a batch's
     // sparse input (slot_of_lookup is then the batch-wide array)
     LaunchScope scope(K_CACHE_SCATTER_SLOTS, s);
-    cache_scatter_slots<<<grid, 256, 0, s>>>(sp, U32(L.uniq_idx), slot_of_uniq, N, n_dev, slot_of_lookup);
+    const bool exp = src.sorted_rows_out != nullptr;
+    cache_scatter_slots<<<grid, 256, 0, s>>>(sp, U32(L.uniq_idx), slot_of_uniq, N, n_dev, slot_of_lookup,
+                                             exp ? U32(L.bag_of_lookup) : nullptr, src.lookup_begin,
+                                             exp ? src.sorted_bag_out + src.lookup_begin : nullptr,
+                                             exp ? src.sorted_slot_out + src.lookup_begin : nullptr);
   }
   return check_launch("cache lists / scatter");
 }
@@ -1246,8 +1262,8 @@ extern "C" int mts_cache_lookup_insert_tables(mts_cache* c, const mts_tables* h,
                                               int64_t* miss_keys, int32_t* miss_slots, int64_t* evict_keys,
                                               int32_t* evict_slots, uint8_t* evict_dirty, int64_t list_capacity,
                                               int64_t* overflow_keys, int64_t overflow_capacity, int64_t* counters,
-                                              uint32_t* sorted_rows_out, uint32_t* sorted_pos_out,
-                                              uint32_t* bag_of_lookup_out, void* workspace, size_t workspace_bytes,
+                                              uint32_t* sorted_rows_out, uint32_t* sorted_bag_out,
+                                              int32_t* sorted_slot_out, void* workspace, size_t workspace_bytes,
                                               void* stream) {
   if (!c || !h || !offsets || B < 1 || t_begin < 0 || t_end > h->T || t_begin >= t_end || n < 0 || lookup_begin < 0 ||
       (n > 0 && !indices))
@@ -1257,14 +1273,14 @@ extern "C" int mts_cache_lookup_insert_tables(mts_cache* c, const mts_tables* h,
                      t_begin, t_end,
                      (long long)(h->h_meta[t_end - 1].row_offset + h->h_meta[t_end - 1].rows - h->h_meta[t_begin].row_offset),
                      (long long)c->key_space);
-  if ((sorted_rows_out == nullptr) != (sorted_pos_out == nullptr) || (bag_of_lookup_out != nullptr && !sorted_rows_out))
-    return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert_tables: pass sorted_rows_out, sorted_pos_out (and bag_of_lookup_out) together");
+  if ((sorted_rows_out == nullptr) != (sorted_bag_out == nullptr) || (sorted_rows_out == nullptr) != (sorted_slot_out == nullptr))
+    return set_error(MTS_ERR_INVALID_ARG, "cache_lookup_insert_tables: pass sorted_rows_out, sorted_bag_out and sorted_slot_out together");
   if (lookup_begin + n >= (1ll << 32) - 1 || (int64_t)h->T * B >= (1ll << 32))
     return set_error(MTS_ERR_UNSUPPORTED, "cache_lookup_insert_tables: lookup positions and bag ids must fit 32 bits");
   KeySource src;
   src.tables = h; src.t_begin = t_begin; src.t_end = t_end; src.B = B;
   src.indices = indices; src.offsets = offsets; src.lookup_begin = lookup_begin;
-  src.sorted_rows_out = sorted_rows_out; src.sorted_pos_out = sorted_pos_out; src.bag_of_lookup_out = bag_of_lookup_out;
+  src.sorted_rows_out = sorted_rows_out; src.sorted_bag_out = sorted_bag_out; src.sorted_slot_out = sorted_slot_out;
   return lookup_insert_impl(c, src, n, step, slot_of_lookup, miss_keys, miss_slots, evict_keys, evict_slots, evict_dirty,
                             overflow_keys, list_capacity, overflow_capacity, counters, workspace, workspace_bytes, stream);
 }
@@ -1514,6 +1530,28 @@ extern "C" int mts_host_gather_rows(const void* host_rows, const int64_t* host_k
       }
       memcpy(dst + (size_t)k * rb, src + (size_t)host_keys[k] * rb, rb);
     }
+  };
+  const int64_t nt = std::max<int64_t>(1, std::min<int64_t>(threads, (n + 1023) / 1024));
+  if (nt == 1) { work(0, n); return MTS_OK; }
+  std::vector<std::thread> pool;
+  const int64_t per = (n + nt - 1) / nt;
+  for (int64_t i = 1; i < nt; ++i) pool.emplace_back(work, std::min(n, i * per), std::min(n, (i + 1) * per));
+  work(0, std::min(n, per));
+  for (auto& t : pool) t.join();
+  return MTS_OK;
+}
+
+extern "C" int mts_host_scatter_rows(void* host_rows, const int64_t* host_keys, const uint8_t* host_mask, int64_t n,
+                                     int64_t row_bytes, const void* host_in, int32_t threads) {
+  if (n < 0 || row_bytes < 1 || (n > 0 && (!host_rows || !host_keys || !host_in)))
+    return set_error(MTS_ERR_INVALID_ARG, "host_scatter_rows: null argument or bad size");
+  if (n == 0) return MTS_OK;
+  char* dst = static_cast<char*>(host_rows);
+  const char* src = static_cast<const char*>(host_in);
+  const size_t rb = (size_t)row_bytes;
+  auto work = [=](int64_t k0, int64_t k1) {
+    for (int64_t k = k0; k < k1; ++k)
+      if (host_mask == nullptr || host_mask[k]) memcpy(dst + (size_t)host_keys[k] * rb, src + (size_t)k * rb, rb);
   };
   const int64_t nt = std::max<int64_t>(1, std::min<int64_t>(threads, (n + 1023) / 1024));
   if (nt == 1) { work(0, n); return MTS_OK; }

@@ -94,8 +94,15 @@ struct RowTarget {
   uint8_t* dirty;     // dirty byte to set, or nullptr
 };
 
-__device__ __forceinline__ RowTarget row_target(const TableMeta& m, int64_t key, uint32_t pos, int eb,
-                                                const int32_t* __restrict__ slot_of_lookup,
+// Cache slot of the lookup at sorted position p (batch position ps): from the array ordered like the sorted
+// lookups when the caller has one, else through the lookup's position.
+__device__ __forceinline__ int32_t slot_at(const TableMeta& m, const int32_t* __restrict__ sorted_slot, int64_t p,
+                                           const int32_t* __restrict__ slot_of_lookup, uint32_t ps) {
+  if (m.cache_id < 0) return -1;
+  return sorted_slot != nullptr ? sorted_slot[p] : slot_of_lookup[ps];
+}
+
+__device__ __forceinline__ RowTarget row_target(const TableMeta& m, int64_t key, int32_t s, int eb,
                                                 const CachePtrs& caches, char* dev_w, char* host_w) {
   RowTarget r;
   const int64_t row_bytes = (int64_t)m.dim * eb;
@@ -104,7 +111,6 @@ __device__ __forceinline__ RowTarget row_target(const TableMeta& m, int64_t key,
   if (m.cache_id < 0) {
     r.w = dev_w + m.weight_offset * eb + idx * row_bytes;
   } else {
-    const int32_t s = slot_of_lookup[pos];
     if (s >= 0) {
       r.w = static_cast<char*>(caches.data[m.cache_id]) + (int64_t)s * row_bytes;
       r.dirty = caches.dirty[m.cache_id] ? caches.dirty[m.cache_id] + s : nullptr;
@@ -241,8 +247,8 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
               const uint32_t* __restrict__ bag_of_pos, int64_t n,
               const int64_t* __restrict__ offsets,
               const void* __restrict__ grad, int64_t grad_stride, float lr, float eps,
-              const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches, char* dev_w,
-                   char* host_w,
+              const int32_t* __restrict__ slot_of_lookup, const int32_t* __restrict__ sorted_slot,
+              const __grid_constant__ CachePtrs caches, char* dev_w, char* host_w,
               float* __restrict__ momentum, float* __restrict__ partial_head,
               float* __restrict__ partial_tail, uint32_t* __restrict__ next_chunk) {
   constexpr int EB = FP16 ? 2 : 4;
@@ -288,7 +294,7 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
       d.z = 0u; d.w = 0u;
       uint8_t* dirty = nullptr;
       if (my_end) {
-        const RowTarget rt = row_target(m, (int64_t)key, ps, EB, slot_of_lookup, caches, dev_w, host_w);
+        const RowTarget rt = row_target(m, (int64_t)key, slot_at(m, sorted_slot, p, slot_of_lookup, ps), EB, caches, dev_w, host_w);
         d.z = (uint32_t)(uintptr_t)rt.w;
         d.w = (uint32_t)((uintptr_t)rt.w >> 32);
         dirty = rt.dirty;
@@ -392,8 +398,8 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
                    const uint32_t* __restrict__ bag_of_pos, int64_t n,
                    const int64_t* __restrict__ offsets,
                    const void* __restrict__ grad, int64_t grad_stride, float lr, float eps,
-                   const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches, char* dev_w,
-                   char* host_w,
+                   const int32_t* __restrict__ slot_of_lookup, const int32_t* __restrict__ sorted_slot,
+                   const __grid_constant__ CachePtrs caches, char* dev_w, char* host_w,
                    float* __restrict__ momentum, float* __restrict__ partial_head,
                    float* __restrict__ partial_tail, uint32_t* __restrict__ next_chunk) {
   constexpr int EB = FP16 ? 2 : 4;
@@ -439,7 +445,7 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
       d.z = 0u; d.w = 0u;
       uint8_t* dirty = nullptr;
       if (my_end) {
-        const RowTarget rt = row_target(m, (int64_t)key, ps, EB, slot_of_lookup, caches, dev_w, host_w);
+        const RowTarget rt = row_target(m, (int64_t)key, slot_at(m, sorted_slot, p, slot_of_lookup, ps), EB, caches, dev_w, host_w);
         d.z = (uint32_t)(uintptr_t)rt.w;
         d.w = (uint32_t)((uintptr_t)rt.w >> 32);
         dirty = rt.dirty;
@@ -573,8 +579,8 @@ template <bool FP16, int NV>
 __global__ void __launch_bounds__(BWD_WARPS * 32)
 combine_partials(const TableMeta* __restrict__ meta, int T, const uint32_t* __restrict__ keys,
                  const uint32_t* __restrict__ pos, int64_t n, float lr, float eps,
-                 const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches, char* dev_w,
-                   char* host_w,
+                 const int32_t* __restrict__ slot_of_lookup, const int32_t* __restrict__ sorted_slot,
+                 const __grid_constant__ CachePtrs caches, char* dev_w, char* host_w,
                  float* __restrict__ momentum, const float* __restrict__ partial_head,
                  const float* __restrict__ partial_tail, const float* __restrict__ partial_group) {
   constexpr int EB = FP16 ? 2 : 4;
@@ -643,7 +649,8 @@ combine_partials(const TableMeta* __restrict__ meta, int T, const uint32_t* __re
   }
   const int t = table_of_key(meta, T, (int64_t)key);
   const TableMeta m = meta[t];
-  const RowTarget rt = row_target(m, (int64_t)key, pos[pe - 1], EB, slot_of_lookup, caches, dev_w, host_w);
+  const RowTarget rt = row_target(m, (int64_t)key, slot_at(m, sorted_slot, pe - 1, slot_of_lookup, pos[pe - 1]), EB, caches,
+                                  dev_w, host_w);
   uint4 w[NV];
   load_row<FP16, NV>(w, rt.w, m.dim);
   adagrad_row<FP16, NV>(acc, w, momentum[key], m.dim, __frcp_rn((float)m.dim), lr, eps, rt.w, momentum + key, rt.dirty);
@@ -730,8 +737,8 @@ template <bool FP16, int NV, int GROUP>
 static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys, const uint32_t* pos,
                            const uint32_t* bag_of_pos, int64_t N, const int64_t* offsets, int32_t pooling_mode,
                            const void* grad, bool grad_half, int64_t grad_stride, float lr, float eps,
-                           const int32_t* slot_of_lookup, const CachePtrs& caches, float* head, float* tail,
-                           float* group, uint32_t* next_chunk, cudaStream_t s) {
+                           const int32_t* slot_of_lookup, const int32_t* sorted_slot, const CachePtrs& caches,
+                           float* head, float* tail, float* group, uint32_t* next_chunk, cudaStream_t s) {
   const int64_t chunks = ceil_div(N, BWD_CHUNK);
   const unsigned grid = (unsigned)ceil_div(chunks, BWD_WARPS);
   // the reduce kernels exist for fp32 and for fp16 upstream gradients
@@ -740,13 +747,13 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
   do {                                                                                                               \
     if (grad_half)                                                                                                   \
       KERNEL<TARGS, true><<<GRID, THREADS, 0, s>>>(h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad,     \
-                                                    grad_stride, lr, eps, slot_of_lookup, caches,                    \
+                                                    grad_stride, lr, eps, slot_of_lookup, sorted_slot, caches,       \
                                                     static_cast<char*>(h->dev_weights),                              \
                                                     static_cast<char*>(h->host_weights), h->momentum, head, tail,    \
                                                     next_chunk);                                                     \
     else                                                                                                             \
       KERNEL<TARGS, false><<<GRID, THREADS, 0, s>>>(h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad,    \
-                                                     grad_stride, lr, eps, slot_of_lookup, caches,                   \
+                                                     grad_stride, lr, eps, slot_of_lookup, sorted_slot, caches,      \
                                                      static_cast<char*>(h->dev_weights),                             \
                                                      static_cast<char*>(h->host_weights), h->momentum, head, tail,   \
                                                      next_chunk);                                                    \
@@ -783,7 +790,7 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
   {
     LaunchScope scope(K_COMBINE_PARTIALS, s);
     combine_partials<FP16, NV><<<grid, BWD_WARPS * 32, 0, s>>>(
-        h->d_meta, h->T, keys, pos, N, lr, eps, slot_of_lookup, caches, static_cast<char*>(h->dev_weights),
+        h->d_meta, h->T, keys, pos, N, lr, eps, slot_of_lookup, sorted_slot, caches, static_cast<char*>(h->dev_weights),
         static_cast<char*>(h->host_weights), h->momentum, head, tail, group);
   }
 #undef MTS_LAUNCH_GH
@@ -878,13 +885,14 @@ extern "C" int mts_tbe_backward_sort(const mts_tables* h, int32_t B, const int64
 }
 
 namespace {
-// sorted_rows / sorted_pos / bag_of_lookup: null = the arrays mts_tbe_backward_sort left in the workspace
+// sorted_rows / sorted_bag / sorted_slot: null = the arrays mts_tbe_backward_sort left in the workspace (and
+// the slots through slot_of_lookup)
 int backward_apply(const mts_tables* h, int32_t B, const int64_t* offsets, int64_t N, int32_t pooling_mode,
                    const void* grad_out, bool grad_half, int64_t grad_stride, float lr, float eps,
                    const int32_t* slot_of_lookup, void* const* host_cache_data, uint8_t* const* host_cache_dirty,
                    int32_t n_caches, void* workspace, size_t workspace_bytes, void* stream,
-                   const uint32_t* sorted_rows = nullptr, const uint32_t* sorted_pos = nullptr,
-                   const uint32_t* bag_of_lookup = nullptr) {
+                   const uint32_t* sorted_rows = nullptr, const uint32_t* sorted_bag = nullptr,
+                   const int32_t* sorted_slot = nullptr) {
   if (!h) return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_apply: null tables");
   const BwdLayout L = bwd_layout(h, N > 0 ? N : 0);
   int rc = check_backward_common(h, B, offsets, N, workspace, workspace_bytes, L, "tbe_backward_apply");
@@ -909,15 +917,15 @@ int backward_apply(const mts_tables* h, int32_t B, const int64_t* offsets, int64
   const uint32_t* bag_of_pos = h->any_cached ? reinterpret_cast<const uint32_t*>(ws + L.bag_of_pos) : nullptr;
   if (sorted_rows != nullptr) {
     keys = sorted_rows;
-    pos = sorted_pos;
-    bag_of_pos = bag_of_lookup;
+    pos = sorted_bag;            // the value that travels with a key is its bag id: no position -> bag lookup
+    bag_of_pos = nullptr;
   }
   float* head = reinterpret_cast<float*>(ws + L.head);
   float* tail = reinterpret_cast<float*>(ws + L.tail);
   float* group = reinterpret_cast<float*>(ws + L.group);
   const int nv = (h->max_dim + 127) / 128;
   const bool fp16 = h->dtype == MTS_DTYPE_FP16;
-#define MTS_BWD(F, V, G) return launch_backward<F, V, G>(h, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad_out, grad_half, grad_stride, lr, eps, slot_of_lookup, caches, head, tail, group, reinterpret_cast<uint32_t*>(ws + L.next_chunk), s)
+#define MTS_BWD(F, V, G) return launch_backward<F, V, G>(h, B, keys, pos, bag_of_pos, N, offsets, pooling_mode, grad_out, grad_half, grad_stride, lr, eps, slot_of_lookup, sorted_slot, caches, head, tail, group, reinterpret_cast<uint32_t*>(ws + L.next_chunk), s)
   if (fp16) {
     if (nv <= 1) MTS_BWD(true, 1, MTS_BWD_GROUP1);
     if (nv <= 2) MTS_BWD(true, 2, MTS_BWD_GROUP2);
@@ -954,18 +962,17 @@ extern "C" int mts_tbe_backward_apply_f16(const mts_tables* h, int32_t B, const 
 extern "C" int mts_tbe_backward_apply_presorted(const mts_tables* h, int32_t B, const int64_t* offsets, int64_t N,
                                                 int32_t pooling_mode, const void* grad_out, int32_t grad_dtype,
                                                 int64_t grad_stride, float lr, float eps,
-                                                const uint32_t* sorted_rows, const uint32_t* sorted_pos,
-                                                const uint32_t* bag_of_lookup, const int32_t* slot_of_lookup,
-                                                void* const* host_cache_data, uint8_t* const* host_cache_dirty,
-                                                int32_t n_caches, void* workspace, size_t workspace_bytes,
-                                                void* stream) {
+                                                const uint32_t* sorted_rows, const uint32_t* sorted_bag,
+                                                const int32_t* sorted_slot, void* const* host_cache_data,
+                                                uint8_t* const* host_cache_dirty, int32_t n_caches,
+                                                void* workspace, size_t workspace_bytes, void* stream) {
   if (grad_dtype != MTS_DTYPE_FP32 && grad_dtype != MTS_DTYPE_FP16)
     return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_apply_presorted: grad_dtype %d", grad_dtype);
-  if (N > 0 && (!sorted_rows || !sorted_pos || !bag_of_lookup))
-    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_apply_presorted: null sorted_rows / sorted_pos / bag_of_lookup");
+  if (N > 0 && (!sorted_rows || !sorted_bag || !sorted_slot))
+    return set_error(MTS_ERR_INVALID_ARG, "tbe_backward_apply_presorted: null sorted_rows / sorted_bag / sorted_slot");
   return backward_apply(h, B, offsets, N, pooling_mode, grad_out, grad_dtype == MTS_DTYPE_FP16, grad_stride, lr, eps,
-                        slot_of_lookup, host_cache_data, host_cache_dirty, n_caches, workspace, workspace_bytes, stream,
-                        sorted_rows, sorted_pos, bag_of_lookup);
+                        sorted_slot, host_cache_data, host_cache_dirty, n_caches, workspace, workspace_bytes, stream,
+                        sorted_rows, sorted_bag, sorted_slot);
 }
 
 extern "C" int mts_tbe_backward_rowwise_adagrad(

@@ -5,6 +5,7 @@ Nothing here computes anything on its own; every step is a call into libmtrains_
 from __future__ import annotations
 
 import os
+import threading
 from typing import List, Optional, Sequence
 
 import numpy as np
@@ -155,8 +156,8 @@ class DeviceModel:
         # the lookups ordered by row (uint32 bit patterns), written by the tag step and reused by the backward
         return dict(slot=torch.full((n,), -1, dtype=torch.int32, device=dev),
                     sorted_rows=torch.empty(n, dtype=torch.int32, device=dev),
-                    sorted_pos=torch.empty(n, dtype=torch.int32, device=dev),
-                    bag_of_lookup=torch.empty(n, dtype=torch.int32, device=dev), lists=lists)
+                    sorted_bag=torch.empty(n, dtype=torch.int32, device=dev),
+                    sorted_slot=torch.empty(n, dtype=torch.int32, device=dev), lists=lists)
 
     @property
     def slot_of_lookup(self):
@@ -191,7 +192,7 @@ class DeviceModel:
             cx = self._ctx(ctx)
             mb.tbe_backward_apply_presorted(
                 self.tables, self.spec.batch, offsets, N, pooling_mode, grad_out, grad_out.shape[1], lr, eps,
-                cx["sorted_rows"], cx["sorted_pos"], cx["bag_of_lookup"], cx["slot"], self.cache_data,
+                cx["sorted_rows"], cx["sorted_bag"], cx["sorted_slot"], self.cache_data,
                 self.cache_dirty, self.workspace, self.ws_bytes, stream, f16=grad_out.dtype == torch.float16)
             return
         if grad_out.dtype == torch.float16:      # fp16 gradients: the two-call form
@@ -252,8 +253,8 @@ class DeviceModel:
                 c, self.tables, t0, t1, B, indices, offsets, begin, n, step, cx["slot"], L["miss_keys"],
                 L["miss_slots"], L["evict_keys"], L["evict_slots"], L["evict_dirty"], L["capacity"],
                 L["overflow_keys"], L["overflow_capacity"], L["counters"], self.cache_ws, self.cache_ws_bytes, stream,
-                sorted_rows_out=cx["sorted_rows"], sorted_pos_out=cx["sorted_pos"],
-                bag_of_lookup_out=cx["bag_of_lookup"])
+                sorted_rows_out=cx["sorted_rows"], sorted_bag_out=cx["sorted_bag"],
+                sorted_slot_out=cx["sorted_slot"])
 
     def cache_move(self, stream=None, ctx: Optional[int] = None) -> None:
         """Data path of one batch: save dirty victims, pull missed rows from the host tier, write victims back."""
@@ -273,7 +274,7 @@ class DeviceModel:
                                  L["evict_slots"], L["evict_dirty"], L["capacity"], L["counters"], L["staging"], stream)
 
     # ---- missed rows gathered by host threads and moved by the copy engine
-    FETCH_STAGE_BYTES = 192 << 20        # per cache and batch context; larger miss lists take cache_fetch
+    FETCH_STAGE_BYTES = 96 << 20         # per cache and batch context; larger miss / evict lists take the kernels
 
     def enable_host_gather(self, threads: Optional[int] = None) -> None:
         """Pinned host buffers (keys and gathered rows, per cache and batch context) and one device
@@ -281,8 +282,10 @@ class DeviceModel:
         if self.fetch_rows is not None:
             return
         esz = 4 if self.spec.dtype == wl.FP32 else 2
-        # the caches gather side by side (one worker each): share the cores out
-        self.gather_threads = threads or max(1, (os.cpu_count() or 1) // max(1, len(self.caches)))
+        # every gather / scatter uses all cores; the caches' workers take turns at it (one lock), so that a cache
+        # with many wide rows is not left with a third of the cores while the others idle
+        self.gather_threads = threads or os.cpu_count() or 1
+        self.host_copy_lock = threading.Lock()
         self.fetch_rows = [max(1, min(self.ctx[0]["lists"][g]["capacity"], self.FETCH_STAGE_BYTES // (c.dim * esz)))
                            for g, c in enumerate(self.caches)]
         self.fetch_dev = [torch.empty(r * c.dim * esz, dtype=torch.uint8, device=self.device)
@@ -291,6 +294,13 @@ class DeviceModel:
                             for r, c in zip(self.fetch_rows, self.caches)] for _ in range(self.N_CTX)]
         self.fetch_keys = [[torch.empty(r, dtype=torch.int64).pin_memory() for r in self.fetch_rows]
                            for _ in range(self.N_CTX)]
+        # the way back: dirty victims, their keys and dirty bytes
+        self.wb_host = [[torch.empty(r * c.dim * esz, dtype=torch.uint8).pin_memory()
+                         for r, c in zip(self.fetch_rows, self.caches)] for _ in range(self.N_CTX)]
+        self.wb_keys = [[torch.empty(r, dtype=torch.int64).pin_memory() for r in self.fetch_rows]
+                        for _ in range(self.N_CTX)]
+        self.wb_dirty = [[torch.empty(r, dtype=torch.uint8).pin_memory() for r in self.fetch_rows]
+                         for _ in range(self.N_CTX)]
 
     def cache_fetch_via_host(self, g: int, n_miss: int, copy_stream, stream, ctx: int, mark=None) -> bool:
         """Cache g, copy-engine path: the first n_miss keys of the miss list come to the host on
@@ -309,7 +319,8 @@ class DeviceModel:
                 keys_h[:n_miss].copy_(L["miss_keys"][:n_miss], non_blocking=True)
             copy_stream.synchronize()
             rows_h = self.fetch_host[ctx][g]
-            mb.host_gather_rows(self.host_rows_ptr(g), keys_h.numpy(), n_miss, rb, rows_h, self.gather_threads)
+            with self.host_copy_lock:
+                mb.host_gather_rows(self.host_rows_ptr(g), keys_h.numpy(), n_miss, rb, rows_h, self.gather_threads)
             with torch.cuda.stream(stream):
                 if mark is not None:
                     mark(f"copy{g}_begin")
@@ -319,6 +330,30 @@ class DeviceModel:
         mb.cache_place_fetched(c, self.fetch_dev[g], L["miss_slots"], L["evict_slots"], L["evict_dirty"],
                                L["capacity"], L["counters"], L["staging"], stream)
         return True
+
+    def cache_writeback_via_host_begin(self, g: int, n_evict: int, stream, ctx: int) -> bool:
+        """Cache g, copy-engine path of the write-back: the first n_evict entries of the evict list (keys, dirty
+        bytes) and of the staging buffer go to pinned host buffers on `stream` (after the placing kernel of the
+        same batch).  Returns False (nothing done) when they do not fit."""
+        if n_evict > self.fetch_rows[g]:
+            return False
+        if n_evict > 0:
+            L = self.ctx[ctx]["lists"][g]
+            rb = self.caches[g].dim * (4 if self.spec.dtype == wl.FP32 else 2)
+            with torch.cuda.stream(stream):
+                self.wb_keys[ctx][g][:n_evict].copy_(L["evict_keys"][:n_evict], non_blocking=True)
+                self.wb_dirty[ctx][g][:n_evict].copy_(L["evict_dirty"][:n_evict], non_blocking=True)
+                self.wb_host[ctx][g][:n_evict * rb].copy_(L["staging"][:n_evict * rb], non_blocking=True)
+        return True
+
+    def cache_writeback_via_host_finish(self, g: int, n_evict: int, ctx: int) -> None:
+        """Host threads put the dirty victims into their rows of the host tier (after the copies of
+        cache_writeback_via_host_begin have completed)."""
+        if n_evict > 0:
+            rb = self.caches[g].dim * (4 if self.spec.dtype == wl.FP32 else 2)
+            with self.host_copy_lock:
+                mb.host_scatter_rows(self.host_rows_ptr(g), self.wb_keys[ctx][g].numpy(), self.wb_dirty[ctx][g].numpy(),
+                                     n_evict, rb, self.wb_host[ctx][g], self.gather_threads)
 
     def cache_writeback(self, g: int, stream=None, ctx: Optional[int] = None) -> None:
         """Cache g: the staged dirty victims back to the host tier (after cache_fetch of the same batch)."""

@@ -139,6 +139,7 @@ class CachedTrainer:
             # the host reads the rows itself: the tag step of this batch is over (its counters are on the
             # host) and this cache's write-backs of earlier batches have reached host memory
             self.ev_tags[t].synchronize()
+            self._finish_writeback(g)
             if t > 0:
                 self.ev_moved[t - 1][g].synchronize()
             n_miss = int(self._host_counters[t, g, mb.COUNTER_NAMES.index("inserted")])
@@ -148,9 +149,31 @@ class CachedTrainer:
         if not done:
             self.m.cache_fetch(g, stream=s, ctx=ctx)
         self._mark(f"placed{g}", t, s)
-        self.m.cache_writeback(g, stream=s, ctx=ctx)
+        wb = False
+        if via_host:
+            # the victims take the copy engine as well; host threads put them into their rows before this
+            # cache's next gather (or at the end of the run)
+            n_evict = int(self._host_counters[t, g, mb.COUNTER_NAMES.index("evicted")])
+            wb = self.m.cache_writeback_via_host_begin(g, n_evict, s, ctx)
+            if wb:
+                e = torch.cuda.Event()
+                e.record(s)
+                self._pending_wb[g] = (e, n_evict, ctx)
+                if not self.pipelined:
+                    self._finish_writeback(g)
+        if not wb:
+            self.m.cache_writeback(g, stream=s, ctx=ctx)
         self._mark(f"move{g}_end", t, s)
         self.ev_moved[t][g].record(s)
+
+    def _finish_writeback(self, g):
+        """Cache g: the victims whose copy to the host was enqueued by an earlier batch go into their rows."""
+        pend = self._pending_wb[g]
+        if pend is not None:
+            e, n_evict, ctx = pend
+            e.synchronize()
+            self.m.cache_writeback_via_host_finish(g, n_evict, ctx)
+            self._pending_wb[g] = None
 
     def _finish_move(self, t):
         """After the data movement of batch t: repair the rows that overflowed in the batches whose backward may
@@ -189,6 +212,7 @@ class CachedTrainer:
             while True:
                 t = self._jobs[g].get()
                 if t is None:
+                    self._finish_writeback(g)
                     return
                 self._move_cache(t, g, True)
                 self._moved_recorded[t][g].set()
@@ -238,6 +262,7 @@ class CachedTrainer:
         self._host_counters = torch.zeros((K, n_c, n_cnt), dtype=torch.int64).pin_memory()
         self._threads = []
         self._worker_error = None
+        self._pending_wb = [None] * n_c
         if out is None:
             out = torch.empty((m.spec.batch, m.spec.total_dim), dtype=torch.float32, device=self.dev)
 
@@ -329,6 +354,8 @@ class CachedTrainer:
                 for th in self._threads:
                     th.join()
                 self._threads = []
+                if self._worker_error is not None:
+                    raise self._worker_error
         for s in [self.tag, self.fix] + self.copies + self.moves:
             self.main.wait_stream(s)
         torch.cuda.synchronize(self.dev)

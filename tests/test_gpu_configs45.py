@@ -215,8 +215,8 @@ def _tag_path_at_size(spec, n_batches, lock=2):
                         ms=torch.empty(n, dtype=torch.int32, device=d), ek=torch.empty(n, dtype=torch.int64, device=d),
                         es=torch.empty(n, dtype=torch.int32, device=d), ed=torch.empty(n, dtype=torch.uint8, device=d),
                         ok=torch.empty(n, dtype=torch.int64, device=d), cnt=torch.empty(mb.NUM_COUNTERS, dtype=torch.int64, device=d),
-                        srow=torch.empty(n, dtype=torch.int32, device=d), spos=torch.empty(n, dtype=torch.int32, device=d),
-                        bag=torch.empty(n, dtype=torch.int32, device=d), ws=torch.empty(wsb, dtype=torch.uint8, device=d), wsb=wsb)
+                        srow=torch.empty(n, dtype=torch.int32, device=d), sbag=torch.empty(n, dtype=torch.int32, device=d),
+                        sslot=torch.empty(n, dtype=torch.int32, device=d), ws=torch.empty(wsb, dtype=torch.uint8, device=d), wsb=wsb)
         d_idx, d_off = to_dev(idx), to_dev(off)
         keys_all = _group_keys(spec, groups, idx, off)
         for g, (dim, t0, t1) in enumerate(groups):
@@ -224,7 +224,7 @@ def _tag_path_at_size(spec, n_batches, lock=2):
             mb.cache_lookup_insert_tables(gc[g], tables, t0, t1, B, d_idx, d_off, lo, hi - lo, k, bufs["slot"], bufs["mk"],
                                           bufs["ms"], bufs["ek"], bufs["es"], bufs["ed"], bufs["n"], bufs["ok"], bufs["n"],
                                           bufs["cnt"], bufs["ws"], bufs["wsb"], sorted_rows_out=bufs["srow"],
-                                          sorted_pos_out=bufs["spos"], bag_of_lookup_out=bufs["bag"])
+                                          sorted_bag_out=bufs["sbag"], sorted_slot_out=bufs["sslot"])
             torch.cuda.synchronize()
             ref = oc[g].lookup_insert(keys_all[g], k)
             cnt = dict(zip(mb.COUNTER_NAMES, bufs["cnt"].cpu().tolist()))
@@ -241,15 +241,15 @@ def _tag_path_at_size(spec, n_batches, lock=2):
             oc[g].dirty[used] = 1
             ones = torch.ones(len(used), dtype=torch.uint8, device="cuda:0")
             as_tensor(gc[g].dirty_ptr, gc[g].num_sets * 32, torch.uint8)[to_dev(used.astype(np.int64))] = ones
-            # the exported order: linear row ids ascending, equal rows by position; positions are a permutation
+            # the exported order: linear row ids ascending, equal rows by position, with the bag and the slot of
+            # every lookup in that order
             srow = bufs["srow"][lo:hi].cpu().numpy().view(np.uint32).astype(np.int64)
-            spos = bufs["spos"][lo:hi].cpu().numpy().view(np.uint32).astype(np.int64)
             lin = keys_all[g] + int(spec.row_offset[t0])
             order = np.argsort(lin, kind="stable")
             np.testing.assert_array_equal(srow, lin[order])
-            np.testing.assert_array_equal(spos, order + lo)
-            bag = bufs["bag"][lo:hi].cpu().numpy().view(np.uint32).astype(np.int64)
-            np.testing.assert_array_equal(bag, np.repeat(np.arange(t0 * B, t1 * B), np.diff(off[t0 * B:t1 * B + 1])))
+            bag_of = np.repeat(np.arange(t0 * B, t1 * B), np.diff(off[t0 * B:t1 * B + 1]))
+            np.testing.assert_array_equal(bufs["sbag"][lo:hi].cpu().numpy().view(np.uint32).astype(np.int64), bag_of[order])
+            np.testing.assert_array_equal(bufs["sslot"][lo:hi].cpu().numpy(), ref["slot_of_lookup"][order])
         assert tables.status() == 0
     for c in gc:
         assert c.status() == 0
