@@ -583,17 +583,21 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
             e = torch.cuda.Event(enable_timing=True)
             e.record(main)
             marks[t] = e
+        if t == warmup - 1 and args.trace:
+            mb.trace_enable(True)          # per-kernel times of the launches from here on (the timed batches)
 
     sampler = ClockSampler(dev.index)
     sampler.start()
     time.sleep(0.3)
     launches0 = mb.launch_count()
-    if args.trace:
-        mb.trace_enable(True)
     sampler.mark(True)
     trainer.run(batches, glist, on_step=on_step)
     torch.cuda.synchronize(dev)
     sampler.mark(False)
+    kernels = None
+    if args.trace:
+        kernels = {k: {"ms_per_step": v[0] / steps, "launches_per_step": v[1] / steps} for k, v in mb.trace_report().items()}
+        mb.trace_enable(False)
     # diagnostics on the last batch, GPU otherwise idle: lookups that bypass the cache, forward and backward alone
     last_ctx = (K - 1) % DeviceModel.N_CTX
     n_last = batches[K - 1][0].numel()
@@ -607,10 +611,6 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
     f1.record(main)
     torch.cuda.synchronize(dev)
     fwd_alone_ms = f0.elapsed_time(f1) / 3
-    kernels = None
-    if args.trace:
-        kernels = {k: {"ms_per_step": v[0] / K, "launches_per_step": v[1] / K} for k, v in mb.trace_report().items()}
-        mb.trace_enable(False)
     clocks = sampler.stop()
     launches = mb.launch_count() - launches0
     ms = marks[warmup - 1].elapsed_time(marks[K - 1])

@@ -14,6 +14,9 @@
 #include <algorithm>
 #include <cstring>
 #include <thread>
+#if defined(__SSE2__)
+#include <emmintrin.h>
+#endif
 
 #include "common.cuh"
 
@@ -323,8 +326,9 @@ cache_probe_second_level(const uint32_t* __restrict__ miss_uidx, const uint32_t*
   }
 }
 
-// One warp per touched set; lane = way.
-__global__ void __launch_bounds__(CACHE_THREADS)
+// One warp per touched set; lane = way.  The walk is a chain of dependent loads per set, so the kernel lives
+// on resident warps: the register allocation is bounded for four blocks per SM.
+__global__ void __launch_bounds__(CACHE_THREADS, 4)
 cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of member j (ascending)
                     const uint32_t* __restrict__ member_uidx,     // distinct-key index of member j
                     const uint32_t* __restrict__ sseg_start, const uint32_t* __restrict__ n_sets,
@@ -344,14 +348,29 @@ cache_probe_replace(const uint32_t* __restrict__ set_sorted,      // set of memb
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   const uint32_t NS = *n_sets;
   unsigned long long c_hit_lookups = 0, c_uhits = 0, c_dirty = 0, c_overflow = 0, c_overflow_dirty = 0;
+  // The state of the warp's next set is requested before the current set is worked on (the sets of one warp
+  // are different sets, so nothing written below is read here): the chain set bounds -> set -> state of
+  // one set overlaps the work on the one before it.
+  uint32_t n_j0 = 0, n_j1 = 0, n_set = 0, n_tag = 0, n_cnt = 0;
+  int32_t n_stamp = 0, n_plc = 0;
+  auto request = [&](int64_t s_i) {
+    if (s_i < NS) {
+      n_j0 = sseg_start[s_i]; n_j1 = sseg_start[s_i + 1];
+      n_set = set_sorted[n_j0];
+      const int64_t at = (int64_t)n_set * 32 + lane;
+      n_tag = tags[at]; n_stamp = ts[at]; n_cnt = freq[at]; n_plc = placed_at[at];
+    }
+  };
+  request(warp0);
   for (int64_t si = warp0; si < NS; si += nwarps) {
-    const uint32_t j0 = sseg_start[si], j1 = sseg_start[si + 1];
-    const uint32_t set = set_sorted[j0];
+    const uint32_t j0 = n_j0, j1 = n_j1;
+    const uint32_t set = n_set;
     const int64_t slot0 = (int64_t)set * 32;
-    uint32_t tag = tags[slot0 + lane];
-    int32_t stamp = ts[slot0 + lane];
-    uint32_t cnt = freq[slot0 + lane];
-    int32_t plc = placed_at[slot0 + lane];
+    uint32_t tag = n_tag;
+    int32_t stamp = n_stamp;
+    uint32_t cnt = n_cnt;
+    int32_t plc = n_plc;
+    request(si + nwarps);
     bool touched = false;
     // pass 1: probe every member against the state before the call, refresh the hits
     for (uint32_t jb = j0; jb < j1; jb += 32) {
@@ -1513,6 +1532,26 @@ extern "C" int mts_cache_prefetch_misses(mts_cache* c, const void* host_rows_map
   return check_launch("cache_save_victims / cache_fetch_misses");
 }
 
+// Host-side row copy whose destination is not read again by this core: non-temporal 16-byte stores where the
+// CPU has them and both sides are 16-byte multiples, so that the rows go to memory instead of filling the
+// cores' caches (the copy engine, which reads the gathered rows next, would have to pull them out of there).
+static inline void host_copy_row_streaming(char* dst, const char* src, size_t bytes) {
+#if defined(__SSE2__)
+  if ((((uintptr_t)dst | bytes) & 15) == 0) {
+    for (size_t b = 0; b < bytes; b += 16)
+      _mm_stream_si128(reinterpret_cast<__m128i*>(dst + b), _mm_loadu_si128(reinterpret_cast<const __m128i*>(src + b)));
+    return;
+  }
+#endif
+  memcpy(dst, src, bytes);
+}
+
+static inline void host_copy_fence() {
+#if defined(__SSE2__)
+  _mm_sfence();
+#endif
+}
+
 extern "C" int mts_host_gather_rows(const void* host_rows, const int64_t* host_keys, int64_t n, int64_t row_bytes,
                                     void* host_out, int32_t threads) {
   if (n < 0 || row_bytes < 1 || (n > 0 && (!host_rows || !host_keys || !host_out)))
@@ -1528,8 +1567,9 @@ extern "C" int mts_host_gather_rows(const void* host_rows, const int64_t* host_k
         const char* ahead = src + (size_t)host_keys[k + AHEAD] * rb;
         for (size_t b = 0; b < rb; b += 64) __builtin_prefetch(ahead + b, 0, 0);
       }
-      memcpy(dst + (size_t)k * rb, src + (size_t)host_keys[k] * rb, rb);
+      host_copy_row_streaming(dst + (size_t)k * rb, src + (size_t)host_keys[k] * rb, rb);
     }
+    host_copy_fence();
   };
   const int64_t nt = std::max<int64_t>(1, std::min<int64_t>(threads, (n + 1023) / 1024));
   if (nt == 1) { work(0, n); return MTS_OK; }
@@ -1551,7 +1591,8 @@ extern "C" int mts_host_scatter_rows(void* host_rows, const int64_t* host_keys, 
   const size_t rb = (size_t)row_bytes;
   auto work = [=](int64_t k0, int64_t k1) {
     for (int64_t k = k0; k < k1; ++k)
-      if (host_mask == nullptr || host_mask[k]) memcpy(dst + (size_t)host_keys[k] * rb, src + (size_t)k * rb, rb);
+      if (host_mask == nullptr || host_mask[k]) host_copy_row_streaming(dst + (size_t)host_keys[k] * rb, src + (size_t)k * rb, rb);
+    host_copy_fence();
   };
   const int64_t nt = std::max<int64_t>(1, std::min<int64_t>(threads, (n + 1023) / 1024));
   if (nt == 1) { work(0, n); return MTS_OK; }

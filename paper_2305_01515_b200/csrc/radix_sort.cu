@@ -404,7 +404,9 @@ int radix_sort_pairs(uint32_t* keys_a, uint32_t* vals_a, uint32_t* keys_b, uint3
   *vals_out = vals_a;
   if (n_max <= 1 || key_bits <= 0) return MTS_OK;
   const int64_t ntiles = ceil_div(n_max, SORT_TILE);
-  const int G = (int)std::min<int64_t>(ntiles, SORT_MAX_BLOCKS);
+  // a device-resident count is usually far below its host bound (the keys that missed, the victims): fewer
+  // blocks then, so that the histogram and its scan are not sized for the bound
+  const int G = (int)std::min<int64_t>(ntiles, n_dev != nullptr ? 256 : SORT_MAX_BLOCKS);
   const SortSegments none{nullptr, 0, nullptr, key_base};
   return run_passes<false>(keys_a, vals_a, keys_b, vals_b, n_max, n_dev, key_bits, hist, G, 1, none, keys_out, vals_out,
                            stream);
