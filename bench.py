@@ -562,14 +562,17 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
     model = DeviceModel(spec, device=dev, lock_depth=args.lock_depth, policy=policy, l2_fraction=args.l2_fraction)
     h2d_gbs, d2h_gbs = host_link_bandwidth(dev)
     stream = wl.BatchStream(spec)
+    # the tag step and the data movement run up to COOLDOWN batches ahead of the training: that many batches
+    # follow the timed ones, so that every timed step carries the side work of a steady state
+    COOLDOWN = 3
     K = warmup + steps
-    host = [stream.next() for _ in range(K)]
+    host = [stream.next() for _ in range(K + COOLDOWN)]
     n_max = max(len(b[0]) for b in host)
     model.reserve(n_max)
     batches = [(torch.from_numpy(i).to(dev), torch.from_numpy(o).to(dev), o) for i, o in host]
     R = min(4, K)
     grads = [torch.from_numpy(wl.gen_grad(spec, k)).to(dev) for k in range(R)]
-    glist = [grads[k % R] for k in range(K)]
+    glist = [grads[k % R] for k in range(K + COOLDOWN)]
     setup_s = time.time() - t_setup
     trainer = CachedTrainer(model, pipelined=not args.sequential, host_gather=args.fetch == "host",
                             tag_on_main=not args.tag_stream)
@@ -577,14 +580,18 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
     gather_gbs = host_gather_rates(model) if args.fetch == "host" else None
     main = torch.cuda.current_stream(dev)
     marks = {}
+    traced = []
 
     def on_step(t):
-        if t >= warmup - 1:
+        if warmup - 1 <= t < K:
             e = torch.cuda.Event(enable_timing=True)
             e.record(main)
             marks[t] = e
         if t == warmup - 1 and args.trace:
-            mb.trace_enable(True)          # per-kernel times of the launches from here on (the timed batches)
+            mb.trace_enable(True)          # per-kernel times of the launches from here on
+        if t == K - 1 and args.trace:
+            traced.append(mb.trace_report())
+            mb.trace_enable(False)
 
     sampler = ClockSampler(dev.index)
     sampler.start()
@@ -595,19 +602,19 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
     torch.cuda.synchronize(dev)
     sampler.mark(False)
     kernels = None
-    if args.trace:
-        kernels = {k: {"ms_per_step": v[0] / steps, "launches_per_step": v[1] / steps} for k, v in mb.trace_report().items()}
-        mb.trace_enable(False)
+    if args.trace and traced:
+        kernels = {k: {"ms_per_step": v[0] / steps, "launches_per_step": v[1] / steps} for k, v in traced[0].items()}
     # diagnostics on the last batch, GPU otherwise idle: lookups that bypass the cache, forward and backward alone
-    last_ctx = (K - 1) % DeviceModel.N_CTX
-    n_last = batches[K - 1][0].numel()
+    K_all = K + COOLDOWN
+    last_ctx = (K_all - 1) % DeviceModel.N_CTX
+    n_last = batches[K_all - 1][0].numel()
     bypass = int((model.ctx[last_ctx]["slot"][:n_last] < 0).sum().item())
     out_d = torch.empty((spec.batch, spec.total_dim), dtype=torch.float32, device=dev)
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    model.forward(batches[K - 1][0], batches[K - 1][1], n_last, out=out_d, stream=main, ctx=last_ctx)
+    model.forward(batches[K_all - 1][0], batches[K_all - 1][1], n_last, out=out_d, stream=main, ctx=last_ctx)
     f0.record(main)
     for _ in range(3):
-        model.forward(batches[K - 1][0], batches[K - 1][1], n_last, out=out_d, stream=main, ctx=last_ctx)
+        model.forward(batches[K_all - 1][0], batches[K_all - 1][1], n_last, out=out_d, stream=main, ctx=last_ctx)
     f1.record(main)
     torch.cuda.synchronize(dev)
     fwd_alone_ms = f0.elapsed_time(f1) / 3
@@ -615,7 +622,7 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
     launches = mb.launch_count() - launches0
     ms = marks[warmup - 1].elapsed_time(marks[K - 1])
     per_step = sorted(marks[t - 1].elapsed_time(marks[t]) for t in range(warmup, K))
-    hist = np.stack(trainer.history)[warmup:]                      # [steps, caches, counters]
+    hist = np.stack(trainer.history)[warmup:K]                     # [steps, caches, counters]
     lookups = float(hist[:, :, 0].sum())
     hit = float(hist[:, :, 2].sum()) / max(lookups, 1.0)
     eb = spec.elem_bytes
@@ -670,7 +677,8 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
         by_batch = {}
         for name, t, ms_at in trainer.timeline():
             by_batch.setdefault(t, {})[name] = round(ms_at, 2)
-        rec["timeline_ms"] = {str(t): dict(sorted(by_batch[t].items(), key=lambda kv: kv[1])) for t in sorted(by_batch)[-4:]}
+        rec["timeline_ms"] = {str(t): dict(sorted(by_batch[t].items(), key=lambda kv: kv[1]))
+                              for t in sorted(by_batch) if K - 4 <= t < K}
     if two_level:
         l2_hits = float(hist[:, :, 10].sum())
         rec["two_level"] = {"l2_fraction": args.l2_fraction, "l1_hit_rate_per_lookup": hit,
