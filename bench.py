@@ -46,7 +46,7 @@ def make_spec(name: str, rank: int, args=None):
     if name == "cfg2":
         return wl.config2(seed=rank, tables=tables) if tables else wl.config2(seed=rank)
     if name == "cfg3":
-        return wl.config3(seed=rank)
+        return wl.config3(seed=rank, tables=tables) if tables else wl.config3(seed=rank)
     if name == "cfg4":
         return wl.config4(seed=rank, hbm_budget_gb=getattr(args, "budget_gb", wl.BENCH_CFG4_BUDGET_GB),
                           n_batches=getattr(args, "warmup", 12) + getattr(args, "steps", 8))
@@ -782,7 +782,7 @@ def main():
     ap.add_argument("--trace", action="store_true",
                     help="cached workloads: CUDA events around every launch of the run (perturbs the timing)")
     ap.add_argument("--tables", type=int, default=0,
-                    help="cfg2 only: fewer tables (a small case for profiler captures; not a bench line)")
+                    help="cfg2 / cfg3: fewer tables (a small case for profiler captures; not a bench line)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

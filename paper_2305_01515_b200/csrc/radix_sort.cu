@@ -426,10 +426,12 @@ int radix_sort_pairs_segmented(uint32_t* keys_a, uint32_t* vals_a, uint32_t* key
 // ------------------------------------------------------------------------------------ distinct keys
 
 constexpr int UNIQ_THREADS = 256;
+constexpr int UNIQ_ITEMS = 4;                       // consecutive keys per thread and round: one block scan per 1024 keys
 
 __device__ __forceinline__ int64_t per_block_of(int64_t n, int G) {
   const int64_t per = (n + G - 1) / G;
-  return (per + UNIQ_THREADS - 1) / UNIQ_THREADS * UNIQ_THREADS;
+  constexpr int64_t ROUND = UNIQ_THREADS * UNIQ_ITEMS;
+  return (per + ROUND - 1) / ROUND * ROUND;
 }
 
 __global__ void __launch_bounds__(UNIQ_THREADS)
@@ -485,14 +487,27 @@ write_heads(const uint32_t* __restrict__ keys, int64_t n_max, const uint32_t* __
   const int64_t begin = (int64_t)blockIdx.x * per_block;
   const int64_t end = min(n, begin + per_block);
   uint32_t base = base_of_block[blockIdx.x];
-  for (int64_t t0 = begin; t0 < end; t0 += UNIQ_THREADS) {
-    const int64_t i = t0 + threadIdx.x;
-    const bool valid = i < end;
-    const uint32_t head = (valid && (i == 0 || keys[i] != keys[i - 1])) ? 1u : 0u;
+  for (int64_t t0 = begin; t0 < end; t0 += UNIQ_THREADS * UNIQ_ITEMS) {
+    // a thread looks at UNIQ_ITEMS consecutive keys
+    const int64_t i0 = t0 + (int64_t)threadIdx.x * UNIQ_ITEMS;
+    uint32_t k[UNIQ_ITEMS + 1];
+    k[0] = (i0 > 0 && i0 < end) ? keys[i0 - 1] : 0u;
+#pragma unroll
+    for (int j = 0; j < UNIQ_ITEMS; ++j) k[j + 1] = i0 + j < end ? keys[i0 + j] : 0u;
+    uint32_t head[UNIQ_ITEMS], mine = 0;
+#pragma unroll
+    for (int j = 0; j < UNIQ_ITEMS; ++j) {
+      head[j] = (i0 + j < end && (i0 + j == 0 || k[j + 1] != k[j])) ? 1u : 0u;
+      mine += head[j];
+    }
     uint32_t total;
-    uint32_t ex = block_exclusive_scan_256(head, sh, &total);
-    if (head) seg_start[base + ex] = (uint32_t)i;
-    if (valid && uniq_idx) uniq_idx[i] = base + ex + head - 1u;
+    uint32_t at = base + block_exclusive_scan_256(mine, sh, &total);
+#pragma unroll
+    for (int j = 0; j < UNIQ_ITEMS; ++j) {
+      if (head[j]) seg_start[at] = (uint32_t)(i0 + j);
+      at += head[j];
+      if (i0 + j < end && uniq_idx) uniq_idx[i0 + j] = at - 1u;
+    }
     base += total;
   }
 }
