@@ -39,6 +39,9 @@ namespace mts {
 #ifndef MTS_BWD_LEAN_MINBLK
 #define MTS_BWD_LEAN_MINBLK 16  // resident blocks per SM reduce_chunks_lean is bounded for (32 registers)
 #endif
+#ifndef MTS_BWD_LEAN_MINBLK2
+#define MTS_BWD_LEAN_MINBLK2 12 // the same for its two-piece form (rows of 129..256 columns)
+#endif
 #ifndef MTS_BWD_GROUP2
 #define MTS_BWD_GROUP2 1        // the same for rows of 129..256 columns
 #endif
@@ -386,13 +389,17 @@ reduce_chunks(const TableMeta* __restrict__ meta, int T, int32_t B,
   }
 }
 
-// ---- reduce_chunks_lean: the same walk for rows of up to 128 columns (one 16-byte piece per lane).
-// The walk is bound by instruction issue and by the latency of dependent instructions, not by
-// bytes in flight, so this form keeps one lookup in flight per warp, fits 32 registers and runs 64
-// warps per SM; a row's loads (gradient slice, and row + state where the row ends) are issued
-// together.  Same summation order and arithmetic as reduce_chunks.
-template <bool FP16, bool MEAN, bool GH>
-__global__ void __launch_bounds__(LEAN_WARPS * 32, MTS_BWD_LEAN_MINBLK)
+// ---- reduce_chunks_lean: the same walk for rows of up to NVL x 128 columns (NVL 16-byte gradient pieces
+// per lane, NVL = 1 or 2).  The walk is bound by instruction issue and by the latency of dependent
+// instructions, not by bytes in flight, so this form keeps one lookup in flight per warp, fits 32 registers
+// (NVL = 1: 64 warps per SM) and issues a row's loads (gradient slice, and row + state where the row
+// ends) together.  Same summation order and arithmetic as reduce_chunks.  PNV = pieces per lane of a stored
+// partial sum (the layout combine_partials reads), >= NVL.
+// `klass` splits the chunks of a model with narrow (<= 128 columns) and wide tables between two launches:
+// 0 = every chunk, 1 = only chunks that touch no wide table, 2 = only the others.  The sorted lookups are
+// ordered by table, so the tables of a chunk are those from its first lookup's to its last one's.
+template <bool FP16, int NVL, int PNV, bool MEAN, bool GH>
+__global__ void __launch_bounds__(LEAN_WARPS * 32, (NVL == 1 ? MTS_BWD_LEAN_MINBLK : MTS_BWD_LEAN_MINBLK2))
 reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
                    const uint32_t* __restrict__ keys, const uint32_t* __restrict__ pos,
                    const uint32_t* __restrict__ bag_of_pos, int64_t n,
@@ -401,15 +408,22 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
                    const int32_t* __restrict__ slot_of_lookup, const int32_t* __restrict__ sorted_slot,
                    const __grid_constant__ CachePtrs caches, char* dev_w, char* host_w,
                    float* __restrict__ momentum, float* __restrict__ partial_head,
-                   float* __restrict__ partial_tail, uint32_t* __restrict__ next_chunk) {
+                   float* __restrict__ partial_tail, uint32_t* __restrict__ next_chunk, int klass) {
+  static_assert(NVL >= 1 && NVL <= 2 && PNV >= NVL, "piece counts");
   constexpr int EB = FP16 ? 2 : 4;
-  constexpr int PSTRIDE = 128;
+  constexpr int PSTRIDE = PNV * 128;
   __shared__ uint4 s_desc[LEAN_WARPS][32];      // {gradient float offset, key, row address lo, hi}
   __shared__ uint2 s_aux[LEAN_WARPS][32];       // {dim, mean-pooling scale bits}
   __shared__ uint8_t* s_dirty[LEAN_WARPS][32];
   const int lane = threadIdx.x & 31;
   const int wib = threadIdx.x >> 5;
   const int64_t lane_elem = lane * 4;
+  auto store_partial = [&](float* dst, int64_t chunk, const float4 (&acc)[NVL]) {
+#pragma unroll
+    for (int q = 0; q < PNV; ++q)
+      *reinterpret_cast<float4*>(dst + chunk * PSTRIDE + (q * 32 + lane) * 4) =
+          q < NVL ? acc[q < NVL ? q : 0] : make_float4(0.f, 0.f, 0.f, 0.f);
+  };
   // Chunks differ a lot in cost (a chunk inside one hot row is a plain sum, a chunk of rows seen
   // once is 128 updates), so a warp takes its next chunk from a counter instead of a fixed share.
   for (;;) {
@@ -419,9 +433,20 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
   const int64_t p0 = chunk * BWD_CHUNK;
   if (p0 >= n) return;
   const int len = (int)min((int64_t)BWD_CHUNK, n - p0);
+  if (klass != 0) {
+    uint32_t bag_a = pos[p0], bag_b = pos[p0 + len - 1];
+    if (bag_of_pos != nullptr) { bag_a = bag_of_pos[bag_a]; bag_b = bag_of_pos[bag_b]; }
+    const int t_a = (int)(bag_a / (uint32_t)B), t_b = (int)(bag_b / (uint32_t)B);
+    bool wide = false;
+    for (int t = t_a + lane; t <= t_b; t += 32) wide |= meta[t].dim > 128;
+    wide = __any_sync(0xffffffffu, wide);
+    if (wide != (klass == 2)) continue;
+  }
   // a row that started in an earlier chunk: its piece here goes to combine_partials
   bool open_head = p0 > 0 && keys[p0 - 1] == keys[p0];
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 acc[NVL];
+#pragma unroll
+  for (int q = 0; q < NVL; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
   bool last_is_end = true;
 
   for (int k0 = 0; k0 < len; k0 += 32) {
@@ -472,61 +497,79 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
     const float inv_dim0 = __frcp_rn((float)dim0);
 
     // walk the 32 lookups run by run: the lookups before the next "last of its row" are only
-    // summed (no test per lookup), then that lookup closes its row.  `full` = every row of the
-    // batch has 128 columns: all lanes take part and the width is a constant.
-    auto walk = [&](auto full) {
-    constexpr bool FULL = decltype(full)::value;
-    auto add_scaled = [&](const GradPiece<GH>& g, int jj) {
-      if (MEAN) fma_piece<GH>(acc, __uint_as_float(s_aux[wib][jj].y), g);
-      else add_piece<GH>(acc, g);
+    // summed (no test per lookup), then that lookup closes its row.  WIDTH = 128 or 256: every row of
+    // the batch has that many columns (all lanes take part, the width is a constant); 0 = any widths.
+    auto walk = [&](auto width) {
+    constexpr int WIDTH = decltype(width)::value;
+    constexpr int NP = WIDTH == 128 ? 1 : NVL;                     // pieces a lane loads per lookup
+    constexpr int RUN = NP == 1 ? LEAN_RUN : (LEAN_RUN > 1 ? LEAN_RUN / 2 : 1);
+    struct Pieces { GradPiece<GH> q[NP]; };
+    auto add_scaled = [&](const Pieces& g, int jj) {
+      if (MEAN) {
+        const float sc = __uint_as_float(s_aux[wib][jj].y);
+#pragma unroll
+        for (int q = 0; q < NP; ++q) fma_piece<GH>(acc[q], sc, g.q[q]);
+      } else {
+#pragma unroll
+        for (int q = 0; q < NP; ++q) add_piece<GH>(acc[q], g.q[q]);
+      }
     };
-    auto load_grad = [&](int jj) {
-      const int dim = FULL ? 128 : uniform ? dim0 : (int)s_aux[wib][jj].x;
-      return load_piece<GH>(grad, lane_elem + s_desc[wib][jj].x, FULL || lane * 4 < dim);
+    auto load_at = [&](uint32_t goff, int dim) {
+      Pieces g;
+#pragma unroll
+      for (int q = 0; q < NP; ++q)
+        g.q[q] = load_piece<GH>(grad, lane_elem + q * 128 + goff, WIDTH != 0 || (q * 32 + lane) * 4 < dim);
+      return g;
     };
+    auto dim_of = [&](int jj) { return WIDTH != 0 ? WIDTH : uniform ? dim0 : (int)s_aux[wib][jj].x; };
+    auto load_grad = [&](int jj) { return load_at(s_desc[wib][jj].x, dim_of(jj)); };
     int j = 0;
     while (j < cnt) {
       const uint32_t rest = ends >> j;
       const int e = rest ? j + __ffs(rest) - 1 : cnt;              // next lookup that ends a row (or none)
-      for (; j + LEAN_RUN <= e; j += LEAN_RUN) {
-        GradPiece<GH> g[LEAN_RUN];
+      for (; j + RUN <= e; j += RUN) {
+        Pieces g[RUN];
 #pragma unroll
-        for (int u = 0; u < LEAN_RUN; ++u) g[u] = load_grad(j + u);
+        for (int u = 0; u < RUN; ++u) g[u] = load_grad(j + u);
 #pragma unroll
-        for (int u = 0; u < LEAN_RUN; ++u) add_scaled(g[u], j + u);
+        for (int u = 0; u < RUN; ++u) add_scaled(g[u], j + u);
       }
       for (; j < e; ++j) add_scaled(load_grad(j), j);
       if (e < cnt) {
         const uint4 d = s_desc[wib][e];
-        const int dim = FULL ? 128 : uniform ? dim0 : (int)s_aux[wib][e].x;
-        const GradPiece<GH> g = load_piece<GH>(grad, lane_elem + d.x, FULL || lane * 4 < dim);
+        const int dim = dim_of(e);
+        const Pieces g = load_at(d.x, dim);
         if (open_head) {
           add_scaled(g, e);
-          *reinterpret_cast<float4*>(partial_head + chunk * PSTRIDE + lane * 4) = acc;
+          store_partial(partial_head, chunk, acc);
           open_head = false;
         } else {
-          uint4 w[1];
+          uint4 w[NP];
           char* wp = reinterpret_cast<char*>((uintptr_t)d.z | ((uintptr_t)d.w << 32));
-          load_row<FP16, 1>(w, wp, dim);
+          load_row<FP16, NP>(w, wp, dim);
           const float m_old = momentum[d.y];
           add_scaled(g, e);
-          float4 a1[1] = {acc};
-          adagrad_row<FP16, 1>(a1, w, m_old, dim, FULL ? 0.0078125f : uniform ? inv_dim0 : __frcp_rn((float)dim), lr, eps, wp,
-                               momentum + d.y, any_dirty ? s_dirty[wib][e] : nullptr);
+          float4 a[NP];
+#pragma unroll
+          for (int q = 0; q < NP; ++q) a[q] = acc[q];
+          adagrad_row<FP16, NP>(a, w, m_old, dim,
+                                WIDTH == 128 ? 0.0078125f : WIDTH == 256 ? 0.00390625f : uniform ? inv_dim0 : __frcp_rn((float)dim),
+                                lr, eps, wp, momentum + d.y, any_dirty ? s_dirty[wib][e] : nullptr);
         }
-        acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int q = 0; q < NVL; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
         j = e + 1;
       }
     }
     };
-    if (uniform && dim0 == 128) walk(std::true_type{});
-    else walk(std::false_type{});
+    if (uniform && dim0 == 128) walk(std::integral_constant<int, 128>{});
+    else if (NVL == 2 && uniform && dim0 == 256) walk(std::integral_constant<int, (NVL == 2 ? 256 : 0)>{});
+    else walk(std::integral_constant<int, 0>{});
     __syncwarp();      // the next batch overwrites the staged descriptions
   }
   if (!last_is_end) {
     // open_head still set: the whole chunk lies inside a row that started earlier
-    float* dst = open_head ? partial_head : partial_tail;
-    *reinterpret_cast<float4*>(dst + chunk * PSTRIDE + lane * 4) = acc;
+    store_partial(open_head ? partial_head : partial_tail, chunk, acc);
   }
   }
 }
@@ -758,20 +801,46 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
                                                      static_cast<char*>(h->host_weights), h->momentum, head, tail,   \
                                                      next_chunk);                                                    \
   } while (0)
-  if constexpr (NV == 1 && MTS_BWD_USE_LEAN) {
+  if constexpr (NV <= 2 && MTS_BWD_USE_LEAN) {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
     // as many blocks as fit on the device at once (or fewer); the warps share out the chunks
     // With cached tables the step shares the GPU with the cache's tag lookup and data movement on other
     // streams: blocks that stay until the last chunk would keep every warp slot for the whole kernel and
     // hold those streams back, so there the grid covers the chunks and a block leaves after one round.
-    const unsigned lean_grid = h->any_cached
-        ? (unsigned)ceil_div(chunks, LEAN_WARPS)
-        : (unsigned)std::min<int64_t>(ceil_div(chunks, LEAN_WARPS), (int64_t)h->sm_count * MTS_BWD_LEAN_MINBLK);
-    if (cudaMemsetAsync(next_chunk, 0, sizeof(uint32_t), s) != cudaSuccess) return check_launch("memset(next_chunk)");
-    if (pooling_mode == MTS_POOL_MEAN)
-      MTS_LAUNCH_GH(reduce_chunks_lean, FP16 COMMA true, lean_grid, LEAN_WARPS * 32);
-    else
-      MTS_LAUNCH_GH(reduce_chunks_lean, FP16 COMMA false, lean_grid, LEAN_WARPS * 32);
+    auto lean_grid = [&](int resident) {
+      return h->any_cached ? (unsigned)ceil_div(chunks, LEAN_WARPS)
+                           : (unsigned)std::min<int64_t>(ceil_div(chunks, LEAN_WARPS), (int64_t)h->sm_count * resident);
+    };
+    // NVL pieces per lane over the chunks of class `klass`
+    auto launch_lean = [&](auto nvl, int klass) -> bool {
+      constexpr int NVL = decltype(nvl)::value;
+      if (cudaMemsetAsync(next_chunk, 0, sizeof(uint32_t), s) != cudaSuccess) return false;
+      const unsigned g = lean_grid(NVL == 1 ? MTS_BWD_LEAN_MINBLK : MTS_BWD_LEAN_MINBLK2);
+      const bool mean = pooling_mode == MTS_POOL_MEAN;
+#define MTS_LEAN(M, G)                                                                                              \
+      reduce_chunks_lean<FP16, NVL, NV, M, G><<<g, LEAN_WARPS * 32, 0, s>>>(                                        \
+          h->d_meta, h->T, B, keys, pos, bag_of_pos, N, offsets, grad, grad_stride, lr, eps, slot_of_lookup,        \
+          sorted_slot, caches, static_cast<char*>(h->dev_weights), static_cast<char*>(h->host_weights), h->momentum, \
+          head, tail, next_chunk, klass)
+      if (mean) { if (grad_half) MTS_LEAN(true, true); else MTS_LEAN(true, false); }
+      else      { if (grad_half) MTS_LEAN(false, true); else MTS_LEAN(false, false); }
+#undef MTS_LEAN
+      return true;
+    };
+    bool ok = true;
+    if constexpr (NV == 1) {
+      ok = launch_lean(std::integral_constant<int, 1>{}, 0);
+    } else {
+      int min_dim = h->max_dim;
+      for (const auto& m : h->h_meta) min_dim = std::min<int>(min_dim, m.dim);
+      if (min_dim > 128) {
+        ok = launch_lean(std::integral_constant<int, 2>{}, 0);
+      } else {
+        // narrow and wide tables: the chunks of the narrow ones keep the one-piece walk and its occupancy
+        ok = launch_lean(std::integral_constant<int, 1>{}, 1) && launch_lean(std::integral_constant<int, 2>{}, 2);
+      }
+    }
+    if (!ok) return check_launch("memset(next_chunk)");
   } else {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
     constexpr int resident = NV == 1 ? MTS_BWD_MINBLK : NV == 2 ? MTS_BWD_MINBLK2 : 2;
