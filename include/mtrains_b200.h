@@ -442,6 +442,7 @@ int mts_cache_prefetch_misses(mts_cache* cache, const void* host_rows_mapped, co
  * host_out to a device buffer `fetched`; (3) mts_cache_place_fetched, on `stream` after that copy: saves
  * the dirty victims like mts_cache_prefetch_misses, then fetched[k] -> slot miss_slots[k] for every k
  * below min(MTS_CNT_INSERTED, list_capacity).  fetched: device [>= that many rows, dim], 16-byte aligned.
+ * evict_staging NULL: the victims were saved already (mts_cache_save_victims), only place.
  * Errors: INVALID_ARG, ALIGNMENT, CUDA. */
 int mts_host_gather_rows(const void* host_rows, const int64_t* host_keys, int64_t n, int64_t row_bytes,
                          void* host_out, int32_t threads);
@@ -455,6 +456,13 @@ int mts_host_scatter_rows(void* host_rows, const int64_t* host_keys, const uint8
 int mts_cache_place_fetched(mts_cache* cache, const void* fetched, const int32_t* miss_slots,
                             const int32_t* evict_slots, const uint8_t* evict_dirty, int64_t list_capacity,
                             const int64_t* counters, void* evict_staging, void* stream);
+/* The first half of mts_cache_place_fetched alone (Section 5.5.4): the rows of the dirty victims, slot ->
+ * evict_staging[k].  A victim's row is final once the lookup that chose it has run (no batch in flight may
+ * use it), so the caller can save and copy the victims out on a second stream while the host still gathers
+ * the missed rows; mts_cache_place_fetched with evict_staging = NULL then only places (the caller orders it
+ * after this call, e.g. with an event).  Errors: INVALID_ARG, ALIGNMENT, CUDA. */
+int mts_cache_save_victims(mts_cache* cache, const int32_t* evict_slots, const uint8_t* evict_dirty,
+                           int64_t list_capacity, const int64_t* counters, void* evict_staging, void* stream);
 
 /* Evicted dirty rows go back to the host tier: evict_staging[k] -> host row evict_keys[k]. */
 int mts_cache_writeback_evicted(mts_cache* cache, void* host_rows_mapped, const int64_t* evict_keys,

@@ -38,7 +38,7 @@ EXPORTS = (
     "mts_tbe_backward_apply_presorted", "mts_cache_create_host_level", "mts_cache2_workspace_bytes",
     "mts_cache2_lookup_insert", "mts_cache2_move", "mts_cache_import_state", "mts_cache_set_fetch_wait_limit",
     "mts_place_tables",
-    "mts_cache_prefetch_misses", "mts_host_gather_rows", "mts_host_scatter_rows", "mts_cache_place_fetched", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
+    "mts_cache_prefetch_misses", "mts_host_gather_rows", "mts_host_scatter_rows", "mts_cache_place_fetched", "mts_cache_save_victims", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
     "mts_cache_export_state",
 )
 
@@ -122,6 +122,7 @@ def lib():
         L.mts_host_gather_rows.argtypes = [vp, vp, i64, i64, vp, i32]
         L.mts_host_scatter_rows.argtypes = [vp, vp, vp, i64, i64, vp, i32]
         L.mts_cache_place_fetched.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, vp]
+        L.mts_cache_save_victims.argtypes = [vp, vp, vp, i64, vp, vp, vp]
         L.mts_cache_flush.argtypes = [vp, vp, vp]
         L.mts_cache_export_state.argtypes = [vp, vp, vp, vp, vp, vp]
         L.mts_cache_import_state.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -437,6 +438,12 @@ def cache_place_fetched(cache: Cache, fetched, miss_slots, evict_slots, evict_di
     _check(lib().mts_cache_place_fetched(cache.handle, _ptr(fetched), _ptr(miss_slots), _ptr(evict_slots),
                                          _ptr(evict_dirty), list_capacity, _ptr(counters), _ptr(evict_staging),
                                          _stream(stream)))
+
+
+def cache_save_victims(cache: Cache, evict_slots, evict_dirty, list_capacity: int, counters, evict_staging,
+                       stream=None) -> None:
+    _check(lib().mts_cache_save_victims(cache.handle, _ptr(evict_slots), _ptr(evict_dirty), list_capacity,
+                                        _ptr(counters), _ptr(evict_staging), _stream(stream)))
 
 
 def cache_writeback_evicted(cache: Cache, host_rows_mapped, evict_keys, evict_dirty, list_capacity: int, counters,

@@ -1604,28 +1604,42 @@ extern "C" int mts_host_scatter_rows(void* host_rows, const int64_t* host_keys, 
   return MTS_OK;
 }
 
+extern "C" int mts_cache_save_victims(mts_cache* c, const int32_t* evict_slots, const uint8_t* evict_dirty,
+                                      int64_t list_capacity, const int64_t* counters, void* evict_staging,
+                                      void* stream) {
+  if (!c || !counters || list_capacity < 0 || (list_capacity > 0 && (!evict_slots || !evict_dirty || !evict_staging)))
+    return set_error(MTS_ERR_INVALID_ARG, "cache_save_victims: null argument");
+  if ((uintptr_t)evict_staging & 15)
+    return set_error(MTS_ERR_ALIGNMENT, "cache_save_victims: the staging buffer must be 16-byte aligned");
+  if (list_capacity == 0) return MTS_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  {
+    LaunchScope scope(K_CACHE_SAVE_VICTIMS, s);
+    cache_save_victims<<<c->sm_count * 8, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, evict_slots, evict_dirty, counters,
+                                                                 list_capacity, static_cast<char*>(evict_staging));
+  }
+  return check_launch("cache_save_victims");
+}
+
 extern "C" int mts_cache_place_fetched(mts_cache* c, const void* fetched, const int32_t* miss_slots,
                                        const int32_t* evict_slots, const uint8_t* evict_dirty, int64_t list_capacity,
                                        const int64_t* counters, void* evict_staging, void* stream) {
-  if (!c || !counters || list_capacity < 0 ||
-      (list_capacity > 0 && (!fetched || !miss_slots || !evict_slots || !evict_dirty || !evict_staging)))
+  if (!c || !counters || list_capacity < 0 || (list_capacity > 0 && (!fetched || !miss_slots)))
     return set_error(MTS_ERR_INVALID_ARG, "cache_place_fetched: null argument");
-  if (((uintptr_t)fetched | (uintptr_t)evict_staging) & 15)
+  if ((uintptr_t)fetched & 15)
     return set_error(MTS_ERR_ALIGNMENT, "cache_place_fetched: buffers must be 16-byte aligned");
   if (list_capacity == 0) return MTS_OK;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const int grid = c->sm_count * 8;
-  {
-    LaunchScope scope(K_CACHE_SAVE_VICTIMS, s);
-    cache_save_victims<<<grid, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, evict_slots, evict_dirty, counters,
-                                                      list_capacity, static_cast<char*>(evict_staging));
+  if (evict_staging != nullptr) {
+    const int rc = mts_cache_save_victims(c, evict_slots, evict_dirty, list_capacity, counters, evict_staging, stream);
+    if (rc != MTS_OK) return rc;
   }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
   {
     LaunchScope scope(K_CACHE_FETCH_MISSES, s);
-    cache_place_fetched<<<grid, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, static_cast<const char*>(fetched),
-                                                       miss_slots, counters, list_capacity);
+    cache_place_fetched<<<c->sm_count * 8, CACHE_THREADS, 0, s>>>(c->data, c->row_bytes, static_cast<const char*>(fetched),
+                                                                  miss_slots, counters, list_capacity);
   }
-  return check_launch("cache_save_victims / cache_place_fetched");
+  return check_launch("cache_place_fetched");
 }
 
 extern "C" int mts_cache_writeback_evicted(mts_cache* c, void* host_rows_mapped, const int64_t* evict_keys,

@@ -42,6 +42,9 @@ namespace mts {
 #ifndef MTS_BWD_LEAN_MINBLK2
 #define MTS_BWD_LEAN_MINBLK2 12 // the same for its two-piece form (rows of 129..256 columns)
 #endif
+#ifndef MTS_BWD_LEAN_RUN2
+#define MTS_BWD_LEAN_RUN2 2     // MTS_BWD_LEAN_RUN of the two-piece form
+#endif
 #ifndef MTS_BWD_GROUP2
 #define MTS_BWD_GROUP2 1        // the same for rows of 129..256 columns
 #endif
@@ -502,7 +505,7 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
     auto walk = [&](auto width) {
     constexpr int WIDTH = decltype(width)::value;
     constexpr int NP = WIDTH == 128 ? 1 : NVL;                     // pieces a lane loads per lookup
-    constexpr int RUN = NP == 1 ? LEAN_RUN : (LEAN_RUN > 1 ? LEAN_RUN / 2 : 1);
+    constexpr int RUN = NP == 1 ? LEAN_RUN : MTS_BWD_LEAN_RUN2;
     struct Pieces { GradPiece<GH> q[NP]; };
     auto add_scaled = [&](const Pieces& g, int jj) {
       if (MEAN) {

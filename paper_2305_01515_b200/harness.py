@@ -302,13 +302,34 @@ class DeviceModel:
         self.wb_dirty = [[torch.empty(r, dtype=torch.uint8).pin_memory() for r in self.fetch_rows]
                          for _ in range(self.N_CTX)]
 
-    def cache_fetch_via_host(self, g: int, n_miss: int, copy_stream, stream, ctx: int, mark=None) -> bool:
+    def host_lists_fit(self, g: int, n_miss: int, n_evict: int) -> bool:
+        """Whether the miss and evict lists of a batch fit the pinned buffers of the copy-engine path."""
+        return n_miss <= self.fetch_rows[g] and n_evict <= self.fetch_rows[g]
+
+    def cache_save_victims_via_host(self, g: int, n_evict: int, stream, ctx: int):
+        """Cache g, copy-engine path of the write-back: the dirty victims are saved to the staging buffer and
+        the first n_evict entries of the evict list (keys, dirty bytes) and of the staging buffer go to pinned
+        host buffers, all on `stream`.  A victim's row is final once its batch's tag step is over, so this
+        needs nothing of the batch's fetch.  Returns the event recorded after the saving kernel (the placing
+        kernel, which overwrites the victims' slots, has to wait for it)."""
+        L = self.ctx[ctx]["lists"][g]
+        mb.cache_save_victims(self.caches[g], L["evict_slots"], L["evict_dirty"], L["capacity"], L["counters"],
+                              L["staging"], stream)
+        saved = torch.cuda.Event()
+        saved.record(stream)
+        if n_evict > 0:
+            rb = self.caches[g].dim * (4 if self.spec.dtype == wl.FP32 else 2)
+            with torch.cuda.stream(stream):
+                self.wb_keys[ctx][g][:n_evict].copy_(L["evict_keys"][:n_evict], non_blocking=True)
+                self.wb_dirty[ctx][g][:n_evict].copy_(L["evict_dirty"][:n_evict], non_blocking=True)
+                self.wb_host[ctx][g][:n_evict * rb].copy_(L["staging"][:n_evict * rb], non_blocking=True)
+        return saved
+
+    def cache_fetch_via_host(self, g: int, n_miss: int, copy_stream, stream, ctx: int, saved, mark=None) -> None:
         """Cache g, copy-engine path: the first n_miss keys of the miss list come to the host on
         `copy_stream` (the caller made sure the tag step is over), host threads gather the rows, one
-        contiguous copy and the placing kernel follow on `stream`.  Blocks the calling thread for the key
-        copy and the gather.  Returns False (nothing done) when the list does not fit the buffers."""
-        if n_miss > self.fetch_rows[g]:
-            return False
+        contiguous copy and the placing kernel (after the event `saved` of cache_save_victims_via_host) follow
+        on `stream`.  Blocks the calling thread for the key copy and the gather, not for the copy of the rows."""
         L = self.ctx[ctx]["lists"][g]
         c = self.caches[g]
         esz = 4 if self.spec.dtype == wl.FP32 else 2
@@ -327,24 +348,8 @@ class DeviceModel:
                 self.fetch_dev[g][:n_miss * rb].copy_(rows_h[:n_miss * rb], non_blocking=True)
                 if mark is not None:
                     mark(f"copy{g}_end")
-        mb.cache_place_fetched(c, self.fetch_dev[g], L["miss_slots"], L["evict_slots"], L["evict_dirty"],
-                               L["capacity"], L["counters"], L["staging"], stream)
-        return True
-
-    def cache_writeback_via_host_begin(self, g: int, n_evict: int, stream, ctx: int) -> bool:
-        """Cache g, copy-engine path of the write-back: the first n_evict entries of the evict list (keys, dirty
-        bytes) and of the staging buffer go to pinned host buffers on `stream` (after the placing kernel of the
-        same batch).  Returns False (nothing done) when they do not fit."""
-        if n_evict > self.fetch_rows[g]:
-            return False
-        if n_evict > 0:
-            L = self.ctx[ctx]["lists"][g]
-            rb = self.caches[g].dim * (4 if self.spec.dtype == wl.FP32 else 2)
-            with torch.cuda.stream(stream):
-                self.wb_keys[ctx][g][:n_evict].copy_(L["evict_keys"][:n_evict], non_blocking=True)
-                self.wb_dirty[ctx][g][:n_evict].copy_(L["evict_dirty"][:n_evict], non_blocking=True)
-                self.wb_host[ctx][g][:n_evict * rb].copy_(L["staging"][:n_evict * rb], non_blocking=True)
-        return True
+        stream.wait_event(saved)
+        mb.cache_place_fetched(c, self.fetch_dev[g], L["miss_slots"], None, None, L["capacity"], L["counters"], None, stream)
 
     def cache_writeback_via_host_finish(self, g: int, n_evict: int, ctx: int) -> None:
         """Host threads put the dirty victims into their rows of the host tier (after the copies of

@@ -4,6 +4,7 @@ lookups).  Streams, ordered by events only:
 
     main    : forward(t), backward(t), tag lookup and replacement for batch t + lock_depth + 1
     move[g] : cache g: save victims / fetch missed rows / write victims back for the batches ahead  (host link)
+    save[g] : cache g, copy-engine path: victims saved and copied to the host beside the fetch on move[g]
     fix     : repair of rows that overflowed in batches t and t-1 and were placed by batch t+1
 
 so the host-link traffic of the batches ahead overlaps the training of the current batch; the launching
@@ -38,7 +39,10 @@ whose overflow list the repair before batch t-4 was the last to read, so it also
 
 With host_gather the missed rows do not cross the host link at the request of SMs (small reads that
 slow every kernel beside them): one worker thread per cache reads the miss list, gathers the rows with
-the host's threads into a pinned buffer and enqueues one contiguous copy and the placing kernel; one more
+the host's threads into a pinned buffer and enqueues one contiguous copy and the placing kernel, without
+waiting for them: while they run it already handles the next batch.  The victims of a batch are final when
+its tag step ends, so they are saved and copied out on save[g] at once (the placing kernel waits for the
+save); the worker puts them into their host rows before its next gather, which may read one of them.  One more
 thread enqueues the repair once all caches of a batch have moved.  The workers run ahead of the launching
 thread; host-side flags tell each side which events the other has recorded.
 """
@@ -80,6 +84,8 @@ class CachedTrainer:
         self.moves = [torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main for _ in range(n_c)]
         self.fix = torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main
         self.copies = [torch.cuda.Stream(self.dev, priority=-1) for _ in range(n_c)]    # miss keys to the host (host_gather)
+        # victims to the host (host_gather), beside the cache's fetch
+        self.saves = [torch.cuda.Stream(self.dev, priority=-1) if pipelined else self.main for _ in range(n_c)]
         self.history: List[np.ndarray] = []           # per batch [n_caches, NUM_COUNTERS], filled when run() returns
         self.record_timeline = False                  # set to True to time every phase with events
         self._marks = []
@@ -128,43 +134,48 @@ class CachedTrainer:
         self.ev_tags[t].record(s)
 
     def _move_cache(self, t, g, via_host):
-        """Data path of batch t for cache g on its move stream: fetch, then write back, in stream order (the
-        next batch's fetch of this cache, which may miss a row written back now, follows on the same stream)."""
+        """Data path of batch t for cache g.  Kernel path: fetch, then write back, on the cache's move stream
+        (the next batch's fetch of this cache, which may miss a row written back now, follows on the same
+        stream).  Copy-engine path: the victims are saved and copied out on the cache's second stream as soon
+        as the tag step is over, while this thread puts the previous batch's victims into their host rows and
+        gathers the missed rows; the copy of the gathered rows and the placing kernel are only enqueued, so
+        the thread goes on to the next batch while they run."""
         s, ctx = self.moves[g], t % DeviceModel.N_CTX
         s.wait_event(self.ev_tags[t])
         self._delay(s)
         self._mark(f"move{g}_begin", t, s)
         done = False
         if via_host:
-            # the host reads the rows itself: the tag step of this batch is over (its counters are on the
-            # host) and this cache's write-backs of earlier batches have reached host memory
+            # the host reads the rows itself: the tag step of this batch is over (its counters are on the host)
             self.ev_tags[t].synchronize()
-            self._finish_writeback(g)
-            if t > 0:
-                self.ev_moved[t - 1][g].synchronize()
             n_miss = int(self._host_counters[t, g, mb.COUNTER_NAMES.index("inserted")])
-            done = self.m.cache_fetch_via_host(
-                g, n_miss, self.copies[g], s, ctx,
-                mark=(lambda name, s=s: self._mark(name, t, s)) if self.record_timeline else None)
-        if not done:
-            self.m.cache_fetch(g, stream=s, ctx=ctx)
-        self._mark(f"placed{g}", t, s)
-        wb = False
-        if via_host:
-            # the victims take the copy engine as well; host threads put them into their rows before this
-            # cache's next gather (or at the end of the run)
             n_evict = int(self._host_counters[t, g, mb.COUNTER_NAMES.index("evicted")])
-            wb = self.m.cache_writeback_via_host_begin(g, n_evict, s, ctx)
-            if wb:
-                e = torch.cuda.Event()
-                e.record(s)
-                self._pending_wb[g] = (e, n_evict, ctx)
+            if self.m.host_lists_fit(g, n_miss, n_evict):
+                w = self.saves[g]
+                w.wait_event(self.ev_tags[t])
+                self._delay(w)
+                saved = self.m.cache_save_victims_via_host(g, n_evict, w, ctx)
+                copied = torch.cuda.Event()
+                copied.record(w)
+                # this cache's write-backs of earlier batches reach host memory before the gather reads it
+                self._finish_writeback(g)
+                self._pending_wb[g] = (copied, n_evict, ctx)
+                self.m.cache_fetch_via_host(
+                    g, n_miss, self.copies[g], s, ctx, saved,
+                    mark=(lambda name, s=s: self._mark(name, t, s)) if self.record_timeline else None)
                 if not self.pipelined:
                     self._finish_writeback(g)
-        if not wb:
+                done = True
+        if not done:
+            if via_host:
+                self._finish_writeback(g)
+            self.m.cache_fetch(g, stream=s, ctx=ctx)
             self.m.cache_writeback(g, stream=s, ctx=ctx)
+        self._mark(f"placed{g}", t, s)
         self._mark(f"move{g}_end", t, s)
         self.ev_moved[t][g].record(s)
+        if via_host and not done:
+            self.ev_moved[t][g].synchronize()       # the kernels' write-back is in host memory before the next gather
 
     def _finish_writeback(self, g):
         """Cache g: the victims whose copy to the host was enqueued by an earlier batch go into their rows."""
@@ -291,7 +302,7 @@ class CachedTrainer:
         # the side streams must see the inputs produced on the main stream
         start = torch.cuda.Event()
         start.record(self.main)
-        for s in [self.tag, self.fix] + self.copies + self.moves:
+        for s in [self.tag, self.fix] + self.copies + self.moves + self.saves:
             s.wait_event(start)
         if self.host_gather:
             self._jobs = [queue.Queue() for _ in range(n_c)]
@@ -356,7 +367,7 @@ class CachedTrainer:
                 self._threads = []
                 if self._worker_error is not None:
                     raise self._worker_error
-        for s in [self.tag, self.fix] + self.copies + self.moves:
+        for s in [self.tag, self.fix] + self.copies + self.moves + self.saves:
             self.main.wait_stream(s)
         torch.cuda.synchronize(self.dev)
         self.history.extend(self._host_counters.numpy().copy())
