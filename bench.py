@@ -672,6 +672,16 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
     }
     if gather_gbs is not None:
         rec["host_link"]["host_gather_gbs_by_dim"] = gather_gbs
+        # what the host threads did over the whole run (warm-up and cooldown batches included), per batch:
+        # the caches take turns at the cores, so the sum of the two times is a floor of the step time
+        st = model.host_copy_stats
+        nb = float(K + COOLDOWN)
+        g_s, s_s = sum(x["gather_s"] for x in st), sum(x["scatter_s"] for x in st)
+        g_b, s_b = sum(x["gather_bytes"] for x in st), sum(x["scatter_bytes"] for x in st)
+        rec["host_threads"] = {"threads": model.gather_threads, "gather_ms_per_batch": g_s * 1e3 / nb,
+                               "scatter_ms_per_batch": s_s * 1e3 / nb,
+                               "gather_gbs": g_b / max(g_s, 1e-9) / 1e9, "scatter_gbs": s_b / max(s_s, 1e-9) / 1e9,
+                               "wait_for_turn_ms_per_batch": sum(x["wait_s"] for x in st) * 1e3 / nb}
     if args.timeline:
         # device time of every phase of the last batches, ms since the first mark (perturbs the run a little)
         by_batch = {}

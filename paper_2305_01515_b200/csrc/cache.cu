@@ -14,6 +14,11 @@
 #include <algorithm>
 #include <cstring>
 #include <thread>
+#include <atomic>
+#include <condition_variable>
+#include <functional>
+#include <mutex>
+#include <vector>
 #if defined(__SSE2__)
 #include <emmintrin.h>
 #endif
@@ -1552,6 +1557,88 @@ static inline void host_copy_fence() {
 #endif
 }
 
+// Host threads for the row copies, kept between calls (a gather of a few hundred thousand rows takes about a
+// millisecond: starting sixteen threads for it would cost a good part of that).  One job at a time; the
+// pieces of a job are handed out through a counter, so a thread that is held up costs one piece, not its share.
+namespace {
+class HostPool {
+ public:
+  static HostPool& get() { static HostPool p; return p; }
+  // fn(k0, k1) over [0, n) in pieces of `grain`, on up to `threads` threads (the caller is one of them)
+  template <class F>
+  void run(int64_t n, int64_t grain, int threads, const F& fn) {
+    const int64_t pieces = (n + grain - 1) / grain;
+    const int helpers = (int)std::max<int64_t>(0, std::min<int64_t>(threads - 1, pieces - 1));
+    if (helpers == 0) { fn(0, n); return; }
+    std::lock_guard<std::mutex> job(job_mu_);
+    auto body = [&](void) {
+      for (;;) {
+        const int64_t k0 = next_.fetch_add(grain, std::memory_order_relaxed);
+        if (k0 >= n) break;
+        fn(k0, std::min(n, k0 + grain));
+      }
+    };
+    std::function<void(void)> erased = body;
+    {
+      std::unique_lock<std::mutex> lk(mu_);
+      while ((int)workers_.size() < helpers) {
+        const int id = (int)workers_.size();
+        workers_.emplace_back([this, id] { worker(id); });
+      }
+      next_.store(0, std::memory_order_relaxed);
+      body_ = &erased;
+      helpers_ = helpers;
+      pending_ = helpers;
+      ++epoch_;
+    }
+    cv_work_.notify_all();
+    body();
+    std::unique_lock<std::mutex> lk(mu_);
+    cv_done_.wait(lk, [this] { return pending_ == 0; });
+    body_ = nullptr;
+  }
+  ~HostPool() {
+    {
+      std::lock_guard<std::mutex> lk(mu_);
+      stop_ = true;
+    }
+    cv_work_.notify_all();
+    for (auto& t : workers_) t.join();
+  }
+
+ private:
+  void worker(int id) {
+    uint64_t seen = 0;
+    for (;;) {
+      const std::function<void(void)>* body = nullptr;
+      {
+        std::unique_lock<std::mutex> lk(mu_);
+        cv_work_.wait(lk, [&] { return stop_ || epoch_ != seen; });
+        if (stop_) return;
+        seen = epoch_;
+        if (id >= helpers_) continue;          // this job uses fewer threads
+        body = body_;
+      }
+      (*body)();
+      {
+        std::lock_guard<std::mutex> lk(mu_);
+        --pending_;
+      }
+      cv_done_.notify_one();
+    }
+  }
+  std::mutex job_mu_, mu_;
+  std::condition_variable cv_work_, cv_done_;
+  std::vector<std::thread> workers_;
+  const std::function<void(void)>* body_ = nullptr;
+  std::atomic<int64_t> next_{0};
+  int helpers_ = 0, pending_ = 0;
+  uint64_t epoch_ = 0;
+  bool stop_ = false;
+};
+constexpr int64_t HOST_COPY_GRAIN = 512;      // rows per piece
+}  // namespace
+
 extern "C" int mts_host_gather_rows(const void* host_rows, const int64_t* host_keys, int64_t n, int64_t row_bytes,
                                     void* host_out, int32_t threads) {
   if (n < 0 || row_bytes < 1 || (n > 0 && (!host_rows || !host_keys || !host_out)))
@@ -1563,7 +1650,7 @@ extern "C" int mts_host_gather_rows(const void* host_rows, const int64_t* host_k
   auto work = [=](int64_t k0, int64_t k1) {
     constexpr int64_t AHEAD = 16;        // rows requested ahead of the copy: the reads are random DRAM accesses
     for (int64_t k = k0; k < k1; ++k) {
-      if (k + AHEAD < k1) {
+      if (k + AHEAD < n) {
         const char* ahead = src + (size_t)host_keys[k + AHEAD] * rb;
         for (size_t b = 0; b < rb; b += 64) __builtin_prefetch(ahead + b, 0, 0);
       }
@@ -1571,13 +1658,7 @@ extern "C" int mts_host_gather_rows(const void* host_rows, const int64_t* host_k
     }
     host_copy_fence();
   };
-  const int64_t nt = std::max<int64_t>(1, std::min<int64_t>(threads, (n + 1023) / 1024));
-  if (nt == 1) { work(0, n); return MTS_OK; }
-  std::vector<std::thread> pool;
-  const int64_t per = (n + nt - 1) / nt;
-  for (int64_t i = 1; i < nt; ++i) pool.emplace_back(work, std::min(n, i * per), std::min(n, (i + 1) * per));
-  work(0, std::min(n, per));
-  for (auto& t : pool) t.join();
+  HostPool::get().run(n, HOST_COPY_GRAIN, threads, work);
   return MTS_OK;
 }
 
@@ -1594,13 +1675,7 @@ extern "C" int mts_host_scatter_rows(void* host_rows, const int64_t* host_keys, 
       if (host_mask == nullptr || host_mask[k]) host_copy_row_streaming(dst + (size_t)host_keys[k] * rb, src + (size_t)k * rb, rb);
     host_copy_fence();
   };
-  const int64_t nt = std::max<int64_t>(1, std::min<int64_t>(threads, (n + 1023) / 1024));
-  if (nt == 1) { work(0, n); return MTS_OK; }
-  std::vector<std::thread> pool;
-  const int64_t per = (n + nt - 1) / nt;
-  for (int64_t i = 1; i < nt; ++i) pool.emplace_back(work, std::min(n, i * per), std::min(n, (i + 1) * per));
-  work(0, std::min(n, per));
-  for (auto& t : pool) t.join();
+  HostPool::get().run(n, HOST_COPY_GRAIN, threads, work);
   return MTS_OK;
 }
 

@@ -6,6 +6,7 @@ from __future__ import annotations
 
 import os
 import threading
+import time
 from typing import List, Optional, Sequence
 
 import numpy as np
@@ -286,6 +287,9 @@ class DeviceModel:
         # with many wide rows is not left with a third of the cores while the others idle
         self.gather_threads = threads or os.cpu_count() or 1
         self.host_copy_lock = threading.Lock()
+        # seconds and bytes the host threads spent on gathers / scatters (and waiting for their turn), per cache
+        self.host_copy_stats = [{"gather_s": 0.0, "gather_bytes": 0, "scatter_s": 0.0, "scatter_bytes": 0, "wait_s": 0.0}
+                                for _ in self.caches]
         self.fetch_rows = [max(1, min(self.ctx[0]["lists"][g]["capacity"], self.FETCH_STAGE_BYTES // (c.dim * esz)))
                            for g, c in enumerate(self.caches)]
         self.fetch_dev = [torch.empty(r * c.dim * esz, dtype=torch.uint8, device=self.device)
@@ -340,8 +344,14 @@ class DeviceModel:
                 keys_h[:n_miss].copy_(L["miss_keys"][:n_miss], non_blocking=True)
             copy_stream.synchronize()
             rows_h = self.fetch_host[ctx][g]
+            t0 = time.perf_counter()
             with self.host_copy_lock:
+                t1 = time.perf_counter()
                 mb.host_gather_rows(self.host_rows_ptr(g), keys_h.numpy(), n_miss, rb, rows_h, self.gather_threads)
+                st = self.host_copy_stats[g]
+                st["gather_s"] += time.perf_counter() - t1
+                st["gather_bytes"] += n_miss * rb
+                st["wait_s"] += t1 - t0
             with torch.cuda.stream(stream):
                 if mark is not None:
                     mark(f"copy{g}_begin")
@@ -356,9 +366,15 @@ class DeviceModel:
         cache_writeback_via_host_begin have completed)."""
         if n_evict > 0:
             rb = self.caches[g].dim * (4 if self.spec.dtype == wl.FP32 else 2)
+            t0 = time.perf_counter()
             with self.host_copy_lock:
+                t1 = time.perf_counter()
                 mb.host_scatter_rows(self.host_rows_ptr(g), self.wb_keys[ctx][g].numpy(), self.wb_dirty[ctx][g].numpy(),
                                      n_evict, rb, self.wb_host[ctx][g], self.gather_threads)
+                st = self.host_copy_stats[g]
+                st["scatter_s"] += time.perf_counter() - t1
+                st["scatter_bytes"] += n_evict * rb
+                st["wait_s"] += t1 - t0
 
     def cache_writeback(self, g: int, stream=None, ctx: Optional[int] = None) -> None:
         """Cache g: the staged dirty victims back to the host tier (after cache_fetch of the same batch)."""
