@@ -86,15 +86,15 @@ def kernel_source_hash(files) -> str:
 
 
 def ncu_traffic_per_lookup(kernel: str, workload: str):
-    """DRAM bytes (read + write) per lookup of `kernel` from the profiler capture recorded in
-    profiles/ncu_dram_traffic.json, or None when there is no capture for this workload or the kernel sources
-    have changed since it was taken (the record carries their hash)."""
+    """DRAM bytes (read + write) per lookup of `kernel` on `workload` from the profiler captures recorded in
+    profiles/ncu_dram_traffic.json ({kernel: {workload: record}}), or None when there is no capture for this
+    workload or the kernel sources have changed since it was taken (the record carries their hash)."""
     try:
         with open(TRAFFIC_FILE) as f:
-            rec = json.load(f).get(kernel)
+            rec = json.load(f).get(kernel, {}).get(workload)
     except (OSError, ValueError):
         return None, "no capture file"
-    if not rec or rec.get("workload") != workload:
+    if not rec:
         return None, "no capture of this kernel on this workload"
     if rec.get("source_sha256") != kernel_source_hash(rec.get("source_files", [])):
         return None, "kernel sources changed since the capture"
@@ -687,6 +687,7 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
         by_batch = {}
         for name, t, ms_at in trainer.timeline():
             by_batch.setdefault(t, {})[name] = round(ms_at, 2)
+        rec["worker_phases_ms"] = trainer.host_phases()
         rec["timeline_ms"] = {str(t): dict(sorted(by_batch[t].items(), key=lambda kv: kv[1]))
                               for t in sorted(by_batch) if K - 4 <= t < K}
     if two_level:

@@ -806,13 +806,11 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
   } while (0)
   if constexpr (NV <= 2 && MTS_BWD_USE_LEAN) {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
-    // as many blocks as fit on the device at once (or fewer); the warps share out the chunks
-    // With cached tables the step shares the GPU with the cache's tag lookup and data movement on other
-    // streams: blocks that stay until the last chunk would keep every warp slot for the whole kernel and
-    // hold those streams back, so there the grid covers the chunks and a block leaves after one round.
+    // as many blocks as fit on the device at once (or fewer); the warps share out the chunks.  (With cached
+    // tables too: the cache's tag step runs between the training steps on the same stream, and the few blocks
+    // of its data movement on the other streams can wait for a kernel of a millisecond or two.)
     auto lean_grid = [&](int resident) {
-      return h->any_cached ? (unsigned)ceil_div(chunks, LEAN_WARPS)
-                           : (unsigned)std::min<int64_t>(ceil_div(chunks, LEAN_WARPS), (int64_t)h->sm_count * resident);
+      return (unsigned)std::min<int64_t>(ceil_div(chunks, LEAN_WARPS), (int64_t)h->sm_count * resident);
     };
     // NVL pieces per lane over the chunks of class `klass`
     auto launch_lean = [&](auto nvl, int klass) -> bool {
@@ -847,7 +845,7 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
   } else {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
     constexpr int resident = NV == 1 ? MTS_BWD_MINBLK : NV == 2 ? MTS_BWD_MINBLK2 : 2;
-    const unsigned dyn_grid = h->any_cached ? grid : (unsigned)std::min<int64_t>(grid, (int64_t)h->sm_count * resident);
+    const unsigned dyn_grid = (unsigned)std::min<int64_t>(grid, (int64_t)h->sm_count * resident);
     if (cudaMemsetAsync(next_chunk, 0, sizeof(uint32_t), s) != cudaSuccess) return check_launch("memset(next_chunk)");
     if (pooling_mode == MTS_POOL_MEAN)
       MTS_LAUNCH_GH(reduce_chunks, FP16 COMMA NV COMMA GROUP COMMA true, dyn_grid, BWD_WARPS * 32);

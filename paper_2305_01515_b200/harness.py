@@ -329,9 +329,16 @@ class DeviceModel:
                 self.wb_host[ctx][g][:n_evict * rb].copy_(L["staging"][:n_evict * rb], non_blocking=True)
         return saved
 
+    def cache_request_miss_keys(self, g: int, n_miss: int, copy_stream, ctx: int) -> None:
+        """Cache g, copy-engine path: the first n_miss keys of the miss list start their way to the host on
+        `copy_stream` (the caller made sure the tag step is over).  Called before the victims' copies are
+        enqueued: the same copy engine serves both, and the gather waits for the keys only."""
+        if n_miss > 0:
+            with torch.cuda.stream(copy_stream):
+                self.fetch_keys[ctx][g][:n_miss].copy_(self.ctx[ctx]["lists"][g]["miss_keys"][:n_miss], non_blocking=True)
+
     def cache_fetch_via_host(self, g: int, n_miss: int, copy_stream, stream, ctx: int, saved, mark=None) -> None:
-        """Cache g, copy-engine path: the first n_miss keys of the miss list come to the host on
-        `copy_stream` (the caller made sure the tag step is over), host threads gather the rows, one
+        """Cache g, copy-engine path, after cache_request_miss_keys: host threads gather the rows, one
         contiguous copy and the placing kernel (after the event `saved` of cache_save_victims_via_host) follow
         on `stream`.  Blocks the calling thread for the key copy and the gather, not for the copy of the rows."""
         L = self.ctx[ctx]["lists"][g]
@@ -340,8 +347,6 @@ class DeviceModel:
         rb = c.dim * esz
         if n_miss > 0:
             keys_h = self.fetch_keys[ctx][g]
-            with torch.cuda.stream(copy_stream):
-                keys_h[:n_miss].copy_(L["miss_keys"][:n_miss], non_blocking=True)
             copy_stream.synchronize()
             rows_h = self.fetch_host[ctx][g]
             t0 = time.perf_counter()

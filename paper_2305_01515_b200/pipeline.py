@@ -50,6 +50,7 @@ from __future__ import annotations
 
 import queue
 import threading
+import time
 from typing import Callable, List, Optional
 
 import numpy as np
@@ -89,6 +90,7 @@ class CachedTrainer:
         self.history: List[np.ndarray] = []           # per batch [n_caches, NUM_COUNTERS], filled when run() returns
         self.record_timeline = False                  # set to True to time every phase with events
         self._marks = []
+        self._host_marks = []
         self._mark_lock = threading.Lock()
         self.debug_delay_cycles = 0                   # > 0: the move and repair streams idle that long before their work
 
@@ -104,6 +106,24 @@ class CachedTrainer:
             e.record(stream)
             with self._mark_lock:
                 self._marks.append((name, t, e))
+
+    def _host_mark(self, name, t, g):
+        if self.record_timeline:
+            with self._mark_lock:
+                self._host_marks.append((name, t, g, time.perf_counter()))
+
+    def host_phases(self):
+        """{phase: mean ms} a cache's worker thread spent between consecutive host marks (record_timeline = True)."""
+        by = {}
+        for name, t, g, at in self._host_marks:
+            by.setdefault((t, g), []).append((at, name))
+        tot, cnt = {}, {}
+        for marks in by.values():
+            marks.sort()
+            for (a0, _), (a1, n1) in zip(marks, marks[1:]):
+                tot[n1] = tot.get(n1, 0.0) + (a1 - a0) * 1e3
+                cnt[n1] = cnt.get(n1, 0) + 1
+        return {n: tot[n] / cnt[n] for n in tot}
 
     def timeline(self):
         """[(phase, batch, ms since the first mark)] after a run with record_timeline = True."""
@@ -147,22 +167,28 @@ class CachedTrainer:
         done = False
         if via_host:
             # the host reads the rows itself: the tag step of this batch is over (its counters are on the host)
+            self._host_mark("job_begin", t, g)
             self.ev_tags[t].synchronize()
+            self._host_mark("tag_waited", t, g)
             n_miss = int(self._host_counters[t, g, mb.COUNTER_NAMES.index("inserted")])
             n_evict = int(self._host_counters[t, g, mb.COUNTER_NAMES.index("evicted")])
             if self.m.host_lists_fit(g, n_miss, n_evict):
+                self.m.cache_request_miss_keys(g, n_miss, self.copies[g], ctx)      # ahead of the victims' copies
                 w = self.saves[g]
                 w.wait_event(self.ev_tags[t])
                 self._delay(w)
                 saved = self.m.cache_save_victims_via_host(g, n_evict, w, ctx)
                 copied = torch.cuda.Event()
                 copied.record(w)
+                self._host_mark("victims_enqueued", t, g)
                 # this cache's write-backs of earlier batches reach host memory before the gather reads it
                 self._finish_writeback(g)
+                self._host_mark("scattered", t, g)
                 self._pending_wb[g] = (copied, n_evict, ctx)
                 self.m.cache_fetch_via_host(
                     g, n_miss, self.copies[g], s, ctx, saved,
                     mark=(lambda name, s=s: self._mark(name, t, s)) if self.record_timeline else None)
+                self._host_mark("gathered_enqueued", t, g)
                 if not self.pipelined:
                     self._finish_writeback(g)
                 done = True
@@ -174,6 +200,8 @@ class CachedTrainer:
         self._mark(f"placed{g}", t, s)
         self._mark(f"move{g}_end", t, s)
         self.ev_moved[t][g].record(s)
+        if via_host:
+            self._host_mark("job_end", t, g)
         if via_host and not done:
             self.ev_moved[t][g].synchronize()       # the kernels' write-back is in host memory before the next gather
 

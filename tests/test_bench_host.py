@@ -51,15 +51,15 @@ def test_profiler_traffic_record_is_dropped_when_the_kernel_source_changes(tmp_p
     import bench
 
     files = ["tbe_backward.cu", "common.cuh"]
-    rec = {"reduce_chunks": {"workload": "cfg2", "dram_bytes_per_lookup": 168.5, "source_files": files,
-                             "source_sha256": bench.kernel_source_hash(files), "capture": "test"}}
+    rec = {"reduce_chunks": {"cfg2": {"dram_bytes_per_lookup": 168.5, "source_files": files,
+                                      "source_sha256": bench.kernel_source_hash(files), "capture": "test"}}}
     path = tmp_path / "traffic.json"
     path.write_text(json.dumps(rec))
     monkeypatch.setattr(bench, "TRAFFIC_FILE", str(path))
     assert bench.ncu_traffic_per_lookup("reduce_chunks", "cfg2")[0] == 168.5
     assert bench.ncu_traffic_per_lookup("reduce_chunks", "cfg3")[0] is None          # another workload
     assert bench.ncu_traffic_per_lookup("tbe_forward_kernel", "cfg2")[0] is None     # no record
-    rec["reduce_chunks"]["source_sha256"] = "0" * 64                                 # the kernel changed since
+    rec["reduce_chunks"]["cfg2"]["source_sha256"] = "0" * 64                                 # the kernel changed since
     path.write_text(json.dumps(rec))
     assert bench.ncu_traffic_per_lookup("reduce_chunks", "cfg2")[0] is None
 
