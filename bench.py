@@ -575,7 +575,7 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
     glist = [grads[k % R] for k in range(K + COOLDOWN)]
     setup_s = time.time() - t_setup
     trainer = CachedTrainer(model, pipelined=not args.sequential, host_gather=args.fetch == "host",
-                            tag_on_main=not args.tag_stream)
+                            tag_on_main=args.tag_on_main)
     trainer.record_timeline = args.timeline
     gather_gbs = host_gather_rates(model) if args.fetch == "host" else None
     main = torch.cuda.current_stream(dev)
@@ -787,9 +787,9 @@ def main():
                     help="cached workloads: batches a stamped way stays unevictable (Section 5.7 invariant)")
     ap.add_argument("--timeline", action="store_true",
                     help="cached workloads: add the device timeline of the last batches (events on every stream) to the line")
-    ap.add_argument("--tag-stream", action="store_true",
-                    help="cached workloads: the tag step on a stream of its own, two batches ahead, instead of between the "
-                         "training steps")
+    ap.add_argument("--tag-on-main", action="store_true",
+                    help="cached workloads: the tag step between the training steps on their stream, instead of two "
+                         "batches ahead on a stream of its own")
     ap.add_argument("--trace", action="store_true",
                     help="cached workloads: CUDA events around every launch of the run (perturbs the timing)")
     ap.add_argument("--tables", type=int, default=0,

@@ -807,8 +807,8 @@ static int launch_backward(const mts_tables* h, int32_t B, const uint32_t* keys,
   if constexpr (NV <= 2 && MTS_BWD_USE_LEAN) {
     LaunchScope scope(K_REDUCE_CHUNKS, s);
     // as many blocks as fit on the device at once (or fewer); the warps share out the chunks.  (With cached
-    // tables too: the cache's tag step runs between the training steps on the same stream, and the few blocks
-    // of its data movement on the other streams can wait for a kernel of a millisecond or two.)
+    // tables too: a grid that covers all chunks, so that blocks retire and the kernels of the cache's other
+    // streams get warp slots during this kernel, measured slower for the step as a whole.)
     auto lean_grid = [&](int resident) {
       return (unsigned)std::min<int64_t>(ceil_div(chunks, LEAN_WARPS), (int64_t)h->sm_count * resident);
     };
