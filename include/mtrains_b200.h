@@ -148,6 +148,9 @@ int mts_tables_status(mts_tables* tables, int32_t* host_status, void* stream);
  * twice.
  * slot_of_lookup (int32 [N], may be NULL when no table is cached): for a lookup of a cached
  * table, the cache slot holding its row, or -1 = read the row from the host tier directly.
+ * A lookup that has a slot may be served without its index being read (the slot names the row);
+ * the index-range check of mts_tables_status then covers the lookups of HBM tables and those without
+ * a slot, and the cache's lookup reports keys outside its key space (mts_cache_status).
  * host_cache_data: host array [n_caches] of device pointers to each cache's row storage.
  * Errors: INVALID_ARG, ALIGNMENT, CUDA (launch failure). */
 int mts_tbe_forward(const mts_tables* tables, int32_t B, const int64_t* indices,

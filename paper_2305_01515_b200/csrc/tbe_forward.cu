@@ -252,11 +252,14 @@ static int launch_forward(const mts_tables* h, int32_t B, const int64_t* indices
   return check_launch("tbe_forward_kernel");
 }
 
-// ---- tbe_forward_lean: the same walk when no table sits behind a cache and a row is at most 32
-// 16-byte pieces.  The walk is bound by latency and instruction issue, not by bytes in flight, so this
-// form trades loads in flight per warp for resident warps: positions and row numbers are 32-bit, there
-// is no cache-slot path, and the register allocation is bounded for MTS_FWD_LEAN_MINBLK blocks per SM.
-// Same summation order and arithmetic as tbe_forward_kernel (bit-identical results).
+// ---- tbe_forward_lean: the same walk when a row is at most 32 16-byte pieces.  The walk is bound by latency
+// and instruction issue, not by bytes in flight, so this form trades loads in flight per warp for resident
+// warps: positions and row numbers are 32-bit and the register allocation is bounded for MTS_FWD_LEAN_MINBLK
+// blocks per SM.  Same summation order and arithmetic as tbe_forward_kernel (bit-identical results).
+// CACHED: tables may sit behind a cache.  A lookup of such a table reads its cache slot instead of its index
+// (the row is cache_data[slot]); only a lookup without a slot (slot < 0: the row is read from the host tier)
+// reads the index too, and a batch of 32 lookups that has one takes a slower form of the inner loop.  An
+// out-of-range index of a cached table is reported by the cache's lookup, not here.
 #ifndef MTS_FWD_LEAN
 #define MTS_FWD_LEAN 1
 #endif
@@ -268,12 +271,13 @@ static int launch_forward(const mts_tables* h, int32_t B, const int64_t* indices
 #endif
 constexpr int LEAN_UNROLL = MTS_FWD_LEAN_UNROLL;
 
-template <bool FP16>
+template <bool FP16, bool CACHED>
 __global__ void __launch_bounds__(FWD_WARPS * 32, MTS_FWD_LEAN_MINBLK)
 tbe_forward_lean(const TableMeta* __restrict__ meta, int32_t n_bags, int32_t B,
                  const int64_t* __restrict__ indices, const int64_t* __restrict__ offsets,
-                 const char* __restrict__ dev_w, int32_t pooling_mode, void* __restrict__ out, int out_kind,
-                 int64_t out_stride, int32_t* status) {
+                 const int32_t* __restrict__ slot_of_lookup, const __grid_constant__ CachePtrs caches,
+                 const char* __restrict__ dev_w, const char* __restrict__ host_w, int32_t pooling_mode,
+                 void* __restrict__ out, int out_kind, int64_t out_stride, int32_t* status) {
   constexpr int EPC = FP16 ? 8 : 4;       // elements per 16-byte chunk
   constexpr int EB = FP16 ? 2 : 4;
   const int lane = threadIdx.x & 31;
@@ -285,17 +289,22 @@ tbe_forward_lean(const TableMeta* __restrict__ meta, int32_t n_bags, int32_t B,
   uint32_t i1 = __shfl_sync(0xffffffffu, my_off, 0);
   int32_t t = (int32_t)((uint32_t)bag0 / (uint32_t)B);
   int32_t b = bag0 - t * B;
-  // first indices of the first bag
-  int64_t pf_idx = 0;
+  // what a lookup's row is found by: its cache slot (cached table) or its index
+  auto reference = [&](uint32_t i, bool cached) -> int64_t {
+    return (CACHED && cached) ? (int64_t)slot_of_lookup[i] : indices[i];
+  };
+  // first references of the first bag
+  int64_t pf_ref = 0;
   {
     const uint32_t e = __shfl_sync(0xffffffffu, my_off, 1);
-    if (i1 + lane < e) pf_idx = indices[i1 + lane];
+    if (i1 + lane < e) pf_ref = reference(i1 + lane, CACHED && meta[t].cache_id >= 0);
   }
   // per-table values, refreshed only when the walk crosses into the next table
   int32_t t_cur = -1;
   int vec16 = 0, logG = 0, row_bytes = 0, out_offset = 0;
   uint32_t rows = 0;
-  const char* lane_base = nullptr;        // the lane's 16-byte piece of row 0
+  bool cached = false;
+  const char* lane_base = nullptr;        // the lane's 16-byte piece of row 0 (of the table, or of the cache's slot 0)
   for (int k = 0; k < nb; ++k, ++b) {
     if (b == B) { b = 0; ++t; }
     if (t != t_cur) {
@@ -307,17 +316,23 @@ tbe_forward_lean(const TableMeta* __restrict__ meta, int32_t n_bags, int32_t B,
       row_bytes = m.dim * EB;
       rows = (uint32_t)m.rows;
       out_offset = m.out_offset;
-      lane_base = dev_w + m.weight_offset * EB + (lane & ((1 << logG) - 1)) * 16;
+      cached = CACHED && m.cache_id >= 0;
+      lane_base = (cached ? static_cast<const char*>(caches.data[m.cache_id]) : dev_w + m.weight_offset * EB) +
+                  (lane & ((1 << logG) - 1)) * 16;
     }
     const int R = 32 >> logG;               // rows per load instruction
     const int sub = lane >> logG;
     const int cl = lane & ((1 << logG) - 1);
     const uint32_t i0 = i1;
     i1 = __shfl_sync(0xffffffffu, my_off, k + 1);
-    const int64_t cur_idx = pf_idx;
+    const int64_t cur_ref = pf_ref;
     if (k + 1 < nb) {
       const uint32_t e = __shfl_sync(0xffffffffu, my_off, k + 2);
-      if (i1 + lane < e) pf_idx = indices[i1 + lane];
+      if (i1 + lane < e) {
+        bool next_cached = cached;
+        if (CACHED && b + 1 == B) next_cached = meta[t + 1].cache_id >= 0;
+        pf_ref = reference(i1 + lane, next_cached);
+      }
     }
 
     float acc[EPC];
@@ -327,23 +342,35 @@ tbe_forward_lean(const TableMeta* __restrict__ meta, int32_t n_bags, int32_t B,
     for (uint32_t base = i0; base < i1; base += 32) {
       const int cnt = (int)min(32u, i1 - base);
       uint32_t my_row = 0;
+      bool no_slot = false;                 // cached table, lookup without a slot: my_row is a row of the host tier
       if (lane < cnt) {
-        int64_t idx = base == i0 ? cur_idx : indices[base + lane];
-        if (idx < 0 || idx >= (int64_t)rows) {
-          atomicOr(status, STATUS_INDEX_CLAMPED);
-          idx = idx < 0 ? 0 : (int64_t)rows - 1;
+        int64_t ref = base == i0 ? cur_ref : reference(base + lane, cached);
+        if (CACHED && cached) {
+          no_slot = ref < 0;
+          if (no_slot) ref = indices[base + lane];
         }
-        my_row = (uint32_t)idx;
+        if (!(CACHED && cached) || no_slot) {
+          if (ref < 0 || ref >= (int64_t)rows) {
+            atomicOr(status, STATUS_INDEX_CLAMPED);
+            ref = ref < 0 ? 0 : (int64_t)rows - 1;
+          }
+        }
+        my_row = (uint32_t)ref;
       }
-      auto walk = [&](auto whole) {
+      const uint32_t no_slot_mask = CACHED ? __ballot_sync(0xffffffffu, no_slot) : 0u;
+      auto walk = [&](auto whole, auto mixed) {
         constexpr bool WHOLE = decltype(whole)::value;
+        constexpr bool MIXED = decltype(mixed)::value;      // some lookups of the batch read the host tier
+        const char* host_base = nullptr;
+        if (MIXED) host_base = host_w + meta[t].weight_offset * EB + cl * 16;
         for (int r = 0; r < cnt; r += R * LEAN_UNROLL) {
           uint4 v[LEAN_UNROLL];
 #pragma unroll
           for (int u = 0; u < LEAN_UNROLL; ++u) {
             const int j = r + u * R + sub;
             const uint32_t row = __shfl_sync(0xffffffffu, my_row, j & 31);
-            if (j < cnt && (WHOLE || cl < vec16)) v[u] = ld_nc_16(lane_base + (int64_t)row * row_bytes);
+            const char* from = (MIXED && ((no_slot_mask >> (j & 31)) & 1u)) ? host_base : lane_base;
+            if (j < cnt && (WHOLE || cl < vec16)) v[u] = ld_nc_16(from + (int64_t)row * row_bytes);
             else v[u] = make_uint4(0u, 0u, 0u, 0u);
           }
 #pragma unroll
@@ -353,8 +380,13 @@ tbe_forward_lean(const TableMeta* __restrict__ meta, int32_t n_bags, int32_t B,
           }
         }
       };
-      if (vec16 == (1 << logG)) walk(std::true_type{});
-      else walk(std::false_type{});
+      if (CACHED && no_slot_mask != 0u) {
+        if (vec16 == (1 << logG)) walk(std::true_type{}, std::true_type{});
+        else walk(std::false_type{}, std::true_type{});
+      } else {
+        if (vec16 == (1 << logG)) walk(std::true_type{}, std::false_type{});
+        else walk(std::false_type{}, std::false_type{});
+      }
     }
     // fold the row groups of the warp together
     for (int o = 1 << logG; o < 32; o <<= 1) {
@@ -375,15 +407,20 @@ tbe_forward_lean(const TableMeta* __restrict__ meta, int32_t n_bags, int32_t B,
 
 template <bool FP16>
 static int launch_forward_lean(const mts_tables* h, int32_t B, const int64_t* indices, const int64_t* offsets,
-                               int32_t pooling_mode, void* out, int out_kind, int64_t out_stride,
-                               cudaStream_t stream) {
+                               int32_t pooling_mode, const int32_t* slot_of_lookup, const CachePtrs& caches,
+                               void* out, int out_kind, int64_t out_stride, cudaStream_t stream) {
   const int64_t n_bags = (int64_t)h->T * B;
   const int64_t grid = ceil_div(n_bags, (int64_t)FWD_WARPS * FWD_BAGS);
   {
     LaunchScope scope(K_FORWARD, stream);
-    tbe_forward_lean<FP16><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
-        h->d_meta, (int32_t)n_bags, B, indices, offsets, static_cast<const char*>(h->dev_weights), pooling_mode, out,
-        out_kind, out_stride, h->d_status);
+    if (h->any_cached)
+      tbe_forward_lean<FP16, true><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
+          h->d_meta, (int32_t)n_bags, B, indices, offsets, slot_of_lookup, caches, static_cast<const char*>(h->dev_weights),
+          static_cast<const char*>(h->host_weights), pooling_mode, out, out_kind, out_stride, h->d_status);
+    else
+      tbe_forward_lean<FP16, false><<<(unsigned)grid, FWD_WARPS * 32, 0, stream>>>(
+          h->d_meta, (int32_t)n_bags, B, indices, offsets, slot_of_lookup, caches, static_cast<const char*>(h->dev_weights),
+          static_cast<const char*>(h->host_weights), pooling_mode, out, out_kind, out_stride, h->d_status);
   }
   return check_launch("tbe_forward_lean");
 }
@@ -430,11 +467,11 @@ int forward_any(const mts_tables* h, int32_t B, const int64_t* indices, const in
   const int nv = max_vec <= 32 ? 1 : max_vec <= 64 ? 2 : max_vec <= 128 ? 4 : 8;
   const bool fp16 = h->dtype == MTS_DTYPE_FP16;
 #if MTS_FWD_LEAN
-  // positions and bag numbers fit 32 bits (row numbers always do), no cached table, rows of at most 32 pieces
-  if (!h->any_cached && nv == 1 && pooling_mode != MTS_POOL_MAX && N < (1ll << 31) &&
+  // positions and bag numbers fit 32 bits (row numbers always do), rows of at most 32 pieces
+  if (nv == 1 && pooling_mode != MTS_POOL_MAX && N < (1ll << 31) &&
       (int64_t)h->T * B < (1ll << 31) - FWD_WARPS * FWD_BAGS) {
-    if (fp16) return launch_forward_lean<true>(h, B, indices, offsets, pooling_mode, out, out_kind, out_stride, s);
-    return launch_forward_lean<false>(h, B, indices, offsets, pooling_mode, out, out_kind, out_stride, s);
+    if (fp16) return launch_forward_lean<true>(h, B, indices, offsets, pooling_mode, slot_of_lookup, caches, out, out_kind, out_stride, s);
+    return launch_forward_lean<false>(h, B, indices, offsets, pooling_mode, slot_of_lookup, caches, out, out_kind, out_stride, s);
   }
 #endif
 #define MTS_FWD(F, V) return launch_forward<F, V>(h, B, indices, offsets, pooling_mode, slot_of_lookup, caches, out, out_kind, out_stride, s)

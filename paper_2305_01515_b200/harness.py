@@ -275,7 +275,7 @@ class DeviceModel:
                                  L["evict_slots"], L["evict_dirty"], L["capacity"], L["counters"], L["staging"], stream)
 
     # ---- missed rows gathered by host threads and moved by the copy engine
-    FETCH_STAGE_BYTES = 96 << 20         # per cache and batch context; larger miss / evict lists take the kernels
+    FETCH_STAGE_BYTES = 96 << 20         # first size of the pinned buffers, per cache and batch context; they grow on demand
 
     def enable_host_gather(self, threads: Optional[int] = None) -> None:
         """Pinned host buffers (keys and gathered rows, per cache and batch context) and one device
@@ -290,21 +290,36 @@ class DeviceModel:
         # seconds and bytes the host threads spent on gathers / scatters (and waiting for their turn), per cache
         self.host_copy_stats = [{"gather_s": 0.0, "gather_bytes": 0, "scatter_s": 0.0, "scatter_bytes": 0, "wait_s": 0.0}
                                 for _ in self.caches]
-        self.fetch_rows = [max(1, min(self.ctx[0]["lists"][g]["capacity"], self.FETCH_STAGE_BYTES // (c.dim * esz)))
-                           for g, c in enumerate(self.caches)]
-        self.fetch_dev = [torch.empty(r * c.dim * esz, dtype=torch.uint8, device=self.device)
-                          for r, c in zip(self.fetch_rows, self.caches)]
-        self.fetch_host = [[torch.empty(r * c.dim * esz, dtype=torch.uint8).pin_memory()
-                            for r, c in zip(self.fetch_rows, self.caches)] for _ in range(self.N_CTX)]
-        self.fetch_keys = [[torch.empty(r, dtype=torch.int64).pin_memory() for r in self.fetch_rows]
-                           for _ in range(self.N_CTX)]
+        n_c = len(self.caches)
+        self.fetch_rows = [0] * n_c
+        self.fetch_dev = [None] * n_c
+        self.fetch_host = [[None] * n_c for _ in range(self.N_CTX)]
+        self.fetch_keys = [[None] * n_c for _ in range(self.N_CTX)]
         # the way back: dirty victims, their keys and dirty bytes
-        self.wb_host = [[torch.empty(r * c.dim * esz, dtype=torch.uint8).pin_memory()
-                         for r, c in zip(self.fetch_rows, self.caches)] for _ in range(self.N_CTX)]
-        self.wb_keys = [[torch.empty(r, dtype=torch.int64).pin_memory() for r in self.fetch_rows]
-                        for _ in range(self.N_CTX)]
-        self.wb_dirty = [[torch.empty(r, dtype=torch.uint8).pin_memory() for r in self.fetch_rows]
-                         for _ in range(self.N_CTX)]
+        self.wb_host = [[None] * n_c for _ in range(self.N_CTX)]
+        self.wb_keys = [[None] * n_c for _ in range(self.N_CTX)]
+        self.wb_dirty = [[None] * n_c for _ in range(self.N_CTX)]
+        for g, c in enumerate(self.caches):
+            self.grow_host_buffers(g, self.FETCH_STAGE_BYTES // (c.dim * esz))
+
+    def grow_host_buffers(self, g: int, rows: int) -> None:
+        """Cache g: buffers of the copy-engine path for lists of up to `rows` rows (never more than the list
+        capacity).  The caller makes sure that no copy of this cache is in flight and no list waits in them."""
+        cap = self.ctx[0]["lists"][g]["capacity"]
+        rows = max(1, min(cap, int(rows)))
+        if rows <= self.fetch_rows[g]:
+            return
+        rb = self.caches[g].dim * (4 if self.spec.dtype == wl.FP32 else 2)
+        pinned = lambda n, dt: torch.empty(n, dtype=dt, pin_memory=True)
+        self.fetch_dev[g] = None
+        self.fetch_dev[g] = torch.empty(rows * rb, dtype=torch.uint8, device=self.device)
+        for x in range(self.N_CTX):
+            self.fetch_host[x][g] = pinned(rows * rb, torch.uint8)
+            self.fetch_keys[x][g] = pinned(rows, torch.int64)
+            self.wb_host[x][g] = pinned(rows * rb, torch.uint8)
+            self.wb_keys[x][g] = pinned(rows, torch.int64)
+            self.wb_dirty[x][g] = pinned(rows, torch.uint8)
+        self.fetch_rows[g] = rows
 
     def host_lists_fit(self, g: int, n_miss: int, n_evict: int) -> bool:
         """Whether the miss and evict lists of a batch fit the pinned buffers of the copy-engine path."""

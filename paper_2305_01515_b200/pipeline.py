@@ -174,6 +174,12 @@ class CachedTrainer:
             self._host_mark("tag_waited", t, g)
             n_miss = int(self._host_counters[t, g, mb.COUNTER_NAMES.index("inserted")])
             n_evict = int(self._host_counters[t, g, mb.COUNTER_NAMES.index("evicted")])
+            if not self.m.host_lists_fit(g, n_miss, n_evict) and max(n_miss, n_evict) <= self.m.ctx[ctx]["lists"][g]["capacity"]:
+                # longer lists than any before: larger buffers, once nothing of this cache is in flight
+                self._finish_writeback(g)
+                for q in (self.copies[g], self.saves[g], s):
+                    q.synchronize()
+                self.m.grow_host_buffers(g, max(n_miss, n_evict) * 5 // 4)
             if self.m.host_lists_fit(g, n_miss, n_evict):
                 self.m.cache_request_miss_keys(g, n_miss, self.copies[g], ctx)      # ahead of the victims' copies
                 w = self.saves[g]
