@@ -33,15 +33,21 @@ def test_pipelined_equals_sequential_and_oracle_tags(frac, lock):
     # sequential with the kernels fetching the missed rows; pipelined the same way; pipelined and
     # sequential with the rows gathered by host threads and moved by the copy engine
     # ... and both places of the tag step: between the training steps, or on a stream of its own
-    for pipelined, host_gather, tag_on_main in ((False, False, True), (True, False, True), (True, True, True),
-                                                (False, True, True), (True, False, False), (True, True, False)):
+    # ... and the copy-engine path starting from pinned buffers of two rows, which have to grow with the lists
+    for pipelined, host_gather, tag_on_main, stage_bytes in (
+            (False, False, True, None), (True, False, True, None), (True, True, True, None), (False, True, True, None),
+            (True, False, False, None), (True, True, False, None), (True, True, False, 512), (False, True, True, 512)):
         m = DeviceModel(spec, weights=W0, lock_depth=lock)
+        if stage_bytes is not None:
+            m.FETCH_STAGE_BYTES = stage_bytes
         m.reserve(max(len(b[0]) for b in host_batches))
         batches = [(to_dev(i), to_dev(o), o) for i, o in host_batches]
         tr = CachedTrainer(m, pipelined=pipelined, host_gather=host_gather, tag_on_main=tag_on_main)
         tr.run(batches, grads)
         m.flush()
         torch.cuda.synchronize()
+        if stage_bytes is not None:
+            assert max(m.fetch_rows) > stage_bytes // 128        # the buffers did grow
         results.append((m.weights_numpy(), m.momentum.cpu().numpy(), np.stack(tr.history)))
         m.close()
     (Wa, ma, ha), (Wb, mb_, hb) = results[0], results[1]
