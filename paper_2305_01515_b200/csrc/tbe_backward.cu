@@ -95,6 +95,13 @@ __device__ __forceinline__ int table_of_key(const TableMeta* __restrict__ meta, 
   return lo;
 }
 
+#ifndef MTS_BWD_PREFETCH_ROWS
+#define MTS_BWD_PREFETCH_ROWS 1   // rows and states that a batch of 32 lookups will update are requested into L2 while it is staged
+#endif
+__device__ __forceinline__ void prefetch_l2(const void* p) {
+  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
+
 struct RowTarget {
   char* w;            // row storage (HBM table, cache slot, or host tier)
   uint8_t* dirty;     // dirty byte to set, or nullptr
@@ -473,10 +480,18 @@ reduce_chunks_lean(const TableMeta* __restrict__ meta, int T, int32_t B,
       d.z = 0u; d.w = 0u;
       uint8_t* dirty = nullptr;
       if (my_end) {
-        const RowTarget rt = row_target(m, (int64_t)key, slot_at(m, sorted_slot, p, slot_of_lookup, ps), EB, caches, dev_w, host_w);
+        const int32_t slot = slot_at(m, sorted_slot, p, slot_of_lookup, ps);
+        const RowTarget rt = row_target(m, (int64_t)key, slot, EB, caches, dev_w, host_w);
         d.z = (uint32_t)(uintptr_t)rt.w;
         d.w = (uint32_t)((uintptr_t)rt.w >> 32);
         dirty = rt.dirty;
+        // the walk reaches this row up to 31 lookups from now: ask for it (device memory only) and its state
+        if (MTS_BWD_PREFETCH_ROWS && (m.cache_id < 0 || slot >= 0)) {
+          const int row_bytes = m.dim * EB;
+          for (int o = 0; o < row_bytes; o += 128) prefetch_l2(rt.w + o);
+          prefetch_l2(rt.w + row_bytes - 1);
+          prefetch_l2(momentum + key);
+        }
       }
       s_desc[wib][lane] = d;
       if (MEAN) {
