@@ -276,6 +276,7 @@ class DeviceModel:
 
     # ---- missed rows gathered by host threads and moved by the copy engine
     FETCH_STAGE_BYTES = 96 << 20         # first size of the pinned buffers, per cache and batch context; they grow on demand
+    FETCH_STAGE_MAX_BYTES = 256 << 20    # ... up to this size; longer lists (a cold cache's first batches) take the kernels
 
     def enable_host_gather(self, threads: Optional[int] = None) -> None:
         """Pinned host buffers (keys and gathered rows, per cache and batch context) and one device
@@ -306,10 +307,10 @@ class DeviceModel:
         """Cache g: buffers of the copy-engine path for lists of up to `rows` rows (never more than the list
         capacity).  The caller makes sure that no copy of this cache is in flight and no list waits in them."""
         cap = self.ctx[0]["lists"][g]["capacity"]
-        rows = max(1, min(cap, int(rows)))
+        rb = self.caches[g].dim * (4 if self.spec.dtype == wl.FP32 else 2)
+        rows = max(1, min(cap, int(rows), max(self.FETCH_STAGE_MAX_BYTES, self.FETCH_STAGE_BYTES) // rb))
         if rows <= self.fetch_rows[g]:
             return
-        rb = self.caches[g].dim * (4 if self.spec.dtype == wl.FP32 else 2)
         pinned = lambda n, dt: torch.empty(n, dtype=dt, pin_memory=True)
         self.fetch_dev[g] = None
         self.fetch_dev[g] = torch.empty(rows * rb, dtype=torch.uint8, device=self.device)
@@ -324,6 +325,11 @@ class DeviceModel:
     def host_lists_fit(self, g: int, n_miss: int, n_evict: int) -> bool:
         """Whether the miss and evict lists of a batch fit the pinned buffers of the copy-engine path."""
         return n_miss <= self.fetch_rows[g] and n_evict <= self.fetch_rows[g]
+
+    def host_buffers_can_hold(self, g: int, rows: int) -> bool:
+        """Whether grow_host_buffers may size cache g's buffers for lists of `rows` rows."""
+        rb = self.caches[g].dim * (4 if self.spec.dtype == wl.FP32 else 2)
+        return rows <= self.ctx[0]["lists"][g]["capacity"] and rows * rb <= self.FETCH_STAGE_MAX_BYTES
 
     def cache_save_victims_via_host(self, g: int, n_evict: int, stream, ctx: int):
         """Cache g, copy-engine path of the write-back: the dirty victims are saved to the staging buffer and

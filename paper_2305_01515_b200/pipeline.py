@@ -174,7 +174,7 @@ class CachedTrainer:
             self._host_mark("tag_waited", t, g)
             n_miss = int(self._host_counters[t, g, mb.COUNTER_NAMES.index("inserted")])
             n_evict = int(self._host_counters[t, g, mb.COUNTER_NAMES.index("evicted")])
-            if not self.m.host_lists_fit(g, n_miss, n_evict) and max(n_miss, n_evict) <= self.m.ctx[ctx]["lists"][g]["capacity"]:
+            if not self.m.host_lists_fit(g, n_miss, n_evict) and self.m.host_buffers_can_hold(g, max(n_miss, n_evict)):
                 # longer lists than any before: larger buffers, once nothing of this cache is in flight
                 self._finish_writeback(g)
                 for q in (self.copies[g], self.saves[g], s):
