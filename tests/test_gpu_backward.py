@@ -88,6 +88,21 @@ def test_mixed_dims_skew_and_long_segments(dtype):
     _run_steps(spec, n_steps=2)
 
 
+@pytest.mark.parametrize("dtype", [wl.FP32, wl.FP16])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_narrow_and_wide_tables_interleaved(dtype, mode):
+    """Tables of up to 128 columns and of 129..256 columns in no order: the reduce step runs once per width
+    class and every chunk of 128 sorted lookups belongs to exactly one of the two launches.  Tables with a
+    handful of lookups sit between large ones, so that chunks span several tables of both classes; a row
+    with thousands of lookups crosses many chunks in each class."""
+    dims = [256, 64, 200, 8, 128, 256, 32, 136, 128]
+    rows = [3000, 5, 2, 40000, 9, 1, 700, 20000, 3]
+    pool = [25, 0.2, 0.1, 30, 0.3, 40, 12, 18, 0.05]
+    spec = custom_spec(rows, dims, 257, dtype, pool, [1.2, 0, 0, 1.0, 0, 0, 0.9, 1.3, 0], seed=19)
+    _run_steps(spec, n_steps=2, mode=mode)
+    _run_steps(spec, n_steps=1, mode=mode, grad_f16=True)
+
+
 def test_mean_pooling_fp16():
     spec = custom_spec([100, 3000], [64, 128], 65, wl.FP16, [5, 25], [1.1, 1.05], seed=2)
     _run_steps(spec, n_steps=2, mode=1)
