@@ -802,7 +802,7 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     headline = args.workload or "cfg3"
-    beside = [] if (args.workload or world > 1) else ["cfg2", "cfg4", "cfg5"]
+    beside = [] if (args.workload or world > 1) else ["cfg2", "cfg5", "cfg4"]
 
     def counts(name):
         k, w = DEFAULT_STEPS.get(name, (8, 8))
