@@ -704,6 +704,7 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
                             "l2_bypass_rows_per_step": float(hist[:, :, 16].sum()) / steps,
                             "l2_dropped_rows_per_step": float(hist[:, :, 18].sum()) / steps,
                             "schedule": "sequential, rows moved by kernels"}
+    trainer.close()
     model.close()
     del model, trainer, batches, grads, glist
     torch.cuda.empty_cache()

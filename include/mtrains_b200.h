@@ -467,6 +467,55 @@ int mts_cache_place_fetched(mts_cache* cache, const void* fetched, const int32_t
 int mts_cache_save_victims(mts_cache* cache, const int32_t* evict_slots, const uint8_t* evict_dirty,
                            int64_t list_capacity, const int64_t* counters, void* evict_staging, void* stream);
 
+/* The copy-engine data movement of one cache run by a host thread of the library (Sections 5.5.3, 5.5.4: rows
+ * between the cache and the lower tier; Section 5.7: ahead of the training of their batch).  A mover owns one
+ * thread, pinned host buffers for `n_contexts` batches in flight (keys and rows, both directions; they start at
+ * first_buffer_bytes per list and grow up to max_buffer_bytes when a batch's lists are longer) and one device
+ * buffer.  Per submitted batch, in submission order, the thread: waits for the event `tag_done` (recorded by
+ * the caller after the batch's mts_cache_lookup_insert* AND after a copy of its `counters` to the pinned
+ * `host_counters`); starts the miss keys on their way to the host on `copy_stream`; saves the victims
+ * (mts_cache_save_victims) and copies them, their keys and dirty bytes out on `save_stream`; puts the previous
+ * batch's victims into their host rows (mts_host_scatter_rows: a row evicted by one batch may be missed by the
+ * next); gathers the missed rows (mts_host_gather_rows); enqueues their copy and mts_cache_place_fetched on
+ * `move_stream`; records the batch's "moved" event there.  It does not wait for the copy of the rows.  Lists
+ * longer than the buffers may grow to are moved by mts_cache_prefetch_misses / mts_cache_writeback_evicted
+ * on `move_stream` instead (the thread then waits for them).
+ * host_rows: base of the cache's keys in the host tier (pinned, device-visible; row k at k * row_bytes).
+ * The job's device pointers are the arguments and results of the batch's mts_cache_lookup_insert*; they and
+ * evict_staging must stay untouched until the batch has moved; one evict_staging may serve all batches of a
+ * mover.  The three streams must not be the legacy default stream's aliases of one another's work in a way
+ * that makes them wait for the caller's later work (the thread enqueues on them while the caller runs).
+ * mts_mover_submit returns at once.  mts_mover_stream_wait_moved blocks the calling host thread until the
+ * batch's "moved" event has been recorded (not until it has completed) and makes `stream` wait for it.
+ * mts_mover_drain waits until every submitted batch has been enqueued and puts the last victims into their
+ * rows (call it with the streams still alive; afterwards the host tier is current once move_stream and
+ * save_stream are idle).  mts_mover_stats: seconds gathering, bytes gathered, seconds scattering, bytes
+ * scattered, batches moved by kernels.  A failure in the thread is returned by every later call.
+ * Errors: INVALID_ARG, CUDA. */
+typedef struct mts_mover mts_mover;
+typedef struct {
+  const int64_t* miss_keys;      /* device lists of the batch (mts_cache_lookup_insert*) */
+  const int32_t* miss_slots;
+  const int64_t* evict_keys;
+  const int32_t* evict_slots;
+  const uint8_t* evict_dirty;
+  int64_t list_capacity;
+  const int64_t* counters;       /* device [MTS_NUM_COUNTERS] */
+  const int64_t* host_counters;  /* pinned copy of `counters`, complete when tag_done is */
+  void* evict_staging;           /* device [list_capacity, dim] */
+  void* tag_done;                /* cudaEvent_t */
+  void* move_stream;             /* cudaStream_t: copy of the gathered rows, placing kernel, "moved" event */
+  void* save_stream;             /* cudaStream_t: victims saved and copied out */
+  void* copy_stream;             /* cudaStream_t: miss keys to the host */
+} mts_move_job;
+int mts_mover_create(mts_mover** out, mts_cache* cache, void* host_rows, int64_t row_bytes, int32_t threads,
+                     int32_t n_contexts, int64_t first_buffer_bytes, int64_t max_buffer_bytes);
+int mts_mover_submit(mts_mover* mover, const mts_move_job* job);
+int mts_mover_stream_wait_moved(mts_mover* mover, int64_t job_index, void* stream);
+int mts_mover_drain(mts_mover* mover);
+int mts_mover_stats(mts_mover* mover, double* out5);
+int mts_mover_destroy(mts_mover* mover);
+
 /* Evicted dirty rows go back to the host tier: evict_staging[k] -> host row evict_keys[k]. */
 int mts_cache_writeback_evicted(mts_cache* cache, void* host_rows_mapped, const int64_t* evict_keys,
                                 const uint8_t* evict_dirty, int64_t list_capacity,

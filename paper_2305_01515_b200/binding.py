@@ -38,7 +38,7 @@ EXPORTS = (
     "mts_tbe_backward_apply_presorted", "mts_cache_create_host_level", "mts_cache2_workspace_bytes",
     "mts_cache2_lookup_insert", "mts_cache2_move", "mts_cache_import_state", "mts_cache_set_fetch_wait_limit",
     "mts_place_tables",
-    "mts_cache_prefetch_misses", "mts_host_gather_rows", "mts_host_scatter_rows", "mts_cache_place_fetched", "mts_cache_save_victims", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
+    "mts_cache_prefetch_misses", "mts_host_gather_rows", "mts_host_scatter_rows", "mts_cache_place_fetched", "mts_cache_save_victims", "mts_mover_create", "mts_mover_submit", "mts_mover_stream_wait_moved", "mts_mover_drain", "mts_mover_stats", "mts_mover_destroy", "mts_cache_writeback_evicted", "mts_cache_refetch_overflowed", "mts_cache_flush",
     "mts_cache_export_state",
 )
 
@@ -123,6 +123,12 @@ def lib():
         L.mts_host_scatter_rows.argtypes = [vp, vp, vp, i64, i64, vp, i32]
         L.mts_cache_place_fetched.argtypes = [vp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.mts_cache_save_victims.argtypes = [vp, vp, vp, i64, vp, vp, vp]
+        L.mts_mover_create.argtypes = [C.POINTER(vp), vp, vp, i64, i32, i32, i64, i64]
+        L.mts_mover_submit.argtypes = [vp, C.POINTER(MoveJob)]
+        L.mts_mover_stream_wait_moved.argtypes = [vp, i64, vp]
+        L.mts_mover_drain.argtypes = [vp]
+        L.mts_mover_stats.argtypes = [vp, C.POINTER(C.c_double)]
+        L.mts_mover_destroy.argtypes = [vp]
         L.mts_cache_flush.argtypes = [vp, vp, vp]
         L.mts_cache_export_state.argtypes = [vp, vp, vp, vp, vp, vp]
         L.mts_cache_import_state.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -438,6 +444,53 @@ def cache_place_fetched(cache: Cache, fetched, miss_slots, evict_slots, evict_di
     _check(lib().mts_cache_place_fetched(cache.handle, _ptr(fetched), _ptr(miss_slots), _ptr(evict_slots),
                                          _ptr(evict_dirty), list_capacity, _ptr(counters), _ptr(evict_staging),
                                          _stream(stream)))
+
+
+class MoveJob(C.Structure):
+    """mts_move_job of the header."""
+    _fields_ = [("miss_keys", C.c_void_p), ("miss_slots", C.c_void_p), ("evict_keys", C.c_void_p),
+                ("evict_slots", C.c_void_p), ("evict_dirty", C.c_void_p), ("list_capacity", C.c_int64),
+                ("counters", C.c_void_p), ("host_counters", C.c_void_p), ("evict_staging", C.c_void_p),
+                ("tag_done", C.c_void_p), ("move_stream", C.c_void_p), ("save_stream", C.c_void_p),
+                ("copy_stream", C.c_void_p)]
+
+
+class Mover:
+    """mts_mover: the copy-engine data movement of one cache on a host thread of the library."""
+
+    def __init__(self, cache: Cache, host_rows: int, row_bytes: int, threads: int, n_contexts: int,
+                 first_buffer_bytes: int, max_buffer_bytes: int):
+        h = C.c_void_p()
+        _check(lib().mts_mover_create(C.byref(h), cache.handle, host_rows, row_bytes, threads, n_contexts,
+                                      first_buffer_bytes, max_buffer_bytes))
+        self.handle = h
+        self.submitted = 0
+
+    def submit(self, miss_keys, miss_slots, evict_keys, evict_slots, evict_dirty, list_capacity: int, counters,
+               host_counters, evict_staging, tag_done: int, move_stream, save_stream, copy_stream) -> int:
+        """Hands the batch to the mover's thread; returns its job index."""
+        job = MoveJob(_ptr(miss_keys), _ptr(miss_slots), _ptr(evict_keys), _ptr(evict_slots), _ptr(evict_dirty),
+                      list_capacity, _ptr(counters), _ptr(host_counters), _ptr(evict_staging), tag_done,
+                      _stream(move_stream), _stream(save_stream), _stream(copy_stream))
+        _check(lib().mts_mover_submit(self.handle, C.byref(job)))
+        self.submitted += 1
+        return self.submitted - 1
+
+    def stream_wait_moved(self, job_index: int, stream) -> None:
+        _check(lib().mts_mover_stream_wait_moved(self.handle, job_index, _stream(stream)))
+
+    def drain(self) -> None:
+        _check(lib().mts_mover_drain(self.handle))
+
+    def stats(self) -> dict:
+        v = (C.c_double * 5)()
+        _check(lib().mts_mover_stats(self.handle, v))
+        return {"gather_s": v[0], "gather_bytes": v[1], "scatter_s": v[2], "scatter_bytes": v[3], "kernel_batches": v[4]}
+
+    def close(self) -> None:
+        if self.handle:
+            lib().mts_mover_destroy(self.handle)
+            self.handle = None
 
 
 def cache_save_victims(cache: Cache, evict_slots, evict_dirty, list_capacity: int, counters, evict_staging,

@@ -63,11 +63,19 @@ from .harness import DeviceModel
 
 
 class CachedTrainer:
-    def __init__(self, model: DeviceModel, pipelined: bool = True, host_gather: bool = False, tag_on_main: bool = False):
+    def __init__(self, model: DeviceModel, pipelined: bool = True, host_gather: bool = False, tag_on_main: bool = False,
+                 native_mover: Optional[bool] = None):
         """host_gather: missed rows are gathered by host threads into a pinned buffer and moved by the
         copy engine, instead of being read over the host link by a kernel.
         tag_on_main: the tag step of batch t + lock_depth + 1 follows the backward of batch t on the training
-        stream, instead of running two batches ahead on a stream of its own (see the module docstring)."""
+        stream, instead of running two batches ahead on a stream of its own (see the module docstring).
+        native_mover (pipelined with host_gather): the caches' data paths run on threads of the library
+        (mts_mover) instead of Python threads; None = yes, unless the phases are timed (record_timeline)."""
+        self.native_mover = native_mover
+        self._movers = None
+        self._mover_seen = [{} for _ in model.caches]
+        self._native = False
+        self._submitted = []
         assert model.cached
         # the side streams run two batches ahead and keep two overflow lists alive: lock depths 1 and 2
         assert not pipelined or 1 <= model.lock_depth <= 2, "the pipelined schedule needs lock_depth 1 or 2"
@@ -95,6 +103,19 @@ class CachedTrainer:
         self._host_marks = []
         self._mark_lock = threading.Lock()
         self.debug_delay_cycles = 0                   # > 0: the move and repair streams idle that long before their work
+
+    def close(self):
+        """Stops the library's mover threads (after run() has returned)."""
+        if self._movers is not None:
+            for mv in self._movers:
+                mv.close()
+            self._movers = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
     def _delay(self, stream):
         """Test aid: hold a side stream back so that the training and the tag step run far ahead of it."""
@@ -222,12 +243,14 @@ class CachedTrainer:
             self.m.cache_writeback_via_host_finish(g, n_evict, ctx)
             self._pending_wb[g] = None
 
-    def _finish_move(self, t):
+    def _finish_move(self, t, waited=False):
         """After the data movement of batch t: repair the rows that overflowed in the batches whose backward may
-        have run after their copy was taken, then batch t is ready to train."""
+        have run after their copy was taken, then batch t is ready to train.  waited: the repair stream already
+        waits for the batch's data movement (the library's movers arranged that)."""
         s = self.fix
-        for e in self.ev_moved[t]:
-            s.wait_event(e)
+        if not waited:
+            for e in self.ev_moved[t]:
+                s.wait_event(e)
         if self.pipelined and t >= 1:
             s.wait_event(self.ev_bwd[t - 1])
             self._delay(s)
@@ -247,6 +270,8 @@ class CachedTrainer:
     def _fail(self, e):
         self._worker_error = e
         for f in self._ready_recorded:
+            f.set()
+        for f in self._submitted:
             f.set()
         for row in self._moved_recorded:
             for f in row:
@@ -272,16 +297,37 @@ class CachedTrainer:
         try:
             torch.cuda.set_device(self.dev)
             for t in range(K):
-                for f in self._moved_recorded[t]:
-                    f.wait()
+                if self._native:
+                    self._submitted[t].wait()
+                    if self._stop.is_set() or self._worker_error is not None:
+                        return
+                    # blocks until each mover has recorded the batch's "moved" event, then the repair stream waits for it
+                    for g, mv in enumerate(self._movers):
+                        mv.stream_wait_moved(self._job_of[t][g], self.fix)
+                else:
+                    for f in self._moved_recorded[t]:
+                        f.wait()
                 if t >= 1:
                     self._bwd_recorded[t - 1].wait()            # the repair waits for that event on the device
                 if self._stop.is_set() or self._worker_error is not None:
                     return
-                self._finish_move(t)
+                self._finish_move(t, waited=self._native)
                 self._ready_recorded[t].set()
         except BaseException as e:
             self._fail(e)
+
+    def _submit_move(self, t):
+        """Batch t to the library's movers (one per cache), which run its data path on their own threads."""
+        m, ctx = self.m, t % DeviceModel.N_CTX
+        tag_done = self.ev_tags[t].cuda_event
+        for g, mv in enumerate(self._movers):
+            self._delay(self.moves[g])
+            self._delay(self.saves[g])
+            L = m.ctx[ctx]["lists"][g]
+            self._job_of[t][g] = mv.submit(L["miss_keys"], L["miss_slots"], L["evict_keys"], L["evict_slots"],
+                                           L["evict_dirty"], L["capacity"], L["counters"], self._host_counters[t, g],
+                                           L["staging"], tag_done, self.moves[g], self.saves[g], self.copies[g])
+        self._submitted[t].set()
 
     def _wait_ready_recorded(self, t):
         if self._threads:
@@ -323,6 +369,7 @@ class CachedTrainer:
         n_cnt = mb.NUM_COUNTERS2 if m.l2 else mb.NUM_COUNTERS
         self._host_counters = torch.zeros((K, n_c, n_cnt), dtype=torch.int64).pin_memory()
         self._threads = []
+        self._native = False
         self._worker_error = None
         self._pending_wb = [None] * n_c
         if out is None:
@@ -361,16 +408,30 @@ class CachedTrainer:
             self._bwd_recorded = [threading.Event() for _ in range(K)]
             self._moved_recorded = [[threading.Event() for _ in range(n_c)] for _ in range(K)]
             self._stop = threading.Event()
-            self._threads = [threading.Thread(target=self._cache_worker, args=(g,), daemon=True) for g in range(n_c)]
+            # the caches' data paths: threads of the library (movers), or Python threads when the phases are
+            # to be timed with events (record_timeline) or the caller asked for them
+            self._native = self.native_mover if self.native_mover is not None else not self.record_timeline
+            self._submitted = [threading.Event() for _ in range(K)]
+            self._job_of = [[0] * n_c for _ in range(K)]
+            if self._native:
+                if self._movers is None:
+                    self._movers = [mb.Mover(c, m.host_rows_ptr(g), c.dim * m.spec.elem_bytes, m.gather_threads,
+                                             DeviceModel.N_CTX, m.FETCH_STAGE_BYTES, max(m.FETCH_STAGE_MAX_BYTES, m.FETCH_STAGE_BYTES))
+                                    for g, c in enumerate(m.caches)]
+                self._threads = []
+            else:
+                self._threads = [threading.Thread(target=self._cache_worker, args=(g,), daemon=True) for g in range(n_c)]
             self._threads.append(threading.Thread(target=self._finisher, args=(K,), daemon=True))
             for th in self._threads:
                 th.start()
 
         def start_move(t):
             """The data path of batch t, as soon as its tag step is enqueued."""
-            if self._threads:
+            if self._threads and self._native:
+                self._submit_move(t)       # ev_tags[t] has been recorded by this thread already
+            elif self._threads:
                 for q in self._jobs:
-                    q.put(t)               # ev_tags[t] has been recorded by this thread already
+                    q.put(t)
             else:
                 for g in range(n_c):
                     self._move_cache(t, g, False)
@@ -413,8 +474,17 @@ class CachedTrainer:
                 for row in self._moved_recorded:
                     for f in row:
                         f.set()
+                for f in self._submitted:
+                    f.set()
                 for th in self._threads:
                     th.join()
+                if self._native and self._worker_error is None:
+                    for g, mv in enumerate(self._movers):
+                        mv.drain()             # the last victims into their host rows
+                        st, cur = m.host_copy_stats[g], mv.stats()
+                        for k in ("gather_s", "gather_bytes", "scatter_s", "scatter_bytes"):
+                            st[k] += cur[k] - self._mover_seen[g].get(k, 0.0)
+                        self._mover_seen[g] = cur
                 self._threads = []
                 if self._worker_error is not None:
                     raise self._worker_error

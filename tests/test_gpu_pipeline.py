@@ -34,20 +34,26 @@ def test_pipelined_equals_sequential_and_oracle_tags(frac, lock):
     # sequential with the rows gathered by host threads and moved by the copy engine
     # ... and both places of the tag step: between the training steps, or on a stream of its own
     # ... and the copy-engine path starting from pinned buffers of two rows, which have to grow with the lists
-    for pipelined, host_gather, tag_on_main, stage_bytes in (
-            (False, False, True, None), (True, False, True, None), (True, True, True, None), (False, True, True, None),
-            (True, False, False, None), (True, True, False, None), (True, True, False, 512), (False, True, True, 512)):
+    # ... and the caches' data paths on the library's mover threads (native) or on Python threads
+    for pipelined, host_gather, tag_on_main, stage_bytes, native in (
+            (False, False, True, None, None), (True, False, True, None, None), (True, True, True, None, True),
+            (False, True, True, None, None), (True, False, False, None, None), (True, True, False, None, True),
+            (True, True, False, None, False), (True, True, True, None, False),
+            (True, True, False, 512, False), (True, True, False, 512, True), (False, True, True, 512, None)):
         m = DeviceModel(spec, weights=W0, lock_depth=lock)
         if stage_bytes is not None:
             m.FETCH_STAGE_BYTES = stage_bytes
         m.reserve(max(len(b[0]) for b in host_batches))
         batches = [(to_dev(i), to_dev(o), o) for i, o in host_batches]
-        tr = CachedTrainer(m, pipelined=pipelined, host_gather=host_gather, tag_on_main=tag_on_main)
+        tr = CachedTrainer(m, pipelined=pipelined, host_gather=host_gather, tag_on_main=tag_on_main, native_mover=native)
         tr.run(batches, grads)
         m.flush()
         torch.cuda.synchronize()
-        if stage_bytes is not None:
+        if stage_bytes is not None and not (pipelined and native):
             assert max(m.fetch_rows) > stage_bytes // 128        # the buffers did grow
+        if pipelined and host_gather and native:
+            assert sum(mv.stats()["gather_bytes"] for mv in tr._movers) > 0      # the movers did the work
+        tr.close()
         results.append((m.weights_numpy(), m.momentum.cpu().numpy(), np.stack(tr.history)))
         m.close()
     (Wa, ma, ha), (Wb, mb_, hb) = results[0], results[1]
