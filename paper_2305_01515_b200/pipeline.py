@@ -46,7 +46,10 @@ waiting for them: while they run it already handles the next batch.  The victims
 its tag step ends, so they are saved and copied out on save[g] at once (the placing kernel waits for the
 save); the worker puts them into their host rows before its next gather, which may read one of them.  One more
 thread enqueues the repair once all caches of a batch have moved.  The workers run ahead of the launching
-thread; host-side flags tell each side which events the other has recorded.
+thread; host-side flags tell each side which events the other has recorded.  By default the worker of a
+cache is a thread of the library (mts_mover: the same calls in the same order, without the interpreter and
+its lock in the loop: 1.9 -> 1.7 ms per batch on configuration 5, 0.43 -> 0.28 ms at batch 1024); the Python
+worker below makes the same calls and is used when the phases are timed with events.
 """
 from __future__ import annotations
 
