@@ -681,7 +681,10 @@ def measure_cached(args, spec, dev, steps: int, warmup: int):
         nb = float(K + COOLDOWN)
         g_s, s_s = sum(x["gather_s"] for x in st), sum(x["scatter_s"] for x in st)
         g_b, s_b = sum(x["gather_bytes"] for x in st), sum(x["scatter_bytes"] for x in st)
-        rec["host_threads"] = {"threads": model.gather_threads, "gather_ms_per_batch": g_s * 1e3 / nb,
+        rec["host_threads"] = {"threads": model.gather_threads,
+                               "workers": "python threads" if args.timeline else "threads of the library (mts_mover); their gather / "
+                                          "scatter times include waiting for the other caches' turn at the cores",
+                               "gather_ms_per_batch": g_s * 1e3 / nb,
                                "scatter_ms_per_batch": s_s * 1e3 / nb,
                                "gather_gbs": g_b / max(g_s, 1e-9) / 1e9, "scatter_gbs": s_b / max(s_s, 1e-9) / 1e9,
                                "wait_for_turn_ms_per_batch": sum(x["wait_s"] for x in st) * 1e3 / nb}
